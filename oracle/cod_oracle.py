@@ -1,0 +1,336 @@
+"""CPU oracle of one Carryover drafting round.  TEST INFRASTRUCTURE ONLY.
+
+A plain, slow, float64 numpy statement of what the round computes, written from
+the paper (Section 2 "Carryover Drafting", Eq. 1, Eq. 2; Appendix A, Algorithm 1
+and its "Cache semantics" paragraph).  It exists to judge the CUDA library; it
+shares no code with it and is never on the product path: only the tests, the
+smoke check and the benchmark's CPU-baseline leg may import it.
+
+Every part below has an exact definition (a prefix rule on integers, linear
+maps, a plane rotation, softmax attention, an argmax), so the oracle is that
+definition written out: no tiling, no online softmax, no fused steps.  numpy's
+``@`` (a library matmul in float64) serves as the contraction step.
+
+Where the paper leaves the drafter body open (the equations "omit attention
+normalisation and positional encoding", Section 2.1), the readings taken are:
+  * F, K_l, V_l, W_q, W_o are bias-free linear maps stored [out, in];
+  * an RMS normalisation with gain follows F (switchable), precedes each
+    attention sub-layer, and precedes the LM head; the residual stream is
+    x <- x + W_o o; there is no MLP;
+  * RoPE is the rotate-half form over the full head dimension, at the absolute
+    token position, applied once to keys when they are projected (Appendix A,
+    "Cache semantics") and to the block's queries and keys at draft time;
+  * the block is [bonus token, MASK, ..., MASK]; every block query sees all
+    committed rows, all carried rows and all block rows (no mask), scale
+    1/sqrt(hd); grouped-query attention maps query head g to KV head
+    g // (n_q / n_kv);
+  * the LM head is the transposed embedding table; argmax ties go to the lowest id.
+
+Parity status: every function here is pinned by tests/test_oracle_pins.py
+against closed forms, brute force, invariants the paper states, and library
+special cases.  What stays unpinned is the choice of the readings above
+themselves: the paper ships no reference numbers for this path, so they are
+pinned to their written definition only ("parity unpinned" against the authors'
+system for the drafter-body glue).
+"""
+from __future__ import annotations
+
+from dataclasses import dataclass
+from typing import Dict, Optional
+
+import numpy as np
+
+MODE_CARRY = 0      # Algorithm 1, right column
+MODE_BASELINE = 1   # Algorithm 1, left column
+
+
+@dataclass
+class OracleConfig:
+    d_target: int
+    n_cap: int
+    d_model: int
+    n_layers: int
+    n_q: int
+    n_kv: int
+    hd: int
+    vocab: int
+    mask_token_id: int
+    W: int
+    page: int
+    rope_theta: float
+    rms_eps: float
+    hidden_norm: bool
+
+    @property
+    def d_in(self) -> int:
+        return self.d_target * self.n_cap
+
+
+def prepare_weights(weights: Dict[str, np.ndarray]) -> Dict[str, np.ndarray]:
+    """float64 copies of the weight arrays (made once; the values are unchanged)."""
+    return {k: np.asarray(v, dtype=np.float64) for k, v in weights.items()}
+
+
+class OracleState:
+    """Committed drafter KV C_l (paged), carried KV U_l, and their lengths.
+
+    pool  [Ld, n_pages, n_kv, 2, page, hd]   index 3: 0 = K (already rotated), 1 = V
+    carry [Ld, S, n_kv, 2, W, hd]            rows >= carry_len[s] are NaN (never to be read)
+    """
+
+    def __init__(self, cfg: OracleConfig, S: int, n_pages: int, block_table: np.ndarray,
+                 committed_len: np.ndarray):
+        self.cfg = cfg
+        self.S = S
+        self.pool = np.zeros((cfg.n_layers, n_pages, cfg.n_kv, 2, cfg.page, cfg.hd), dtype=np.float64)
+        self.block_table = np.array(block_table, dtype=np.int64)
+        self.committed_len = np.array(committed_len, dtype=np.int64)
+        self.carry = np.full((cfg.n_layers, S, cfg.n_kv, 2, cfg.W, cfg.hd), np.nan, dtype=np.float64)
+        # Algorithm 1: "Initialize U_l = empty".
+        self.carry_len = np.zeros(S, dtype=np.int64)
+
+
+# =========================================================================== part 1
+def verify_accept(draft: np.ndarray, target: np.ndarray, committed_len: np.ndarray,
+                  block_table: np.ndarray, page: int, n_forced: int) -> Dict[str, np.ndarray]:
+    """Greedy verification (Section 2, "Preliminaries"; Algorithm 2 "GreedyVerify").
+
+    The target accepts the longest PREFIX of the window whose tokens equal its own
+    greedy tokens; rejection stops acceptance of the whole suffix (Appendix B.1).
+    target[s, p] is the target's greedy token for window row p (W+1 entries), so the
+    token after the accepted prefix, target[s, m], is the bonus token.  The first
+    n_forced rows (the anchor) count as accepted whatever they hold.
+
+    Rows p < m are accepted (H^acc), rows p >= m are rejected (H^rej), Eq. 1.  Row p
+    sits at absolute position L_s + p ("each rejected state keeps the absolute
+    position of the token at which it was computed").
+    """
+    draft = np.asarray(draft)
+    target = np.asarray(target)
+    S, W = draft.shape
+    accept_len = np.zeros(S, dtype=np.int32)
+    bonus = np.zeros(S, dtype=np.int32)
+    row_pos = np.zeros(S * W, dtype=np.int32)
+    commit_slot = np.full(S * W, -1, dtype=np.int32)
+    carry_slot = np.full(S * W, -1, dtype=np.int32)
+    acc_rows, rej_rows = [], []
+    acc_off, rej_off = [0], [0]
+    for s in range(S):
+        m = 0
+        while m < W and (m < n_forced or int(draft[s, m]) == int(target[s, m])):
+            m += 1
+        accept_len[s] = m
+        bonus[s] = target[s, m]
+        L = int(committed_len[s])
+        for p in range(W):
+            row = s * W + p
+            pos = L + p
+            row_pos[row] = pos
+            if p < m:
+                commit_slot[row] = int(block_table[s, pos // page]) * page + pos % page
+                acc_rows.append(row)
+            else:
+                carry_slot[row] = s * W + (p - m)
+                rej_rows.append(row)
+        acc_off.append(len(acc_rows))
+        rej_off.append(len(rej_rows))
+    pad = lambda lst: np.array(lst + [-1] * (S * W - len(lst)), dtype=np.int32)
+    return {
+        "accept_len": accept_len, "bonus": bonus, "row_pos": row_pos,
+        "commit_slot": commit_slot, "carry_slot": carry_slot,
+        "acc_rows": pad(acc_rows), "acc_off": np.array(acc_off, dtype=np.int32),
+        "rej_rows": pad(rej_rows), "rej_off": np.array(rej_off, dtype=np.int32),
+    }
+
+
+# =========================================================================== shared pieces
+def rope(x: np.ndarray, pos, theta: float) -> np.ndarray:
+    """Rotate-half rotary embedding of x[..., hd] at absolute position(s) pos.
+
+    Pair (j, j + hd/2) is rotated by the angle pos * theta^(-2j/hd).
+    pos broadcasts against x[..., 0].
+    """
+    x = np.asarray(x, dtype=np.float64)
+    hd = x.shape[-1]
+    half = hd // 2
+    j = np.arange(half, dtype=np.float64)
+    inv_freq = np.float64(theta) ** (-2.0 * j / hd)
+    ang = np.asarray(pos, dtype=np.float64)[..., None] * inv_freq
+    c, s = np.cos(ang), np.sin(ang)
+    x1, x2 = x[..., :half], x[..., half:]
+    return np.concatenate([x1 * c - x2 * s, x2 * c + x1 * s], axis=-1)
+
+
+def rmsnorm(x: np.ndarray, g: np.ndarray, eps: float) -> np.ndarray:
+    """g * x / sqrt(mean(x^2) + eps) over the last axis."""
+    x = np.asarray(x, dtype=np.float64)
+    return g * x / np.sqrt(np.mean(x * x, axis=-1, keepdims=True) + eps)
+
+
+# =========================================================================== part 2
+def fuse_features(H: np.ndarray, rejected: np.ndarray, w: Dict[str, np.ndarray],
+                  cfg: OracleConfig) -> np.ndarray:
+    """Z = F(H^keep) with E_carry added to the rejected rows first (Eq. 2; Algorithm 1
+    right column, steps 2-3: the embedding is added "before projection by F")."""
+    Hk = np.asarray(H, dtype=np.float64).copy()
+    Hk[rejected] = Hk[rejected] + w["e_carry"]
+    Z = Hk @ w["fc"].T
+    if cfg.hidden_norm:
+        Z = rmsnorm(Z, w["g_hidden"], cfg.rms_eps)
+    return Z
+
+
+def project_kv(H: np.ndarray, split: Dict[str, np.ndarray], w: Dict[str, np.ndarray],
+               cfg: OracleConfig, mode: int) -> np.ndarray:
+    """J_l = (K_l(Z), V_l(Z)) for every drafter layer (Eq. 1; Algorithm 1 step "J_l").
+
+    Carry mode keeps all window rows; baseline mode keeps the accepted rows only
+    (the others come back as NaN: they do not exist in that column of Algorithm 1).
+    Keys are rotated at their row's absolute position.  Output [Ld, R, 2, n_kv, hd].
+    """
+    R = H.shape[0]
+    W = cfg.W
+    m_of_row = np.repeat(np.asarray(split["accept_len"], dtype=np.int64), W)
+    p_of_row = np.tile(np.arange(W), R // W)
+    rejected = p_of_row >= m_of_row
+    keep = np.ones(R, dtype=bool) if mode == MODE_CARRY else ~rejected
+    Z = fuse_features(H, rejected, w, cfg)
+    J = np.full((cfg.n_layers, R, 2, cfg.n_kv, cfg.hd), np.nan, dtype=np.float64)
+    pos = np.asarray(split["row_pos"], dtype=np.float64)
+    for l in range(cfg.n_layers):
+        K = (Z @ w["wk"][l].T).reshape(R, cfg.n_kv, cfg.hd)
+        V = (Z @ w["wv"][l].T).reshape(R, cfg.n_kv, cfg.hd)
+        K = rope(K, pos[:, None], cfg.rope_theta)
+        J[l, keep, 0] = K[keep]
+        J[l, keep, 1] = V[keep]
+    return J
+
+
+# =========================================================================== part 3
+def scatter_kv(J: np.ndarray, split: Dict[str, np.ndarray], st: OracleState, mode: int) -> None:
+    """C_l <- [C_l; J_{l,1:m}],  U_l <- J_{l,m+1:B} replacing the old U_l (Algorithm 1,
+    right column, last three steps); the baseline column appends only and leaves U empty."""
+    cfg = st.cfg
+    W, page = cfg.W, cfg.page
+    for s in range(st.S):
+        m = int(split["accept_len"][s])
+        L = int(st.committed_len[s])
+        for l in range(cfg.n_layers):
+            for p in range(m):
+                pos = L + p
+                pg = int(st.block_table[s, pos // page])
+                st.pool[l, pg, :, 0, pos % page, :] = J[l, s * W + p, 0]
+                st.pool[l, pg, :, 1, pos % page, :] = J[l, s * W + p, 1]
+            st.carry[l, s] = np.nan                       # the previous U_l is gone
+            if mode == MODE_CARRY:
+                for p in range(m, W):
+                    st.carry[l, s, :, 0, p - m, :] = J[l, s * W + p, 0]
+                    st.carry[l, s, :, 1, p - m, :] = J[l, s * W + p, 1]
+        st.committed_len[s] = L + m
+        st.carry_len[s] = (W - m) if mode == MODE_CARRY else 0
+
+
+# =========================================================================== part 4
+def gather_ctx(st: OracleState, layer: int, s: int, use_carry: bool):
+    """ctx_l = [C_l; U_l] of sequence s as dense arrays K, V [n_kv, L' + c, hd] (Eq. 2)."""
+    cfg = st.cfg
+    L = int(st.committed_len[s])
+    t = np.arange(L)
+    pages = st.block_table[s, t // cfg.page]
+    Kc = st.pool[layer, pages, :, 0, t % cfg.page, :]      # [L, n_kv, hd]
+    Vc = st.pool[layer, pages, :, 1, t % cfg.page, :]
+    K = np.transpose(Kc, (1, 0, 2))
+    V = np.transpose(Vc, (1, 0, 2))
+    c = int(st.carry_len[s]) if use_carry else 0
+    if c > 0:
+        K = np.concatenate([K, st.carry[layer, s, :, 0, :c, :]], axis=1)
+        V = np.concatenate([V, st.carry[layer, s, :, 1, :c, :]], axis=1)
+    return K, V, c
+
+
+def block_attn(layer: int, q: np.ndarray, k_blk: np.ndarray, v_blk: np.ndarray,
+               st: OracleState, use_carry: bool):
+    """Block attention over [C_l; U_l; block] (Section 2 "Preliminaries": draft positions
+    attend to the keys and values made from target hidden states; Algorithm 1: "the next
+    draft reads ctx_l").
+
+    q [S, W, n_q, hd], k_blk / v_blk [S, W, n_kv, hd], q and k_blk NOT yet rotated: block
+    row i of sequence s sits at position L'_s + i.  Returns out [S, W, n_q, hd] and the
+    softmax mass that falls on the carried rows [S, W, n_q] (Appendix C's diagnostic).
+    """
+    cfg = st.cfg
+    S, W = q.shape[0], q.shape[1]
+    rep = cfg.n_q // cfg.n_kv
+    out = np.zeros((S, W, cfg.n_q, cfg.hd), dtype=np.float64)
+    mass = np.zeros((S, W, cfg.n_q), dtype=np.float64)
+    for s in range(S):
+        L = int(st.committed_len[s])
+        pos = (L + np.arange(W)).astype(np.float64)
+        qr = rope(np.asarray(q[s], dtype=np.float64), pos[:, None], cfg.rope_theta)
+        kr = rope(np.asarray(k_blk[s], dtype=np.float64), pos[:, None], cfg.rope_theta)
+        Kctx, Vctx, c = gather_ctx(st, layer, s, use_carry)
+        K = np.concatenate([Kctx, np.transpose(kr, (1, 0, 2))], axis=1)        # [n_kv, T, hd]
+        V = np.concatenate([Vctx, np.transpose(np.asarray(v_blk[s], dtype=np.float64), (1, 0, 2))], axis=1)
+        for g in range(cfg.n_q):
+            h = g // rep
+            sc = (qr[:, g, :] @ K[h].T) / np.sqrt(np.float64(cfg.hd))          # [W, T]
+            sc = sc - sc.max(axis=1, keepdims=True)
+            pr = np.exp(sc)
+            pr = pr / pr.sum(axis=1, keepdims=True)
+            out[s, :, g, :] = pr @ V[h]
+            mass[s, :, g] = pr[:, L:L + c].sum(axis=1)
+    return out, mass
+
+
+# =========================================================================== part 5
+def lm_head_argmax(x: np.ndarray, w: Dict[str, np.ndarray], cfg: OracleConfig):
+    """logits = N_f(x) Emb^T; token = lowest-index argmax; also the top-2 logit gap."""
+    y = rmsnorm(x, w["g_final"], cfg.rms_eps)
+    logits = y @ w["emb"].T
+    tok = np.argmax(logits, axis=1).astype(np.int32)          # first occurrence = lowest id
+    top2 = np.partition(logits, -2, axis=1)[:, -2:]
+    gap = top2[:, 1] - top2[:, 0]
+    return tok, gap, logits
+
+
+# =========================================================================== the drafter pass
+def draft_block(st: OracleState, bonus: np.ndarray, w: Dict[str, np.ndarray],
+                use_carry: bool, keep_logits: bool = False) -> Dict[str, np.ndarray]:
+    """One parallel block prediction from [bonus, MASK, ...] reading ctx_l in every layer."""
+    cfg = st.cfg
+    S, W, D = st.S, cfg.W, cfg.d_model
+    toks = np.full((S, W), cfg.mask_token_id, dtype=np.int64)
+    toks[:, 0] = bonus
+    x = w["emb"][toks.reshape(-1)].copy()                                     # [R, D]
+    attn_out = np.zeros((cfg.n_layers, S * W, cfg.n_q * cfg.hd), dtype=np.float64)
+    mass = np.zeros((cfg.n_layers, S, W, cfg.n_q), dtype=np.float64)
+    for l in range(cfg.n_layers):
+        a = rmsnorm(x, w["g_attn"][l], cfg.rms_eps)
+        q = (a @ w["wq"][l].T).reshape(S, W, cfg.n_q, cfg.hd)
+        kb = (a @ w["wk"][l].T).reshape(S, W, cfg.n_kv, cfg.hd)
+        vb = (a @ w["wv"][l].T).reshape(S, W, cfg.n_kv, cfg.hd)
+        o, mass[l] = block_attn(l, q, kb, vb, st, use_carry)
+        attn_out[l] = o.reshape(S * W, cfg.n_q * cfg.hd)
+        x = x + attn_out[l] @ w["wo"][l].T
+    tok, gap, logits = lm_head_argmax(x, w, cfg)
+    res = {"tok": tok.reshape(S, W), "gap": gap.reshape(S, W), "x_final": x,
+           "attn_out": attn_out, "carry_mass": mass}
+    if keep_logits:
+        res["logits"] = logits
+    return res
+
+
+def draft_round(draft: np.ndarray, target: np.ndarray, H: np.ndarray, st: OracleState,
+                w: Dict[str, np.ndarray], n_forced: int, mode: int,
+                keep_logits: bool = False) -> Dict[str, np.ndarray]:
+    """verify-accept -> project -> scatter -> draft the next block (Algorithm 1, then
+    "the next draft reads ctx_l").  Mutates st.  next_draft = [bonus, tok_1 .. tok_{W-1}]."""
+    cfg = st.cfg
+    split = verify_accept(draft, target, st.committed_len, st.block_table, cfg.page, n_forced)
+    J = project_kv(H, split, w, cfg, mode)
+    scatter_kv(J, split, st, mode)
+    res = draft_block(st, split["bonus"], w, use_carry=(mode == MODE_CARRY), keep_logits=keep_logits)
+    next_draft = res["tok"].copy()
+    next_draft[:, 0] = split["bonus"]
+    res.update(split=split, J=J, next_draft=next_draft.astype(np.int32))
+    return res

@@ -1,0 +1,594 @@
+"""Pins for the CPU oracle: each part is checked against something other than itself —
+closed forms, brute force on tiny inputs, invariants the paper states (Section 2.1 and
+Appendix A "Cache semantics"), and library routines it must reduce to.
+
+The paper prints no worked numeric example for the drafting round (all of its numbers
+need trained checkpoints), so there is no table of printed values to compare with; see
+tests/golden/README.md.
+"""
+import itertools
+import math
+
+import numpy as np
+import pytest
+import torch
+
+from oracle import cod_oracle as orc
+from paper_2609_14717_b200 import synth
+from tests.helpers import oracle_config, oracle_state, small_bf16
+
+
+# ----------------------------------------------------------------------------- part 1
+def _first_zero(bits):
+    """Index of the first False in a tuple of booleans (len if none) — via string search."""
+    s = "".join("1" if b else "0" for b in bits)
+    i = s.find("0")
+    return len(s) if i < 0 else i
+
+
+@pytest.mark.parametrize("n_forced", [0, 1])
+def test_accept_is_prefix_rule_exhaustive_W8(n_forced):
+    W, page = 8, 16
+    pats = list(itertools.product([False, True], repeat=W))
+    S = len(pats)
+    rng = np.random.default_rng(1)
+    draft = rng.integers(0, 50, size=(S, W)).astype(np.int32)
+    target = rng.integers(0, 50, size=(S, W + 1)).astype(np.int32)
+    for s, bits in enumerate(pats):
+        for p, b in enumerate(bits):
+            target[s, p] = draft[s, p] if b else draft[s, p] + 100   # mismatch for certain
+    L = rng.integers(0, 100, size=S).astype(np.int32)
+    bt = rng.permutation(S * 8).reshape(S, 8).astype(np.int32)
+    out = orc.verify_accept(draft, target, L, bt, page, n_forced)
+    for s, bits in enumerate(pats):
+        eff = tuple(b or p < n_forced for p, b in enumerate(bits))
+        m = _first_zero(eff)
+        assert out["accept_len"][s] == m                      # a later match never counts
+        assert out["bonus"][s] == target[s, m]
+    # counts and offsets
+    assert out["acc_off"][-1] + out["rej_off"][-1] == S * W
+    assert np.array_equal(np.diff(out["acc_off"]), out["accept_len"])
+    assert np.array_equal(np.diff(out["rej_off"]), W - out["accept_len"])
+    # lists are the row ids in increasing order, split by acceptance
+    acc = out["acc_rows"][:out["acc_off"][-1]]
+    rej = out["rej_rows"][:out["rej_off"][-1]]
+    assert np.all(np.diff(acc) > 0) and np.all(np.diff(rej) > 0)
+    assert sorted(list(acc) + list(rej)) == list(range(S * W))
+    # slots by the direct formula
+    for row in range(S * W):
+        s, p = divmod(row, W)
+        pos = int(L[s]) + p
+        assert out["row_pos"][row] == pos
+        if p < out["accept_len"][s]:
+            assert out["commit_slot"][row] == bt[s, pos // page] * page + pos % page
+            assert out["carry_slot"][row] == -1
+        else:
+            assert out["commit_slot"][row] == -1
+            assert out["carry_slot"][row] == s * W + p - out["accept_len"][s]
+
+
+@pytest.mark.parametrize("name", ["cfg1", "cfg3"])
+def test_accept_matches_generator_intent(name):
+    """The token generator builds draft/target to realise a chosen m; the oracle must find it."""
+    wl = synth.workload(name)
+    lay = synth.make_layout(wl, 3)
+    for r in range(8):
+        rng = np.random.default_rng([3, 99, r])
+        m = synth.draw_accept(wl, rng)
+        draft, target = synth.make_tokens(wl, rng, m)
+        out = orc.verify_accept(draft, target, lay["committed_len"], lay["block_table"],
+                                wl.shape.page, wl.n_forced)
+        assert np.array_equal(out["accept_len"], m)
+        assert 0 <= (wl.shape.W - out["accept_len"]).max() <= wl.shape.W
+
+
+def test_forced_anchor_row_is_accepted_even_if_tokens_differ():
+    draft = np.array([[5, 6, 7, 8]], dtype=np.int32)
+    target = np.array([[9, 6, 7, 1, 2]], dtype=np.int32)
+    L = np.array([3], dtype=np.int32)
+    bt = np.array([[4, 2]], dtype=np.int32)
+    assert orc.verify_accept(draft, target, L, bt, 16, 0)["accept_len"][0] == 0
+    out = orc.verify_accept(draft, target, L, bt, 16, 1)
+    assert out["accept_len"][0] == 3 and out["bonus"][0] == 1
+
+
+# ----------------------------------------------------------------------------- RoPE / norm
+def test_rope_hand_values():
+    # hd = 2: one pair, frequency 1: (1, 0) at position p turns into (cos p, sin p).
+    out = orc.rope(np.array([1.0, 0.0]), 0.5, 10000.0)
+    assert np.allclose(out, [math.cos(0.5), math.sin(0.5)], atol=1e-15)
+    out = orc.rope(np.array([0.0, 1.0]), 0.5, 10000.0)
+    assert np.allclose(out, [-math.sin(0.5), math.cos(0.5)], atol=1e-15)
+    # hd = 4: pairs (0,2) and (1,3); the second pair turns at theta^(-1/2).
+    x = np.array([1.0, 2.0, 3.0, 4.0])
+    p, th = 7.0, 100.0
+    a0, a1 = p * 1.0, p * th ** -0.5
+    want = [1 * math.cos(a0) - 3 * math.sin(a0), 2 * math.cos(a1) - 4 * math.sin(a1),
+            3 * math.cos(a0) + 1 * math.sin(a0), 4 * math.cos(a1) + 2 * math.sin(a1)]
+    assert np.allclose(orc.rope(x, p, th), want, atol=1e-13)
+
+
+def test_rope_invariants():
+    rng = np.random.default_rng(0)
+    hd = 64
+    q = rng.standard_normal((5, hd))
+    k = rng.standard_normal((5, hd))
+    assert np.array_equal(orc.rope(q, np.zeros(5), 1e6), q)            # position 0 = identity
+    r = orc.rope(q, np.arange(5) * 1000.0, 1e6)
+    assert np.allclose((r ** 2).sum(-1), (q ** 2).sum(-1), rtol=1e-12)  # a rotation
+    half = hd // 2
+    assert np.allclose(r[:, :half] ** 2 + r[:, half:] ** 2,
+                       q[:, :half] ** 2 + q[:, half:] ** 2, rtol=1e-10)
+    # scores depend on the position difference only
+    d1 = (orc.rope(q, np.full(5, 17.0), 1e4) * orc.rope(k, np.full(5, 5.0), 1e4)).sum(-1)
+    d2 = (orc.rope(q, np.full(5, 1012.0), 1e4) * orc.rope(k, np.full(5, 1000.0), 1e4)).sum(-1)
+    assert np.allclose(d1, d2, atol=1e-9)
+
+
+def test_rmsnorm_closed_form():
+    x = np.array([[3.0, 4.0]])
+    g = np.array([2.0, 0.5])
+    # mean square = 12.5
+    want = g * x / math.sqrt(12.5 + 1e-6)
+    assert np.allclose(orc.rmsnorm(x, g, 1e-6), want, atol=1e-15)
+    y = orc.rmsnorm(np.random.default_rng(0).standard_normal((4, 256)) * 7, np.ones(256), 0.0)
+    assert np.allclose((y ** 2).mean(-1), 1.0)
+
+
+# ----------------------------------------------------------------------------- part 2
+def _tiny(norm=True, **kw):
+    wl = synth.workload("cfg1")
+    wl = synth.scaled(wl, hidden_norm=norm, **kw)
+    cfg = oracle_config(wl.shape)
+    w = orc.prepare_weights(synth.make_weights(wl.shape, 5))
+    return wl, cfg, w
+
+
+def _split_for(wl, m, seed=0):
+    lay = synth.make_layout(wl, seed)
+    rng = np.random.default_rng(seed + 77)
+    draft, target = synth.make_tokens(wl, rng, np.asarray(m, dtype=np.int32))
+    sp = orc.verify_accept(draft, target, lay["committed_len"], lay["block_table"], wl.shape.page, 0)
+    assert np.array_equal(sp["accept_len"], m)
+    return sp, lay
+
+
+def test_project_linearity_in_carry_embedding():
+    """Norm off: Phi(h + E) = Phi(h) + Phi(E) row-wise, also after the key rotation."""
+    wl, cfg, w = _tiny(norm=False, S=2)
+    sp, _ = _split_for(wl, [3, 0])
+    H = synth.make_round(wl, 0, 0)["H"].astype(np.float64)
+    J = orc.project_kv(H, sp, w, cfg, orc.MODE_CARRY)
+    w0 = dict(w, e_carry=np.zeros_like(w["e_carry"]))
+    J0 = orc.project_kv(H, sp, w0, cfg, orc.MODE_CARRY)
+    # Phi(E) alone, at each row's own position
+    HE = np.tile(w["e_carry"], (wl.R, 1))
+    sp_all = dict(sp, accept_len=np.array([wl.shape.W] * wl.S))       # nothing rejected
+    JE = orc.project_kv(HE, sp_all, w0, cfg, orc.MODE_CARRY)
+    rej = np.repeat(sp["accept_len"], wl.shape.W) <= np.tile(np.arange(wl.shape.W), wl.S)
+    assert rej.sum() == 5 + 8
+    assert np.allclose(J[:, rej], J0[:, rej] + JE[:, rej], atol=1e-12)
+    assert np.array_equal(J[:, ~rej], J0[:, ~rej])                  # accepted rows never see E
+
+
+@pytest.mark.parametrize("norm", [False, True])
+def test_rejected_rows_use_the_same_path_when_E_is_zero(norm):
+    """E_carry = 0: a rejected row's K/V equal what the accepted-row path gives for it."""
+    wl, cfg, w = _tiny(norm=norm, S=2)
+    w0 = dict(w, e_carry=np.zeros_like(w["e_carry"]))
+    H = synth.make_round(wl, 0, 1)["H"]
+    sp, _ = _split_for(wl, [2, 5])
+    J = orc.project_kv(H, sp, w0, cfg, orc.MODE_CARRY)
+    sp_all = dict(sp, accept_len=np.array([wl.shape.W] * wl.S))
+    Jb = orc.project_kv(H, sp_all, w0, cfg, orc.MODE_BASELINE)
+    assert np.array_equal(J, Jb)
+    # and with E != 0 the rejected rows do change, the accepted ones do not
+    JE = orc.project_kv(H, sp, w, cfg, orc.MODE_CARRY)
+    rej = np.repeat(sp["accept_len"], wl.shape.W) <= np.tile(np.arange(wl.shape.W), wl.S)
+    assert np.array_equal(JE[:, ~rej], J[:, ~rej])
+    assert np.abs(JE[:, rej] - J[:, rej]).max() > 1e-3
+
+
+def test_baseline_projects_accepted_rows_only():
+    wl, cfg, w = _tiny(S=2)
+    H = synth.make_round(wl, 0, 2)["H"]
+    sp, _ = _split_for(wl, [2, 8])
+    Jb = orc.project_kv(H, sp, w, cfg, orc.MODE_BASELINE)
+    Jc = orc.project_kv(H, sp, w, cfg, orc.MODE_CARRY)
+    rej = np.repeat(sp["accept_len"], wl.shape.W) <= np.tile(np.arange(wl.shape.W), wl.S)
+    assert np.isnan(Jb[:, rej]).all()
+    assert np.array_equal(Jb[:, ~rej], Jc[:, ~rej])
+
+
+def test_project_with_selection_weights_is_a_copy():
+    """One-hot F, K, V (norm off) and position 0: the outputs are exact copies of H entries."""
+    wl, cfg, w = _tiny(norm=False)
+    D, Din, kvw = cfg.d_model, cfg.d_in, cfg.n_kv * cfg.hd
+    rng = np.random.default_rng(4)
+    sel_f = rng.permutation(Din)[:D]
+    sel_k = rng.permutation(D)[:kvw]
+    sel_v = rng.permutation(D)[:kvw]
+    w = dict(w)
+    w["fc"] = np.zeros((D, Din)); w["fc"][np.arange(D), sel_f] = 1.0
+    w["wk"] = np.zeros((1, kvw, D)); w["wk"][0, np.arange(kvw), sel_k] = 1.0
+    w["wv"] = np.zeros((1, kvw, D)); w["wv"][0, np.arange(kvw), sel_v] = 1.0
+    H = synth.make_round(wl, 0, 0)["H"].astype(np.float64)
+    W = cfg.W
+    sp = {"accept_len": np.array([3]), "row_pos": np.zeros(W, dtype=np.int32)}
+    J = orc.project_kv(H, sp, w, cfg, orc.MODE_CARRY)
+    Hk = H.copy(); Hk[3:] += w["e_carry"]
+    assert np.array_equal(J[0, :, 1].reshape(W, kvw), Hk[:, sel_f][:, sel_v])
+    assert np.array_equal(J[0, :, 0].reshape(W, kvw), Hk[:, sel_f][:, sel_k])
+
+
+def test_project_against_torch_linear():
+    """The same maps through torch's float64 linear layers and an explicit rotation."""
+    wl, cfg, w = _tiny(S=2)
+    H = synth.make_round(wl, 0, 3)["H"]
+    sp, _ = _split_for(wl, [4, 1])
+    J = orc.project_kv(H, sp, w, cfg, orc.MODE_CARRY)
+    t = lambda a: torch.from_numpy(np.asarray(a, dtype=np.float64))
+    Ht = t(H).clone()
+    for s, m in enumerate([4, 1]):
+        Ht[s * 8 + m:(s + 1) * 8] += t(w["e_carry"])
+    Z = torch.nn.functional.linear(Ht, t(w["fc"]))
+    Z = Z * torch.rsqrt((Z * Z).mean(-1, keepdim=True) + cfg.rms_eps) * t(w["g_hidden"])
+    K = torch.nn.functional.linear(Z, t(w["wk"][0])).reshape(-1, cfg.n_kv, cfg.hd)
+    V = torch.nn.functional.linear(Z, t(w["wv"][0])).reshape(-1, cfg.n_kv, cfg.hd)
+    half = cfg.hd // 2
+    inv = cfg.rope_theta ** (-torch.arange(half, dtype=torch.float64) * 2 / cfg.hd)
+    ang = t(sp["row_pos"])[:, None, None] * inv
+    Kr = torch.cat([K[..., :half] * ang.cos() - K[..., half:] * ang.sin(),
+                    K[..., half:] * ang.cos() + K[..., :half] * ang.sin()], -1)
+    assert np.allclose(J[0, :, 0], Kr.numpy(), atol=1e-12)
+    assert np.allclose(J[0, :, 1], V.numpy(), atol=1e-12)
+
+
+# ----------------------------------------------------------------------------- part 3
+def test_scatter_semantics_over_rounds():
+    """Carry never exceeds W rows, is replaced each round, starts empty; rejected rows never
+    reach the committed cache; committed rows are exact copies and older rows never change."""
+    wl = synth.scaled(synth.workload("cfg1"), S=3, ctx=(5, 40), n_rounds=6)
+    cfg, st, lay = oracle_state(wl, 2)
+    w = orc.prepare_weights(synth.make_weights(wl.shape, 2))
+    assert (st.carry_len == 0).all() and np.isnan(st.carry).all()
+    W, page = cfg.W, cfg.page
+    for r in range(6):
+        rd = synth.make_round(wl, 2, r)
+        pool_before = st.pool.copy()
+        L0 = st.committed_len.copy()
+        sp = orc.verify_accept(rd["draft"], rd["target"], st.committed_len, st.block_table, page, wl.n_forced)
+        J = orc.project_kv(rd["H"], sp, w, cfg, orc.MODE_CARRY)
+        orc.scatter_kv(J, sp, st, orc.MODE_CARRY)
+        m = sp["accept_len"]
+        assert np.array_equal(st.committed_len, L0 + m)
+        assert np.array_equal(st.carry_len, W - m) and (st.carry_len <= W).all()
+        changed = np.zeros(st.pool.shape, dtype=bool)
+        for s in range(wl.S):
+            c = int(st.carry_len[s])
+            assert np.isnan(st.carry[:, s, :, :, c:, :]).all()          # old carry is gone
+            for p in range(W):
+                pos = int(L0[s]) + p
+                pg, off = st.block_table[s, pos // page], pos % page
+                if p < m[s]:
+                    assert np.array_equal(st.pool[:, pg, :, :, off, :],
+                                          np.transpose(J[:, s * W + p], (0, 2, 1, 3)))
+                    changed[:, pg, :, :, off, :] = True
+                else:
+                    assert np.array_equal(st.carry[:, s, :, :, p - m[s], :],
+                                          np.transpose(J[:, s * W + p], (0, 2, 1, 3)))
+        assert np.array_equal(st.pool[~changed], pool_before[~changed])
+
+
+def test_baseline_scatter_leaves_carry_empty():
+    wl = synth.scaled(synth.workload("cfg1"), S=2, ctx=(5, 40))
+    cfg, st, _ = oracle_state(wl, 2)
+    w = orc.prepare_weights(synth.make_weights(wl.shape, 2))
+    rd = synth.make_round(wl, 2, 0)
+    orc.draft_round(rd["draft"], rd["target"], rd["H"], st, w, wl.n_forced, orc.MODE_BASELINE)
+    assert (st.carry_len == 0).all() and np.isnan(st.carry).all()
+
+
+# ----------------------------------------------------------------------------- part 4
+def _attn_case(seed=0, S=2, carry=True):
+    wl = synth.scaled(synth.workload("cfg1"), S=S, ctx=(3, 45))
+    cfg, st, lay = oracle_state(wl, seed)
+    rng = np.random.default_rng(seed + 10)
+    if carry:
+        st.carry_len[:] = rng.integers(1, cfg.W + 1, size=S)
+        for s in range(S):
+            c = int(st.carry_len[s])
+            st.carry[:, s, :, :, :c, :] = rng.standard_normal((cfg.n_layers, cfg.n_kv, 2, c, cfg.hd))
+    q = rng.standard_normal((S, cfg.W, cfg.n_q, cfg.hd))
+    kb = rng.standard_normal((S, cfg.W, cfg.n_kv, cfg.hd))
+    vb = rng.standard_normal((S, cfg.W, cfg.n_kv, cfg.hd))
+    return wl, cfg, st, q, kb, vb
+
+
+def _rope_scalar(x, pos, theta):
+    """Independent scalar-loop rotation used by the brute-force attention."""
+    hd = len(x)
+    half = hd // 2
+    out = [0.0] * hd
+    for j in range(half):
+        a = pos * theta ** (-2.0 * j / hd)
+        out[j] = x[j] * math.cos(a) - x[j + half] * math.sin(a)
+        out[j + half] = x[j + half] * math.cos(a) + x[j] * math.sin(a)
+    return out
+
+
+def test_attention_brute_force_loops():
+    """Materialised scores in pure Python loops with a page-table walk of its own."""
+    wl, cfg, st, q, kb, vb = _attn_case(seed=1, S=2)
+    out, mass = orc.block_attn(0, q, kb, vb, st, use_carry=True)
+    rep = cfg.n_q // cfg.n_kv
+    for s in range(2):
+        L, c = int(st.committed_len[s]), int(st.carry_len[s])
+        for i in (0, cfg.W - 1):
+            for g in (0, cfg.n_q - 1):
+                h = g // rep
+                qq = _rope_scalar(list(q[s, i, g]), L + i, cfg.rope_theta)
+                keys, vals = [], []
+                for t in range(L):
+                    pg = int(st.block_table[s, t // cfg.page])
+                    keys.append(list(st.pool[0, pg, h, 0, t % cfg.page]))
+                    vals.append(list(st.pool[0, pg, h, 1, t % cfg.page]))
+                for u in range(c):
+                    keys.append(list(st.carry[0, s, h, 0, u]))
+                    vals.append(list(st.carry[0, s, h, 1, u]))
+                for jb in range(cfg.W):
+                    keys.append(_rope_scalar(list(kb[s, jb, h]), L + jb, cfg.rope_theta))
+                    vals.append(list(vb[s, jb, h]))
+                sc = [sum(a * b for a, b in zip(qq, k)) / math.sqrt(cfg.hd) for k in keys]
+                mx = max(sc)
+                e = [math.exp(v - mx) for v in sc]
+                z = sum(e)
+                o = [sum(e[t] * vals[t][d] for t in range(len(e))) / z for d in range(cfg.hd)]
+                assert np.allclose(out[s, i, g], o, atol=1e-12)
+                assert abs(mass[s, i, g] - sum(e[L:L + c]) / z) < 1e-12
+
+
+def test_attention_is_plain_sdpa_over_concatenated_keys():
+    """Once [C; U; block] is concatenated and GQA heads repeated, it is library SDPA."""
+    wl, cfg, st, q, kb, vb = _attn_case(seed=2, S=2)
+    out, _ = orc.block_attn(0, q, kb, vb, st, use_carry=True)
+    rep = cfg.n_q // cfg.n_kv
+    for s in range(2):
+        L, c = int(st.committed_len[s]), int(st.carry_len[s])
+        pos = L + np.arange(cfg.W)
+        t_idx = np.arange(L)
+        pg = st.block_table[s, t_idx // cfg.page]
+        Kc = np.stack([st.pool[0, pg[t], :, 0, t % cfg.page] for t in range(L)], 0)    # [L, n_kv, hd]
+        Vc = np.stack([st.pool[0, pg[t], :, 1, t % cfg.page] for t in range(L)], 0)
+        Ku = np.transpose(st.carry[0, s, :, 0, :c], (1, 0, 2))
+        Vu = np.transpose(st.carry[0, s, :, 1, :c], (1, 0, 2))
+        Kb = np.stack([[_rope_scalar(list(kb[s, j, h]), int(pos[j]), cfg.rope_theta)
+                        for h in range(cfg.n_kv)] for j in range(cfg.W)], 0)
+        K = np.concatenate([Kc, Ku, Kb], 0)
+        V = np.concatenate([Vc, Vu, vb[s]], 0)
+        Q = np.stack([[_rope_scalar(list(q[s, i, g]), int(pos[i]), cfg.rope_theta)
+                       for g in range(cfg.n_q)] for i in range(cfg.W)], 0)
+        Kt = torch.from_numpy(K).permute(1, 0, 2).repeat_interleave(rep, 0)   # [n_q, T, hd]
+        Vt = torch.from_numpy(V).permute(1, 0, 2).repeat_interleave(rep, 0)
+        Qt = torch.from_numpy(Q).permute(1, 0, 2)
+        ref = torch.nn.functional.scaled_dot_product_attention(Qt, Kt, Vt)      # [n_q, W, hd]
+        assert np.allclose(out[s], ref.permute(1, 0, 2).numpy(), atol=1e-11)
+
+
+def test_attention_closed_forms():
+    wl = synth.scaled(synth.workload("cfg1"), S=1, ctx=(0, 0), W=1)
+    cfg, st, _ = oracle_state(wl, 0)
+    rng = np.random.default_rng(0)
+    # one key in total (the block row itself): output = its V
+    q = rng.standard_normal((1, 1, cfg.n_q, cfg.hd))
+    kb = rng.standard_normal((1, 1, cfg.n_kv, cfg.hd))
+    vb = rng.standard_normal((1, 1, cfg.n_kv, cfg.hd))
+    out, _ = orc.block_attn(0, q, kb, vb, st, use_carry=True)
+    rep = cfg.n_q // cfg.n_kv
+    for g in range(cfg.n_q):
+        assert np.allclose(out[0, 0, g], vb[0, 0, g // rep], atol=1e-15)
+    # identical keys everywhere: output = mean of the values
+    wl = synth.scaled(synth.workload("cfg1"), S=1, ctx=(20, 20))
+    cfg, st, _ = oracle_state(wl, 0)
+    st.pool[:, :, :, 0] = 0.0                                    # all committed keys = 0
+    kb = np.zeros((1, cfg.W, cfg.n_kv, cfg.hd))                  # rotation of 0 is 0
+    vb = rng.standard_normal((1, cfg.W, cfg.n_kv, cfg.hd))
+    q = rng.standard_normal((1, cfg.W, cfg.n_q, cfg.hd))
+    out, _ = orc.block_attn(0, q, kb, vb, st, use_carry=False)
+    pg = st.block_table[0, np.arange(20) // cfg.page]
+    for g in range(cfg.n_q):
+        h = g // rep
+        vals = [st.pool[0, pg[t], h, 1, t % cfg.page] for t in range(20)] + list(vb[0, :, h])
+        assert np.allclose(out[0, 3, g], np.mean(vals, axis=0), atol=1e-13)
+    # two keys with scores 0 and ln 3 (hd = 4, scale 1/2): weights 1/4 and 3/4
+    wl = synth.scaled(synth.workload("cfg1"), S=1, ctx=(1, 1), W=1, hd=4, n_q=1, n_kv=1, d_model=4)
+    cfg, st, _ = oracle_state(wl, 0)
+    pg = st.block_table[0, 0]
+    st.pool[0, pg, 0, 0, 0] = [0.0, 0.0, 0.0, 0.0]
+    st.pool[0, pg, 0, 1, 0] = [1.0, 0.0, 0.0, 0.0]
+    q = np.array([[[[2 * math.log(3.0), 0.0, 0.0, 0.0]]]])
+    kb = np.array([[[[1.0, 0.0, 0.0, 0.0]]]])
+    vb = np.array([[[[0.0, 1.0, 0.0, 0.0]]]])
+    # q and k_blk sit at the same position, so the rotation leaves their product unchanged
+    out, _ = orc.block_attn(0, q, kb, vb, st, use_carry=True)
+    assert np.allclose(out[0, 0, 0], [0.25, 0.75, 0.0, 0.0], atol=1e-14)
+
+
+def test_attention_masked_carry_equals_baseline_and_mass():
+    wl, cfg, st, q, kb, vb = _attn_case(seed=3)
+    out_c, mass_c = orc.block_attn(0, q, kb, vb, st, use_carry=True)
+    out_b, mass_b = orc.block_attn(0, q, kb, vb, st, use_carry=False)
+    assert np.abs(out_c - out_b).max() > 1e-3 and (mass_c > 0).all() and (mass_c < 1).all()
+    assert (mass_b == 0).all()
+    keep = st.carry_len.copy()
+    st.carry_len[:] = 0                                            # empty carry = baseline
+    out_0, _ = orc.block_attn(0, q, kb, vb, st, use_carry=True)
+    assert np.array_equal(out_0, out_b)
+    st.carry_len[:] = keep
+
+
+def test_attention_page_permutation_invariance():
+    wl, cfg, st, q, kb, vb = _attn_case(seed=4)
+    out, _ = orc.block_attn(0, q, kb, vb, st, use_carry=True)
+    n_pages = st.pool.shape[1]
+    perm = np.random.default_rng(9).permutation(n_pages)
+    inv = np.argsort(perm)
+    st2 = orc.OracleState(cfg, st.S, n_pages, perm[st.block_table], st.committed_len)
+    st2.pool = st.pool[:, inv]
+    st2.carry, st2.carry_len = st.carry, st.carry_len
+    out2, _ = orc.block_attn(0, q, kb, vb, st2, use_carry=True)
+    assert np.array_equal(out, out2)
+
+
+def test_attention_depends_on_relative_position_only():
+    """Move every row (committed, carried, block) delta positions later, re-rotating the stored
+    keys by delta: the outputs must not change.  The delta vacated leading positions hold
+    zero keys / zero values, whose scores are 0 whatever the rotation; the expected result is
+    computed directly with those filler rows in front."""
+    wl, cfg, st, q, kb, vb = _attn_case(seed=4)
+    delta = 37
+    n_pages = st.pool.shape[1]
+    bt = np.zeros((st.S, 16), dtype=np.int64)
+    shifted = orc.OracleState(cfg, st.S, n_pages + 64, bt, st.committed_len + delta)
+    stale = orc.OracleState(cfg, st.S, n_pages + 64, bt, st.committed_len + delta)
+    nxt = 0
+    for s in range(st.S):
+        L = int(st.committed_len[s])
+        npg = (L + delta + cfg.page - 1) // cfg.page
+        bt[s, :npg] = np.arange(nxt, nxt + npg); nxt += npg
+        shifted.block_table[s] = bt[s]; stale.block_table[s] = bt[s]
+        K, V, c = orc.gather_ctx(st, 0, s, True)                   # [n_kv, L + c, hd]
+        Kr = orc.rope(K, np.full(K.shape[1], float(delta))[None, :], cfg.rope_theta)
+        for dst, Kuse in ((shifted, Kr), (stale, K)):
+            for t in range(L):
+                pos = t + delta
+                pg = dst.block_table[s, pos // cfg.page]
+                dst.pool[0, pg, :, 0, pos % cfg.page] = Kuse[:, t]
+                dst.pool[0, pg, :, 1, pos % cfg.page] = V[:, t]
+            dst.carry[0, s, :, 0, :c] = Kuse[:, L:L + c]
+            dst.carry[0, s, :, 1, :c] = V[:, L:L + c]
+            dst.carry_len[s] = c
+    out_shift, _ = orc.block_attn(0, q, kb, vb, shifted, use_carry=True)
+    out_stale, _ = orc.block_attn(0, q, kb, vb, stale, use_carry=True)
+    assert np.abs(out_stale - out_shift).max() > 1e-4              # keys do carry their position
+    rep = cfg.n_q // cfg.n_kv
+    for s in range(st.S):
+        L = int(st.committed_len[s])
+        K, V, c = orc.gather_ctx(st, 0, s, True)
+        pos = (L + np.arange(cfg.W)).astype(np.float64)
+        qr = orc.rope(q[s], pos[:, None], cfg.rope_theta)
+        kr = orc.rope(kb[s], pos[:, None], cfg.rope_theta)
+        for g in range(cfg.n_q):
+            h = g // rep
+            Kall = np.concatenate([np.zeros((delta, cfg.hd)), K[h], kr[:, h]], 0)
+            Vall = np.concatenate([np.zeros((delta, cfg.hd)), V[h], vb[s][:, h]], 0)
+            sc = qr[:, g] @ Kall.T / math.sqrt(cfg.hd)
+            pr = np.exp(sc - sc.max(1, keepdims=True)); pr /= pr.sum(1, keepdims=True)
+            assert np.allclose(out_shift[s, :, g], pr @ Vall, atol=1e-9)
+
+
+# ----------------------------------------------------------------------------- part 5
+def test_lm_head_planted_maximum_and_ties():
+    wl, cfg, w = _tiny()
+    rng = np.random.default_rng(0)
+    x = rng.standard_normal((6, cfg.d_model))
+    y = orc.rmsnorm(x, w["g_final"], cfg.rms_eps)
+    for row, v in enumerate([0, 127, 128, 500, cfg.vocab - 2, cfg.vocab - 1]):
+        w2 = dict(w); emb = w["emb"].copy(); emb[v] = y[row] * 10.0; w2["emb"] = emb
+        tok, gap, _ = orc.lm_head_argmax(x, w2, cfg)
+        assert tok[row] == v and gap[row] > 0
+    # exact tie between two vocabulary rows: the lower id wins, the gap is zero
+    w2 = dict(w); emb = w["emb"].copy(); emb[700] = y[2] * 10.0; emb[33] = emb[700]; w2["emb"] = emb
+    tok, gap, _ = orc.lm_head_argmax(x, w2, cfg)
+    assert tok[2] == 33 and gap[2] == 0.0
+
+
+def test_lm_head_brute_force():
+    wl, cfg, w = _tiny()
+    x = np.random.default_rng(1).standard_normal((3, cfg.d_model))
+    tok, gap, _ = orc.lm_head_argmax(x, w, cfg)
+    for r in range(3):
+        ms = math.sqrt(sum(v * v for v in x[r]) / cfg.d_model + cfg.rms_eps)
+        y = [w["g_final"][d] * x[r, d] / ms for d in range(cfg.d_model)]
+        logits = [math.fsum(w["emb"][v, d] * y[d] for d in range(cfg.d_model)) for v in range(cfg.vocab)]
+        best = max(range(cfg.vocab), key=lambda v: (logits[v], -v))
+        srt = sorted(logits)
+        assert tok[r] == best
+        assert abs(gap[r] - (srt[-1] - srt[-2])) < 1e-12
+
+
+# ----------------------------------------------------------------------------- whole round
+def test_full_acceptance_round_equals_baseline_round():
+    """Full acceptance leaves U empty, so the round is the no-carryover drafter's round."""
+    wl = synth.scaled(synth.workload("cfg1"), S=2, ctx=(20, 60), accept=("fixed_m", 8), n_forced=0)
+    cfg, st_c, _ = oracle_state(wl, 1)
+    _, st_b, _ = oracle_state(wl, 1)
+    w = orc.prepare_weights(synth.make_weights(wl.shape, 1))
+    w["wo"] = w["wo"] * 40.0                                       # make the attention path matter
+    for r in range(3):
+        rd = synth.make_round(wl, 1, r)
+        rc = orc.draft_round(rd["draft"], rd["target"], rd["H"], st_c, w, 0, orc.MODE_CARRY, keep_logits=True)
+        rb = orc.draft_round(rd["draft"], rd["target"], rd["H"], st_b, w, 0, orc.MODE_BASELINE, keep_logits=True)
+        assert (st_c.carry_len == 0).all()
+        assert np.array_equal(rc["logits"], rb["logits"])
+        assert np.array_equal(rc["next_draft"], rb["next_draft"])
+        assert np.array_equal(st_c.pool, st_b.pool)
+
+
+def test_partial_acceptance_differs_from_baseline_and_commits_the_same():
+    wl = synth.scaled(synth.workload("cfg1"), S=2, ctx=(20, 60))
+    cfg, st_c, _ = oracle_state(wl, 1)
+    _, st_b, _ = oracle_state(wl, 1)
+    w = orc.prepare_weights(synth.make_weights(wl.shape, 1))
+    w["wo"] = w["wo"] * 40.0
+    differs = False
+    for r in range(4):
+        rd = synth.make_round(wl, 1, r)
+        rc = orc.draft_round(rd["draft"], rd["target"], rd["H"], st_c, w, 1, orc.MODE_CARRY)
+        rb = orc.draft_round(rd["draft"], rd["target"], rd["H"], st_b, w, 1, orc.MODE_BASELINE)
+        # the acceptance rule and the committed cache do not depend on carryover
+        assert np.array_equal(rc["split"]["accept_len"], rb["split"]["accept_len"])
+        assert np.array_equal(st_c.pool, st_b.pool)
+        assert np.array_equal(st_c.committed_len, st_b.committed_len)
+        differs |= np.abs(rc["x_final"] - rb["x_final"]).max() > 1e-6
+    assert differs
+
+
+def test_committed_cache_equals_from_scratch_recomputation():
+    """After many rounds the committed rows are exactly Phi of the concatenated accepted
+    hiddens at positions 0.., computed in one go without any paging."""
+    wl = synth.scaled(synth.workload("cfg1"), S=2, ctx=(0, 0), n_rounds=16)
+    cfg, st, _ = oracle_state(wl, 6, fill_pool=False)
+    w = orc.prepare_weights(synth.make_weights(wl.shape, 6))
+    kept = [[], []]
+    for r in range(16):
+        rd = synth.make_round(wl, 6, r)
+        res = orc.draft_round(rd["draft"], rd["target"], rd["H"], st, w, 1, orc.MODE_CARRY)
+        for s in range(2):
+            kept[s].append(rd["H"][s * cfg.W: s * cfg.W + int(rd["m"][s])])
+    for s in range(2):
+        Hs = np.concatenate(kept[s], 0).astype(np.float64)
+        L = Hs.shape[0]
+        assert L == st.committed_len[s]
+        Z = Hs @ w["fc"].T
+        Z = w["g_hidden"] * Z / np.sqrt((Z * Z).mean(-1, keepdims=True) + cfg.rms_eps)
+        K = orc.rope((Z @ w["wk"][0].T).reshape(L, cfg.n_kv, cfg.hd), np.arange(L)[:, None], cfg.rope_theta)
+        V = (Z @ w["wv"][0].T).reshape(L, cfg.n_kv, cfg.hd)
+        Kc, Vc, _ = orc.gather_ctx(st, 0, s, use_carry=False)
+        assert np.allclose(np.transpose(Kc, (1, 0, 2)), K, atol=1e-12)
+        assert np.allclose(np.transpose(Vc, (1, 0, 2)), V, atol=1e-12)
+
+
+def test_round_is_deterministic_and_next_draft_shape():
+    wl = small_bf16()
+    outs = []
+    for _ in range(2):
+        cfg, st, _ = oracle_state(wl, 0)
+        w = orc.prepare_weights(synth.make_weights(wl.shape, 0))
+        rd = synth.make_round(wl, 0, 0)
+        res = orc.draft_round(rd["draft"], rd["target"], rd["H"], st, w, 1, orc.MODE_CARRY)
+        outs.append(res)
+    assert np.array_equal(outs[0]["x_final"], outs[1]["x_final"])
+    nd = outs[0]["next_draft"]
+    assert nd.shape == (wl.S, wl.shape.W) and np.array_equal(nd[:, 0], outs[0]["split"]["bonus"])
+    assert np.array_equal(nd[:, 1:], outs[0]["tok"][:, 1:])
