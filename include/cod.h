@@ -1,0 +1,210 @@
+/* cod.h — C ABI of the Carryover drafting round for NVIDIA B200 (sm_100a).
+ *
+ * One "round" is what a block-diffusion drafter does between two target
+ * verifications (paper: Section 2 "Carryover Drafting", Eq. 1-2; Appendix A,
+ * Algorithm 1 and its "Cache semantics" paragraph):
+ *
+ *   1. greedy verify-accept of the drafted block against the target's tokens;
+ *   2. projection of the target's concatenated multi-layer hidden states into
+ *      drafter K/V through the existing fusion map F and the per-layer K_l, V_l,
+ *      with the learned embedding E_carry added to the REJECTED rows only;
+ *   3. accepted rows are appended to the paged committed drafter cache C_l,
+ *      rejected rows replace the one-block carryover slot U_l;
+ *   4. the next block ([bonus, MASK, ...]) attends to [C_l; U_l; block];
+ *   5. the tied LM head with a fused argmax gives the next proposals.
+ *
+ * Conventions
+ *   - Every function returns 0 (COD_OK) or a negative cod_status. Nothing throws.
+ *   - "device" pointers are CUDA device addresses owned by the caller and only
+ *     borrowed for the call; "host" pointers are ordinary host addresses.
+ *   - All work is enqueued on the caller's stream (a cudaStream_t passed as
+ *     void*); no call synchronises the host except cod_create, cod_destroy
+ *     and cod_poll_status. Results are valid once the stream has been
+ *     synchronised by the caller.
+ *   - After cod_create the library allocates nothing (the workspace is sized
+ *     from cod_config at creation).
+ *   - What only the device can see (a position beyond the page table, a token
+ *     id outside the vocabulary, an expired bounded wait) sets a bit in a sticky
+ *     device status word; the offending access is skipped and the kernel ends
+ *     normally. cod_poll_status copies the word out.
+ *   - Element type: COD_BF16 = bfloat16 storage, COD_F32 = float storage, for
+ *     weights, H, the KV pool, the carry slot, J, q/k/v/out. Accumulation,
+ *     norms, softmax and the residual stream are float in both.
+ *   - Layouts are row-major with the last index contiguous.
+ */
+#ifndef COD_H_
+#define COD_H_
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct cod_ctx cod_ctx;
+typedef void* cod_stream_t; /* a cudaStream_t */
+
+enum cod_status {
+  COD_OK = 0,
+  COD_ERR_INVALID_ARG = -1, /* NULL pointer, size out of range, misaligned pointer */
+  COD_ERR_UNSUPPORTED = -2, /* a shape or flag this build has no kernel for */
+  COD_ERR_CUDA = -3,        /* a CUDA runtime call or launch failed */
+  COD_ERR_NO_WEIGHTS = -4,  /* cod_set_weights has not been called */
+  COD_ERR_ALLOC = -5        /* cod_create could not allocate its workspace */
+};
+
+enum cod_dtype { COD_F32 = 0, COD_BF16 = 1 };
+enum cod_mode {
+  COD_CARRY = 0,   /* Algorithm 1, right column: all rows projected, rejected rows carried */
+  COD_BASELINE = 1 /* Algorithm 1, left column: accepted rows only, U_l left empty */
+};
+
+/* cod_config.flags */
+#define COD_F_HIDDEN_NORM 1u /* RMS-normalise (with gain g_hidden) the output of F */
+
+/* bits of the sticky device status word */
+#define COD_DEV_BAD_TOKEN 1u      /* a token id outside [0, vocab) was met (treated as id 0) */
+#define COD_DEV_PAGE_OVERFLOW 2u  /* a position fell beyond max_pages_per_seq (row not stored) */
+#define COD_DEV_BAD_PAGE 4u       /* block_table held a page id outside [0, n_pages) */
+#define COD_DEV_TIMEOUT 8u        /* a bounded device-side wait gave up */
+#define COD_DEV_BAD_LEN 16u       /* committed_len / carry_len outside its range */
+
+/* Immutable description of the drafter and of the capacities the workspace is sized for. */
+typedef struct {
+  int32_t d_target;          /* width of one captured target layer                         */
+  int32_t n_cap;             /* captured target layers; D_in = d_target * n_cap            */
+  int32_t d_model;           /* drafter width D; must equal n_q_heads * head_dim           */
+  int32_t n_layers;          /* drafter layers Ld                                          */
+  int32_t n_q_heads, n_kv_heads, head_dim;
+  int32_t vocab;             /* LM head = transposed embedding table                       */
+  int32_t mask_token_id;
+  int32_t block;             /* W: rows of the verified window = drafted block size        */
+  int32_t page_size;         /* tokens per KV page                                         */
+  int32_t max_batch;         /* largest S any call will pass                               */
+  int32_t max_pages_per_seq; /* row length of block_table                                  */
+  int32_t n_pages;           /* pages in kv_pool (per layer)                               */
+  int32_t dtype;             /* cod_dtype                                                  */
+  uint32_t flags;
+  float rope_theta, rms_eps;
+  int32_t attn_split_len;    /* keys per attention split (a multiple of 32); 0 = library default */
+} cod_config;
+
+/* Borrowed device pointers, element type per cod_config.dtype, each matrix [out, in]. */
+typedef struct {
+  const void* fc;       /* [D, D_in]            the fusion map F                           */
+  const void* e_carry;  /* [D_in]               E_carry (Eq. 2)                            */
+  const void* g_hidden; /* [D]                  gain of the norm after F                   */
+  const void* wk;       /* [Ld][n_kv*hd, D]     K_l                                        */
+  const void* wv;       /* [Ld][n_kv*hd, D]     V_l                                        */
+  const void* wq;       /* [Ld][n_q*hd, D]                                                 */
+  const void* wo;       /* [Ld][D, n_q*hd]                                                 */
+  const void* g_attn;   /* [Ld][D]              gain of the pre-attention norm             */
+  const void* g_final;  /* [D]                  gain of the final norm                     */
+  const void* emb;      /* [vocab, D]           embedding table = LM head                  */
+} cod_weights;
+
+/* Mutable drafter state of a batch (device, caller-owned). */
+typedef struct {
+  void* kv_pool;          /* [Ld][n_pages][n_kv][2][page][hd]  C_l; index 3: 0 = K (rotated), 1 = V */
+  int32_t* block_table;   /* [S][max_pages_per_seq]            physical page of each logical page  */
+  int32_t* committed_len; /* [S]   L_s; cod_scatter_kv adds the accepted rows                      */
+  void* carry_kv;         /* [Ld][max_batch][n_kv][2][W][hd]   U_l (rows >= carry_len are stale)   */
+  int32_t* carry_len;     /* [S]   c_s in 0..W, overwritten every round                            */
+} cod_state;
+
+/* Output of cod_verify_accept (device, caller-owned). Row ids are s*W + p. */
+typedef struct {
+  int32_t* accept_len;  /* [S]     m_s                                                      */
+  int32_t* bonus;       /* [S]     target[s, m_s]                                           */
+  int32_t* row_pos;     /* [S*W]   absolute position L_s + p                                */
+  int32_t* commit_slot; /* [S*W]   page*page_size + offset for accepted rows, else -1       */
+  int32_t* carry_slot;  /* [S*W]   s*W + (p - m_s) for rejected rows, else -1               */
+  int32_t* acc_rows;    /* [S*W]   accepted row ids, increasing; tail filled with -1        */
+  int32_t* acc_off;     /* [S+1]   exclusive prefix sums of m_s                             */
+  int32_t* rej_rows;    /* [S*W]   rejected row ids, increasing; tail filled with -1        */
+  int32_t* rej_off;     /* [S+1]   exclusive prefix sums of W - m_s                         */
+} cod_split;
+
+/* Optional float32 taps of cod_draft_round for parity tests (device; any member may be NULL). */
+typedef struct {
+  float* z;         /* [S*W, D]            normalised fused features of the window rows (rows not
+                                           projected in baseline mode are left untouched)   */
+  float* attn_out;  /* [Ld][S*W, n_q*hd]   attention output of every layer                  */
+  float* x_final;   /* [S*W, D]            residual stream before the final norm            */
+  float* top_logit; /* [S*W]               the winning logit of every block row             */
+} cod_taps;
+
+/* Creates a context on the CURRENT CUDA device and allocates its workspace.
+   cfg: host pointer. out: host pointer receiving the handle. */
+int cod_create(const cod_config* cfg, cod_ctx** out);
+int cod_destroy(cod_ctx* ctx);
+
+/* Records the weight pointers (they must stay valid while the context is used) and
+   precomputes F(E_carry) = fc . e_carry: F is linear and bias-free, so
+   F(h + E_carry) = F(h) + F(E_carry) (Eq. 2 with Algorithm 1's "add before F"). */
+int cod_set_weights(cod_ctx* ctx, const cod_weights* w, cod_stream_t stream);
+
+/* Part 1 — greedy verification (Section 2 "Preliminaries"; Algorithm 2 "GreedyVerify").
+   draft  [S, W]   device int32: the window's tokens (row 0 = anchor when n_forced = 1).
+   target [S, W+1] device int32: the target's greedy token for each window row, so
+                   target[s, m_s] is the bonus token.
+   m_s = longest prefix with draft == target, the first n_forced (0 or 1) rows always
+   accepted. Reads st->committed_len and st->block_table; modifies no state. */
+int cod_verify_accept(cod_ctx* ctx, const int32_t* draft, const int32_t* target, int S,
+                      int n_forced, const cod_state* st, cod_split* out, cod_stream_t stream);
+
+/* Part 2 — J_l = (K_l(Z), V_l(Z)), Z = F(H + [rejected] E_carry) (Eq. 1-2; Algorithm 1).
+   H [S*W, D_in] device. J [Ld][S*W][2][n_kv][hd] device; keys rotated (RoPE) at row_pos.
+   COD_CARRY writes every row; COD_BASELINE writes accepted rows only and leaves the
+   other rows of J untouched. */
+int cod_project_kv(cod_ctx* ctx, const void* H, const cod_split* split, int S, int mode,
+                   void* J, cod_stream_t stream);
+
+/* Part 3 — C_l <- [C_l; J_l accepted], U_l <- J_l rejected (Algorithm 1, last steps).
+   Copies accepted rows to their page slots and, in COD_CARRY, rejected rows to the carry
+   slot; then committed_len[s] += m_s and carry_len[s] = W - m_s (0 in COD_BASELINE). */
+int cod_scatter_kv(cod_ctx* ctx, const void* J, const cod_split* split, int S, int mode,
+                   cod_state* st, cod_stream_t stream);
+
+/* Part 4 — block attention of one drafter layer over [C_l; U_l; block]
+   (Section 2 "Preliminaries"; Algorithm 1 "the next draft reads ctx_l").
+   q [S, W, n_q, hd], k_blk / v_blk [S, W, n_kv, hd] device, q and k_blk NOT rotated: the
+   call rotates them at positions committed_len[s] + i. No mask; scale 1/sqrt(hd); query
+   head g reads KV head g / (n_q / n_kv). use_carry = 0 ignores U_l.
+   out [S, W, n_q, hd]. carry_mass (nullable) float [S, W, n_q]: share of softmax mass on
+   the carried rows (the diagnostic of Appendix C). */
+int cod_block_attn(cod_ctx* ctx, int layer, const void* q, const void* k_blk, const void* v_blk,
+                   const cod_state* st, int S, int use_carry, void* out, float* carry_mass,
+                   cod_stream_t stream);
+
+/* Part 5 — tied LM head with fused argmax: tok[r] = lowest-index argmax_v Emb[v] . N_f(x[r]).
+   x [n_rows, D] device float32 (the residual stream); tok [n_rows] device int32;
+   top_logit (nullable) [n_rows] device float. Logits are never materialised. */
+int cod_lm_head_argmax(cod_ctx* ctx, const float* x, int n_rows, int32_t* tok, float* top_logit,
+                       cod_stream_t stream);
+
+/* The whole round: parts 1-3 on (draft, target, H), then one parallel block prediction from
+   [bonus, MASK, ...] through every drafter layer, then part 5.
+   next_draft [S, W] device int32 = [bonus_s, tok_1, ..., tok_{W-1}].
+   Leaves st exactly as cod_verify_accept + cod_project_kv + cod_scatter_kv would.
+   taps: host pointer to a struct of device pointers, or NULL. */
+int cod_draft_round(cod_ctx* ctx, const int32_t* draft, const int32_t* target, const void* H,
+                    int S, int n_forced, int mode, cod_state* st, cod_split* split_out,
+                    int32_t* next_draft, const cod_taps* taps, cod_stream_t stream);
+
+/* Copies the sticky device status word to *dev_flags (host) after synchronising the stream;
+   clear != 0 also resets it. */
+int cod_poll_status(cod_ctx* ctx, uint32_t* dev_flags, int clear, cod_stream_t stream);
+
+/* Number of kernels this context has launched since creation (host-side counter). */
+int64_t cod_launch_count(const cod_ctx* ctx);
+
+/* Bytes of device workspace the context holds. */
+int64_t cod_workspace_bytes(const cod_ctx* ctx);
+
+const char* cod_error_string(int status);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* COD_H_ */

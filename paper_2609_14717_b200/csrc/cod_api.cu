@@ -1,0 +1,340 @@
+// The C ABI: argument validation, workspace, and the order of kernels in one round.
+#include <math.h>
+#include <stdlib.h>
+#include <string.h>
+
+#include <new>
+
+#include "cod_internal.cuh"
+
+namespace {
+
+inline size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
+inline size_t esize(const cod_ctx* c) { return c->cfg.dtype == COD_BF16 ? 2 : 4; }
+inline bool misaligned(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) != 0; }
+
+struct Carver {
+  char* base;
+  size_t off;
+  template <typename P>
+  void take(P*& ptr, size_t bytes) {
+    off = align_up(off, 256);
+    if (base) ptr = reinterpret_cast<P*>(base + off);
+    off += bytes;
+  }
+};
+
+// Lays out the workspace; with c->ws == nullptr it only measures.
+size_t carve(cod_ctx* c) {
+  const cod_config& f = c->cfg;
+  const size_t R = c->R_max, es = esize(c), D = c->D;
+  Carver cv{c->ws, 0};
+  cv.take(c->status, 256);
+  cv.take(c->inv_freq_d, sizeof(double) * c->half);
+  cv.take(c->inv_freq, sizeof(float) * c->half);
+  cv.take(c->fcE, sizeof(float) * D);
+  cv.take(c->rope_win, sizeof(float) * R * f.head_dim);
+  cv.take(c->rope_blk, sizeof(float) * R * f.head_dim);
+  size_t widest = D;
+  widest = widest > static_cast<size_t>(2 * f.n_layers * c->kvw) ? widest : static_cast<size_t>(2 * f.n_layers * c->kvw);
+  widest = widest > static_cast<size_t>(c->qw + 2 * c->kvw) ? widest : static_cast<size_t>(c->qw + 2 * c->kvw);
+  c->gemm_out_floats = static_cast<size_t>(COD_MAX_SPLITS) * R * widest;
+  cv.take(c->gemm_out, sizeof(float) * c->gemm_out_floats);
+  cv.take(c->z, es * R * D);
+  cv.take(c->x, sizeof(float) * R * D);
+  cv.take(c->a, es * R * D);
+  cv.take(c->q, es * R * c->qw);
+  cv.take(c->kb, es * R * c->kvw);
+  cv.take(c->vb, es * R * c->kvw);
+  cv.take(c->o, es * R * c->qw);
+  const size_t M = static_cast<size_t>(f.block) * (f.n_q_heads / f.n_kv_heads);
+  const size_t parts = static_cast<size_t>(f.max_batch) * f.n_kv_heads * c->max_splits * M;
+  cv.take(c->attn_o, sizeof(float) * parts * f.head_dim);
+  cv.take(c->attn_ml, sizeof(float) * parts * 4);
+  cv.take(c->amax, sizeof(unsigned long long) * R);
+  cv.take(c->tok, sizeof(int32_t) * R);
+  cv.take(c->sp.accept_len, sizeof(int32_t) * f.max_batch);
+  cv.take(c->sp.bonus, sizeof(int32_t) * f.max_batch);
+  cv.take(c->sp.row_pos, sizeof(int32_t) * R);
+  cv.take(c->sp.commit_slot, sizeof(int32_t) * R);
+  cv.take(c->sp.carry_slot, sizeof(int32_t) * R);
+  cv.take(c->sp.acc_rows, sizeof(int32_t) * R);
+  cv.take(c->sp.acc_off, sizeof(int32_t) * (f.max_batch + 1));
+  cv.take(c->sp.rej_rows, sizeof(int32_t) * R);
+  cv.take(c->sp.rej_off, sizeof(int32_t) * (f.max_batch + 1));
+  return align_up(cv.off, 256);
+}
+
+bool split_has_null(const cod_split* s) {
+  return !s || !s->accept_len || !s->bonus || !s->row_pos || !s->commit_slot || !s->carry_slot || !s->acc_rows ||
+         !s->acc_off || !s->rej_rows || !s->rej_off;
+}
+bool state_has_null(const cod_state* s) {
+  return !s || !s->kv_pool || !s->block_table || !s->committed_len || !s->carry_kv || !s->carry_len;
+}
+
+// split-K factor so that (feature tiles x splits) fills the machine; partial slabs must fit
+int pick_splits(const cod_ctx* c, int n_out, int K, int rows) {
+  (void)c; (void)n_out; (void)K; (void)rows;
+  return 1;
+}
+
+int check_S(const cod_ctx* c, int S) { return (S >= 1 && S <= c->cfg.max_batch) ? COD_OK : COD_ERR_INVALID_ARG; }
+
+}  // namespace
+
+int cod_launch_gemm(cod_ctx* c, const GemmArgs& g, cudaStream_t st) { return cod_launch_gemm_simt(c, g, st); }
+
+int cod_launch_attn(cod_ctx* c, int layer, const void* q, const void* kb, const void* vb, const cod_state* state,
+                    int S, int use_carry, void* out, float* tap_out, float* carry_mass, cudaStream_t st) {
+  return cod_launch_attn_simt(c, layer, q, kb, vb, state, S, use_carry, out, tap_out, carry_mass, st);
+}
+
+extern "C" {
+
+int cod_create(const cod_config* cfg, cod_ctx** out) {
+  if (!cfg || !out) return COD_ERR_INVALID_ARG;
+  *out = nullptr;
+  const cod_config& f = *cfg;
+  if (f.d_target < 1 || f.n_cap < 1 || f.d_model < 1 || f.n_layers < 1 || f.n_q_heads < 1 || f.n_kv_heads < 1 ||
+      f.head_dim < 1 || f.vocab < 2 || f.block < 1 || f.page_size < 1 || f.max_batch < 1 ||
+      f.max_pages_per_seq < 1 || f.n_pages < 1)
+    return COD_ERR_INVALID_ARG;
+  if (f.dtype != COD_F32 && f.dtype != COD_BF16) return COD_ERR_INVALID_ARG;
+  if (f.mask_token_id < 0 || f.mask_token_id >= f.vocab) return COD_ERR_INVALID_ARG;
+  if (f.n_q_heads % f.n_kv_heads) return COD_ERR_INVALID_ARG;
+  if (f.d_model != f.n_q_heads * f.head_dim) return COD_ERR_INVALID_ARG;
+  if (f.attn_split_len < 0 || f.attn_split_len % 32) return COD_ERR_INVALID_ARG;
+  if (!(f.rope_theta > 0.f) || !(f.rms_eps >= 0.f)) return COD_ERR_INVALID_ARG;
+  if (f.head_dim != 64 && f.head_dim != 128) return COD_ERR_UNSUPPORTED;
+  if (f.block > COD_MAX_W || f.block * (f.n_q_heads / f.n_kv_heads) > 128) return COD_ERR_UNSUPPORTED;
+  if ((f.d_target * f.n_cap) % 8 || f.d_model % 8) return COD_ERR_UNSUPPORTED;
+  if ((f.n_kv_heads * f.head_dim) % 64) return COD_ERR_UNSUPPORTED;
+  if (static_cast<int64_t>(f.n_pages) * f.page_size > (1ll << 31) - 1) return COD_ERR_UNSUPPORTED;
+
+  cod_ctx* c = new (std::nothrow) cod_ctx();
+  if (!c) return COD_ERR_ALLOC;
+  memset(c, 0, sizeof(*c));
+  c->cfg = f;
+  if (cudaGetDevice(&c->device) != cudaSuccess) { delete c; return COD_ERR_CUDA; }
+  c->D = f.d_model;
+  c->D_in = f.d_target * f.n_cap;
+  c->kvw = f.n_kv_heads * f.head_dim;
+  c->qw = f.n_q_heads * f.head_dim;
+  c->R_max = f.max_batch * f.block;
+  c->half = f.head_dim / 2;
+  c->split_len = f.attn_split_len > 0 ? f.attn_split_len : 512;
+  const int64_t max_keys = static_cast<int64_t>(f.max_pages_per_seq) * f.page_size + 2 * f.block;
+  c->max_splits = static_cast<int>((max_keys + c->split_len - 1) / c->split_len);
+
+  c->ws = nullptr;
+  c->ws_bytes = carve(c);
+  if (cudaMalloc(&c->ws, c->ws_bytes) != cudaSuccess) { cudaGetLastError(); delete c; return COD_ERR_ALLOC; }
+  carve(c);
+  bool ok = cudaMemset(c->ws, 0, c->ws_bytes) == cudaSuccess;
+  double* fr = static_cast<double*>(malloc(sizeof(double) * c->half));
+  float* frf = static_cast<float*>(malloc(sizeof(float) * c->half));
+  if (!fr || !frf) ok = false;
+  if (ok) {
+    for (int j = 0; j < c->half; ++j) {
+      fr[j] = pow(static_cast<double>(f.rope_theta), -2.0 * j / f.head_dim);
+      frf[j] = static_cast<float>(fr[j]);
+    }
+    ok = cudaMemcpy(c->inv_freq_d, fr, sizeof(double) * c->half, cudaMemcpyHostToDevice) == cudaSuccess &&
+         cudaMemcpy(c->inv_freq, frf, sizeof(float) * c->half, cudaMemcpyHostToDevice) == cudaSuccess;
+  }
+  free(fr);
+  free(frf);
+  if (!ok) { cudaFree(c->ws); cudaGetLastError(); delete c; return COD_ERR_CUDA; }
+  *out = c;
+  return COD_OK;
+}
+
+int cod_destroy(cod_ctx* c) {
+  if (!c) return COD_ERR_INVALID_ARG;
+  cudaDeviceSynchronize();
+  cudaFree(c->ws);
+  delete c;
+  return COD_OK;
+}
+
+int cod_set_weights(cod_ctx* c, const cod_weights* w, cod_stream_t stream) {
+  if (!c || !w) return COD_ERR_INVALID_ARG;
+  const void* ps[] = {w->fc, w->e_carry, w->g_hidden, w->wk, w->wv, w->wq, w->wo, w->g_attn, w->g_final, w->emb};
+  for (const void* p : ps)
+    if (!p || misaligned(p)) return COD_ERR_INVALID_ARG;
+  c->w = *w;
+  c->has_weights = true;
+  return cod_launch_fcE(c, static_cast<cudaStream_t>(stream));
+}
+
+int cod_verify_accept(cod_ctx* c, const int32_t* draft, const int32_t* target, int S, int n_forced,
+                      const cod_state* st, cod_split* out, cod_stream_t stream) {
+  if (!c || !draft || !target || !st || !st->committed_len || !st->block_table || split_has_null(out))
+    return COD_ERR_INVALID_ARG;
+  if (check_S(c, S) != COD_OK || n_forced < 0 || n_forced > 1) return COD_ERR_INVALID_ARG;
+  return cod_launch_verify(c, draft, target, S, n_forced, st, out, static_cast<cudaStream_t>(stream));
+}
+
+// fc and K/V contractions of the kept rows; the finish kernel writes J or the state.
+static int project_impl(cod_ctx* c, const void* H, const cod_split* sp, int S, int mode, void* J,
+                        const cod_state* dest, float* tap_z, cudaStream_t st) {
+  const cod_config& f = c->cfg;
+  const int R = S * f.block;
+  const int* a_rows = mode == COD_BASELINE ? sp->acc_rows : nullptr;
+  const int* n_dev = mode == COD_BASELINE ? sp->acc_off + S : nullptr;
+  int rc;
+
+  GemmArgs g{};
+  g.A = H; g.lda = c->D_in; g.a_rows = a_rows; g.n_rows_dev = n_dev; g.n_rows = R; g.K = c->D_in;
+  g.seg[0] = {c->w.fc, c->D}; g.n_seg = 1;
+  g.C = c->gemm_out; g.ldc = c->D; g.splits = pick_splits(c, c->D, c->D_in, R);
+  if ((rc = cod_launch_gemm(c, g, st)) != COD_OK) return rc;
+  if ((rc = cod_launch_fc_finish(c, c->gemm_out, g.splits, R, n_dev, a_rows, sp->carry_slot, tap_z, st)) != COD_OK)
+    return rc;
+
+  GemmArgs k{};
+  k.A = c->z; k.lda = c->D; k.a_rows = a_rows; k.n_rows_dev = n_dev; k.n_rows = R; k.K = c->D;
+  k.seg[0] = {c->w.wk, f.n_layers * c->kvw};
+  k.seg[1] = {c->w.wv, f.n_layers * c->kvw};
+  k.n_seg = 2;
+  k.C = c->gemm_out; k.ldc = 2 * f.n_layers * c->kvw; k.splits = 1;
+  if ((rc = cod_launch_gemm(c, k, st)) != COD_OK) return rc;
+  return cod_launch_kv_finish(c, c->gemm_out, 1, R, n_dev, a_rows, sp, J, dest, R, st);
+}
+
+int cod_project_kv(cod_ctx* c, const void* H, const cod_split* split, int S, int mode, void* J,
+                   cod_stream_t stream) {
+  if (!c || !H || !J || split_has_null(split) || misaligned(H) || misaligned(J)) return COD_ERR_INVALID_ARG;
+  if (check_S(c, S) != COD_OK || (mode != COD_CARRY && mode != COD_BASELINE)) return COD_ERR_INVALID_ARG;
+  if (!c->has_weights) return COD_ERR_NO_WEIGHTS;
+  return project_impl(c, H, split, S, mode, J, nullptr, nullptr, static_cast<cudaStream_t>(stream));
+}
+
+int cod_scatter_kv(cod_ctx* c, const void* J, const cod_split* split, int S, int mode, cod_state* st,
+                   cod_stream_t stream) {
+  if (!c || !J || split_has_null(split) || state_has_null(st) || misaligned(J) || misaligned(st->kv_pool) ||
+      misaligned(st->carry_kv))
+    return COD_ERR_INVALID_ARG;
+  if (check_S(c, S) != COD_OK || (mode != COD_CARRY && mode != COD_BASELINE)) return COD_ERR_INVALID_ARG;
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  int rc = cod_launch_scatter(c, J, split, S, mode, st, s);
+  if (rc != COD_OK) return rc;
+  return cod_launch_update_lens(c, split, S, mode, st, s);
+}
+
+int cod_block_attn(cod_ctx* c, int layer, const void* q, const void* k_blk, const void* v_blk,
+                   const cod_state* st, int S, int use_carry, void* out, float* carry_mass,
+                   cod_stream_t stream) {
+  if (!c || !q || !k_blk || !v_blk || !out || state_has_null(st)) return COD_ERR_INVALID_ARG;
+  if (misaligned(q) || misaligned(k_blk) || misaligned(v_blk) || misaligned(out) || misaligned(st->kv_pool) ||
+      misaligned(st->carry_kv))
+    return COD_ERR_INVALID_ARG;
+  if (check_S(c, S) != COD_OK || layer < 0 || layer >= c->cfg.n_layers) return COD_ERR_INVALID_ARG;
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  int rc = cod_launch_rope_blk_only(c, st->committed_len, S, s);
+  if (rc != COD_OK) return rc;
+  if ((rc = cod_launch_rope_qk(c, q, k_blk, st->committed_len, S, s)) != COD_OK) return rc;
+  return cod_launch_attn(c, layer, c->q, c->kb, v_blk, st, S, use_carry ? 1 : 0, out, nullptr, carry_mass, s);
+}
+
+static int lm_head_impl(cod_ctx* c, int n_rows, cudaStream_t st) {
+  GemmArgs g{};
+  g.A = c->a; g.lda = c->D; g.n_rows = n_rows; g.K = c->D;
+  g.seg[0] = {c->w.emb, c->cfg.vocab}; g.n_seg = 1;
+  g.splits = 1; g.amax = c->amax;
+  return cod_launch_gemm(c, g, st);
+}
+
+int cod_lm_head_argmax(cod_ctx* c, const float* x, int n_rows, int32_t* tok, float* top_logit,
+                       cod_stream_t stream) {
+  if (!c || !x || !tok || misaligned(x)) return COD_ERR_INVALID_ARG;
+  if (n_rows < 1 || n_rows > c->R_max) return COD_ERR_INVALID_ARG;
+  if (!c->has_weights) return COD_ERR_NO_WEIGHTS;
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  int rc = cod_launch_resid_norm(c, nullptr, 0, n_rows, const_cast<float*>(x), c->w.g_final, nullptr, s);
+  if (rc != COD_OK) return rc;
+  if ((rc = lm_head_impl(c, n_rows, s)) != COD_OK) return rc;
+  return cod_launch_finalize(c, n_rows, 1, nullptr, tok, nullptr, top_logit, s);
+}
+
+int cod_draft_round(cod_ctx* c, const int32_t* draft, const int32_t* target, const void* H, int S,
+                    int n_forced, int mode, cod_state* st, cod_split* split_out, int32_t* next_draft,
+                    const cod_taps* taps, cod_stream_t stream) {
+  if (!c || !draft || !target || !H || !next_draft || state_has_null(st)) return COD_ERR_INVALID_ARG;
+  if (misaligned(H) || misaligned(st->kv_pool) || misaligned(st->carry_kv)) return COD_ERR_INVALID_ARG;
+  if (split_out && split_has_null(split_out)) return COD_ERR_INVALID_ARG;
+  if (check_S(c, S) != COD_OK || n_forced < 0 || n_forced > 1) return COD_ERR_INVALID_ARG;
+  if (mode != COD_CARRY && mode != COD_BASELINE) return COD_ERR_INVALID_ARG;
+  if (!c->has_weights) return COD_ERR_NO_WEIGHTS;
+  const cod_config& f = c->cfg;
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  const cod_split* sp = split_out ? split_out : &c->sp;
+  const int R = S * f.block;
+  const size_t es = esize(c);
+  int rc;
+
+  // parts 1-3
+  if ((rc = cod_launch_verify(c, draft, target, S, n_forced, st, sp, s)) != COD_OK) return rc;
+  if ((rc = project_impl(c, H, sp, S, mode, nullptr, st, taps ? taps->z : nullptr, s)) != COD_OK) return rc;
+  if ((rc = cod_launch_update_lens(c, sp, S, mode, st, s)) != COD_OK) return rc;
+
+  // the next block: [bonus, MASK, ...] through every drafter layer
+  if ((rc = cod_launch_embed_norm(c, sp->bonus, S, s)) != COD_OK) return rc;
+  for (int l = 0; l < f.n_layers; ++l) {
+    GemmArgs g{};
+    g.A = c->a; g.lda = c->D; g.n_rows = R; g.K = c->D;
+    g.seg[0] = {static_cast<const char*>(c->w.wq) + es * l * c->qw * c->D, c->qw};
+    g.seg[1] = {static_cast<const char*>(c->w.wk) + es * l * c->kvw * c->D, c->kvw};
+    g.seg[2] = {static_cast<const char*>(c->w.wv) + es * l * c->kvw * c->D, c->kvw};
+    g.n_seg = 3;
+    g.C = c->gemm_out; g.ldc = c->qw + 2 * c->kvw; g.splits = pick_splits(c, g.ldc, c->D, R);
+    if ((rc = cod_launch_gemm(c, g, s)) != COD_OK) return rc;
+    if ((rc = cod_launch_qkv_finish(c, c->gemm_out, g.splits, R, s)) != COD_OK) return rc;
+
+    float* tap_o = (taps && taps->attn_out) ? taps->attn_out + static_cast<size_t>(l) * R * c->qw : nullptr;
+    if ((rc = cod_launch_attn(c, l, c->q, c->kb, c->vb, st, S, mode == COD_CARRY ? 1 : 0, c->o, tap_o, nullptr, s)) != COD_OK)
+      return rc;
+
+    GemmArgs o{};
+    o.A = c->o; o.lda = c->qw; o.n_rows = R; o.K = c->qw;
+    o.seg[0] = {static_cast<const char*>(c->w.wo) + es * l * c->D * c->qw, c->D};
+    o.n_seg = 1;
+    o.C = c->gemm_out; o.ldc = c->D; o.splits = pick_splits(c, c->D, c->qw, R);
+    if ((rc = cod_launch_gemm(c, o, s)) != COD_OK) return rc;
+    const bool last = l + 1 == f.n_layers;
+    const void* gain = last ? c->w.g_final : static_cast<const char*>(c->w.g_attn) + es * (l + 1) * c->D;
+    if ((rc = cod_launch_resid_norm(c, c->gemm_out, o.splits, R, c->x, gain,
+                                    (last && taps) ? taps->x_final : nullptr, s)) != COD_OK)
+      return rc;
+  }
+  // part 5
+  if ((rc = lm_head_impl(c, R, s)) != COD_OK) return rc;
+  return cod_launch_finalize(c, R, f.block, sp->bonus, c->tok, next_draft, taps ? taps->top_logit : nullptr, s);
+}
+
+int cod_poll_status(cod_ctx* c, uint32_t* dev_flags, int clear, cod_stream_t stream) {
+  if (!c || !dev_flags) return COD_ERR_INVALID_ARG;
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  if (cudaMemcpyAsync(dev_flags, c->status, sizeof(uint32_t), cudaMemcpyDeviceToHost, s) != cudaSuccess) return COD_ERR_CUDA;
+  if (clear && cudaMemsetAsync(c->status, 0, sizeof(uint32_t), s) != cudaSuccess) return COD_ERR_CUDA;
+  if (cudaStreamSynchronize(s) != cudaSuccess) return COD_ERR_CUDA;
+  return COD_OK;
+}
+
+int64_t cod_launch_count(const cod_ctx* c) { return c ? c->launches : 0; }
+int64_t cod_workspace_bytes(const cod_ctx* c) { return c ? static_cast<int64_t>(c->ws_bytes) : 0; }
+
+const char* cod_error_string(int status) {
+  switch (status) {
+    case COD_OK: return "ok";
+    case COD_ERR_INVALID_ARG: return "invalid argument";
+    case COD_ERR_UNSUPPORTED: return "unsupported shape or flag";
+    case COD_ERR_CUDA: return "CUDA runtime error";
+    case COD_ERR_NO_WEIGHTS: return "weights not set";
+    case COD_ERR_ALLOC: return "workspace allocation failed";
+    default: return "unknown status";
+  }
+}
+
+}  // extern "C"

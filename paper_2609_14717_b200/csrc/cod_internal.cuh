@@ -1,0 +1,164 @@
+// Internal declarations shared by the library's translation units (not part of the C ABI).
+#pragma once
+
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "cod.h"
+
+#define COD_MAX_SPLITS 8          // split-K partial slabs the GEMM workspace can hold
+#define COD_MAX_W 128             // largest supported block size
+
+// ---------------------------------------------------------------------------- element access
+__device__ __forceinline__ float cod_ld(const float* p) { return *p; }
+__device__ __forceinline__ float cod_ld(const __nv_bfloat16* p) { return __bfloat162float(*p); }
+__device__ __forceinline__ void cod_st(float* p, float v) { *p = v; }
+__device__ __forceinline__ void cod_st(__nv_bfloat16* p, float v) { *p = __float2bfloat16_rn(v); }
+
+// four consecutive elements (pointer aligned to 4 elements)
+__device__ __forceinline__ float4 cod_ld4(const float* p) { return *reinterpret_cast<const float4*>(p); }
+__device__ __forceinline__ float4 cod_ld4(const __nv_bfloat16* p) {
+  uint2 u = *reinterpret_cast<const uint2*>(p);
+  __nv_bfloat162 a = *reinterpret_cast<__nv_bfloat162*>(&u.x);
+  __nv_bfloat162 b = *reinterpret_cast<__nv_bfloat162*>(&u.y);
+  float2 fa = __bfloat1622float2(a), fb = __bfloat1622float2(b);
+  return make_float4(fa.x, fa.y, fb.x, fb.y);
+}
+
+__device__ __forceinline__ float cod_warp_sum(float v) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+  return v;
+}
+__device__ __forceinline__ float cod_warp_max(float v) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v = fmaxf(v, __shfl_xor_sync(0xffffffffu, v, o));
+  return v;
+}
+
+// Sum over a thread block (blockDim.x a multiple of 32, at most 1024); result in every thread.
+__device__ __forceinline__ float cod_block_sum(float v, float* red /* >= 33 floats of shared */) {
+  v = cod_warp_sum(v);
+  const int lane = threadIdx.x & 31, wid = threadIdx.x >> 5, nw = (blockDim.x + 31) >> 5;
+  __syncthreads();
+  if (lane == 0) red[wid] = v;
+  __syncthreads();
+  if (wid == 0) {
+    float t = lane < nw ? red[lane] : 0.f;
+    t = cod_warp_sum(t);
+    if (lane == 0) red[32] = t;
+  }
+  __syncthreads();
+  return red[32];
+}
+
+// Packed (logit, index) key whose unsigned order is: larger logit first, then lower index.
+__device__ __forceinline__ unsigned long long cod_pack_argmax(float v, int idx) {
+  unsigned u = __float_as_uint(v);
+  u = (u & 0x80000000u) ? ~u : (u | 0x80000000u);
+  return (static_cast<unsigned long long>(u) << 32) | static_cast<unsigned long long>(0xFFFFFFFFu - static_cast<unsigned>(idx));
+}
+__device__ __forceinline__ float cod_unpack_logit(unsigned long long key) {
+  unsigned u = static_cast<unsigned>(key >> 32);
+  u = (u & 0x80000000u) ? (u & 0x7FFFFFFFu) : ~u;
+  return __uint_as_float(u);
+}
+__device__ __forceinline__ int cod_unpack_index(unsigned long long key) {
+  return static_cast<int>(0xFFFFFFFFu - static_cast<unsigned>(key & 0xFFFFFFFFull));
+}
+
+// ---------------------------------------------------------------------------- GEMM arguments
+// C[i, n] = sum_k A[row(i), k] * B[n, k]   (A: activations, B: weights, both K contiguous)
+struct GemmSeg {
+  const void* B;  // [N, K]
+  int N;
+};
+struct GemmArgs {
+  const void* A;          // [*, K] with row stride lda
+  int lda;
+  const int* a_rows;      // optional gather list: row(i) = a_rows[i]; else row(i) = i
+  const int* n_rows_dev;  // optional device count of valid rows (<= n_rows)
+  int n_rows;             // rows (or their upper bound when n_rows_dev is set)
+  int K;
+  GemmSeg seg[3];         // weight segments laid side by side along N
+  int n_seg;
+  float* C;               // [splits][n_rows][ldc] float partial sums
+  int ldc;
+  int splits;             // split-K factor (1 = none)
+  unsigned long long* amax;  // if non-null: per-row packed argmax over N instead of storing C
+};
+
+struct cod_ctx {
+  cod_config cfg;
+  cod_weights w;
+  bool has_weights;
+  int device;
+  int D, D_in, kvw, qw, R_max, half;
+  int split_len, max_splits;   // attention split-KV
+  int64_t launches;
+  size_t ws_bytes;
+  char* ws;
+  // carved out of ws
+  uint32_t* status;
+  float* inv_freq;             // [hd/2]  theta^(-2j/hd), rounded from double
+  double* inv_freq_d;          // [hd/2]
+  float* fcE;                  // [D]     F(E_carry)
+  float* rope_win;             // [R_max][hd]  cos | sin of the window rows' positions
+  float* rope_blk;             // [R_max][hd]  cos | sin of the block rows' positions
+  float* gemm_out;             // split-K / unfused GEMM results
+  size_t gemm_out_floats;
+  void* z;                     // [R_max, D]
+  float* x;                    // [R_max, D]   residual stream
+  void* a;                     // [R_max, D]   normalised activations
+  void* q;                     // [R_max, qw]
+  void* kb;                    // [R_max, kvw]
+  void* vb;                    // [R_max, kvw]
+  void* o;                     // [R_max, qw]
+  float* attn_o;               // [S][n_kv][splits][M][hd]
+  float* attn_ml;              // [S][n_kv][splits][M][4]  (m, l, l_carry, -)
+  unsigned long long* amax;    // [R_max]
+  int32_t* tok;                // [R_max]
+  cod_split sp;                // internal split arrays (used when the caller passes none)
+};
+
+// ---------------------------------------------------------------------------- launchers
+// Every launcher enqueues on `st`, bumps ctx->launches, and returns a cod_status.
+int cod_launch_verify(cod_ctx* c, const int32_t* draft, const int32_t* target, int S, int n_forced,
+                      const cod_state* state, const cod_split* out, cudaStream_t st);
+int cod_launch_gemm(cod_ctx* c, const GemmArgs& g, cudaStream_t st);
+int cod_launch_gemm_simt(cod_ctx* c, const GemmArgs& g, cudaStream_t st);
+int cod_launch_attn_simt(cod_ctx* c, int layer, const void* q, const void* kb, const void* vb,
+                         const cod_state* stt, int S, int use_carry, void* out, float* tap, float* mass,
+                         cudaStream_t st);
+// cos/sin tables of the block rows only, at positions committed_len[s] + i
+int cod_launch_rope_blk_only(cod_ctx* c, const int32_t* committed_len, int S, cudaStream_t st);
+int cod_launch_fcE(cod_ctx* c, cudaStream_t st);
+int cod_launch_fc_finish(cod_ctx* c, const float* part, int splits, int n_rows, const int* n_rows_dev,
+                         const int* a_rows, const int* carry_slot, float* tap_z, cudaStream_t st);
+// dest_state == nullptr: write J; else write the pool / carry slot directly
+int cod_launch_kv_finish(cod_ctx* c, const float* part, int splits, int n_rows, const int* n_rows_dev,
+                         const int* a_rows, const cod_split* sp, void* J, const cod_state* dest_state,
+                         int R_total, cudaStream_t st);
+int cod_launch_scatter(cod_ctx* c, const void* J, const cod_split* sp, int S, int mode,
+                       const cod_state* state, cudaStream_t st);
+int cod_launch_update_lens(cod_ctx* c, const cod_split* sp, int S, int mode, const cod_state* state,
+                           cudaStream_t st);
+int cod_launch_embed_norm(cod_ctx* c, const int32_t* bonus, int S, cudaStream_t st);
+int cod_launch_qkv_finish(cod_ctx* c, const float* part, int splits, int R, cudaStream_t st);
+int cod_launch_rope_qk(cod_ctx* c, const void* q, const void* k, const int32_t* committed_len, int S,
+                       cudaStream_t st);  // standalone attention entry: rotate into c->q / c->kb
+int cod_launch_attn(cod_ctx* c, int layer, const void* q, const void* kb, const void* vb,
+                    const cod_state* state, int S, int use_carry, void* out, float* tap_out,
+                    float* carry_mass, cudaStream_t st);
+// x += sum of partials (if part != nullptr); a = N(x) * gain; optional copy of x to tap_x
+int cod_launch_resid_norm(cod_ctx* c, const float* part, int splits, int R, float* x, const void* gain,
+                          float* tap_x, cudaStream_t st);
+int cod_launch_finalize(cod_ctx* c, int R, int W, const int32_t* bonus, int32_t* tok, int32_t* next_draft,
+                        float* top_logit, cudaStream_t st);
+
+#define COD_CHECK_LAUNCH(c)                                   \
+  do {                                                        \
+    (c)->launches++;                                          \
+    if (cudaPeekAtLastError() != cudaSuccess) return COD_ERR_CUDA; \
+  } while (0)

@@ -1,0 +1,131 @@
+// Plain FP32-FMA GEMM: C[i, n] = sum_k A[row(i), k] * B[n, k].
+// This is the float32 path (TF32 would be too coarse for the 1e-3 parity bound of the
+// float configuration) and the general-shape path for bf16 shapes the tensor-core kernels
+// do not cover. Both operands are K-contiguous; accumulation is float.
+#include "cod_internal.cuh"
+
+namespace {
+
+constexpr int BM = 32;   // activation rows per tile
+constexpr int BN = 64;   // weight rows (output features) per tile
+constexpr int BK = 32;
+constexpr int NT = 256;  // threads: 16 (features, 4 each) x 16 (rows, 2 each)
+
+template <typename T, bool ARGMAX>
+__global__ void __launch_bounds__(NT) k_gemm_simt(GemmArgs g) {
+  __shared__ float As[BK][BM + 1];
+  __shared__ float Bs[BK][BN + 1];
+
+  const int n_rows = g.n_rows_dev ? min(*g.n_rows_dev, g.n_rows) : g.n_rows;
+  const int i0 = blockIdx.y * BM;
+  if (i0 >= n_rows) return;
+
+  // which weight segment does this feature tile fall in
+  int n0 = blockIdx.x * BN, col0 = n0, sidx = 0;
+  while (sidx < g.n_seg - 1 && n0 >= g.seg[sidx].N) { n0 -= g.seg[sidx].N; ++sidx; }
+  const T* __restrict__ B = static_cast<const T*>(g.seg[sidx].B);
+  const int N = g.seg[sidx].N;
+  const T* __restrict__ A = static_cast<const T*>(g.A);
+
+  // K range of this split (multiples of BK)
+  const int kblocks = (g.K + BK - 1) / BK;
+  const int per = (kblocks + g.splits - 1) / g.splits;
+  const int kb0 = blockIdx.z * per, kb1 = min(kblocks, kb0 + per);
+
+  const int t = threadIdx.x;
+  const int tx = t & 15, ty = t >> 4;
+
+  // loader mapping: each thread moves groups of 4 consecutive k
+  const int la_r = t >> 3, la_k = (t & 7) * 4;        // A: 32 rows x 8 groups
+  int a_row = -1;
+  if (i0 + la_r < n_rows) a_row = g.a_rows ? g.a_rows[i0 + la_r] : i0 + la_r;
+
+  float acc[2][4] = {};
+  for (int kb = kb0; kb < kb1; ++kb) {
+    const int k0 = kb * BK;
+    {
+      float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
+      if (a_row >= 0 && k0 + la_k < g.K) v = cod_ld4(A + static_cast<size_t>(a_row) * g.lda + k0 + la_k);
+      As[la_k + 0][la_r] = v.x; As[la_k + 1][la_r] = v.y; As[la_k + 2][la_r] = v.z; As[la_k + 3][la_r] = v.w;
+    }
+#pragma unroll
+    for (int it = 0; it < 2; ++it) {
+      const int idx = t + it * NT;                    // B: 64 rows x 8 groups
+      const int r = idx >> 3, kk = (idx & 7) * 4;
+      float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
+      if (n0 + r < N && k0 + kk < g.K) v = cod_ld4(B + static_cast<size_t>(n0 + r) * g.K + k0 + kk);
+      Bs[kk + 0][r] = v.x; Bs[kk + 1][r] = v.y; Bs[kk + 2][r] = v.z; Bs[kk + 3][r] = v.w;
+    }
+    __syncthreads();
+#pragma unroll
+    for (int k = 0; k < BK; ++k) {
+      float a[2], b[4];
+#pragma unroll
+      for (int i = 0; i < 2; ++i) a[i] = As[k][ty * 2 + i];
+#pragma unroll
+      for (int j = 0; j < 4; ++j) b[j] = Bs[k][tx + 16 * j];
+#pragma unroll
+      for (int i = 0; i < 2; ++i)
+#pragma unroll
+        for (int j = 0; j < 4; ++j) acc[i][j] = fmaf(a[i], b[j], acc[i][j]);
+    }
+    __syncthreads();
+  }
+
+  if (!ARGMAX) {
+    float* C = g.C + static_cast<size_t>(blockIdx.z) * g.n_rows * g.ldc;
+#pragma unroll
+    for (int i = 0; i < 2; ++i) {
+      const int row = i0 + ty * 2 + i;
+      if (row >= n_rows) continue;
+#pragma unroll
+      for (int j = 0; j < 4; ++j) {
+        const int n = tx + 16 * j;
+        if (n0 + n < N) C[static_cast<size_t>(row) * g.ldc + col0 + n] = acc[i][j];
+      }
+    }
+  } else {
+    // per-row (max, lowest index) over this tile's features, then one atomic per row
+#pragma unroll
+    for (int i = 0; i < 2; ++i) {
+      unsigned long long best = 0ull;
+#pragma unroll
+      for (int j = 0; j < 4; ++j) {
+        const int n = tx + 16 * j;
+        if (n0 + n < N) {
+          const unsigned long long key = cod_pack_argmax(acc[i][j], col0 + n);
+          best = key > best ? key : best;
+        }
+      }
+#pragma unroll
+      for (int o = 8; o > 0; o >>= 1) {
+        const unsigned long long other = __shfl_xor_sync(0xffffffffu, best, o);
+        best = other > best ? other : best;
+      }
+      const int row = i0 + ty * 2 + i;
+      if (tx == 0 && row < n_rows) atomicMax(g.amax + row, best);
+    }
+  }
+}
+
+template <typename T>
+int launch_t(cod_ctx* c, const GemmArgs& g, cudaStream_t st) {
+  int n_total = 0;
+  for (int i = 0; i < g.n_seg; ++i) n_total += g.seg[i].N;
+  dim3 grid((n_total + BN - 1) / BN, (g.n_rows + BM - 1) / BM, g.splits);
+  if (g.amax) k_gemm_simt<T, true><<<grid, NT, 0, st>>>(g);
+  else k_gemm_simt<T, false><<<grid, NT, 0, st>>>(g);
+  COD_CHECK_LAUNCH(c);
+  return COD_OK;
+}
+
+}  // namespace
+
+int cod_launch_gemm_simt(cod_ctx* c, const GemmArgs& g, cudaStream_t st) {
+  if (g.n_rows <= 0) return COD_OK;
+  // segments other than the last must be whole tiles so no tile straddles two matrices
+  for (int i = 0; i + 1 < g.n_seg; ++i)
+    if (g.seg[i].N % BN) return COD_ERR_UNSUPPORTED;
+  if (g.K % 4 || g.lda % 4) return COD_ERR_UNSUPPORTED;
+  return c->cfg.dtype == COD_BF16 ? launch_t<__nv_bfloat16>(c, g, st) : launch_t<float>(c, g, st);
+}

@@ -1,0 +1,376 @@
+// Row-wise kernels between the contractions: split-K reduction, E_carry on rejected rows,
+// RMS norms, RoPE, the K/V scatter, the embedding gather and the argmax read-out.
+#include "cod_internal.cuh"
+
+namespace {
+
+__device__ __forceinline__ int valid_rows(const int* n_rows_dev, int n_rows) {
+  return n_rows_dev ? min(*n_rows_dev, n_rows) : n_rows;
+}
+
+// ------------------------------------------------------------------ F(E_carry) = fc . e_carry
+// F is linear and bias-free, so F(h + E_carry) = F(h) + F(E_carry) (Eq. 2; Algorithm 1, right
+// column, step 2): the embedding can be added after the contraction, before the norm.
+template <typename T>
+__global__ void k_fcE(const T* __restrict__ fc, const T* __restrict__ e, int D_in, float* __restrict__ out) {
+  __shared__ float red[33];
+  const int n = blockIdx.x;
+  float acc = 0.f;
+  for (int k = threadIdx.x; k < D_in; k += blockDim.x) acc = fmaf(cod_ld(fc + static_cast<size_t>(n) * D_in + k), cod_ld(e + k), acc);
+  acc = cod_block_sum(acc, red);
+  if (threadIdx.x == 0) out[n] = acc;
+}
+
+// ------------------------------------------------------------------ fc finish
+// z[row] = N_h( sum_splits part[i] + [row rejected] F(E_carry) )   (one block per kept row)
+template <typename T>
+__global__ void k_fc_finish(const float* __restrict__ part, int splits, int n_rows, const int* n_rows_dev,
+                            const int* __restrict__ a_rows, const int* __restrict__ carry_slot,
+                            const float* __restrict__ fcE, const T* __restrict__ gain, int D, float eps,
+                            int do_norm, T* __restrict__ z, float* __restrict__ tap) {
+  extern __shared__ float sh[];   // [D] values + 33 reduction slots
+  float* vals = sh;
+  float* red = sh + D;
+  const int i = blockIdx.x;
+  if (i >= valid_rows(n_rows_dev, n_rows)) return;
+  const int row = a_rows ? a_rows[i] : i;
+  const bool rej = carry_slot[row] >= 0;
+  float ss = 0.f;
+  for (int d = threadIdx.x; d < D; d += blockDim.x) {
+    float v = 0.f;
+    for (int s = 0; s < splits; ++s) v += part[(static_cast<size_t>(s) * n_rows + i) * D + d];
+    if (rej) v += fcE[d];
+    vals[d] = v;
+    ss = fmaf(v, v, ss);
+  }
+  ss = cod_block_sum(ss, red);
+  const float scale = do_norm ? rsqrtf(ss / static_cast<float>(D) + eps) : 1.f;
+  for (int d = threadIdx.x; d < D; d += blockDim.x) {
+    const float v = do_norm ? vals[d] * scale * cod_ld(gain + d) : vals[d];
+    cod_st(z + static_cast<size_t>(row) * D + d, v);
+    if (tap) tap[static_cast<size_t>(row) * D + d] = v;
+  }
+}
+
+// ------------------------------------------------------------------ K/V finish
+// part: [splits][n_rows][2 * Ld * kvw]; columns [0, Ld*kvw) are K of every layer, the rest V.
+// Rotates K at the row's position and writes either J[l][row][2][n_kv][hd] or straight to the
+// row's destination (page slot if accepted, carry slot if rejected).
+template <typename T>
+__global__ void k_kv_finish(const float* __restrict__ part, int splits, int n_rows, const int* n_rows_dev,
+                            const int* __restrict__ a_rows, const float* __restrict__ rope_win, int Ld,
+                            int n_kv, int hd, T* __restrict__ J, int R_total,
+                            const int* __restrict__ commit_slot, const int* __restrict__ carry_slot,
+                            T* __restrict__ pool, T* __restrict__ carry, int page, int n_pages, int W,
+                            int max_batch, int to_state) {
+  const int i = blockIdx.x, l = blockIdx.y;
+  if (i >= valid_rows(n_rows_dev, n_rows)) return;
+  const int row = a_rows ? a_rows[i] : i;
+  const int kvw = n_kv * hd, half = hd >> 1, ldc = 2 * Ld * kvw;
+  const float* cs = rope_win + static_cast<size_t>(row) * hd;
+
+  T* dstK = nullptr;   // address of [h = 0][K][..][d = 0]; strides below
+  size_t h_stride, kv_stride;
+  if (!to_state) {
+    dstK = J + ((static_cast<size_t>(l) * R_total + row) * 2) * kvw;
+    h_stride = hd;
+    kv_stride = kvw;
+  } else {
+    const int cslot = commit_slot[row], uslot = carry_slot[row];
+    if (cslot >= 0) {
+      const int pg = cslot / page, off = cslot - pg * page;
+      dstK = pool + (((static_cast<size_t>(l) * n_pages + pg) * n_kv) * 2) * page * hd + static_cast<size_t>(off) * hd;
+      h_stride = static_cast<size_t>(2) * page * hd;
+      kv_stride = static_cast<size_t>(page) * hd;
+    } else if (uslot >= 0 && carry) {
+      const int s = uslot / W, u = uslot - s * W;
+      dstK = carry + (((static_cast<size_t>(l) * max_batch + s) * n_kv) * 2) * W * hd + static_cast<size_t>(u) * hd;
+      h_stride = static_cast<size_t>(2) * W * hd;
+      kv_stride = static_cast<size_t>(W) * hd;
+    } else {
+      return;   // nowhere to go (position beyond the page table: already flagged)
+    }
+  }
+  for (int e = threadIdx.x; e < n_kv * half; e += blockDim.x) {
+    const int h = e / half, j = e - h * half;
+    float k1 = 0.f, k2 = 0.f, v1 = 0.f, v2 = 0.f;
+    for (int s = 0; s < splits; ++s) {
+      const float* p = part + (static_cast<size_t>(s) * n_rows + i) * ldc;
+      k1 += p[l * kvw + h * hd + j];
+      k2 += p[l * kvw + h * hd + j + half];
+      v1 += p[Ld * kvw + l * kvw + h * hd + j];
+      v2 += p[Ld * kvw + l * kvw + h * hd + j + half];
+    }
+    const float c = cs[j], sn = cs[half + j];
+    T* kd = dstK + h * h_stride;
+    cod_st(kd + j, k1 * c - k2 * sn);
+    cod_st(kd + j + half, k2 * c + k1 * sn);
+    cod_st(kd + kv_stride + j, v1);
+    cod_st(kd + kv_stride + j + half, v2);
+  }
+}
+
+// ------------------------------------------------------------------ scatter (unfused form)
+// One block per (row, layer): copies the row's K and V (n_kv heads of hd elements each) from J
+// to its page slot or carry slot with 128-bit accesses.
+template <typename T>
+__global__ void k_scatter_kv(const T* __restrict__ J, int R_total, int n_kv, int hd,
+                             const int* __restrict__ commit_slot, const int* __restrict__ carry_slot,
+                             T* __restrict__ pool, T* __restrict__ carry, int page, int n_pages, int W,
+                             int max_batch, int use_carry) {
+  const int row = blockIdx.x, l = blockIdx.y;
+  const int kvw = n_kv * hd;
+  const int cslot = commit_slot[row], uslot = carry_slot[row];
+  T* dst;
+  size_t h_stride, kv_stride;
+  if (cslot >= 0) {
+    const int pg = cslot / page, off = cslot - pg * page;
+    dst = pool + (((static_cast<size_t>(l) * n_pages + pg) * n_kv) * 2) * page * hd + static_cast<size_t>(off) * hd;
+    h_stride = static_cast<size_t>(2) * page * hd;
+    kv_stride = static_cast<size_t>(page) * hd;
+  } else if (uslot >= 0 && use_carry) {
+    const int s = uslot / W, u = uslot - s * W;
+    dst = carry + (((static_cast<size_t>(l) * max_batch + s) * n_kv) * 2) * W * hd + static_cast<size_t>(u) * hd;
+    h_stride = static_cast<size_t>(2) * W * hd;
+    kv_stride = static_cast<size_t>(W) * hd;
+  } else {
+    return;
+  }
+  constexpr int VEC = 16 / sizeof(T);
+  const T* src = J + ((static_cast<size_t>(l) * R_total + row) * 2) * kvw;
+  const int per_head = hd / VEC;
+  for (int e = threadIdx.x; e < 2 * n_kv * per_head; e += blockDim.x) {
+    const int kv = e / (n_kv * per_head), rem = e - kv * n_kv * per_head;
+    const int h = rem / per_head, v = rem - h * per_head;
+    const uint4 val = *reinterpret_cast<const uint4*>(src + static_cast<size_t>(kv) * kvw + h * hd + v * VEC);
+    *reinterpret_cast<uint4*>(dst + h * h_stride + kv * kv_stride + v * VEC) = val;
+  }
+}
+
+__global__ void k_update_lens(const int* __restrict__ accept_len, int S, int W, int mode, int max_tokens,
+                              int* __restrict__ committed_len, int* __restrict__ carry_len, uint32_t* status) {
+  const int s = blockIdx.x * blockDim.x + threadIdx.x;
+  if (s >= S) return;
+  const int m = accept_len[s];
+  const int L = committed_len[s] + m;
+  if (L > max_tokens) atomicOr(status, COD_DEV_PAGE_OVERFLOW);
+  committed_len[s] = L;
+  carry_len[s] = mode == COD_CARRY ? W - m : 0;
+}
+
+// ------------------------------------------------------------------ block input
+// x = Emb[[bonus, MASK, ...]], a = N(x) * g_attn[0]; also clears the argmax keys.
+template <typename T>
+__global__ void k_embed_norm(const T* __restrict__ emb, const int* __restrict__ bonus, int W, int mask_id,
+                             int vocab, const T* __restrict__ gain, int D, float eps, float* __restrict__ x,
+                             T* __restrict__ a, unsigned long long* __restrict__ amax) {
+  __shared__ float red[33];
+  const int r = blockIdx.x, s = r / W, p = r - s * W;
+  int tok = p == 0 ? bonus[s] : mask_id;
+  if (tok < 0 || tok >= vocab) tok = 0;
+  float ss = 0.f;
+  for (int d = threadIdx.x; d < D; d += blockDim.x) {
+    const float v = cod_ld(emb + static_cast<size_t>(tok) * D + d);
+    x[static_cast<size_t>(r) * D + d] = v;
+    ss = fmaf(v, v, ss);
+  }
+  ss = cod_block_sum(ss, red);
+  const float scale = rsqrtf(ss / static_cast<float>(D) + eps);
+  for (int d = threadIdx.x; d < D; d += blockDim.x)
+    cod_st(a + static_cast<size_t>(r) * D + d, x[static_cast<size_t>(r) * D + d] * scale * cod_ld(gain + d));
+  if (threadIdx.x == 0) amax[r] = 0ull;
+}
+
+// ------------------------------------------------------------------ Q/K/V of the block rows
+// part: [splits][R][qw + 2 kvw] -> q (rotated), k_blk (rotated), v_blk
+template <typename T>
+__global__ void k_qkv_finish(const float* __restrict__ part, int splits, int R, int n_q, int n_kv, int hd,
+                             const float* __restrict__ rope_blk, T* __restrict__ q, T* __restrict__ kb,
+                             T* __restrict__ vb) {
+  const int r = blockIdx.x;
+  const int qw = n_q * hd, kvw = n_kv * hd, half = hd >> 1, ldc = qw + 2 * kvw;
+  const float* cs = rope_blk + static_cast<size_t>(r) * hd;
+  const int n_rot = (n_q + n_kv) * half;
+  for (int e = threadIdx.x; e < n_rot + kvw; e += blockDim.x) {
+    if (e < n_rot) {
+      const int h = e / half, j = e - h * half;        // heads 0..n_q-1 are q, then k
+      float a = 0.f, b = 0.f;
+      for (int s = 0; s < splits; ++s) {
+        const float* p = part + (static_cast<size_t>(s) * R + r) * ldc + h * hd;
+        a += p[j];
+        b += p[j + half];
+      }
+      const float c = cs[j], sn = cs[half + j];
+      T* dst = h < n_q ? q + static_cast<size_t>(r) * qw + h * hd : kb + static_cast<size_t>(r) * kvw + (h - n_q) * hd;
+      cod_st(dst + j, a * c - b * sn);
+      cod_st(dst + j + half, b * c + a * sn);
+    } else {
+      const int d = e - n_rot;
+      float v = 0.f;
+      for (int s = 0; s < splits; ++s) v += part[(static_cast<size_t>(s) * R + r) * ldc + qw + kvw + d];
+      cod_st(vb + static_cast<size_t>(r) * kvw + d, v);
+    }
+  }
+}
+
+// Rotates caller-supplied q / k_blk (the stand-alone attention entry point).
+template <typename T>
+__global__ void k_rope_qk(const T* __restrict__ qin, const T* __restrict__ kin, int n_q, int n_kv, int hd,
+                          const float* __restrict__ rope_blk, T* __restrict__ q, T* __restrict__ kb) {
+  const int r = blockIdx.x;
+  const int qw = n_q * hd, kvw = n_kv * hd, half = hd >> 1;
+  const float* cs = rope_blk + static_cast<size_t>(r) * hd;
+  for (int e = threadIdx.x; e < (n_q + n_kv) * half; e += blockDim.x) {
+    const int h = e / half, j = e - h * half;
+    const T* src = h < n_q ? qin + static_cast<size_t>(r) * qw + h * hd : kin + static_cast<size_t>(r) * kvw + (h - n_q) * hd;
+    T* dst = h < n_q ? q + static_cast<size_t>(r) * qw + h * hd : kb + static_cast<size_t>(r) * kvw + (h - n_q) * hd;
+    const float a = cod_ld(src + j), b = cod_ld(src + j + half);
+    const float c = cs[j], sn = cs[half + j];
+    cod_st(dst + j, a * c - b * sn);
+    cod_st(dst + j + half, b * c + a * sn);
+  }
+}
+
+// ------------------------------------------------------------------ residual + norm
+// x[r] += sum_splits part (if any); a[r] = N(x[r]) * gain
+template <typename T>
+__global__ void k_resid_norm(const float* __restrict__ part, int splits, int R, int D, float* x,
+                             const T* __restrict__ gain, float eps, T* __restrict__ a, float* __restrict__ tap,
+                             unsigned long long* __restrict__ amax) {
+  __shared__ float red[33];
+  const int r = blockIdx.x;
+  float ss = 0.f;
+  for (int d = threadIdx.x; d < D; d += blockDim.x) {
+    float v = x[static_cast<size_t>(r) * D + d];
+    if (part)
+      for (int s = 0; s < splits; ++s) v += part[(static_cast<size_t>(s) * R + r) * D + d];
+    if (part) x[static_cast<size_t>(r) * D + d] = v;   // without partials x is read-only input
+    if (tap) tap[static_cast<size_t>(r) * D + d] = v;
+    ss = fmaf(v, v, ss);
+  }
+  ss = cod_block_sum(ss, red);
+  const float scale = rsqrtf(ss / static_cast<float>(D) + eps);
+  for (int d = threadIdx.x; d < D; d += blockDim.x)
+    cod_st(a + static_cast<size_t>(r) * D + d, x[static_cast<size_t>(r) * D + d] * scale * cod_ld(gain + d));
+  if (amax && threadIdx.x == 0) amax[r] = 0ull;
+}
+
+__global__ void k_finalize(const unsigned long long* __restrict__ amax, int R, int W, const int* __restrict__ bonus,
+                           int* __restrict__ tok, int* __restrict__ next_draft, float* __restrict__ top_logit) {
+  const int r = blockIdx.x * blockDim.x + threadIdx.x;
+  if (r >= R) return;
+  const unsigned long long key = amax[r];
+  const int t = cod_unpack_index(key);
+  if (tok) tok[r] = t;
+  if (top_logit) top_logit[r] = cod_unpack_logit(key);
+  if (next_draft) next_draft[r] = (r % W == 0) ? bonus[r / W] : t;
+}
+
+}  // namespace
+
+#define DISPATCH_T(c, CALL_BF16, CALL_F32) \
+  do {                                     \
+    if ((c)->cfg.dtype == COD_BF16) { CALL_BF16; } else { CALL_F32; } \
+  } while (0)
+
+int cod_launch_fcE(cod_ctx* c, cudaStream_t st) {
+  DISPATCH_T(c,
+             (k_fcE<__nv_bfloat16><<<c->D, 256, 0, st>>>(static_cast<const __nv_bfloat16*>(c->w.fc), static_cast<const __nv_bfloat16*>(c->w.e_carry), c->D_in, c->fcE)),
+             (k_fcE<float><<<c->D, 256, 0, st>>>(static_cast<const float*>(c->w.fc), static_cast<const float*>(c->w.e_carry), c->D_in, c->fcE)));
+  COD_CHECK_LAUNCH(c);
+  return COD_OK;
+}
+
+int cod_launch_fc_finish(cod_ctx* c, const float* part, int splits, int n_rows, const int* n_rows_dev,
+                         const int* a_rows, const int* carry_slot, float* tap_z, cudaStream_t st) {
+  if (n_rows <= 0) return COD_OK;
+  const size_t smem = (c->D + 33) * sizeof(float);
+  const int do_norm = (c->cfg.flags & COD_F_HIDDEN_NORM) ? 1 : 0;
+  DISPATCH_T(c,
+             (k_fc_finish<__nv_bfloat16><<<n_rows, 256, smem, st>>>(part, splits, n_rows, n_rows_dev, a_rows, carry_slot, c->fcE, static_cast<const __nv_bfloat16*>(c->w.g_hidden), c->D, c->cfg.rms_eps, do_norm, static_cast<__nv_bfloat16*>(c->z), tap_z)),
+             (k_fc_finish<float><<<n_rows, 256, smem, st>>>(part, splits, n_rows, n_rows_dev, a_rows, carry_slot, c->fcE, static_cast<const float*>(c->w.g_hidden), c->D, c->cfg.rms_eps, do_norm, static_cast<float*>(c->z), tap_z)));
+  COD_CHECK_LAUNCH(c);
+  return COD_OK;
+}
+
+int cod_launch_kv_finish(cod_ctx* c, const float* part, int splits, int n_rows, const int* n_rows_dev,
+                         const int* a_rows, const cod_split* sp, void* J, const cod_state* ds, int R_total,
+                         cudaStream_t st) {
+  if (n_rows <= 0) return COD_OK;
+  const cod_config& f = c->cfg;
+  dim3 grid(n_rows, f.n_layers);
+  const int to_state = ds ? 1 : 0;
+  DISPATCH_T(c,
+             (k_kv_finish<__nv_bfloat16><<<grid, 128, 0, st>>>(part, splits, n_rows, n_rows_dev, a_rows, c->rope_win, f.n_layers, f.n_kv_heads, f.head_dim, static_cast<__nv_bfloat16*>(J), R_total, sp->commit_slot, sp->carry_slot, ds ? static_cast<__nv_bfloat16*>(ds->kv_pool) : nullptr, ds ? static_cast<__nv_bfloat16*>(ds->carry_kv) : nullptr, f.page_size, f.n_pages, f.block, f.max_batch, to_state)),
+             (k_kv_finish<float><<<grid, 128, 0, st>>>(part, splits, n_rows, n_rows_dev, a_rows, c->rope_win, f.n_layers, f.n_kv_heads, f.head_dim, static_cast<float*>(J), R_total, sp->commit_slot, sp->carry_slot, ds ? static_cast<float*>(ds->kv_pool) : nullptr, ds ? static_cast<float*>(ds->carry_kv) : nullptr, f.page_size, f.n_pages, f.block, f.max_batch, to_state)));
+  COD_CHECK_LAUNCH(c);
+  return COD_OK;
+}
+
+int cod_launch_scatter(cod_ctx* c, const void* J, const cod_split* sp, int S, int mode, const cod_state* ds,
+                       cudaStream_t st) {
+  const cod_config& f = c->cfg;
+  const int R = S * f.block;
+  dim3 grid(R, f.n_layers);
+  const int use_carry = mode == COD_CARRY;
+  DISPATCH_T(c,
+             (k_scatter_kv<__nv_bfloat16><<<grid, 128, 0, st>>>(static_cast<const __nv_bfloat16*>(J), R, f.n_kv_heads, f.head_dim, sp->commit_slot, sp->carry_slot, static_cast<__nv_bfloat16*>(ds->kv_pool), static_cast<__nv_bfloat16*>(ds->carry_kv), f.page_size, f.n_pages, f.block, f.max_batch, use_carry)),
+             (k_scatter_kv<float><<<grid, 128, 0, st>>>(static_cast<const float*>(J), R, f.n_kv_heads, f.head_dim, sp->commit_slot, sp->carry_slot, static_cast<float*>(ds->kv_pool), static_cast<float*>(ds->carry_kv), f.page_size, f.n_pages, f.block, f.max_batch, use_carry)));
+  COD_CHECK_LAUNCH(c);
+  return COD_OK;
+}
+
+int cod_launch_update_lens(cod_ctx* c, const cod_split* sp, int S, int mode, const cod_state* ds, cudaStream_t st) {
+  k_update_lens<<<(S + 127) / 128, 128, 0, st>>>(sp->accept_len, S, c->cfg.block, mode,
+                                                 c->cfg.max_pages_per_seq * c->cfg.page_size, ds->committed_len,
+                                                 ds->carry_len, c->status);
+  COD_CHECK_LAUNCH(c);
+  return COD_OK;
+}
+
+int cod_launch_embed_norm(cod_ctx* c, const int32_t* bonus, int S, cudaStream_t st) {
+  const cod_config& f = c->cfg;
+  const int R = S * f.block;
+  DISPATCH_T(c,
+             (k_embed_norm<__nv_bfloat16><<<R, 256, 0, st>>>(static_cast<const __nv_bfloat16*>(c->w.emb), bonus, f.block, f.mask_token_id, f.vocab, static_cast<const __nv_bfloat16*>(c->w.g_attn), c->D, f.rms_eps, c->x, static_cast<__nv_bfloat16*>(c->a), c->amax)),
+             (k_embed_norm<float><<<R, 256, 0, st>>>(static_cast<const float*>(c->w.emb), bonus, f.block, f.mask_token_id, f.vocab, static_cast<const float*>(c->w.g_attn), c->D, f.rms_eps, c->x, static_cast<float*>(c->a), c->amax)));
+  COD_CHECK_LAUNCH(c);
+  return COD_OK;
+}
+
+int cod_launch_qkv_finish(cod_ctx* c, const float* part, int splits, int R, cudaStream_t st) {
+  const cod_config& f = c->cfg;
+  DISPATCH_T(c,
+             (k_qkv_finish<__nv_bfloat16><<<R, 256, 0, st>>>(part, splits, R, f.n_q_heads, f.n_kv_heads, f.head_dim, c->rope_blk, static_cast<__nv_bfloat16*>(c->q), static_cast<__nv_bfloat16*>(c->kb), static_cast<__nv_bfloat16*>(c->vb))),
+             (k_qkv_finish<float><<<R, 256, 0, st>>>(part, splits, R, f.n_q_heads, f.n_kv_heads, f.head_dim, c->rope_blk, static_cast<float*>(c->q), static_cast<float*>(c->kb), static_cast<float*>(c->vb))));
+  COD_CHECK_LAUNCH(c);
+  return COD_OK;
+}
+
+// rope_blk must already hold the block rows' tables
+int cod_launch_rope_qk(cod_ctx* c, const void* q, const void* k, const int32_t* committed_len, int S, cudaStream_t st) {
+  (void)committed_len;
+  const cod_config& f = c->cfg;
+  const int R = S * f.block;
+  DISPATCH_T(c,
+             (k_rope_qk<__nv_bfloat16><<<R, 256, 0, st>>>(static_cast<const __nv_bfloat16*>(q), static_cast<const __nv_bfloat16*>(k), f.n_q_heads, f.n_kv_heads, f.head_dim, c->rope_blk, static_cast<__nv_bfloat16*>(c->q), static_cast<__nv_bfloat16*>(c->kb))),
+             (k_rope_qk<float><<<R, 256, 0, st>>>(static_cast<const float*>(q), static_cast<const float*>(k), f.n_q_heads, f.n_kv_heads, f.head_dim, c->rope_blk, static_cast<float*>(c->q), static_cast<float*>(c->kb))));
+  COD_CHECK_LAUNCH(c);
+  return COD_OK;
+}
+
+int cod_launch_resid_norm(cod_ctx* c, const float* part, int splits, int R, float* x, const void* gain,
+                          float* tap_x, cudaStream_t st) {
+  DISPATCH_T(c,
+             (k_resid_norm<__nv_bfloat16><<<R, 256, 0, st>>>(part, splits, R, c->D, x, static_cast<const __nv_bfloat16*>(gain), c->cfg.rms_eps, static_cast<__nv_bfloat16*>(c->a), tap_x, c->amax)),
+             (k_resid_norm<float><<<R, 256, 0, st>>>(part, splits, R, c->D, x, static_cast<const float*>(gain), c->cfg.rms_eps, static_cast<float*>(c->a), tap_x, c->amax)));
+  COD_CHECK_LAUNCH(c);
+  return COD_OK;
+}
+
+int cod_launch_finalize(cod_ctx* c, int R, int W, const int32_t* bonus, int32_t* tok, int32_t* next_draft,
+                        float* top_logit, cudaStream_t st) {
+  k_finalize<<<(R + 127) / 128, 128, 0, st>>>(c->amax, R, W, bonus, tok, next_draft, top_logit);
+  COD_CHECK_LAUNCH(c);
+  return COD_OK;
+}

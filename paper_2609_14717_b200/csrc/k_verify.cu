@@ -1,0 +1,139 @@
+// Part 1: greedy verify-accept and the row split (Section 2 "Preliminaries"; Algorithm 2
+// "GreedyVerify"), plus the cos/sin tables of the positions this round touches.
+#include "cod_internal.cuh"
+
+// One block. A warp handles one sequence at a time: each lane compares one window row,
+// a ballot finds the first mismatch (acceptance is a PREFIX rule: a later match after the
+// first mismatch does not count). Then a scan over sequences gives the CSR offsets and
+// all threads write the per-row arrays.
+__global__ void __launch_bounds__(1024)
+k_verify_accept(const int32_t* __restrict__ draft, const int32_t* __restrict__ target, int S, int W,
+                int n_forced, int vocab, int page, int max_pages, int n_pages,
+                const int32_t* __restrict__ committed_len, const int32_t* __restrict__ block_table,
+                cod_split out, uint32_t* status) {
+  extern __shared__ int sm[];
+  int* s_m = sm;              // [S]
+  int* s_acc = sm + S;        // [S+1]
+  const int lane = threadIdx.x & 31, wid = threadIdx.x >> 5, nw = blockDim.x >> 5;
+  uint32_t flags = 0;
+
+  for (int s = wid; s < S; s += nw) {
+    int m = W;
+    for (int p0 = 0; p0 < W && m == W; p0 += 32) {
+      const int p = p0 + lane;
+      bool ok = true;
+      if (p < W) {
+        const int d = draft[s * W + p], t = target[s * (W + 1) + p];
+        if (d < 0 || d >= vocab || t < 0 || t >= vocab) flags |= COD_DEV_BAD_TOKEN;
+        ok = (p < n_forced) || (d == t);
+      }
+      const unsigned miss = __ballot_sync(0xffffffffu, !ok);
+      if (miss) m = p0 + __ffs(miss) - 1;
+    }
+    if (lane == 0) {
+      s_m[s] = m;
+      int b = target[s * (W + 1) + m];
+      if (b < 0 || b >= vocab) { flags |= COD_DEV_BAD_TOKEN; b = 0; }
+      out.accept_len[s] = m;
+      out.bonus[s] = b;
+    }
+  }
+  __syncthreads();
+
+  // exclusive prefix sums of m_s (warp 0, chunks of 32 with a running carry)
+  if (wid == 0) {
+    int run = 0;
+    for (int s0 = 0; s0 < S; s0 += 32) {
+      const int s = s0 + lane;
+      const int v = s < S ? s_m[s] : 0;
+      int inc = v;
+#pragma unroll
+      for (int o = 1; o < 32; o <<= 1) {
+        const int n = __shfl_up_sync(0xffffffffu, inc, o);
+        if (lane >= o) inc += n;
+      }
+      if (s < S) s_acc[s] = run + inc - v;
+      run += __shfl_sync(0xffffffffu, inc, 31);
+    }
+    if (lane == 0) s_acc[S] = run;
+  }
+  __syncthreads();
+
+  for (int s = threadIdx.x; s <= S; s += blockDim.x) {
+    out.acc_off[s] = s_acc[s];
+    out.rej_off[s] = s * W - s_acc[s];
+  }
+  const int R = S * W, acc_total = s_acc[S];
+  for (int r = threadIdx.x; r < R; r += blockDim.x) {
+    const int s = r / W, p = r - s * W, m = s_m[s];
+    const int L = committed_len[s];
+    if (L < 0) flags |= COD_DEV_BAD_LEN;
+    const int pos = L + p;
+    out.row_pos[r] = pos;
+    int cslot = -1, uslot = -1;
+    if (p < m) {
+      const int lp = pos / page;
+      if (L < 0 || lp >= max_pages) {
+        flags |= COD_DEV_PAGE_OVERFLOW;
+      } else {
+        const int pg = block_table[s * max_pages + lp];
+        if (pg < 0 || pg >= n_pages) flags |= COD_DEV_BAD_PAGE;
+        else cslot = pg * page + pos % page;
+      }
+      out.acc_rows[s_acc[s] + p] = r;
+    } else {
+      uslot = s * W + (p - m);
+      out.rej_rows[(s * W - s_acc[s]) + (p - m)] = r;
+    }
+    out.commit_slot[r] = cslot;
+    out.carry_slot[r] = uslot;
+    if (r >= acc_total) out.acc_rows[r] = -1;
+    if (r >= R - acc_total) out.rej_rows[r] = -1;
+  }
+  if (flags) atomicOr(status, flags);
+}
+
+// cos/sin of pos * theta^(-2j/hd) for the window rows (pos = L_s + p) and the next block's
+// rows (pos = L_s + m_s + i). The angle is formed and reduced modulo 2*pi in double, so
+// positions of tens of thousands lose nothing in float.
+__global__ void k_rope_tables(const int32_t* __restrict__ committed_len, const int32_t* __restrict__ accept_len,
+                              const double* __restrict__ inv_freq, int S, int W, int half,
+                              float* __restrict__ rope_win, float* __restrict__ rope_blk) {
+  const int r = blockIdx.x, s = r / W, p = r - s * W;
+  const int L = max(committed_len[s], 0);
+  const int m = accept_len ? accept_len[s] : 0;
+  const double two_pi = 6.283185307179586476925286766559;
+  for (int j = threadIdx.x; j < half; j += blockDim.x) {
+    const double f = inv_freq[j];
+    double a = static_cast<double>(L + p) * f;
+    a -= two_pi * rint(a / two_pi);
+    float sn, cs;
+    sincosf(static_cast<float>(a), &sn, &cs);
+    if (rope_win) { rope_win[r * 2 * half + j] = cs; rope_win[r * 2 * half + half + j] = sn; }
+    double b = static_cast<double>(L + m + p) * f;
+    b -= two_pi * rint(b / two_pi);
+    sincosf(static_cast<float>(b), &sn, &cs);
+    if (rope_blk) { rope_blk[r * 2 * half + j] = cs; rope_blk[r * 2 * half + half + j] = sn; }
+  }
+}
+
+int cod_launch_verify(cod_ctx* c, const int32_t* draft, const int32_t* target, int S, int n_forced,
+                      const cod_state* state, const cod_split* out, cudaStream_t st) {
+  const int W = c->cfg.block;
+  const size_t smem = static_cast<size_t>(2 * S + 2) * sizeof(int);
+  k_verify_accept<<<1, 1024, smem, st>>>(draft, target, S, W, n_forced, c->cfg.vocab, c->cfg.page_size,
+                                         c->cfg.max_pages_per_seq, c->cfg.n_pages, state->committed_len,
+                                         state->block_table, *out, c->status);
+  COD_CHECK_LAUNCH(c);
+  k_rope_tables<<<S * W, 64, 0, st>>>(state->committed_len, out->accept_len, c->inv_freq_d, S, W, c->half,
+                                      c->rope_win, c->rope_blk);
+  COD_CHECK_LAUNCH(c);
+  return COD_OK;
+}
+
+int cod_launch_rope_blk_only(cod_ctx* c, const int32_t* committed_len, int S, cudaStream_t st) {
+  k_rope_tables<<<S * c->cfg.block, 64, 0, st>>>(committed_len, nullptr, c->inv_freq_d, S, c->cfg.block, c->half,
+                                                 nullptr, c->rope_blk);
+  COD_CHECK_LAUNCH(c);
+  return COD_OK;
+}

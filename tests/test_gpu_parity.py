@@ -1,0 +1,394 @@
+"""GPU parity: the CUDA library (through its C ABI) against the CPU oracle, element by element,
+on the same seeded inputs.  Integers must be bit-exact; floating point within the stated
+relative tolerance per tensor (2e-2 bf16, 1e-3 float32); argmax tokens equal wherever the
+oracle's top-2 logit gap is at least 1e-2."""
+import itertools
+
+import numpy as np
+import pytest
+import torch
+
+from oracle import cod_oracle as orc
+from paper_2609_14717_b200 import synth
+from tests.helpers import rel_err, small_bf16
+
+pytestmark = pytest.mark.gpu
+
+
+def _B():
+    from paper_2609_14717_b200 import binding
+    return binding
+
+
+def _H():
+    from tests import gpu_harness
+    return gpu_harness
+
+
+# ----------------------------------------------------------------------------- part 1
+@pytest.mark.parametrize("n_forced", [0, 1])
+def test_verify_accept_exhaustive_W8(n_forced):
+    B, Hn = _B(), _H()
+    W, page = 8, 16
+    pats = list(itertools.product([False, True], repeat=W))
+    S = len(pats)
+    wl = synth.scaled(synth.workload("cfg1"), S=S, ctx=(0, 200))
+    lay = synth.make_layout(wl, 1)
+    rng = np.random.default_rng(1)
+    draft = rng.integers(0, 500, size=(S, W)).astype(np.int32)
+    target = rng.integers(0, 500, size=(S, W + 1)).astype(np.int32)
+    for s, bits in enumerate(pats):
+        for p, b in enumerate(bits):
+            target[s, p] = draft[s, p] if b else draft[s, p] + 500
+    cfg = B.make_config(wl.shape, S, int(lay["max_pages_per_seq"]), int(lay["n_pages"]))
+    ctx = B.Context(cfg)
+    st = B.State(cfg, "f32", S, lay["block_table"], lay["committed_len"])
+    sp = B.Split(S, W)
+    ctx.verify_accept(Hn.dev_i32(draft), Hn.dev_i32(target), S, n_forced, st, sp)
+    torch.cuda.synchronize()
+    ref = orc.verify_accept(draft, target, lay["committed_len"], lay["block_table"], page, n_forced)
+    got = sp.to_host()
+    for k in ref:
+        assert np.array_equal(got[k], ref[k]), k
+    assert ctx.poll_status() == 0
+    assert np.array_equal(st.committed_len.cpu().numpy(), lay["committed_len"])     # state untouched
+    ctx.close()
+
+
+@pytest.mark.parametrize("W,S", [(16, 32), (32, 4), (16, 64), (32, 33)])
+def test_verify_accept_random(W, S):
+    B, Hn = _B(), _H()
+    wl = synth.scaled(synth.workload("cfg3"), S=S, W=W, ctx=(17, 900), d_target=64, d_model=512, n_q=4, n_kv=1,
+                      vocab=5000, n_layers=1)
+    lay = synth.make_layout(wl, 2)
+    cfg = B.make_config(wl.shape, S, int(lay["max_pages_per_seq"]), int(lay["n_pages"]))
+    ctx = B.Context(cfg)
+    st = B.State(cfg, "bf16", S, lay["block_table"], lay["committed_len"])
+    sp = B.Split(S, W)
+    for r, nf in enumerate([1, 0, 1]):
+        rng = np.random.default_rng([7, r])
+        m = rng.integers(nf, W + 1, size=S).astype(np.int32)
+        draft, target = synth.make_tokens(wl, rng, m)
+        # sprinkle later matches after the first mismatch: they must not count
+        for s in range(S):
+            if m[s] + 2 < W:
+                target[s, m[s] + 2] = draft[s, m[s] + 2]
+        ctx.verify_accept(Hn.dev_i32(draft), Hn.dev_i32(target), S, nf, st, sp)
+        torch.cuda.synchronize()
+        ref = orc.verify_accept(draft, target, lay["committed_len"], lay["block_table"], wl.shape.page, nf)
+        assert np.array_equal(ref["accept_len"], m)
+        got = sp.to_host()
+        for k in ref:
+            assert np.array_equal(got[k], ref[k]), k
+    assert ctx.poll_status() == 0
+    ctx.close()
+
+
+# ----------------------------------------------------------------------------- parts 2, 3
+def _workloads():
+    return {
+        "tiny_f32": synth.scaled(synth.workload("cfg1"), S=3, ctx=(5, 140), n_rounds=6),
+        "tiny_f32_nonorm": synth.scaled(synth.workload("cfg1"), S=2, ctx=(30, 60), hidden_norm=False, n_rounds=4),
+        "small_bf16": small_bf16(S=3, W=16, n_layers=2, ctx=(40, 300)),
+        "small_bf16_W32": small_bf16(S=2, W=32, n_layers=1, ctx=(100, 200)),
+        "small_bf16_W8": small_bf16(S=5, W=8, n_layers=1, ctx=(0, 50)),
+    }
+
+
+@pytest.mark.parametrize("name", list(_workloads()))
+@pytest.mark.parametrize("mode", [orc.MODE_CARRY, orc.MODE_BASELINE])
+def test_project_and_scatter_unfused(name, mode):
+    """cod_verify_accept -> cod_project_kv -> cod_scatter_kv against the oracle's three steps."""
+    B, Hn = _B(), _H()
+    wl = _workloads()[name]
+    sh = wl.shape
+    P = Hn.Pair(wl, seed=3)
+    tol = Hn.TOL[sh.dtype]
+    J = torch.full((sh.n_layers, wl.R, 2, sh.n_kv, sh.hd), float("nan"), dtype=B.torch_dtype(sh.dtype), device="cuda")
+    m_cases = [None, np.full(wl.S, sh.W), np.zeros(wl.S, dtype=int)]
+    for r, m_fix in enumerate(m_cases):
+        rd, dev = P.round_inputs(r)
+        nf = wl.n_forced
+        if m_fix is not None:
+            rng = np.random.default_rng(r)
+            rd["draft"], rd["target"] = synth.make_tokens(wl, rng, m_fix.astype(np.int32))
+            dev["draft"], dev["target"] = Hn.dev_i32(rd["draft"]), Hn.dev_i32(rd["target"])
+            nf = 0
+        L0 = P.st_o.committed_len.copy()
+        pool0 = P.st_g.kv_pool.clone()
+        sp_o = orc.verify_accept(rd["draft"], rd["target"], P.st_o.committed_len, P.st_o.block_table, sh.page, nf)
+        J_o = orc.project_kv(rd["H"], sp_o, P.w_o, P.cfg_o, mode)
+        orc.scatter_kv(J_o, sp_o, P.st_o, mode)
+
+        J.fill_(float("nan"))
+        P.ctx.verify_accept(dev["draft"], dev["target"], wl.S, nf, P.st_g, P.split)
+        P.ctx.project_kv(dev["H"], P.split, wl.S, mode, J)
+        P.ctx.scatter_kv(J, P.split, wl.S, mode, P.st_g)
+        torch.cuda.synchronize()
+        P.check_split({"split": sp_o})
+        P.check_lens()
+        Jg = J.float().cpu().numpy().astype(np.float64)
+        kept = ~np.isnan(J_o[0, :, 0, 0, 0])
+        assert np.array_equal(np.isnan(Jg[0, :, 0, 0, 0]), ~kept)            # untouched rows stay untouched
+        if kept.any():
+            for l in range(sh.n_layers):
+                assert rel_err(Jg[l, kept, 0], J_o[l, kept, 0]) <= tol       # K
+                assert rel_err(Jg[l, kept, 1], J_o[l, kept, 1]) <= tol       # V
+        # the scatter is a copy: committed slots and carry rows hold J's bits exactly
+        Jh = J.cpu()
+        pool_g = P.st_g.kv_pool.cpu()
+        carry_g = P.st_g.carry_kv.cpu()
+        touched = torch.zeros(pool_g.shape, dtype=torch.bool)
+        for s in range(wl.S):
+            ms = int(sp_o["accept_len"][s])
+            for p in range(sh.W):
+                row = s * sh.W + p
+                if p < ms:
+                    pos = int(L0[s]) + p
+                    pg, off = int(P.st_o.block_table[s, pos // sh.page]), pos % sh.page
+                    assert torch.equal(pool_g[:, pg, :, :, off, :], Jh[:, row].transpose(1, 2))
+                    touched[:, pg, :, :, off, :] = True
+                elif mode == orc.MODE_CARRY:
+                    assert torch.equal(carry_g[:, s, :, :, p - ms, :], Jh[:, row].transpose(1, 2))
+        assert torch.equal(pool_g[~touched], pool0.cpu()[~touched])           # nothing else moved
+    assert P.ctx.poll_status() == 0
+    P.close()
+
+
+# ----------------------------------------------------------------------------- part 4
+def _attn_inputs(P, rng):
+    sh, S = P.wl.shape, P.wl.S
+    q = synth.to_storage(rng.standard_normal((S, sh.W, sh.n_q, sh.hd)).astype(np.float32), sh.dtype)
+    kb = synth.to_storage(rng.standard_normal((S, sh.W, sh.n_kv, sh.hd)).astype(np.float32), sh.dtype)
+    vb = synth.to_storage(rng.standard_normal((S, sh.W, sh.n_kv, sh.hd)).astype(np.float32), sh.dtype)
+    return q, kb, vb
+
+
+def _set_carry(P, rng, lens):
+    sh = P.wl.shape
+    for s, c in enumerate(lens):
+        P.st_o.carry_len[s] = c
+        P.st_o.carry[:, s] = np.nan
+        if c:
+            blk = synth.to_storage(rng.standard_normal((sh.n_layers, sh.n_kv, 2, c, sh.hd)).astype(np.float32), sh.dtype)
+            P.st_o.carry[:, s, :, :, :c, :] = blk
+            P.st_g.carry_kv[:, s, :, :, :c, :] = _B().to_device(blk, sh.dtype)
+    P.st_g.carry_len.copy_(torch.tensor(lens, dtype=torch.int32))
+
+
+@pytest.mark.parametrize("name,split_len", [("tiny_f32", 32), ("tiny_f32", 0), ("small_bf16", 64),
+                                            ("small_bf16_W32", 32), ("small_bf16_W8", 0)])
+def test_block_attn_parity(name, split_len):
+    B, Hn = _B(), _H()
+    wl = _workloads()[name]
+    sh = wl.shape
+    P = Hn.Pair(wl, seed=4, attn_split_len=split_len, poison=True)
+    rng = np.random.default_rng(11)
+    tol = Hn.TOL[sh.dtype]
+    out = torch.zeros((wl.S, sh.W, sh.n_q, sh.hd), dtype=B.torch_dtype(sh.dtype), device="cuda")
+    mass = torch.zeros((wl.S, sh.W, sh.n_q), dtype=torch.float32, device="cuda")
+    for lens in ([0] * wl.S, [sh.W] * wl.S, [1] + [sh.W // 2] * (wl.S - 1)):
+        _set_carry(P, rng, lens)
+        q, kb, vb = _attn_inputs(P, rng)
+        for layer in range(sh.n_layers):
+            for use_carry in (True, False):
+                ref, mref = orc.block_attn(layer, q, kb, vb, P.st_o, use_carry)
+                P.ctx.block_attn(layer, B.to_device(q, sh.dtype), B.to_device(kb, sh.dtype), B.to_device(vb, sh.dtype),
+                                 P.st_g, wl.S, use_carry, out, mass)
+                torch.cuda.synchronize()
+                got = out.float().cpu().numpy()
+                assert np.isfinite(got).all()            # poisoned pages / stale carry rows never read
+                assert rel_err(got, ref) <= tol
+                assert np.max(np.abs(mass.cpu().numpy() - mref)) <= tol
+    assert P.ctx.poll_status() == 0
+    P.close()
+
+
+def test_block_attn_split_and_page_invariance():
+    """Same inputs, different split lengths: equal to 1e-6 (float32). Permuted physical pages: same bits."""
+    B, Hn = _B(), _H()
+    wl = synth.scaled(synth.workload("cfg1"), S=2, ctx=(150, 300))
+    sh = wl.shape
+    rng = np.random.default_rng(5)
+    outs = []
+    for split_len in (32, 96, 0):
+        P = Hn.Pair(wl, seed=6, attn_split_len=split_len)
+        _set_carry(P, np.random.default_rng(1), [3, 8])
+        q, kb, vb = _attn_inputs(P, np.random.default_rng(2))
+        out = torch.zeros((wl.S, sh.W, sh.n_q, sh.hd), dtype=torch.float32, device="cuda")
+        P.ctx.block_attn(0, B.to_device(q, "f32"), B.to_device(kb, "f32"), B.to_device(vb, "f32"), P.st_g, wl.S, 1, out)
+        torch.cuda.synchronize()
+        outs.append(out.cpu().numpy())
+        if split_len == 32:
+            # permute the physical pages of the same logical content
+            n_pages = P.cfg_g.n_pages
+            perm = torch.from_numpy(np.random.default_rng(3).permutation(n_pages)).cuda()
+            inv = torch.argsort(perm)
+            P.st_g.kv_pool.copy_(P.st_g.kv_pool[:, inv].clone())
+            P.st_g.block_table.copy_(perm[P.st_g.block_table.long()].int())
+            out2 = torch.zeros_like(out)
+            P.ctx.block_attn(0, B.to_device(q, "f32"), B.to_device(kb, "f32"), B.to_device(vb, "f32"), P.st_g, wl.S, 1, out2)
+            torch.cuda.synchronize()
+            assert np.array_equal(out2.cpu().numpy(), outs[0])
+        P.close()
+    assert np.max(np.abs(outs[0] - outs[1])) <= 1e-6 and np.max(np.abs(outs[0] - outs[2])) <= 1e-6
+
+
+# ----------------------------------------------------------------------------- part 5
+@pytest.mark.parametrize("name", ["tiny_f32", "small_bf16"])
+def test_lm_head_planted_and_ties(name):
+    B, Hn = _B(), _H()
+    wl = _workloads()[name]
+    sh = wl.shape
+    P = Hn.Pair(wl, seed=8, fill_pool=False)
+    rng = np.random.default_rng(0)
+    V = sh.vocab
+    plant = [0, 63, 64, 127, 128, V // 2 + 1, V - 2, V - 1]
+    n = len(plant) + 1
+    x = rng.standard_normal((n, sh.d_model)).astype(np.float32)
+    y = orc.rmsnorm(x.astype(np.float64), P.w_o["g_final"], sh.rms_eps)
+    emb = P.w_host["emb"].copy()
+    for row, v in enumerate(plant):
+        emb[v] = synth.to_storage((y[row] * 3.0).astype(np.float32), sh.dtype)
+    emb[V - 7] = synth.to_storage((y[n - 1] * 3.0).astype(np.float32), sh.dtype)      # an exact tie ...
+    emb[5] = emb[V - 7]                                                               # ... lower id must win
+    w_o = dict(P.w_o, emb=emb.astype(np.float64))
+    P.w_g["emb"] = B.to_device(emb, sh.dtype)
+    P.ctx.set_weights(P.w_g)
+    tok = torch.zeros(n, dtype=torch.int32, device="cuda")
+    top = torch.zeros(n, dtype=torch.float32, device="cuda")
+    P.ctx.lm_head_argmax(torch.from_numpy(x).cuda(), n, tok, top)
+    torch.cuda.synchronize()
+    ref_tok, gap, logits = orc.lm_head_argmax(x.astype(np.float64), w_o, P.cfg_o)
+    assert list(ref_tok[:-1]) == plant and ref_tok[-1] == 5 and gap[-1] == 0.0
+    assert np.array_equal(tok.cpu().numpy(), ref_tok)
+    assert rel_err(top.cpu().numpy(), logits.max(axis=1)) <= Hn.TOL[sh.dtype]
+    P.close()
+
+
+# ----------------------------------------------------------------------------- whole rounds
+def _check_round(P, res_o, L0, tol):
+    Hn = _H()
+    sh = P.wl.shape
+    P.check_split(res_o)
+    P.check_lens()
+    for e in P.written_kv_errors(res_o, L0):
+        assert e <= tol
+    kept = ~np.isnan(res_o["J"][0, :, 0, 0, 0])
+    for l in range(sh.n_layers):
+        assert rel_err(P.taps.attn_out[l].cpu().numpy(), res_o["attn_out"][l]) <= tol
+    assert rel_err(P.taps.x_final.cpu().numpy(), res_o["x_final"]) <= tol
+    nd = P.next_draft.cpu().numpy()
+    assert np.array_equal(nd[:, 0], res_o["split"]["bonus"])
+    sure = res_o["gap"] >= Hn.GAP
+    sure[:, 0] = False
+    assert np.array_equal(nd[sure], res_o["next_draft"][sure])
+    return int((~sure[:, 1:]).sum())
+
+
+def test_round_parity_cfg1_every_round():
+    """The tiny float32 configuration: 16 rounds, context 128, rejected count uniform 0..7."""
+    Hn = _H()
+    wl = synth.workload("cfg1")
+    P = Hn.Pair(wl, seed=0, attn_split_len=64)
+    exempt = 0
+    for r in range(wl.n_rounds):
+        L0 = P.st_o.committed_len.copy()
+        res_o = P.run_round(r, orc.MODE_CARRY)
+        exempt += _check_round(P, res_o, L0, Hn.TOL["f32"])
+    assert exempt <= 2
+    assert P.ctx.poll_status() == 0
+    P.close()
+
+
+@pytest.mark.parametrize("name,wo_scale,mode", [
+    ("tiny_f32", 40.0, orc.MODE_CARRY), ("tiny_f32", 40.0, orc.MODE_BASELINE), ("tiny_f32_nonorm", 1.0, orc.MODE_CARRY),
+    ("small_bf16", 30.0, orc.MODE_CARRY), ("small_bf16", 30.0, orc.MODE_BASELINE),
+    ("small_bf16_W32", 1.0, orc.MODE_CARRY), ("small_bf16_W8", 30.0, orc.MODE_CARRY)])
+def test_round_parity_multi_round(name, wo_scale, mode):
+    """Open-loop rounds (inputs pre-generated), ragged acceptance, attention path made to matter."""
+    Hn = _H()
+    wl = _workloads()[name]
+    P = Hn.Pair(wl, seed=5, attn_split_len=64, wo_scale=wo_scale, poison=True)
+    tol = Hn.TOL[wl.shape.dtype]
+    toks_differ = False
+    for r in range(4):
+        L0 = P.st_o.committed_len.copy()
+        res_o = P.run_round(r, mode)
+        _check_round(P, res_o, L0, tol)
+        toks_differ |= len(np.unique(res_o["next_draft"][:, 1:])) > 1
+    if wo_scale > 1.0:
+        assert toks_differ                       # the argmax really depends on the attention path
+    assert P.ctx.poll_status() == 0
+    P.close()
+
+
+def test_full_acceptance_carry_equals_baseline_bitwise():
+    """m = W for every sequence: U is empty and the carry-mode round is the baseline round."""
+    Hn = _H()
+    wl = synth.scaled(small_bf16(S=2), accept=("fixed_m", 16), n_forced=0)
+    outs = []
+    for mode in (orc.MODE_CARRY, orc.MODE_BASELINE):
+        P = Hn.Pair(wl, seed=9, wo_scale=30.0)
+        for r in range(2):
+            P.run_round(r, mode)
+        assert (P.st_g.carry_len == 0).all()
+        outs.append((P.taps.x_final.cpu().numpy().copy(), P.next_draft.cpu().numpy().copy(),
+                     P.st_g.kv_pool.cpu().view(torch.int16).numpy().copy()))
+        P.close()
+    for a, b in zip(*outs):
+        assert np.array_equal(a, b)
+
+
+def test_determinism_two_runs_identical_bits():
+    Hn = _H()
+    wl = _workloads()["small_bf16"]
+    outs = []
+    for _ in range(2):
+        P = Hn.Pair(wl, seed=2, attn_split_len=64, wo_scale=30.0)
+        for r in range(3):
+            P.run_round(r, orc.MODE_CARRY)
+        outs.append((P.taps.x_final.cpu().numpy().copy(), P.taps.top_logit.cpu().numpy().copy(),
+                     P.st_g.carry_kv.cpu().view(torch.int16).numpy().copy()))
+        P.close()
+    for a, b in zip(*outs):
+        assert np.array_equal(a, b)
+
+
+# ----------------------------------------------------------------------------- host-made failures
+def test_status_word_and_argument_errors():
+    B, Hn = _B(), _H()
+    wl = synth.scaled(synth.workload("cfg1"), S=2, ctx=(10, 20))
+    P = Hn.Pair(wl, seed=1)
+    rd, dev = P.round_inputs(0)
+    # a token id outside the vocabulary is flagged, nothing faults
+    bad = rd["target"].copy(); bad[0, :] = wl.shape.vocab + 5
+    bd = rd["draft"].copy(); bd[0, :] = wl.shape.vocab + 5
+    P.ctx.draft_round(Hn.dev_i32(bd), Hn.dev_i32(bad), dev["H"], wl.S, 1, 0, P.st_g, P.split, P.next_draft, None)
+    assert P.ctx.poll_status() & B.DEV_BAD_TOKEN
+    assert P.ctx.poll_status() == 0                                   # cleared by the previous poll
+    # a committed length beyond the page table: rows are dropped and flagged
+    P.st_g.committed_len.fill_(int(P.cfg_g.max_pages_per_seq) * 16 - 2)
+    P.ctx.verify_accept(dev["draft"], dev["draft"].new_zeros((wl.S, wl.shape.W + 1)), wl.S, 1, P.st_g, P.split)
+    rdm = torch.cat([dev["draft"], dev["draft"][:, :1]], 1).contiguous()
+    P.ctx.verify_accept(dev["draft"], rdm, wl.S, 1, P.st_g, P.split)
+    assert P.ctx.poll_status() & B.DEV_PAGE_OVERFLOW
+    assert (P.split.commit_slot.cpu().numpy()[2:wl.shape.W] == -1).all()
+    # host-visible argument errors
+    with pytest.raises(B.CodError) as e:
+        P.ctx.draft_round(dev["draft"], dev["target"], dev["H"], wl.S + 1, 1, 0, P.st_g, P.split, P.next_draft, None)
+    assert e.value.status == -1
+    with pytest.raises(B.CodError):
+        P.ctx.draft_round(dev["draft"], dev["target"], dev["H"], wl.S, 2, 0, P.st_g, P.split, P.next_draft, None)
+    with pytest.raises(B.CodError):
+        P.ctx.block_attn(5, dev["H"], dev["H"], dev["H"], P.st_g, wl.S, 1, dev["H"])
+    cfg = B.make_config(wl.shape, 2, 4, 8)
+    cfg.head_dim = 48
+    with pytest.raises(B.CodError):
+        B.Context(cfg)
+    ctx2 = B.Context(B.make_config(wl.shape, 2, 4, 8))
+    with pytest.raises(B.CodError) as e:
+        ctx2.draft_round(dev["draft"], dev["target"], dev["H"], wl.S, 1, 0, P.st_g, P.split, P.next_draft, None)
+    assert e.value.status == -4
+    ctx2.close()
+    P.close()
