@@ -1,0 +1,431 @@
+#!/usr/bin/env python
+"""Benchmark of the Carryover drafting round (one step = one whole round: verify-accept,
+K/V projection with E_carry, scatter, block attention in every drafter layer, LM head + argmax).
+
+    python bench.py --gpus 1 --steps 64 --warmup 3            # batch-1 configuration (default)
+    python bench.py --workload cfg3                           # batch 32
+    python bench.py --impl reference                          # the CPU oracle on the host cores
+
+Prints ONE JSON line.  Inputs are seeded and synthetic (see the design doc for the recipe); the
+weights (about 2 GB) are re-read from HBM every round, so no L2 flush is needed between steps.
+With N > 1 (torchrun) every rank runs an independent replica: the round has no exchange step.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+from paper_2609_14717_b200 import synth  # noqa: E402
+
+METRIC = "drafting rounds/s"
+UNIT = "rounds/s"
+# dram__bytes_read.sum + dram__bytes_write.sum per launch of the dominant kernel, from the ncu
+# capture summarised under profiles/ (None until a capture exists for the current kernel).
+NCU_TRAFFIC_BYTES = {"cfg2": None, "cfg3": None}
+
+
+def load_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        p = json.load(open(path))
+        return {"hbm_gbs": float(p["hbm_gbs"]), "tflops": float(p.get("bf16_tflops_sustained", p["bf16_tflops"])),
+                "tflops_burst": float(p["bf16_tflops"]), "source": "measured"}
+    return {"hbm_gbs": 6650.0, "tflops": 1400.0, "tflops_burst": 1590.0, "source": "fallback"}
+
+
+# --------------------------------------------------------------------------- byte / flop model
+def round_model(wl, L_after, carry, kept_rows, es=2):
+    """Algorithmic bytes and flops of one round, per kernel class (weights read once per round,
+    committed KV read once per layer per sequence)."""
+    sh = wl.shape
+    D, Din, Ld = sh.d_model, sh.d_in, sh.n_layers
+    kvw, qw, R, V = sh.n_kv * sh.hd, sh.n_q * sh.hd, wl.R, sh.vocab
+    keys = float(np.sum(L_after + carry))
+    out = {
+        "fc": (D * Din * es + kept_rows * Din * es + kept_rows * D * es, 2.0 * kept_rows * Din * D),
+        "kv": (2 * Ld * kvw * D * es + kept_rows * Ld * 2 * kvw * es, 2.0 * kept_rows * D * 2 * Ld * kvw),
+        "qkv": (Ld * ((qw + 2 * kvw) * D * es + R * (D + qw + 2 * kvw) * es), 2.0 * R * D * (qw + 2 * kvw) * Ld),
+        "oproj": (Ld * (D * qw * es + R * (qw * es + D * 4)), 2.0 * R * qw * D * Ld),
+        "attn": (Ld * (keys * 2 * kvw * es + 2 * R * qw * es),
+                 Ld * 4.0 * sh.W * sh.n_q * sh.hd * float(np.sum(L_after + carry + sh.W))),
+        "lmhead": (V * D * es + R * D * es, 2.0 * R * D * V),
+    }
+    return out
+
+
+# --------------------------------------------------------------------------- clocks
+class ClockSampler:
+    """Polls NVML (read-only) for SM clock, power and throttle reasons while the timed region runs."""
+
+    def __init__(self, device_index: int):
+        self.samples, self.reasons, self.max_mhz = [], set(), None
+        self._stop = threading.Event()
+        self._thread = None
+        self._h = None
+        try:
+            import pynvml
+            import torch
+            pynvml.nvmlInit()
+            self._nv = pynvml
+            try:
+                uuid = str(torch.cuda.get_device_properties(device_index).uuid)
+                if not uuid.startswith("GPU-"):
+                    uuid = "GPU-" + uuid
+                self._h = pynvml.nvmlDeviceGetHandleByUUID(uuid.encode())
+            except Exception:
+                self._h = pynvml.nvmlDeviceGetHandleByIndex(device_index)
+            self.max_mhz = pynvml.nvmlDeviceGetMaxClockInfo(self._h, pynvml.NVML_CLOCK_SM)
+        except Exception:
+            self._h = None
+
+    def _loop(self):
+        nv = self._nv
+        names = {"hw_slowdown": 0x8, "sw_power_cap": 0x4, "sw_thermal_slowdown": 0x20,
+                 "hw_thermal_slowdown": 0x40, "hw_power_brake": 0x80}
+        while not self._stop.is_set():
+            try:
+                self.samples.append(nv.nvmlDeviceGetClockInfo(self._h, nv.NVML_CLOCK_SM))
+                try:
+                    bits = nv.nvmlDeviceGetCurrentClocksEventReasons(self._h)
+                except Exception:
+                    bits = nv.nvmlDeviceGetCurrentClocksThrottleReasons(self._h)
+                for k, b in names.items():
+                    if bits & b:
+                        self.reasons.add(k)
+            except Exception:
+                pass
+            time.sleep(0.004)
+
+    def __enter__(self):
+        if self._h is not None:
+            self._thread = threading.Thread(target=self._loop, daemon=True)
+            self._thread.start()
+        return self
+
+    def __exit__(self, *a):
+        self._stop.set()
+        if self._thread:
+            self._thread.join()
+
+    def summary(self):
+        if not self.samples:
+            return {"sm_mhz": None, "sm_max_mhz": self.max_mhz, "reasons": sorted(self.reasons), "samples": 0}
+        return {"sm_mhz": statistics.median(self.samples), "sm_max_mhz": self.max_mhz,
+                "reasons": sorted(self.reasons), "samples": len(self.samples)}
+
+
+# --------------------------------------------------------------------------- workload set-up
+def bench_workload(name: str, n_rounds: int):
+    wl = synth.workload(name)
+    return synth.scaled(wl, n_rounds=n_rounds)
+
+
+def host_rounds(wl, seed, n, ring):
+    """Tokens for n rounds and a ring of H tensors (open loop: inputs never depend on outputs)."""
+    toks, Hs = [], []
+    for r in range(n):
+        rng = np.random.default_rng([seed, 4, r])
+        m = synth.draw_accept(wl, rng)
+        draft, target = synth.make_tokens(wl, rng, m)
+        toks.append((draft, target, m))
+        if r < ring:
+            Hs.append(synth.make_hidden(wl, rng))
+    return toks, Hs
+
+
+# --------------------------------------------------------------------------- the CPU oracle leg
+def oracle_objects(wl, seed, weights, S_sample):
+    from oracle import cod_oracle as orc
+    sh = wl.shape
+    sub = synth.scaled(wl, S=S_sample)
+    lay = synth.make_layout(sub, seed)
+    cfg = orc.OracleConfig(d_target=sh.d_target, n_cap=sh.n_cap, d_model=sh.d_model, n_layers=sh.n_layers,
+                           n_q=sh.n_q, n_kv=sh.n_kv, hd=sh.hd, vocab=sh.vocab, mask_token_id=sh.mask_token_id,
+                           W=sh.W, page=sh.page, rope_theta=sh.rope_theta, rms_eps=sh.rms_eps,
+                           hidden_norm=sh.hidden_norm)
+    # compact page table: only the pages this sample can touch
+    L = lay["committed_len"]
+    per = (int(L.max()) + (sub.n_rounds + 2) * sh.W) // sh.page + 2
+    bt = np.arange(S_sample * per, dtype=np.int64).reshape(S_sample, per)
+    st = orc.OracleState(cfg, S_sample, S_sample * per, bt, L)
+    rng = np.random.default_rng([seed, 3])
+    for s in range(S_sample):
+        used = (int(L[s]) + sh.page - 1) // sh.page
+        st.pool[:, bt[s, :used]] = synth.to_storage(
+            rng.standard_normal((sh.n_layers, used, sh.n_kv, 2, sh.page, sh.hd), dtype=np.float32), sh.dtype)
+    return orc, sub, st, orc.prepare_weights(weights)
+
+
+def time_oracle(wl, seed, weights, n_rounds, S_sample, budget_s=None):
+    """Runs the oracle, as it stands, for n_rounds rounds of the first S_sample sequences."""
+    orc, sub, st, w64 = oracle_objects(wl, seed, weights, S_sample)
+    times = []
+    for r in range(n_rounds):
+        rd = synth.make_round(sub, seed, r)
+        t0 = time.perf_counter()
+        orc.draft_round(rd["draft"], rd["target"], rd["H"], st, w64, sub.n_forced, orc.MODE_CARRY)
+        times.append(time.perf_counter() - t0)
+        if budget_s is not None and sum(times) > budget_s and len(times) >= 1:
+            break
+    return times
+
+
+def cores_used():
+    try:
+        return len(os.sched_getaffinity(0))
+    except Exception:
+        return os.cpu_count() or 1
+
+
+def run_reference(args):
+    """--impl reference: the CPU oracle timed on the host cores (rank 0 only)."""
+    if int(os.environ.get("RANK", "0")) != 0:
+        return
+    wl = bench_workload(args.workload, args.steps + args.warmup + 1)
+    weights = synth.make_weights(wl.shape, args.seed)
+    S_sample = 1 if wl.S == 1 else 2
+    orc, sub, st, w64 = oracle_objects(wl, args.seed, weights, S_sample)
+    per_step = []
+    budget = 240.0
+    t_start = time.perf_counter()
+    done = 0
+    for r in range(args.warmup + args.steps):
+        rd = synth.make_round(sub, args.seed, r)
+        t0 = time.perf_counter()
+        orc.draft_round(rd["draft"], rd["target"], rd["H"], st, w64, sub.n_forced, orc.MODE_CARRY)
+        dt = time.perf_counter() - t0
+        if r >= args.warmup:
+            per_step.append(dt)
+            done += 1
+        if time.perf_counter() - t_start > budget and done >= 1:
+            break
+    mean = sum(per_step) / len(per_step)
+    # a step of the sample covers S_sample of the S sequences of a round
+    value = (S_sample / wl.S) / mean
+    sample = (f"{len(per_step)} whole rounds of {S_sample} of {wl.S} sequences at full shapes, float64 numpy; "
+              f"rounds/s scaled by {S_sample}/{wl.S}")
+    line = {
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+        "steps": len(per_step), "steps_requested": args.steps, "warmup": args.warmup,
+        "ms_per_step": 1e3 * mean * wl.S / S_sample, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": wl.name, "batch": wl.S, "block": wl.shape.W, "context": list(wl.ctx)},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": cores_used(), "kind": "oracle", "sample": sample},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+    }
+    print(json.dumps(line))
+
+
+# --------------------------------------------------------------------------- the GPU arm
+def run_gpu(args):
+    import torch
+    import torch.distributed as dist
+
+    import __graft_entry__ as entry
+    from paper_2609_14717_b200 import binding as B
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    torch.cuda.set_device(local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    if rank == 0:
+        entry.build()
+    if world > 1:
+        dist.barrier()
+
+    peaks = load_peaks()
+    K, Wm = args.steps, args.warmup
+    n_rounds = K + Wm
+    wl = bench_workload(args.workload, n_rounds + 1)
+    sh = wl.shape
+    seed = args.seed + rank
+    es = 2 if sh.dtype == "bf16" else 4
+
+    # ---- inputs: weights (host, seeded) -> device; layout; pool filled on the device
+    weights = synth.make_weights(sh, seed)
+    lay = synth.make_layout(wl, seed)
+    n_pages, mp = int(lay["n_pages"]), int(lay["max_pages_per_seq"])
+    cfg = B.make_config(sh, wl.S, mp, n_pages)
+    ctx = B.Context(cfg)
+    w_dev = B.weights_to_device(weights, sh.dtype)
+    ctx.set_weights(w_dev)
+    state = B.State(cfg, sh.dtype, wl.S, lay["block_table"], lay["committed_len"])
+    gen = torch.Generator(device="cuda").manual_seed(seed)
+    for l in range(sh.n_layers):
+        state.kv_pool[l].copy_(torch.randn(state.kv_pool[l].shape, generator=gen, device="cuda",
+                                           dtype=torch.float32).to(state.kv_pool.dtype))
+    ring = 8
+    toks, Hs = host_rounds(wl, seed, n_rounds, ring)
+    H_pin = [torch.from_numpy(h).to(B.torch_dtype(sh.dtype)).pin_memory() for h in Hs]
+    d_pin = [torch.from_numpy(t[0]).pin_memory() for t in toks]
+    t_pin = [torch.from_numpy(t[1]).pin_memory() for t in toks]
+    H_dev = [h.cuda() for h in H_pin]
+    d_dev = [d.cuda() for d in d_pin]
+    t_dev = [t.cuda() for t in t_pin]
+    next_draft = torch.zeros((wl.S, sh.W), dtype=torch.int32, device="cuda")
+    L0 = state.committed_len.clone()
+
+    def reset():
+        state.committed_len.copy_(L0)
+        state.carry_len.zero_()
+
+    def barrier():
+        torch.cuda.synchronize()
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    def timed_pass(mode, e2e=False, profile=(), K=K):
+        reset()
+        ctx.profile_enable(())
+        stage_H = torch.empty_like(H_dev[0])
+        stage_d = torch.empty_like(d_dev[0])
+        stage_t = torch.empty_like(t_dev[0])
+
+        def step(r):
+            if e2e:
+                stage_H.copy_(H_pin[r % ring], non_blocking=True)
+                stage_d.copy_(d_pin[r], non_blocking=True)
+                stage_t.copy_(t_pin[r], non_blocking=True)
+                ctx.draft_round(stage_d, stage_t, stage_H, wl.S, wl.n_forced, mode, state, None, next_draft, None)
+                return next_draft.cpu()
+            ctx.draft_round(d_dev[r], t_dev[r], H_dev[r % ring], wl.S, wl.n_forced, mode, state, None, next_draft, None)
+            return None
+
+        for r in range(Wm):
+            step(r)
+        barrier()
+        ctx.profile_enable(profile)
+        n0 = ctx.launch_count()
+        ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        ev0.record()
+        for r in range(Wm, Wm + K):
+            step(r)
+        ev1.record()
+        barrier()
+        ms = ev0.elapsed_time(ev1)
+        launches = ctx.launch_count() - n0
+        if world > 1:
+            t = torch.tensor([ms], device="cuda")
+            dist.all_reduce(t, op=dist.ReduceOp.MAX)
+            ms = float(t.item())
+        return ms, launches
+
+    # ---- which kernel dominates, by the byte/flop model at the measured peaks
+    L_run = lay["committed_len"].astype(np.int64).copy()
+    models = []
+    for r in range(n_rounds):
+        m = toks[r][2].astype(np.int64)
+        L_run = L_run + m
+        if r >= Wm:
+            models.append(round_model(wl, L_run, sh.W - m, wl.R, es))
+    mean_model = {k: (float(np.mean([mm[k][0] for mm in models])), float(np.mean([mm[k][1] for mm in models])))
+                  for k in models[0]}
+    t_class = {k: max(b / (peaks["hbm_gbs"] * 1e9), f / (peaks["tflops"] * 1e12)) for k, (b, f) in mean_model.items()}
+    dominant = max(t_class, key=t_class.get)
+
+    with ClockSampler(local) as clk:
+        ms, launches = timed_pass(B.COD_CARRY, profile=(dominant,))
+    dom_ms, dom_n = ctx.profile_read(dominant)
+    ms_base, _ = timed_pass(B.COD_BASELINE)
+    ms_e2e, _ = timed_pass(B.COD_CARRY, e2e=True)
+    K_prof = min(K, 32)                                     # bounded by the library's event slots
+    timed_pass(B.COD_CARRY, profile=B.KERNEL_CLASSES, K=K_prof)
+    per_class = {k: ctx.profile_read(k) for k in B.KERNEL_CLASSES}
+    status = ctx.poll_status()
+
+    if rank != 0:
+        if world > 1:
+            dist.destroy_process_group()
+        return
+
+    # ---- roofline of the dominant kernel and of the whole round
+    b_dom, f_dom = mean_model[dominant]
+    launches_per_round = max(dom_n // K, 1)
+    dur = dom_ms / max(dom_n, 1) * 1e-3                      # seconds per launch
+    b_launch, f_launch = b_dom / launches_per_round, f_dom / launches_per_round
+    hbm_bound = b_launch / (peaks["hbm_gbs"] * 1e9) >= f_launch / (peaks["tflops"] * 1e12)
+    if hbm_bound:
+        achieved, peak, unit, bound = b_launch / dur / 1e9, peaks["hbm_gbs"], "GB/s", "hbm"
+    else:
+        achieved, peak, unit, bound = f_launch / dur / 1e12, peaks["tflops"], "TFLOP/s", "tensor"
+    roofline = {"bound": bound, "kernel": dominant, "achieved": achieved, "peak": peak, "unit": unit,
+                "frac": achieved / peak, "traffic": NCU_TRAFFIC_BYTES.get(wl.name),
+                "peak_source": peaks["source"], "algorithmic_bytes_per_launch": b_launch,
+                "algorithmic_flops_per_launch": f_launch, "us_per_launch": dur * 1e6, "launches_timed": dom_n}
+    tot_b = sum(v[0] for v in mean_model.values())
+    tot_f = sum(v[1] for v in mean_model.values())
+    strict_s = max(tot_b / (peaks["hbm_gbs"] * 1e9), tot_f / (peaks["tflops_burst"] * 1e12))
+    serial_s = sum(max(b / (peaks["hbm_gbs"] * 1e9), f / (peaks["tflops_burst"] * 1e12)) for b, f in mean_model.values())
+    us_round = ms / K * 1e3
+    round_roofline = {"strict_us": strict_s * 1e6, "serial_us": serial_s * 1e6, "measured_us": us_round,
+                      "frac_of_strict": strict_s * 1e6 / us_round, "bytes": tot_b, "flops": tot_f}
+
+    # ---- the CPU oracle on a bounded sample (rank 0, N = 1 only)
+    cpu = None
+    if world == 1 and not args.no_cpu_baseline:
+        S_sample = 1 if wl.S == 1 else 2
+        times = time_oracle(wl, seed, weights, n_rounds=3, S_sample=S_sample, budget_s=25.0)
+        mean = sum(times) / len(times)
+        cpu = {"value": (S_sample / wl.S) / mean, "unit": UNIT, "cores": cores_used(), "kind": "oracle",
+               "sample": f"{len(times)} whole rounds of {S_sample} of {wl.S} sequences at full shapes "
+                         f"(float64 numpy, {mean:.2f} s each); rounds/s scaled by {S_sample}/{wl.S}"}
+
+    h2d = int(H_pin[0].numel() * H_pin[0].element_size() + d_pin[0].numel() * 4 + t_pin[0].numel() * 4)
+    line = {
+        "metric": METRIC, "value": world * K / (ms * 1e-3), "unit": UNIT, "n_gpus": world, "steps": K, "warmup": Wm,
+        "ms_per_step": ms / K, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": sh.dtype, "data": "synthetic",
+        "config": {"workload": wl.name, "batch": wl.S, "block": sh.W, "context": list(wl.ctx),
+                   "drafter_layers": sh.n_layers, "vocab": sh.vocab, "parallelism": f"replicas x{world}",
+                   "l2": "inputs larger than L2 (weights re-read every round)"},
+        "us_per_round": us_round, "seq_rounds_per_s": world * wl.S * K / (ms * 1e-3),
+        "carryover_overhead_pct": 100.0 * (ms - ms_base) / ms_base,
+        "baseline_us_per_round": ms_base / K * 1e3,
+        "roofline": roofline, "round_roofline": round_roofline,
+        "kernels_us_per_round": {k: v[0] / K_prof * 1e3 for k, v in per_class.items()},
+        "cpu_baseline": cpu,
+        "e2e": {"value": world * K / (ms_e2e * 1e-3), "unit": UNIT, "h2d_bytes_per_step": h2d,
+                "d2h_bytes_per_step": int(next_draft.numel() * 4)},
+        "gpu_launches": launches, "clocks": clk.summary(), "device_status": status,
+        "workspace_bytes": ctx.workspace_bytes(),
+    }
+    print(json.dumps(line))
+    ctx.close()
+    if world > 1:
+        dist.destroy_process_group()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=64)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="cfg2", choices=["cfg1", "cfg2", "cfg3", "cfg4", "cfg5"])
+    ap.add_argument("--seed", type=int, default=0)
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    if args.warmup < 3:
+        args.warmup = 3
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_gpu(args)
+
+
+if __name__ == "__main__":
+    main()

@@ -61,6 +61,7 @@ enum cod_mode {
 
 /* cod_config.flags */
 #define COD_F_HIDDEN_NORM 1u /* RMS-normalise (with gain g_hidden) the output of F */
+#define COD_F_NO_TENSOR_CORES 2u /* use the plain-FMA kernels only (an on-GPU cross-check) */
 
 /* bits of the sticky device status word */
 #define COD_DEV_BAD_TOKEN 1u      /* a token id outside [0, vocab) was met (treated as id 0) */
@@ -195,6 +196,28 @@ int cod_draft_round(cod_ctx* ctx, const int32_t* draft, const int32_t* target, c
 /* Copies the sticky device status word to *dev_flags (host) after synchronising the stream;
    clear != 0 also resets it. */
 int cod_poll_status(cod_ctx* ctx, uint32_t* dev_flags, int clear, cod_stream_t stream);
+
+/* Kernel classes for the optional per-kernel timing below. */
+enum cod_kernel_class {
+  COD_K_VERIFY = 0, /* verify-accept + position tables      */
+  COD_K_FC = 1,     /* contraction with F                   */
+  COD_K_KV = 2,     /* contraction with K_l, V_l (all l)    */
+  COD_K_QKV = 3,    /* Q/K/V of the block rows (per layer)  */
+  COD_K_ATTN = 4,   /* block attention (split + combine)    */
+  COD_K_OPROJ = 5,  /* output projection (per layer)        */
+  COD_K_LMHEAD = 6, /* LM head + argmax                     */
+  COD_K_ROWOPS = 7, /* norms, rotations, scatter, read-out  */
+  COD_K_CLASSES = 8
+};
+
+/* Measurement aid (the paper has no counterpart): while class_mask has bit (1 << k) set,
+   every launch of class k is bracketed by CUDA events on the launching stream (at most
+   4096 launches are recorded between two calls). class_mask = 0 switches it off.
+   Calling it also discards earlier records. */
+int cod_profile_enable(cod_ctx* ctx, uint32_t class_mask);
+/* Synchronises the recorded events and returns the summed duration and launch count of one
+   class since cod_profile_enable. total_ms, launches: host pointers. */
+int cod_profile_read(cod_ctx* ctx, int kernel_class, float* total_ms, int32_t* launches);
 
 /* Number of kernels this context has launched since creation (host-side counter). */
 int64_t cod_launch_count(const cod_ctx* ctx);

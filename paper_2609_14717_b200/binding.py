@@ -19,11 +19,14 @@ LIB_PATH = os.path.join(_HERE, "libcod.so")
 COD_F32, COD_BF16 = 0, 1
 COD_CARRY, COD_BASELINE = 0, 1
 COD_F_HIDDEN_NORM = 1
+COD_F_NO_TENSOR_CORES = 2
 DEV_BAD_TOKEN, DEV_PAGE_OVERFLOW, DEV_BAD_PAGE, DEV_TIMEOUT, DEV_BAD_LEN = 1, 2, 4, 8, 16
 
 EXPORTS = ("cod_create", "cod_destroy", "cod_set_weights", "cod_verify_accept", "cod_project_kv",
            "cod_scatter_kv", "cod_block_attn", "cod_lm_head_argmax", "cod_draft_round",
-           "cod_poll_status", "cod_launch_count", "cod_workspace_bytes", "cod_error_string")
+           "cod_poll_status", "cod_profile_enable", "cod_profile_read", "cod_launch_count",
+           "cod_workspace_bytes", "cod_error_string")
+KERNEL_CLASSES = ("verify", "fc", "kv", "qkv", "attn", "oproj", "lmhead", "rowops")
 
 
 class CodConfig(C.Structure):
@@ -73,6 +76,8 @@ def load_library() -> C.CDLL:
     lib.cod_draft_round.argtypes = [vp, vp, vp, vp, i32, i32, i32, C.POINTER(CodState), C.POINTER(CodSplit),
                                     vp, C.POINTER(CodTaps), vp]
     lib.cod_poll_status.argtypes = [vp, C.POINTER(C.c_uint32), i32, vp]
+    lib.cod_profile_enable.argtypes = [vp, C.c_uint32]
+    lib.cod_profile_read.argtypes = [vp, i32, C.POINTER(C.c_float), C.POINTER(C.c_int32)]
     lib.cod_launch_count.argtypes = [vp]
     lib.cod_launch_count.restype = i64
     lib.cod_workspace_bytes.argtypes = [vp]
@@ -249,6 +254,17 @@ class Context:
         _check("cod_poll_status", lib().cod_poll_status(self._h, C.byref(flags), int(clear), _stream()))
         return int(flags.value)
 
+    def profile_enable(self, classes=()) -> None:
+        mask = 0
+        for k in classes:
+            mask |= 1 << KERNEL_CLASSES.index(k)
+        _check("cod_profile_enable", lib().cod_profile_enable(self._h, mask))
+
+    def profile_read(self, klass: str):
+        ms, n = C.c_float(0), C.c_int32(0)
+        _check("cod_profile_read", lib().cod_profile_read(self._h, KERNEL_CLASSES.index(klass), C.byref(ms), C.byref(n)))
+        return float(ms.value), int(n.value)
+
     def launch_count(self) -> int:
         return int(lib().cod_launch_count(self._h))
 
@@ -256,14 +272,16 @@ class Context:
         return int(lib().cod_workspace_bytes(self._h))
 
 
-def make_config(sh, max_batch: int, max_pages_per_seq: int, n_pages: int, attn_split_len: int = 0) -> CodConfig:
+def make_config(sh, max_batch: int, max_pages_per_seq: int, n_pages: int, attn_split_len: int = 0,
+                no_tensor_cores: bool = False) -> CodConfig:
     """cod_config from a synthetic DrafterShape."""
     return CodConfig(
         d_target=sh.d_target, n_cap=sh.n_cap, d_model=sh.d_model, n_layers=sh.n_layers, n_q_heads=sh.n_q,
         n_kv_heads=sh.n_kv, head_dim=sh.hd, vocab=sh.vocab, mask_token_id=sh.mask_token_id, block=sh.W,
         page_size=sh.page, max_batch=max_batch, max_pages_per_seq=max_pages_per_seq, n_pages=n_pages,
         dtype=COD_BF16 if sh.dtype == "bf16" else COD_F32,
-        flags=COD_F_HIDDEN_NORM if sh.hidden_norm else 0, rope_theta=sh.rope_theta, rms_eps=sh.rms_eps,
+        flags=(COD_F_HIDDEN_NORM if sh.hidden_norm else 0) | (COD_F_NO_TENSOR_CORES if no_tensor_cores else 0),
+        rope_theta=sh.rope_theta, rms_eps=sh.rms_eps,
         attn_split_len=attn_split_len)
 
 

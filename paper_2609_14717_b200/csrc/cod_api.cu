@@ -40,6 +40,7 @@ size_t carve(cod_ctx* c) {
   widest = widest > static_cast<size_t>(c->qw + 2 * c->kvw) ? widest : static_cast<size_t>(c->qw + 2 * c->kvw);
   c->gemm_out_floats = static_cast<size_t>(COD_MAX_SPLITS) * R * widest;
   cv.take(c->gemm_out, sizeof(float) * c->gemm_out_floats);
+  cv.take(c->hc, es * R * c->D_in);
   cv.take(c->z, es * R * D);
   cv.take(c->x, sizeof(float) * R * D);
   cv.take(c->a, es * R * D);
@@ -75,18 +76,30 @@ bool state_has_null(const cod_state* s) {
 
 // split-K factor so that (feature tiles x splits) fills the machine; partial slabs must fit
 int pick_splits(const cod_ctx* c, int n_out, int K, int rows) {
-  (void)c; (void)n_out; (void)K; (void)rows;
-  return 1;
+  if (c->cfg.dtype != COD_BF16 || c->force_simt) return 1;
+  const int ctas = ((n_out + 127) / 128) * ((rows + 255) / 256);
+  const int kb = (K + 63) / 64;
+  int splits = c->n_sm / ctas;
+  if (splits > COD_MAX_SPLITS) splits = COD_MAX_SPLITS;
+  if (splits > kb / 4) splits = kb / 4;
+  if (splits < 1) splits = 1;
+  const int per = (kb + splits - 1) / splits;
+  return (kb + per - 1) / per;            // no empty split
 }
 
 int check_S(const cod_ctx* c, int S) { return (S >= 1 && S <= c->cfg.max_batch) ? COD_OK : COD_ERR_INVALID_ARG; }
 
 }  // namespace
 
-int cod_launch_gemm(cod_ctx* c, const GemmArgs& g, cudaStream_t st) { return cod_launch_gemm_simt(c, g, st); }
+int cod_launch_gemm(cod_ctx* c, const GemmArgs& g, cudaStream_t st) {
+  ProfScope prof(c, g.klass, st);
+  if (!c->force_simt && cod_gemm_tc_supported(c, g)) return cod_launch_gemm_tc(c, g, st);
+  return cod_launch_gemm_simt(c, g, st);
+}
 
 int cod_launch_attn(cod_ctx* c, int layer, const void* q, const void* kb, const void* vb, const cod_state* state,
                     int S, int use_carry, void* out, float* tap_out, float* carry_mass, cudaStream_t st) {
+  ProfScope prof(c, COD_K_ATTN, st);
   return cod_launch_attn_simt(c, layer, q, kb, vb, state, S, use_carry, out, tap_out, carry_mass, st);
 }
 
@@ -123,6 +136,8 @@ int cod_create(const cod_config* cfg, cod_ctx** out) {
   c->qw = f.n_q_heads * f.head_dim;
   c->R_max = f.max_batch * f.block;
   c->half = f.head_dim / 2;
+  c->force_simt = (f.flags & COD_F_NO_TENSOR_CORES) != 0;
+  if (cudaDeviceGetAttribute(&c->n_sm, cudaDevAttrMultiProcessorCount, c->device) != cudaSuccess || c->n_sm < 1) c->n_sm = 148;
   c->split_len = f.attn_split_len > 0 ? f.attn_split_len : 512;
   const int64_t max_keys = static_cast<int64_t>(f.max_pages_per_seq) * f.page_size + 2 * f.block;
   c->max_splits = static_cast<int>((max_keys + c->split_len - 1) / c->split_len);
@@ -145,7 +160,11 @@ int cod_create(const cod_config* cfg, cod_ctx** out) {
   }
   free(fr);
   free(frf);
-  if (!ok) { cudaFree(c->ws); cudaGetLastError(); delete c; return COD_ERR_CUDA; }
+  c->prof_ev = static_cast<cudaEvent_t*>(calloc(2 * COD_PROF_SLOTS, sizeof(cudaEvent_t)));
+  c->prof_class = static_cast<unsigned char*>(calloc(COD_PROF_SLOTS, 1));
+  if (!c->prof_ev || !c->prof_class) ok = false;
+  for (int i = 0; ok && i < 2 * COD_PROF_SLOTS; ++i) ok = cudaEventCreate(&c->prof_ev[i]) == cudaSuccess;
+  if (!ok) { cudaFree(c->ws); cudaGetLastError(); free(c->prof_ev); free(c->prof_class); delete c; return COD_ERR_CUDA; }
   *out = c;
   return COD_OK;
 }
@@ -154,6 +173,9 @@ int cod_destroy(cod_ctx* c) {
   if (!c) return COD_ERR_INVALID_ARG;
   cudaDeviceSynchronize();
   cudaFree(c->ws);
+  for (int i = 0; i < 2 * COD_PROF_SLOTS; ++i) cudaEventDestroy(c->prof_ev[i]);
+  free(c->prof_ev);
+  free(c->prof_class);
   delete c;
   return COD_OK;
 }
@@ -185,22 +207,26 @@ static int project_impl(cod_ctx* c, const void* H, const cod_split* sp, int S, i
   const int* n_dev = mode == COD_BASELINE ? sp->acc_off + S : nullptr;
   int rc;
 
+  if (a_rows) {   // baseline: pack the accepted rows, then the same dense kernels on fewer rows
+    if ((rc = cod_launch_gather_rows(c, H, a_rows, n_dev, R, c->D_in, c->hc, st)) != COD_OK) return rc;
+    H = c->hc;
+  }
   GemmArgs g{};
-  g.A = H; g.lda = c->D_in; g.a_rows = a_rows; g.n_rows_dev = n_dev; g.n_rows = R; g.K = c->D_in;
-  g.seg[0] = {c->w.fc, c->D}; g.n_seg = 1;
+  g.A = H; g.lda = c->D_in; g.a_rows = nullptr; g.n_rows_dev = n_dev; g.n_rows = R; g.K = c->D_in;
+  g.seg[0] = {c->w.fc, c->D}; g.n_seg = 1; g.klass = COD_K_FC;
   g.C = c->gemm_out; g.ldc = c->D; g.splits = pick_splits(c, c->D, c->D_in, R);
   if ((rc = cod_launch_gemm(c, g, st)) != COD_OK) return rc;
   if ((rc = cod_launch_fc_finish(c, c->gemm_out, g.splits, R, n_dev, a_rows, sp->carry_slot, tap_z, st)) != COD_OK)
     return rc;
 
   GemmArgs k{};
-  k.A = c->z; k.lda = c->D; k.a_rows = a_rows; k.n_rows_dev = n_dev; k.n_rows = R; k.K = c->D;
+  k.A = c->z; k.lda = c->D; k.a_rows = nullptr; k.n_rows_dev = n_dev; k.n_rows = R; k.K = c->D;
   k.seg[0] = {c->w.wk, f.n_layers * c->kvw};
   k.seg[1] = {c->w.wv, f.n_layers * c->kvw};
-  k.n_seg = 2;
-  k.C = c->gemm_out; k.ldc = 2 * f.n_layers * c->kvw; k.splits = 1;
+  k.n_seg = 2; k.klass = COD_K_KV;
+  k.C = c->gemm_out; k.ldc = 2 * f.n_layers * c->kvw; k.splits = pick_splits(c, k.ldc, c->D, R);
   if ((rc = cod_launch_gemm(c, k, st)) != COD_OK) return rc;
-  return cod_launch_kv_finish(c, c->gemm_out, 1, R, n_dev, a_rows, sp, J, dest, R, st);
+  return cod_launch_kv_finish(c, c->gemm_out, k.splits, R, n_dev, a_rows, sp, J, dest, R, st);
 }
 
 int cod_project_kv(cod_ctx* c, const void* H, const cod_split* split, int S, int mode, void* J,
@@ -242,7 +268,7 @@ static int lm_head_impl(cod_ctx* c, int n_rows, cudaStream_t st) {
   GemmArgs g{};
   g.A = c->a; g.lda = c->D; g.n_rows = n_rows; g.K = c->D;
   g.seg[0] = {c->w.emb, c->cfg.vocab}; g.n_seg = 1;
-  g.splits = 1; g.amax = c->amax;
+  g.splits = 1; g.amax = c->amax; g.klass = COD_K_LMHEAD;
   return cod_launch_gemm(c, g, st);
 }
 
@@ -287,7 +313,7 @@ int cod_draft_round(cod_ctx* c, const int32_t* draft, const int32_t* target, con
     g.seg[0] = {static_cast<const char*>(c->w.wq) + es * l * c->qw * c->D, c->qw};
     g.seg[1] = {static_cast<const char*>(c->w.wk) + es * l * c->kvw * c->D, c->kvw};
     g.seg[2] = {static_cast<const char*>(c->w.wv) + es * l * c->kvw * c->D, c->kvw};
-    g.n_seg = 3;
+    g.n_seg = 3; g.klass = COD_K_QKV;
     g.C = c->gemm_out; g.ldc = c->qw + 2 * c->kvw; g.splits = pick_splits(c, g.ldc, c->D, R);
     if ((rc = cod_launch_gemm(c, g, s)) != COD_OK) return rc;
     if ((rc = cod_launch_qkv_finish(c, c->gemm_out, g.splits, R, s)) != COD_OK) return rc;
@@ -299,7 +325,7 @@ int cod_draft_round(cod_ctx* c, const int32_t* draft, const int32_t* target, con
     GemmArgs o{};
     o.A = c->o; o.lda = c->qw; o.n_rows = R; o.K = c->qw;
     o.seg[0] = {static_cast<const char*>(c->w.wo) + es * l * c->D * c->qw, c->D};
-    o.n_seg = 1;
+    o.n_seg = 1; o.klass = COD_K_OPROJ;
     o.C = c->gemm_out; o.ldc = c->D; o.splits = pick_splits(c, c->D, c->qw, R);
     if ((rc = cod_launch_gemm(c, o, s)) != COD_OK) return rc;
     const bool last = l + 1 == f.n_layers;
@@ -319,6 +345,30 @@ int cod_poll_status(cod_ctx* c, uint32_t* dev_flags, int clear, cod_stream_t str
   if (cudaMemcpyAsync(dev_flags, c->status, sizeof(uint32_t), cudaMemcpyDeviceToHost, s) != cudaSuccess) return COD_ERR_CUDA;
   if (clear && cudaMemsetAsync(c->status, 0, sizeof(uint32_t), s) != cudaSuccess) return COD_ERR_CUDA;
   if (cudaStreamSynchronize(s) != cudaSuccess) return COD_ERR_CUDA;
+  return COD_OK;
+}
+
+int cod_profile_enable(cod_ctx* c, uint32_t class_mask) {
+  if (!c) return COD_ERR_INVALID_ARG;
+  c->prof_mask = class_mask & ((1u << COD_K_CLASSES) - 1u);
+  c->prof_n = 0;
+  return COD_OK;
+}
+
+int cod_profile_read(cod_ctx* c, int kernel_class, float* total_ms, int32_t* launches) {
+  if (!c || !total_ms || !launches || kernel_class < 0 || kernel_class >= COD_K_CLASSES) return COD_ERR_INVALID_ARG;
+  float tot = 0.f;
+  int n = 0;
+  for (int i = 0; i < c->prof_n; ++i) {
+    if (c->prof_class[i] != kernel_class) continue;
+    if (cudaEventSynchronize(c->prof_ev[2 * i + 1]) != cudaSuccess) return COD_ERR_CUDA;
+    float ms = 0.f;
+    if (cudaEventElapsedTime(&ms, c->prof_ev[2 * i], c->prof_ev[2 * i + 1]) != cudaSuccess) return COD_ERR_CUDA;
+    tot += ms;
+    ++n;
+  }
+  *total_ms = tot;
+  *launches = n;
   return COD_OK;
 }
 

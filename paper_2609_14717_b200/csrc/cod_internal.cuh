@@ -87,7 +87,10 @@ struct GemmArgs {
   int ldc;
   int splits;             // split-K factor (1 = none)
   unsigned long long* amax;  // if non-null: per-row packed argmax over N instead of storing C
+  int klass;              // cod_kernel_class, for the optional timing
 };
+
+#define COD_PROF_SLOTS 4096
 
 struct cod_ctx {
   cod_config cfg;
@@ -96,6 +99,8 @@ struct cod_ctx {
   int device;
   int D, D_in, kvw, qw, R_max, half;
   int split_len, max_splits;   // attention split-KV
+  int n_sm;
+  bool force_simt;             // COD_F_NO_TENSOR_CORES: plain-FMA kernels only
   int64_t launches;
   size_t ws_bytes;
   char* ws;
@@ -108,6 +113,7 @@ struct cod_ctx {
   float* rope_blk;             // [R_max][hd]  cos | sin of the block rows' positions
   float* gemm_out;             // split-K / unfused GEMM results
   size_t gemm_out_floats;
+  void* hc;                    // [R_max, D_in] accepted rows of H packed densely (baseline mode)
   void* z;                     // [R_max, D]
   float* x;                    // [R_max, D]   residual stream
   void* a;                     // [R_max, D]   normalised activations
@@ -120,6 +126,26 @@ struct cod_ctx {
   unsigned long long* amax;    // [R_max]
   int32_t* tok;                // [R_max]
   cod_split sp;                // internal split arrays (used when the caller passes none)
+  // optional per-kernel timing
+  uint32_t prof_mask;
+  int prof_n;
+  cudaEvent_t* prof_ev;        // [2 * COD_PROF_SLOTS], created at cod_create
+  unsigned char* prof_class;   // [COD_PROF_SLOTS]
+};
+
+// Brackets the launches made inside its scope with two events when the class is being timed.
+struct ProfScope {
+  cod_ctx* c; cudaStream_t st; int slot;
+  ProfScope(cod_ctx* c_, int klass, cudaStream_t st_) : c(c_), st(st_), slot(-1) {
+    if ((c->prof_mask >> klass) & 1u) {
+      if (c->prof_n < COD_PROF_SLOTS) {
+        slot = c->prof_n++;
+        c->prof_class[slot] = static_cast<unsigned char>(klass);
+        cudaEventRecord(c->prof_ev[2 * slot], st);
+      }
+    }
+  }
+  ~ProfScope() { if (slot >= 0) cudaEventRecord(c->prof_ev[2 * slot + 1], st); }
 };
 
 // ---------------------------------------------------------------------------- launchers
@@ -128,12 +154,16 @@ int cod_launch_verify(cod_ctx* c, const int32_t* draft, const int32_t* target, i
                       const cod_state* state, const cod_split* out, cudaStream_t st);
 int cod_launch_gemm(cod_ctx* c, const GemmArgs& g, cudaStream_t st);
 int cod_launch_gemm_simt(cod_ctx* c, const GemmArgs& g, cudaStream_t st);
+bool cod_gemm_tc_supported(const cod_ctx* c, const GemmArgs& g);
+int cod_launch_gemm_tc(cod_ctx* c, const GemmArgs& g, cudaStream_t st);
 int cod_launch_attn_simt(cod_ctx* c, int layer, const void* q, const void* kb, const void* vb,
                          const cod_state* stt, int S, int use_carry, void* out, float* tap, float* mass,
                          cudaStream_t st);
 // cos/sin tables of the block rows only, at positions committed_len[s] + i
 int cod_launch_rope_blk_only(cod_ctx* c, const int32_t* committed_len, int S, cudaStream_t st);
 int cod_launch_fcE(cod_ctx* c, cudaStream_t st);
+int cod_launch_gather_rows(cod_ctx* c, const void* src, const int* rows, const int* n_dev, int n_max, int width,
+                           void* dst, cudaStream_t st);
 int cod_launch_fc_finish(cod_ctx* c, const float* part, int splits, int n_rows, const int* n_rows_dev,
                          const int* a_rows, const int* carry_slot, float* tap_z, cudaStream_t st);
 // dest_state == nullptr: write J; else write the pool / carry slot directly

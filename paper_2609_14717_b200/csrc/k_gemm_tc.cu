@@ -1,0 +1,390 @@
+// Weight-streaming GEMM on the 5th-generation tensor cores (tcgen05), bf16 in / float out:
+//   C[i, n] = sum_k A[i, k] * B[n, k]     A: activations [rows, K], B: weights [N, K].
+//
+// The operands are swapped for the MMA: the 128 weight rows of a tile are the MMA's M
+// dimension and the (few) activation rows its N dimension (16..256), so a round with 16
+// token rows wastes no tensor work and every CTA streams a disjoint slab of the weight
+// matrix exactly once. Both tiles are staged K-major by TMA with the 128-byte swizzle into
+// a multi-stage shared-memory ring; one elected thread issues tcgen05.mma, the accumulator
+// lives in tensor memory (one lane per weight row, one column per token) and is read back
+// with tcgen05.ld by four epilogue warps.
+//
+//   warp 0-3  epilogue (TMEM lanes 32*w .. 32*w+31)     warp 4  TMA producer     warp 5  MMA issuer
+//
+// Epilogues: float partial sums (split-K slabs, reduced by the row-wise kernels), or a fused
+// per-token argmax over the weight rows for the LM head (logits are never stored).
+// Every mbarrier wait is bounded: on expiry the CTA raises COD_DEV_TIMEOUT and leaves cleanly.
+#include <cuda.h>
+
+#include "cod_internal.cuh"
+
+namespace {
+
+constexpr int BM = 128;       // weight rows per CTA (MMA M)
+constexpr int BK = 64;        // K elements per stage = one 128-byte swizzled row of bf16
+constexpr int UK = 16;        // K elements per tcgen05.mma (kind::f16)
+constexpr int NTHREADS = 192;
+constexpr uint32_t A_TILE_BYTES = BM * BK * 2;   // 16 KB
+constexpr unsigned long long WAIT_LIMIT_NS = 2000000000ull;
+
+struct TcParams {
+  int K;
+  int kb_total, kb_per_split;
+  int n_rows;                 // rows (upper bound when n_rows_dev is set)
+  const int* n_rows_dev;
+  int NT;                     // token rows per CTA = MMA N (multiple of 16, <= 256)
+  int tmem_cols;              // power of two >= max(32, NT)
+  int stages;
+  int seg_tile_end[3];        // cumulative count of 128-row tiles after each weight segment
+  int seg_N[3];
+  int n_seg;
+  float* C;
+  int ldc;
+  unsigned long long* amax;
+  uint32_t* status;
+};
+
+// ------------------------------------------------------------------ PTX wrappers
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return static_cast<uint32_t>(__cvta_generic_to_shared(p)); }
+
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count));
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+  return ok != 0;
+}
+__device__ __forceinline__ unsigned long long global_ns() {
+  unsigned long long t;
+  asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
+  return t;
+}
+// Bounded wait: false if the limit expired or another role already gave up.
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, uint32_t* status) {
+  const unsigned long long t0 = global_ns();
+  for (;;) {
+#pragma unroll 1
+    for (int i = 0; i < 256; ++i)
+      if (mbar_try_wait(bar, parity)) return true;
+    if (*abort_flag) return false;
+    if (global_ns() - t0 > WAIT_LIMIT_NS) {
+      *abort_flag = 1;
+      atomicOr(status, COD_DEV_TIMEOUT);
+      return false;
+    }
+  }
+}
+
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, int c0, int c1, uint32_t bar) {
+  asm volatile(
+      "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
+      ::"r"(dst), "l"(reinterpret_cast<uint64_t>(map)), "r"(c0), "r"(c1), "r"(bar) : "memory");
+}
+
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+
+__device__ __forceinline__ void tmem_alloc(uint32_t dst_smem, uint32_t cols) {
+  asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(dst_smem), "r"(cols) : "memory");
+  asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void tmem_dealloc(uint32_t taddr, uint32_t cols) {
+  asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(cols) : "memory");
+}
+
+// D[tmem] (+)= A[smem] * B[smem]^T, bf16 operands, float accumulator
+__device__ __forceinline__ void umma_bf16(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, uint32_t accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+      ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate) : "memory");
+}
+// the mbarrier is arrived on once all MMAs issued so far by this thread have completed
+__device__ __forceinline__ void umma_commit(uint32_t bar) {
+  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+
+__device__ __forceinline__ void tmem_ld16(uint32_t taddr, uint32_t (&v)[16]) {
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15}, [%16];"
+      : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]),
+        "=r"(v[8]), "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15])
+      : "r"(taddr) : "memory");
+  asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+}
+
+// Shared-memory operand descriptor: K-major tile whose rows are 128 bytes (64 bf16), 128-byte
+// swizzle, groups of 8 rows 1024 bytes apart; descriptor version 1 (Blackwell).
+__device__ __forceinline__ uint64_t smem_desc_sw128(uint32_t saddr) {
+  uint64_t d = 0;
+  d |= static_cast<uint64_t>((saddr & 0x3FFFFu) >> 4);          // start address            bits [0,14)
+  d |= static_cast<uint64_t>(1) << 16;                          // leading byte offset (unused for swizzled K-major)
+  d |= static_cast<uint64_t>(1024 >> 4) << 32;                  // stride byte offset        bits [32,46)
+  d |= static_cast<uint64_t>(1) << 46;                          // version                   bits [46,48)
+  d |= static_cast<uint64_t>(2) << 61;                          // layout: 128-byte swizzle  bits [61,64)
+  return d;
+}
+// Instruction descriptor: bf16 x bf16 -> float, both operands K-major, M = 128, N = n.
+__device__ __forceinline__ uint32_t instr_desc(int n) {
+  uint32_t d = 0;
+  d |= 1u << 4;                                  // accumulator format: float
+  d |= 1u << 7;                                  // A format: bf16
+  d |= 1u << 10;                                 // B format: bf16
+  d |= static_cast<uint32_t>(n >> 3) << 17;      // N / 8
+  d |= static_cast<uint32_t>(BM >> 4) << 24;     // M / 16
+  return d;
+}
+
+__device__ __forceinline__ unsigned order_key(float v) {
+  const unsigned u = __float_as_uint(v);
+  return (u & 0x80000000u) ? ~u : (u | 0x80000000u);
+}
+
+__global__ void __launch_bounds__(NTHREADS, 1)
+k_gemm_tc(const __grid_constant__ CUtensorMap map_w0, const __grid_constant__ CUtensorMap map_w1,
+          const __grid_constant__ CUtensorMap map_w2, const __grid_constant__ CUtensorMap map_a, const TcParams p) {
+  extern __shared__ uint8_t smem_raw[];
+  // tiles need 1024-byte alignment for the 128-byte swizzle pattern
+  const uint32_t raw = smem_u32(smem_raw);
+  const uint32_t base = (raw + 1023u) & ~1023u;
+  uint8_t* sm = smem_raw + (base - raw);
+  const uint32_t b_tile_bytes = static_cast<uint32_t>(p.NT) * BK * 2;
+  const uint32_t stage_bytes = A_TILE_BYTES + b_tile_bytes;
+  uint8_t* ctl = sm + static_cast<size_t>(p.stages) * stage_bytes;     // barriers and small state
+  uint64_t* full_bar = reinterpret_cast<uint64_t*>(ctl);               // [stages]
+  uint64_t* empty_bar = full_bar + 16;                                 // [stages]
+  uint64_t* acc_bar = full_bar + 32;                                   // accumulator ready
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(full_bar + 33);
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+  unsigned long long* red = reinterpret_cast<unsigned long long*>(full_bar + 34);   // [NT] argmax keys
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int n_tile = blockIdx.x, m_tile = blockIdx.y, split = blockIdx.z;
+  const int n_rows = p.n_rows_dev ? min(*p.n_rows_dev, p.n_rows) : p.n_rows;
+  const int i0 = n_tile * p.NT;
+  if (i0 >= n_rows) return;                       // whole CTA: no token rows here
+
+  // weight segment of this tile
+  int sidx = 0;
+  while (sidx < p.n_seg - 1 && m_tile >= p.seg_tile_end[sidx]) ++sidx;
+  const int tile_in_seg = m_tile - (sidx ? p.seg_tile_end[sidx - 1] : 0);
+  const int f0 = tile_in_seg * BM;                // first weight row within the segment
+  int col0 = f0;                                  // first output column
+  for (int s = 0; s < sidx; ++s) col0 += p.seg_N[s];
+  const int seg_N = p.seg_N[sidx];
+  const CUtensorMap* map_w = sidx == 0 ? &map_w0 : (sidx == 1 ? &map_w1 : &map_w2);
+
+  const int kb0 = split * p.kb_per_split, kb1 = min(p.kb_total, kb0 + p.kb_per_split);
+  const int n_kb = kb1 - kb0;
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < p.stages; ++s) { mbar_init(smem_u32(full_bar + s), 1); mbar_init(smem_u32(empty_bar + s), 1); }
+    mbar_init(smem_u32(acc_bar), 1);
+    *abort_flag = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  for (int t = threadIdx.x; t < p.NT; t += NTHREADS) red[t] = 0ull;
+  if (warp == 5) tmem_alloc(smem_u32(tmem_slot), static_cast<uint32_t>(p.tmem_cols));
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = *tmem_slot;
+
+  if (warp == 4) {
+    // ------------------------------------------------ TMA producer
+    if (lane == 0) {
+      for (int it = 0; it < n_kb; ++it) {
+        const int s = it % p.stages, use = it / p.stages;
+        if (use > 0 && !mbar_wait(smem_u32(empty_bar + s), (use - 1) & 1, abort_flag, p.status)) break;
+        const uint32_t fb = smem_u32(full_bar + s);
+        mbar_expect_tx(fb, stage_bytes);
+        const uint32_t a_dst = base + s * stage_bytes;
+        const int k = (kb0 + it) * BK;
+        tma_load_2d(a_dst, map_w, k, f0, fb);
+        tma_load_2d(a_dst + A_TILE_BYTES, &map_a, k, i0, fb);
+      }
+    }
+  } else if (warp == 5) {
+    // ------------------------------------------------ MMA issuer
+    if (lane == 0) {
+      const uint32_t idesc = instr_desc(p.NT);
+      bool ok = true;
+      for (int it = 0; it < n_kb && ok; ++it) {
+        const int s = it % p.stages, use = it / p.stages;
+        ok = mbar_wait(smem_u32(full_bar + s), use & 1, abort_flag, p.status);
+        if (!ok) break;
+        tc_fence_after();
+        const uint32_t a_addr = base + s * stage_bytes;
+        const uint64_t a_desc = smem_desc_sw128(a_addr), b_desc = smem_desc_sw128(a_addr + A_TILE_BYTES);
+#pragma unroll
+        for (int k = 0; k < BK / UK; ++k)       // advance 32 bytes (16 bf16) along K inside the swizzled row
+          umma_bf16(tmem_base, a_desc + (k * UK * 2 >> 4), b_desc + (k * UK * 2 >> 4), idesc, (it | k) ? 1u : 0u);
+        umma_commit(smem_u32(empty_bar + s));   // frees the stage when these MMAs retire
+      }
+      if (ok) umma_commit(smem_u32(acc_bar));
+    }
+  } else {
+    // ------------------------------------------------ epilogue warps 0..3
+    const bool ok = mbar_wait(smem_u32(acc_bar), 0, abort_flag, p.status);
+    tc_fence_after();
+    const int f = f0 + warp * 32 + lane;                    // weight row within the segment
+    const bool f_ok = f < seg_N;
+    const uint32_t t_lane = tmem_base + (static_cast<uint32_t>(warp * 32) << 16);
+    if (ok && p.amax == nullptr) {
+      float* C = p.C + static_cast<size_t>(split) * p.n_rows * p.ldc;
+      for (int c = 0; c < p.NT; c += 16) {
+        uint32_t v[16];
+        tmem_ld16(t_lane + c, v);
+#pragma unroll
+        for (int j = 0; j < 16; ++j) {
+          const int i = i0 + c + j;
+          if (f_ok && i < n_rows) C[static_cast<size_t>(i) * p.ldc + col0 + warp * 32 + lane] = __uint_as_float(v[j]);
+        }
+      }
+    } else if (ok) {
+      for (int c = 0; c < p.NT; c += 16) {
+        uint32_t v[16];
+        tmem_ld16(t_lane + c, v);
+#pragma unroll
+        for (int j = 0; j < 16; ++j) {
+          const unsigned u = f_ok ? order_key(__uint_as_float(v[j])) : 0u;
+          const unsigned mx = __reduce_max_sync(0xffffffffu, u);
+          const unsigned who = __ballot_sync(0xffffffffu, u == mx);
+          if (lane == 0) {
+            const int idx = col0 + warp * 32 + (__ffs(who) - 1);      // lowest weight row among equals
+            atomicMax(red + c + j, (static_cast<unsigned long long>(mx) << 32) |
+                                       static_cast<unsigned long long>(0xFFFFFFFFu - static_cast<unsigned>(idx)));
+          }
+        }
+      }
+    }
+  }
+
+  // ---------------------------------------------------- teardown
+  tc_fence_before();
+  __syncthreads();
+  if (*abort_flag) {
+    // give copies that may still be in flight time to land before the shared memory is released
+    for (int i = 0; i < 64; ++i) __nanosleep(1000);
+    __syncthreads();
+  }
+  else if (p.amax != nullptr) {
+    // the four epilogue warps merged their per-token keys in shared memory: one atomic per token
+    for (int t = threadIdx.x; t < p.NT; t += NTHREADS)
+      if (i0 + t < n_rows) atomicMax(p.amax + i0 + t, red[t]);
+  }
+  if (warp == 5) {
+    __syncwarp();
+    tc_fence_after();
+    tmem_dealloc(tmem_base, static_cast<uint32_t>(p.tmem_cols));
+  }
+}
+
+// ------------------------------------------------------------------ host side
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn encode_fn() {
+  static EncodeTiledFn fn = nullptr;
+  static bool tried = false;
+  if (!tried) {
+    tried = true;
+    void* p = nullptr;
+    cudaDriverEntryPointQueryResult q;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) == cudaSuccess &&
+        q == cudaDriverEntryPointSuccess)
+      fn = reinterpret_cast<EncodeTiledFn>(p);
+  }
+  return fn;
+}
+
+// bf16 matrix [rows, K] with row stride ld (elements); box = box_rows x 64 columns, 128-byte swizzle
+bool make_map(CUtensorMap* m, const void* ptr, uint64_t rows, uint64_t K, uint64_t ld, uint32_t box_rows) {
+  EncodeTiledFn fn = encode_fn();
+  if (!fn) return false;
+  cuuint64_t gdim[2] = {K, rows};
+  cuuint64_t gstride[1] = {ld * 2};
+  cuuint32_t box[2] = {static_cast<cuuint32_t>(BK), box_rows};
+  cuuint32_t estr[2] = {1, 1};
+  return fn(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(ptr), gdim, gstride, box, estr,
+            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+}  // namespace
+
+bool cod_gemm_tc_supported(const cod_ctx* c, const GemmArgs& g) {
+  if (c->cfg.dtype != COD_BF16 || g.a_rows != nullptr) return false;
+  if (g.K % 8 || g.lda % 8 || g.n_rows < 1) return false;
+  if ((reinterpret_cast<uintptr_t>(g.A) & 15u) != 0) return false;
+  for (int i = 0; i < g.n_seg; ++i) {
+    if ((reinterpret_cast<uintptr_t>(g.seg[i].B) & 15u) != 0) return false;
+    if (i + 1 < g.n_seg && g.seg[i].N % BM) return false;     // a tile must not straddle two matrices
+  }
+  return encode_fn() != nullptr;
+}
+
+int cod_launch_gemm_tc(cod_ctx* c, const GemmArgs& g, cudaStream_t st) {
+  TcParams p{};
+  p.K = g.K;
+  p.kb_total = (g.K + BK - 1) / BK;
+  int splits = g.splits < 1 ? 1 : g.splits;
+  p.kb_per_split = (p.kb_total + splits - 1) / splits;
+  splits = (p.kb_total + p.kb_per_split - 1) / p.kb_per_split;     // no empty split
+  if (splits != g.splits) return COD_ERR_INVALID_ARG;               // the caller sized the partial slabs
+  p.n_rows = g.n_rows;
+  p.n_rows_dev = g.n_rows_dev;
+  const int r16 = (g.n_rows + 15) / 16 * 16;
+  p.NT = r16 < 256 ? r16 : 256;
+  int cols = 32;
+  while (cols < p.NT) cols <<= 1;
+  p.tmem_cols = cols;
+  const uint32_t stage_bytes = A_TILE_BYTES + static_cast<uint32_t>(p.NT) * BK * 2;
+  int stages = static_cast<int>((200u * 1024u) / stage_bytes);
+  if (stages > 8) stages = 8;
+  if (p.NT <= 32 && stages > 5) stages = 5;      // small tiles: leave room for two CTAs per SM
+  if (stages > p.kb_per_split) stages = p.kb_per_split;
+  if (stages < 1) stages = 1;
+  p.stages = stages;
+  int tiles = 0;
+  for (int i = 0; i < 3; ++i) {
+    if (i < g.n_seg) {
+      tiles += (g.seg[i].N + BM - 1) / BM;
+      p.seg_N[i] = g.seg[i].N;
+    }
+    p.seg_tile_end[i] = tiles;
+  }
+  p.n_seg = g.n_seg;
+  p.C = g.C;
+  p.ldc = g.ldc;
+  p.amax = g.amax;
+  p.status = c->status;
+
+  CUtensorMap mw[3], ma;
+  for (int i = 0; i < 3; ++i) {
+    const int j = i < g.n_seg ? i : 0;
+    if (!make_map(&mw[i], g.seg[j].B, g.seg[j].N, g.K, g.K, BM)) return COD_ERR_CUDA;
+  }
+  if (!make_map(&ma, g.A, g.n_rows, g.K, g.lda, p.NT)) return COD_ERR_CUDA;
+
+  const size_t smem = static_cast<size_t>(stages) * stage_bytes + 1024 /* alignment slack */ + 34 * 8 + 4 * p.NT * 8;
+  static size_t configured = 0;
+  if (smem > configured) {
+    if (cudaFuncSetAttribute(k_gemm_tc, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem)) != cudaSuccess)
+      return COD_ERR_CUDA;
+    configured = smem;
+  }
+  dim3 grid((g.n_rows + p.NT - 1) / p.NT, tiles, splits);
+  k_gemm_tc<<<grid, NTHREADS, smem, st>>>(mw[0], mw[1], mw[2], ma, p);
+  COD_CHECK_LAUNCH(c);
+  return COD_OK;
+}

@@ -21,13 +21,28 @@ __global__ void k_fcE(const T* __restrict__ fc, const T* __restrict__ e, int D_i
   if (threadIdx.x == 0) out[n] = acc;
 }
 
+// ------------------------------------------------------------------ row compaction (baseline mode)
+// dst[i] = src[rows[i]] for i < *n_dev: the accepted rows of H packed densely, so the baseline
+// column of Algorithm 1 ("collect accepted states") runs the same dense contractions on fewer rows.
+template <typename T>
+__global__ void k_gather_rows(const T* __restrict__ src, const int* __restrict__ rows, const int* __restrict__ n_dev,
+                              int width, T* __restrict__ dst) {
+  const int i = blockIdx.x;
+  if (i >= *n_dev) return;
+  const int row = rows[i];
+  constexpr int VEC = 16 / sizeof(T);
+  const uint4* s4 = reinterpret_cast<const uint4*>(src + static_cast<size_t>(row) * width);
+  uint4* d4 = reinterpret_cast<uint4*>(dst + static_cast<size_t>(i) * width);
+  for (int e = threadIdx.x; e < width / VEC; e += blockDim.x) d4[e] = s4[e];
+}
+
 // ------------------------------------------------------------------ fc finish
 // z[row] = N_h( sum_splits part[i] + [row rejected] F(E_carry) )   (one block per kept row)
 template <typename T>
 __global__ void k_fc_finish(const float* __restrict__ part, int splits, int n_rows, const int* n_rows_dev,
                             const int* __restrict__ a_rows, const int* __restrict__ carry_slot,
                             const float* __restrict__ fcE, const T* __restrict__ gain, int D, float eps,
-                            int do_norm, T* __restrict__ z, float* __restrict__ tap) {
+                            int do_norm, T* __restrict__ z, int z_compact, float* __restrict__ tap) {
   extern __shared__ float sh[];   // [D] values + 33 reduction slots
   float* vals = sh;
   float* red = sh + D;
@@ -47,7 +62,7 @@ __global__ void k_fc_finish(const float* __restrict__ part, int splits, int n_ro
   const float scale = do_norm ? rsqrtf(ss / static_cast<float>(D) + eps) : 1.f;
   for (int d = threadIdx.x; d < D; d += blockDim.x) {
     const float v = do_norm ? vals[d] * scale * cod_ld(gain + d) : vals[d];
-    cod_st(z + static_cast<size_t>(row) * D + d, v);
+    cod_st(z + static_cast<size_t>(z_compact ? i : row) * D + d, v);
     if (tap) tap[static_cast<size_t>(row) * D + d] = v;
   }
 }
@@ -273,7 +288,19 @@ __global__ void k_finalize(const unsigned long long* __restrict__ amax, int R, i
     if ((c)->cfg.dtype == COD_BF16) { CALL_BF16; } else { CALL_F32; } \
   } while (0)
 
+int cod_launch_gather_rows(cod_ctx* c, const void* src, const int* rows, const int* n_dev, int n_max, int width,
+                           void* dst, cudaStream_t st) {
+  ProfScope prof(c, COD_K_ROWOPS, st);
+  if (n_max <= 0) return COD_OK;
+  DISPATCH_T(c,
+             (k_gather_rows<__nv_bfloat16><<<n_max, 256, 0, st>>>(static_cast<const __nv_bfloat16*>(src), rows, n_dev, width, static_cast<__nv_bfloat16*>(dst))),
+             (k_gather_rows<float><<<n_max, 256, 0, st>>>(static_cast<const float*>(src), rows, n_dev, width, static_cast<float*>(dst))));
+  COD_CHECK_LAUNCH(c);
+  return COD_OK;
+}
+
 int cod_launch_fcE(cod_ctx* c, cudaStream_t st) {
+  ProfScope prof(c, COD_K_ROWOPS, st);
   DISPATCH_T(c,
              (k_fcE<__nv_bfloat16><<<c->D, 256, 0, st>>>(static_cast<const __nv_bfloat16*>(c->w.fc), static_cast<const __nv_bfloat16*>(c->w.e_carry), c->D_in, c->fcE)),
              (k_fcE<float><<<c->D, 256, 0, st>>>(static_cast<const float*>(c->w.fc), static_cast<const float*>(c->w.e_carry), c->D_in, c->fcE)));
@@ -283,12 +310,13 @@ int cod_launch_fcE(cod_ctx* c, cudaStream_t st) {
 
 int cod_launch_fc_finish(cod_ctx* c, const float* part, int splits, int n_rows, const int* n_rows_dev,
                          const int* a_rows, const int* carry_slot, float* tap_z, cudaStream_t st) {
+  ProfScope prof(c, COD_K_ROWOPS, st);
   if (n_rows <= 0) return COD_OK;
   const size_t smem = (c->D + 33) * sizeof(float);
   const int do_norm = (c->cfg.flags & COD_F_HIDDEN_NORM) ? 1 : 0;
   DISPATCH_T(c,
-             (k_fc_finish<__nv_bfloat16><<<n_rows, 256, smem, st>>>(part, splits, n_rows, n_rows_dev, a_rows, carry_slot, c->fcE, static_cast<const __nv_bfloat16*>(c->w.g_hidden), c->D, c->cfg.rms_eps, do_norm, static_cast<__nv_bfloat16*>(c->z), tap_z)),
-             (k_fc_finish<float><<<n_rows, 256, smem, st>>>(part, splits, n_rows, n_rows_dev, a_rows, carry_slot, c->fcE, static_cast<const float*>(c->w.g_hidden), c->D, c->cfg.rms_eps, do_norm, static_cast<float*>(c->z), tap_z)));
+             (k_fc_finish<__nv_bfloat16><<<n_rows, 256, smem, st>>>(part, splits, n_rows, n_rows_dev, a_rows, carry_slot, c->fcE, static_cast<const __nv_bfloat16*>(c->w.g_hidden), c->D, c->cfg.rms_eps, do_norm, static_cast<__nv_bfloat16*>(c->z), a_rows ? 1 : 0, tap_z)),
+             (k_fc_finish<float><<<n_rows, 256, smem, st>>>(part, splits, n_rows, n_rows_dev, a_rows, carry_slot, c->fcE, static_cast<const float*>(c->w.g_hidden), c->D, c->cfg.rms_eps, do_norm, static_cast<float*>(c->z), a_rows ? 1 : 0, tap_z)));
   COD_CHECK_LAUNCH(c);
   return COD_OK;
 }
@@ -296,6 +324,7 @@ int cod_launch_fc_finish(cod_ctx* c, const float* part, int splits, int n_rows, 
 int cod_launch_kv_finish(cod_ctx* c, const float* part, int splits, int n_rows, const int* n_rows_dev,
                          const int* a_rows, const cod_split* sp, void* J, const cod_state* ds, int R_total,
                          cudaStream_t st) {
+  ProfScope prof(c, COD_K_ROWOPS, st);
   if (n_rows <= 0) return COD_OK;
   const cod_config& f = c->cfg;
   dim3 grid(n_rows, f.n_layers);
@@ -309,6 +338,7 @@ int cod_launch_kv_finish(cod_ctx* c, const float* part, int splits, int n_rows, 
 
 int cod_launch_scatter(cod_ctx* c, const void* J, const cod_split* sp, int S, int mode, const cod_state* ds,
                        cudaStream_t st) {
+  ProfScope prof(c, COD_K_ROWOPS, st);
   const cod_config& f = c->cfg;
   const int R = S * f.block;
   dim3 grid(R, f.n_layers);
@@ -321,6 +351,7 @@ int cod_launch_scatter(cod_ctx* c, const void* J, const cod_split* sp, int S, in
 }
 
 int cod_launch_update_lens(cod_ctx* c, const cod_split* sp, int S, int mode, const cod_state* ds, cudaStream_t st) {
+  ProfScope prof(c, COD_K_ROWOPS, st);
   k_update_lens<<<(S + 127) / 128, 128, 0, st>>>(sp->accept_len, S, c->cfg.block, mode,
                                                  c->cfg.max_pages_per_seq * c->cfg.page_size, ds->committed_len,
                                                  ds->carry_len, c->status);
@@ -329,6 +360,7 @@ int cod_launch_update_lens(cod_ctx* c, const cod_split* sp, int S, int mode, con
 }
 
 int cod_launch_embed_norm(cod_ctx* c, const int32_t* bonus, int S, cudaStream_t st) {
+  ProfScope prof(c, COD_K_ROWOPS, st);
   const cod_config& f = c->cfg;
   const int R = S * f.block;
   DISPATCH_T(c,
@@ -339,6 +371,7 @@ int cod_launch_embed_norm(cod_ctx* c, const int32_t* bonus, int S, cudaStream_t 
 }
 
 int cod_launch_qkv_finish(cod_ctx* c, const float* part, int splits, int R, cudaStream_t st) {
+  ProfScope prof(c, COD_K_ROWOPS, st);
   const cod_config& f = c->cfg;
   DISPATCH_T(c,
              (k_qkv_finish<__nv_bfloat16><<<R, 256, 0, st>>>(part, splits, R, f.n_q_heads, f.n_kv_heads, f.head_dim, c->rope_blk, static_cast<__nv_bfloat16*>(c->q), static_cast<__nv_bfloat16*>(c->kb), static_cast<__nv_bfloat16*>(c->vb))),
@@ -349,6 +382,7 @@ int cod_launch_qkv_finish(cod_ctx* c, const float* part, int splits, int R, cuda
 
 // rope_blk must already hold the block rows' tables
 int cod_launch_rope_qk(cod_ctx* c, const void* q, const void* k, const int32_t* committed_len, int S, cudaStream_t st) {
+  ProfScope prof(c, COD_K_ROWOPS, st);
   (void)committed_len;
   const cod_config& f = c->cfg;
   const int R = S * f.block;
@@ -361,6 +395,7 @@ int cod_launch_rope_qk(cod_ctx* c, const void* q, const void* k, const int32_t* 
 
 int cod_launch_resid_norm(cod_ctx* c, const float* part, int splits, int R, float* x, const void* gain,
                           float* tap_x, cudaStream_t st) {
+  ProfScope prof(c, COD_K_ROWOPS, st);
   DISPATCH_T(c,
              (k_resid_norm<__nv_bfloat16><<<R, 256, 0, st>>>(part, splits, R, c->D, x, static_cast<const __nv_bfloat16*>(gain), c->cfg.rms_eps, static_cast<__nv_bfloat16*>(c->a), tap_x, c->amax)),
              (k_resid_norm<float><<<R, 256, 0, st>>>(part, splits, R, c->D, x, static_cast<const float*>(gain), c->cfg.rms_eps, static_cast<float*>(c->a), tap_x, c->amax)));
@@ -370,6 +405,7 @@ int cod_launch_resid_norm(cod_ctx* c, const float* part, int splits, int R, floa
 
 int cod_launch_finalize(cod_ctx* c, int R, int W, const int32_t* bonus, int32_t* tok, int32_t* next_draft,
                         float* top_logit, cudaStream_t st) {
+  ProfScope prof(c, COD_K_ROWOPS, st);
   k_finalize<<<(R + 127) / 128, 128, 0, st>>>(c->amax, R, W, bonus, tok, next_draft, top_logit);
   COD_CHECK_LAUNCH(c);
   return COD_OK;

@@ -119,6 +119,7 @@ __global__ void k_rope_tables(const int32_t* __restrict__ committed_len, const i
 
 int cod_launch_verify(cod_ctx* c, const int32_t* draft, const int32_t* target, int S, int n_forced,
                       const cod_state* state, const cod_split* out, cudaStream_t st) {
+  ProfScope prof(c, COD_K_VERIFY, st);
   const int W = c->cfg.block;
   const size_t smem = static_cast<size_t>(2 * S + 2) * sizeof(int);
   k_verify_accept<<<1, 1024, smem, st>>>(draft, target, S, W, n_forced, c->cfg.vocab, c->cfg.page_size,
@@ -132,6 +133,7 @@ int cod_launch_verify(cod_ctx* c, const int32_t* draft, const int32_t* target, i
 }
 
 int cod_launch_rope_blk_only(cod_ctx* c, const int32_t* committed_len, int S, cudaStream_t st) {
+  ProfScope prof(c, COD_K_VERIFY, st);
   k_rope_tables<<<S * c->cfg.block, 64, 0, st>>>(committed_len, nullptr, c->inv_freq_d, S, c->cfg.block, c->half,
                                                  nullptr, c->rope_blk);
   COD_CHECK_LAUNCH(c);

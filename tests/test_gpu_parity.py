@@ -92,6 +92,9 @@ def _workloads():
         "small_bf16": small_bf16(S=3, W=16, n_layers=2, ctx=(40, 300)),
         "small_bf16_W32": small_bf16(S=2, W=32, n_layers=1, ctx=(100, 200)),
         "small_bf16_W8": small_bf16(S=5, W=8, n_layers=1, ctx=(0, 50)),
+        # wide enough for split-K, several token tiles with a ragged last one, a ragged vocab tile
+        "mid_bf16": small_bf16(S=34, W=16, n_layers=2, ctx=(100, 600), d_target=512, n_cap=5, d_model=1024,
+                               n_q=8, n_kv=2, vocab=3000),
     }
 
 
@@ -235,7 +238,7 @@ def test_block_attn_split_and_page_invariance():
 
 
 # ----------------------------------------------------------------------------- part 5
-@pytest.mark.parametrize("name", ["tiny_f32", "small_bf16"])
+@pytest.mark.parametrize("name", ["tiny_f32", "small_bf16", "mid_bf16"])
 def test_lm_head_planted_and_ties(name):
     B, Hn = _B(), _H()
     wl = _workloads()[name]
@@ -304,7 +307,8 @@ def test_round_parity_cfg1_every_round():
 @pytest.mark.parametrize("name,wo_scale,mode", [
     ("tiny_f32", 40.0, orc.MODE_CARRY), ("tiny_f32", 40.0, orc.MODE_BASELINE), ("tiny_f32_nonorm", 1.0, orc.MODE_CARRY),
     ("small_bf16", 30.0, orc.MODE_CARRY), ("small_bf16", 30.0, orc.MODE_BASELINE),
-    ("small_bf16_W32", 1.0, orc.MODE_CARRY), ("small_bf16_W8", 30.0, orc.MODE_CARRY)])
+    ("small_bf16_W32", 1.0, orc.MODE_CARRY), ("small_bf16_W8", 30.0, orc.MODE_CARRY),
+    ("mid_bf16", 30.0, orc.MODE_CARRY), ("mid_bf16", 30.0, orc.MODE_BASELINE)])
 def test_round_parity_multi_round(name, wo_scale, mode):
     """Open-loop rounds (inputs pre-generated), ragged acceptance, attention path made to matter."""
     Hn = _H()
