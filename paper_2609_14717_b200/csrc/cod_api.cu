@@ -49,7 +49,9 @@ size_t carve(cod_ctx* c) {
   cv.take(c->vb, es * R * c->kvw);
   cv.take(c->o, es * R * c->qw);
   const size_t M = static_cast<size_t>(f.block) * (f.n_q_heads / f.n_kv_heads);
-  const size_t parts = static_cast<size_t>(f.max_batch) * f.n_kv_heads * c->max_splits * M;
+  const size_t per_head = static_cast<size_t>(c->max_splits > c->tc_max_parts ? c->max_splits : c->tc_max_parts);
+  const size_t parts = static_cast<size_t>(f.max_batch) * f.n_kv_heads * per_head * M;
+  cv.take(c->zero_page, 4096);
   cv.take(c->attn_o, sizeof(float) * parts * f.head_dim);
   cv.take(c->attn_ml, sizeof(float) * parts * 4);
   cv.take(c->amax, sizeof(unsigned long long) * R);
@@ -100,6 +102,7 @@ int cod_launch_gemm(cod_ctx* c, const GemmArgs& g, cudaStream_t st) {
 int cod_launch_attn(cod_ctx* c, int layer, const void* q, const void* kb, const void* vb, const cod_state* state,
                     int S, int use_carry, void* out, float* tap_out, float* carry_mass, cudaStream_t st) {
   ProfScope prof(c, COD_K_ATTN, st);
+  if (cod_attn_tc_supported(c)) return cod_launch_attn_tc(c, layer, q, kb, vb, state, S, use_carry, out, tap_out, carry_mass, st);
   return cod_launch_attn_simt(c, layer, q, kb, vb, state, S, use_carry, out, tap_out, carry_mass, st);
 }
 
@@ -142,6 +145,22 @@ int cod_create(const cod_config* cfg, cod_ctx** out) {
   const int64_t max_keys = static_cast<int64_t>(f.max_pages_per_seq) * f.page_size + 2 * f.block;
   c->max_splits = static_cast<int>((max_keys + c->split_len - 1) / c->split_len);
 
+  {
+    // tensor-core attention: keys of the paged region per CTA, and partial slots per (sequence, head)
+    const int M = f.block * (f.n_q_heads / f.n_kv_heads);
+    const int64_t cap = static_cast<int64_t>(f.max_pages_per_seq) * f.page_size;
+    int64_t sl;
+    if (f.attn_split_len > 0) sl = (f.attn_split_len + 127) / 128 * 128;
+    else {
+      sl = (cap * f.max_batch * f.n_kv_heads / (8 * static_cast<int64_t>(c->n_sm)) + 127) / 128 * 128;
+      if (sl < 128) sl = 128;
+      if (sl > 2048) sl = 2048;
+    }
+    c->tc_split_len = static_cast<int>(sl);
+    const int keys_it = M <= 64 ? 128 : 64, ring = M <= 64 ? 2 : 4;
+    const bool tail_fits = (15 + 2 * f.block + keys_it - 1) / keys_it <= ring;
+    c->tc_max_parts = tail_fits ? static_cast<int>((cap + sl - 1) / sl + 1) * (M <= 64 ? 2 : 1) : 0;
+  }
   c->ws = nullptr;
   c->ws_bytes = carve(c);
   if (cudaMalloc(&c->ws, c->ws_bytes) != cudaSuccess) { cudaGetLastError(); delete c; return COD_ERR_ALLOC; }

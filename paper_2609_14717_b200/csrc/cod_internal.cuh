@@ -98,7 +98,9 @@ struct cod_ctx {
   bool has_weights;
   int device;
   int D, D_in, kvw, qw, R_max, half;
-  int split_len, max_splits;   // attention split-KV
+  int split_len, max_splits;   // attention split-KV (plain-FMA kernel)
+  int tc_split_len, tc_max_parts;  // attention split-KV (tensor-core kernel); 0 parts = not usable
+  void* zero_page;             // 16 x 128 bf16 zeros (stands in for pages past the end of a split)
   int n_sm;
   bool force_simt;             // COD_F_NO_TENSOR_CORES: plain-FMA kernels only
   int64_t launches;
@@ -155,6 +157,9 @@ int cod_launch_verify(cod_ctx* c, const int32_t* draft, const int32_t* target, i
 int cod_launch_gemm(cod_ctx* c, const GemmArgs& g, cudaStream_t st);
 int cod_launch_gemm_simt(cod_ctx* c, const GemmArgs& g, cudaStream_t st);
 bool cod_gemm_tc_supported(const cod_ctx* c, const GemmArgs& g);
+bool cod_attn_tc_supported(const cod_ctx* c);
+int cod_launch_attn_tc(cod_ctx* c, int layer, const void* q, const void* kb, const void* vb, const cod_state* stt,
+                       int S, int use_carry, void* out, float* tap, float* mass, cudaStream_t st);
 int cod_launch_gemm_tc(cod_ctx* c, const GemmArgs& g, cudaStream_t st);
 int cod_launch_attn_simt(cod_ctx* c, int layer, const void* q, const void* kb, const void* vb,
                          const cod_state* stt, int S, int use_carry, void* out, float* tap, float* mass,

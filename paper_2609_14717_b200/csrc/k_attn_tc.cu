@@ -1,0 +1,609 @@
+// Part 4 on the tensor cores: split-KV block attention over [C_l; U_l; block] for bf16, head
+// size 128, page size 16 (Section 2 "Preliminaries"; Algorithm 1 "the next draft reads ctx_l").
+//
+// A CTA owns one (sequence, KV head, split). The W * (n_q / n_kv) query rows that share the KV
+// head are the MMA's M dimension, so every K/V byte is read once per sequence.
+//   S = Q K^T   tcgen05.mma, Q and the K tile K-major in shared memory, S in tensor memory
+//   P = exp2(S * c - m)   one thread per query row: row max and row sum are thread-local
+//   O = P V     tcgen05.mma, P (bf16) K-major in shared memory, the V tile MN-major
+// With 64 query rows (block 16, GQA 4) an M = 64 accumulator uses lanes 0-15 of each 32-lane
+// quarter of tensor memory; a second, independent M = 64 tile is placed on lanes 16-31, so the
+// CTA works on two 64-key tiles at once and all 128 softmax threads have a row. With 128 query
+// rows (block 32) one M = 128 tile is used.
+//
+// Keys: [0, F) with F = 16 * floor(L / 16) come from whole pages, fetched by TMA straight from the
+// block table into a shared-memory ring (two 16 x 64-element boxes per page and operand, no
+// multi-destination loads). The remaining L - F committed rows, the c carried rows and the W
+// block rows form the tail, gathered with plain 128-bit loads by one extra CTA per (sequence, head)
+// which zero-fills the padding, so stale or unallocated rows are never read.
+// Each 64-key tile yields an unnormalised partial (o, m, l); a second kernel merges them.
+//
+//   warps 0-3 softmax / accumulation     warp 4 TMA producer     warp 5 MMA issuer
+// Every mbarrier wait is bounded and raises COD_DEV_TIMEOUT instead of spinning forever.
+#include <cuda.h>
+
+#include "cod_internal.cuh"
+
+namespace {
+
+constexpr int HD = 128, PAGE = 16, KT = 64;           // head size, page size, keys per tile
+constexpr int NTHREADS = 192;
+constexpr uint32_t TILE_BYTES = KT * HD * 2;           // one 64-key K or V tile: 16 KB
+constexpr uint32_t HALF_BYTES = KT * 128;              // 64 keys x 64 elements: 8 KB
+constexpr unsigned long long WAIT_LIMIT_NS = 2000000000ull;
+
+struct AttnParams {
+  const __nv_bfloat16 *q, *kb, *vb;     // rotated q [R, n_q*hd]; rotated k_blk, v_blk [R, n_kv*hd]
+  const __nv_bfloat16 *pool, *carry;
+  const int *block_table, *committed_len, *carry_len;
+  int use_carry, layer, W, rep, n_kv, n_pages, max_pages, max_batch;
+  int split_len;                        // keys of the paged region per CTA (multiple of 128)
+  int max_parts;                        // partial slots per (sequence, KV head)
+  float* part_o;                        // [S][n_kv][max_parts][M][hd]
+  float* part_ml;                       // [S][n_kv][max_parts][M][4]   m (natural log units), l, l_carry
+  uint32_t* status;
+};
+
+// ------------------------------------------------------------------ PTX wrappers
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return static_cast<uint32_t>(__cvta_generic_to_shared(p)); }
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count));
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+  return ok != 0;
+}
+__device__ __forceinline__ unsigned long long global_ns() {
+  unsigned long long t;
+  asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
+  return t;
+}
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, uint32_t* status) {
+  const unsigned long long t0 = global_ns();
+  for (;;) {
+#pragma unroll 1
+    for (int i = 0; i < 256; ++i)
+      if (mbar_try_wait(bar, parity)) return true;
+    if (*abort_flag) return false;
+    if (global_ns() - t0 > WAIT_LIMIT_NS) {
+      *abort_flag = 1;
+      atomicOr(status, COD_DEV_TIMEOUT);
+      return false;
+    }
+  }
+}
+__device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap* map, int c0, int c1, int c2, uint32_t bar) {
+  asm volatile(
+      "cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4}], [%5];"
+      ::"r"(dst), "l"(reinterpret_cast<uint64_t>(map)), "r"(c0), "r"(c1), "r"(c2), "r"(bar) : "memory");
+}
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void fence_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
+__device__ __forceinline__ void tmem_alloc(uint32_t dst_smem, uint32_t cols) {
+  asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(dst_smem), "r"(cols) : "memory");
+  asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void tmem_dealloc(uint32_t taddr, uint32_t cols) {
+  asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(cols) : "memory");
+}
+__device__ __forceinline__ void umma_bf16(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, uint32_t accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+      ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate) : "memory");
+}
+__device__ __forceinline__ void umma_commit(uint32_t bar) {
+  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&v)[32]) {
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+      "{%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31}, [%32];"
+      : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]),
+        "=r"(v[8]), "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15]),
+        "=r"(v[16]), "=r"(v[17]), "=r"(v[18]), "=r"(v[19]), "=r"(v[20]), "=r"(v[21]), "=r"(v[22]), "=r"(v[23]),
+        "=r"(v[24]), "=r"(v[25]), "=r"(v[26]), "=r"(v[27]), "=r"(v[28]), "=r"(v[29]), "=r"(v[30]), "=r"(v[31])
+      : "r"(taddr) : "memory");
+  asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+}
+
+// K-major operand, 128-byte rows, 128-byte swizzle, 8-row groups 1024 bytes apart.
+__device__ __forceinline__ uint64_t desc_kmajor(uint32_t saddr) {
+  uint64_t d = 0;
+  d |= static_cast<uint64_t>((saddr & 0x3FFFFu) >> 4);
+  d |= static_cast<uint64_t>(1) << 16;
+  d |= static_cast<uint64_t>(1024 >> 4) << 32;
+  d |= static_cast<uint64_t>(1) << 46;
+  d |= static_cast<uint64_t>(2) << 61;
+  return d;
+}
+// MN-major operand (V tile: rows are keys, 64 contiguous head elements per 128-byte row): the
+// next 64 head elements sit HALF_BYTES further (leading offset), the next 8 keys 1024 bytes
+// further (stride offset).
+__device__ __forceinline__ uint64_t desc_mnmajor(uint32_t saddr) {
+  uint64_t d = 0;
+  d |= static_cast<uint64_t>((saddr & 0x3FFFFu) >> 4);
+  d |= static_cast<uint64_t>(HALF_BYTES >> 4) << 16;
+  d |= static_cast<uint64_t>(1024 >> 4) << 32;
+  d |= static_cast<uint64_t>(1) << 46;
+  d |= static_cast<uint64_t>(2) << 61;
+  return d;
+}
+__device__ __forceinline__ uint32_t instr_desc(int m, int n, int b_mn_major) {
+  uint32_t d = 0;
+  d |= 1u << 4;                                  // float accumulator
+  d |= 1u << 7;                                  // A: bf16
+  d |= 1u << 10;                                 // B: bf16
+  d |= static_cast<uint32_t>(b_mn_major) << 16;  // B major
+  d |= static_cast<uint32_t>(n >> 3) << 17;
+  d |= static_cast<uint32_t>(m >> 4) << 24;
+  return d;
+}
+
+template <bool DUAL>
+struct Geo {
+  static constexpr int TILES = DUAL ? 2 : 1;             // 64-key tiles per iteration
+  static constexpr int MROWS = DUAL ? 64 : 128;          // MMA M
+  static constexpr int KEYS_IT = KT * TILES;
+  static constexpr int NK = DUAL ? 2 : 4;                // K ring slots
+  static constexpr int NV = DUAL ? 3 : 5;                // V ring slots
+  static constexpr uint32_t SLOT = TILE_BYTES * TILES;
+  static constexpr uint32_t Q_BYTES = MROWS * HD * 2;
+  static constexpr uint32_t Q_HALF = MROWS * 128;
+  static constexpr uint32_t P_TILE = MROWS * 128;        // [MROWS][64 keys] bf16
+  static constexpr uint32_t P_BUF = P_TILE * TILES;
+  static constexpr uint32_t OFF_P = Q_BYTES;
+  static constexpr uint32_t OFF_K = OFF_P + 2 * P_BUF;
+  static constexpr uint32_t OFF_V = OFF_K + NK * SLOT;
+  static constexpr uint32_t OFF_CTL = OFF_V + NV * SLOT;
+  static constexpr uint32_t SMEM = OFF_CTL + 256 + 1024;
+  // tensor memory columns: S[2] (64 each) then O[2] (128 each)
+  static constexpr uint32_t COL_S = 0, COL_O = 128, TMEM_COLS = 512;
+};
+
+template <bool DUAL>
+__global__ void __launch_bounds__(NTHREADS, 1)
+k_attn_tc(const __grid_constant__ CUtensorMap map_pool, const __grid_constant__ CUtensorMap map_zero, const AttnParams p) {
+  using G = Geo<DUAL>;
+  extern __shared__ uint8_t smem_raw[];
+  const uint32_t raw = smem_u32(smem_raw);
+  const uint32_t base = (raw + 1023u) & ~1023u;
+  uint8_t* sm = smem_raw + (base - raw);
+  uint64_t* bars = reinterpret_cast<uint64_t*>(sm + G::OFF_CTL);
+  uint64_t* k_full = bars;                  // [NK]
+  uint64_t* k_empty = bars + 5;             // [NK]
+  uint64_t* v_full = bars + 10;             // [NV]
+  uint64_t* v_empty = bars + 15;            // [NV]
+  uint64_t* s_full = bars + 20;             // [2]
+  uint64_t* p_full = bars + 22;             // [2]
+  uint64_t* o_full = bars + 24;             // [2]
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 26);
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int split = blockIdx.x, h = blockIdx.y, s = blockIdx.z;
+  const int M = p.W * p.rep;
+
+  uint32_t flags = 0;
+  int L = p.committed_len[s];
+  int c = p.use_carry ? p.carry_len[s] : 0;
+  if (L < 0 || L > p.max_pages * PAGE) { flags |= COD_DEV_BAD_LEN; L = max(0, min(L, p.max_pages * PAGE)); }
+  if (c < 0 || c > p.W) { flags |= COD_DEV_BAD_LEN; c = max(0, min(c, p.W)); }
+  const int F = (L / PAGE) * PAGE;                       // keys held in whole pages
+  const int n_reg = (F + p.split_len - 1) / p.split_len; // CTAs over the paged region
+  if (split > n_reg) return;
+  const bool is_tail = split == n_reg;
+  const int Lr = L - F;                                  // committed rows in the last, partial page
+  const int n_tail = Lr + c + p.W;
+  const int k_begin = is_tail ? 0 : split * p.split_len;
+  const int k_end = is_tail ? n_tail : min(F, k_begin + p.split_len);
+  const int n_it = (k_end - k_begin + G::KEYS_IT - 1) / G::KEYS_IT;
+
+  if (threadIdx.x == 0) {
+    for (int i = 0; i < G::NK; ++i) { mbar_init(smem_u32(k_full + i), is_tail ? 128 : 1); mbar_init(smem_u32(k_empty + i), 1); }
+    for (int i = 0; i < G::NV; ++i) { mbar_init(smem_u32(v_full + i), is_tail ? 128 : 1); mbar_init(smem_u32(v_empty + i), 1); }
+    for (int i = 0; i < 2; ++i) { mbar_init(smem_u32(s_full + i), 1); mbar_init(smem_u32(p_full + i), 128); mbar_init(smem_u32(o_full + i), 1); }
+    *abort_flag = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  if (warp == 5) tmem_alloc(smem_u32(tmem_slot), G::TMEM_COLS);
+
+  // Q tile: [half][row][64 elements], 128-byte rows, chunks of 16 bytes XOR-swizzled by (row & 7);
+  // rows beyond the real query rows are zero.
+  if (warp < 4) {
+    const int qw = p.n_kv * p.rep * HD;
+    for (int idx = threadIdx.x; idx < G::MROWS * 16; idx += 128) {
+      const int r = idx >> 4, ch = idx & 15;
+      uint4 v = make_uint4(0u, 0u, 0u, 0u);
+      if (r < M) {
+        const int i = r / p.rep, gg = r - i * p.rep;
+        v = *reinterpret_cast<const uint4*>(p.q + static_cast<size_t>(s * p.W + i) * qw + (h * p.rep + gg) * HD + ch * 8);
+      }
+      const uint32_t off = (ch >> 3) * G::Q_HALF + r * 128 + (((ch & 7) ^ (r & 7)) << 4);
+      *reinterpret_cast<uint4*>(sm + off) = v;
+    }
+    fence_async_smem();
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = *tmem_slot;
+
+  if (warp == 4) {
+    // ------------------------------------------------ TMA producer (paged region only)
+    if (!is_tail) {
+      const int pages_it = G::KEYS_IT / PAGE;           // 8 or 4 pages per iteration, one per lane
+      bool ok = true;
+      for (int it = 0; it < n_it && ok; ++it) {
+        const int key0 = k_begin + it * G::KEYS_IT + lane * PAGE;
+        int row_k = -1;                                 // first key row of this lane's page in the pool map
+        if (lane < pages_it && key0 < k_end) {
+          int pg = p.block_table[s * p.max_pages + key0 / PAGE];
+          if (pg < 0 || pg >= p.n_pages) { flags |= COD_DEV_BAD_PAGE; }
+          else row_k = (((p.layer * p.n_pages + pg) * p.n_kv + h) * 2) * PAGE;
+        }
+        const uint32_t in_slot = (lane / (KT / PAGE)) * TILE_BYTES + (lane % (KT / PAGE)) * (PAGE * 128);
+        // K
+        {
+          const int slot = it % G::NK, use = it / G::NK;
+          if (lane == 0 && use > 0) ok = mbar_wait(smem_u32(k_empty + slot), (use - 1) & 1, abort_flag, p.status);
+          ok = __shfl_sync(0xffffffffu, ok, 0);
+          if (!ok) break;
+          const uint32_t fb = smem_u32(k_full + slot);
+          if (lane == 0) mbar_expect_tx(fb, G::SLOT);
+          __syncwarp();
+          if (lane < pages_it) {
+            const uint32_t dst = base + G::OFF_K + slot * G::SLOT + in_slot;
+            if (row_k >= 0) {
+              tma_load_3d(dst, &map_pool, 0, 0, row_k, fb);
+              tma_load_3d(dst + HALF_BYTES, &map_pool, 0, 1, row_k, fb);
+            } else {
+              tma_load_3d(dst, &map_zero, 0, 0, 0, fb);
+              tma_load_3d(dst + HALF_BYTES, &map_zero, 0, 1, 0, fb);
+            }
+          }
+        }
+        // V
+        {
+          const int slot = it % G::NV, use = it / G::NV;
+          if (lane == 0 && use > 0) ok = mbar_wait(smem_u32(v_empty + slot), (use - 1) & 1, abort_flag, p.status);
+          ok = __shfl_sync(0xffffffffu, ok, 0);
+          if (!ok) break;
+          const uint32_t fb = smem_u32(v_full + slot);
+          if (lane == 0) mbar_expect_tx(fb, G::SLOT);
+          __syncwarp();
+          if (lane < pages_it) {
+            const uint32_t dst = base + G::OFF_V + slot * G::SLOT + in_slot;
+            if (row_k >= 0) {
+              tma_load_3d(dst, &map_pool, 0, 0, row_k + PAGE, fb);
+              tma_load_3d(dst + HALF_BYTES, &map_pool, 0, 1, row_k + PAGE, fb);
+            } else {
+              tma_load_3d(dst, &map_zero, 0, 0, 0, fb);
+              tma_load_3d(dst + HALF_BYTES, &map_zero, 0, 1, 0, fb);
+            }
+          }
+        }
+      }
+    }
+  } else if (warp == 5) {
+    // ------------------------------------------------ MMA issuer
+    if (lane == 0 && n_it > 0) {
+      const uint32_t idesc_qk = instr_desc(G::MROWS, KT, 0);
+      const uint32_t idesc_pv = instr_desc(G::MROWS, HD, 1);
+      const uint64_t q_desc = desc_kmajor(base);
+      bool ok = true;
+      auto issue_qk = [&](int it) -> bool {
+        const int slot = it % G::NK;
+        if (!mbar_wait(smem_u32(k_full + slot), (it / G::NK) & 1, abort_flag, p.status)) return false;
+        tc_fence_after();
+#pragma unroll
+        for (int t = 0; t < G::TILES; ++t) {
+          const uint64_t k_desc = desc_kmajor(base + G::OFF_K + slot * G::SLOT + t * TILE_BYTES);
+          const uint32_t d = tmem_base + G::COL_S + (it & 1) * KT + (static_cast<uint32_t>(16 * t) << 16);
+#pragma unroll
+          for (int k = 0; k < HD / 16; ++k) {
+            const uint32_t qa = (k < 4 ? 0u : (G::Q_HALF >> 4)) + (k & 3) * 2;
+            const uint32_t ka = (k < 4 ? 0u : (HALF_BYTES >> 4)) + (k & 3) * 2;
+            umma_bf16(d, q_desc + qa, k_desc + ka, idesc_qk, k ? 1u : 0u);
+          }
+        }
+        umma_commit(smem_u32(s_full + (it & 1)));
+        umma_commit(smem_u32(k_empty + slot));
+        return true;
+      };
+      ok = issue_qk(0);
+      for (int it = 0; it < n_it && ok; ++it) {
+        if (it + 1 < n_it) ok = issue_qk(it + 1);
+        if (!ok) break;
+        const int slot = it % G::NV;
+        ok = mbar_wait(smem_u32(p_full + (it & 1)), (it >> 1) & 1, abort_flag, p.status) &&
+             mbar_wait(smem_u32(v_full + slot), (it / G::NV) & 1, abort_flag, p.status);
+        if (!ok) break;
+        tc_fence_after();
+#pragma unroll
+        for (int t = 0; t < G::TILES; ++t) {
+          const uint64_t p_desc = desc_kmajor(base + G::OFF_P + (it & 1) * G::P_BUF + t * G::P_TILE);
+          const uint64_t v_desc = desc_mnmajor(base + G::OFF_V + slot * G::SLOT + t * TILE_BYTES);
+          const uint32_t d = tmem_base + G::COL_O + (it & 1) * HD + (static_cast<uint32_t>(16 * t) << 16);
+#pragma unroll
+          for (int kk = 0; kk < KT / 16; ++kk)       // 16 keys per MMA: 32 bytes along P's rows, 16 rows of V
+            umma_bf16(d, p_desc + kk * 2, v_desc + kk * ((16 * 128) >> 4), idesc_pv, kk ? 1u : 0u);
+        }
+        umma_commit(smem_u32(o_full + (it & 1)));
+        umma_commit(smem_u32(v_empty + slot));
+      }
+    }
+  } else {
+    // ------------------------------------------------ softmax / accumulation: one thread per (row, tile)
+    const int T = threadIdx.x;
+    const int tile = DUAL ? (lane >> 4) : 0;
+    const int r = DUAL ? (16 * warp + (lane & 15)) : T;
+    const uint32_t t_lane = tmem_base + (static_cast<uint32_t>(32 * warp) << 16);
+    const float sl2 = rsqrtf(static_cast<float>(HD)) * 1.4426950408889634f;
+    float m_run = -INFINITY, l_run = 0.f, lc_run = 0.f, corr_pending = 1.f;
+    float o_acc[HD];
+#pragma unroll
+    for (int d = 0; d < HD; ++d) o_acc[d] = 0.f;
+    bool ok = true;
+
+    auto accumulate_o = [&](int it) -> bool {
+      if (!mbar_wait(smem_u32(o_full + (it & 1)), (it >> 1) & 1, abort_flag, p.status)) return false;
+      tc_fence_after();
+#pragma unroll
+      for (int q4 = 0; q4 < HD / 32; ++q4) {
+        uint32_t v[32];
+        tmem_ld32(t_lane + G::COL_O + (it & 1) * HD + q4 * 32, v);
+#pragma unroll
+        for (int j = 0; j < 32; ++j) o_acc[q4 * 32 + j] = fmaf(o_acc[q4 * 32 + j], corr_pending, __uint_as_float(v[j]));
+      }
+      return true;
+    };
+
+    for (int it = 0; it < n_it && ok; ++it) {
+      if (is_tail) {
+        // gather this iteration's rows (partial page, carried rows, block rows) with plain loads
+        const int kslot = it % G::NK, vslot = it % G::NV;
+        for (int idx0 = T; idx0 < G::KEYS_IT * 32; idx0 += 128 * 4) {
+          uint4 val[4];
+          uint32_t dst[4];
+#pragma unroll
+          for (int u = 0; u < 4; ++u) {
+            const int idx = idx0 + u * 128;
+            const int ch = idx & 15, kv = (idx >> 4) & 1, j = idx >> 5;       // chunk, K|V, key within iteration
+            const int g = it * G::KEYS_IT + j;
+            const __nv_bfloat16* src = nullptr;
+            if (g < Lr) {
+              int pg = p.block_table[s * p.max_pages + F / PAGE];
+              if (pg < 0 || pg >= p.n_pages) { flags |= COD_DEV_BAD_PAGE; }
+              else src = p.pool + ((((static_cast<size_t>(p.layer) * p.n_pages + pg) * p.n_kv + h) * 2 + kv) * PAGE + g) * HD;
+            } else if (g < Lr + c) {
+              src = p.carry + ((((static_cast<size_t>(p.layer) * p.max_batch + s) * p.n_kv + h) * 2 + kv) * p.W + (g - Lr)) * HD;
+            } else if (g < n_tail) {
+              src = (kv ? p.vb : p.kb) + static_cast<size_t>(s * p.W + (g - Lr - c)) * (p.n_kv * HD) + h * HD;
+            }
+            val[u] = src ? *reinterpret_cast<const uint4*>(src + ch * 8) : make_uint4(0u, 0u, 0u, 0u);
+            const int jj = j & (KT - 1), tl = j / KT;
+            dst[u] = (kv ? G::OFF_V + vslot * G::SLOT : G::OFF_K + kslot * G::SLOT) + tl * TILE_BYTES +
+                     (ch >> 3) * HALF_BYTES + jj * 128 + (((ch & 7) ^ (jj & 7)) << 4);
+          }
+#pragma unroll
+          for (int u = 0; u < 4; ++u) *reinterpret_cast<uint4*>(sm + dst[u]) = val[u];
+        }
+        fence_async_smem();
+        mbar_arrive(smem_u32(k_full + kslot));
+        mbar_arrive(smem_u32(v_full + vslot));
+      }
+
+      ok = mbar_wait(smem_u32(s_full + (it & 1)), (it >> 1) & 1, abort_flag, p.status);
+      if (!ok) break;
+      tc_fence_after();
+      const int key_t0 = k_begin + it * G::KEYS_IT + tile * KT;         // first key of this thread's tile
+      const int n_valid = max(0, min(KT, k_end - key_t0));
+      float sc[KT];
+      {
+        uint32_t v[32];
+        tmem_ld32(t_lane + G::COL_S + (it & 1) * KT, v);
+#pragma unroll
+        for (int j = 0; j < 32; ++j) sc[j] = __uint_as_float(v[j]);
+        tmem_ld32(t_lane + G::COL_S + (it & 1) * KT + 32, v);
+#pragma unroll
+        for (int j = 0; j < 32; ++j) sc[32 + j] = __uint_as_float(v[j]);
+      }
+      float mx = -INFINITY;
+#pragma unroll
+      for (int j = 0; j < KT; ++j) {
+        sc[j] = j < n_valid ? sc[j] * sl2 : -INFINITY;
+        mx = fmaxf(mx, sc[j]);
+      }
+      const float m_new = fmaxf(m_run, mx);
+      const float m_use = m_new == -INFINITY ? 0.f : m_new;              // nothing valid yet: all p = 0
+      const float corr = exp2f(m_run - m_use);                            // exp2(-inf) = 0
+      float psum = 0.f, pcar = 0.f;
+      uint8_t* prow = sm + G::OFF_P + (it & 1) * G::P_BUF + tile * G::P_TILE + r * 128;
+      const int car0 = is_tail ? Lr - (it * G::KEYS_IT + tile * KT) : KT;  // carried keys: [car0, car0 + c)
+#pragma unroll
+      for (int ch = 0; ch < 8; ++ch) {
+        uint32_t packed[4];
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+          const int j = ch * 8 + e * 2;
+          const float p0 = exp2f(sc[j] - m_use), p1 = exp2f(sc[j + 1] - m_use);
+          psum += p0 + p1;
+          if (is_tail) {
+            if (j >= car0 && j < car0 + c) pcar += p0;
+            if (j + 1 >= car0 && j + 1 < car0 + c) pcar += p1;
+          }
+          const __nv_bfloat162 b = __floats2bfloat162_rn(p0, p1);
+          packed[e] = *reinterpret_cast<const uint32_t*>(&b);
+        }
+        *reinterpret_cast<uint4*>(prow + ((ch ^ (r & 7)) << 4)) = make_uint4(packed[0], packed[1], packed[2], packed[3]);
+      }
+      fence_async_smem();
+      tc_fence_before();
+      mbar_arrive(smem_u32(p_full + (it & 1)));
+      l_run = l_run * corr + psum;
+      lc_run = lc_run * corr + pcar;
+      m_run = m_new;
+      if (it > 0) ok = accumulate_o(it - 1);
+      corr_pending = corr;
+    }
+    if (ok && n_it > 0) ok = accumulate_o(n_it - 1);
+
+    // partial results of this (row, tile)
+    const int part = (DUAL ? 2 : 1) * split + tile;
+    if (r < M && (ok || n_it == 0)) {
+      const size_t rowi = ((static_cast<size_t>(s) * p.n_kv + h) * p.max_parts + part) * M + r;
+      float4* po = reinterpret_cast<float4*>(p.part_o + rowi * HD);
+#pragma unroll
+      for (int d = 0; d < HD / 4; ++d) po[d] = make_float4(o_acc[4 * d], o_acc[4 * d + 1], o_acc[4 * d + 2], o_acc[4 * d + 3]);
+      float* ml = p.part_ml + rowi * 4;
+      ml[0] = m_run * 0.6931471805599453f;      // back to natural-log units
+      ml[1] = l_run;
+      ml[2] = lc_run;
+    }
+  }
+
+  // ---------------------------------------------------- teardown
+  if (flags) atomicOr(p.status, flags);
+  tc_fence_before();
+  __syncthreads();
+  if (*abort_flag) {
+    for (int i = 0; i < 64; ++i) __nanosleep(1000);
+    __syncthreads();
+  }
+  if (warp == 5) {
+    __syncwarp();
+    tc_fence_after();
+    tmem_dealloc(tmem_base, G::TMEM_COLS);
+  }
+}
+
+// Merges the partials of one (row, query head); one warp each. Empty partials carry m = -inf, l = 0.
+template <bool DUAL>
+__global__ void k_attn_tc_combine(const float* __restrict__ part_o, const float* __restrict__ part_ml,
+                                  const int* __restrict__ committed_len, int S, int W, int rep, int n_kv,
+                                  int max_pages, int split_len, int max_parts, __nv_bfloat16* __restrict__ out,
+                                  float* __restrict__ tap, float* __restrict__ mass) {
+  const int lane = threadIdx.x & 31;
+  const int item = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+  const int n_q = n_kv * rep;
+  if (item >= S * W * n_q) return;
+  const int g = item % n_q, i = (item / n_q) % W, s = item / (n_q * W);
+  const int h = g / rep, mrow = i * rep + (g - h * rep), M = W * rep;
+  const int L = max(0, min(committed_len[s], max_pages * PAGE));
+  const int F = (L / PAGE) * PAGE;
+  const int n_parts = ((F + split_len - 1) / split_len + 1) * (DUAL ? 2 : 1);
+  const size_t base = (static_cast<size_t>(s) * n_kv + h) * max_parts;
+  float mg = -INFINITY;
+  for (int k = 0; k < n_parts; ++k) mg = fmaxf(mg, part_ml[((base + k) * M + mrow) * 4]);
+  float acc[4] = {0.f, 0.f, 0.f, 0.f}, l = 0.f, lc = 0.f;
+  for (int k = 0; k < n_parts; ++k) {
+    const float* ml = part_ml + ((base + k) * M + mrow) * 4;
+    const float w = __expf(ml[0] - mg);
+    l = fmaf(w, ml[1], l);
+    lc = fmaf(w, ml[2], lc);
+    const float4 v = *reinterpret_cast<const float4*>(part_o + ((base + k) * M + mrow) * HD + lane * 4);
+    acc[0] = fmaf(w, v.x, acc[0]); acc[1] = fmaf(w, v.y, acc[1]); acc[2] = fmaf(w, v.z, acc[2]); acc[3] = fmaf(w, v.w, acc[3]);
+  }
+  const float inv = 1.f / l;
+  const size_t ob = static_cast<size_t>(item) * HD + lane * 4;
+  const __nv_bfloat162 b0 = __floats2bfloat162_rn(acc[0] * inv, acc[1] * inv), b1 = __floats2bfloat162_rn(acc[2] * inv, acc[3] * inv);
+  uint2 pk;
+  pk.x = *reinterpret_cast<const uint32_t*>(&b0);
+  pk.y = *reinterpret_cast<const uint32_t*>(&b1);
+  *reinterpret_cast<uint2*>(out + ob) = pk;
+  if (tap) *reinterpret_cast<float4*>(tap + ob) = make_float4(acc[0] * inv, acc[1] * inv, acc[2] * inv, acc[3] * inv);
+  if (mass && lane == 0) mass[item] = lc * inv;
+}
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+EncodeTiledFn encode_fn() {
+  static EncodeTiledFn fn = nullptr;
+  static bool tried = false;
+  if (!tried) {
+    tried = true;
+    void* ptr = nullptr;
+    cudaDriverEntryPointQueryResult q;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &ptr, cudaEnableDefault, &q) == cudaSuccess &&
+        q == cudaDriverEntryPointSuccess)
+      fn = reinterpret_cast<EncodeTiledFn>(ptr);
+  }
+  return fn;
+}
+
+// Rows of 128 bf16 seen as (64 elements, 2 halves, rows); a box is one half of 16 consecutive rows.
+bool make_rows_map(CUtensorMap* m, const void* ptr, uint64_t rows) {
+  EncodeTiledFn fn = encode_fn();
+  if (!fn) return false;
+  cuuint64_t gdim[3] = {64, 2, rows};
+  cuuint64_t gstride[2] = {128, 256};
+  cuuint32_t box[3] = {64, 1, PAGE};
+  cuuint32_t estr[3] = {1, 1, 1};
+  return fn(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(ptr), gdim, gstride, box, estr,
+            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+template <bool DUAL>
+int launch(cod_ctx* c, int layer, const void* q, const void* kb, const void* vb, const cod_state* stt, int S,
+           int use_carry, void* out, float* tap, float* mass, cudaStream_t st) {
+  using G = Geo<DUAL>;
+  const cod_config& f = c->cfg;
+  CUtensorMap mp, mz;
+  const uint64_t rows = static_cast<uint64_t>(f.n_layers) * f.n_pages * f.n_kv_heads * 2 * PAGE;
+  if (!make_rows_map(&mp, stt->kv_pool, rows) || !make_rows_map(&mz, c->zero_page, PAGE)) return COD_ERR_CUDA;
+  AttnParams p{};
+  p.q = static_cast<const __nv_bfloat16*>(q); p.kb = static_cast<const __nv_bfloat16*>(kb); p.vb = static_cast<const __nv_bfloat16*>(vb);
+  p.pool = static_cast<const __nv_bfloat16*>(stt->kv_pool); p.carry = static_cast<const __nv_bfloat16*>(stt->carry_kv);
+  p.block_table = stt->block_table; p.committed_len = stt->committed_len; p.carry_len = stt->carry_len;
+  p.use_carry = use_carry; p.layer = layer; p.W = f.block; p.rep = f.n_q_heads / f.n_kv_heads; p.n_kv = f.n_kv_heads;
+  p.n_pages = f.n_pages; p.max_pages = f.max_pages_per_seq; p.max_batch = f.max_batch;
+  p.split_len = c->tc_split_len; p.max_parts = c->tc_max_parts;
+  p.part_o = c->attn_o; p.part_ml = c->attn_ml; p.status = c->status;
+  static bool configured = false;
+  if (!configured) {
+    if (cudaFuncSetAttribute(k_attn_tc<DUAL>, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(G::SMEM)) != cudaSuccess)
+      return COD_ERR_CUDA;
+    configured = true;
+  }
+  dim3 grid(c->tc_max_parts / (DUAL ? 2 : 1), f.n_kv_heads, S);
+  k_attn_tc<DUAL><<<grid, NTHREADS, G::SMEM, st>>>(mp, mz, p);
+  COD_CHECK_LAUNCH(c);
+  const int items = S * f.block * f.n_q_heads;
+  k_attn_tc_combine<DUAL><<<(items + 3) / 4, 128, 0, st>>>(c->attn_o, c->attn_ml, stt->committed_len, S, f.block, p.rep,
+                                                           f.n_kv_heads, f.max_pages_per_seq, c->tc_split_len,
+                                                           c->tc_max_parts, static_cast<__nv_bfloat16*>(out), tap, mass);
+  COD_CHECK_LAUNCH(c);
+  return COD_OK;
+}
+
+}  // namespace
+
+bool cod_attn_tc_supported(const cod_ctx* c) {
+  const cod_config& f = c->cfg;
+  const int M = f.block * (f.n_q_heads / f.n_kv_heads);
+  return f.dtype == COD_BF16 && f.head_dim == HD && f.page_size == PAGE && M <= 128 && !c->force_simt &&
+         c->tc_max_parts > 0 && encode_fn() != nullptr;
+}
+
+// q / kb already rotated. Layout of the partial buffers is private to this file.
+int cod_launch_attn_tc(cod_ctx* c, int layer, const void* q, const void* kb, const void* vb, const cod_state* stt,
+                       int S, int use_carry, void* out, float* tap, float* mass, cudaStream_t st) {
+  const int M = c->cfg.block * (c->cfg.n_q_heads / c->cfg.n_kv_heads);
+  if (M <= 64) return launch<true>(c, layer, q, kb, vb, stt, S, use_carry, out, tap, mass, st);
+  return launch<false>(c, layer, q, kb, vb, stt, S, use_carry, out, tap, mass, st);
+}

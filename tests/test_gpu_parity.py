@@ -92,6 +92,9 @@ def _workloads():
         "small_bf16": small_bf16(S=3, W=16, n_layers=2, ctx=(40, 300)),
         "small_bf16_W32": small_bf16(S=2, W=32, n_layers=1, ctx=(100, 200)),
         "small_bf16_W8": small_bf16(S=5, W=8, n_layers=1, ctx=(0, 50)),
+        # contexts long enough for several pipeline iterations per CTA (ring slots get reused)
+        "long_bf16": small_bf16(S=2, W=16, n_layers=1, ctx=(700, 1500)),
+        "long_bf16_W32": small_bf16(S=2, W=32, n_layers=1, ctx=(500, 900)),
         # wide enough for split-K, several token tiles with a ragged last one, a ragged vocab tile
         "mid_bf16": small_bf16(S=34, W=16, n_layers=2, ctx=(100, 600), d_target=512, n_cap=5, d_model=1024,
                                n_q=8, n_kv=2, vocab=3000),
@@ -180,7 +183,8 @@ def _set_carry(P, rng, lens):
 
 
 @pytest.mark.parametrize("name,split_len", [("tiny_f32", 32), ("tiny_f32", 0), ("small_bf16", 64),
-                                            ("small_bf16_W32", 32), ("small_bf16_W8", 0)])
+                                            ("small_bf16_W32", 32), ("small_bf16_W8", 0), ("long_bf16", 1024),
+                                            ("long_bf16", 256), ("long_bf16_W32", 512), ("mid_bf16", 0)])
 def test_block_attn_parity(name, split_len):
     B, Hn = _B(), _H()
     wl = _workloads()[name]
