@@ -268,13 +268,14 @@ def run_gpu(args):
         state.kv_pool[l].copy_(torch.randn(state.kv_pool[l].shape, generator=gen, device="cuda",
                                            dtype=torch.float32).to(state.kv_pool.dtype))
     ring = 8
-    toks, Hs = host_rounds(wl, seed, n_rounds, ring)
+    toks, Hs = host_rounds(wl, seed, ring, ring)           # inputs repeat with period 8 (open loop)
     H_pin = [torch.from_numpy(h).to(B.torch_dtype(sh.dtype)).pin_memory() for h in Hs]
     d_pin = [torch.from_numpy(t[0]).pin_memory() for t in toks]
     t_pin = [torch.from_numpy(t[1]).pin_memory() for t in toks]
     H_dev = [h.cuda() for h in H_pin]
     d_dev = [d.cuda() for d in d_pin]
     t_dev = [t.cuda() for t in t_pin]
+    stage_H, stage_d, stage_t = torch.empty_like(H_dev[0]), torch.empty_like(d_dev[0]), torch.empty_like(t_dev[0])
     next_draft = torch.zeros((wl.S, sh.W), dtype=torch.int32, device="cuda")
     L0 = state.committed_len.clone()
 
@@ -288,21 +289,54 @@ def run_gpu(args):
             dist.barrier()
         torch.cuda.synchronize()
 
-    def timed_pass(mode, e2e=False, profile=(), K=K):
+    def launch_round(i, mode, staged=False):
+        if staged:
+            ctx.draft_round(stage_d, stage_t, stage_H, wl.S, wl.n_forced, mode, state, None, next_draft, None)
+        else:
+            ctx.draft_round(d_dev[i], t_dev[i], H_dev[i], wl.S, wl.n_forced, mode, state, None, next_draft, None)
+
+    # One CUDA graph per input slot (and one bound to the staging buffers for the end-to-end
+    # pass): a replay enqueues the round's ~40 kernels with a single launch.
+    graphs = {}
+
+    def graph_for(i, mode, staged=False):
+        key = (i, mode, staged)
+        if key not in graphs:
+            side = torch.cuda.Stream()
+            side.wait_stream(torch.cuda.current_stream())
+            with torch.cuda.stream(side):                   # warm-up outside capture
+                launch_round(i, mode, staged)
+            torch.cuda.current_stream().wait_stream(side)
+            torch.cuda.synchronize()
+            g = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(g):
+                launch_round(i, mode, staged)
+            graphs[key] = g
+        return graphs[key]
+
+    def timed_pass(mode, e2e=False, profile=(), K=K, use_graph=True):
+        reset()
+        if use_graph:
+            for i in range(1 if e2e else ring):
+                graph_for(0 if e2e else i, mode, staged=e2e)
         reset()
         ctx.profile_enable(())
-        stage_H = torch.empty_like(H_dev[0])
-        stage_d = torch.empty_like(d_dev[0])
-        stage_t = torch.empty_like(t_dev[0])
 
         def step(r):
+            i = r % ring
             if e2e:
-                stage_H.copy_(H_pin[r % ring], non_blocking=True)
-                stage_d.copy_(d_pin[r], non_blocking=True)
-                stage_t.copy_(t_pin[r], non_blocking=True)
-                ctx.draft_round(stage_d, stage_t, stage_H, wl.S, wl.n_forced, mode, state, None, next_draft, None)
+                stage_H.copy_(H_pin[i], non_blocking=True)
+                stage_d.copy_(d_pin[i], non_blocking=True)
+                stage_t.copy_(t_pin[i], non_blocking=True)
+                if use_graph:
+                    graphs[(0, mode, True)].replay()
+                else:
+                    launch_round(i, mode, staged=True)
                 return next_draft.cpu()
-            ctx.draft_round(d_dev[r], t_dev[r], H_dev[r % ring], wl.S, wl.n_forced, mode, state, None, next_draft, None)
+            if use_graph:
+                graphs[(i, mode, False)].replay()
+            else:
+                launch_round(i, mode)
             return None
 
         for r in range(Wm):
@@ -328,7 +362,7 @@ def run_gpu(args):
     L_run = lay["committed_len"].astype(np.int64).copy()
     models = []
     for r in range(n_rounds):
-        m = toks[r][2].astype(np.int64)
+        m = toks[r % ring][2].astype(np.int64)
         L_run = L_run + m
         if r >= Wm:
             models.append(round_model(wl, L_run, sh.W - m, wl.R, es))
@@ -337,14 +371,18 @@ def run_gpu(args):
     t_class = {k: max(b / (peaks["hbm_gbs"] * 1e9), f / (peaks["tflops"] * 1e12)) for k, (b, f) in mean_model.items()}
     dominant = max(t_class, key=t_class.get)
 
-    with ClockSampler(local) as clk:
-        ms, launches = timed_pass(B.COD_CARRY, profile=(dominant,))
+    # stream launches first (also counts the kernels of a round and times the dominant one) ...
+    ms_stream, launches = timed_pass(B.COD_CARRY, profile=(dominant,), use_graph=False)
     dom_ms, dom_n = ctx.profile_read(dominant)
-    ms_base, _ = timed_pass(B.COD_BASELINE)
-    ms_e2e, _ = timed_pass(B.COD_CARRY, e2e=True)
     K_prof = min(K, 32)                                     # bounded by the library's event slots
-    timed_pass(B.COD_CARRY, profile=B.KERNEL_CLASSES, K=K_prof)
+    timed_pass(B.COD_CARRY, profile=B.KERNEL_CLASSES, K=K_prof, use_graph=False)
     per_class = {k: ctx.profile_read(k) for k in B.KERNEL_CLASSES}
+    # ... then the same rounds replayed as CUDA graphs: the headline numbers
+    use_graph = not args.no_graph
+    with ClockSampler(local) as clk:
+        ms, _ = timed_pass(B.COD_CARRY, use_graph=use_graph)
+    ms_base, _ = timed_pass(B.COD_BASELINE, use_graph=use_graph)
+    ms_e2e, _ = timed_pass(B.COD_CARRY, e2e=True, use_graph=use_graph)
     status = ctx.poll_status()
 
     if rank != 0:
@@ -391,7 +429,9 @@ def run_gpu(args):
         "dtype": sh.dtype, "data": "synthetic",
         "config": {"workload": wl.name, "batch": wl.S, "block": sh.W, "context": list(wl.ctx),
                    "drafter_layers": sh.n_layers, "vocab": sh.vocab, "parallelism": f"replicas x{world}",
-                   "l2": "inputs larger than L2 (weights re-read every round)"},
+                   "l2": "inputs larger than L2 (weights re-read every round)",
+                   "launch": "cuda_graph" if use_graph else "stream"},
+        "stream_us_per_round": ms_stream / K * 1e3,
         "us_per_round": us_round, "seq_rounds_per_s": world * wl.S * K / (ms * 1e-3),
         "carryover_overhead_pct": 100.0 * (ms - ms_base) / ms_base,
         "baseline_us_per_round": ms_base / K * 1e3,
@@ -409,6 +449,63 @@ def run_gpu(args):
         dist.destroy_process_group()
 
 
+def run_micro(args):
+    """--micro attn|lmhead: one entry point alone on the workload's shapes (one drafter layer, so the
+    device footprint stays small enough for a profiler capture). Prints its own JSON line."""
+    import torch
+
+    import __graft_entry__ as entry
+    from paper_2609_14717_b200 import binding as B
+
+    entry.build()
+    torch.cuda.set_device(0)
+    peaks = load_peaks()
+    wl = synth.scaled(bench_workload(args.workload, 4), n_layers=1)
+    sh = wl.shape
+    lay = synth.make_layout(wl, args.seed)
+    n_pages, mp = int(lay["n_pages"]), int(lay["max_pages_per_seq"])
+    cfg = B.make_config(sh, wl.S, mp, n_pages)
+    ctx = B.Context(cfg)
+    td = B.torch_dtype(sh.dtype)
+    gen = torch.Generator(device="cuda").manual_seed(args.seed)
+    rnd = lambda *shape, scale=1.0: (torch.randn(*shape, generator=gen, device="cuda") * scale).to(td)
+    K, Wm = args.steps, args.warmup
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    if args.micro == "attn":
+        state = B.State(cfg, sh.dtype, wl.S, lay["block_table"], lay["committed_len"])
+        state.kv_pool.copy_(rnd(*state.kv_pool.shape))
+        state.carry_kv.copy_(rnd(*state.carry_kv.shape))
+        state.carry_len.fill_(sh.W // 2)
+        q, kb, vb = rnd(wl.S, sh.W, sh.n_q, sh.hd), rnd(wl.S, sh.W, sh.n_kv, sh.hd), rnd(wl.S, sh.W, sh.n_kv, sh.hd)
+        out = torch.empty_like(q)
+        call = lambda: ctx.block_attn(0, q, kb, vb, state, wl.S, 1, out)
+        L = lay["committed_len"].astype(np.int64)
+        nbytes = float(np.sum(L + sh.W // 2) * 2 * sh.n_kv * sh.hd * 2 + 2 * q.numel() * 2)
+        flops = 4.0 * sh.W * sh.n_q * sh.hd * float(np.sum(L + sh.W // 2 + sh.W))
+    else:
+        w = {k: (rnd(*v, scale=0.02) if k not in ("g_hidden", "g_attn", "g_final") else torch.ones(*v, device="cuda", dtype=td))
+             for k, v in synth.weight_shapes(sh).items()}
+        ctx.set_weights(w)
+        x = torch.randn(wl.R, sh.d_model, generator=gen, device="cuda")
+        tok = torch.zeros(wl.R, dtype=torch.int32, device="cuda")
+        call = lambda: ctx.lm_head_argmax(x, wl.R, tok)
+        nbytes = float(sh.vocab * sh.d_model * 2 + wl.R * sh.d_model * 2)
+        flops = 2.0 * wl.R * sh.d_model * sh.vocab
+    for _ in range(Wm):
+        call()
+    torch.cuda.synchronize()
+    ev0.record()
+    for _ in range(K):
+        call()
+    ev1.record()
+    torch.cuda.synchronize()
+    us = ev0.elapsed_time(ev1) / K * 1e3
+    print(json.dumps({"micro": args.micro, "workload": wl.name, "us_per_call": us, "GBps": nbytes / us / 1e3,
+                      "TFLOPs": flops / us / 1e6, "hbm_frac": nbytes / us / 1e3 / peaks["hbm_gbs"],
+                      "tensor_frac": flops / us / 1e6 / peaks["tflops"], "device_status": ctx.poll_status()}))
+    ctx.close()
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -418,10 +515,15 @@ def main():
     ap.add_argument("--workload", default="cfg2", choices=["cfg1", "cfg2", "cfg3", "cfg4", "cfg5"])
     ap.add_argument("--seed", type=int, default=0)
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-graph", action="store_true", help="time plain stream launches instead of graph replays")
+    ap.add_argument("--micro", default=None, choices=["attn", "lmhead"],
+                    help="time one entry point alone (small footprint; meant for profiler captures)")
     args = ap.parse_args()
     if args.warmup < 3:
         args.warmup = 3
-    if args.impl == "reference":
+    if args.micro:
+        run_micro(args)
+    elif args.impl == "reference":
         run_reference(args)
     else:
         run_gpu(args)

@@ -124,7 +124,7 @@ int cod_create(const cod_config* cfg, cod_ctx** out) {
   if (!(f.rope_theta > 0.f) || !(f.rms_eps >= 0.f)) return COD_ERR_INVALID_ARG;
   if (f.head_dim != 64 && f.head_dim != 128) return COD_ERR_UNSUPPORTED;
   if (f.block > COD_MAX_W || f.block * (f.n_q_heads / f.n_kv_heads) > 128) return COD_ERR_UNSUPPORTED;
-  if ((f.d_target * f.n_cap) % 8 || f.d_model % 8) return COD_ERR_UNSUPPORTED;
+  if ((f.d_target * f.n_cap) % 8 || f.d_model % 8 || f.d_model > 32768) return COD_ERR_UNSUPPORTED;
   if ((f.n_kv_heads * f.head_dim) % 64) return COD_ERR_UNSUPPORTED;
   if (static_cast<int64_t>(f.n_pages) * f.page_size > (1ll << 31) - 1) return COD_ERR_UNSUPPORTED;
 
@@ -150,16 +150,16 @@ int cod_create(const cod_config* cfg, cod_ctx** out) {
     const int M = f.block * (f.n_q_heads / f.n_kv_heads);
     const int64_t cap = static_cast<int64_t>(f.max_pages_per_seq) * f.page_size;
     int64_t sl;
-    if (f.attn_split_len > 0) sl = (f.attn_split_len + 127) / 128 * 128;
+    if (f.attn_split_len > 0) sl = (f.attn_split_len + 127) / 128 * 128 > 4096 ? 4096 : (f.attn_split_len + 127) / 128 * 128;
     else {
       sl = (cap * f.max_batch * f.n_kv_heads / (8 * static_cast<int64_t>(c->n_sm)) + 127) / 128 * 128;
       if (sl < 128) sl = 128;
       if (sl > 2048) sl = 2048;
     }
     c->tc_split_len = static_cast<int>(sl);
-    const int keys_it = M <= 64 ? 128 : 64, ring = M <= 64 ? 2 : 4;
+    const int keys_it = M <= 64 ? 128 : 64, ring = M <= 64 ? 1 : 2;
     const bool tail_fits = (15 + 2 * f.block + keys_it - 1) / keys_it <= ring;
-    c->tc_max_parts = tail_fits ? static_cast<int>((cap + sl - 1) / sl + 1) * (M <= 64 ? 2 : 1) : 0;
+    c->tc_max_parts = tail_fits ? static_cast<int>((cap + sl - 1) / sl + 1) : 0;
   }
   c->ws = nullptr;
   c->ws_bytes = carve(c);

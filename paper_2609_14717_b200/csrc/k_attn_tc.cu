@@ -27,10 +27,10 @@
 namespace {
 
 constexpr int HD = 128, PAGE = 16, KT = 64;           // head size, page size, keys per tile
-constexpr int NTHREADS = 192;
+constexpr int NTHREADS = 224;     // 4 softmax warps, K producer, MMA issuer, V producer
 constexpr uint32_t TILE_BYTES = KT * HD * 2;           // one 64-key K or V tile: 16 KB
 constexpr uint32_t HALF_BYTES = KT * 128;              // 64 keys x 64 elements: 8 KB
-constexpr unsigned long long WAIT_LIMIT_NS = 2000000000ull;
+constexpr long long WAIT_LIMIT_CYCLES = 4000000000ll;
 
 struct AttnParams {
   const __nv_bfloat16 *q, *kb, *vb;     // rotated q [R, n_q*hd]; rotated k_blk, v_blk [R, n_kv*hd]
@@ -64,19 +64,20 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
       : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
   return ok != 0;
 }
-__device__ __forceinline__ unsigned long long global_ns() {
-  unsigned long long t;
-  asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
-  return t;
-}
+// Bounded wait. The common case (phase already complete, or completing within a few polls) never
+// reads a timer; after that the SM cycle counter bounds the wait (about 2 s at the maximum clock),
+// then the CTA raises COD_DEV_TIMEOUT and every role leaves through the abort flag.
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, uint32_t* status) {
-  const unsigned long long t0 = global_ns();
+#pragma unroll 1
+  for (int i = 0; i < 64; ++i)
+    if (mbar_try_wait(bar, parity)) return true;
+  const long long t0 = clock64();
   for (;;) {
 #pragma unroll 1
     for (int i = 0; i < 256; ++i)
       if (mbar_try_wait(bar, parity)) return true;
     if (*abort_flag) return false;
-    if (global_ns() - t0 > WAIT_LIMIT_NS) {
+    if (clock64() - t0 > WAIT_LIMIT_CYCLES) {
       *abort_flag = 1;
       atomicOr(status, COD_DEV_TIMEOUT);
       return false;
@@ -117,6 +118,23 @@ __device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&v)[32]) {
         "=r"(v[24]), "=r"(v[25]), "=r"(v[26]), "=r"(v[27]), "=r"(v[28]), "=r"(v[29]), "=r"(v[30]), "=r"(v[31])
       : "r"(taddr) : "memory");
   asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+}
+
+__device__ __forceinline__ void tmem_st32(uint32_t taddr, const uint32_t (&v)[32]) {
+  asm volatile(
+      "tcgen05.st.sync.aligned.32x32b.x32.b32 [%0], "
+      "{%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31,%32};"
+      ::"r"(taddr), "r"(v[0]), "r"(v[1]), "r"(v[2]), "r"(v[3]), "r"(v[4]), "r"(v[5]), "r"(v[6]), "r"(v[7]),
+        "r"(v[8]), "r"(v[9]), "r"(v[10]), "r"(v[11]), "r"(v[12]), "r"(v[13]), "r"(v[14]), "r"(v[15]),
+        "r"(v[16]), "r"(v[17]), "r"(v[18]), "r"(v[19]), "r"(v[20]), "r"(v[21]), "r"(v[22]), "r"(v[23]),
+        "r"(v[24]), "r"(v[25]), "r"(v[26]), "r"(v[27]), "r"(v[28]), "r"(v[29]), "r"(v[30]), "r"(v[31])
+      : "memory");
+  asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
+}
+__device__ __forceinline__ float ex2_approx(float x) {
+  float y;
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
 }
 
 // K-major operand, 128-byte rows, 128-byte swizzle, 8-row groups 1024 bytes apart.
@@ -168,9 +186,9 @@ struct Geo {
   static constexpr uint32_t OFF_K = OFF_P + 2 * P_BUF;
   static constexpr uint32_t OFF_V = OFF_K + NK * SLOT;
   static constexpr uint32_t OFF_CTL = OFF_V + NV * SLOT;
-  static constexpr uint32_t SMEM = OFF_CTL + 256 + 1024;
-  // tensor memory columns: S[2] (64 each) then O[2] (128 each)
-  static constexpr uint32_t COL_S = 0, COL_O = 128, TMEM_COLS = 512;
+  static constexpr uint32_t SMEM = OFF_CTL + 256 + 1024 + 1024;   // barriers, page ids, alignment slack
+  // tensor memory columns: S[2] (64 each) then O (128)
+  static constexpr uint32_t COL_S = 0, COL_O = 128, TMEM_COLS = 256;
 };
 
 template <bool DUAL>
@@ -191,6 +209,7 @@ k_attn_tc(const __grid_constant__ CUtensorMap map_pool, const __grid_constant__ 
   uint64_t* o_full = bars + 24;             // [2]
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 26);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+  int* page_ids = reinterpret_cast<int*>(bars + 28);       // [split_len / 16] <= 256 entries
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int split = blockIdx.x, h = blockIdx.y, s = blockIdx.z;
@@ -224,75 +243,73 @@ k_attn_tc(const __grid_constant__ CUtensorMap map_pool, const __grid_constant__ 
   // rows beyond the real query rows are zero.
   if (warp < 4) {
     const int qw = p.n_kv * p.rep * HD;
-    for (int idx = threadIdx.x; idx < G::MROWS * 16; idx += 128) {
-      const int r = idx >> 4, ch = idx & 15;
-      uint4 v = make_uint4(0u, 0u, 0u, 0u);
-      if (r < M) {
-        const int i = r / p.rep, gg = r - i * p.rep;
-        v = *reinterpret_cast<const uint4*>(p.q + static_cast<size_t>(s * p.W + i) * qw + (h * p.rep + gg) * HD + ch * 8);
+    constexpr int QB = 8;                                   // independent 16-byte loads in flight per thread
+    for (int idx0 = threadIdx.x; idx0 < G::MROWS * 16; idx0 += 128 * QB) {
+      uint4 v[QB];
+#pragma unroll
+      for (int u = 0; u < QB; ++u) {
+        const int idx = idx0 + u * 128, r = idx >> 4, ch = idx & 15;
+        v[u] = make_uint4(0u, 0u, 0u, 0u);
+        if (r < M) {
+          const int i = r / p.rep, gg = r - i * p.rep;
+          v[u] = *reinterpret_cast<const uint4*>(p.q + static_cast<size_t>(s * p.W + i) * qw + (h * p.rep + gg) * HD + ch * 8);
+        }
       }
-      const uint32_t off = (ch >> 3) * G::Q_HALF + r * 128 + (((ch & 7) ^ (r & 7)) << 4);
-      *reinterpret_cast<uint4*>(sm + off) = v;
+#pragma unroll
+      for (int u = 0; u < QB; ++u) {
+        const int idx = idx0 + u * 128, r = idx >> 4, ch = idx & 15;
+        *reinterpret_cast<uint4*>(sm + (ch >> 3) * G::Q_HALF + r * 128 + (((ch & 7) ^ (r & 7)) << 4)) = v[u];
+      }
     }
     fence_async_smem();
+  } else if (warp == 4 && !is_tail) {
+    // physical page of every logical page this CTA will touch, fetched once
+    for (int i = lane; i < (k_end - k_begin + PAGE - 1) / PAGE; i += 32) {
+      int pg = p.block_table[s * p.max_pages + k_begin / PAGE + i];
+      if (pg < 0 || pg >= p.n_pages) { flags |= COD_DEV_BAD_PAGE; pg = -1; }
+      page_ids[i] = pg;
+    }
+    __syncwarp();
   }
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
 
-  if (warp == 4) {
-    // ------------------------------------------------ TMA producer (paged region only)
+  if (warp == 4 || warp == 6) {
+    // ------------------------------------------------ TMA producers (paged region only): warp 4 streams
+    // the K tiles, warp 6 the V tiles, so the two rings are fed independently
     if (!is_tail) {
+      const bool is_v = warp == 6;
       const int pages_it = G::KEYS_IT / PAGE;           // 8 or 4 pages per iteration, one per lane
+      const int ring = is_v ? G::NV : G::NK;
+      uint64_t* full = is_v ? v_full : k_full;
+      uint64_t* empty = is_v ? v_empty : k_empty;
+      const uint32_t ring_off = is_v ? G::OFF_V : G::OFF_K;
       bool ok = true;
       for (int it = 0; it < n_it && ok; ++it) {
         const int key0 = k_begin + it * G::KEYS_IT + lane * PAGE;
-        int row_k = -1;                                 // first key row of this lane's page in the pool map
+        int row = -1;                                   // first row of this lane's page tile in the pool map
         if (lane < pages_it && key0 < k_end) {
-          int pg = p.block_table[s * p.max_pages + key0 / PAGE];
-          if (pg < 0 || pg >= p.n_pages) { flags |= COD_DEV_BAD_PAGE; }
-          else row_k = (((p.layer * p.n_pages + pg) * p.n_kv + h) * 2) * PAGE;
+          const int pg = page_ids[(key0 - k_begin) / PAGE];
+          if (pg >= 0) row = (((p.layer * p.n_pages + pg) * p.n_kv + h) * 2 + (is_v ? 1 : 0)) * PAGE;
         }
         const uint32_t in_slot = (lane / (KT / PAGE)) * TILE_BYTES + (lane % (KT / PAGE)) * (PAGE * 128);
-        // K
-        {
-          const int slot = it % G::NK, use = it / G::NK;
-          if (lane == 0 && use > 0) ok = mbar_wait(smem_u32(k_empty + slot), (use - 1) & 1, abort_flag, p.status);
-          ok = __shfl_sync(0xffffffffu, ok, 0);
-          if (!ok) break;
-          const uint32_t fb = smem_u32(k_full + slot);
-          if (lane == 0) mbar_expect_tx(fb, G::SLOT);
-          __syncwarp();
-          if (lane < pages_it) {
-            const uint32_t dst = base + G::OFF_K + slot * G::SLOT + in_slot;
-            if (row_k >= 0) {
-              tma_load_3d(dst, &map_pool, 0, 0, row_k, fb);
-              tma_load_3d(dst + HALF_BYTES, &map_pool, 0, 1, row_k, fb);
-            } else {
-              tma_load_3d(dst, &map_zero, 0, 0, 0, fb);
-              tma_load_3d(dst + HALF_BYTES, &map_zero, 0, 1, 0, fb);
-            }
-          }
-        }
-        // V
-        {
-          const int slot = it % G::NV, use = it / G::NV;
-          if (lane == 0 && use > 0) ok = mbar_wait(smem_u32(v_empty + slot), (use - 1) & 1, abort_flag, p.status);
-          ok = __shfl_sync(0xffffffffu, ok, 0);
-          if (!ok) break;
-          const uint32_t fb = smem_u32(v_full + slot);
-          if (lane == 0) mbar_expect_tx(fb, G::SLOT);
-          __syncwarp();
-          if (lane < pages_it) {
-            const uint32_t dst = base + G::OFF_V + slot * G::SLOT + in_slot;
-            if (row_k >= 0) {
-              tma_load_3d(dst, &map_pool, 0, 0, row_k + PAGE, fb);
-              tma_load_3d(dst + HALF_BYTES, &map_pool, 0, 1, row_k + PAGE, fb);
-            } else {
-              tma_load_3d(dst, &map_zero, 0, 0, 0, fb);
-              tma_load_3d(dst + HALF_BYTES, &map_zero, 0, 1, 0, fb);
-            }
+        const int slot = it % ring, use = it / ring;
+        if (lane == 0 && use > 0) ok = mbar_wait(smem_u32(empty + slot), (use - 1) & 1, abort_flag, p.status);
+        ok = __shfl_sync(0xffffffffu, ok, 0);
+        if (!ok) break;
+        const uint32_t fb = smem_u32(full + slot);
+        if (lane == 0) mbar_expect_tx(fb, G::SLOT);
+        __syncwarp();
+        if (lane < pages_it) {
+          const uint32_t dst = base + ring_off + slot * G::SLOT + in_slot;
+          if (row >= 0) {
+            tma_load_3d(dst, &map_pool, 0, 0, row, fb);
+            tma_load_3d(dst + HALF_BYTES, &map_pool, 0, 1, row, fb);
+          } else {
+            tma_load_3d(dst, &map_zero, 0, 0, 0, fb);
+            tma_load_3d(dst + HALF_BYTES, &map_zero, 0, 1, 0, fb);
           }
         }
       }
@@ -336,50 +353,40 @@ k_attn_tc(const __grid_constant__ CUtensorMap map_pool, const __grid_constant__ 
         for (int t = 0; t < G::TILES; ++t) {
           const uint64_t p_desc = desc_kmajor(base + G::OFF_P + (it & 1) * G::P_BUF + t * G::P_TILE);
           const uint64_t v_desc = desc_mnmajor(base + G::OFF_V + slot * G::SLOT + t * TILE_BYTES);
-          const uint32_t d = tmem_base + G::COL_O + (it & 1) * HD + (static_cast<uint32_t>(16 * t) << 16);
+          const uint32_t d = tmem_base + G::COL_O + (static_cast<uint32_t>(16 * t) << 16);
 #pragma unroll
           for (int kk = 0; kk < KT / 16; ++kk)       // 16 keys per MMA: 32 bytes along P's rows, 16 rows of V
-            umma_bf16(d, p_desc + kk * 2, v_desc + kk * ((16 * 128) >> 4), idesc_pv, kk ? 1u : 0u);
+            umma_bf16(d, p_desc + kk * 2, v_desc + kk * ((16 * 128) >> 4), idesc_pv, (it | kk) ? 1u : 0u);
         }
         umma_commit(smem_u32(o_full + (it & 1)));
         umma_commit(smem_u32(v_empty + slot));
       }
     }
   } else {
-    // ------------------------------------------------ softmax / accumulation: one thread per (row, tile)
+    // ------------------------------------------------ softmax: one thread per (row, tile)
+    // O = sum_j p_j v_j accumulates in tensor memory across iterations, relative to a per-row
+    // reference maximum m_ref. The reference only moves when the row maximum grows by more than
+    // 2^8 in probability terms (then this warp rescales its rows of O in tensor memory), so the
+    // common iteration touches S only: load scores, exponentiate, store P.
     const int T = threadIdx.x;
     const int tile = DUAL ? (lane >> 4) : 0;
     const int r = DUAL ? (16 * warp + (lane & 15)) : T;
     const uint32_t t_lane = tmem_base + (static_cast<uint32_t>(32 * warp) << 16);
-    const float sl2 = rsqrtf(static_cast<float>(HD)) * 1.4426950408889634f;
-    float m_run = -INFINITY, l_run = 0.f, lc_run = 0.f, corr_pending = 1.f;
-    float o_acc[HD];
-#pragma unroll
-    for (int d = 0; d < HD; ++d) o_acc[d] = 0.f;
+    const float sl2 = rsqrtf(static_cast<float>(HD)) * 1.4426950408889634f;   // raw score -> log2 units
+    const float rescale_gap = 8.f / sl2;
+    float m_ref = -INFINITY, l_run = 0.f, lc_run = 0.f;
     bool ok = true;
-
-    auto accumulate_o = [&](int it) -> bool {
-      if (!mbar_wait(smem_u32(o_full + (it & 1)), (it >> 1) & 1, abort_flag, p.status)) return false;
-      tc_fence_after();
-#pragma unroll
-      for (int q4 = 0; q4 < HD / 32; ++q4) {
-        uint32_t v[32];
-        tmem_ld32(t_lane + G::COL_O + (it & 1) * HD + q4 * 32, v);
-#pragma unroll
-        for (int j = 0; j < 32; ++j) o_acc[q4 * 32 + j] = fmaf(o_acc[q4 * 32 + j], corr_pending, __uint_as_float(v[j]));
-      }
-      return true;
-    };
 
     for (int it = 0; it < n_it && ok; ++it) {
       if (is_tail) {
         // gather this iteration's rows (partial page, carried rows, block rows) with plain loads
         const int kslot = it % G::NK, vslot = it % G::NV;
-        for (int idx0 = T; idx0 < G::KEYS_IT * 32; idx0 += 128 * 4) {
-          uint4 val[4];
-          uint32_t dst[4];
+        constexpr int GB = 8;                               // independent 16-byte loads in flight per thread
+        for (int idx0 = T; idx0 < G::KEYS_IT * 32; idx0 += 128 * GB) {
+          uint4 val[GB];
+          uint32_t dst[GB];
 #pragma unroll
-          for (int u = 0; u < 4; ++u) {
+          for (int u = 0; u < GB; ++u) {
             const int idx = idx0 + u * 128;
             const int ch = idx & 15, kv = (idx >> 4) & 1, j = idx >> 5;       // chunk, K|V, key within iteration
             const int g = it * G::KEYS_IT + j;
@@ -399,14 +406,14 @@ k_attn_tc(const __grid_constant__ CUtensorMap map_pool, const __grid_constant__ 
                      (ch >> 3) * HALF_BYTES + jj * 128 + (((ch & 7) ^ (jj & 7)) << 4);
           }
 #pragma unroll
-          for (int u = 0; u < 4; ++u) *reinterpret_cast<uint4*>(sm + dst[u]) = val[u];
+          for (int u = 0; u < GB; ++u) *reinterpret_cast<uint4*>(sm + dst[u]) = val[u];
         }
         fence_async_smem();
         mbar_arrive(smem_u32(k_full + kslot));
         mbar_arrive(smem_u32(v_full + vslot));
       }
 
-      ok = mbar_wait(smem_u32(s_full + (it & 1)), (it >> 1) & 1, abort_flag, p.status);
+      ok = __all_sync(0xffffffffu, mbar_wait(smem_u32(s_full + (it & 1)), (it >> 1) & 1, abort_flag, p.status));
       if (!ok) break;
       tc_fence_after();
       const int key_t0 = k_begin + it * G::KEYS_IT + tile * KT;         // first key of this thread's tile
@@ -421,16 +428,45 @@ k_attn_tc(const __grid_constant__ CUtensorMap map_pool, const __grid_constant__ 
 #pragma unroll
         for (int j = 0; j < 32; ++j) sc[32 + j] = __uint_as_float(v[j]);
       }
-      float mx = -INFINITY;
+      if (n_valid < KT) {                                  // only the last iteration of a split is ragged
 #pragma unroll
-      for (int j = 0; j < KT; ++j) {
-        sc[j] = j < n_valid ? sc[j] * sl2 : -INFINITY;
-        mx = fmaxf(mx, sc[j]);
+        for (int j = 0; j < KT; ++j) sc[j] = j < n_valid ? sc[j] : -INFINITY;
       }
-      const float m_new = fmaxf(m_run, mx);
-      const float m_use = m_new == -INFINITY ? 0.f : m_new;              // nothing valid yet: all p = 0
-      const float corr = exp2f(m_run - m_use);                            // exp2(-inf) = 0
-      float psum = 0.f, pcar = 0.f;
+      float mx4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};      // four independent chains
+#pragma unroll
+      for (int j = 0; j < KT; j += 4) {
+        mx4[0] = fmaxf(mx4[0], sc[j]); mx4[1] = fmaxf(mx4[1], sc[j + 1]);
+        mx4[2] = fmaxf(mx4[2], sc[j + 2]); mx4[3] = fmaxf(mx4[3], sc[j + 3]);
+      }
+      const float mx = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3]));
+      const bool need = mx > m_ref + rescale_gap;        // also true for the first finite maximum
+      if (__any_sync(0xffffffffu, need)) {
+        const float m_new = need ? mx : m_ref;
+        const float factor = need ? ex2_approx((m_ref - m_new) * sl2) : 1.f;     // ex2(-inf) = 0
+        if (it > 0) {
+          // O is relative to the old reference: once PV(it-1) has landed, scale this warp's rows
+          ok = __all_sync(0xffffffffu, mbar_wait(smem_u32(o_full + ((it - 1) & 1)), ((it - 1) >> 1) & 1, abort_flag, p.status));
+          if (!ok) break;
+          tc_fence_after();
+#pragma unroll
+          for (int q4 = 0; q4 < HD / 32; ++q4) {
+            uint32_t v[32];
+            tmem_ld32(t_lane + G::COL_O + q4 * 32, v);
+#pragma unroll
+            for (int j = 0; j < 32; ++j) v[j] = __float_as_uint(__uint_as_float(v[j]) * factor);
+            tmem_st32(t_lane + G::COL_O + q4 * 32, v);
+          }
+        }
+        l_run *= factor;
+        lc_run *= factor;
+        m_ref = m_new;
+      }
+      if (it >= 2) {   // the P buffer about to be overwritten was read by PV(it-2)
+        ok = __all_sync(0xffffffffu, mbar_wait(smem_u32(o_full + (it & 1)), ((it - 2) >> 1) & 1, abort_flag, p.status));
+        if (!ok) break;
+      }
+      const float neg = m_ref == -INFINITY ? 0.f : -m_ref * sl2;
+      float ps4[4] = {0.f, 0.f, 0.f, 0.f}, pcar = 0.f;
       uint8_t* prow = sm + G::OFF_P + (it & 1) * G::P_BUF + tile * G::P_TILE + r * 128;
       const int car0 = is_tail ? Lr - (it * G::KEYS_IT + tile * KT) : KT;  // carried keys: [car0, car0 + c)
 #pragma unroll
@@ -439,8 +475,8 @@ k_attn_tc(const __grid_constant__ CUtensorMap map_pool, const __grid_constant__ 
 #pragma unroll
         for (int e = 0; e < 4; ++e) {
           const int j = ch * 8 + e * 2;
-          const float p0 = exp2f(sc[j] - m_use), p1 = exp2f(sc[j + 1] - m_use);
-          psum += p0 + p1;
+          const float p0 = ex2_approx(fmaf(sc[j], sl2, neg)), p1 = ex2_approx(fmaf(sc[j + 1], sl2, neg));
+          ps4[e] += p0 + p1;
           if (is_tail) {
             if (j >= car0 && j < car0 + c) pcar += p0;
             if (j + 1 >= car0 && j + 1 < car0 + c) pcar += p1;
@@ -453,25 +489,54 @@ k_attn_tc(const __grid_constant__ CUtensorMap map_pool, const __grid_constant__ 
       fence_async_smem();
       tc_fence_before();
       mbar_arrive(smem_u32(p_full + (it & 1)));
-      l_run = l_run * corr + psum;
-      lc_run = lc_run * corr + pcar;
-      m_run = m_new;
-      if (it > 0) ok = accumulate_o(it - 1);
-      corr_pending = corr;
+      l_run += (ps4[0] + ps4[1]) + (ps4[2] + ps4[3]);
+      lc_run += pcar;
     }
-    if (ok && n_it > 0) ok = accumulate_o(n_it - 1);
 
-    // partial results of this (row, tile)
-    const int part = (DUAL ? 2 : 1) * split + tile;
-    if (r < M && (ok || n_it == 0)) {
-      const size_t rowi = ((static_cast<size_t>(s) * p.n_kv + h) * p.max_parts + part) * M + r;
-      float4* po = reinterpret_cast<float4*>(p.part_o + rowi * HD);
+    // partial result of this row: O from tensor memory once the last PV has landed. With two
+    // interleaved tiles, lanes l and l + 16 hold the same query row for different keys: they are
+    // merged with shuffles (log-sum-exp weights) so the CTA writes one partial per row.
+    if (ok && n_it > 0) {
+      ok = __all_sync(0xffffffffu, mbar_wait(smem_u32(o_full + ((n_it - 1) & 1)), ((n_it - 1) >> 1) & 1, abort_flag, p.status));
+      if (ok) {
+        tc_fence_after();
+        float w_me = 1.f, w_other = 0.f;
+        float m_out = m_ref;
+        if (DUAL) {
+          const float m_o = __shfl_xor_sync(0xffffffffu, m_ref, 16);
+          const float l_o = __shfl_xor_sync(0xffffffffu, l_run, 16), lc_o = __shfl_xor_sync(0xffffffffu, lc_run, 16);
+          m_out = fmaxf(m_ref, m_o);
+          const float base_m = m_out == -INFINITY ? 0.f : m_out;
+          w_me = ex2_approx((m_ref - base_m) * sl2);
+          w_other = ex2_approx((m_o - base_m) * sl2);
+          l_run = w_me * l_run + w_other * l_o;
+          lc_run = w_me * lc_run + w_other * lc_o;
+        }
+        const size_t rowi = ((static_cast<size_t>(s) * p.n_kv + h) * p.max_parts + split) * M + min(r, M - 1);
+        float4* po = reinterpret_cast<float4*>(p.part_o + rowi * HD);
 #pragma unroll
-      for (int d = 0; d < HD / 4; ++d) po[d] = make_float4(o_acc[4 * d], o_acc[4 * d + 1], o_acc[4 * d + 2], o_acc[4 * d + 3]);
-      float* ml = p.part_ml + rowi * 4;
-      ml[0] = m_run * 0.6931471805599453f;      // back to natural-log units
-      ml[1] = l_run;
-      ml[2] = lc_run;
+        for (int q4 = 0; q4 < HD / 32; ++q4) {
+          uint32_t v[32];
+          tmem_ld32(t_lane + G::COL_O + q4 * 32, v);
+          float o[32];
+#pragma unroll
+          for (int j = 0; j < 32; ++j) {
+            o[j] = __uint_as_float(v[j]) * w_me;
+            if (DUAL) o[j] += __shfl_xor_sync(0xffffffffu, __uint_as_float(v[j]), 16) * w_other;
+          }
+          // the two lanes of a row share the stores: even chunks from the first tile's lane
+          if (r < M && (!DUAL || ((q4 & 1) == tile))) {
+#pragma unroll
+            for (int j = 0; j < 8; ++j) po[q4 * 8 + j] = make_float4(o[4 * j], o[4 * j + 1], o[4 * j + 2], o[4 * j + 3]);
+          }
+        }
+        if (r < M && tile == 0) {
+          float* ml = p.part_ml + rowi * 4;
+          ml[0] = m_out * rsqrtf(static_cast<float>(HD));      // natural-log units of the scaled score
+          ml[1] = l_run;
+          ml[2] = lc_run;
+        }
+      }
     }
   }
 
@@ -504,19 +569,31 @@ __global__ void k_attn_tc_combine(const float* __restrict__ part_o, const float*
   const int h = g / rep, mrow = i * rep + (g - h * rep), M = W * rep;
   const int L = max(0, min(committed_len[s], max_pages * PAGE));
   const int F = (L / PAGE) * PAGE;
-  const int n_parts = ((F + split_len - 1) / split_len + 1) * (DUAL ? 2 : 1);
+  const int n_parts = (F + split_len - 1) / split_len + 1;
   const size_t base = (static_cast<size_t>(s) * n_kv + h) * max_parts;
+  // every lane fetches the (m, l, l_carry) record of its parts; weights stay in registers
   float mg = -INFINITY;
-  for (int k = 0; k < n_parts; ++k) mg = fmaxf(mg, part_ml[((base + k) * M + mrow) * 4]);
+  for (int k = lane; k < n_parts; k += 32) mg = fmaxf(mg, part_ml[((base + k) * M + mrow) * 4]);
+  mg = cod_warp_max(mg);
   float acc[4] = {0.f, 0.f, 0.f, 0.f}, l = 0.f, lc = 0.f;
-  for (int k = 0; k < n_parts; ++k) {
-    const float* ml = part_ml + ((base + k) * M + mrow) * 4;
-    const float w = __expf(ml[0] - mg);
-    l = fmaf(w, ml[1], l);
-    lc = fmaf(w, ml[2], lc);
-    const float4 v = *reinterpret_cast<const float4*>(part_o + ((base + k) * M + mrow) * HD + lane * 4);
-    acc[0] = fmaf(w, v.x, acc[0]); acc[1] = fmaf(w, v.y, acc[1]); acc[2] = fmaf(w, v.z, acc[2]); acc[3] = fmaf(w, v.w, acc[3]);
+  for (int k0 = 0; k0 < n_parts; k0 += 32) {
+    float w_mine = 0.f;
+    if (k0 + lane < n_parts) {
+      const float4 ml = *reinterpret_cast<const float4*>(part_ml + ((base + k0 + lane) * M + mrow) * 4);
+      w_mine = __expf(ml.x - mg);
+      l = fmaf(w_mine, ml.y, l);
+      lc = fmaf(w_mine, ml.z, lc);
+    }
+    const int nk = min(32, n_parts - k0);
+#pragma unroll 8
+    for (int k = 0; k < nk; ++k) {
+      const float w = __shfl_sync(0xffffffffu, w_mine, k);
+      const float4 v = *reinterpret_cast<const float4*>(part_o + ((base + k0 + k) * M + mrow) * HD + lane * 4);
+      acc[0] = fmaf(w, v.x, acc[0]); acc[1] = fmaf(w, v.y, acc[1]); acc[2] = fmaf(w, v.z, acc[2]); acc[3] = fmaf(w, v.w, acc[3]);
+    }
   }
+  l = cod_warp_sum(l);
+  lc = cod_warp_sum(lc);
   const float inv = 1.f / l;
   const size_t ob = static_cast<size_t>(item) * HD + lane * 4;
   const __nv_bfloat162 b0 = __floats2bfloat162_rn(acc[0] * inv, acc[1] * inv), b1 = __floats2bfloat162_rn(acc[2] * inv, acc[3] * inv);
@@ -580,7 +657,7 @@ int launch(cod_ctx* c, int layer, const void* q, const void* kb, const void* vb,
       return COD_ERR_CUDA;
     configured = true;
   }
-  dim3 grid(c->tc_max_parts / (DUAL ? 2 : 1), f.n_kv_heads, S);
+  dim3 grid(c->tc_max_parts, f.n_kv_heads, S);
   k_attn_tc<DUAL><<<grid, NTHREADS, G::SMEM, st>>>(mp, mz, p);
   COD_CHECK_LAUNCH(c);
   const int items = S * f.block * f.n_q_heads;

@@ -25,7 +25,7 @@ constexpr int BK = 64;        // K elements per stage = one 128-byte swizzled ro
 constexpr int UK = 16;        // K elements per tcgen05.mma (kind::f16)
 constexpr int NTHREADS = 192;
 constexpr uint32_t A_TILE_BYTES = BM * BK * 2;   // 16 KB
-constexpr unsigned long long WAIT_LIMIT_NS = 2000000000ull;
+constexpr long long WAIT_LIMIT_CYCLES = 4000000000ll;
 
 struct TcParams {
   int K;
@@ -35,6 +35,7 @@ struct TcParams {
   int NT;                     // token rows per CTA = MMA N (multiple of 16, <= 256)
   int tmem_cols;              // power of two >= max(32, NT)
   int stages;
+  int prefetch;
   int seg_tile_end[3];        // cumulative count of 128-row tiles after each weight segment
   int seg_N[3];
   int n_seg;
@@ -62,33 +63,37 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
       : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
   return ok != 0;
 }
-__device__ __forceinline__ unsigned long long global_ns() {
-  unsigned long long t;
-  asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
-  return t;
-}
-// Bounded wait: false if the limit expired or another role already gave up.
+// Bounded wait. The common case (phase already complete, or completing within a few polls) never
+// reads a timer; after that the SM cycle counter bounds the wait (about 2 s at the maximum clock),
+// then the CTA raises COD_DEV_TIMEOUT and every role leaves through the abort flag.
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, uint32_t* status) {
-  const unsigned long long t0 = global_ns();
+#pragma unroll 1
+  for (int i = 0; i < 64; ++i)
+    if (mbar_try_wait(bar, parity)) return true;
+  const long long t0 = clock64();
   for (;;) {
 #pragma unroll 1
     for (int i = 0; i < 256; ++i)
       if (mbar_try_wait(bar, parity)) return true;
     if (*abort_flag) return false;
-    if (global_ns() - t0 > WAIT_LIMIT_NS) {
+    if (clock64() - t0 > WAIT_LIMIT_CYCLES) {
       *abort_flag = 1;
       atomicOr(status, COD_DEV_TIMEOUT);
       return false;
     }
   }
 }
-
 __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, int c0, int c1, uint32_t bar) {
   asm volatile(
       "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
       ::"r"(dst), "l"(reinterpret_cast<uint64_t>(map)), "r"(c0), "r"(c1), "r"(bar) : "memory");
 }
 
+// brings a weight tile into L2 only: the HBM latency is paid long before the tile's ring slot frees up
+__device__ __forceinline__ void tma_prefetch_2d(const CUtensorMap* map, int c0, int c1) {
+  asm volatile("cp.async.bulk.prefetch.tensor.2d.L2.global.tile [%0, {%1, %2}];"
+               ::"l"(reinterpret_cast<uint64_t>(map)), "r"(c0), "r"(c1) : "memory");
+}
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
 
@@ -164,7 +169,7 @@ k_gemm_tc(const __grid_constant__ CUtensorMap map_w0, const __grid_constant__ CU
   uint64_t* acc_bar = full_bar + 32;                                   // accumulator ready
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(full_bar + 33);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
-  unsigned long long* red = reinterpret_cast<unsigned long long*>(full_bar + 34);   // [NT] argmax keys
+  unsigned long long* red = reinterpret_cast<unsigned long long*>(full_bar + 34);   // [4][NT] argmax keys, one row per epilogue warp
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int n_tile = blockIdx.x, m_tile = blockIdx.y, split = blockIdx.z;
@@ -191,7 +196,7 @@ k_gemm_tc(const __grid_constant__ CUtensorMap map_w0, const __grid_constant__ CU
     *abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
-  for (int t = threadIdx.x; t < p.NT; t += NTHREADS) red[t] = 0ull;
+  for (int t = threadIdx.x; t < 4 * p.NT; t += NTHREADS) red[t] = 0ull;
   if (warp == 5) tmem_alloc(smem_u32(tmem_slot), static_cast<uint32_t>(p.tmem_cols));
   tc_fence_before();
   __syncthreads();
@@ -201,7 +206,10 @@ k_gemm_tc(const __grid_constant__ CUtensorMap map_w0, const __grid_constant__ CU
   if (warp == 4) {
     // ------------------------------------------------ TMA producer
     if (lane == 0) {
+      const int pf = p.prefetch;                          // k-blocks of weights kept in flight towards L2
+      for (int it = p.stages; it < min(n_kb, p.stages + pf); ++it) tma_prefetch_2d(map_w, (kb0 + it) * BK, f0);
       for (int it = 0; it < n_kb; ++it) {
+        if (pf > 0 && it + p.stages + pf < n_kb) tma_prefetch_2d(map_w, (kb0 + it + p.stages + pf) * BK, f0);
         const int s = it % p.stages, use = it / p.stages;
         if (use > 0 && !mbar_wait(smem_u32(empty_bar + s), (use - 1) & 1, abort_flag, p.status)) break;
         const uint32_t fb = smem_u32(full_bar + s);
@@ -250,20 +258,23 @@ k_gemm_tc(const __grid_constant__ CUtensorMap map_w0, const __grid_constant__ CU
         }
       }
     } else if (ok) {
+      // per-token (max, lowest row) over this warp's 32 weight rows; lane j keeps column c + j
       for (int c = 0; c < p.NT; c += 16) {
         uint32_t v[16];
         tmem_ld16(t_lane + c, v);
+        unsigned long long mine = 0ull;
 #pragma unroll
         for (int j = 0; j < 16; ++j) {
           const unsigned u = f_ok ? order_key(__uint_as_float(v[j])) : 0u;
           const unsigned mx = __reduce_max_sync(0xffffffffu, u);
           const unsigned who = __ballot_sync(0xffffffffu, u == mx);
-          if (lane == 0) {
+          if (lane == j) {
             const int idx = col0 + warp * 32 + (__ffs(who) - 1);      // lowest weight row among equals
-            atomicMax(red + c + j, (static_cast<unsigned long long>(mx) << 32) |
-                                       static_cast<unsigned long long>(0xFFFFFFFFu - static_cast<unsigned>(idx)));
+            mine = (static_cast<unsigned long long>(mx) << 32) |
+                   static_cast<unsigned long long>(0xFFFFFFFFu - static_cast<unsigned>(idx));
           }
         }
+        if (lane < 16) red[warp * p.NT + c + lane] = mine;
       }
     }
   }
@@ -278,8 +289,14 @@ k_gemm_tc(const __grid_constant__ CUtensorMap map_w0, const __grid_constant__ CU
   }
   else if (p.amax != nullptr) {
     // the four epilogue warps merged their per-token keys in shared memory: one atomic per token
-    for (int t = threadIdx.x; t < p.NT; t += NTHREADS)
-      if (i0 + t < n_rows) atomicMax(p.amax + i0 + t, red[t]);
+    for (int t = threadIdx.x; t < p.NT; t += NTHREADS) {
+      if (i0 + t < n_rows) {
+        unsigned long long best = red[t];
+#pragma unroll
+        for (int w = 1; w < 4; ++w) best = red[w * p.NT + t] > best ? red[w * p.NT + t] : best;
+        atomicMax(p.amax + i0 + t, best);
+      }
+    }
   }
   if (warp == 5) {
     __syncwarp();
@@ -355,6 +372,7 @@ int cod_launch_gemm_tc(cod_ctx* c, const GemmArgs& g, cudaStream_t st) {
   if (stages > p.kb_per_split) stages = p.kb_per_split;
   if (stages < 1) stages = 1;
   p.stages = stages;
+  p.prefetch = 0;
   int tiles = 0;
   for (int i = 0; i < 3; ++i) {
     if (i < g.n_seg) {

@@ -4,6 +4,19 @@
 
 namespace {
 
+constexpr int ROW_MAXV = 8;   // float4 slots a thread keeps in registers: D <= 4 * ROW_MAXV * blockDim.x
+
+__device__ __forceinline__ void cod_st4(float* p, float4 v) { *reinterpret_cast<float4*>(p) = v; }
+__device__ __forceinline__ void cod_st4(__nv_bfloat16* p, float4 v) {
+  const __nv_bfloat162 a = __floats2bfloat162_rn(v.x, v.y), b = __floats2bfloat162_rn(v.z, v.w);
+  uint2 u;
+  u.x = *reinterpret_cast<const uint32_t*>(&a);
+  u.y = *reinterpret_cast<const uint32_t*>(&b);
+  *reinterpret_cast<uint2*>(p) = u;
+}
+__device__ __forceinline__ float4 f4_add(float4 a, float4 b) { return make_float4(a.x + b.x, a.y + b.y, a.z + b.z, a.w + b.w); }
+__device__ __forceinline__ float f4_ss(float4 a) { return a.x * a.x + a.y * a.y + a.z * a.z + a.w * a.w; }
+
 __device__ __forceinline__ int valid_rows(const int* n_rows_dev, int n_rows) {
   return n_rows_dev ? min(*n_rows_dev, n_rows) : n_rows;
 }
@@ -43,27 +56,39 @@ __global__ void k_fc_finish(const float* __restrict__ part, int splits, int n_ro
                             const int* __restrict__ a_rows, const int* __restrict__ carry_slot,
                             const float* __restrict__ fcE, const T* __restrict__ gain, int D, float eps,
                             int do_norm, T* __restrict__ z, int z_compact, float* __restrict__ tap) {
-  extern __shared__ float sh[];   // [D] values + 33 reduction slots
-  float* vals = sh;
-  float* red = sh + D;
+  __shared__ float red[33];
   const int i = blockIdx.x;
   if (i >= valid_rows(n_rows_dev, n_rows)) return;
   const int row = a_rows ? a_rows[i] : i;
   const bool rej = carry_slot[row] >= 0;
+  const int nv = D >> 2;
+  float4 v[ROW_MAXV];
   float ss = 0.f;
-  for (int d = threadIdx.x; d < D; d += blockDim.x) {
-    float v = 0.f;
-    for (int s = 0; s < splits; ++s) v += part[(static_cast<size_t>(s) * n_rows + i) * D + d];
-    if (rej) v += fcE[d];
-    vals[d] = v;
-    ss = fmaf(v, v, ss);
+#pragma unroll
+  for (int t = 0; t < ROW_MAXV; ++t) {
+    const int j = threadIdx.x + t * blockDim.x;
+    v[t] = make_float4(0.f, 0.f, 0.f, 0.f);
+    if (j < nv) {
+      for (int s = 0; s < splits; ++s)
+        v[t] = f4_add(v[t], *reinterpret_cast<const float4*>(part + (static_cast<size_t>(s) * n_rows + i) * D + 4 * j));
+      if (rej) v[t] = f4_add(v[t], *reinterpret_cast<const float4*>(fcE + 4 * j));
+      ss += f4_ss(v[t]);
+    }
   }
   ss = cod_block_sum(ss, red);
   const float scale = do_norm ? rsqrtf(ss / static_cast<float>(D) + eps) : 1.f;
-  for (int d = threadIdx.x; d < D; d += blockDim.x) {
-    const float v = do_norm ? vals[d] * scale * cod_ld(gain + d) : vals[d];
-    cod_st(z + static_cast<size_t>(z_compact ? i : row) * D + d, v);
-    if (tap) tap[static_cast<size_t>(row) * D + d] = v;
+#pragma unroll
+  for (int t = 0; t < ROW_MAXV; ++t) {
+    const int j = threadIdx.x + t * blockDim.x;
+    if (j < nv) {
+      float4 o = v[t];
+      if (do_norm) {
+        const float4 g = cod_ld4(gain + 4 * j);
+        o = make_float4(o.x * scale * g.x, o.y * scale * g.y, o.z * scale * g.z, o.w * scale * g.w);
+      }
+      cod_st4(z + static_cast<size_t>(z_compact ? i : row) * D + 4 * j, o);
+      if (tap) *reinterpret_cast<float4*>(tap + static_cast<size_t>(row) * D + 4 * j) = o;
+    }
   }
 }
 
@@ -183,16 +208,30 @@ __global__ void k_embed_norm(const T* __restrict__ emb, const int* __restrict__ 
   const int r = blockIdx.x, s = r / W, p = r - s * W;
   int tok = p == 0 ? bonus[s] : mask_id;
   if (tok < 0 || tok >= vocab) tok = 0;
+  const int nv = D >> 2;
+  float4 v[ROW_MAXV];
   float ss = 0.f;
-  for (int d = threadIdx.x; d < D; d += blockDim.x) {
-    const float v = cod_ld(emb + static_cast<size_t>(tok) * D + d);
-    x[static_cast<size_t>(r) * D + d] = v;
-    ss = fmaf(v, v, ss);
+#pragma unroll
+  for (int t = 0; t < ROW_MAXV; ++t) {
+    const int j = threadIdx.x + t * blockDim.x;
+    v[t] = make_float4(0.f, 0.f, 0.f, 0.f);
+    if (j < nv) {
+      v[t] = cod_ld4(emb + static_cast<size_t>(tok) * D + 4 * j);
+      *reinterpret_cast<float4*>(x + static_cast<size_t>(r) * D + 4 * j) = v[t];
+      ss += f4_ss(v[t]);
+    }
   }
   ss = cod_block_sum(ss, red);
   const float scale = rsqrtf(ss / static_cast<float>(D) + eps);
-  for (int d = threadIdx.x; d < D; d += blockDim.x)
-    cod_st(a + static_cast<size_t>(r) * D + d, x[static_cast<size_t>(r) * D + d] * scale * cod_ld(gain + d));
+#pragma unroll
+  for (int t = 0; t < ROW_MAXV; ++t) {
+    const int j = threadIdx.x + t * blockDim.x;
+    if (j < nv) {
+      const float4 g = cod_ld4(gain + 4 * j);
+      cod_st4(a + static_cast<size_t>(r) * D + 4 * j,
+              make_float4(v[t].x * scale * g.x, v[t].y * scale * g.y, v[t].z * scale * g.z, v[t].w * scale * g.w));
+    }
+  }
   if (threadIdx.x == 0) amax[r] = 0ull;
 }
 
@@ -202,28 +241,28 @@ template <typename T>
 __global__ void k_qkv_finish(const float* __restrict__ part, int splits, int R, int n_q, int n_kv, int hd,
                              const float* __restrict__ rope_blk, T* __restrict__ q, T* __restrict__ kb,
                              T* __restrict__ vb) {
-  const int r = blockIdx.x;
+  // one block per (row, head): heads 0..n_q-1 are q, then n_kv heads of k (both rotated), then n_kv of v
+  const int r = blockIdx.x, hh = blockIdx.y;
   const int qw = n_q * hd, kvw = n_kv * hd, half = hd >> 1, ldc = qw + 2 * kvw;
   const float* cs = rope_blk + static_cast<size_t>(r) * hd;
-  const int n_rot = (n_q + n_kv) * half;
-  for (int e = threadIdx.x; e < n_rot + kvw; e += blockDim.x) {
-    if (e < n_rot) {
-      const int h = e / half, j = e - h * half;        // heads 0..n_q-1 are q, then k
-      float a = 0.f, b = 0.f;
-      for (int s = 0; s < splits; ++s) {
-        const float* p = part + (static_cast<size_t>(s) * R + r) * ldc + h * hd;
-        a += p[j];
-        b += p[j + half];
-      }
+  const bool rot = hh < n_q + n_kv;
+  T* dst = hh < n_q ? q + static_cast<size_t>(r) * qw + hh * hd
+                    : (rot ? kb + static_cast<size_t>(r) * kvw + (hh - n_q) * hd
+                           : vb + static_cast<size_t>(r) * kvw + (hh - n_q - n_kv) * hd);
+  for (int j = threadIdx.x; j < half; j += blockDim.x) {
+    float a = 0.f, b = 0.f;
+    for (int s = 0; s < splits; ++s) {
+      const float* p = part + (static_cast<size_t>(s) * R + r) * ldc + hh * hd;
+      a += p[j];
+      b += p[j + half];
+    }
+    if (rot) {
       const float c = cs[j], sn = cs[half + j];
-      T* dst = h < n_q ? q + static_cast<size_t>(r) * qw + h * hd : kb + static_cast<size_t>(r) * kvw + (h - n_q) * hd;
       cod_st(dst + j, a * c - b * sn);
       cod_st(dst + j + half, b * c + a * sn);
     } else {
-      const int d = e - n_rot;
-      float v = 0.f;
-      for (int s = 0; s < splits; ++s) v += part[(static_cast<size_t>(s) * R + r) * ldc + qw + kvw + d];
-      cod_st(vb + static_cast<size_t>(r) * kvw + d, v);
+      cod_st(dst + j, a);
+      cod_st(dst + j + half, b);
     }
   }
 }
@@ -254,19 +293,35 @@ __global__ void k_resid_norm(const float* __restrict__ part, int splits, int R, 
                              unsigned long long* __restrict__ amax) {
   __shared__ float red[33];
   const int r = blockIdx.x;
+  const int nv = D >> 2;
+  float4 v[ROW_MAXV];
   float ss = 0.f;
-  for (int d = threadIdx.x; d < D; d += blockDim.x) {
-    float v = x[static_cast<size_t>(r) * D + d];
-    if (part)
-      for (int s = 0; s < splits; ++s) v += part[(static_cast<size_t>(s) * R + r) * D + d];
-    if (part) x[static_cast<size_t>(r) * D + d] = v;   // without partials x is read-only input
-    if (tap) tap[static_cast<size_t>(r) * D + d] = v;
-    ss = fmaf(v, v, ss);
+#pragma unroll
+  for (int t = 0; t < ROW_MAXV; ++t) {
+    const int j = threadIdx.x + t * blockDim.x;
+    v[t] = make_float4(0.f, 0.f, 0.f, 0.f);
+    if (j < nv) {
+      v[t] = *reinterpret_cast<const float4*>(x + static_cast<size_t>(r) * D + 4 * j);
+      if (part) {
+        for (int s = 0; s < splits; ++s)
+          v[t] = f4_add(v[t], *reinterpret_cast<const float4*>(part + (static_cast<size_t>(s) * R + r) * D + 4 * j));
+        *reinterpret_cast<float4*>(x + static_cast<size_t>(r) * D + 4 * j) = v[t];   // without partials x is read-only
+      }
+      if (tap) *reinterpret_cast<float4*>(tap + static_cast<size_t>(r) * D + 4 * j) = v[t];
+      ss += f4_ss(v[t]);
+    }
   }
   ss = cod_block_sum(ss, red);
   const float scale = rsqrtf(ss / static_cast<float>(D) + eps);
-  for (int d = threadIdx.x; d < D; d += blockDim.x)
-    cod_st(a + static_cast<size_t>(r) * D + d, x[static_cast<size_t>(r) * D + d] * scale * cod_ld(gain + d));
+#pragma unroll
+  for (int t = 0; t < ROW_MAXV; ++t) {
+    const int j = threadIdx.x + t * blockDim.x;
+    if (j < nv) {
+      const float4 g = cod_ld4(gain + 4 * j);
+      cod_st4(a + static_cast<size_t>(r) * D + 4 * j,
+              make_float4(v[t].x * scale * g.x, v[t].y * scale * g.y, v[t].z * scale * g.z, v[t].w * scale * g.w));
+    }
+  }
   if (amax && threadIdx.x == 0) amax[r] = 0ull;
 }
 
@@ -282,6 +337,8 @@ __global__ void k_finalize(const unsigned long long* __restrict__ amax, int R, i
 }
 
 }  // namespace
+
+static inline int row_threads(int D) { return D <= 4 * ROW_MAXV * 256 ? 256 : 1024; }
 
 #define DISPATCH_T(c, CALL_BF16, CALL_F32) \
   do {                                     \
@@ -312,11 +369,11 @@ int cod_launch_fc_finish(cod_ctx* c, const float* part, int splits, int n_rows, 
                          const int* a_rows, const int* carry_slot, float* tap_z, cudaStream_t st) {
   ProfScope prof(c, COD_K_ROWOPS, st);
   if (n_rows <= 0) return COD_OK;
-  const size_t smem = (c->D + 33) * sizeof(float);
+  const int nt = row_threads(c->D);
   const int do_norm = (c->cfg.flags & COD_F_HIDDEN_NORM) ? 1 : 0;
   DISPATCH_T(c,
-             (k_fc_finish<__nv_bfloat16><<<n_rows, 256, smem, st>>>(part, splits, n_rows, n_rows_dev, a_rows, carry_slot, c->fcE, static_cast<const __nv_bfloat16*>(c->w.g_hidden), c->D, c->cfg.rms_eps, do_norm, static_cast<__nv_bfloat16*>(c->z), a_rows ? 1 : 0, tap_z)),
-             (k_fc_finish<float><<<n_rows, 256, smem, st>>>(part, splits, n_rows, n_rows_dev, a_rows, carry_slot, c->fcE, static_cast<const float*>(c->w.g_hidden), c->D, c->cfg.rms_eps, do_norm, static_cast<float*>(c->z), a_rows ? 1 : 0, tap_z)));
+             (k_fc_finish<__nv_bfloat16><<<n_rows, nt, 0, st>>>(part, splits, n_rows, n_rows_dev, a_rows, carry_slot, c->fcE, static_cast<const __nv_bfloat16*>(c->w.g_hidden), c->D, c->cfg.rms_eps, do_norm, static_cast<__nv_bfloat16*>(c->z), a_rows ? 1 : 0, tap_z)),
+             (k_fc_finish<float><<<n_rows, nt, 0, st>>>(part, splits, n_rows, n_rows_dev, a_rows, carry_slot, c->fcE, static_cast<const float*>(c->w.g_hidden), c->D, c->cfg.rms_eps, do_norm, static_cast<float*>(c->z), a_rows ? 1 : 0, tap_z)));
   COD_CHECK_LAUNCH(c);
   return COD_OK;
 }
@@ -364,8 +421,8 @@ int cod_launch_embed_norm(cod_ctx* c, const int32_t* bonus, int S, cudaStream_t 
   const cod_config& f = c->cfg;
   const int R = S * f.block;
   DISPATCH_T(c,
-             (k_embed_norm<__nv_bfloat16><<<R, 256, 0, st>>>(static_cast<const __nv_bfloat16*>(c->w.emb), bonus, f.block, f.mask_token_id, f.vocab, static_cast<const __nv_bfloat16*>(c->w.g_attn), c->D, f.rms_eps, c->x, static_cast<__nv_bfloat16*>(c->a), c->amax)),
-             (k_embed_norm<float><<<R, 256, 0, st>>>(static_cast<const float*>(c->w.emb), bonus, f.block, f.mask_token_id, f.vocab, static_cast<const float*>(c->w.g_attn), c->D, f.rms_eps, c->x, static_cast<float*>(c->a), c->amax)));
+             (k_embed_norm<__nv_bfloat16><<<R, row_threads(c->D), 0, st>>>(static_cast<const __nv_bfloat16*>(c->w.emb), bonus, f.block, f.mask_token_id, f.vocab, static_cast<const __nv_bfloat16*>(c->w.g_attn), c->D, f.rms_eps, c->x, static_cast<__nv_bfloat16*>(c->a), c->amax)),
+             (k_embed_norm<float><<<R, row_threads(c->D), 0, st>>>(static_cast<const float*>(c->w.emb), bonus, f.block, f.mask_token_id, f.vocab, static_cast<const float*>(c->w.g_attn), c->D, f.rms_eps, c->x, static_cast<float*>(c->a), c->amax)));
   COD_CHECK_LAUNCH(c);
   return COD_OK;
 }
@@ -373,9 +430,10 @@ int cod_launch_embed_norm(cod_ctx* c, const int32_t* bonus, int S, cudaStream_t 
 int cod_launch_qkv_finish(cod_ctx* c, const float* part, int splits, int R, cudaStream_t st) {
   ProfScope prof(c, COD_K_ROWOPS, st);
   const cod_config& f = c->cfg;
+  const dim3 grid(R, f.n_q_heads + 2 * f.n_kv_heads);
   DISPATCH_T(c,
-             (k_qkv_finish<__nv_bfloat16><<<R, 256, 0, st>>>(part, splits, R, f.n_q_heads, f.n_kv_heads, f.head_dim, c->rope_blk, static_cast<__nv_bfloat16*>(c->q), static_cast<__nv_bfloat16*>(c->kb), static_cast<__nv_bfloat16*>(c->vb))),
-             (k_qkv_finish<float><<<R, 256, 0, st>>>(part, splits, R, f.n_q_heads, f.n_kv_heads, f.head_dim, c->rope_blk, static_cast<float*>(c->q), static_cast<float*>(c->kb), static_cast<float*>(c->vb))));
+             (k_qkv_finish<__nv_bfloat16><<<grid, 64, 0, st>>>(part, splits, R, f.n_q_heads, f.n_kv_heads, f.head_dim, c->rope_blk, static_cast<__nv_bfloat16*>(c->q), static_cast<__nv_bfloat16*>(c->kb), static_cast<__nv_bfloat16*>(c->vb))),
+             (k_qkv_finish<float><<<grid, 64, 0, st>>>(part, splits, R, f.n_q_heads, f.n_kv_heads, f.head_dim, c->rope_blk, static_cast<float*>(c->q), static_cast<float*>(c->kb), static_cast<float*>(c->vb))));
   COD_CHECK_LAUNCH(c);
   return COD_OK;
 }
@@ -397,8 +455,8 @@ int cod_launch_resid_norm(cod_ctx* c, const float* part, int splits, int R, floa
                           float* tap_x, cudaStream_t st) {
   ProfScope prof(c, COD_K_ROWOPS, st);
   DISPATCH_T(c,
-             (k_resid_norm<__nv_bfloat16><<<R, 256, 0, st>>>(part, splits, R, c->D, x, static_cast<const __nv_bfloat16*>(gain), c->cfg.rms_eps, static_cast<__nv_bfloat16*>(c->a), tap_x, c->amax)),
-             (k_resid_norm<float><<<R, 256, 0, st>>>(part, splits, R, c->D, x, static_cast<const float*>(gain), c->cfg.rms_eps, static_cast<float*>(c->a), tap_x, c->amax)));
+             (k_resid_norm<__nv_bfloat16><<<R, row_threads(c->D), 0, st>>>(part, splits, R, c->D, x, static_cast<const __nv_bfloat16*>(gain), c->cfg.rms_eps, static_cast<__nv_bfloat16*>(c->a), tap_x, c->amax)),
+             (k_resid_norm<float><<<R, row_threads(c->D), 0, st>>>(part, splits, R, c->D, x, static_cast<const float*>(gain), c->cfg.rms_eps, static_cast<float*>(c->a), tap_x, c->amax)));
   COD_CHECK_LAUNCH(c);
   return COD_OK;
 }
