@@ -50,7 +50,8 @@ enum cod_status {
   COD_ERR_UNSUPPORTED = -2, /* a shape or flag this build has no kernel for */
   COD_ERR_CUDA = -3,        /* a CUDA runtime call or launch failed */
   COD_ERR_NO_WEIGHTS = -4,  /* cod_set_weights has not been called */
-  COD_ERR_ALLOC = -5        /* cod_create could not allocate its workspace */
+  COD_ERR_ALLOC = -5,       /* cod_create could not allocate its workspace */
+  COD_ERR_TOO_LARGE = -6    /* a size exceeds a fixed capacity (see cod_lm_head_argmax_static) */
 };
 
 enum cod_dtype { COD_F32 = 0, COD_BF16 = 1 };
@@ -183,6 +184,25 @@ int cod_block_attn(cod_ctx* ctx, int layer, const void* q, const void* k_blk, co
    top_logit (nullable) [n_rows] device float. Logits are never materialised. */
 int cod_lm_head_argmax(cod_ctx* ctx, const float* x, int n_rows, int32_t* tok, float* top_logit,
                        cod_stream_t stream);
+
+/* The same argmax as cod_lm_head_argmax for callers that may not allocate device memory: it needs
+   no cod_ctx and calls no cudaMalloc / cudaFree or any allocating routine. (The paper has no
+   counterpart for this entry point; it exists for integration.) Such callers are, for example, a
+   server whose device memory is entirely owned by its own pool, or a latency-critical loop that
+   cannot afford cudaMalloc's device-wide synchronisation.
+   Its scratch (normalised activations, packed argmax keys) is a fixed array inside the library:
+   each GPU that loads the library holds about 2 MiB of it until the process exits.
+     emb [vocab, d_model], g_final [d_model]: device, element type `dtype` (cod_dtype);
+     x [n_rows, d_model] device float32; tok [n_rows] device int32; top_logit [n_rows] device
+     float32 or NULL.
+   Limits: n_rows <= 64 and d_model <= 8192, otherwise COD_ERR_TOO_LARGE and nothing is launched.
+   All calls on a device share the scratch, which keeps the last call's contents (what must start
+   at zero is cleared by the call itself): calls that overlap on the GPU race with each other.
+   The first call on a device looks up the scratch's device address with that device current; it
+   should be made before any stream capture begins. Device-side status bits are not reported. */
+int cod_lm_head_argmax_static(const void* emb, const void* g_final, const float* x, int n_rows,
+                              int d_model, int vocab, int dtype, float rms_eps, int32_t* tok,
+                              float* top_logit, cod_stream_t stream);
 
 /* The whole round: parts 1-3 on (draft, target, H), then one parallel block prediction from
    [bonus, MASK, ...] through every drafter layer, then part 5.

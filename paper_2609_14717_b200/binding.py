@@ -23,7 +23,8 @@ COD_F_NO_TENSOR_CORES = 2
 DEV_BAD_TOKEN, DEV_PAGE_OVERFLOW, DEV_BAD_PAGE, DEV_TIMEOUT, DEV_BAD_LEN = 1, 2, 4, 8, 16
 
 EXPORTS = ("cod_create", "cod_destroy", "cod_set_weights", "cod_verify_accept", "cod_project_kv",
-           "cod_scatter_kv", "cod_block_attn", "cod_lm_head_argmax", "cod_draft_round",
+           "cod_scatter_kv", "cod_block_attn", "cod_lm_head_argmax", "cod_lm_head_argmax_static",
+           "cod_draft_round",
            "cod_poll_status", "cod_profile_enable", "cod_profile_read", "cod_launch_count",
            "cod_workspace_bytes", "cod_error_string")
 KERNEL_CLASSES = ("verify", "fc", "kv", "qkv", "attn", "oproj", "lmhead", "rowops")
@@ -73,6 +74,7 @@ def load_library() -> C.CDLL:
     lib.cod_scatter_kv.argtypes = [vp, vp, C.POINTER(CodSplit), i32, i32, C.POINTER(CodState), vp]
     lib.cod_block_attn.argtypes = [vp, i32, vp, vp, vp, C.POINTER(CodState), i32, i32, vp, vp, vp]
     lib.cod_lm_head_argmax.argtypes = [vp, vp, i32, vp, vp, vp]
+    lib.cod_lm_head_argmax_static.argtypes = [vp, vp, vp, i32, i32, i32, i32, C.c_float, vp, vp, vp]
     lib.cod_draft_round.argtypes = [vp, vp, vp, vp, i32, i32, i32, C.POINTER(CodState), C.POINTER(CodSplit),
                                     vp, C.POINTER(CodTaps), vp]
     lib.cod_poll_status.argtypes = [vp, C.POINTER(C.c_uint32), i32, vp]
@@ -270,6 +272,20 @@ class Context:
 
     def workspace_bytes(self) -> int:
         return int(lib().cod_workspace_bytes(self._h))
+
+
+def lm_head_argmax_static(emb: torch.Tensor, g_final: torch.Tensor, x: torch.Tensor, tok: torch.Tensor,
+                          top_logit: Optional[torch.Tensor], rms_eps: float) -> None:
+    """cod_lm_head_argmax_static: the LM-head argmax for callers that may not allocate device memory.
+
+    Needs no Context. The scratch is a fixed array inside the library (rows <= 64, width <= 8192);
+    calls that overlap on the GPU race on it, and the first call on a device should precede any
+    stream capture."""
+    n_rows, d_model = x.shape
+    dtype = COD_BF16 if emb.dtype == torch.bfloat16 else COD_F32
+    _check("cod_lm_head_argmax_static", lib().cod_lm_head_argmax_static(
+        _ptr(emb), _ptr(g_final), _ptr(x), n_rows, d_model, emb.shape[0], dtype, C.c_float(rms_eps),
+        _ptr(tok), _ptr(top_logit), _stream()))
 
 
 def make_config(sh, max_batch: int, max_pages_per_seq: int, n_pages: int, attn_split_len: int = 0,

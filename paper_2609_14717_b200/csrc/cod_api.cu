@@ -402,6 +402,7 @@ const char* cod_error_string(int status) {
     case COD_ERR_CUDA: return "CUDA runtime error";
     case COD_ERR_NO_WEIGHTS: return "weights not set";
     case COD_ERR_ALLOC: return "workspace allocation failed";
+    case COD_ERR_TOO_LARGE: return "size exceeds a fixed capacity of this entry point";
     default: return "unknown status";
   }
 }
