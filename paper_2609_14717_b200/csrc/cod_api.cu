@@ -79,7 +79,9 @@ bool state_has_null(const cod_state* s) {
 // split-K factor so that (feature tiles x splits) fills the machine; partial slabs must fit
 int pick_splits(const cod_ctx* c, int n_out, int K, int rows) {
   if (c->cfg.dtype != COD_BF16 || c->force_simt) return 1;
-  const int ctas = ((n_out + 127) / 128) * ((rows + 255) / 256);
+  const int tiles = (n_out + 127) / 128;
+  int ctas = tiles * ((rows + 255) / 256);
+  if (rows > 128 && tiles >= c->n_sm) ctas = tiles * ((rows + 511) / 512);   // the paired kernel's 512-row tiles
   const int kb = (K + 63) / 64;
   int splits = c->n_sm / ctas;
   if (splits > COD_MAX_SPLITS) splits = COD_MAX_SPLITS;
@@ -95,6 +97,7 @@ int check_S(const cod_ctx* c, int S) { return (S >= 1 && S <= c->cfg.max_batch) 
 
 int cod_launch_gemm(cod_ctx* c, const GemmArgs& g, cudaStream_t st) {
   ProfScope prof(c, g.klass, st);
+  if (!c->force_simt && cod_gemm_tc2_supported(c, g)) return cod_launch_gemm_tc2(c, g, st);
   if (!c->force_simt && cod_gemm_tc_supported(c, g)) return cod_launch_gemm_tc(c, g, st);
   return cod_launch_gemm_simt(c, g, st);
 }

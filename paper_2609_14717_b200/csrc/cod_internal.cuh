@@ -157,6 +157,8 @@ int cod_launch_verify(cod_ctx* c, const int32_t* draft, const int32_t* target, i
 int cod_launch_gemm(cod_ctx* c, const GemmArgs& g, cudaStream_t st);
 int cod_launch_gemm_simt(cod_ctx* c, const GemmArgs& g, cudaStream_t st);
 bool cod_gemm_tc_supported(const cod_ctx* c, const GemmArgs& g);
+bool cod_gemm_tc2_supported(const cod_ctx* c, const GemmArgs& g);
+int cod_launch_gemm_tc2(cod_ctx* c, const GemmArgs& g, cudaStream_t st);
 bool cod_attn_tc_supported(const cod_ctx* c);
 int cod_launch_attn_tc(cod_ctx* c, int layer, const void* q, const void* kb, const void* vb, const cod_state* stt,
                        int S, int use_carry, void* out, float* tap, float* mass, cudaStream_t st);

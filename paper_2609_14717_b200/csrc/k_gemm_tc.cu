@@ -153,6 +153,36 @@ __device__ __forceinline__ unsigned order_key(float v) {
   return (u & 0x80000000u) ? ~u : (u | 0x80000000u);
 }
 
+// Column-wise maximum over the 32 lanes of a warp for 32 columns at once: every lane brings one
+// packed key per column; after five exchange rounds (16 + 8 + 4 + 2 + 1 shuffles) lane L holds
+// the maximum of column L. The keys carry the row index, so this is an argmax with the lowest
+// row winning ties.
+__device__ __forceinline__ unsigned long long warp_colmax32(unsigned long long (&k)[32], int lane) {
+#pragma unroll
+  for (int off = 16; off >= 1; off >>= 1) {
+    const bool hi = (lane & off) != 0;
+#pragma unroll
+    for (int c = 0; c < off; ++c) {
+      const unsigned long long send = hi ? k[c] : k[c + off];
+      const unsigned long long mine = hi ? k[c + off] : k[c];
+      const unsigned long long recv = __shfl_xor_sync(0xffffffffu, send, off);
+      k[c] = recv > mine ? recv : mine;
+    }
+  }
+  return k[0];
+}
+__device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&v)[32]) {
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+      "{%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31}, [%32];"
+      : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]),
+        "=r"(v[8]), "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15]),
+        "=r"(v[16]), "=r"(v[17]), "=r"(v[18]), "=r"(v[19]), "=r"(v[20]), "=r"(v[21]), "=r"(v[22]), "=r"(v[23]),
+        "=r"(v[24]), "=r"(v[25]), "=r"(v[26]), "=r"(v[27]), "=r"(v[28]), "=r"(v[29]), "=r"(v[30]), "=r"(v[31])
+      : "r"(taddr) : "memory");
+  asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+}
+
 __global__ void __launch_bounds__(NTHREADS, 1)
 k_gemm_tc(const __grid_constant__ CUtensorMap map_w0, const __grid_constant__ CUtensorMap map_w1,
           const __grid_constant__ CUtensorMap map_w2, const __grid_constant__ CUtensorMap map_a, const TcParams p) {
@@ -258,23 +288,27 @@ k_gemm_tc(const __grid_constant__ CUtensorMap map_w0, const __grid_constant__ CU
         }
       }
     } else if (ok) {
-      // per-token (max, lowest row) over this warp's 32 weight rows; lane j keeps column c + j
-      for (int c = 0; c < p.NT; c += 16) {
-        uint32_t v[16];
-        tmem_ld16(t_lane + c, v);
-        unsigned long long mine = 0ull;
+      // per-token (max, lowest row) over this warp's 32 weight rows, 32 token columns at a time
+      const unsigned long long low = static_cast<unsigned long long>(0xFFFFFFFFu - static_cast<unsigned>(col0 + warp * 32 + lane));
+      for (int c = 0; c < p.NT; c += 32) {
+        unsigned long long k[32];
+        if (c + 32 <= p.NT) {
+          uint32_t v[32];
+          tmem_ld32(t_lane + c, v);
 #pragma unroll
-        for (int j = 0; j < 16; ++j) {
-          const unsigned u = f_ok ? order_key(__uint_as_float(v[j])) : 0u;
-          const unsigned mx = __reduce_max_sync(0xffffffffu, u);
-          const unsigned who = __ballot_sync(0xffffffffu, u == mx);
-          if (lane == j) {
-            const int idx = col0 + warp * 32 + (__ffs(who) - 1);      // lowest weight row among equals
-            mine = (static_cast<unsigned long long>(mx) << 32) |
-                   static_cast<unsigned long long>(0xFFFFFFFFu - static_cast<unsigned>(idx));
+          for (int j = 0; j < 32; ++j)
+            k[j] = f_ok ? ((static_cast<unsigned long long>(order_key(__uint_as_float(v[j]))) << 32) | low) : 0ull;
+        } else {                                   // NT is a multiple of 16: a last half chunk
+          uint32_t v[16];
+          tmem_ld16(t_lane + c, v);
+#pragma unroll
+          for (int j = 0; j < 16; ++j) {
+            k[j] = f_ok ? ((static_cast<unsigned long long>(order_key(__uint_as_float(v[j]))) << 32) | low) : 0ull;
+            k[16 + j] = 0ull;
           }
         }
-        if (lane < 16) red[warp * p.NT + c + lane] = mine;
+        const unsigned long long best = warp_colmax32(k, lane);
+        if (c + lane < p.NT) red[warp * p.NT + c + lane] = best;
       }
     }
   }

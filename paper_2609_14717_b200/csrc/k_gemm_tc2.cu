@@ -1,0 +1,415 @@
+// Weight-streaming GEMM for many token rows (more than 128): the same swap-AB scheme as
+// k_gemm_tc, but two CTAs of a thread-block cluster (two SMs) work on one 256 x 256 tile with
+// tcgen05.mma.cta_group::2:
+//   C[i, n] = sum_k A[i, k] * B[n, k]     A: activations [rows, K], B: weights [N, K].
+// Each CTA stages its own 128 weight rows and its own half (128) of the 256 token rows, so per
+// unit of tensor work every SM pulls half as many operand bytes through its TMA engine as a
+// single-CTA 128 x 256 tile does - the engine (about 36 B/clk per SM), not the tensor pipe,
+// is what limits the single-CTA kernel once the GEMM is compute-bound.
+//
+// Protocol (rank 0 of the pair is the leader):
+//   * both CTAs: TMA producer warp loads its tiles with the cta_group::2 form of the copy, which
+//     signals the LEADER's "full" barrier; the leader expects the bytes of both CTAs;
+//   * leader only: one thread issues the MMAs (M = 256 spans both CTAs' tensor memory) and commits
+//     with a cluster-wide arrive to the "empty" barrier of both CTAs (and, at the end, to both
+//     "accumulator ready" barriers);
+//   * both CTAs: four epilogue warps read their own 128 accumulator rows.
+// No load is delivered to more than one CTA. Waits are bounded as in k_gemm_tc; the only
+// unbounded synchronisation is the hardware cluster barrier, which every thread reaches
+// unconditionally.
+#include <cuda.h>
+
+#include "cod_internal.cuh"
+
+namespace {
+
+constexpr int BM = 128;       // weight rows per CTA (256 per pair)
+constexpr int BK = 64;
+constexpr int UK = 16;
+constexpr int NT = 256;       // token rows per pair = MMA N; each CTA stages NT / 2 of them
+constexpr int NTHREADS = 192;
+constexpr uint32_t A_TILE_BYTES = BM * BK * 2;          // 16 KB
+constexpr uint32_t B_TILE_BYTES = (NT / 2) * BK * 2;    // 16 KB
+constexpr int MAX_STAGES = 6;   // one accumulator: 6 stages of 32 KB; two: 4 stages of 48 KB
+constexpr long long WAIT_LIMIT_CYCLES = 4000000000ll;
+constexpr uint32_t PEER_MASK = 0xFEFFFFFFu;             // shared::cluster address of the even-ranked CTA's copy
+
+struct Tc2Params {
+  int K, kb_total, kb_per_split;
+  int n_rows;
+  const int* n_rows_dev;
+  int pair_end[3];            // cumulative count of 256-row tile pairs after each weight segment
+  int seg_N[3];
+  int n_seg;
+  int n_tiles_n;              // token tiles
+  int n_acc;                  // accumulators per pair: 1 (256 token rows) or 2 (512)
+  int stages;
+  float* C;
+  int ldc;
+  unsigned long long* amax;
+  uint32_t* status;
+};
+
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return static_cast<uint32_t>(__cvta_generic_to_shared(p)); }
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count));
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+  return ok != 0;
+}
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, uint32_t* status) {
+#pragma unroll 1
+  for (int i = 0; i < 64; ++i)
+    if (mbar_try_wait(bar, parity)) return true;
+  const long long t0 = clock64();
+  for (;;) {
+#pragma unroll 1
+    for (int i = 0; i < 256; ++i)
+      if (mbar_try_wait(bar, parity)) return true;
+    if (*abort_flag) return false;
+    if (clock64() - t0 > WAIT_LIMIT_CYCLES) {
+      *abort_flag = 1;
+      atomicOr(status, COD_DEV_TIMEOUT);
+      return false;
+    }
+  }
+}
+// the copy lands in this CTA's shared memory; its bytes are counted on the leader's barrier
+__device__ __forceinline__ void tma_load_2d_pair(uint32_t dst, const CUtensorMap* map, int c0, int c1, uint32_t leader_bar) {
+  asm volatile(
+      "cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
+      ::"r"(dst), "l"(reinterpret_cast<uint64_t>(map)), "r"(c0), "r"(c1), "r"(leader_bar) : "memory");
+}
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void cluster_sync_all() {
+  asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
+  asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void tmem_alloc_pair(uint32_t dst_smem, uint32_t cols) {
+  asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(dst_smem), "r"(cols) : "memory");
+  asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void tmem_dealloc_pair(uint32_t taddr, uint32_t cols) {
+  asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(cols) : "memory");
+}
+__device__ __forceinline__ void umma_bf16_pair(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, uint32_t accumulate) {
+  const uint32_t z = 0u;   // no accumulator lane is masked off
+  asm volatile(
+      "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::2.kind::f16 [%0], %1, %2, %3, {%5, %5, %5, %5, %5, %5, %5, %5}, p;\n\t}"
+      ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate), "r"(z) : "memory");
+}
+// arrive on the barrier at this offset in every CTA of the mask once the MMAs issued so far are done
+__device__ __forceinline__ void umma_commit_pair(uint32_t bar, uint16_t cta_mask) {
+  asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;"
+               ::"r"(bar), "h"(cta_mask) : "memory");
+}
+__device__ __forceinline__ void tmem_ld16(uint32_t taddr, uint32_t (&v)[16]) {
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15}, [%16];"
+      : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]),
+        "=r"(v[8]), "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15])
+      : "r"(taddr) : "memory");
+  asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+}
+__device__ __forceinline__ uint64_t smem_desc_sw128(uint32_t saddr) {
+  uint64_t d = 0;
+  d |= static_cast<uint64_t>((saddr & 0x3FFFFu) >> 4);
+  d |= static_cast<uint64_t>(1) << 16;
+  d |= static_cast<uint64_t>(1024 >> 4) << 32;
+  d |= static_cast<uint64_t>(1) << 46;
+  d |= static_cast<uint64_t>(2) << 61;
+  return d;
+}
+__device__ __forceinline__ unsigned order_key(float v) {
+  const unsigned u = __float_as_uint(v);
+  return (u & 0x80000000u) ? ~u : (u | 0x80000000u);
+}
+
+// Column-wise maximum over the 32 lanes of a warp for 32 columns at once: every lane brings one
+// packed key per column; after five exchange rounds (16 + 8 + 4 + 2 + 1 shuffles) lane L holds
+// the maximum of column L. The keys carry the row index, so this is an argmax with the lowest
+// row winning ties.
+__device__ __forceinline__ unsigned long long warp_colmax32(unsigned long long (&k)[32], int lane) {
+#pragma unroll
+  for (int off = 16; off >= 1; off >>= 1) {
+    const bool hi = (lane & off) != 0;
+#pragma unroll
+    for (int c = 0; c < off; ++c) {
+      const unsigned long long send = hi ? k[c] : k[c + off];
+      const unsigned long long mine = hi ? k[c + off] : k[c];
+      const unsigned long long recv = __shfl_xor_sync(0xffffffffu, send, off);
+      k[c] = recv > mine ? recv : mine;
+    }
+  }
+  return k[0];
+}
+__device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&v)[32]) {
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+      "{%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31}, [%32];"
+      : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]),
+        "=r"(v[8]), "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15]),
+        "=r"(v[16]), "=r"(v[17]), "=r"(v[18]), "=r"(v[19]), "=r"(v[20]), "=r"(v[21]), "=r"(v[22]), "=r"(v[23]),
+        "=r"(v[24]), "=r"(v[25]), "=r"(v[26]), "=r"(v[27]), "=r"(v[28]), "=r"(v[29]), "=r"(v[30]), "=r"(v[31])
+      : "r"(taddr) : "memory");
+  asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+}
+
+__global__ void __launch_bounds__(NTHREADS, 1)
+k_gemm_tc2(const __grid_constant__ CUtensorMap map_w0, const __grid_constant__ CUtensorMap map_w1,
+           const __grid_constant__ CUtensorMap map_w2, const __grid_constant__ CUtensorMap map_a, const Tc2Params p) {
+  extern __shared__ uint8_t smem_raw[];
+  const uint32_t raw = smem_u32(smem_raw);
+  const uint32_t base = (raw + 1023u) & ~1023u;
+  uint8_t* sm = smem_raw + (base - raw);
+  const uint32_t STAGE_BYTES = A_TILE_BYTES + p.n_acc * B_TILE_BYTES;
+  const int STAGES = p.stages;
+  const int NTOK = p.n_acc * NT;                                       // token rows of this pair's tile
+  const uint32_t TMEM_COLS = static_cast<uint32_t>(NTOK);
+  uint8_t* ctl = sm + STAGES * STAGE_BYTES;
+  uint64_t* full_bar = reinterpret_cast<uint64_t*>(ctl);               // [STAGES], used in the leader
+  uint64_t* empty_bar = full_bar + 8;                                  // [STAGES]
+  uint64_t* acc_bar = full_bar + 16;
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(full_bar + 17);
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+  unsigned long long* red = reinterpret_cast<unsigned long long*>(full_bar + 18);   // [4][NT]
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int rank = blockIdx.x;                    // position in the pair; 0 leads
+  const int n_tile = blockIdx.y % p.n_tiles_n, pair = blockIdx.y / p.n_tiles_n, split = blockIdx.z;
+  const int n_rows = p.n_rows_dev ? min(*p.n_rows_dev, p.n_rows) : p.n_rows;
+  const int i0 = n_tile * NTOK;
+  // NOTE: both CTAs of a pair take the same decision here (it depends on the pair's tile only)
+  const bool idle = i0 >= n_rows;
+
+  int sidx = 0;
+  while (sidx < p.n_seg - 1 && pair >= p.pair_end[sidx]) ++sidx;
+  const int pair_in_seg = pair - (sidx ? p.pair_end[sidx - 1] : 0);
+  const int f0 = pair_in_seg * 2 * BM + rank * BM;           // this CTA's first weight row within the segment
+  int col0 = f0;
+  for (int s = 0; s < sidx; ++s) col0 += p.seg_N[s];
+  const int seg_N = p.seg_N[sidx];
+  const CUtensorMap* map_w = sidx == 0 ? &map_w0 : (sidx == 1 ? &map_w1 : &map_w2);
+  const int kb0 = split * p.kb_per_split, kb1 = min(p.kb_total, kb0 + p.kb_per_split);
+  const int n_kb = idle ? 0 : kb1 - kb0;
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < STAGES; ++s) { mbar_init(smem_u32(full_bar + s), 1); mbar_init(smem_u32(empty_bar + s), 1); }
+    mbar_init(smem_u32(acc_bar), 1);
+    *abort_flag = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  for (int t = threadIdx.x; t < 4 * NTOK; t += NTHREADS) red[t] = 0ull;
+  if (warp == 5) tmem_alloc_pair(smem_u32(tmem_slot), TMEM_COLS);
+  tc_fence_before();
+  __syncthreads();
+  cluster_sync_all();                 // the partner's barriers exist before anything signals them
+  tc_fence_after();
+  const uint32_t tmem_base = *tmem_slot;
+
+  if (warp == 4) {
+    if (lane == 0) {
+      for (int it = 0; it < n_kb; ++it) {
+        const int s = it % STAGES, use = it / STAGES;
+        if (use > 0 && !mbar_wait(smem_u32(empty_bar + s), (use - 1) & 1, abort_flag, p.status)) break;
+        const uint32_t fb = smem_u32(full_bar + s);
+        if (rank == 0) mbar_expect_tx(fb, 2 * STAGE_BYTES);     // both CTAs' bytes land on the leader's barrier
+        const uint32_t a_dst = base + s * STAGE_BYTES;
+        const int k = (kb0 + it) * BK;
+        tma_load_2d_pair(a_dst, map_w, k, f0, fb & PEER_MASK);
+        for (int a = 0; a < p.n_acc; ++a)      // accumulator a covers tokens [i0 + a*256, +256): this CTA stages its half
+          tma_load_2d_pair(a_dst + A_TILE_BYTES + a * B_TILE_BYTES, &map_a, k, i0 + a * NT + rank * (NT / 2), fb & PEER_MASK);
+      }
+    }
+  } else if (warp == 5) {
+    if (lane == 0 && rank == 0) {
+      // bf16 x bf16 -> float, K-major operands, M = 256 (both CTAs), N = 256
+      const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | (static_cast<uint32_t>(NT >> 3) << 17) |
+                             (static_cast<uint32_t>((2 * BM) >> 4) << 24);
+      bool ok = true;
+      for (int it = 0; it < n_kb && ok; ++it) {
+        const int s = it % STAGES, use = it / STAGES;
+        ok = mbar_wait(smem_u32(full_bar + s), use & 1, abort_flag, p.status);
+        if (!ok) break;
+        tc_fence_after();
+        const uint32_t a_addr = base + s * STAGE_BYTES;
+        const uint64_t a_desc = smem_desc_sw128(a_addr);
+        for (int a = 0; a < p.n_acc; ++a) {
+          const uint64_t b_desc = smem_desc_sw128(a_addr + A_TILE_BYTES + a * B_TILE_BYTES);
+#pragma unroll
+          for (int k = 0; k < BK / UK; ++k)
+            umma_bf16_pair(tmem_base + a * NT, a_desc + (k * UK * 2 >> 4), b_desc + (k * UK * 2 >> 4), idesc, (it | k) ? 1u : 0u);
+        }
+        umma_commit_pair(smem_u32(empty_bar + s), 3);
+      }
+      if (ok && n_kb > 0) umma_commit_pair(smem_u32(acc_bar), 3);
+    }
+  } else if (n_kb > 0) {
+    const bool ok = mbar_wait(smem_u32(acc_bar), 0, abort_flag, p.status);
+    tc_fence_after();
+    const int f = f0 + warp * 32 + lane;
+    const bool f_ok = f < seg_N;
+    const uint32_t t_lane = tmem_base + (static_cast<uint32_t>(warp * 32) << 16);
+    if (ok && p.amax == nullptr) {
+      float* C = p.C + static_cast<size_t>(split) * p.n_rows * p.ldc;
+      for (int c = 0; c < NTOK; c += 16) {
+        if (i0 + c >= n_rows) break;
+        uint32_t v[16];
+        tmem_ld16(t_lane + c, v);
+#pragma unroll
+        for (int j = 0; j < 16; ++j) {
+          const int i = i0 + c + j;
+          if (f_ok && i < n_rows) C[static_cast<size_t>(i) * p.ldc + col0 + warp * 32 + lane] = __uint_as_float(v[j]);
+        }
+      }
+    } else if (ok) {
+      const unsigned long long low = static_cast<unsigned long long>(0xFFFFFFFFu - static_cast<unsigned>(col0 + warp * 32 + lane));
+      for (int c = 0; c < NTOK; c += 32) {
+        if (i0 + c >= n_rows) break;
+        uint32_t v[32];
+        tmem_ld32(t_lane + c, v);
+        unsigned long long k[32];
+#pragma unroll
+        for (int j = 0; j < 32; ++j)
+          k[j] = f_ok ? ((static_cast<unsigned long long>(order_key(__uint_as_float(v[j]))) << 32) | low) : 0ull;
+        red[warp * NTOK + c + lane] = warp_colmax32(k, lane);
+      }
+    }
+  }
+
+  // ---------------------------------------------------- teardown
+  tc_fence_before();
+  __syncthreads();
+  if (*abort_flag) {
+    for (int i = 0; i < 64; ++i) __nanosleep(1000);
+    __syncthreads();
+  } else if (p.amax != nullptr && n_kb > 0) {
+    for (int t = threadIdx.x; t < NTOK; t += NTHREADS) {
+      if (i0 + t < n_rows) {
+        unsigned long long best = red[t];
+#pragma unroll
+        for (int w = 1; w < 4; ++w) best = red[w * NTOK + t] > best ? red[w * NTOK + t] : best;
+        if (best) atomicMax(p.amax + i0 + t, best);
+      }
+    }
+  }
+  cluster_sync_all();                 // neither CTA frees tensor memory or exits while the other may still touch it
+  if (warp == 5) {
+    tc_fence_after();
+    tmem_dealloc_pair(tmem_base, TMEM_COLS);
+  }
+}
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+EncodeTiledFn encode_fn() {
+  static EncodeTiledFn fn = nullptr;
+  static bool tried = false;
+  if (!tried) {
+    tried = true;
+    void* ptr = nullptr;
+    cudaDriverEntryPointQueryResult q;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &ptr, cudaEnableDefault, &q) == cudaSuccess &&
+        q == cudaDriverEntryPointSuccess)
+      fn = reinterpret_cast<EncodeTiledFn>(ptr);
+  }
+  return fn;
+}
+bool make_map(CUtensorMap* m, const void* ptr, uint64_t rows, uint64_t K, uint64_t ld, uint32_t box_rows) {
+  EncodeTiledFn fn = encode_fn();
+  if (!fn) return false;
+  cuuint64_t gdim[2] = {K, rows};
+  cuuint64_t gstride[1] = {ld * 2};
+  cuuint32_t box[2] = {static_cast<cuuint32_t>(BK), box_rows};
+  cuuint32_t estr[2] = {1, 1};
+  return fn(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(ptr), gdim, gstride, box, estr,
+            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+}  // namespace
+
+// Used for more than 128 token rows; every weight segment but the last must be whole 256-row pairs.
+bool cod_gemm_tc2_supported(const cod_ctx* c, const GemmArgs& g) {
+  if (c->cfg.dtype != COD_BF16 || g.a_rows != nullptr || g.n_rows <= 128) return false;
+  if (g.K % 8 || g.lda % 8) return false;
+  if ((reinterpret_cast<uintptr_t>(g.A) & 15u) != 0) return false;
+  for (int i = 0; i < g.n_seg; ++i) {
+    if ((reinterpret_cast<uintptr_t>(g.seg[i].B) & 15u) != 0) return false;
+    if (i + 1 < g.n_seg && g.seg[i].N % (2 * BM)) return false;
+  }
+  return encode_fn() != nullptr;
+}
+
+int cod_launch_gemm_tc2(cod_ctx* c, const GemmArgs& g, cudaStream_t st) {
+  Tc2Params p{};
+  p.K = g.K;
+  p.kb_total = (g.K + BK - 1) / BK;
+  int splits = g.splits < 1 ? 1 : g.splits;
+  p.kb_per_split = (p.kb_total + splits - 1) / splits;
+  splits = (p.kb_total + p.kb_per_split - 1) / p.kb_per_split;
+  if (splits != g.splits) return COD_ERR_INVALID_ARG;
+  p.n_rows = g.n_rows;
+  p.n_rows_dev = g.n_rows_dev;
+  int pairs = 0;
+  for (int i = 0; i < 3; ++i) {
+    if (i < g.n_seg) {
+      pairs += (g.seg[i].N + 2 * BM - 1) / (2 * BM);
+      p.seg_N[i] = g.seg[i].N;
+    }
+    p.pair_end[i] = pairs;
+  }
+  p.n_seg = g.n_seg;
+  // two accumulators (512 token rows per pair, weights streamed once) only when there are enough
+  // weight-row pairs to fill the machine that way
+  p.n_acc = (g.n_rows > NT && 2 * pairs >= c->n_sm) ? 2 : 1;
+  p.stages = p.n_acc == 2 ? 4 : MAX_STAGES;
+  p.n_tiles_n = (g.n_rows + p.n_acc * NT - 1) / (p.n_acc * NT);
+  p.C = g.C;
+  p.ldc = g.ldc;
+  p.amax = g.amax;
+  p.status = c->status;
+
+  CUtensorMap mw[3], ma;
+  for (int i = 0; i < 3; ++i) {
+    const int j = i < g.n_seg ? i : 0;
+    if (!make_map(&mw[i], g.seg[j].B, g.seg[j].N, g.K, g.K, BM)) return COD_ERR_CUDA;
+  }
+  if (!make_map(&ma, g.A, g.n_rows, g.K, g.lda, NT / 2)) return COD_ERR_CUDA;
+
+  const size_t smem = static_cast<size_t>(p.stages) * (A_TILE_BYTES + p.n_acc * B_TILE_BYTES) + 1024 + 18 * 8 +
+                      static_cast<size_t>(4) * p.n_acc * NT * 8;
+  static size_t configured = 0;
+  if (smem > configured) {
+    if (cudaFuncSetAttribute(k_gemm_tc2, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem)) != cudaSuccess)
+      return COD_ERR_CUDA;
+    configured = smem;
+  }
+  cudaLaunchConfig_t cfg{};
+  cfg.gridDim = dim3(2, pairs * p.n_tiles_n, splits);
+  cfg.blockDim = dim3(NTHREADS, 1, 1);
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = st;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeClusterDimension;
+  attr[0].val.clusterDim.x = 2;
+  attr[0].val.clusterDim.y = 1;
+  attr[0].val.clusterDim.z = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  if (cudaLaunchKernelEx(&cfg, k_gemm_tc2, mw[0], mw[1], mw[2], ma, p) != cudaSuccess) return COD_ERR_CUDA;
+  COD_CHECK_LAUNCH(c);
+  return COD_OK;
+}
