@@ -258,7 +258,7 @@ def run_gpu(args):
     weights = synth.make_weights(sh, seed)
     lay = synth.make_layout(wl, seed)
     n_pages, mp = int(lay["n_pages"]), int(lay["max_pages_per_seq"])
-    cfg = B.make_config(sh, wl.S, mp, n_pages)
+    cfg = B.make_config(sh, wl.S, mp, n_pages, attn_split_len=args.attn_split)
     ctx = B.Context(cfg)
     w_dev = B.weights_to_device(weights, sh.dtype)
     ctx.set_weights(w_dev)
@@ -464,7 +464,7 @@ def run_micro(args):
     sh = wl.shape
     lay = synth.make_layout(wl, args.seed)
     n_pages, mp = int(lay["n_pages"]), int(lay["max_pages_per_seq"])
-    cfg = B.make_config(sh, wl.S, mp, n_pages)
+    cfg = B.make_config(sh, wl.S, mp, n_pages, attn_split_len=args.attn_split)
     ctx = B.Context(cfg)
     td = B.torch_dtype(sh.dtype)
     gen = torch.Generator(device="cuda").manual_seed(args.seed)
@@ -516,6 +516,7 @@ def main():
     ap.add_argument("--seed", type=int, default=0)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-graph", action="store_true", help="time plain stream launches instead of graph replays")
+    ap.add_argument("--attn-split", type=int, default=0, help="keys per attention split (0 = library default)")
     ap.add_argument("--micro", default=None, choices=["attn", "lmhead"],
                     help="time one entry point alone (small footprint; meant for profiler captures)")
     args = ap.parse_args()

@@ -175,15 +175,15 @@ struct Geo {
   static constexpr int TILES = DUAL ? 2 : 1;             // 64-key tiles per iteration
   static constexpr int MROWS = DUAL ? 64 : 128;          // MMA M
   static constexpr int KEYS_IT = KT * TILES;
-  static constexpr int NK = DUAL ? 2 : 4;                // K ring slots
-  static constexpr int NV = DUAL ? 3 : 5;                // V ring slots
+  static constexpr int NK = DUAL ? 1 : 2;                // K ring slots
+  static constexpr int NV = DUAL ? 1 : 2;                // V ring slots
   static constexpr uint32_t SLOT = TILE_BYTES * TILES;
   static constexpr uint32_t Q_BYTES = MROWS * HD * 2;
   static constexpr uint32_t Q_HALF = MROWS * 128;
   static constexpr uint32_t P_TILE = MROWS * 128;        // [MROWS][64 keys] bf16
   static constexpr uint32_t P_BUF = P_TILE * TILES;
   static constexpr uint32_t OFF_P = Q_BYTES;
-  static constexpr uint32_t OFF_K = OFF_P + 2 * P_BUF;
+  static constexpr uint32_t OFF_K = OFF_P + P_BUF;       // P is single-buffered
   static constexpr uint32_t OFF_V = OFF_K + NK * SLOT;
   static constexpr uint32_t OFF_CTL = OFF_V + NV * SLOT;
   static constexpr uint32_t SMEM = OFF_CTL + 256 + 1024 + 1024;   // barriers, page ids, alignment slack
@@ -192,7 +192,7 @@ struct Geo {
 };
 
 template <bool DUAL>
-__global__ void __launch_bounds__(NTHREADS, 1)
+__global__ void __launch_bounds__(NTHREADS, 2)
 k_attn_tc(const __grid_constant__ CUtensorMap map_pool, const __grid_constant__ CUtensorMap map_zero, const AttnParams p) {
   using G = Geo<DUAL>;
   extern __shared__ uint8_t smem_raw[];
@@ -351,7 +351,7 @@ k_attn_tc(const __grid_constant__ CUtensorMap map_pool, const __grid_constant__ 
         tc_fence_after();
 #pragma unroll
         for (int t = 0; t < G::TILES; ++t) {
-          const uint64_t p_desc = desc_kmajor(base + G::OFF_P + (it & 1) * G::P_BUF + t * G::P_TILE);
+          const uint64_t p_desc = desc_kmajor(base + G::OFF_P + t * G::P_TILE);
           const uint64_t v_desc = desc_mnmajor(base + G::OFF_V + slot * G::SLOT + t * TILE_BYTES);
           const uint32_t d = tmem_base + G::COL_O + (static_cast<uint32_t>(16 * t) << 16);
 #pragma unroll
@@ -461,13 +461,13 @@ k_attn_tc(const __grid_constant__ CUtensorMap map_pool, const __grid_constant__ 
         lc_run *= factor;
         m_ref = m_new;
       }
-      if (it >= 2) {   // the P buffer about to be overwritten was read by PV(it-2)
-        ok = __all_sync(0xffffffffu, mbar_wait(smem_u32(o_full + (it & 1)), ((it - 2) >> 1) & 1, abort_flag, p.status));
+      if (it >= 1) {   // the P buffer about to be overwritten was read by PV(it-1)
+        ok = __all_sync(0xffffffffu, mbar_wait(smem_u32(o_full + ((it - 1) & 1)), ((it - 1) >> 1) & 1, abort_flag, p.status));
         if (!ok) break;
       }
       const float neg = m_ref == -INFINITY ? 0.f : -m_ref * sl2;
       float ps4[4] = {0.f, 0.f, 0.f, 0.f}, pcar = 0.f;
-      uint8_t* prow = sm + G::OFF_P + (it & 1) * G::P_BUF + tile * G::P_TILE + r * 128;
+      uint8_t* prow = sm + G::OFF_P + tile * G::P_TILE + r * 128;
       const int car0 = is_tail ? Lr - (it * G::KEYS_IT + tile * KT) : KT;  // carried keys: [car0, car0 + c)
 #pragma unroll
       for (int ch = 0; ch < 8; ++ch) {
