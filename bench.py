@@ -44,6 +44,28 @@ def load_peaks():
     return {"hbm_gbs": 6650.0, "tflops": 1400.0, "tflops_burst": 1590.0, "source": "fallback"}
 
 
+# --------------------------------------------------------------------------- replicas
+def replica_seed(seed: int, rank: int) -> int:
+    """Every rank runs its own replica of the workload on its own inputs."""
+    return seed + rank
+
+
+def max_over_ranks(ms: float, world: int, device="cuda") -> float:
+    """The timed region of the job is that of its slowest replica."""
+    if world <= 1:
+        return ms
+    import torch
+    import torch.distributed as dist
+    t = torch.tensor([ms], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def job_throughput(ms: float, steps: int, world: int) -> float:
+    """Rounds per second of the whole job: all replicas' rounds over the slowest replica's time."""
+    return world * steps / (ms * 1e-3)
+
+
 # --------------------------------------------------------------------------- byte / flop model
 def round_model(wl, L_after, carry, kept_rows, es=2):
     """Algorithmic bytes and flops of one round, per kernel class (weights read once per round,
@@ -251,7 +273,7 @@ def run_gpu(args):
     n_rounds = K + Wm
     wl = bench_workload(args.workload, n_rounds + 1)
     sh = wl.shape
-    seed = args.seed + rank
+    seed = replica_seed(args.seed, rank)
     es = 2 if sh.dtype == "bf16" else 4
 
     # ---- inputs: weights (host, seeded) -> device; layout; pool filled on the device
@@ -352,11 +374,7 @@ def run_gpu(args):
         barrier()
         ms = ev0.elapsed_time(ev1)
         launches = ctx.launch_count() - n0
-        if world > 1:
-            t = torch.tensor([ms], device="cuda")
-            dist.all_reduce(t, op=dist.ReduceOp.MAX)
-            ms = float(t.item())
-        return ms, launches
+        return max_over_ranks(ms, world), launches
 
     # ---- which kernel dominates, by the byte/flop model at the measured peaks
     L_run = lay["committed_len"].astype(np.int64).copy()
@@ -424,7 +442,7 @@ def run_gpu(args):
 
     h2d = int(H_pin[0].numel() * H_pin[0].element_size() + d_pin[0].numel() * 4 + t_pin[0].numel() * 4)
     line = {
-        "metric": METRIC, "value": world * K / (ms * 1e-3), "unit": UNIT, "n_gpus": world, "steps": K, "warmup": Wm,
+        "metric": METRIC, "value": job_throughput(ms, K, world), "unit": UNIT, "n_gpus": world, "steps": K, "warmup": Wm,
         "ms_per_step": ms / K, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
         "dtype": sh.dtype, "data": "synthetic",
         "config": {"workload": wl.name, "batch": wl.S, "block": sh.W, "context": list(wl.ctx),

@@ -1,0 +1,135 @@
+"""Parity at the sizes and in the launch configuration bench.py times (batch-1 and batch-32
+configurations, default split lengths, tensor-core kernels), on outputs the oracle can
+afford: the whole batch-1 round, and two sampled sequences of the batch-32 round."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import cod_oracle as orc
+from paper_2609_14717_b200 import synth
+from tests.helpers import oracle_config, rel_err
+
+pytestmark = pytest.mark.gpu
+TOL, GAP = 2e-2, 1e-2
+# Inside a whole round the inputs of layer l > 0 already differ between the two sides: the residual
+# stream, the normalised activations, q/k/v and the attention output are stored in bf16 between the
+# kernels (five layers deep), and in this random-weight model the attention branch dominates the
+# residual stream, so those roundings compound (about 0.5 % per layer; the plain-FMA kernels show the
+# same growth). Each part ALONE, on identical inputs, is held to TOL (K/V rows below, the stand-alone
+# attention test below, the LM-head tests); the downstream taps of the fused round get this bound.
+TOL_COMPOUNDED = 5e-2
+
+
+def _setup(name, seed, sample):
+    """GPU state for the whole batch; oracle state for the sampled sequences only (they are
+    independent of the rest), with identical pool contents for those sequences."""
+    from paper_2609_14717_b200 import binding as B
+    wl = synth.scaled(synth.workload(name), n_rounds=4)
+    sh = wl.shape
+    lay = synth.make_layout(wl, seed)
+    n_pages, mp = int(lay["n_pages"]), int(lay["max_pages_per_seq"])
+    w = synth.make_weights(sh, seed)
+    cfg = B.make_config(sh, wl.S, mp, n_pages)
+    ctx = B.Context(cfg)
+    ctx.set_weights(B.weights_to_device(w, sh.dtype))
+    st_g = B.State(cfg, sh.dtype, wl.S, lay["block_table"], lay["committed_len"])
+    gen = torch.Generator(device="cuda").manual_seed(seed)
+    for l in range(sh.n_layers):                              # everything random, then the sampled sequences exactly
+        st_g.kv_pool[l].copy_(torch.randn(st_g.kv_pool[l].shape, generator=gen, device="cuda").to(torch.bfloat16))
+    cfg_o = oracle_config(sh)
+    L = lay["committed_len"][sample]
+    per = (int(L.max()) + 6 * sh.W) // sh.page + 2
+    bt_o = np.arange(len(sample) * per, dtype=np.int64).reshape(len(sample), per)
+    st_o = orc.OracleState(cfg_o, len(sample), len(sample) * per, bt_o, L)
+    for j, s in enumerate(sample):
+        rng = np.random.default_rng([seed, 77, s])
+        used = (int(L[j]) + sh.page - 1) // sh.page
+        blk = synth.to_storage(rng.standard_normal((sh.n_layers, used, sh.n_kv, 2, sh.page, sh.hd), dtype=np.float32), sh.dtype)
+        st_o.pool[:, bt_o[j, :used]] = blk
+        phys = torch.from_numpy(lay["block_table"][s, :used].astype(np.int64)).cuda()
+        st_g.kv_pool[:, phys] = torch.from_numpy(blk).to(device="cuda", dtype=torch.bfloat16)
+    return wl, lay, w, ctx, cfg, st_g, cfg_o, st_o
+
+
+@pytest.mark.parametrize("name,sample", [("cfg2", [0]), ("cfg3", [5, 22])])
+def test_full_size_round_on_sampled_sequences(name, sample):
+    from paper_2609_14717_b200 import binding as B
+    wl, lay, w, ctx, cfg, st_g, cfg_o, st_o = _setup(name, 11, sample)
+    sh = wl.shape
+    w_o = orc.prepare_weights(w)
+    split, taps = B.Split(wl.S, sh.W), B.Taps(cfg, wl.S)
+    nd = torch.zeros((wl.S, sh.W), dtype=torch.int32, device="cuda")
+    rows = np.concatenate([np.arange(s * sh.W, (s + 1) * sh.W) for s in sample])
+    exempt = 0
+    for r in range(2):
+        rd = synth.make_round(wl, 11, r)
+        ctx.draft_round(torch.from_numpy(rd["draft"]).cuda(), torch.from_numpy(rd["target"]).cuda(),
+                        B.to_device(rd["H"], sh.dtype), wl.S, wl.n_forced, B.COD_CARRY, st_g, split, nd, taps)
+        torch.cuda.synchronize()
+        L0 = st_o.committed_len.copy()
+        res = orc.draft_round(rd["draft"][sample], rd["target"][sample], rd["H"][rows], st_o, w_o, wl.n_forced, orc.MODE_CARRY)
+        got = split.to_host()
+        # integers: exact (slot numbers differ because the oracle uses a compact page table)
+        assert np.array_equal(got["accept_len"], rd["m"])
+        assert np.array_equal(got["accept_len"][sample], res["split"]["accept_len"])
+        assert np.array_equal(got["bonus"][sample], res["split"]["bonus"])
+        assert np.array_equal(got["row_pos"][rows], res["split"]["row_pos"])
+        assert np.array_equal(st_g.committed_len.cpu().numpy()[sample], st_o.committed_len)
+        assert np.array_equal(st_g.carry_len.cpu().numpy()[sample], st_o.carry_len)
+        # K/V rows written this round, through the real page table
+        pool_g, carry_g = st_g.kv_pool, st_g.carry_kv
+        for j, s in enumerate(sample):
+            m = int(res["split"]["accept_len"][j])
+            for l in (0, sh.n_layers - 1):
+                ref, gpu = [], []
+                for p in range(m):
+                    pos = int(L0[j]) + p
+                    pg_o, pg_g, off = int(st_o.block_table[j, pos // sh.page]), int(lay["block_table"][s, pos // sh.page]), pos % sh.page
+                    ref.append(st_o.pool[l, pg_o, :, :, off, :]); gpu.append(pool_g[l, pg_g, :, :, off, :].float().cpu().numpy())
+                c = int(st_o.carry_len[j])
+                if c:
+                    ref.append(st_o.carry[l, j, :, :, :c, :].reshape(-1, sh.hd)); gpu.append(carry_g[l, s, :, :, :c, :].float().cpu().numpy().reshape(-1, sh.hd))
+                assert rel_err(np.concatenate([a.reshape(-1) for a in gpu]), np.concatenate([a.reshape(-1) for a in ref])) <= TOL
+        for l in range(sh.n_layers):
+            assert rel_err(taps.attn_out[l].cpu().numpy()[rows], res["attn_out"][l]) <= (TOL if l == 0 else TOL_COMPOUNDED)
+        assert rel_err(taps.x_final.cpu().numpy()[rows], res["x_final"]) <= TOL_COMPOUNDED
+        sure = res["gap"] >= GAP
+        sure[:, 0] = False
+        assert np.array_equal(nd.cpu().numpy()[sample][sure], res["next_draft"][sure])
+        exempt += int((~sure[:, 1:]).sum())
+    assert ctx.poll_status() == 0
+    assert exempt <= len(sample) * sh.W          # only a handful of near-ties may be exempt
+    ctx.close()
+
+
+@pytest.mark.parametrize("name,sample", [("cfg2", [0]), ("cfg3", [5, 22]), ("cfg4", [1])])
+def test_full_size_attention_alone_on_identical_inputs(name, sample):
+    """cod_block_attn at the benchmark's context lengths and split configuration, same q/k/v and
+    same cache contents on both sides: the 2e-2 bound proper for part 4."""
+    from paper_2609_14717_b200 import binding as B
+    wl, lay, w, ctx, cfg, st_g, cfg_o, st_o = _setup(name, 13, sample)
+    sh = wl.shape
+    rng = np.random.default_rng(5)
+    q = synth.to_storage(rng.standard_normal((wl.S, sh.W, sh.n_q, sh.hd)).astype(np.float32), "bf16")
+    kb = synth.to_storage(rng.standard_normal((wl.S, sh.W, sh.n_kv, sh.hd)).astype(np.float32), "bf16")
+    vb = synth.to_storage(rng.standard_normal((wl.S, sh.W, sh.n_kv, sh.hd)).astype(np.float32), "bf16")
+    lens = rng.integers(0, sh.W + 1, size=wl.S)
+    lens[sample[0]] = sh.W
+    for j, s in enumerate(sample):
+        c = int(lens[s])
+        st_o.carry_len[j] = c
+        if c:
+            blk = synth.to_storage(rng.standard_normal((sh.n_layers, sh.n_kv, 2, c, sh.hd)).astype(np.float32), "bf16")
+            st_o.carry[:, j, :, :, :c, :] = blk
+            st_g.carry_kv[:, s, :, :, :c, :] = B.to_device(blk, "bf16")
+    st_g.carry_len.copy_(torch.from_numpy(lens.astype(np.int32)))
+    out = torch.zeros((wl.S, sh.W, sh.n_q, sh.hd), dtype=torch.bfloat16, device="cuda")
+    mass = torch.zeros((wl.S, sh.W, sh.n_q), dtype=torch.float32, device="cuda")
+    for layer in (0, sh.n_layers - 1):
+        ctx.block_attn(layer, B.to_device(q, "bf16"), B.to_device(kb, "bf16"), B.to_device(vb, "bf16"), st_g, wl.S, 1, out, mass)
+        torch.cuda.synchronize()
+        ref, mref = orc.block_attn(layer, q[sample], kb[sample], vb[sample], st_o, True)
+        assert rel_err(out.float().cpu().numpy()[sample], ref) <= TOL
+        assert np.max(np.abs(mass.cpu().numpy()[sample] - mref)) <= TOL
+    assert ctx.poll_status() == 0
+    ctx.close()
