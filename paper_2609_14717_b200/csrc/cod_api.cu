@@ -81,7 +81,7 @@ int pick_splits(const cod_ctx* c, int n_out, int K, int rows) {
   if (c->cfg.dtype != COD_BF16 || c->force_simt) return 1;
   const int tiles = (n_out + 127) / 128;
   int ctas = tiles * ((rows + 255) / 256);
-  if (rows > 128 && tiles >= c->n_sm) ctas = tiles * ((rows + 511) / 512);   // the paired kernel's 512-row tiles
+  if (rows > 128 && tiles >= c->n_sm / 2) ctas = tiles * ((rows + 511) / 512);   // the paired kernel's 512-row tiles
   const int kb = (K + 63) / 64;
   int splits = c->n_sm / ctas;
   if (splits > COD_MAX_SPLITS) splits = COD_MAX_SPLITS;

@@ -372,9 +372,16 @@ int cod_launch_gemm_tc2(cod_ctx* c, const GemmArgs& g, cudaStream_t st) {
     p.pair_end[i] = pairs;
   }
   p.n_seg = g.n_seg;
-  // two accumulators (512 token rows per pair, weights streamed once) only when there are enough
-  // weight-row pairs to fill the machine that way
-  p.n_acc = (g.n_rows > NT && 2 * pairs >= c->n_sm) ? 2 : 1;
+  // One or two accumulators per pair (256 or 512 token rows; with two the weights stream once):
+  // take whichever needs less time in waves of (SMs / 2) pairs. A k-block costs about 0.42 us with
+  // one accumulator and 0.55 us with two (both are bound by the barrier round trip, not the MMAs).
+  p.n_acc = 1;
+  if (g.n_rows > NT) {
+    const int per_wave = c->n_sm / 2;
+    const int c1 = pairs * ((g.n_rows + NT - 1) / NT) * splits, c2 = pairs * ((g.n_rows + 2 * NT - 1) / (2 * NT)) * splits;
+    const float t1 = 0.42f * ((c1 + per_wave - 1) / per_wave), t2 = 0.55f * ((c2 + per_wave - 1) / per_wave);
+    p.n_acc = t2 < t1 ? 2 : 1;
+  }
   p.stages = p.n_acc == 2 ? 4 : MAX_STAGES;
   p.n_tiles_n = (g.n_rows + p.n_acc * NT - 1) / (p.n_acc * NT);
   p.C = g.C;
