@@ -524,6 +524,72 @@ def run_micro(args):
     ctx.close()
 
 
+def run_sweep(args):
+    """--sweep: the carryover-overhead sweep (configuration 5): batch x block x rejected fraction,
+    each point timed with carryover and with the baseline drafter on identical inputs (graph replay,
+    fixed accepted length m = W - rejected, no forced anchor; plus the anchor corner m = 1)."""
+    import torch
+
+    import __graft_entry__ as entry
+    from paper_2609_14717_b200 import binding as B
+
+    entry.build()
+    torch.cuda.set_device(0)
+    base = synth.workload("cfg5")
+    weights = B.weights_to_device(synth.make_weights(base.shape, args.seed), "bf16")
+    K, Wm = args.steps, args.warmup
+    rows = []
+    for W in (8, 16):
+        for S in (1, 4, 16, 64):
+            points = [(W, 0), (W // 2, 0), (0, 0), (1, 1)]            # (accepted rows m, n_forced)
+            for m, nf in points:
+                wl = synth.sweep_point(S, W, m, n_forced=nf, n_rounds=K + Wm + 2)
+                sh = wl.shape
+                lay = synth.make_layout(wl, args.seed)
+                n_pages, mp = int(lay["n_pages"]), int(lay["max_pages_per_seq"])
+                ctx = B.Context(B.make_config(sh, S, mp, n_pages))
+                ctx.set_weights(weights)
+                state = B.State(ctx.cfg, "bf16", S, lay["block_table"], lay["committed_len"])
+                gen = torch.Generator(device="cuda").manual_seed(args.seed)
+                for l in range(sh.n_layers):
+                    state.kv_pool[l].copy_(torch.randn(state.kv_pool[l].shape, generator=gen, device="cuda").to(torch.bfloat16))
+                rd = synth.make_round(wl, args.seed, 0)
+                d, t = torch.from_numpy(rd["draft"]).cuda(), torch.from_numpy(rd["target"]).cuda()
+                H = B.to_device(rd["H"], "bf16")
+                nd = torch.zeros((S, W), dtype=torch.int32, device="cuda")
+                L0 = state.committed_len.clone()
+                res = {}
+                for mode, name in ((B.COD_CARRY, "carry"), (B.COD_BASELINE, "baseline")):
+                    def one():
+                        ctx.draft_round(d, t, H, S, nf, mode, state, None, nd, None)
+                    state.committed_len.copy_(L0); state.carry_len.zero_()
+                    side = torch.cuda.Stream(); side.wait_stream(torch.cuda.current_stream())
+                    with torch.cuda.stream(side):
+                        one()
+                    torch.cuda.current_stream().wait_stream(side); torch.cuda.synchronize()
+                    g = torch.cuda.CUDAGraph()
+                    with torch.cuda.graph(g):
+                        one()
+                    state.committed_len.copy_(L0); state.carry_len.zero_()
+                    for _ in range(Wm):
+                        g.replay()
+                    torch.cuda.synchronize()
+                    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                    e0.record()
+                    for _ in range(K):
+                        g.replay()
+                    e1.record(); torch.cuda.synchronize()
+                    res[name] = e0.elapsed_time(e1) / K * 1e3
+                status = ctx.poll_status()
+                rows.append({"S": S, "W": W, "m": m, "rejected": W - m, "n_forced": nf, "carry_us": res["carry"],
+                             "baseline_us": res["baseline"], "overhead_pct": 100.0 * (res["carry"] - res["baseline"]) / res["baseline"],
+                             "device_status": status})
+                ctx.close()
+                del state
+                torch.cuda.empty_cache()
+    print(json.dumps({"sweep": "cfg5", "context": 4096, "steps": K, "points": rows}))
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -534,13 +600,16 @@ def main():
     ap.add_argument("--seed", type=int, default=0)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-graph", action="store_true", help="time plain stream launches instead of graph replays")
+    ap.add_argument("--sweep", action="store_true", help="carryover-overhead sweep over batch, block and rejected fraction")
     ap.add_argument("--attn-split", type=int, default=0, help="keys per attention split (0 = library default)")
     ap.add_argument("--micro", default=None, choices=["attn", "lmhead"],
                     help="time one entry point alone (small footprint; meant for profiler captures)")
     args = ap.parse_args()
     if args.warmup < 3:
         args.warmup = 3
-    if args.micro:
+    if args.sweep:
+        run_sweep(args)
+    elif args.micro:
         run_micro(args)
     elif args.impl == "reference":
         run_reference(args)

@@ -209,6 +209,7 @@ int cod_set_weights(cod_ctx* c, const cod_weights* w, cod_stream_t stream) {
     if (!p || misaligned(p)) return COD_ERR_INVALID_ARG;
   c->w = *w;
   c->has_weights = true;
+  c->pdl = false;
   return cod_launch_fcE(c, static_cast<cudaStream_t>(stream));
 }
 
@@ -217,6 +218,7 @@ int cod_verify_accept(cod_ctx* c, const int32_t* draft, const int32_t* target, i
   if (!c || !draft || !target || !st || !st->committed_len || !st->block_table || split_has_null(out))
     return COD_ERR_INVALID_ARG;
   if (check_S(c, S) != COD_OK || n_forced < 0 || n_forced > 1) return COD_ERR_INVALID_ARG;
+  c->pdl = true;
   return cod_launch_verify(c, draft, target, S, n_forced, st, out, static_cast<cudaStream_t>(stream));
 }
 
@@ -256,6 +258,7 @@ int cod_project_kv(cod_ctx* c, const void* H, const cod_split* split, int S, int
   if (!c || !H || !J || split_has_null(split) || misaligned(H) || misaligned(J)) return COD_ERR_INVALID_ARG;
   if (check_S(c, S) != COD_OK || (mode != COD_CARRY && mode != COD_BASELINE)) return COD_ERR_INVALID_ARG;
   if (!c->has_weights) return COD_ERR_NO_WEIGHTS;
+  c->pdl = true;
   return project_impl(c, H, split, S, mode, J, nullptr, nullptr, static_cast<cudaStream_t>(stream));
 }
 
@@ -266,6 +269,7 @@ int cod_scatter_kv(cod_ctx* c, const void* J, const cod_split* split, int S, int
     return COD_ERR_INVALID_ARG;
   if (check_S(c, S) != COD_OK || (mode != COD_CARRY && mode != COD_BASELINE)) return COD_ERR_INVALID_ARG;
   cudaStream_t s = static_cast<cudaStream_t>(stream);
+  c->pdl = true;
   int rc = cod_launch_scatter(c, J, split, S, mode, st, s);
   if (rc != COD_OK) return rc;
   return cod_launch_update_lens(c, split, S, mode, st, s);
@@ -280,6 +284,7 @@ int cod_block_attn(cod_ctx* c, int layer, const void* q, const void* k_blk, cons
     return COD_ERR_INVALID_ARG;
   if (check_S(c, S) != COD_OK || layer < 0 || layer >= c->cfg.n_layers) return COD_ERR_INVALID_ARG;
   cudaStream_t s = static_cast<cudaStream_t>(stream);
+  c->pdl = true;
   int rc = cod_launch_rope_blk_only(c, st->committed_len, S, s);
   if (rc != COD_OK) return rc;
   if ((rc = cod_launch_rope_qk(c, q, k_blk, st->committed_len, S, s)) != COD_OK) return rc;
@@ -300,6 +305,7 @@ int cod_lm_head_argmax(cod_ctx* c, const float* x, int n_rows, int32_t* tok, flo
   if (n_rows < 1 || n_rows > c->R_max) return COD_ERR_INVALID_ARG;
   if (!c->has_weights) return COD_ERR_NO_WEIGHTS;
   cudaStream_t s = static_cast<cudaStream_t>(stream);
+  c->pdl = true;
   int rc = cod_launch_resid_norm(c, nullptr, 0, n_rows, const_cast<float*>(x), c->w.g_final, nullptr, s);
   if (rc != COD_OK) return rc;
   if ((rc = lm_head_impl(c, n_rows, s)) != COD_OK) return rc;
@@ -321,6 +327,7 @@ int cod_draft_round(cod_ctx* c, const int32_t* draft, const int32_t* target, con
   const int R = S * f.block;
   const size_t es = esize(c);
   int rc;
+  c->pdl = true;
 
   // parts 1-3
   if ((rc = cod_launch_verify(c, draft, target, S, n_forced, st, sp, s)) != COD_OK) return rc;

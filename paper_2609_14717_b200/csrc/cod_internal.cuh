@@ -10,6 +10,20 @@
 #define COD_MAX_SPLITS 8          // split-K partial slabs the GEMM workspace can hold
 #define COD_MAX_W 128             // largest supported block size
 
+// ---------------------------------------------------------------------------- dependent launches
+// With few token rows a round is ~45 short kernels, and every kernel is launched with programmatic
+// stream serialisation: its CTAs may become resident while the previous kernel of the stream is
+// still running, so launch latency and CTA set-up overlap that kernel's tail. The first statement
+// of every kernel waits until the previous grid has completed and its memory is visible (before
+// any global access and before any tensor-memory allocation, so a waiting CTA holds nothing an
+// earlier grid still needs). Small grids then let the next grid start launching at once; for
+// grids of more than ~1000 CTAs the early trigger measured slower (the many waiting CTAs of the
+// next grid get in the way) and the next grid starts as this one drains.
+__device__ __forceinline__ void cod_pdl_prologue() {
+  asm volatile("griddepcontrol.wait;" ::: "memory");
+  if (gridDim.x * gridDim.y * gridDim.z <= 1024u) asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+}
+
 // ---------------------------------------------------------------------------- element access
 __device__ __forceinline__ float cod_ld(const float* p) { return *p; }
 __device__ __forceinline__ float cod_ld(const __nv_bfloat16* p) { return __bfloat162float(*p); }
@@ -103,6 +117,7 @@ struct cod_ctx {
   void* zero_page;             // 16 x 128 bf16 zeros (stands in for pages past the end of a split)
   int n_sm;
   bool force_simt;             // COD_F_NO_TENSOR_CORES: plain-FMA kernels only
+  bool pdl;                    // launch kernels as programmatic dependents of their predecessor in the stream
   int64_t launches;
   size_t ws_bytes;
   char* ws;
@@ -149,6 +164,22 @@ struct ProfScope {
   }
   ~ProfScope() { if (slot >= 0) cudaEventRecord(c->prof_ev[2 * slot + 1], st); }
 };
+
+template <typename... KArgs, typename... Args>
+inline cudaError_t cod_launch_pdl(const cod_ctx* c, void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st,
+                                  Args&&... args) {
+  cudaLaunchConfig_t cfg{};
+  cfg.gridDim = grid;
+  cfg.blockDim = block;
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = st;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = c->pdl ? 1 : 0;
+  return cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
+}
 
 // ---------------------------------------------------------------------------- launchers
 // Every launcher enqueues on `st`, bumps ctx->launches, and returns a cod_status.

@@ -23,6 +23,7 @@ k_attn_split(const T* __restrict__ q, const T* __restrict__ kb, const T* __restr
              int layer, int W, int rep, int n_kv, int page, int max_pages, int n_pages, int max_batch,
              int split_len, int max_splits, float* __restrict__ part_o, float* __restrict__ part_ml,
              uint32_t* status) {
+  cod_pdl_prologue();
   extern __shared__ float smem[];
   const int M = W * rep;
   float* Qs = smem;                       // [M][HD]   (pre-scaled by 1/sqrt(hd))
@@ -157,6 +158,7 @@ __global__ void k_attn_combine(const float* __restrict__ part_o, const float* __
                                int use_carry, int S, int W, int rep, int n_kv, int page, int max_pages,
                                int split_len, int max_splits, T* __restrict__ out, float* __restrict__ tap,
                                float* __restrict__ mass) {
+  cod_pdl_prologue();
   const int lane = threadIdx.x & 31;
   const int item = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);   // (s, i, g)
   const int n_q = n_kv * rep;
@@ -204,7 +206,7 @@ int launch_split(cod_ctx* c, int layer, const void* q, const void* kb, const voi
       return COD_ERR_CUDA;
   }
   dim3 grid(c->max_splits, f.n_kv_heads, S);
-  kern<<<grid, NWARP * 32, smem, st>>>(static_cast<const T*>(q), static_cast<const T*>(kb), static_cast<const T*>(vb),
+  cod_launch_pdl(c, kern, grid, NWARP * 32, smem, st, static_cast<const T*>(q), static_cast<const T*>(kb), static_cast<const T*>(vb),
                                        static_cast<const T*>(stt->kv_pool), static_cast<const T*>(stt->carry_kv),
                                        stt->block_table, stt->committed_len, stt->carry_len, use_carry, layer, f.block,
                                        rep, f.n_kv_heads, f.page_size, f.max_pages_per_seq, f.n_pages, f.max_batch,
@@ -225,7 +227,7 @@ int launch_all(cod_ctx* c, int layer, const void* q, const void* kb, const void*
   else return COD_ERR_UNSUPPORTED;
   if (rc != COD_OK) return rc;
   const int items = S * f.block * f.n_q_heads;
-  k_attn_combine<T, HD><<<(items + 3) / 4, 128, 0, st>>>(c->attn_o, c->attn_ml, stt->committed_len, stt->carry_len,
+  cod_launch_pdl(c, k_attn_combine<T, HD>, (items + 3) / 4, 128, 0, st, c->attn_o, c->attn_ml, stt->committed_len, stt->carry_len,
                                                          use_carry, S, f.block, rep, f.n_kv_heads, f.page_size,
                                                          f.max_pages_per_seq, c->split_len, c->max_splits,
                                                          static_cast<T*>(out), tap, mass);

@@ -194,6 +194,7 @@ struct Geo {
 template <bool DUAL>
 __global__ void __launch_bounds__(NTHREADS, 2)
 k_attn_tc(const __grid_constant__ CUtensorMap map_pool, const __grid_constant__ CUtensorMap map_zero, const AttnParams p) {
+  cod_pdl_prologue();
   using G = Geo<DUAL>;
   extern __shared__ uint8_t smem_raw[];
   const uint32_t raw = smem_u32(smem_raw);
@@ -561,6 +562,7 @@ __global__ void k_attn_tc_combine(const float* __restrict__ part_o, const float*
                                   const int* __restrict__ committed_len, int S, int W, int rep, int n_kv,
                                   int max_pages, int split_len, int max_parts, __nv_bfloat16* __restrict__ out,
                                   float* __restrict__ tap, float* __restrict__ mass) {
+  cod_pdl_prologue();
   const int lane = threadIdx.x & 31;
   const int item = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
   const int n_q = n_kv * rep;
@@ -658,10 +660,10 @@ int launch(cod_ctx* c, int layer, const void* q, const void* kb, const void* vb,
     configured = true;
   }
   dim3 grid(c->tc_max_parts, f.n_kv_heads, S);
-  k_attn_tc<DUAL><<<grid, NTHREADS, G::SMEM, st>>>(mp, mz, p);
+  cod_launch_pdl(c, k_attn_tc<DUAL>, grid, NTHREADS, G::SMEM, st, mp, mz, p);
   COD_CHECK_LAUNCH(c);
   const int items = S * f.block * f.n_q_heads;
-  k_attn_tc_combine<DUAL><<<(items + 3) / 4, 128, 0, st>>>(c->attn_o, c->attn_ml, stt->committed_len, S, f.block, p.rep,
+  cod_launch_pdl(c, k_attn_tc_combine<DUAL>, (items + 3) / 4, 128, 0, st, c->attn_o, c->attn_ml, stt->committed_len, S, f.block, p.rep,
                                                            f.n_kv_heads, f.max_pages_per_seq, c->tc_split_len,
                                                            c->tc_max_parts, static_cast<__nv_bfloat16*>(out), tap, mass);
   COD_CHECK_LAUNCH(c);

@@ -13,6 +13,7 @@ constexpr int NT = 256;  // threads: 16 (features, 4 each) x 16 (rows, 2 each)
 
 template <typename T, bool ARGMAX>
 __global__ void __launch_bounds__(NT) k_gemm_simt(GemmArgs g) {
+  cod_pdl_prologue();
   __shared__ float As[BK][BM + 1];
   __shared__ float Bs[BK][BN + 1];
 
@@ -113,8 +114,8 @@ int launch_t(cod_ctx* c, const GemmArgs& g, cudaStream_t st) {
   int n_total = 0;
   for (int i = 0; i < g.n_seg; ++i) n_total += g.seg[i].N;
   dim3 grid((n_total + BN - 1) / BN, (g.n_rows + BM - 1) / BM, g.splits);
-  if (g.amax) k_gemm_simt<T, true><<<grid, NT, 0, st>>>(g);
-  else k_gemm_simt<T, false><<<grid, NT, 0, st>>>(g);
+  if (g.amax) cod_launch_pdl(c, k_gemm_simt<T, true>, grid, NT, 0, st, g);
+  else cod_launch_pdl(c, k_gemm_simt<T, false>, grid, NT, 0, st, g);
   COD_CHECK_LAUNCH(c);
   return COD_OK;
 }

@@ -186,6 +186,7 @@ __device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&v)[32]) {
 __global__ void __launch_bounds__(NTHREADS, 1)
 k_gemm_tc(const __grid_constant__ CUtensorMap map_w0, const __grid_constant__ CUtensorMap map_w1,
           const __grid_constant__ CUtensorMap map_w2, const __grid_constant__ CUtensorMap map_a, const TcParams p) {
+  cod_pdl_prologue();
   extern __shared__ uint8_t smem_raw[];
   // tiles need 1024-byte alignment for the 128-byte swizzle pattern
   const uint32_t raw = smem_u32(smem_raw);
@@ -436,7 +437,7 @@ int cod_launch_gemm_tc(cod_ctx* c, const GemmArgs& g, cudaStream_t st) {
     configured = smem;
   }
   dim3 grid((g.n_rows + p.NT - 1) / p.NT, tiles, splits);
-  k_gemm_tc<<<grid, NTHREADS, smem, st>>>(mw[0], mw[1], mw[2], ma, p);
+  cod_launch_pdl(c, k_gemm_tc, grid, NTHREADS, smem, st, mw[0], mw[1], mw[2], ma, p);
   COD_CHECK_LAUNCH(c);
   return COD_OK;
 }

@@ -26,6 +26,7 @@ __device__ __forceinline__ int valid_rows(const int* n_rows_dev, int n_rows) {
 // column, step 2): the embedding can be added after the contraction, before the norm.
 template <typename T>
 __global__ void k_fcE(const T* __restrict__ fc, const T* __restrict__ e, int D_in, float* __restrict__ out) {
+  cod_pdl_prologue();
   __shared__ float red[33];
   const int n = blockIdx.x;
   float acc = 0.f;
@@ -40,6 +41,7 @@ __global__ void k_fcE(const T* __restrict__ fc, const T* __restrict__ e, int D_i
 template <typename T>
 __global__ void k_gather_rows(const T* __restrict__ src, const int* __restrict__ rows, const int* __restrict__ n_dev,
                               int width, T* __restrict__ dst) {
+  cod_pdl_prologue();
   const int i = blockIdx.x;
   if (i >= *n_dev) return;
   const int row = rows[i];
@@ -56,6 +58,7 @@ __global__ void k_fc_finish(const float* __restrict__ part, int splits, int n_ro
                             const int* __restrict__ a_rows, const int* __restrict__ carry_slot,
                             const float* __restrict__ fcE, const T* __restrict__ gain, int D, float eps,
                             int do_norm, T* __restrict__ z, int z_compact, float* __restrict__ tap) {
+  cod_pdl_prologue();
   __shared__ float red[33];
   const int i = blockIdx.x;
   if (i >= valid_rows(n_rows_dev, n_rows)) return;
@@ -103,6 +106,7 @@ __global__ void k_kv_finish(const float* __restrict__ part, int splits, int n_ro
                             const int* __restrict__ commit_slot, const int* __restrict__ carry_slot,
                             T* __restrict__ pool, T* __restrict__ carry, int page, int n_pages, int W,
                             int max_batch, int to_state) {
+  cod_pdl_prologue();
   const int i = blockIdx.x, l = blockIdx.y;
   if (i >= valid_rows(n_rows_dev, n_rows)) return;
   const int row = a_rows ? a_rows[i] : i;
@@ -158,6 +162,7 @@ __global__ void k_scatter_kv(const T* __restrict__ J, int R_total, int n_kv, int
                              const int* __restrict__ commit_slot, const int* __restrict__ carry_slot,
                              T* __restrict__ pool, T* __restrict__ carry, int page, int n_pages, int W,
                              int max_batch, int use_carry) {
+  cod_pdl_prologue();
   const int row = blockIdx.x, l = blockIdx.y;
   const int kvw = n_kv * hd;
   const int cslot = commit_slot[row], uslot = carry_slot[row];
@@ -189,6 +194,7 @@ __global__ void k_scatter_kv(const T* __restrict__ J, int R_total, int n_kv, int
 
 __global__ void k_update_lens(const int* __restrict__ accept_len, int S, int W, int mode, int max_tokens,
                               int* __restrict__ committed_len, int* __restrict__ carry_len, uint32_t* status) {
+  cod_pdl_prologue();
   const int s = blockIdx.x * blockDim.x + threadIdx.x;
   if (s >= S) return;
   const int m = accept_len[s];
@@ -204,6 +210,7 @@ template <typename T>
 __global__ void k_embed_norm(const T* __restrict__ emb, const int* __restrict__ bonus, int W, int mask_id,
                              int vocab, const T* __restrict__ gain, int D, float eps, float* __restrict__ x,
                              T* __restrict__ a, unsigned long long* __restrict__ amax) {
+  cod_pdl_prologue();
   __shared__ float red[33];
   const int r = blockIdx.x, s = r / W, p = r - s * W;
   int tok = p == 0 ? bonus[s] : mask_id;
@@ -241,6 +248,7 @@ template <typename T>
 __global__ void k_qkv_finish(const float* __restrict__ part, int splits, int R, int n_q, int n_kv, int hd,
                              const float* __restrict__ rope_blk, T* __restrict__ q, T* __restrict__ kb,
                              T* __restrict__ vb) {
+  cod_pdl_prologue();
   // one block per (row, head): heads 0..n_q-1 are q, then n_kv heads of k (both rotated), then n_kv of v
   const int r = blockIdx.x, hh = blockIdx.y;
   const int qw = n_q * hd, kvw = n_kv * hd, half = hd >> 1, ldc = qw + 2 * kvw;
@@ -271,6 +279,7 @@ __global__ void k_qkv_finish(const float* __restrict__ part, int splits, int R, 
 template <typename T>
 __global__ void k_rope_qk(const T* __restrict__ qin, const T* __restrict__ kin, int n_q, int n_kv, int hd,
                           const float* __restrict__ rope_blk, T* __restrict__ q, T* __restrict__ kb) {
+  cod_pdl_prologue();
   const int r = blockIdx.x;
   const int qw = n_q * hd, kvw = n_kv * hd, half = hd >> 1;
   const float* cs = rope_blk + static_cast<size_t>(r) * hd;
@@ -291,6 +300,7 @@ template <typename T>
 __global__ void k_resid_norm(const float* __restrict__ part, int splits, int R, int D, float* x,
                              const T* __restrict__ gain, float eps, T* __restrict__ a, float* __restrict__ tap,
                              unsigned long long* __restrict__ amax) {
+  cod_pdl_prologue();
   __shared__ float red[33];
   const int r = blockIdx.x;
   const int nv = D >> 2;
@@ -327,6 +337,7 @@ __global__ void k_resid_norm(const float* __restrict__ part, int splits, int R, 
 
 __global__ void k_finalize(const unsigned long long* __restrict__ amax, int R, int W, const int* __restrict__ bonus,
                            int* __restrict__ tok, int* __restrict__ next_draft, float* __restrict__ top_logit) {
+  cod_pdl_prologue();
   const int r = blockIdx.x * blockDim.x + threadIdx.x;
   if (r >= R) return;
   const unsigned long long key = amax[r];
@@ -350,8 +361,8 @@ int cod_launch_gather_rows(cod_ctx* c, const void* src, const int* rows, const i
   ProfScope prof(c, COD_K_ROWOPS, st);
   if (n_max <= 0) return COD_OK;
   DISPATCH_T(c,
-             (k_gather_rows<__nv_bfloat16><<<n_max, 256, 0, st>>>(static_cast<const __nv_bfloat16*>(src), rows, n_dev, width, static_cast<__nv_bfloat16*>(dst))),
-             (k_gather_rows<float><<<n_max, 256, 0, st>>>(static_cast<const float*>(src), rows, n_dev, width, static_cast<float*>(dst))));
+             (cod_launch_pdl(c, k_gather_rows<__nv_bfloat16>, n_max, 256, 0, st, static_cast<const __nv_bfloat16*>(src), rows, n_dev, width, static_cast<__nv_bfloat16*>(dst))),
+             (cod_launch_pdl(c, k_gather_rows<float>, n_max, 256, 0, st, static_cast<const float*>(src), rows, n_dev, width, static_cast<float*>(dst))));
   COD_CHECK_LAUNCH(c);
   return COD_OK;
 }
@@ -359,8 +370,8 @@ int cod_launch_gather_rows(cod_ctx* c, const void* src, const int* rows, const i
 int cod_launch_fcE(cod_ctx* c, cudaStream_t st) {
   ProfScope prof(c, COD_K_ROWOPS, st);
   DISPATCH_T(c,
-             (k_fcE<__nv_bfloat16><<<c->D, 256, 0, st>>>(static_cast<const __nv_bfloat16*>(c->w.fc), static_cast<const __nv_bfloat16*>(c->w.e_carry), c->D_in, c->fcE)),
-             (k_fcE<float><<<c->D, 256, 0, st>>>(static_cast<const float*>(c->w.fc), static_cast<const float*>(c->w.e_carry), c->D_in, c->fcE)));
+             (cod_launch_pdl(c, k_fcE<__nv_bfloat16>, c->D, 256, 0, st, static_cast<const __nv_bfloat16*>(c->w.fc), static_cast<const __nv_bfloat16*>(c->w.e_carry), c->D_in, c->fcE)),
+             (cod_launch_pdl(c, k_fcE<float>, c->D, 256, 0, st, static_cast<const float*>(c->w.fc), static_cast<const float*>(c->w.e_carry), c->D_in, c->fcE)));
   COD_CHECK_LAUNCH(c);
   return COD_OK;
 }
@@ -372,8 +383,8 @@ int cod_launch_fc_finish(cod_ctx* c, const float* part, int splits, int n_rows, 
   const int nt = row_threads(c->D);
   const int do_norm = (c->cfg.flags & COD_F_HIDDEN_NORM) ? 1 : 0;
   DISPATCH_T(c,
-             (k_fc_finish<__nv_bfloat16><<<n_rows, nt, 0, st>>>(part, splits, n_rows, n_rows_dev, a_rows, carry_slot, c->fcE, static_cast<const __nv_bfloat16*>(c->w.g_hidden), c->D, c->cfg.rms_eps, do_norm, static_cast<__nv_bfloat16*>(c->z), a_rows ? 1 : 0, tap_z)),
-             (k_fc_finish<float><<<n_rows, nt, 0, st>>>(part, splits, n_rows, n_rows_dev, a_rows, carry_slot, c->fcE, static_cast<const float*>(c->w.g_hidden), c->D, c->cfg.rms_eps, do_norm, static_cast<float*>(c->z), a_rows ? 1 : 0, tap_z)));
+             (cod_launch_pdl(c, k_fc_finish<__nv_bfloat16>, n_rows, nt, 0, st, part, splits, n_rows, n_rows_dev, a_rows, carry_slot, c->fcE, static_cast<const __nv_bfloat16*>(c->w.g_hidden), c->D, c->cfg.rms_eps, do_norm, static_cast<__nv_bfloat16*>(c->z), a_rows ? 1 : 0, tap_z)),
+             (cod_launch_pdl(c, k_fc_finish<float>, n_rows, nt, 0, st, part, splits, n_rows, n_rows_dev, a_rows, carry_slot, c->fcE, static_cast<const float*>(c->w.g_hidden), c->D, c->cfg.rms_eps, do_norm, static_cast<float*>(c->z), a_rows ? 1 : 0, tap_z)));
   COD_CHECK_LAUNCH(c);
   return COD_OK;
 }
@@ -387,8 +398,8 @@ int cod_launch_kv_finish(cod_ctx* c, const float* part, int splits, int n_rows, 
   dim3 grid(n_rows, f.n_layers);
   const int to_state = ds ? 1 : 0;
   DISPATCH_T(c,
-             (k_kv_finish<__nv_bfloat16><<<grid, 128, 0, st>>>(part, splits, n_rows, n_rows_dev, a_rows, c->rope_win, f.n_layers, f.n_kv_heads, f.head_dim, static_cast<__nv_bfloat16*>(J), R_total, sp->commit_slot, sp->carry_slot, ds ? static_cast<__nv_bfloat16*>(ds->kv_pool) : nullptr, ds ? static_cast<__nv_bfloat16*>(ds->carry_kv) : nullptr, f.page_size, f.n_pages, f.block, f.max_batch, to_state)),
-             (k_kv_finish<float><<<grid, 128, 0, st>>>(part, splits, n_rows, n_rows_dev, a_rows, c->rope_win, f.n_layers, f.n_kv_heads, f.head_dim, static_cast<float*>(J), R_total, sp->commit_slot, sp->carry_slot, ds ? static_cast<float*>(ds->kv_pool) : nullptr, ds ? static_cast<float*>(ds->carry_kv) : nullptr, f.page_size, f.n_pages, f.block, f.max_batch, to_state)));
+             (cod_launch_pdl(c, k_kv_finish<__nv_bfloat16>, grid, 128, 0, st, part, splits, n_rows, n_rows_dev, a_rows, c->rope_win, f.n_layers, f.n_kv_heads, f.head_dim, static_cast<__nv_bfloat16*>(J), R_total, sp->commit_slot, sp->carry_slot, ds ? static_cast<__nv_bfloat16*>(ds->kv_pool) : nullptr, ds ? static_cast<__nv_bfloat16*>(ds->carry_kv) : nullptr, f.page_size, f.n_pages, f.block, f.max_batch, to_state)),
+             (cod_launch_pdl(c, k_kv_finish<float>, grid, 128, 0, st, part, splits, n_rows, n_rows_dev, a_rows, c->rope_win, f.n_layers, f.n_kv_heads, f.head_dim, static_cast<float*>(J), R_total, sp->commit_slot, sp->carry_slot, ds ? static_cast<float*>(ds->kv_pool) : nullptr, ds ? static_cast<float*>(ds->carry_kv) : nullptr, f.page_size, f.n_pages, f.block, f.max_batch, to_state)));
   COD_CHECK_LAUNCH(c);
   return COD_OK;
 }
@@ -401,15 +412,15 @@ int cod_launch_scatter(cod_ctx* c, const void* J, const cod_split* sp, int S, in
   dim3 grid(R, f.n_layers);
   const int use_carry = mode == COD_CARRY;
   DISPATCH_T(c,
-             (k_scatter_kv<__nv_bfloat16><<<grid, 128, 0, st>>>(static_cast<const __nv_bfloat16*>(J), R, f.n_kv_heads, f.head_dim, sp->commit_slot, sp->carry_slot, static_cast<__nv_bfloat16*>(ds->kv_pool), static_cast<__nv_bfloat16*>(ds->carry_kv), f.page_size, f.n_pages, f.block, f.max_batch, use_carry)),
-             (k_scatter_kv<float><<<grid, 128, 0, st>>>(static_cast<const float*>(J), R, f.n_kv_heads, f.head_dim, sp->commit_slot, sp->carry_slot, static_cast<float*>(ds->kv_pool), static_cast<float*>(ds->carry_kv), f.page_size, f.n_pages, f.block, f.max_batch, use_carry)));
+             (cod_launch_pdl(c, k_scatter_kv<__nv_bfloat16>, grid, 128, 0, st, static_cast<const __nv_bfloat16*>(J), R, f.n_kv_heads, f.head_dim, sp->commit_slot, sp->carry_slot, static_cast<__nv_bfloat16*>(ds->kv_pool), static_cast<__nv_bfloat16*>(ds->carry_kv), f.page_size, f.n_pages, f.block, f.max_batch, use_carry)),
+             (cod_launch_pdl(c, k_scatter_kv<float>, grid, 128, 0, st, static_cast<const float*>(J), R, f.n_kv_heads, f.head_dim, sp->commit_slot, sp->carry_slot, static_cast<float*>(ds->kv_pool), static_cast<float*>(ds->carry_kv), f.page_size, f.n_pages, f.block, f.max_batch, use_carry)));
   COD_CHECK_LAUNCH(c);
   return COD_OK;
 }
 
 int cod_launch_update_lens(cod_ctx* c, const cod_split* sp, int S, int mode, const cod_state* ds, cudaStream_t st) {
   ProfScope prof(c, COD_K_ROWOPS, st);
-  k_update_lens<<<(S + 127) / 128, 128, 0, st>>>(sp->accept_len, S, c->cfg.block, mode,
+  cod_launch_pdl(c, k_update_lens, (S + 127) / 128, 128, 0, st, sp->accept_len, S, c->cfg.block, mode,
                                                  c->cfg.max_pages_per_seq * c->cfg.page_size, ds->committed_len,
                                                  ds->carry_len, c->status);
   COD_CHECK_LAUNCH(c);
@@ -421,8 +432,8 @@ int cod_launch_embed_norm(cod_ctx* c, const int32_t* bonus, int S, cudaStream_t 
   const cod_config& f = c->cfg;
   const int R = S * f.block;
   DISPATCH_T(c,
-             (k_embed_norm<__nv_bfloat16><<<R, row_threads(c->D), 0, st>>>(static_cast<const __nv_bfloat16*>(c->w.emb), bonus, f.block, f.mask_token_id, f.vocab, static_cast<const __nv_bfloat16*>(c->w.g_attn), c->D, f.rms_eps, c->x, static_cast<__nv_bfloat16*>(c->a), c->amax)),
-             (k_embed_norm<float><<<R, row_threads(c->D), 0, st>>>(static_cast<const float*>(c->w.emb), bonus, f.block, f.mask_token_id, f.vocab, static_cast<const float*>(c->w.g_attn), c->D, f.rms_eps, c->x, static_cast<float*>(c->a), c->amax)));
+             (cod_launch_pdl(c, k_embed_norm<__nv_bfloat16>, R, row_threads(c->D), 0, st, static_cast<const __nv_bfloat16*>(c->w.emb), bonus, f.block, f.mask_token_id, f.vocab, static_cast<const __nv_bfloat16*>(c->w.g_attn), c->D, f.rms_eps, c->x, static_cast<__nv_bfloat16*>(c->a), c->amax)),
+             (cod_launch_pdl(c, k_embed_norm<float>, R, row_threads(c->D), 0, st, static_cast<const float*>(c->w.emb), bonus, f.block, f.mask_token_id, f.vocab, static_cast<const float*>(c->w.g_attn), c->D, f.rms_eps, c->x, static_cast<float*>(c->a), c->amax)));
   COD_CHECK_LAUNCH(c);
   return COD_OK;
 }
@@ -432,8 +443,8 @@ int cod_launch_qkv_finish(cod_ctx* c, const float* part, int splits, int R, cuda
   const cod_config& f = c->cfg;
   const dim3 grid(R, f.n_q_heads + 2 * f.n_kv_heads);
   DISPATCH_T(c,
-             (k_qkv_finish<__nv_bfloat16><<<grid, 64, 0, st>>>(part, splits, R, f.n_q_heads, f.n_kv_heads, f.head_dim, c->rope_blk, static_cast<__nv_bfloat16*>(c->q), static_cast<__nv_bfloat16*>(c->kb), static_cast<__nv_bfloat16*>(c->vb))),
-             (k_qkv_finish<float><<<grid, 64, 0, st>>>(part, splits, R, f.n_q_heads, f.n_kv_heads, f.head_dim, c->rope_blk, static_cast<float*>(c->q), static_cast<float*>(c->kb), static_cast<float*>(c->vb))));
+             (cod_launch_pdl(c, k_qkv_finish<__nv_bfloat16>, grid, 64, 0, st, part, splits, R, f.n_q_heads, f.n_kv_heads, f.head_dim, c->rope_blk, static_cast<__nv_bfloat16*>(c->q), static_cast<__nv_bfloat16*>(c->kb), static_cast<__nv_bfloat16*>(c->vb))),
+             (cod_launch_pdl(c, k_qkv_finish<float>, grid, 64, 0, st, part, splits, R, f.n_q_heads, f.n_kv_heads, f.head_dim, c->rope_blk, static_cast<float*>(c->q), static_cast<float*>(c->kb), static_cast<float*>(c->vb))));
   COD_CHECK_LAUNCH(c);
   return COD_OK;
 }
@@ -445,8 +456,8 @@ int cod_launch_rope_qk(cod_ctx* c, const void* q, const void* k, const int32_t* 
   const cod_config& f = c->cfg;
   const int R = S * f.block;
   DISPATCH_T(c,
-             (k_rope_qk<__nv_bfloat16><<<R, 256, 0, st>>>(static_cast<const __nv_bfloat16*>(q), static_cast<const __nv_bfloat16*>(k), f.n_q_heads, f.n_kv_heads, f.head_dim, c->rope_blk, static_cast<__nv_bfloat16*>(c->q), static_cast<__nv_bfloat16*>(c->kb))),
-             (k_rope_qk<float><<<R, 256, 0, st>>>(static_cast<const float*>(q), static_cast<const float*>(k), f.n_q_heads, f.n_kv_heads, f.head_dim, c->rope_blk, static_cast<float*>(c->q), static_cast<float*>(c->kb))));
+             (cod_launch_pdl(c, k_rope_qk<__nv_bfloat16>, R, 256, 0, st, static_cast<const __nv_bfloat16*>(q), static_cast<const __nv_bfloat16*>(k), f.n_q_heads, f.n_kv_heads, f.head_dim, c->rope_blk, static_cast<__nv_bfloat16*>(c->q), static_cast<__nv_bfloat16*>(c->kb))),
+             (cod_launch_pdl(c, k_rope_qk<float>, R, 256, 0, st, static_cast<const float*>(q), static_cast<const float*>(k), f.n_q_heads, f.n_kv_heads, f.head_dim, c->rope_blk, static_cast<float*>(c->q), static_cast<float*>(c->kb))));
   COD_CHECK_LAUNCH(c);
   return COD_OK;
 }
@@ -455,8 +466,8 @@ int cod_launch_resid_norm(cod_ctx* c, const float* part, int splits, int R, floa
                           float* tap_x, cudaStream_t st) {
   ProfScope prof(c, COD_K_ROWOPS, st);
   DISPATCH_T(c,
-             (k_resid_norm<__nv_bfloat16><<<R, row_threads(c->D), 0, st>>>(part, splits, R, c->D, x, static_cast<const __nv_bfloat16*>(gain), c->cfg.rms_eps, static_cast<__nv_bfloat16*>(c->a), tap_x, c->amax)),
-             (k_resid_norm<float><<<R, row_threads(c->D), 0, st>>>(part, splits, R, c->D, x, static_cast<const float*>(gain), c->cfg.rms_eps, static_cast<float*>(c->a), tap_x, c->amax)));
+             (cod_launch_pdl(c, k_resid_norm<__nv_bfloat16>, R, row_threads(c->D), 0, st, part, splits, R, c->D, x, static_cast<const __nv_bfloat16*>(gain), c->cfg.rms_eps, static_cast<__nv_bfloat16*>(c->a), tap_x, c->amax)),
+             (cod_launch_pdl(c, k_resid_norm<float>, R, row_threads(c->D), 0, st, part, splits, R, c->D, x, static_cast<const float*>(gain), c->cfg.rms_eps, static_cast<float*>(c->a), tap_x, c->amax)));
   COD_CHECK_LAUNCH(c);
   return COD_OK;
 }
@@ -464,7 +475,7 @@ int cod_launch_resid_norm(cod_ctx* c, const float* part, int splits, int R, floa
 int cod_launch_finalize(cod_ctx* c, int R, int W, const int32_t* bonus, int32_t* tok, int32_t* next_draft,
                         float* top_logit, cudaStream_t st) {
   ProfScope prof(c, COD_K_ROWOPS, st);
-  k_finalize<<<(R + 127) / 128, 128, 0, st>>>(c->amax, R, W, bonus, tok, next_draft, top_logit);
+  cod_launch_pdl(c, k_finalize, (R + 127) / 128, 128, 0, st, c->amax, R, W, bonus, tok, next_draft, top_logit);
   COD_CHECK_LAUNCH(c);
   return COD_OK;
 }

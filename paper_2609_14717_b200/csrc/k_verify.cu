@@ -11,6 +11,7 @@ k_verify_accept(const int32_t* __restrict__ draft, const int32_t* __restrict__ t
                 int n_forced, int vocab, int page, int max_pages, int n_pages,
                 const int32_t* __restrict__ committed_len, const int32_t* __restrict__ block_table,
                 cod_split out, uint32_t* status) {
+  cod_pdl_prologue();
   extern __shared__ int sm[];
   int* s_m = sm;              // [S]
   int* s_acc = sm + S;        // [S+1]
@@ -99,6 +100,7 @@ k_verify_accept(const int32_t* __restrict__ draft, const int32_t* __restrict__ t
 __global__ void k_rope_tables(const int32_t* __restrict__ committed_len, const int32_t* __restrict__ accept_len,
                               const double* __restrict__ inv_freq, int S, int W, int half,
                               float* __restrict__ rope_win, float* __restrict__ rope_blk) {
+  cod_pdl_prologue();
   const int r = blockIdx.x, s = r / W, p = r - s * W;
   const int L = max(committed_len[s], 0);
   const int m = accept_len ? accept_len[s] : 0;
@@ -122,11 +124,11 @@ int cod_launch_verify(cod_ctx* c, const int32_t* draft, const int32_t* target, i
   ProfScope prof(c, COD_K_VERIFY, st);
   const int W = c->cfg.block;
   const size_t smem = static_cast<size_t>(2 * S + 2) * sizeof(int);
-  k_verify_accept<<<1, 1024, smem, st>>>(draft, target, S, W, n_forced, c->cfg.vocab, c->cfg.page_size,
+  cod_launch_pdl(c, k_verify_accept, 1, 1024, smem, st, draft, target, S, W, n_forced, c->cfg.vocab, c->cfg.page_size,
                                          c->cfg.max_pages_per_seq, c->cfg.n_pages, state->committed_len,
                                          state->block_table, *out, c->status);
   COD_CHECK_LAUNCH(c);
-  k_rope_tables<<<S * W, 64, 0, st>>>(state->committed_len, out->accept_len, c->inv_freq_d, S, W, c->half,
+  cod_launch_pdl(c, k_rope_tables, S * W, 64, 0, st, state->committed_len, out->accept_len, c->inv_freq_d, S, W, c->half,
                                       c->rope_win, c->rope_blk);
   COD_CHECK_LAUNCH(c);
   return COD_OK;
@@ -134,7 +136,7 @@ int cod_launch_verify(cod_ctx* c, const int32_t* draft, const int32_t* target, i
 
 int cod_launch_rope_blk_only(cod_ctx* c, const int32_t* committed_len, int S, cudaStream_t st) {
   ProfScope prof(c, COD_K_VERIFY, st);
-  k_rope_tables<<<S * c->cfg.block, 64, 0, st>>>(committed_len, nullptr, c->inv_freq_d, S, c->cfg.block, c->half,
+  cod_launch_pdl(c, k_rope_tables, S * c->cfg.block, 64, 0, st, committed_len, nullptr, c->inv_freq_d, S, c->cfg.block, c->half,
                                                  nullptr, c->rope_blk);
   COD_CHECK_LAUNCH(c);
   return COD_OK;
