@@ -20,17 +20,16 @@
 //
 //   warps 0-3 softmax / accumulation     warp 4 TMA producer     warp 5 MMA issuer
 // Every mbarrier wait is bounded and raises COD_DEV_TIMEOUT instead of spinning forever.
-#include <cuda.h>
-
-#include "cod_internal.cuh"
+#include "tc_common.cuh"
 
 namespace {
+
+using namespace tc;
 
 constexpr int HD = 128, PAGE = 16, KT = 64;           // head size, page size, keys per tile
 constexpr int NTHREADS = 224;     // 4 softmax warps, K producer, MMA issuer, V producer
 constexpr uint32_t TILE_BYTES = KT * HD * 2;           // one 64-key K or V tile: 16 KB
 constexpr uint32_t HALF_BYTES = KT * 128;              // 64 keys x 64 elements: 8 KB
-constexpr long long WAIT_LIMIT_CYCLES = 4000000000ll;
 
 struct AttnParams {
   const __nv_bfloat16 *q, *kb, *vb;     // rotated q [R, n_q*hd]; rotated k_blk, v_blk [R, n_kv*hd]
@@ -44,131 +43,8 @@ struct AttnParams {
   uint32_t* status;
 };
 
-// ------------------------------------------------------------------ PTX wrappers
-__device__ __forceinline__ uint32_t smem_u32(const void* p) { return static_cast<uint32_t>(__cvta_generic_to_shared(p)); }
-__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
-  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count));
-}
-__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
-  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
-}
-__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
-  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
-}
-__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
-  uint32_t ok;
-  asm volatile(
-      "{\n\t.reg .pred p;\n\t"
-      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
-      "selp.u32 %0, 1, 0, p;\n\t}"
-      : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
-  return ok != 0;
-}
-// Bounded wait. The common case (phase already complete, or completing within a few polls) never
-// reads a timer; after that the SM cycle counter bounds the wait (about 2 s at the maximum clock),
-// then the CTA raises COD_DEV_TIMEOUT and every role leaves through the abort flag.
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, uint32_t* status) {
-#pragma unroll 1
-  for (int i = 0; i < 64; ++i)
-    if (mbar_try_wait(bar, parity)) return true;
-  const long long t0 = clock64();
-  for (;;) {
-#pragma unroll 1
-    for (int i = 0; i < 256; ++i)
-      if (mbar_try_wait(bar, parity)) return true;
-    if (*abort_flag) return false;
-    if (clock64() - t0 > WAIT_LIMIT_CYCLES) {
-      *abort_flag = 1;
-      atomicOr(status, COD_DEV_TIMEOUT);
-      return false;
-    }
-  }
-}
-__device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap* map, int c0, int c1, int c2, uint32_t bar) {
-  asm volatile(
-      "cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4}], [%5];"
-      ::"r"(dst), "l"(reinterpret_cast<uint64_t>(map)), "r"(c0), "r"(c1), "r"(c2), "r"(bar) : "memory");
-}
-__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
-__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
-__device__ __forceinline__ void fence_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
-__device__ __forceinline__ void tmem_alloc(uint32_t dst_smem, uint32_t cols) {
-  asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(dst_smem), "r"(cols) : "memory");
-  asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
-}
-__device__ __forceinline__ void tmem_dealloc(uint32_t taddr, uint32_t cols) {
-  asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(cols) : "memory");
-}
-__device__ __forceinline__ void umma_bf16(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, uint32_t accumulate) {
-  asm volatile(
-      "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
-      "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
-      ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate) : "memory");
-}
-__device__ __forceinline__ void umma_commit(uint32_t bar) {
-  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
-}
-__device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&v)[32]) {
-  asm volatile(
-      "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
-      "{%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31}, [%32];"
-      : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]),
-        "=r"(v[8]), "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15]),
-        "=r"(v[16]), "=r"(v[17]), "=r"(v[18]), "=r"(v[19]), "=r"(v[20]), "=r"(v[21]), "=r"(v[22]), "=r"(v[23]),
-        "=r"(v[24]), "=r"(v[25]), "=r"(v[26]), "=r"(v[27]), "=r"(v[28]), "=r"(v[29]), "=r"(v[30]), "=r"(v[31])
-      : "r"(taddr) : "memory");
-  asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
-}
 
-__device__ __forceinline__ void tmem_st32(uint32_t taddr, const uint32_t (&v)[32]) {
-  asm volatile(
-      "tcgen05.st.sync.aligned.32x32b.x32.b32 [%0], "
-      "{%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31,%32};"
-      ::"r"(taddr), "r"(v[0]), "r"(v[1]), "r"(v[2]), "r"(v[3]), "r"(v[4]), "r"(v[5]), "r"(v[6]), "r"(v[7]),
-        "r"(v[8]), "r"(v[9]), "r"(v[10]), "r"(v[11]), "r"(v[12]), "r"(v[13]), "r"(v[14]), "r"(v[15]),
-        "r"(v[16]), "r"(v[17]), "r"(v[18]), "r"(v[19]), "r"(v[20]), "r"(v[21]), "r"(v[22]), "r"(v[23]),
-        "r"(v[24]), "r"(v[25]), "r"(v[26]), "r"(v[27]), "r"(v[28]), "r"(v[29]), "r"(v[30]), "r"(v[31])
-      : "memory");
-  asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
-}
-__device__ __forceinline__ float ex2_approx(float x) {
-  float y;
-  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
-  return y;
-}
 
-// K-major operand, 128-byte rows, 128-byte swizzle, 8-row groups 1024 bytes apart.
-__device__ __forceinline__ uint64_t desc_kmajor(uint32_t saddr) {
-  uint64_t d = 0;
-  d |= static_cast<uint64_t>((saddr & 0x3FFFFu) >> 4);
-  d |= static_cast<uint64_t>(1) << 16;
-  d |= static_cast<uint64_t>(1024 >> 4) << 32;
-  d |= static_cast<uint64_t>(1) << 46;
-  d |= static_cast<uint64_t>(2) << 61;
-  return d;
-}
-// MN-major operand (V tile: rows are keys, 64 contiguous head elements per 128-byte row): the
-// next 64 head elements sit HALF_BYTES further (leading offset), the next 8 keys 1024 bytes
-// further (stride offset).
-__device__ __forceinline__ uint64_t desc_mnmajor(uint32_t saddr) {
-  uint64_t d = 0;
-  d |= static_cast<uint64_t>((saddr & 0x3FFFFu) >> 4);
-  d |= static_cast<uint64_t>(HALF_BYTES >> 4) << 16;
-  d |= static_cast<uint64_t>(1024 >> 4) << 32;
-  d |= static_cast<uint64_t>(1) << 46;
-  d |= static_cast<uint64_t>(2) << 61;
-  return d;
-}
-__device__ __forceinline__ uint32_t instr_desc(int m, int n, int b_mn_major) {
-  uint32_t d = 0;
-  d |= 1u << 4;                                  // float accumulator
-  d |= 1u << 7;                                  // A: bf16
-  d |= 1u << 10;                                 // B: bf16
-  d |= static_cast<uint32_t>(b_mn_major) << 16;  // B major
-  d |= static_cast<uint32_t>(n >> 3) << 17;
-  d |= static_cast<uint32_t>(m >> 4) << 24;
-  return d;
-}
 
 template <bool DUAL>
 struct Geo {
@@ -320,7 +196,7 @@ k_attn_tc(const __grid_constant__ CUtensorMap map_pool, const __grid_constant__ 
     if (lane == 0 && n_it > 0) {
       const uint32_t idesc_qk = instr_desc(G::MROWS, KT, 0);
       const uint32_t idesc_pv = instr_desc(G::MROWS, HD, 1);
-      const uint64_t q_desc = desc_kmajor(base);
+      const uint64_t q_desc = desc_kmajor_sw128(base);
       bool ok = true;
       auto issue_qk = [&](int it) -> bool {
         const int slot = it % G::NK;
@@ -328,7 +204,7 @@ k_attn_tc(const __grid_constant__ CUtensorMap map_pool, const __grid_constant__ 
         tc_fence_after();
 #pragma unroll
         for (int t = 0; t < G::TILES; ++t) {
-          const uint64_t k_desc = desc_kmajor(base + G::OFF_K + slot * G::SLOT + t * TILE_BYTES);
+          const uint64_t k_desc = desc_kmajor_sw128(base + G::OFF_K + slot * G::SLOT + t * TILE_BYTES);
           const uint32_t d = tmem_base + G::COL_S + (it & 1) * KT + (static_cast<uint32_t>(16 * t) << 16);
 #pragma unroll
           for (int k = 0; k < HD / 16; ++k) {
@@ -352,8 +228,8 @@ k_attn_tc(const __grid_constant__ CUtensorMap map_pool, const __grid_constant__ 
         tc_fence_after();
 #pragma unroll
         for (int t = 0; t < G::TILES; ++t) {
-          const uint64_t p_desc = desc_kmajor(base + G::OFF_P + t * G::P_TILE);
-          const uint64_t v_desc = desc_mnmajor(base + G::OFF_V + slot * G::SLOT + t * TILE_BYTES);
+          const uint64_t p_desc = desc_kmajor_sw128(base + G::OFF_P + t * G::P_TILE);
+          const uint64_t v_desc = desc_mnmajor_sw128(base + G::OFF_V + slot * G::SLOT + t * TILE_BYTES, HALF_BYTES);
           const uint32_t d = tmem_base + G::COL_O + (static_cast<uint32_t>(16 * t) << 16);
 #pragma unroll
           for (int kk = 0; kk < KT / 16; ++kk)       // 16 keys per MMA: 32 bytes along P's rows, 16 rows of V
@@ -607,35 +483,7 @@ __global__ void k_attn_tc_combine(const float* __restrict__ part_o, const float*
   if (mass && lane == 0) mass[item] = lc * inv;
 }
 
-typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
-                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
-                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
-EncodeTiledFn encode_fn() {
-  static EncodeTiledFn fn = nullptr;
-  static bool tried = false;
-  if (!tried) {
-    tried = true;
-    void* ptr = nullptr;
-    cudaDriverEntryPointQueryResult q;
-    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &ptr, cudaEnableDefault, &q) == cudaSuccess &&
-        q == cudaDriverEntryPointSuccess)
-      fn = reinterpret_cast<EncodeTiledFn>(ptr);
-  }
-  return fn;
-}
 
-// Rows of 128 bf16 seen as (64 elements, 2 halves, rows); a box is one half of 16 consecutive rows.
-bool make_rows_map(CUtensorMap* m, const void* ptr, uint64_t rows) {
-  EncodeTiledFn fn = encode_fn();
-  if (!fn) return false;
-  cuuint64_t gdim[3] = {64, 2, rows};
-  cuuint64_t gstride[2] = {128, 256};
-  cuuint32_t box[3] = {64, 1, PAGE};
-  cuuint32_t estr[3] = {1, 1, 1};
-  return fn(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(ptr), gdim, gstride, box, estr,
-            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
-            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
-}
 
 template <bool DUAL>
 int launch(cod_ctx* c, int layer, const void* q, const void* kb, const void* vb, const cod_state* stt, int S,
@@ -644,7 +492,7 @@ int launch(cod_ctx* c, int layer, const void* q, const void* kb, const void* vb,
   const cod_config& f = c->cfg;
   CUtensorMap mp, mz;
   const uint64_t rows = static_cast<uint64_t>(f.n_layers) * f.n_pages * f.n_kv_heads * 2 * PAGE;
-  if (!make_rows_map(&mp, stt->kv_pool, rows) || !make_rows_map(&mz, c->zero_page, PAGE)) return COD_ERR_CUDA;
+  if (!make_map_rows128(&mp, stt->kv_pool, rows, PAGE) || !make_map_rows128(&mz, c->zero_page, PAGE, PAGE)) return COD_ERR_CUDA;
   AttnParams p{};
   p.q = static_cast<const __nv_bfloat16*>(q); p.kb = static_cast<const __nv_bfloat16*>(kb); p.vb = static_cast<const __nv_bfloat16*>(vb);
   p.pool = static_cast<const __nv_bfloat16*>(stt->kv_pool); p.carry = static_cast<const __nv_bfloat16*>(stt->carry_kv);

@@ -14,18 +14,17 @@
 // Epilogues: float partial sums (split-K slabs, reduced by the row-wise kernels), or a fused
 // per-token argmax over the weight rows for the LM head (logits are never stored).
 // Every mbarrier wait is bounded: on expiry the CTA raises COD_DEV_TIMEOUT and leaves cleanly.
-#include <cuda.h>
-
-#include "cod_internal.cuh"
+#include "tc_common.cuh"
 
 namespace {
+
+using namespace tc;
 
 constexpr int BM = 128;       // weight rows per CTA (MMA M)
 constexpr int BK = 64;        // K elements per stage = one 128-byte swizzled row of bf16
 constexpr int UK = 16;        // K elements per tcgen05.mma (kind::f16)
 constexpr int NTHREADS = 192;
 constexpr uint32_t A_TILE_BYTES = BM * BK * 2;   // 16 KB
-constexpr long long WAIT_LIMIT_CYCLES = 4000000000ll;
 
 struct TcParams {
   int K;
@@ -35,7 +34,6 @@ struct TcParams {
   int NT;                     // token rows per CTA = MMA N (multiple of 16, <= 256)
   int tmem_cols;              // power of two >= max(32, NT)
   int stages;
-  int prefetch;
   int seg_tile_end[3];        // cumulative count of 128-row tiles after each weight segment
   int seg_N[3];
   int n_seg;
@@ -45,143 +43,14 @@ struct TcParams {
   uint32_t* status;
 };
 
-// ------------------------------------------------------------------ PTX wrappers
-__device__ __forceinline__ uint32_t smem_u32(const void* p) { return static_cast<uint32_t>(__cvta_generic_to_shared(p)); }
 
-__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
-  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count));
-}
-__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
-  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
-}
-__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
-  uint32_t ok;
-  asm volatile(
-      "{\n\t.reg .pred p;\n\t"
-      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
-      "selp.u32 %0, 1, 0, p;\n\t}"
-      : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
-  return ok != 0;
-}
-// Bounded wait. The common case (phase already complete, or completing within a few polls) never
-// reads a timer; after that the SM cycle counter bounds the wait (about 2 s at the maximum clock),
-// then the CTA raises COD_DEV_TIMEOUT and every role leaves through the abort flag.
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, uint32_t* status) {
-#pragma unroll 1
-  for (int i = 0; i < 64; ++i)
-    if (mbar_try_wait(bar, parity)) return true;
-  const long long t0 = clock64();
-  for (;;) {
-#pragma unroll 1
-    for (int i = 0; i < 256; ++i)
-      if (mbar_try_wait(bar, parity)) return true;
-    if (*abort_flag) return false;
-    if (clock64() - t0 > WAIT_LIMIT_CYCLES) {
-      *abort_flag = 1;
-      atomicOr(status, COD_DEV_TIMEOUT);
-      return false;
-    }
-  }
-}
-__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, int c0, int c1, uint32_t bar) {
-  asm volatile(
-      "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
-      ::"r"(dst), "l"(reinterpret_cast<uint64_t>(map)), "r"(c0), "r"(c1), "r"(bar) : "memory");
-}
 
-// brings a weight tile into L2 only: the HBM latency is paid long before the tile's ring slot frees up
-__device__ __forceinline__ void tma_prefetch_2d(const CUtensorMap* map, int c0, int c1) {
-  asm volatile("cp.async.bulk.prefetch.tensor.2d.L2.global.tile [%0, {%1, %2}];"
-               ::"l"(reinterpret_cast<uint64_t>(map)), "r"(c0), "r"(c1) : "memory");
-}
-__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
-__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
 
-__device__ __forceinline__ void tmem_alloc(uint32_t dst_smem, uint32_t cols) {
-  asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(dst_smem), "r"(cols) : "memory");
-  asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
-}
-__device__ __forceinline__ void tmem_dealloc(uint32_t taddr, uint32_t cols) {
-  asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(cols) : "memory");
-}
 
-// D[tmem] (+)= A[smem] * B[smem]^T, bf16 operands, float accumulator
-__device__ __forceinline__ void umma_bf16(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, uint32_t accumulate) {
-  asm volatile(
-      "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
-      "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
-      ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate) : "memory");
-}
-// the mbarrier is arrived on once all MMAs issued so far by this thread have completed
-__device__ __forceinline__ void umma_commit(uint32_t bar) {
-  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
-}
 
-__device__ __forceinline__ void tmem_ld16(uint32_t taddr, uint32_t (&v)[16]) {
-  asm volatile(
-      "tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15}, [%16];"
-      : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]),
-        "=r"(v[8]), "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15])
-      : "r"(taddr) : "memory");
-  asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
-}
 
-// Shared-memory operand descriptor: K-major tile whose rows are 128 bytes (64 bf16), 128-byte
-// swizzle, groups of 8 rows 1024 bytes apart; descriptor version 1 (Blackwell).
-__device__ __forceinline__ uint64_t smem_desc_sw128(uint32_t saddr) {
-  uint64_t d = 0;
-  d |= static_cast<uint64_t>((saddr & 0x3FFFFu) >> 4);          // start address            bits [0,14)
-  d |= static_cast<uint64_t>(1) << 16;                          // leading byte offset (unused for swizzled K-major)
-  d |= static_cast<uint64_t>(1024 >> 4) << 32;                  // stride byte offset        bits [32,46)
-  d |= static_cast<uint64_t>(1) << 46;                          // version                   bits [46,48)
-  d |= static_cast<uint64_t>(2) << 61;                          // layout: 128-byte swizzle  bits [61,64)
-  return d;
-}
-// Instruction descriptor: bf16 x bf16 -> float, both operands K-major, M = 128, N = n.
-__device__ __forceinline__ uint32_t instr_desc(int n) {
-  uint32_t d = 0;
-  d |= 1u << 4;                                  // accumulator format: float
-  d |= 1u << 7;                                  // A format: bf16
-  d |= 1u << 10;                                 // B format: bf16
-  d |= static_cast<uint32_t>(n >> 3) << 17;      // N / 8
-  d |= static_cast<uint32_t>(BM >> 4) << 24;     // M / 16
-  return d;
-}
 
-__device__ __forceinline__ unsigned order_key(float v) {
-  const unsigned u = __float_as_uint(v);
-  return (u & 0x80000000u) ? ~u : (u | 0x80000000u);
-}
 
-// Column-wise maximum over the 32 lanes of a warp for 32 columns at once: every lane brings one
-// packed key per column; after five exchange rounds (16 + 8 + 4 + 2 + 1 shuffles) lane L holds
-// the maximum of column L. The keys carry the row index, so this is an argmax with the lowest
-// row winning ties.
-__device__ __forceinline__ unsigned long long warp_colmax32(unsigned long long (&k)[32], int lane) {
-#pragma unroll
-  for (int off = 16; off >= 1; off >>= 1) {
-    const bool hi = (lane & off) != 0;
-#pragma unroll
-    for (int c = 0; c < off; ++c) {
-      const unsigned long long send = hi ? k[c] : k[c + off];
-      const unsigned long long mine = hi ? k[c + off] : k[c];
-      const unsigned long long recv = __shfl_xor_sync(0xffffffffu, send, off);
-      k[c] = recv > mine ? recv : mine;
-    }
-  }
-  return k[0];
-}
-__device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&v)[32]) {
-  asm volatile(
-      "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
-      "{%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31}, [%32];"
-      : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]),
-        "=r"(v[8]), "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15]),
-        "=r"(v[16]), "=r"(v[17]), "=r"(v[18]), "=r"(v[19]), "=r"(v[20]), "=r"(v[21]), "=r"(v[22]), "=r"(v[23]),
-        "=r"(v[24]), "=r"(v[25]), "=r"(v[26]), "=r"(v[27]), "=r"(v[28]), "=r"(v[29]), "=r"(v[30]), "=r"(v[31])
-      : "r"(taddr) : "memory");
-  asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
-}
 
 __global__ void __launch_bounds__(NTHREADS, 1)
 k_gemm_tc(const __grid_constant__ CUtensorMap map_w0, const __grid_constant__ CUtensorMap map_w1,
@@ -237,10 +106,7 @@ k_gemm_tc(const __grid_constant__ CUtensorMap map_w0, const __grid_constant__ CU
   if (warp == 4) {
     // ------------------------------------------------ TMA producer
     if (lane == 0) {
-      const int pf = p.prefetch;                          // k-blocks of weights kept in flight towards L2
-      for (int it = p.stages; it < min(n_kb, p.stages + pf); ++it) tma_prefetch_2d(map_w, (kb0 + it) * BK, f0);
       for (int it = 0; it < n_kb; ++it) {
-        if (pf > 0 && it + p.stages + pf < n_kb) tma_prefetch_2d(map_w, (kb0 + it + p.stages + pf) * BK, f0);
         const int s = it % p.stages, use = it / p.stages;
         if (use > 0 && !mbar_wait(smem_u32(empty_bar + s), (use - 1) & 1, abort_flag, p.status)) break;
         const uint32_t fb = smem_u32(full_bar + s);
@@ -254,7 +120,7 @@ k_gemm_tc(const __grid_constant__ CUtensorMap map_w0, const __grid_constant__ CU
   } else if (warp == 5) {
     // ------------------------------------------------ MMA issuer
     if (lane == 0) {
-      const uint32_t idesc = instr_desc(p.NT);
+      const uint32_t idesc = instr_desc(BM, p.NT, 0);
       bool ok = true;
       for (int it = 0; it < n_kb && ok; ++it) {
         const int s = it % p.stages, use = it / p.stages;
@@ -262,7 +128,7 @@ k_gemm_tc(const __grid_constant__ CUtensorMap map_w0, const __grid_constant__ CU
         if (!ok) break;
         tc_fence_after();
         const uint32_t a_addr = base + s * stage_bytes;
-        const uint64_t a_desc = smem_desc_sw128(a_addr), b_desc = smem_desc_sw128(a_addr + A_TILE_BYTES);
+        const uint64_t a_desc = desc_kmajor_sw128(a_addr), b_desc = desc_kmajor_sw128(a_addr + A_TILE_BYTES);
 #pragma unroll
         for (int k = 0; k < BK / UK; ++k)       // advance 32 bytes (16 bf16) along K inside the swizzled row
           umma_bf16(tmem_base, a_desc + (k * UK * 2 >> 4), b_desc + (k * UK * 2 >> 4), idesc, (it | k) ? 1u : 0u);
@@ -341,36 +207,8 @@ k_gemm_tc(const __grid_constant__ CUtensorMap map_w0, const __grid_constant__ CU
 }
 
 // ------------------------------------------------------------------ host side
-typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
-                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
-                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
 
-EncodeTiledFn encode_fn() {
-  static EncodeTiledFn fn = nullptr;
-  static bool tried = false;
-  if (!tried) {
-    tried = true;
-    void* p = nullptr;
-    cudaDriverEntryPointQueryResult q;
-    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) == cudaSuccess &&
-        q == cudaDriverEntryPointSuccess)
-      fn = reinterpret_cast<EncodeTiledFn>(p);
-  }
-  return fn;
-}
 
-// bf16 matrix [rows, K] with row stride ld (elements); box = box_rows x 64 columns, 128-byte swizzle
-bool make_map(CUtensorMap* m, const void* ptr, uint64_t rows, uint64_t K, uint64_t ld, uint32_t box_rows) {
-  EncodeTiledFn fn = encode_fn();
-  if (!fn) return false;
-  cuuint64_t gdim[2] = {K, rows};
-  cuuint64_t gstride[1] = {ld * 2};
-  cuuint32_t box[2] = {static_cast<cuuint32_t>(BK), box_rows};
-  cuuint32_t estr[2] = {1, 1};
-  return fn(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(ptr), gdim, gstride, box, estr,
-            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
-            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
-}
 
 }  // namespace
 
@@ -407,7 +245,6 @@ int cod_launch_gemm_tc(cod_ctx* c, const GemmArgs& g, cudaStream_t st) {
   if (stages > p.kb_per_split) stages = p.kb_per_split;
   if (stages < 1) stages = 1;
   p.stages = stages;
-  p.prefetch = 0;
   int tiles = 0;
   for (int i = 0; i < 3; ++i) {
     if (i < g.n_seg) {
@@ -425,9 +262,9 @@ int cod_launch_gemm_tc(cod_ctx* c, const GemmArgs& g, cudaStream_t st) {
   CUtensorMap mw[3], ma;
   for (int i = 0; i < 3; ++i) {
     const int j = i < g.n_seg ? i : 0;
-    if (!make_map(&mw[i], g.seg[j].B, g.seg[j].N, g.K, g.K, BM)) return COD_ERR_CUDA;
+    if (!make_map_2d(&mw[i], g.seg[j].B, g.seg[j].N, g.K, g.K, BM)) return COD_ERR_CUDA;
   }
-  if (!make_map(&ma, g.A, g.n_rows, g.K, g.lda, p.NT)) return COD_ERR_CUDA;
+  if (!make_map_2d(&ma, g.A, g.n_rows, g.K, g.lda, p.NT)) return COD_ERR_CUDA;
 
   const size_t smem = static_cast<size_t>(stages) * stage_bytes + 1024 /* alignment slack */ + 34 * 8 + 4 * p.NT * 8;
   static size_t configured = 0;

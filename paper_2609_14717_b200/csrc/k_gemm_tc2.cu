@@ -17,11 +17,11 @@
 // No load is delivered to more than one CTA. Waits are bounded as in k_gemm_tc; the only
 // unbounded synchronisation is the hardware cluster barrier, which every thread reaches
 // unconditionally.
-#include <cuda.h>
-
-#include "cod_internal.cuh"
+#include "tc_common.cuh"
 
 namespace {
+
+using namespace tc;
 
 constexpr int BM = 128;       // weight rows per CTA (256 per pair)
 constexpr int BK = 64;
@@ -31,8 +31,6 @@ constexpr int NTHREADS = 192;
 constexpr uint32_t A_TILE_BYTES = BM * BK * 2;          // 16 KB
 constexpr uint32_t B_TILE_BYTES = (NT / 2) * BK * 2;    // 16 KB
 constexpr int MAX_STAGES = 6;   // one accumulator: 6 stages of 32 KB; two: 4 stages of 48 KB
-constexpr long long WAIT_LIMIT_CYCLES = 4000000000ll;
-constexpr uint32_t PEER_MASK = 0xFEFFFFFFu;             // shared::cluster address of the even-ranked CTA's copy
 
 struct Tc2Params {
   int K, kb_total, kb_per_split;
@@ -50,121 +48,7 @@ struct Tc2Params {
   uint32_t* status;
 };
 
-__device__ __forceinline__ uint32_t smem_u32(const void* p) { return static_cast<uint32_t>(__cvta_generic_to_shared(p)); }
-__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
-  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count));
-}
-__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
-  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
-}
-__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
-  uint32_t ok;
-  asm volatile(
-      "{\n\t.reg .pred p;\n\t"
-      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
-      "selp.u32 %0, 1, 0, p;\n\t}"
-      : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
-  return ok != 0;
-}
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, uint32_t* status) {
-#pragma unroll 1
-  for (int i = 0; i < 64; ++i)
-    if (mbar_try_wait(bar, parity)) return true;
-  const long long t0 = clock64();
-  for (;;) {
-#pragma unroll 1
-    for (int i = 0; i < 256; ++i)
-      if (mbar_try_wait(bar, parity)) return true;
-    if (*abort_flag) return false;
-    if (clock64() - t0 > WAIT_LIMIT_CYCLES) {
-      *abort_flag = 1;
-      atomicOr(status, COD_DEV_TIMEOUT);
-      return false;
-    }
-  }
-}
-// the copy lands in this CTA's shared memory; its bytes are counted on the leader's barrier
-__device__ __forceinline__ void tma_load_2d_pair(uint32_t dst, const CUtensorMap* map, int c0, int c1, uint32_t leader_bar) {
-  asm volatile(
-      "cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
-      ::"r"(dst), "l"(reinterpret_cast<uint64_t>(map)), "r"(c0), "r"(c1), "r"(leader_bar) : "memory");
-}
-__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
-__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
-__device__ __forceinline__ void cluster_sync_all() {
-  asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
-  asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
-}
-__device__ __forceinline__ void tmem_alloc_pair(uint32_t dst_smem, uint32_t cols) {
-  asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(dst_smem), "r"(cols) : "memory");
-  asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
-}
-__device__ __forceinline__ void tmem_dealloc_pair(uint32_t taddr, uint32_t cols) {
-  asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(cols) : "memory");
-}
-__device__ __forceinline__ void umma_bf16_pair(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, uint32_t accumulate) {
-  const uint32_t z = 0u;   // no accumulator lane is masked off
-  asm volatile(
-      "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
-      "tcgen05.mma.cta_group::2.kind::f16 [%0], %1, %2, %3, {%5, %5, %5, %5, %5, %5, %5, %5}, p;\n\t}"
-      ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate), "r"(z) : "memory");
-}
-// arrive on the barrier at this offset in every CTA of the mask once the MMAs issued so far are done
-__device__ __forceinline__ void umma_commit_pair(uint32_t bar, uint16_t cta_mask) {
-  asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;"
-               ::"r"(bar), "h"(cta_mask) : "memory");
-}
-__device__ __forceinline__ void tmem_ld16(uint32_t taddr, uint32_t (&v)[16]) {
-  asm volatile(
-      "tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15}, [%16];"
-      : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]),
-        "=r"(v[8]), "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15])
-      : "r"(taddr) : "memory");
-  asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
-}
-__device__ __forceinline__ uint64_t smem_desc_sw128(uint32_t saddr) {
-  uint64_t d = 0;
-  d |= static_cast<uint64_t>((saddr & 0x3FFFFu) >> 4);
-  d |= static_cast<uint64_t>(1) << 16;
-  d |= static_cast<uint64_t>(1024 >> 4) << 32;
-  d |= static_cast<uint64_t>(1) << 46;
-  d |= static_cast<uint64_t>(2) << 61;
-  return d;
-}
-__device__ __forceinline__ unsigned order_key(float v) {
-  const unsigned u = __float_as_uint(v);
-  return (u & 0x80000000u) ? ~u : (u | 0x80000000u);
-}
 
-// Column-wise maximum over the 32 lanes of a warp for 32 columns at once: every lane brings one
-// packed key per column; after five exchange rounds (16 + 8 + 4 + 2 + 1 shuffles) lane L holds
-// the maximum of column L. The keys carry the row index, so this is an argmax with the lowest
-// row winning ties.
-__device__ __forceinline__ unsigned long long warp_colmax32(unsigned long long (&k)[32], int lane) {
-#pragma unroll
-  for (int off = 16; off >= 1; off >>= 1) {
-    const bool hi = (lane & off) != 0;
-#pragma unroll
-    for (int c = 0; c < off; ++c) {
-      const unsigned long long send = hi ? k[c] : k[c + off];
-      const unsigned long long mine = hi ? k[c + off] : k[c];
-      const unsigned long long recv = __shfl_xor_sync(0xffffffffu, send, off);
-      k[c] = recv > mine ? recv : mine;
-    }
-  }
-  return k[0];
-}
-__device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&v)[32]) {
-  asm volatile(
-      "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
-      "{%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31}, [%32];"
-      : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]),
-        "=r"(v[8]), "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15]),
-        "=r"(v[16]), "=r"(v[17]), "=r"(v[18]), "=r"(v[19]), "=r"(v[20]), "=r"(v[21]), "=r"(v[22]), "=r"(v[23]),
-        "=r"(v[24]), "=r"(v[25]), "=r"(v[26]), "=r"(v[27]), "=r"(v[28]), "=r"(v[29]), "=r"(v[30]), "=r"(v[31])
-      : "r"(taddr) : "memory");
-  asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
-}
 
 __global__ void __launch_bounds__(NTHREADS, 1)
 k_gemm_tc2(const __grid_constant__ CUtensorMap map_w0, const __grid_constant__ CUtensorMap map_w1,
@@ -236,8 +120,7 @@ k_gemm_tc2(const __grid_constant__ CUtensorMap map_w0, const __grid_constant__ C
   } else if (warp == 5) {
     if (lane == 0 && rank == 0) {
       // bf16 x bf16 -> float, K-major operands, M = 256 (both CTAs), N = 256
-      const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | (static_cast<uint32_t>(NT >> 3) << 17) |
-                             (static_cast<uint32_t>((2 * BM) >> 4) << 24);
+      const uint32_t idesc = instr_desc(2 * BM, NT, 0);
       bool ok = true;
       for (int it = 0; it < n_kb && ok; ++it) {
         const int s = it % STAGES, use = it / STAGES;
@@ -245,9 +128,9 @@ k_gemm_tc2(const __grid_constant__ CUtensorMap map_w0, const __grid_constant__ C
         if (!ok) break;
         tc_fence_after();
         const uint32_t a_addr = base + s * STAGE_BYTES;
-        const uint64_t a_desc = smem_desc_sw128(a_addr);
+        const uint64_t a_desc = desc_kmajor_sw128(a_addr);
         for (int a = 0; a < p.n_acc; ++a) {
-          const uint64_t b_desc = smem_desc_sw128(a_addr + A_TILE_BYTES + a * B_TILE_BYTES);
+          const uint64_t b_desc = desc_kmajor_sw128(a_addr + A_TILE_BYTES + a * B_TILE_BYTES);
 #pragma unroll
           for (int k = 0; k < BK / UK; ++k)
             umma_bf16_pair(tmem_base + a * NT, a_desc + (k * UK * 2 >> 4), b_desc + (k * UK * 2 >> 4), idesc, (it | k) ? 1u : 0u);
@@ -312,33 +195,6 @@ k_gemm_tc2(const __grid_constant__ CUtensorMap map_w0, const __grid_constant__ C
   }
 }
 
-typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
-                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
-                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
-EncodeTiledFn encode_fn() {
-  static EncodeTiledFn fn = nullptr;
-  static bool tried = false;
-  if (!tried) {
-    tried = true;
-    void* ptr = nullptr;
-    cudaDriverEntryPointQueryResult q;
-    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &ptr, cudaEnableDefault, &q) == cudaSuccess &&
-        q == cudaDriverEntryPointSuccess)
-      fn = reinterpret_cast<EncodeTiledFn>(ptr);
-  }
-  return fn;
-}
-bool make_map(CUtensorMap* m, const void* ptr, uint64_t rows, uint64_t K, uint64_t ld, uint32_t box_rows) {
-  EncodeTiledFn fn = encode_fn();
-  if (!fn) return false;
-  cuuint64_t gdim[2] = {K, rows};
-  cuuint64_t gstride[1] = {ld * 2};
-  cuuint32_t box[2] = {static_cast<cuuint32_t>(BK), box_rows};
-  cuuint32_t estr[2] = {1, 1};
-  return fn(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(ptr), gdim, gstride, box, estr,
-            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
-            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
-}
 
 }  // namespace
 
@@ -393,9 +249,9 @@ int cod_launch_gemm_tc2(cod_ctx* c, const GemmArgs& g, cudaStream_t st) {
   CUtensorMap mw[3], ma;
   for (int i = 0; i < 3; ++i) {
     const int j = i < g.n_seg ? i : 0;
-    if (!make_map(&mw[i], g.seg[j].B, g.seg[j].N, g.K, g.K, BM)) return COD_ERR_CUDA;
+    if (!make_map_2d(&mw[i], g.seg[j].B, g.seg[j].N, g.K, g.K, BM)) return COD_ERR_CUDA;
   }
-  if (!make_map(&ma, g.A, g.n_rows, g.K, g.lda, NT / 2)) return COD_ERR_CUDA;
+  if (!make_map_2d(&ma, g.A, g.n_rows, g.K, g.lda, NT / 2)) return COD_ERR_CUDA;
 
   const size_t smem = static_cast<size_t>(p.stages) * (A_TILE_BYTES + p.n_acc * B_TILE_BYTES) + 1024 + 18 * 8 +
                       static_cast<size_t>(4) * p.n_acc * NT * 8;
