@@ -42,6 +42,7 @@ struct Tc2Params {
   int n_tiles_n;              // token tiles
   int n_acc;                  // accumulators per pair: 1 (256 token rows) or 2 (512)
   int stages;
+  int staged;                 // epilogue transposes through shared memory (needs 16-byte aligned feature runs)
   float* C;
   int ldc;
   unsigned long long* amax;
@@ -49,6 +50,17 @@ struct Tc2Params {
 };
 
 
+
+// AND of a predicate over the 128 threads of warps 0-3 (named barrier 1)
+__device__ __forceinline__ bool bar_and_128(bool v) {
+  uint32_t r;
+  asm volatile(
+      "{\n\t.reg .pred p, q;\n\tsetp.ne.b32 q, %1, 0;\n\t"
+      "bar.red.and.pred p, 1, 128, q;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(r) : "r"(static_cast<uint32_t>(v)) : "memory");
+  return r != 0;
+}
 
 __global__ void __launch_bounds__(NTHREADS, 1)
 k_gemm_tc2(const __grid_constant__ CUtensorMap map_w0, const __grid_constant__ CUtensorMap map_w1,
@@ -140,12 +152,36 @@ k_gemm_tc2(const __grid_constant__ CUtensorMap map_w0, const __grid_constant__ C
       if (ok && n_kb > 0) umma_commit_pair(smem_u32(acc_bar), 3);
     }
   } else if (n_kb > 0) {
-    const bool ok = mbar_wait(smem_u32(acc_bar), 0, abort_flag, p.status);
+    // one verdict for the four epilogue warps (they meet at a named barrier below)
+    const bool ok = bar_and_128(mbar_wait(smem_u32(acc_bar), 0, abort_flag, p.status));
     tc_fence_after();
     const int f = f0 + warp * 32 + lane;
     const bool f_ok = f < seg_N;
     const uint32_t t_lane = tmem_base + (static_cast<uint32_t>(warp * 32) << 16);
-    if (ok && p.amax == nullptr) {
+    if (ok && p.amax == nullptr && p.staged) {
+      // The accumulator has features on lanes and tokens on columns; C wants a token's features
+      // contiguous. Transpose 32 tokens at a time through the (now idle) pipeline buffers and
+      // store whole 512-byte feature runs: two 16 KB buffers, one barrier of the four epilogue
+      // warps per chunk.
+      float* C = p.C + static_cast<size_t>(split) * p.n_rows * p.ldc + col0;
+      float* stage = reinterpret_cast<float*>(sm);
+      const int f_left = seg_N - f0;                       // features of this CTA that exist
+      for (int c = 0, q = 0; c < NTOK && i0 + c < n_rows; c += 32, q ^= 1) {
+        uint32_t v[32];
+        tmem_ld32(t_lane + c, v);
+        float* buf = stage + q * (32 * BM);
+#pragma unroll
+        for (int j = 0; j < 32; ++j) buf[j * BM + warp * 32 + lane] = __uint_as_float(v[j]);
+        asm volatile("bar.sync 1, 128;" ::: "memory");
+#pragma unroll
+        for (int t = 0; t < 8; ++t) {
+          const int tok = warp * 8 + t, i = i0 + c + tok;
+          if (i < n_rows && lane * 4 < f_left)
+            *reinterpret_cast<float4*>(C + static_cast<size_t>(i) * p.ldc + lane * 4) =
+                *reinterpret_cast<const float4*>(buf + tok * BM + lane * 4);
+        }
+      }
+    } else if (ok && p.amax == nullptr) {
       float* C = p.C + static_cast<size_t>(split) * p.n_rows * p.ldc;
       for (int c = 0; c < NTOK; c += 16) {
         if (i0 + c >= n_rows) break;
@@ -243,6 +279,8 @@ int cod_launch_gemm_tc2(cod_ctx* c, const GemmArgs& g, cudaStream_t st) {
   p.n_tiles_n = (g.n_rows + p.n_acc * NT - 1) / (p.n_acc * NT);
   p.C = g.C;
   p.ldc = g.ldc;
+  p.staged = (g.ldc % 4 == 0) && ((reinterpret_cast<uintptr_t>(g.C) & 15u) == 0);
+  for (int i = 0; i < g.n_seg; ++i) p.staged = p.staged && (g.seg[i].N % 4 == 0);
   p.amax = g.amax;
   p.status = c->status;
 
