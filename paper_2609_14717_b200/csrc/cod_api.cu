@@ -79,11 +79,14 @@ bool state_has_null(const cod_state* s) {
 // split-K factor so that (feature tiles x splits) fills the machine; partial slabs must fit
 int pick_splits(const cod_ctx* c, int n_out, int K, int rows) {
   if (c->cfg.dtype != COD_BF16 || c->force_simt) return 1;
+  if (rows > 128) {                         // the paired kernel: its own time model picks tiles and splits
+    int splits, n_acc;
+    cod_plan_gemm_tc2(c->n_sm, n_out, K, rows, COD_MAX_SPLITS, 0, &splits, &n_acc);
+    return splits;
+  }
   const int tiles = (n_out + 127) / 128;
-  int ctas = tiles * ((rows + 255) / 256);
-  if (rows > 128 && tiles >= c->n_sm / 2) ctas = tiles * ((rows + 511) / 512);   // the paired kernel's 512-row tiles
   const int kb = (K + 63) / 64;
-  int splits = c->n_sm / ctas;
+  int splits = c->n_sm / tiles;
   if (splits > COD_MAX_SPLITS) splits = COD_MAX_SPLITS;
   if (splits > kb / 4) splits = kb / 4;
   if (splits < 1) splits = 1;

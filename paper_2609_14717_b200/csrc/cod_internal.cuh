@@ -100,6 +100,7 @@ struct GemmArgs {
   float* C;               // [splits][n_rows][ldc] float partial sums
   int ldc;
   int splits;             // split-K factor (1 = none)
+  int n_acc;              // paired kernel: accumulators per CTA pair (1 or 2); 0 = let the launcher choose
   unsigned long long* amax;  // if non-null: per-row packed argmax over N instead of storing C
   int klass;              // cod_kernel_class, for the optional timing
 };
@@ -189,6 +190,11 @@ int cod_launch_gemm(cod_ctx* c, const GemmArgs& g, cudaStream_t st);
 int cod_launch_gemm_simt(cod_ctx* c, const GemmArgs& g, cudaStream_t st);
 bool cod_gemm_tc_supported(const cod_ctx* c, const GemmArgs& g);
 bool cod_gemm_tc2_supported(const cod_ctx* c, const GemmArgs& g);
+// Tile plan of the paired kernel for n_out weight rows, K and `rows` token rows: split-K factor and
+// accumulators per pair with the least modelled time (no split is left empty). fixed_splits > 0 pins
+// the split-K factor and only chooses the accumulators.
+void cod_plan_gemm_tc2(int n_sm, int n_out, int K, int rows, int max_splits, int fixed_splits, int* splits,
+                       int* n_acc);
 int cod_launch_gemm_tc2(cod_ctx* c, const GemmArgs& g, cudaStream_t st);
 bool cod_attn_tc_supported(const cod_ctx* c);
 int cod_launch_attn_tc(cod_ctx* c, int layer, const void* q, const void* kb, const void* vb, const cod_state* stt,

@@ -234,6 +234,37 @@ k_gemm_tc2(const __grid_constant__ CUtensorMap map_w0, const __grid_constant__ C
 
 }  // namespace
 
+// Modelled time of one launch in SM cycles, from device-side cycle stamps of this kernel:
+//   per CTA pair: ~7500 cycles before the first MMA (setup, first operands), then per 64-wide
+//   k-block ~760 cycles with one accumulator (the operand fetch of 32 KB per SM is the limit) and
+//   ~1000 with two (48 KB per SM, the tensor pipe is the limit), then ~3000 cycles of epilogue per
+//   accumulator; pairs run in waves of n_sm / 2;
+//   every split beyond the first costs one more float slab written here and read by the
+//   finishing kernel (~30 bytes per cycle per SM through L2).
+void cod_plan_gemm_tc2(int n_sm, int n_out, int K, int rows, int max_splits, int fixed_splits, int* splits_out,
+                       int* n_acc_out) {
+  const int kb = (K + BK - 1) / BK;
+  const int pairs = (n_out + 2 * BM - 1) / (2 * BM);
+  const int per_wave = n_sm / 2 > 0 ? n_sm / 2 : 1;
+  double best = 0.0;
+  int best_s = 1, best_a = 1;
+  for (int a = 1; a <= (rows > NT ? 2 : 1); ++a) {
+    const int tiles_n = (rows + a * NT - 1) / (a * NT);
+    for (int s = 1; s <= max_splits && s <= (kb / 4 > 0 ? kb / 4 : 1); ++s) {
+      const int per = (kb + s - 1) / s;
+      if ((kb + per - 1) / per != s) continue;              // would leave an empty split
+      if (fixed_splits > 0 && s != fixed_splits) continue;
+      const int waves = (pairs * tiles_n * s + per_wave - 1) / per_wave;
+      const double t_main = waves * (7500.0 + per * (a == 2 ? 1000.0 : 760.0) + a * 3000.0);
+      const double t_slabs = (s - 1) * 2.0 * rows * static_cast<double>(n_out) * 4.0 / (30.0 * n_sm);
+      const double t = t_main + t_slabs;
+      if (best == 0.0 || t < best) { best = t; best_s = s; best_a = a; }
+    }
+  }
+  *splits_out = best_s;
+  *n_acc_out = best_a;
+}
+
 // Used for more than 128 token rows; every weight segment but the last must be whole 256-row pairs.
 bool cod_gemm_tc2_supported(const cod_ctx* c, const GemmArgs& g) {
   if (c->cfg.dtype != COD_BF16 || g.a_rows != nullptr || g.n_rows <= 128) return false;
@@ -265,15 +296,11 @@ int cod_launch_gemm_tc2(cod_ctx* c, const GemmArgs& g, cudaStream_t st) {
     p.pair_end[i] = pairs;
   }
   p.n_seg = g.n_seg;
-  // One or two accumulators per pair (256 or 512 token rows; with two the weights stream once):
-  // take whichever needs less time in waves of (SMs / 2) pairs. A k-block costs about 0.42 us with
-  // one accumulator and 0.55 us with two (both are bound by the barrier round trip, not the MMAs).
-  p.n_acc = 1;
-  if (g.n_rows > NT) {
-    const int per_wave = c->n_sm / 2;
-    const int c1 = pairs * ((g.n_rows + NT - 1) / NT) * splits, c2 = pairs * ((g.n_rows + 2 * NT - 1) / (2 * NT)) * splits;
-    const float t1 = 0.42f * ((c1 + per_wave - 1) / per_wave), t2 = 0.55f * ((c2 + per_wave - 1) / per_wave);
-    p.n_acc = t2 < t1 ? 2 : 1;
+  p.n_acc = g.n_acc;
+  if (p.n_acc != 1 && p.n_acc != 2) {
+    int s_unused, n_out = 0;
+    for (int i = 0; i < g.n_seg; ++i) n_out += g.seg[i].N;
+    cod_plan_gemm_tc2(c->n_sm, n_out, g.K, g.n_rows, COD_MAX_SPLITS, splits, &s_unused, &p.n_acc);
   }
   p.stages = p.n_acc == 2 ? 4 : MAX_STAGES;
   p.n_tiles_n = (g.n_rows + p.n_acc * NT - 1) / (p.n_acc * NT);
