@@ -71,13 +71,17 @@ __global__ void k_fc_finish(const float* __restrict__ part, int splits, int n_ro
   for (int t = 0; t < ROW_MAXV; ++t) {
     const int j = threadIdx.x + t * blockDim.x;
     v[t] = make_float4(0.f, 0.f, 0.f, 0.f);
-    if (j < nv) {
-      for (int s = 0; s < splits; ++s)
-        v[t] = f4_add(v[t], *reinterpret_cast<const float4*>(part + (static_cast<size_t>(s) * n_rows + i) * D + 4 * j));
-      if (rej) v[t] = f4_add(v[t], *reinterpret_cast<const float4*>(fcE + 4 * j));
-      ss += f4_ss(v[t]);
+    if (j < nv && rej) v[t] = *reinterpret_cast<const float4*>(fcE + 4 * j);
+  }
+  for (int s = 0; s < splits; ++s) {        // slots inside: all of a slab's loads are in flight together
+#pragma unroll
+    for (int t = 0; t < ROW_MAXV; ++t) {
+      const int j = threadIdx.x + t * blockDim.x;
+      if (j < nv) v[t] = f4_add(v[t], *reinterpret_cast<const float4*>(part + (static_cast<size_t>(s) * n_rows + i) * D + 4 * j));
     }
   }
+#pragma unroll
+  for (int t = 0; t < ROW_MAXV; ++t) ss += f4_ss(v[t]);
   ss = cod_block_sum(ss, red);
   const float scale = do_norm ? rsqrtf(ss / static_cast<float>(D) + eps) : 1.f;
 #pragma unroll
@@ -135,22 +139,25 @@ __global__ void k_kv_finish(const float* __restrict__ part, int splits, int n_ro
       return;   // nowhere to go (position beyond the page table: already flagged)
     }
   }
-  for (int e = threadIdx.x; e < n_kv * half; e += blockDim.x) {
-    const int h = e / half, j = e - h * half;
-    float k1 = 0.f, k2 = 0.f, v1 = 0.f, v2 = 0.f;
+  // hd / 8 threads per head: 4 consecutive elements of the lower half and their RoPE partners
+  const int tph = half >> 2;
+  for (int e = threadIdx.x; e < n_kv * tph; e += blockDim.x) {
+    const int h = e / tph, j = (e - h * tph) * 4;
+    float4 k1 = make_float4(0.f, 0.f, 0.f, 0.f), k2 = k1, v1 = k1, v2 = k1;
+    const float* p = part + static_cast<size_t>(i) * ldc + l * kvw + h * hd + j;
+    const size_t slab = static_cast<size_t>(n_rows) * ldc;
     for (int s = 0; s < splits; ++s) {
-      const float* p = part + (static_cast<size_t>(s) * n_rows + i) * ldc;
-      k1 += p[l * kvw + h * hd + j];
-      k2 += p[l * kvw + h * hd + j + half];
-      v1 += p[Ld * kvw + l * kvw + h * hd + j];
-      v2 += p[Ld * kvw + l * kvw + h * hd + j + half];
+      k1 = f4_add(k1, *reinterpret_cast<const float4*>(p + s * slab));
+      k2 = f4_add(k2, *reinterpret_cast<const float4*>(p + s * slab + half));
+      v1 = f4_add(v1, *reinterpret_cast<const float4*>(p + s * slab + Ld * kvw));
+      v2 = f4_add(v2, *reinterpret_cast<const float4*>(p + s * slab + Ld * kvw + half));
     }
-    const float c = cs[j], sn = cs[half + j];
+    const float4 c = *reinterpret_cast<const float4*>(cs + j), sn = *reinterpret_cast<const float4*>(cs + half + j);
     T* kd = dstK + h * h_stride;
-    cod_st(kd + j, k1 * c - k2 * sn);
-    cod_st(kd + j + half, k2 * c + k1 * sn);
-    cod_st(kd + kv_stride + j, v1);
-    cod_st(kd + kv_stride + j + half, v2);
+    cod_st4(kd + j, make_float4(k1.x * c.x - k2.x * sn.x, k1.y * c.y - k2.y * sn.y, k1.z * c.z - k2.z * sn.z, k1.w * c.w - k2.w * sn.w));
+    cod_st4(kd + j + half, make_float4(k2.x * c.x + k1.x * sn.x, k2.y * c.y + k1.y * sn.y, k2.z * c.z + k1.z * sn.z, k2.w * c.w + k1.w * sn.w));
+    cod_st4(kd + kv_stride + j, v1);
+    cod_st4(kd + kv_stride + j + half, v2);
   }
 }
 
@@ -247,31 +254,34 @@ __global__ void k_embed_norm(const T* __restrict__ emb, const int* __restrict__ 
 template <typename T>
 __global__ void k_qkv_finish(const float* __restrict__ part, int splits, int R, int n_q, int n_kv, int hd,
                              const float* __restrict__ rope_blk, T* __restrict__ q, T* __restrict__ kb,
-                             T* __restrict__ vb) {
+                             T* __restrict__ vb, int hpb) {
   cod_pdl_prologue();
-  // one block per (row, head): heads 0..n_q-1 are q, then n_kv heads of k (both rotated), then n_kv of v
-  const int r = blockIdx.x, hh = blockIdx.y;
-  const int qw = n_q * hd, kvw = n_kv * hd, half = hd >> 1, ldc = qw + 2 * kvw;
-  const float* cs = rope_blk + static_cast<size_t>(r) * hd;
+  // A block covers hpb heads of one row; hd / 8 threads per head, each owning 4 consecutive
+  // elements of the lower half and their partners in the upper half (the pairs RoPE mixes).
+  // Heads 0..n_q-1 are q, then n_kv heads of k (both rotated), then n_kv heads of v.
+  const int half = hd >> 1, tph = half >> 2;
+  const int r = blockIdx.x, hh = blockIdx.y * hpb + threadIdx.x / tph, j = (threadIdx.x % tph) * 4;
+  if (hh >= n_q + 2 * n_kv) return;
+  const int qw = n_q * hd, kvw = n_kv * hd, ldc = qw + 2 * kvw;
+  const float* p = part + static_cast<size_t>(r) * ldc + hh * hd + j;
+  const size_t slab = static_cast<size_t>(R) * ldc;
+  float4 a = make_float4(0.f, 0.f, 0.f, 0.f), b = a;
+  for (int s = 0; s < splits; ++s) {
+    a = f4_add(a, *reinterpret_cast<const float4*>(p + s * slab));
+    b = f4_add(b, *reinterpret_cast<const float4*>(p + s * slab + half));
+  }
   const bool rot = hh < n_q + n_kv;
   T* dst = hh < n_q ? q + static_cast<size_t>(r) * qw + hh * hd
                     : (rot ? kb + static_cast<size_t>(r) * kvw + (hh - n_q) * hd
                            : vb + static_cast<size_t>(r) * kvw + (hh - n_q - n_kv) * hd);
-  for (int j = threadIdx.x; j < half; j += blockDim.x) {
-    float a = 0.f, b = 0.f;
-    for (int s = 0; s < splits; ++s) {
-      const float* p = part + (static_cast<size_t>(s) * R + r) * ldc + hh * hd;
-      a += p[j];
-      b += p[j + half];
-    }
-    if (rot) {
-      const float c = cs[j], sn = cs[half + j];
-      cod_st(dst + j, a * c - b * sn);
-      cod_st(dst + j + half, b * c + a * sn);
-    } else {
-      cod_st(dst + j, a);
-      cod_st(dst + j + half, b);
-    }
+  if (rot) {
+    const float* cs = rope_blk + static_cast<size_t>(r) * hd;
+    const float4 c = *reinterpret_cast<const float4*>(cs + j), sn = *reinterpret_cast<const float4*>(cs + half + j);
+    cod_st4(dst + j, make_float4(a.x * c.x - b.x * sn.x, a.y * c.y - b.y * sn.y, a.z * c.z - b.z * sn.z, a.w * c.w - b.w * sn.w));
+    cod_st4(dst + j + half, make_float4(b.x * c.x + a.x * sn.x, b.y * c.y + a.y * sn.y, b.z * c.z + a.z * sn.z, b.w * c.w + a.w * sn.w));
+  } else {
+    cod_st4(dst + j, a);
+    cod_st4(dst + j + half, b);
   }
 }
 
@@ -310,13 +320,22 @@ __global__ void k_resid_norm(const float* __restrict__ part, int splits, int R, 
   for (int t = 0; t < ROW_MAXV; ++t) {
     const int j = threadIdx.x + t * blockDim.x;
     v[t] = make_float4(0.f, 0.f, 0.f, 0.f);
-    if (j < nv) {
-      v[t] = *reinterpret_cast<const float4*>(x + static_cast<size_t>(r) * D + 4 * j);
-      if (part) {
-        for (int s = 0; s < splits; ++s)
-          v[t] = f4_add(v[t], *reinterpret_cast<const float4*>(part + (static_cast<size_t>(s) * R + r) * D + 4 * j));
-        *reinterpret_cast<float4*>(x + static_cast<size_t>(r) * D + 4 * j) = v[t];   // without partials x is read-only
+    if (j < nv) v[t] = *reinterpret_cast<const float4*>(x + static_cast<size_t>(r) * D + 4 * j);
+  }
+  if (part) {
+    for (int s = 0; s < splits; ++s) {      // slots inside: all of a slab's loads are in flight together
+#pragma unroll
+      for (int t = 0; t < ROW_MAXV; ++t) {
+        const int j = threadIdx.x + t * blockDim.x;
+        if (j < nv) v[t] = f4_add(v[t], *reinterpret_cast<const float4*>(part + (static_cast<size_t>(s) * R + r) * D + 4 * j));
       }
+    }
+  }
+#pragma unroll
+  for (int t = 0; t < ROW_MAXV; ++t) {
+    const int j = threadIdx.x + t * blockDim.x;
+    if (j < nv) {
+      if (part) *reinterpret_cast<float4*>(x + static_cast<size_t>(r) * D + 4 * j) = v[t];   // without partials x is read-only
       if (tap) *reinterpret_cast<float4*>(tap + static_cast<size_t>(r) * D + 4 * j) = v[t];
       ss += f4_ss(v[t]);
     }
@@ -441,10 +460,14 @@ int cod_launch_embed_norm(cod_ctx* c, const int32_t* bonus, int S, cudaStream_t 
 int cod_launch_qkv_finish(cod_ctx* c, const float* part, int splits, int R, cudaStream_t st) {
   ProfScope prof(c, COD_K_ROWOPS, st);
   const cod_config& f = c->cfg;
-  const dim3 grid(R, f.n_q_heads + 2 * f.n_kv_heads);
+  // heads per block: as many (up to 8) as still leave a couple of blocks per SM
+  const int nh = f.n_q_heads + 2 * f.n_kv_heads, tph = f.head_dim / 8;
+  int hpb = 8;
+  while (hpb > 1 && R * ((nh + hpb - 1) / hpb) < 2 * c->n_sm) hpb >>= 1;
+  const dim3 grid(R, (nh + hpb - 1) / hpb);
   DISPATCH_T(c,
-             (cod_launch_pdl(c, k_qkv_finish<__nv_bfloat16>, grid, 64, 0, st, part, splits, R, f.n_q_heads, f.n_kv_heads, f.head_dim, c->rope_blk, static_cast<__nv_bfloat16*>(c->q), static_cast<__nv_bfloat16*>(c->kb), static_cast<__nv_bfloat16*>(c->vb))),
-             (cod_launch_pdl(c, k_qkv_finish<float>, grid, 64, 0, st, part, splits, R, f.n_q_heads, f.n_kv_heads, f.head_dim, c->rope_blk, static_cast<float*>(c->q), static_cast<float*>(c->kb), static_cast<float*>(c->vb))));
+             (cod_launch_pdl(c, k_qkv_finish<__nv_bfloat16>, grid, tph * hpb, 0, st, part, splits, R, f.n_q_heads, f.n_kv_heads, f.head_dim, c->rope_blk, static_cast<__nv_bfloat16*>(c->q), static_cast<__nv_bfloat16*>(c->kb), static_cast<__nv_bfloat16*>(c->vb), hpb)),
+             (cod_launch_pdl(c, k_qkv_finish<float>, grid, tph * hpb, 0, st, part, splits, R, f.n_q_heads, f.n_kv_heads, f.head_dim, c->rope_blk, static_cast<float*>(c->q), static_cast<float*>(c->kb), static_cast<float*>(c->vb), hpb)));
   COD_CHECK_LAUNCH(c);
   return COD_OK;
 }
