@@ -4,7 +4,9 @@
 
 namespace {
 
-constexpr int ROW_MAXV = 8;   // float4 slots a thread keeps in registers: D <= 4 * ROW_MAXV * blockDim.x
+// Row kernels keep a row in registers as NV float4 slots per thread (D <= 4 * NV * blockDim.x):
+// one slot with up to 1024 threads for rows of up to 4096 elements, eight slots beyond.
+constexpr int ROW_WIDE_NV = 8;
 
 __device__ __forceinline__ void cod_st4(float* p, float4 v) { *reinterpret_cast<float4*>(p) = v; }
 __device__ __forceinline__ void cod_st4(__nv_bfloat16* p, float4 v) {
@@ -53,8 +55,8 @@ __global__ void k_gather_rows(const T* __restrict__ src, const int* __restrict__
 
 // ------------------------------------------------------------------ fc finish
 // z[row] = N_h( sum_splits part[i] + [row rejected] F(E_carry) )   (one block per kept row)
-template <typename T>
-__global__ void k_fc_finish(const float* __restrict__ part, int splits, int n_rows, const int* n_rows_dev,
+template <typename T, int NV>
+__global__ void __launch_bounds__(1024) k_fc_finish(const float* __restrict__ part, int splits, int n_rows, const int* n_rows_dev,
                             const int* __restrict__ a_rows, const int* __restrict__ carry_slot,
                             const float* __restrict__ fcE, const T* __restrict__ gain, int D, float eps,
                             int do_norm, T* __restrict__ z, int z_compact, float* __restrict__ tap) {
@@ -65,27 +67,28 @@ __global__ void k_fc_finish(const float* __restrict__ part, int splits, int n_ro
   const int row = a_rows ? a_rows[i] : i;
   const bool rej = carry_slot[row] >= 0;
   const int nv = D >> 2;
-  float4 v[ROW_MAXV];
+  float4 v[NV];
   float ss = 0.f;
 #pragma unroll
-  for (int t = 0; t < ROW_MAXV; ++t) {
+  for (int t = 0; t < NV; ++t) {
     const int j = threadIdx.x + t * blockDim.x;
     v[t] = make_float4(0.f, 0.f, 0.f, 0.f);
     if (j < nv && rej) v[t] = *reinterpret_cast<const float4*>(fcE + 4 * j);
   }
-  for (int s = 0; s < splits; ++s) {        // slots inside: all of a slab's loads are in flight together
+#pragma unroll 4
+  for (int s = 0; s < splits; ++s) {        // slots inside, four slabs unrolled: their loads are all in flight together
 #pragma unroll
-    for (int t = 0; t < ROW_MAXV; ++t) {
+    for (int t = 0; t < NV; ++t) {
       const int j = threadIdx.x + t * blockDim.x;
       if (j < nv) v[t] = f4_add(v[t], *reinterpret_cast<const float4*>(part + (static_cast<size_t>(s) * n_rows + i) * D + 4 * j));
     }
   }
 #pragma unroll
-  for (int t = 0; t < ROW_MAXV; ++t) ss += f4_ss(v[t]);
+  for (int t = 0; t < NV; ++t) ss += f4_ss(v[t]);
   ss = cod_block_sum(ss, red);
   const float scale = do_norm ? rsqrtf(ss / static_cast<float>(D) + eps) : 1.f;
 #pragma unroll
-  for (int t = 0; t < ROW_MAXV; ++t) {
+  for (int t = 0; t < NV; ++t) {
     const int j = threadIdx.x + t * blockDim.x;
     if (j < nv) {
       float4 o = v[t];
@@ -213,8 +216,8 @@ __global__ void k_update_lens(const int* __restrict__ accept_len, int S, int W, 
 
 // ------------------------------------------------------------------ block input
 // x = Emb[[bonus, MASK, ...]], a = N(x) * g_attn[0]; also clears the argmax keys.
-template <typename T>
-__global__ void k_embed_norm(const T* __restrict__ emb, const int* __restrict__ bonus, int W, int mask_id,
+template <typename T, int NV>
+__global__ void __launch_bounds__(1024) k_embed_norm(const T* __restrict__ emb, const int* __restrict__ bonus, int W, int mask_id,
                              int vocab, const T* __restrict__ gain, int D, float eps, float* __restrict__ x,
                              T* __restrict__ a, unsigned long long* __restrict__ amax) {
   cod_pdl_prologue();
@@ -223,10 +226,10 @@ __global__ void k_embed_norm(const T* __restrict__ emb, const int* __restrict__ 
   int tok = p == 0 ? bonus[s] : mask_id;
   if (tok < 0 || tok >= vocab) tok = 0;
   const int nv = D >> 2;
-  float4 v[ROW_MAXV];
+  float4 v[NV];
   float ss = 0.f;
 #pragma unroll
-  for (int t = 0; t < ROW_MAXV; ++t) {
+  for (int t = 0; t < NV; ++t) {
     const int j = threadIdx.x + t * blockDim.x;
     v[t] = make_float4(0.f, 0.f, 0.f, 0.f);
     if (j < nv) {
@@ -238,7 +241,7 @@ __global__ void k_embed_norm(const T* __restrict__ emb, const int* __restrict__ 
   ss = cod_block_sum(ss, red);
   const float scale = rsqrtf(ss / static_cast<float>(D) + eps);
 #pragma unroll
-  for (int t = 0; t < ROW_MAXV; ++t) {
+  for (int t = 0; t < NV; ++t) {
     const int j = threadIdx.x + t * blockDim.x;
     if (j < nv) {
       const float4 g = cod_ld4(gain + 4 * j);
@@ -306,33 +309,34 @@ __global__ void k_rope_qk(const T* __restrict__ qin, const T* __restrict__ kin, 
 
 // ------------------------------------------------------------------ residual + norm
 // x[r] += sum_splits part (if any); a[r] = N(x[r]) * gain
-template <typename T>
-__global__ void k_resid_norm(const float* __restrict__ part, int splits, int R, int D, float* x,
+template <typename T, int NV>
+__global__ void __launch_bounds__(1024) k_resid_norm(const float* __restrict__ part, int splits, int R, int D, float* x,
                              const T* __restrict__ gain, float eps, T* __restrict__ a, float* __restrict__ tap,
                              unsigned long long* __restrict__ amax) {
   cod_pdl_prologue();
   __shared__ float red[33];
   const int r = blockIdx.x;
   const int nv = D >> 2;
-  float4 v[ROW_MAXV];
+  float4 v[NV];
   float ss = 0.f;
 #pragma unroll
-  for (int t = 0; t < ROW_MAXV; ++t) {
+  for (int t = 0; t < NV; ++t) {
     const int j = threadIdx.x + t * blockDim.x;
     v[t] = make_float4(0.f, 0.f, 0.f, 0.f);
     if (j < nv) v[t] = *reinterpret_cast<const float4*>(x + static_cast<size_t>(r) * D + 4 * j);
   }
   if (part) {
-    for (int s = 0; s < splits; ++s) {      // slots inside: all of a slab's loads are in flight together
+#pragma unroll 4
+    for (int s = 0; s < splits; ++s) {      // slots inside, four slabs unrolled: their loads are all in flight together
 #pragma unroll
-      for (int t = 0; t < ROW_MAXV; ++t) {
+      for (int t = 0; t < NV; ++t) {
         const int j = threadIdx.x + t * blockDim.x;
         if (j < nv) v[t] = f4_add(v[t], *reinterpret_cast<const float4*>(part + (static_cast<size_t>(s) * R + r) * D + 4 * j));
       }
     }
   }
 #pragma unroll
-  for (int t = 0; t < ROW_MAXV; ++t) {
+  for (int t = 0; t < NV; ++t) {
     const int j = threadIdx.x + t * blockDim.x;
     if (j < nv) {
       if (part) *reinterpret_cast<float4*>(x + static_cast<size_t>(r) * D + 4 * j) = v[t];   // without partials x is read-only
@@ -343,7 +347,7 @@ __global__ void k_resid_norm(const float* __restrict__ part, int splits, int R, 
   ss = cod_block_sum(ss, red);
   const float scale = rsqrtf(ss / static_cast<float>(D) + eps);
 #pragma unroll
-  for (int t = 0; t < ROW_MAXV; ++t) {
+  for (int t = 0; t < NV; ++t) {
     const int j = threadIdx.x + t * blockDim.x;
     if (j < nv) {
       const float4 g = cod_ld4(gain + 4 * j);
@@ -368,7 +372,14 @@ __global__ void k_finalize(const unsigned long long* __restrict__ amax, int R, i
 
 }  // namespace
 
-static inline int row_threads(int D) { return D <= 4 * ROW_MAXV * 256 ? 256 : 1024; }
+// One float4 slot per thread where the row allows it: these kernels are latency-bound, so the more
+// independent loads a row has in flight the better.
+static inline bool row_narrow(int D) { return D <= 4096; }
+static inline int row_threads(int D) {
+  if (!row_narrow(D)) return 1024;
+  const int nt = ((D / 4 + 31) / 32) * 32;
+  return nt < 128 ? 128 : nt;
+}
 
 #define DISPATCH_T(c, CALL_BF16, CALL_F32) \
   do {                                     \
@@ -401,9 +412,15 @@ int cod_launch_fc_finish(cod_ctx* c, const float* part, int splits, int n_rows, 
   if (n_rows <= 0) return COD_OK;
   const int nt = row_threads(c->D);
   const int do_norm = (c->cfg.flags & COD_F_HIDDEN_NORM) ? 1 : 0;
-  DISPATCH_T(c,
-             (cod_launch_pdl(c, k_fc_finish<__nv_bfloat16>, n_rows, nt, 0, st, part, splits, n_rows, n_rows_dev, a_rows, carry_slot, c->fcE, static_cast<const __nv_bfloat16*>(c->w.g_hidden), c->D, c->cfg.rms_eps, do_norm, static_cast<__nv_bfloat16*>(c->z), a_rows ? 1 : 0, tap_z)),
-             (cod_launch_pdl(c, k_fc_finish<float>, n_rows, nt, 0, st, part, splits, n_rows, n_rows_dev, a_rows, carry_slot, c->fcE, static_cast<const float*>(c->w.g_hidden), c->D, c->cfg.rms_eps, do_norm, static_cast<float*>(c->z), a_rows ? 1 : 0, tap_z)));
+  if (row_narrow(c->D)) {
+    DISPATCH_T(c,
+               (cod_launch_pdl(c, k_fc_finish<__nv_bfloat16, 1>, n_rows, nt, 0, st, part, splits, n_rows, n_rows_dev, a_rows, carry_slot, c->fcE, static_cast<const __nv_bfloat16*>(c->w.g_hidden), c->D, c->cfg.rms_eps, do_norm, static_cast<__nv_bfloat16*>(c->z), a_rows ? 1 : 0, tap_z)),
+               (cod_launch_pdl(c, k_fc_finish<float, 1>, n_rows, nt, 0, st, part, splits, n_rows, n_rows_dev, a_rows, carry_slot, c->fcE, static_cast<const float*>(c->w.g_hidden), c->D, c->cfg.rms_eps, do_norm, static_cast<float*>(c->z), a_rows ? 1 : 0, tap_z)));
+  } else {
+    DISPATCH_T(c,
+               (cod_launch_pdl(c, k_fc_finish<__nv_bfloat16, ROW_WIDE_NV>, n_rows, nt, 0, st, part, splits, n_rows, n_rows_dev, a_rows, carry_slot, c->fcE, static_cast<const __nv_bfloat16*>(c->w.g_hidden), c->D, c->cfg.rms_eps, do_norm, static_cast<__nv_bfloat16*>(c->z), a_rows ? 1 : 0, tap_z)),
+               (cod_launch_pdl(c, k_fc_finish<float, ROW_WIDE_NV>, n_rows, nt, 0, st, part, splits, n_rows, n_rows_dev, a_rows, carry_slot, c->fcE, static_cast<const float*>(c->w.g_hidden), c->D, c->cfg.rms_eps, do_norm, static_cast<float*>(c->z), a_rows ? 1 : 0, tap_z)));
+  }
   COD_CHECK_LAUNCH(c);
   return COD_OK;
 }
@@ -450,9 +467,15 @@ int cod_launch_embed_norm(cod_ctx* c, const int32_t* bonus, int S, cudaStream_t 
   ProfScope prof(c, COD_K_ROWOPS, st);
   const cod_config& f = c->cfg;
   const int R = S * f.block;
-  DISPATCH_T(c,
-             (cod_launch_pdl(c, k_embed_norm<__nv_bfloat16>, R, row_threads(c->D), 0, st, static_cast<const __nv_bfloat16*>(c->w.emb), bonus, f.block, f.mask_token_id, f.vocab, static_cast<const __nv_bfloat16*>(c->w.g_attn), c->D, f.rms_eps, c->x, static_cast<__nv_bfloat16*>(c->a), c->amax)),
-             (cod_launch_pdl(c, k_embed_norm<float>, R, row_threads(c->D), 0, st, static_cast<const float*>(c->w.emb), bonus, f.block, f.mask_token_id, f.vocab, static_cast<const float*>(c->w.g_attn), c->D, f.rms_eps, c->x, static_cast<float*>(c->a), c->amax)));
+  if (row_narrow(c->D)) {
+    DISPATCH_T(c,
+               (cod_launch_pdl(c, k_embed_norm<__nv_bfloat16, 1>, R, row_threads(c->D), 0, st, static_cast<const __nv_bfloat16*>(c->w.emb), bonus, f.block, f.mask_token_id, f.vocab, static_cast<const __nv_bfloat16*>(c->w.g_attn), c->D, f.rms_eps, c->x, static_cast<__nv_bfloat16*>(c->a), c->amax)),
+               (cod_launch_pdl(c, k_embed_norm<float, 1>, R, row_threads(c->D), 0, st, static_cast<const float*>(c->w.emb), bonus, f.block, f.mask_token_id, f.vocab, static_cast<const float*>(c->w.g_attn), c->D, f.rms_eps, c->x, static_cast<float*>(c->a), c->amax)));
+  } else {
+    DISPATCH_T(c,
+               (cod_launch_pdl(c, k_embed_norm<__nv_bfloat16, ROW_WIDE_NV>, R, row_threads(c->D), 0, st, static_cast<const __nv_bfloat16*>(c->w.emb), bonus, f.block, f.mask_token_id, f.vocab, static_cast<const __nv_bfloat16*>(c->w.g_attn), c->D, f.rms_eps, c->x, static_cast<__nv_bfloat16*>(c->a), c->amax)),
+               (cod_launch_pdl(c, k_embed_norm<float, ROW_WIDE_NV>, R, row_threads(c->D), 0, st, static_cast<const float*>(c->w.emb), bonus, f.block, f.mask_token_id, f.vocab, static_cast<const float*>(c->w.g_attn), c->D, f.rms_eps, c->x, static_cast<float*>(c->a), c->amax)));
+  }
   COD_CHECK_LAUNCH(c);
   return COD_OK;
 }
@@ -488,9 +511,15 @@ int cod_launch_rope_qk(cod_ctx* c, const void* q, const void* k, const int32_t* 
 int cod_launch_resid_norm(cod_ctx* c, const float* part, int splits, int R, float* x, const void* gain,
                           float* tap_x, cudaStream_t st) {
   ProfScope prof(c, COD_K_ROWOPS, st);
-  DISPATCH_T(c,
-             (cod_launch_pdl(c, k_resid_norm<__nv_bfloat16>, R, row_threads(c->D), 0, st, part, splits, R, c->D, x, static_cast<const __nv_bfloat16*>(gain), c->cfg.rms_eps, static_cast<__nv_bfloat16*>(c->a), tap_x, c->amax)),
-             (cod_launch_pdl(c, k_resid_norm<float>, R, row_threads(c->D), 0, st, part, splits, R, c->D, x, static_cast<const float*>(gain), c->cfg.rms_eps, static_cast<float*>(c->a), tap_x, c->amax)));
+  if (row_narrow(c->D)) {
+    DISPATCH_T(c,
+               (cod_launch_pdl(c, k_resid_norm<__nv_bfloat16, 1>, R, row_threads(c->D), 0, st, part, splits, R, c->D, x, static_cast<const __nv_bfloat16*>(gain), c->cfg.rms_eps, static_cast<__nv_bfloat16*>(c->a), tap_x, c->amax)),
+               (cod_launch_pdl(c, k_resid_norm<float, 1>, R, row_threads(c->D), 0, st, part, splits, R, c->D, x, static_cast<const float*>(gain), c->cfg.rms_eps, static_cast<float*>(c->a), tap_x, c->amax)));
+  } else {
+    DISPATCH_T(c,
+               (cod_launch_pdl(c, k_resid_norm<__nv_bfloat16, ROW_WIDE_NV>, R, row_threads(c->D), 0, st, part, splits, R, c->D, x, static_cast<const __nv_bfloat16*>(gain), c->cfg.rms_eps, static_cast<__nv_bfloat16*>(c->a), tap_x, c->amax)),
+               (cod_launch_pdl(c, k_resid_norm<float, ROW_WIDE_NV>, R, row_threads(c->D), 0, st, part, splits, R, c->D, x, static_cast<const float*>(gain), c->cfg.rms_eps, static_cast<float*>(c->a), tap_x, c->amax)));
+  }
   COD_CHECK_LAUNCH(c);
   return COD_OK;
 }
