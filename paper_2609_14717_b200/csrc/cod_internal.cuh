@@ -13,12 +13,16 @@
 // ---------------------------------------------------------------------------- dependent launches
 // With few token rows a round is ~45 short kernels, and every kernel is launched with programmatic
 // stream serialisation: its CTAs may become resident while the previous kernel of the stream is
-// still running, so launch latency and CTA set-up overlap that kernel's tail. The first statement
-// of every kernel waits until the previous grid has completed and its memory is visible (before
-// any global access and before any tensor-memory allocation, so a waiting CTA holds nothing an
-// earlier grid still needs). Small grids then let the next grid start launching at once; for
-// grids of more than ~1000 CTAs the early trigger measured slower (the many waiting CTAs of the
-// next grid get in the way) and the next grid starts as this one drains.
+// still running, so launch latency and CTA set-up overlap that kernel's tail. cod_pdl_prologue()
+// waits until the previous grid has completed and its memory is visible, then (small grids only)
+// lets the next grid start launching. Before that call a kernel touches only what no kernel writes:
+// its parameters, its own shared and tensor memory and - in the tensor-core GEMMs - the weights,
+// whose first tiles are requested ahead of the wait. A GEMM always follows a row-wise kernel, never
+// another tensor-memory user, so the tensor memory it allocates ahead of its wait is never needed
+// by the grid it waits for.
+// For grids of more than ~1000 CTAs the explicit trigger measured slower (the many waiting CTAs of
+// the next grid get in the way) and the next grid starts as this one drains; triggering ahead of
+// the wait (several grids running ahead) measured slower as well.
 __device__ __forceinline__ void cod_pdl_prologue() {
   asm volatile("griddepcontrol.wait;" ::: "memory");
   if (gridDim.x * gridDim.y * gridDim.z <= 1024u) asm volatile("griddepcontrol.launch_dependents;" ::: "memory");

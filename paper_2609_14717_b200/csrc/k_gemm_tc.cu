@@ -55,7 +55,6 @@ struct TcParams {
 __global__ void __launch_bounds__(NTHREADS, 1)
 k_gemm_tc(const __grid_constant__ CUtensorMap map_w0, const __grid_constant__ CUtensorMap map_w1,
           const __grid_constant__ CUtensorMap map_w2, const __grid_constant__ CUtensorMap map_a, const TcParams p) {
-  cod_pdl_prologue();
   extern __shared__ uint8_t smem_raw[];
   // tiles need 1024-byte alignment for the 128-byte swizzle pattern
   const uint32_t raw = smem_u32(smem_raw);
@@ -73,9 +72,7 @@ k_gemm_tc(const __grid_constant__ CUtensorMap map_w0, const __grid_constant__ CU
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int n_tile = blockIdx.x, m_tile = blockIdx.y, split = blockIdx.z;
-  const int n_rows = p.n_rows_dev ? min(*p.n_rows_dev, p.n_rows) : p.n_rows;
   const int i0 = n_tile * p.NT;
-  if (i0 >= n_rows) return;                       // whole CTA: no token rows here
 
   // weight segment of this tile
   int sidx = 0;
@@ -88,8 +85,12 @@ k_gemm_tc(const __grid_constant__ CUtensorMap map_w0, const __grid_constant__ CU
   const CUtensorMap* map_w = sidx == 0 ? &map_w0 : (sidx == 1 ? &map_w1 : &map_w2);
 
   const int kb0 = split * p.kb_per_split, kb1 = min(p.kb_total, kb0 + p.kb_per_split);
-  const int n_kb = kb1 - kb0;
+  const int n_pre = min(p.stages, kb1 - kb0);     // stages whose weight tile is requested ahead of the dependency
 
+  // ---- before the dependency on the previous kernel resolves: set up, and start streaming the
+  // weights (nothing in the stream writes them) so the first stages are in flight or landed by the
+  // time the activations exist. Their bytes are counted on the stage's barrier before its
+  // expect_tx below, which the transaction count allows.
   if (threadIdx.x == 0) {
     for (int s = 0; s < p.stages; ++s) { mbar_init(smem_u32(full_bar + s), 1); mbar_init(smem_u32(empty_bar + s), 1); }
     mbar_init(smem_u32(acc_bar), 1);
@@ -102,10 +103,23 @@ k_gemm_tc(const __grid_constant__ CUtensorMap map_w0, const __grid_constant__ CU
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
+  if (warp == 4 && lane == 0)
+    for (int it = 0; it < n_pre; ++it)
+      tma_load_2d(base + it * stage_bytes, map_w, (kb0 + it) * BK, f0, smem_u32(full_bar + it));
+
+  cod_pdl_prologue();
+  const int n_rows = p.n_rows_dev ? min(*p.n_rows_dev, p.n_rows) : p.n_rows;
+  const int n_kb = i0 < n_rows ? kb1 - kb0 : 0;   // 0: no token rows here, only the requested weights to absorb
 
   if (warp == 4) {
     // ------------------------------------------------ TMA producer
     if (lane == 0) {
+      if (n_kb == 0) {
+        for (int it = 0; it < n_pre; ++it) {
+          mbar_expect_tx(smem_u32(full_bar + it), A_TILE_BYTES);
+          if (!mbar_wait(smem_u32(full_bar + it), 0, abort_flag, p.status)) break;
+        }
+      }
       for (int it = 0; it < n_kb; ++it) {
         const int s = it % p.stages, use = it / p.stages;
         if (use > 0 && !mbar_wait(smem_u32(empty_bar + s), (use - 1) & 1, abort_flag, p.status)) break;
@@ -113,7 +127,7 @@ k_gemm_tc(const __grid_constant__ CUtensorMap map_w0, const __grid_constant__ CU
         mbar_expect_tx(fb, stage_bytes);
         const uint32_t a_dst = base + s * stage_bytes;
         const int k = (kb0 + it) * BK;
-        tma_load_2d(a_dst, map_w, k, f0, fb);
+        if (it >= n_pre) tma_load_2d(a_dst, map_w, k, f0, fb);
         tma_load_2d(a_dst + A_TILE_BYTES, &map_a, k, i0, fb);
       }
     }
@@ -134,9 +148,9 @@ k_gemm_tc(const __grid_constant__ CUtensorMap map_w0, const __grid_constant__ CU
           umma_bf16(tmem_base, a_desc + (k * UK * 2 >> 4), b_desc + (k * UK * 2 >> 4), idesc, (it | k) ? 1u : 0u);
         umma_commit(smem_u32(empty_bar + s));   // frees the stage when these MMAs retire
       }
-      if (ok) umma_commit(smem_u32(acc_bar));
+      if (ok && n_kb > 0) umma_commit(smem_u32(acc_bar));
     }
-  } else {
+  } else if (n_kb > 0) {
     // ------------------------------------------------ epilogue warps 0..3
     const bool ok = mbar_wait(smem_u32(acc_bar), 0, abort_flag, p.status);
     tc_fence_after();
@@ -188,7 +202,7 @@ k_gemm_tc(const __grid_constant__ CUtensorMap map_w0, const __grid_constant__ CU
     for (int i = 0; i < 64; ++i) __nanosleep(1000);
     __syncthreads();
   }
-  else if (p.amax != nullptr) {
+  else if (p.amax != nullptr && n_kb > 0) {
     // the four epilogue warps merged their per-token keys in shared memory: one atomic per token
     for (int t = threadIdx.x; t < p.NT; t += NTHREADS) {
       if (i0 + t < n_rows) {

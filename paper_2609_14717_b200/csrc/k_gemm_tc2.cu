@@ -65,7 +65,6 @@ __device__ __forceinline__ bool bar_and_128(bool v) {
 __global__ void __launch_bounds__(NTHREADS, 1)
 k_gemm_tc2(const __grid_constant__ CUtensorMap map_w0, const __grid_constant__ CUtensorMap map_w1,
            const __grid_constant__ CUtensorMap map_w2, const __grid_constant__ CUtensorMap map_a, const Tc2Params p) {
-  cod_pdl_prologue();
   extern __shared__ uint8_t smem_raw[];
   const uint32_t raw = smem_u32(smem_raw);
   const uint32_t base = (raw + 1023u) & ~1023u;
@@ -85,10 +84,7 @@ k_gemm_tc2(const __grid_constant__ CUtensorMap map_w0, const __grid_constant__ C
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int rank = blockIdx.x;                    // position in the pair; 0 leads
   const int n_tile = blockIdx.y % p.n_tiles_n, pair = blockIdx.y / p.n_tiles_n, split = blockIdx.z;
-  const int n_rows = p.n_rows_dev ? min(*p.n_rows_dev, p.n_rows) : p.n_rows;
   const int i0 = n_tile * NTOK;
-  // NOTE: both CTAs of a pair take the same decision here (it depends on the pair's tile only)
-  const bool idle = i0 >= n_rows;
 
   int sidx = 0;
   while (sidx < p.n_seg - 1 && pair >= p.pair_end[sidx]) ++sidx;
@@ -99,8 +95,11 @@ k_gemm_tc2(const __grid_constant__ CUtensorMap map_w0, const __grid_constant__ C
   const int seg_N = p.seg_N[sidx];
   const CUtensorMap* map_w = sidx == 0 ? &map_w0 : (sidx == 1 ? &map_w1 : &map_w2);
   const int kb0 = split * p.kb_per_split, kb1 = min(p.kb_total, kb0 + p.kb_per_split);
-  const int n_kb = idle ? 0 : kb1 - kb0;
+  const int n_pre = min(STAGES, kb1 - kb0);       // stages whose weight tile is requested ahead of the dependency
 
+  // ---- before the dependency on the previous kernel resolves: set up, and start streaming the
+  // weights (nothing in the stream writes them). Their bytes are counted on the leader's stage
+  // barrier before its expect_tx below, which the transaction count allows.
   if (threadIdx.x == 0) {
     for (int s = 0; s < STAGES; ++s) { mbar_init(smem_u32(full_bar + s), 1); mbar_init(smem_u32(empty_bar + s), 1); }
     mbar_init(smem_u32(acc_bar), 1);
@@ -114,9 +113,23 @@ k_gemm_tc2(const __grid_constant__ CUtensorMap map_w0, const __grid_constant__ C
   cluster_sync_all();                 // the partner's barriers exist before anything signals them
   tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
+  if (warp == 4 && lane == 0)
+    for (int it = 0; it < n_pre; ++it)
+      tma_load_2d_pair(base + it * STAGE_BYTES, map_w, (kb0 + it) * BK, f0, smem_u32(full_bar + it) & PEER_MASK);
+
+  cod_pdl_prologue();
+  const int n_rows = p.n_rows_dev ? min(*p.n_rows_dev, p.n_rows) : p.n_rows;
+  // NOTE: both CTAs of a pair take the same decision here (it depends on the pair's tile only)
+  const int n_kb = i0 < n_rows ? kb1 - kb0 : 0;   // 0: no token rows here, only the requested weights to absorb
 
   if (warp == 4) {
     if (lane == 0) {
+      if (n_kb == 0 && rank == 0) {
+        for (int it = 0; it < n_pre; ++it) {
+          mbar_expect_tx(smem_u32(full_bar + it), 2 * A_TILE_BYTES);
+          if (!mbar_wait(smem_u32(full_bar + it), 0, abort_flag, p.status)) break;
+        }
+      }
       for (int it = 0; it < n_kb; ++it) {
         const int s = it % STAGES, use = it / STAGES;
         if (use > 0 && !mbar_wait(smem_u32(empty_bar + s), (use - 1) & 1, abort_flag, p.status)) break;
@@ -124,7 +137,7 @@ k_gemm_tc2(const __grid_constant__ CUtensorMap map_w0, const __grid_constant__ C
         if (rank == 0) mbar_expect_tx(fb, 2 * STAGE_BYTES);     // both CTAs' bytes land on the leader's barrier
         const uint32_t a_dst = base + s * STAGE_BYTES;
         const int k = (kb0 + it) * BK;
-        tma_load_2d_pair(a_dst, map_w, k, f0, fb & PEER_MASK);
+        if (it >= n_pre) tma_load_2d_pair(a_dst, map_w, k, f0, fb & PEER_MASK);
         for (int a = 0; a < p.n_acc; ++a)      // accumulator a covers tokens [i0 + a*256, +256): this CTA stages its half
           tma_load_2d_pair(a_dst + A_TILE_BYTES + a * B_TILE_BYTES, &map_a, k, i0 + a * NT + rank * (NT / 2), fb & PEER_MASK);
       }
