@@ -13,7 +13,8 @@
 //   * leader only: one thread issues the MMAs (M = 256 spans both CTAs' tensor memory) and commits
 //     with a cluster-wide arrive to the "empty" barrier of both CTAs (and, at the end, to both
 //     "accumulator ready" barriers);
-//   * both CTAs: four epilogue warps read their own 128 accumulator rows.
+//   * both CTAs: all eight warps read the CTA's own 128 accumulator rows back (two warps per 32 lanes,
+//     each taking half of the token columns).
 // No load is delivered to more than one CTA. Waits are bounded as in k_gemm_tc; the only
 // unbounded synchronisation is the hardware cluster barrier, which every thread reaches
 // unconditionally.
@@ -27,7 +28,7 @@ constexpr int BM = 128;       // weight rows per CTA (256 per pair)
 constexpr int BK = 64;
 constexpr int UK = 16;
 constexpr int NT = 256;       // token rows per pair = MMA N; each CTA stages NT / 2 of them
-constexpr int NTHREADS = 192;
+constexpr int NTHREADS = 256;   // 8 warps: all of them read the accumulator back; warps 4 and 5 first produce / issue
 constexpr uint32_t A_TILE_BYTES = BM * BK * 2;          // 16 KB
 constexpr uint32_t B_TILE_BYTES = (NT / 2) * BK * 2;    // 16 KB
 constexpr int MAX_STAGES = 6;   // one accumulator: 6 stages of 32 KB; two: 4 stages of 48 KB
@@ -50,17 +51,6 @@ struct Tc2Params {
 };
 
 
-
-// AND of a predicate over the 128 threads of warps 0-3 (named barrier 1)
-__device__ __forceinline__ bool bar_and_128(bool v) {
-  uint32_t r;
-  asm volatile(
-      "{\n\t.reg .pred p, q;\n\tsetp.ne.b32 q, %1, 0;\n\t"
-      "bar.red.and.pred p, 1, 128, q;\n\t"
-      "selp.u32 %0, 1, 0, p;\n\t}"
-      : "=r"(r) : "r"(static_cast<uint32_t>(v)) : "memory");
-  return r != 0;
-}
 
 __global__ void __launch_bounds__(NTHREADS, 1)
 k_gemm_tc2(const __grid_constant__ CUtensorMap map_w0, const __grid_constant__ CUtensorMap map_w1,
@@ -164,31 +154,39 @@ k_gemm_tc2(const __grid_constant__ CUtensorMap map_w0, const __grid_constant__ C
       }
       if (ok && n_kb > 0) umma_commit_pair(smem_u32(acc_bar), 3);
     }
-  } else if (n_kb > 0) {
-    // one verdict for the four epilogue warps (they meet at a named barrier below)
-    const bool ok = bar_and_128(mbar_wait(smem_u32(acc_bar), 0, abort_flag, p.status));
+  }
+  __syncwarp();
+
+  // ---------------------------------------------------- epilogue, all 8 warps
+  // Warp w reads tensor-memory lanes 32 * (w % 4) .. +31 (the only lanes it may touch); warps 0-3
+  // take the first half of the token columns, warps 4-7 the second.
+  if (n_kb > 0) {
+    // one verdict for everyone (the warps meet at named barriers below)
+    const bool ok = __syncthreads_and(mbar_wait(smem_u32(acc_bar), 0, abort_flag, p.status)) != 0;
     tc_fence_after();
-    const int f = f0 + warp * 32 + lane;
+    const int qw = warp & 3, grp = warp >> 2;
+    const int c_begin = grp * (NTOK / 2), c_end = c_begin + NTOK / 2;
+    const int f = f0 + qw * 32 + lane;
     const bool f_ok = f < seg_N;
-    const uint32_t t_lane = tmem_base + (static_cast<uint32_t>(warp * 32) << 16);
+    const uint32_t t_lane = tmem_base + (static_cast<uint32_t>(qw * 32) << 16);
     if (ok && p.amax == nullptr && p.staged) {
       // The accumulator has features on lanes and tokens on columns; C wants a token's features
-      // contiguous. Transpose 32 tokens at a time through the (now idle) pipeline buffers and
-      // store whole 512-byte feature runs: two 16 KB buffers, one barrier of the four epilogue
-      // warps per chunk.
+      // contiguous. Each group of four warps transposes 32 tokens at a time through the (now idle)
+      // pipeline buffers and stores whole 512-byte feature runs: two 16 KB buffers per group, one
+      // named barrier of the group per chunk.
       float* C = p.C + static_cast<size_t>(split) * p.n_rows * p.ldc + col0;
-      float* stage = reinterpret_cast<float*>(sm);
+      float* stage = reinterpret_cast<float*>(sm) + grp * (2 * 32 * BM);
       const int f_left = seg_N - f0;                       // features of this CTA that exist
-      for (int c = 0, q = 0; c < NTOK && i0 + c < n_rows; c += 32, q ^= 1) {
+      for (int c = c_begin, q = 0; c < c_end && i0 + c < n_rows; c += 32, q ^= 1) {
         uint32_t v[32];
         tmem_ld32(t_lane + c, v);
         float* buf = stage + q * (32 * BM);
 #pragma unroll
-        for (int j = 0; j < 32; ++j) buf[j * BM + warp * 32 + lane] = __uint_as_float(v[j]);
-        asm volatile("bar.sync 1, 128;" ::: "memory");
+        for (int j = 0; j < 32; ++j) buf[j * BM + qw * 32 + lane] = __uint_as_float(v[j]);
+        asm volatile("bar.sync %0, 128;" ::"r"(1 + grp) : "memory");
 #pragma unroll
         for (int t = 0; t < 8; ++t) {
-          const int tok = warp * 8 + t, i = i0 + c + tok;
+          const int tok = qw * 8 + t, i = i0 + c + tok;
           if (i < n_rows && lane * 4 < f_left)
             *reinterpret_cast<float4*>(C + static_cast<size_t>(i) * p.ldc + lane * 4) =
                 *reinterpret_cast<const float4*>(buf + tok * BM + lane * 4);
@@ -196,19 +194,19 @@ k_gemm_tc2(const __grid_constant__ CUtensorMap map_w0, const __grid_constant__ C
       }
     } else if (ok && p.amax == nullptr) {
       float* C = p.C + static_cast<size_t>(split) * p.n_rows * p.ldc;
-      for (int c = 0; c < NTOK; c += 16) {
+      for (int c = c_begin; c < c_end; c += 16) {
         if (i0 + c >= n_rows) break;
         uint32_t v[16];
         tmem_ld16(t_lane + c, v);
 #pragma unroll
         for (int j = 0; j < 16; ++j) {
           const int i = i0 + c + j;
-          if (f_ok && i < n_rows) C[static_cast<size_t>(i) * p.ldc + col0 + warp * 32 + lane] = __uint_as_float(v[j]);
+          if (f_ok && i < n_rows) C[static_cast<size_t>(i) * p.ldc + col0 + qw * 32 + lane] = __uint_as_float(v[j]);
         }
       }
     } else if (ok) {
-      const unsigned long long low = static_cast<unsigned long long>(0xFFFFFFFFu - static_cast<unsigned>(col0 + warp * 32 + lane));
-      for (int c = 0; c < NTOK; c += 32) {
+      const unsigned long long low = static_cast<unsigned long long>(0xFFFFFFFFu - static_cast<unsigned>(col0 + qw * 32 + lane));
+      for (int c = c_begin; c < c_end; c += 32) {
         if (i0 + c >= n_rows) break;
         uint32_t v[32];
         tmem_ld32(t_lane + c, v);
@@ -216,7 +214,7 @@ k_gemm_tc2(const __grid_constant__ CUtensorMap map_w0, const __grid_constant__ C
 #pragma unroll
         for (int j = 0; j < 32; ++j)
           k[j] = f_ok ? ((static_cast<unsigned long long>(order_key(__uint_as_float(v[j]))) << 32) | low) : 0ull;
-        red[warp * NTOK + c + lane] = warp_colmax32(k, lane);
+        red[qw * NTOK + c + lane] = warp_colmax32(k, lane);
       }
     }
   }
