@@ -86,7 +86,8 @@ int pick_splits(const cod_ctx* c, int n_out, int K, int rows) {
   }
   const int tiles = (n_out + 127) / 128;
   const int kb = (K + 63) / 64;
-  int splits = c->n_sm / tiles;
+  // up to 32 token rows two CTAs fit on an SM (the launcher keeps their rings small): aim for two waves' worth
+  int splits = (rows <= 32 ? 2 * c->n_sm : c->n_sm) / tiles;
   if (splits > COD_MAX_SPLITS) splits = COD_MAX_SPLITS;
   if (splits > kb / 4) splits = kb / 4;
   if (splits < 1) splits = 1;
