@@ -154,19 +154,25 @@ int cod_create(const cod_config* cfg, cod_ctx** out) {
 
   {
     // tensor-core attention: keys of the paged region per CTA, and partial slots per (sequence, head)
-    const int M = f.block * (f.n_q_heads / f.n_kv_heads);
     const int64_t cap = static_cast<int64_t>(f.max_pages_per_seq) * f.page_size;
     int64_t sl;
     if (f.attn_split_len > 0) sl = (f.attn_split_len + 127) / 128 * 128 > 4096 ? 4096 : (f.attn_split_len + 127) / 128 * 128;
     else {
+      // large batches: enough parts to keep every SM fed for several waves
       sl = (cap * f.max_batch * f.n_kv_heads / (8 * static_cast<int64_t>(c->n_sm)) + 127) / 128 * 128;
       if (sl < 256) sl = 256;   // fewer, longer parts beat more CTAs at batch 1 (measured at 2K context)
       if (sl > 2048) sl = 2048;
+      // small batches: all parts in ONE wave of two CTAs per SM if at least four parts per
+      // (sequence, head) fit (a second, mostly empty wave cost 10 % at 4 x 32K keys)
+      const int64_t per_seq = 2 * static_cast<int64_t>(c->n_sm) / (static_cast<int64_t>(f.max_batch) * f.n_kv_heads);
+      if (per_seq >= 4) {
+        int64_t one_wave = ((cap + per_seq - 1) / per_seq + 127) / 128 * 128;
+        if (one_wave < 256) one_wave = 256;
+        if (one_wave <= 4096) sl = one_wave;
+      }
     }
     c->tc_split_len = static_cast<int>(sl);
-    const int keys_it = M <= 64 ? 128 : 64, ring = M <= 64 ? 1 : 2;
-    const bool tail_fits = (15 + 2 * f.block + keys_it - 1) / keys_it <= ring;
-    c->tc_max_parts = tail_fits ? static_cast<int>((cap + sl - 1) / sl + 1) : 0;
+    c->tc_max_parts = static_cast<int>((cap + sl - 1) / sl + 1);
   }
   c->ws = nullptr;
   c->ws_bytes = carve(c);

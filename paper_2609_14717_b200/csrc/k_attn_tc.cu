@@ -52,7 +52,7 @@ struct Geo {
   static constexpr int MROWS = DUAL ? 64 : 128;          // MMA M
   static constexpr int KEYS_IT = KT * TILES;
   static constexpr int NK = DUAL ? 1 : 2;                // K ring slots
-  static constexpr int NV = DUAL ? 1 : 2;                // V ring slots
+  static constexpr int NV = 1;                           // V ring slots (two CTAs fit on an SM either way)
   static constexpr uint32_t SLOT = TILE_BYTES * TILES;
   static constexpr uint32_t Q_BYTES = MROWS * HD * 2;
   static constexpr uint32_t Q_HALF = MROWS * 128;
@@ -256,38 +256,50 @@ k_attn_tc(const __grid_constant__ CUtensorMap map_pool, const __grid_constant__ 
 
     for (int it = 0; it < n_it && ok; ++it) {
       if (is_tail) {
-        // gather this iteration's rows (partial page, carried rows, block rows) with plain loads
-        const int kslot = it % G::NK, vslot = it % G::NV;
+        // gather this iteration's rows (partial page, carried rows, block rows) with plain loads:
+        // first the K rows (the MMA warp asks for them first), then the V rows. A ring slot that was
+        // used before is taken only once the MMAs that read it have retired.
         constexpr int GB = 8;                               // independent 16-byte loads in flight per thread
-        for (int idx0 = T; idx0 < G::KEYS_IT * 32; idx0 += 128 * GB) {
-          uint4 val[GB];
-          uint32_t dst[GB];
-#pragma unroll
-          for (int u = 0; u < GB; ++u) {
-            const int idx = idx0 + u * 128;
-            const int ch = idx & 15, kv = (idx >> 4) & 1, j = idx >> 5;       // chunk, K|V, key within iteration
-            const int g = it * G::KEYS_IT + j;
-            const __nv_bfloat16* src = nullptr;
-            if (g < Lr) {
-              int pg = p.block_table[s * p.max_pages + F / PAGE];
-              if (pg < 0 || pg >= p.n_pages) { flags |= COD_DEV_BAD_PAGE; }
-              else src = p.pool + ((((static_cast<size_t>(p.layer) * p.n_pages + pg) * p.n_kv + h) * 2 + kv) * PAGE + g) * HD;
-            } else if (g < Lr + c) {
-              src = p.carry + ((((static_cast<size_t>(p.layer) * p.max_batch + s) * p.n_kv + h) * 2 + kv) * p.W + (g - Lr)) * HD;
-            } else if (g < n_tail) {
-              src = (kv ? p.vb : p.kb) + static_cast<size_t>(s * p.W + (g - Lr - c)) * (p.n_kv * HD) + h * HD;
-            }
-            val[u] = src ? *reinterpret_cast<const uint4*>(src + ch * 8) : make_uint4(0u, 0u, 0u, 0u);
-            const int jj = j & (KT - 1), tl = j / KT;
-            dst[u] = (kv ? G::OFF_V + vslot * G::SLOT : G::OFF_K + kslot * G::SLOT) + tl * TILE_BYTES +
-                     (ch >> 3) * HALF_BYTES + jj * 128 + (((ch & 7) ^ (jj & 7)) << 4);
+#pragma unroll 1
+        for (int kv = 0; kv < 2; ++kv) {
+          const int ring = kv ? G::NV : G::NK;
+          const int slot = it % ring, use = it / ring;
+          uint64_t* full = kv ? v_full : k_full;
+          uint64_t* empty = kv ? v_empty : k_empty;
+          if (use > 0) {
+            ok = __all_sync(0xffffffffu, mbar_wait(smem_u32(empty + slot), (use - 1) & 1, abort_flag, p.status));
+            if (!ok) break;
           }
+          for (int idx0 = T; idx0 < G::KEYS_IT * 16; idx0 += 128 * GB) {
+            uint4 val[GB];
+            uint32_t dst[GB];
 #pragma unroll
-          for (int u = 0; u < GB; ++u) *reinterpret_cast<uint4*>(sm + dst[u]) = val[u];
+            for (int u = 0; u < GB; ++u) {
+              const int idx = idx0 + u * 128;
+              const int ch = idx & 15, j = idx >> 4;                          // chunk, key within iteration
+              const int g = it * G::KEYS_IT + j;
+              const __nv_bfloat16* src = nullptr;
+              if (g < Lr) {
+                int pg = p.block_table[s * p.max_pages + F / PAGE];
+                if (pg < 0 || pg >= p.n_pages) { flags |= COD_DEV_BAD_PAGE; }
+                else src = p.pool + ((((static_cast<size_t>(p.layer) * p.n_pages + pg) * p.n_kv + h) * 2 + kv) * PAGE + g) * HD;
+              } else if (g < Lr + c) {
+                src = p.carry + ((((static_cast<size_t>(p.layer) * p.max_batch + s) * p.n_kv + h) * 2 + kv) * p.W + (g - Lr)) * HD;
+              } else if (g < n_tail) {
+                src = (kv ? p.vb : p.kb) + static_cast<size_t>(s * p.W + (g - Lr - c)) * (p.n_kv * HD) + h * HD;
+              }
+              val[u] = src ? *reinterpret_cast<const uint4*>(src + ch * 8) : make_uint4(0u, 0u, 0u, 0u);
+              const int jj = j & (KT - 1), tl = j / KT;
+              dst[u] = (kv ? G::OFF_V : G::OFF_K) + slot * G::SLOT + tl * TILE_BYTES +
+                       (ch >> 3) * HALF_BYTES + jj * 128 + (((ch & 7) ^ (jj & 7)) << 4);
+            }
+#pragma unroll
+            for (int u = 0; u < GB; ++u) *reinterpret_cast<uint4*>(sm + dst[u]) = val[u];
+          }
+          fence_async_smem();
+          mbar_arrive(smem_u32(full + slot));
         }
-        fence_async_smem();
-        mbar_arrive(smem_u32(k_full + kslot));
-        mbar_arrive(smem_u32(v_full + vslot));
+        if (!ok) break;
       }
 
       ok = __all_sync(0xffffffffu, mbar_wait(smem_u32(s_full + (it & 1)), (it >> 1) & 1, abort_flag, p.status));
