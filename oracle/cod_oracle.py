@@ -16,7 +16,12 @@ normalisation and positional encoding", Section 2.1), the readings taken are:
   * F, K_l, V_l, W_q, W_o are bias-free linear maps stored [out, in];
   * an RMS normalisation with gain follows F (switchable), precedes each
     attention sub-layer, and precedes the LM head; the residual stream is
-    x <- x + W_o o; there is no MLP;
+    x <- x + W_o o; by default there is no MLP;
+  * the complete layer (d_ff > 0, qk_norm; the shape of the Qwen3 blocks the
+    paper's DFlash drafters are built from, Section 4 "Targets and drafters")
+    adds a per-head RMS norm with gain on queries and on ALL keys (cached and
+    block keys alike) before the rotation, and after the attention residual
+    x <- x + W_down( silu(W_gate b) * (W_up b) ) with b = N(x) * g_mlp;
   * RoPE is the rotate-half form over the full head dimension, at the absolute
     token position, applied once to keys when they are projected (Appendix A,
     "Cache semantics") and to the block's queries and keys at draft time;
@@ -60,6 +65,8 @@ class OracleConfig:
     rope_theta: float
     rms_eps: float
     hidden_norm: bool
+    d_ff: int = 0            # > 0: every drafter layer has a gated MLP of this width
+    qk_norm: bool = False    # per-head RMS norm of queries and keys before the rotation
 
     @property
     def d_in(self) -> int:
@@ -167,6 +174,17 @@ def rmsnorm(x: np.ndarray, g: np.ndarray, eps: float) -> np.ndarray:
     return g * x / np.sqrt(np.mean(x * x, axis=-1, keepdims=True) + eps)
 
 
+def silu(x: np.ndarray) -> np.ndarray:
+    """x * sigmoid(x)."""
+    x = np.asarray(x, dtype=np.float64)
+    return x / (1.0 + np.exp(-x))
+
+
+def gated_mlp(b: np.ndarray, w_gate: np.ndarray, w_up: np.ndarray, w_down: np.ndarray) -> np.ndarray:
+    """W_down( silu(W_gate b) * (W_up b) ) for rows b [R, D]; matrices stored [out, in]."""
+    return (silu(b @ w_gate.T) * (b @ w_up.T)) @ w_down.T
+
+
 # =========================================================================== part 2
 def fuse_features(H: np.ndarray, rejected: np.ndarray, w: Dict[str, np.ndarray],
                   cfg: OracleConfig) -> np.ndarray:
@@ -200,6 +218,8 @@ def project_kv(H: np.ndarray, split: Dict[str, np.ndarray], w: Dict[str, np.ndar
     for l in range(cfg.n_layers):
         K = (Z @ w["wk"][l].T).reshape(R, cfg.n_kv, cfg.hd)
         V = (Z @ w["wv"][l].T).reshape(R, cfg.n_kv, cfg.hd)
+        if cfg.qk_norm:
+            K = rmsnorm(K, w["g_knorm"][l], cfg.rms_eps)
         K = rope(K, pos[:, None], cfg.rope_theta)
         J[l, keep, 0] = K[keep]
         J[l, keep, 1] = V[keep]
@@ -309,9 +329,15 @@ def draft_block(st: OracleState, bonus: np.ndarray, w: Dict[str, np.ndarray],
         q = (a @ w["wq"][l].T).reshape(S, W, cfg.n_q, cfg.hd)
         kb = (a @ w["wk"][l].T).reshape(S, W, cfg.n_kv, cfg.hd)
         vb = (a @ w["wv"][l].T).reshape(S, W, cfg.n_kv, cfg.hd)
+        if cfg.qk_norm:
+            q = rmsnorm(q, w["g_qnorm"][l], cfg.rms_eps)
+            kb = rmsnorm(kb, w["g_knorm"][l], cfg.rms_eps)
         o, mass[l] = block_attn(l, q, kb, vb, st, use_carry)
         attn_out[l] = o.reshape(S * W, cfg.n_q * cfg.hd)
         x = x + attn_out[l] @ w["wo"][l].T
+        if cfg.d_ff > 0:
+            b = rmsnorm(x, w["g_mlp"][l], cfg.rms_eps)
+            x = x + gated_mlp(b, w["w_gate"][l], w["w_up"][l], w["w_down"][l])
     tok, gap, logits = lm_head_argmax(x, w, cfg)
     res = {"tok": tok.reshape(S, W), "gap": gap.reshape(S, W), "x_final": x,
            "attn_out": attn_out, "carry_mass": mass}

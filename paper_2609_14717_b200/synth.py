@@ -50,6 +50,8 @@ class DrafterShape:
     rms_eps: float = 1.0e-6
     hidden_norm: bool = True
     h_rms: Optional[Tuple[float, float]] = None  # per-layer RMS range of H
+    d_ff: int = 0         # width of the gated MLP of a drafter layer; 0 = attention sub-layer only
+    qk_norm: bool = False # per-head RMS norm (with gain) of queries and keys before the rotation
 
     @property
     def d_in(self) -> int:
@@ -105,6 +107,10 @@ def workload(name: str) -> Workload:
     if name == "cfg5":
         return Workload("cfg5", _FULL, S=1, ctx=(4096, 4096), accept=("fixed_m", 8),
                         n_forced=0, n_rounds=16)
+    if name in ("cfg2f", "cfg3f"):
+        # the same batches with a complete drafter layer: gated MLP of width 9728 and q/k norms
+        base = workload(name[:-1])
+        return replace(base, name=name, shape=replace(base.shape, d_ff=9728, qk_norm=True))
     raise KeyError(name)
 
 
@@ -144,12 +150,13 @@ def _normal(rng: np.random.Generator, shape, scale: float = 1.0) -> np.ndarray:
 
 
 # --------------------------------------------------------------------------- weights
-_WEIGHT_ORDER = ("fc", "e_carry", "g_hidden", "wk", "wv", "wq", "wo", "g_attn", "g_final", "emb")
+_WEIGHT_ORDER = ("fc", "e_carry", "g_hidden", "wk", "wv", "wq", "wo", "g_attn", "g_final", "emb",
+                 "w_gate", "w_up", "w_down", "g_mlp", "g_qnorm", "g_knorm")   # new names go last: stream index = position
 
 
 def weight_shapes(sh: DrafterShape) -> Dict[str, Tuple[int, ...]]:
     D, Ld = sh.d_model, sh.n_layers
-    return {
+    out = {
         "fc": (D, sh.d_in),
         "e_carry": (sh.d_in,),
         "g_hidden": (D,),
@@ -161,6 +168,12 @@ def weight_shapes(sh: DrafterShape) -> Dict[str, Tuple[int, ...]]:
         "g_final": (D,),
         "emb": (sh.vocab, D),
     }
+    if sh.d_ff > 0:
+        out.update({"w_gate": (Ld, sh.d_ff, D), "w_up": (Ld, sh.d_ff, D), "w_down": (Ld, D, sh.d_ff),
+                    "g_mlp": (Ld, D)})
+    if sh.qk_norm:
+        out.update({"g_qnorm": (Ld, sh.hd), "g_knorm": (Ld, sh.hd)})
+    return out
 
 
 def make_weights(sh: DrafterShape, seed: int) -> Dict[str, np.ndarray]:
@@ -168,6 +181,8 @@ def make_weights(sh: DrafterShape, seed: int) -> Dict[str, np.ndarray]:
     out = {}
     shapes = weight_shapes(sh)
     for i, name in enumerate(_WEIGHT_ORDER):
+        if name not in shapes:
+            continue
         rng = np.random.default_rng([seed, _STREAM_WEIGHTS, i])
         if name.startswith("g_"):
             w = np.float32(1.0) + _normal(rng, shapes[name], 0.1)

@@ -592,3 +592,129 @@ def test_round_is_deterministic_and_next_draft_shape():
     nd = outs[0]["next_draft"]
     assert nd.shape == (wl.S, wl.shape.W) and np.array_equal(nd[:, 0], outs[0]["split"]["bonus"])
     assert np.array_equal(nd[:, 1:], outs[0]["tok"][:, 1:])
+
+
+# ----------------------------------------------------------------------------- the complete layer
+def _full_layer_workload(**kw):
+    args = dict(S=2, ctx=(20, 60), d_ff=96, qk_norm=True, n_layers=2, n_rounds=4)
+    args.update(kw)
+    return synth.scaled(synth.workload("cfg1"), **args)
+
+
+def test_silu_closed_form():
+    x = np.array([0.0, 1.0, -1.0, 30.0, -30.0, math.log(3.0)])
+    got = orc.silu(x)
+    exp = [0.0, 1.0 / (1.0 + math.exp(-1.0)), -1.0 / (1.0 + math.e), 30.0, 0.0, math.log(3.0) * 0.75]
+    assert np.allclose(got, exp, atol=1e-11)
+    # silu(x) - silu(-x) = x  (sigmoid(x) + sigmoid(-x) = 1)
+    y = np.linspace(-6, 6, 41)
+    assert np.allclose(orc.silu(y) - orc.silu(-y), y, atol=1e-12)
+
+
+def test_gated_mlp_against_torch_and_loops():
+    rng = np.random.default_rng(3)
+    b = rng.standard_normal((5, 12)); wg = rng.standard_normal((7, 12)); wu = rng.standard_normal((7, 12))
+    wd = rng.standard_normal((12, 7))
+    got = orc.gated_mlp(b, wg, wu, wd)
+    F = torch.nn.functional
+    tb, tg, tu, td = (torch.from_numpy(a) for a in (b, wg, wu, wd))
+    ref = F.linear(F.silu(F.linear(tb, tg)) * F.linear(tb, tu), td).numpy()
+    assert np.allclose(got, ref, atol=1e-12)
+    # and element by element: a transposed operand or a swapped gate/up would show here
+    for r in range(5):
+        h = [sum(b[r, k] * wg[j, k] for k in range(12)) for j in range(7)]
+        u = [sum(b[r, k] * wu[j, k] for k in range(12)) for j in range(7)]
+        act = [hj / (1.0 + math.exp(-hj)) * uj for hj, uj in zip(h, u)]
+        for i in range(12):
+            assert abs(got[r, i] - sum(act[j] * wd[i, j] for j in range(7))) < 1e-10
+
+
+@pytest.mark.parametrize("zeroed", ["w_down", "w_gate", "w_up"])
+def test_mlp_with_a_zero_factor_is_the_attention_only_layer(zeroed):
+    """silu(0) = 0, so a zero gate, a zero up-projection or a zero down-projection removes the MLP."""
+    wl = _full_layer_workload(qk_norm=False)
+    wl0 = synth.scaled(wl, d_ff=0)
+    w = orc.prepare_weights(synth.make_weights(wl.shape, 2))
+    w[zeroed] = np.zeros_like(w[zeroed])
+    w0 = {k: v for k, v in w.items() if k not in ("w_gate", "w_up", "w_down", "g_mlp")}
+    _, st, _ = oracle_state(wl, 2)
+    _, st0, _ = oracle_state(wl0, 2)
+    for r in range(2):
+        rd = synth.make_round(wl, 2, r)
+        a = orc.draft_round(rd["draft"], rd["target"], rd["H"], st, w, 1, orc.MODE_CARRY)
+        b = orc.draft_round(rd["draft"], rd["target"], rd["H"], st0, w0, 1, orc.MODE_CARRY)
+        assert np.array_equal(a["x_final"], b["x_final"]) and np.array_equal(a["tok"], b["tok"])
+
+
+def test_mlp_residual_written_out_for_one_layer():
+    """One layer with W_o = 0: x_final = x0 + MLP(N(x0) g_mlp), x0 the embedded block."""
+    wl = _full_layer_workload(n_layers=1, qk_norm=False, S=1)
+    cfg, st, _ = oracle_state(wl, 4)
+    w = orc.prepare_weights(synth.make_weights(wl.shape, 4))
+    w["wo"] = np.zeros_like(w["wo"])
+    for k in ("w_gate", "w_up", "w_down"):
+        w[k] = w[k] * 25.0                                   # make the MLP term large enough to matter
+    rd = synth.make_round(wl, 4, 0)
+    res = orc.draft_round(rd["draft"], rd["target"], rd["H"], st, w, 1, orc.MODE_CARRY)
+    toks = [int(res["split"]["bonus"][0])] + [cfg.mask_token_id] * (cfg.W - 1)
+    for i, t in enumerate(toks):
+        x0 = w["emb"][t]
+        b = w["g_mlp"][0] * x0 / math.sqrt(float(np.mean(x0 * x0)) + cfg.rms_eps)
+        g = w["w_gate"][0] @ b
+        u = w["w_up"][0] @ b
+        want = x0 + w["w_down"][0] @ (g / (1.0 + np.exp(-g)) * u)
+        assert np.allclose(res["x_final"][i], want, atol=1e-10)
+        assert np.abs(want - x0).max() > 1e-3
+
+
+def test_qk_norm_makes_unit_mean_square_keys_and_ignores_projection_scale():
+    wl = _full_layer_workload(d_ff=0, rms_eps=0.0)
+    cfg, st, _ = oracle_state(wl, 5)
+    w = orc.prepare_weights(synth.make_weights(wl.shape, 5))
+    w["wo"] = w["wo"] * 40.0
+    rd = synth.make_round(wl, 5, 0)
+    res = orc.draft_round(rd["draft"], rd["target"], rd["H"], st, w, 1, orc.MODE_CARRY)
+    # the rotation keeps a head's length, so with unit gains every cached key has mean square exactly 1
+    w1 = dict(w); w1["g_knorm"] = np.ones_like(w["g_knorm"]); w1["g_qnorm"] = np.ones_like(w["g_qnorm"])
+    _, st1, _ = oracle_state(wl, 5)
+    res1 = orc.draft_round(rd["draft"], rd["target"], rd["H"], st1, w1, 1, orc.MODE_CARRY)
+    ms = np.mean(res1["J"][:, :, 0] ** 2, axis=-1)
+    assert np.allclose(ms, 1.0, atol=1e-12)
+    # values are not normalised
+    assert np.abs(np.mean(res1["J"][:, :, 1] ** 2, axis=-1) - 1.0).min() > 1e-3
+    # a rescaled W_q or W_k changes nothing (eps = 0): queries, cached keys and block keys are all normalised
+    w2 = dict(w); w2["wq"] = w["wq"] * 7.0; w2["wk"] = w["wk"] * 0.25
+    _, st2, _ = oracle_state(wl, 5)
+    res2 = orc.draft_round(rd["draft"], rd["target"], rd["H"], st2, w2, 1, orc.MODE_CARRY)
+    assert np.allclose(res2["x_final"], res["x_final"], rtol=0, atol=1e-11)
+    assert np.allclose(st2.pool, st.pool, atol=1e-12)
+    # ... and without the norms the same rescaling does change the result
+    wl_off = synth.scaled(wl, qk_norm=False)
+    _, sa, _ = oracle_state(wl_off, 5)
+    _, sb, _ = oracle_state(wl_off, 5)
+    ra = orc.draft_round(rd["draft"], rd["target"], rd["H"], sa, w, 1, orc.MODE_CARRY)
+    rb = orc.draft_round(rd["draft"], rd["target"], rd["H"], sb, w2, 1, orc.MODE_CARRY)
+    assert np.abs(ra["x_final"] - rb["x_final"]).max() > 1e-6
+
+
+def test_qk_norm_is_applied_before_the_rotation():
+    """N(RoPE(k)) = RoPE(N(k)) only for a uniform gain; with a non-uniform gain the order shows.
+    The cached key must equal RoPE(g * k / rms(k)) computed by hand."""
+    wl = _full_layer_workload(d_ff=0, n_layers=1, S=1)
+    cfg, st, _ = oracle_state(wl, 7)
+    w = orc.prepare_weights(synth.make_weights(wl.shape, 7))
+    rd = synth.make_round(wl, 7, 0)
+    res = orc.draft_round(rd["draft"], rd["target"], rd["H"], st, w, 1, orc.MODE_CARRY)
+    Z = orc.fuse_features(rd["H"], np.repeat(np.arange(cfg.W)[None] >= res["split"]["accept_len"][:, None], 1, 0).reshape(-1), w, cfg)
+    row = 0
+    pos = int(res["split"]["row_pos"][row])
+    k = (w["wk"][0] @ Z[row]).reshape(cfg.n_kv, cfg.hd)
+    half = cfg.hd // 2
+    for h in range(cfg.n_kv):
+        kn = w["g_knorm"][0] * k[h] / math.sqrt(float(np.mean(k[h] ** 2)) + cfg.rms_eps)
+        for j in range(half):
+            ang = pos * cfg.rope_theta ** (-2.0 * j / cfg.hd)
+            want1 = kn[j] * math.cos(ang) - kn[j + half] * math.sin(ang)
+            want2 = kn[j + half] * math.cos(ang) + kn[j] * math.sin(ang)
+            assert abs(res["J"][0, row, 0, h, j] - want1) < 1e-10
+            assert abs(res["J"][0, row, 0, h, j + half] - want2) < 1e-10
