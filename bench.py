@@ -83,6 +83,8 @@ def round_model(wl, L_after, carry, kept_rows, es=2):
                  Ld * 4.0 * sh.W * sh.n_q * sh.hd * float(np.sum(L_after + carry + sh.W))),
         "lmhead": (V * D * es + R * D * es, 2.0 * R * D * V),
     }
+    if sh.d_ff > 0:      # complete layer: gate, up and down matrices once per layer
+        out["mlp"] = (Ld * (3 * D * sh.d_ff * es + R * (D + 2 * sh.d_ff) * es), 2.0 * R * 3 * D * sh.d_ff * Ld)
     return out
 
 
@@ -596,7 +598,8 @@ def main():
     ap.add_argument("--steps", type=int, default=64)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--workload", default="cfg2", choices=["cfg1", "cfg2", "cfg3", "cfg4", "cfg5"])
+    ap.add_argument("--workload", default="cfg2", choices=["cfg1", "cfg2", "cfg3", "cfg4", "cfg5", "cfg2f", "cfg3f"],
+                    help="cfg2 (default): batch 1; cfg3: batch 32; cfg2f / cfg3f: the same with the complete drafter layer (gated MLP 9728, q/k norms)")
     ap.add_argument("--seed", type=int, default=0)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-graph", action="store_true", help="time plain stream launches instead of graph replays")

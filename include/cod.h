@@ -63,6 +63,8 @@ enum cod_mode {
 /* cod_config.flags */
 #define COD_F_HIDDEN_NORM 1u /* RMS-normalise (with gain g_hidden) the output of F */
 #define COD_F_NO_TENSOR_CORES 2u /* use the plain-FMA kernels only (an on-GPU cross-check) */
+#define COD_F_QK_NORM 4u /* per-head RMS norm with gain (g_qnorm, g_knorm) of queries and of all keys,
+                            cached and block keys alike, before the rotation */
 
 /* bits of the sticky device status word */
 #define COD_DEV_BAD_TOKEN 1u      /* a token id outside [0, vocab) was met (treated as id 0) */
@@ -89,6 +91,9 @@ typedef struct {
   uint32_t flags;
   float rope_theta, rms_eps;
   int32_t attn_split_len;    /* keys per attention split (a multiple of 32); 0 = library default */
+  int32_t d_ff;              /* width of the gated MLP that follows the attention sub-layer of every
+                                drafter layer (a multiple of 64); 0 = no MLP. The paper leaves the
+                                drafter body open (Section 2.1); this is the complete-layer reading  */
 } cod_config;
 
 /* Borrowed device pointers, element type per cod_config.dtype, each matrix [out, in]. */
@@ -103,6 +108,13 @@ typedef struct {
   const void* g_attn;   /* [Ld][D]              gain of the pre-attention norm             */
   const void* g_final;  /* [D]                  gain of the final norm                     */
   const void* emb;      /* [vocab, D]           embedding table = LM head                  */
+  /* complete layer only; may be NULL when d_ff == 0 resp. COD_F_QK_NORM is not set:               */
+  const void* w_gate;   /* [Ld][d_ff, D]        x += W_down( silu(W_gate b) * (W_up b) ),          */
+  const void* w_up;     /* [Ld][d_ff, D]        b = N(x) * g_mlp, after the attention residual     */
+  const void* w_down;   /* [Ld][D, d_ff]                                                           */
+  const void* g_mlp;    /* [Ld][D]              gain of the pre-MLP norm                           */
+  const void* g_qnorm;  /* [Ld][hd]             gain of the per-head query norm                    */
+  const void* g_knorm;  /* [Ld][hd]             gain of the per-head key norm                      */
 } cod_weights;
 
 /* Mutable drafter state of a batch (device, caller-owned). */
@@ -172,7 +184,8 @@ int cod_scatter_kv(cod_ctx* ctx, const void* J, const cod_split* split, int S, i
    (Section 2 "Preliminaries"; Algorithm 1 "the next draft reads ctx_l").
    q [S, W, n_q, hd], k_blk / v_blk [S, W, n_kv, hd] device, q and k_blk NOT rotated: the
    call rotates them at positions committed_len[s] + i. No mask; scale 1/sqrt(hd); query
-   head g reads KV head g / (n_q / n_kv). use_carry = 0 ignores U_l.
+   head g reads KV head g / (n_q / n_kv). use_carry = 0 ignores U_l. With COD_F_QK_NORM
+   the caller passes q and k_blk already normalised (cod_draft_round does that itself).
    out [S, W, n_q, hd]. carry_mass (nullable) float [S, W, n_q]: share of softmax mass on
    the carried rows (the diagnostic of Appendix C). */
 int cod_block_attn(cod_ctx* ctx, int layer, const void* q, const void* k_blk, const void* v_blk,
@@ -227,7 +240,8 @@ enum cod_kernel_class {
   COD_K_OPROJ = 5,  /* output projection (per layer)        */
   COD_K_LMHEAD = 6, /* LM head + argmax                     */
   COD_K_ROWOPS = 7, /* norms, rotations, scatter, read-out  */
-  COD_K_CLASSES = 8
+  COD_K_MLP = 8,    /* gate/up and down contractions (d_ff > 0) */
+  COD_K_CLASSES = 9
 };
 
 /* Measurement aid (the paper has no counterpart): while class_mask has bit (1 << k) set,

@@ -20,6 +20,7 @@ COD_F32, COD_BF16 = 0, 1
 COD_CARRY, COD_BASELINE = 0, 1
 COD_F_HIDDEN_NORM = 1
 COD_F_NO_TENSOR_CORES = 2
+COD_F_QK_NORM = 4
 DEV_BAD_TOKEN, DEV_PAGE_OVERFLOW, DEV_BAD_PAGE, DEV_TIMEOUT, DEV_BAD_LEN = 1, 2, 4, 8, 16
 
 EXPORTS = ("cod_create", "cod_destroy", "cod_set_weights", "cod_verify_accept", "cod_project_kv",
@@ -27,7 +28,7 @@ EXPORTS = ("cod_create", "cod_destroy", "cod_set_weights", "cod_verify_accept", 
            "cod_draft_round",
            "cod_poll_status", "cod_profile_enable", "cod_profile_read", "cod_launch_count",
            "cod_workspace_bytes", "cod_error_string")
-KERNEL_CLASSES = ("verify", "fc", "kv", "qkv", "attn", "oproj", "lmhead", "rowops")
+KERNEL_CLASSES = ("verify", "fc", "kv", "qkv", "attn", "oproj", "lmhead", "rowops", "mlp")
 
 
 class CodConfig(C.Structure):
@@ -35,10 +36,11 @@ class CodConfig(C.Structure):
         "d_target", "n_cap", "d_model", "n_layers", "n_q_heads", "n_kv_heads", "head_dim", "vocab",
         "mask_token_id", "block", "page_size", "max_batch", "max_pages_per_seq", "n_pages", "dtype")] + [
         ("flags", C.c_uint32), ("rope_theta", C.c_float), ("rms_eps", C.c_float),
-        ("attn_split_len", C.c_int32)]
+        ("attn_split_len", C.c_int32), ("d_ff", C.c_int32)]
 
 
-_WEIGHT_FIELDS = ("fc", "e_carry", "g_hidden", "wk", "wv", "wq", "wo", "g_attn", "g_final", "emb")
+_WEIGHT_FIELDS = ("fc", "e_carry", "g_hidden", "wk", "wv", "wq", "wo", "g_attn", "g_final", "emb",
+                  "w_gate", "w_up", "w_down", "g_mlp", "g_qnorm", "g_knorm")   # the last six: complete layer only
 _SPLIT_FIELDS = ("accept_len", "bonus", "row_pos", "commit_slot", "carry_slot", "acc_rows", "acc_off",
                  "rej_rows", "rej_off")
 _STATE_FIELDS = ("kv_pool", "block_table", "committed_len", "carry_kv", "carry_len")
@@ -213,8 +215,8 @@ class Context:
 
     # ---- set-up
     def set_weights(self, w: Dict[str, torch.Tensor]) -> None:
-        self._weights = {k: w[k] for k in _WEIGHT_FIELDS}      # keep the tensors alive
-        ws = CodWeights(*[_ptr(self._weights[k]) for k in _WEIGHT_FIELDS])
+        self._weights = {k: w[k] for k in _WEIGHT_FIELDS if k in w}      # keep the tensors alive
+        ws = CodWeights(*[_ptr(self._weights.get(k)) for k in _WEIGHT_FIELDS])
         _check("cod_set_weights", lib().cod_set_weights(self._h, C.byref(ws), _stream()))
 
     # ---- the five parts
@@ -296,9 +298,10 @@ def make_config(sh, max_batch: int, max_pages_per_seq: int, n_pages: int, attn_s
         n_kv_heads=sh.n_kv, head_dim=sh.hd, vocab=sh.vocab, mask_token_id=sh.mask_token_id, block=sh.W,
         page_size=sh.page, max_batch=max_batch, max_pages_per_seq=max_pages_per_seq, n_pages=n_pages,
         dtype=COD_BF16 if sh.dtype == "bf16" else COD_F32,
-        flags=(COD_F_HIDDEN_NORM if sh.hidden_norm else 0) | (COD_F_NO_TENSOR_CORES if no_tensor_cores else 0),
+        flags=(COD_F_HIDDEN_NORM if sh.hidden_norm else 0) | (COD_F_NO_TENSOR_CORES if no_tensor_cores else 0)
+        | (COD_F_QK_NORM if sh.qk_norm else 0),
         rope_theta=sh.rope_theta, rms_eps=sh.rms_eps,
-        attn_split_len=attn_split_len)
+        attn_split_len=attn_split_len, d_ff=sh.d_ff)
 
 
 def weights_to_device(w: Dict[str, np.ndarray], dtype: str) -> Dict[str, torch.Tensor]:

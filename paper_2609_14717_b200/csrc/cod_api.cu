@@ -38,6 +38,7 @@ size_t carve(cod_ctx* c) {
   size_t widest = D;
   widest = widest > static_cast<size_t>(2 * f.n_layers * c->kvw) ? widest : static_cast<size_t>(2 * f.n_layers * c->kvw);
   widest = widest > static_cast<size_t>(c->qw + 2 * c->kvw) ? widest : static_cast<size_t>(c->qw + 2 * c->kvw);
+  widest = widest > static_cast<size_t>(2 * f.d_ff) ? widest : static_cast<size_t>(2 * f.d_ff);
   c->gemm_out_floats = static_cast<size_t>(COD_MAX_SPLITS) * R * widest;
   cv.take(c->gemm_out, sizeof(float) * c->gemm_out_floats);
   cv.take(c->hc, es * R * c->D_in);
@@ -48,6 +49,7 @@ size_t carve(cod_ctx* c) {
   cv.take(c->kb, es * R * c->kvw);
   cv.take(c->vb, es * R * c->kvw);
   cv.take(c->o, es * R * c->qw);
+  if (f.d_ff > 0) cv.take(c->hmid, es * R * f.d_ff);
   const size_t M = static_cast<size_t>(f.block) * (f.n_q_heads / f.n_kv_heads);
   const size_t per_head = static_cast<size_t>(c->max_splits > c->tc_max_parts ? c->max_splits : c->tc_max_parts);
   const size_t parts = static_cast<size_t>(f.max_batch) * f.n_kv_heads * per_head * M;
@@ -133,6 +135,8 @@ int cod_create(const cod_config* cfg, cod_ctx** out) {
   if (f.block > COD_MAX_W || f.block * (f.n_q_heads / f.n_kv_heads) > 128) return COD_ERR_UNSUPPORTED;
   if ((f.d_target * f.n_cap) % 8 || f.d_model % 8 || f.d_model > 32768) return COD_ERR_UNSUPPORTED;
   if ((f.n_kv_heads * f.head_dim) % 64) return COD_ERR_UNSUPPORTED;
+  if (f.d_ff < 0) return COD_ERR_INVALID_ARG;
+  if (f.d_ff % 64) return COD_ERR_UNSUPPORTED;   // gate and up share one contraction: tiles must not straddle them
   if (static_cast<int64_t>(f.n_pages) * f.page_size > (1ll << 31) - 1) return COD_ERR_UNSUPPORTED;
 
   cod_ctx* c = new (std::nothrow) cod_ctx();
@@ -217,6 +221,12 @@ int cod_set_weights(cod_ctx* c, const cod_weights* w, cod_stream_t stream) {
   const void* ps[] = {w->fc, w->e_carry, w->g_hidden, w->wk, w->wv, w->wq, w->wo, w->g_attn, w->g_final, w->emb};
   for (const void* p : ps)
     if (!p || misaligned(p)) return COD_ERR_INVALID_ARG;
+  if (c->cfg.d_ff > 0)
+    for (const void* p : {w->w_gate, w->w_up, w->w_down, w->g_mlp})
+      if (!p || misaligned(p)) return COD_ERR_INVALID_ARG;
+  if (c->cfg.flags & COD_F_QK_NORM)
+    for (const void* p : {w->g_qnorm, w->g_knorm})
+      if (!p || misaligned(p)) return COD_ERR_INVALID_ARG;
   c->w = *w;
   c->has_weights = true;
   c->pdl = false;
@@ -355,7 +365,7 @@ int cod_draft_round(cod_ctx* c, const int32_t* draft, const int32_t* target, con
     g.n_seg = 3; g.klass = COD_K_QKV;
     g.C = c->gemm_out; g.ldc = c->qw + 2 * c->kvw; g.splits = pick_splits(c, g.ldc, c->D, R);
     if ((rc = cod_launch_gemm(c, g, s)) != COD_OK) return rc;
-    if ((rc = cod_launch_qkv_finish(c, c->gemm_out, g.splits, R, s)) != COD_OK) return rc;
+    if ((rc = cod_launch_qkv_finish(c, c->gemm_out, g.splits, R, l, s)) != COD_OK) return rc;
 
     float* tap_o = (taps && taps->attn_out) ? taps->attn_out + static_cast<size_t>(l) * R * c->qw : nullptr;
     if ((rc = cod_launch_attn(c, l, c->q, c->kb, c->vb, st, S, mode == COD_CARRY ? 1 : 0, c->o, tap_o, nullptr, s)) != COD_OK)
@@ -369,7 +379,30 @@ int cod_draft_round(cod_ctx* c, const int32_t* draft, const int32_t* target, con
     if ((rc = cod_launch_gemm(c, o, s)) != COD_OK) return rc;
     const bool last = l + 1 == f.n_layers;
     const void* gain = last ? c->w.g_final : static_cast<const char*>(c->w.g_attn) + es * (l + 1) * c->D;
-    if ((rc = cod_launch_resid_norm(c, c->gemm_out, o.splits, R, c->x, gain,
+    if (f.d_ff == 0) {
+      if ((rc = cod_launch_resid_norm(c, c->gemm_out, o.splits, R, c->x, gain,
+                                      (last && taps) ? taps->x_final : nullptr, s)) != COD_OK)
+        return rc;
+      continue;
+    }
+    // the gated MLP of the complete layer: b = N(x) g_mlp; x += W_down( silu(W_gate b) * (W_up b) )
+    const void* g_mlp = static_cast<const char*>(c->w.g_mlp) + es * l * c->D;
+    if ((rc = cod_launch_resid_norm(c, c->gemm_out, o.splits, R, c->x, g_mlp, nullptr, s)) != COD_OK) return rc;
+    GemmArgs gu{};
+    gu.A = c->a; gu.lda = c->D; gu.n_rows = R; gu.K = c->D;
+    gu.seg[0] = {static_cast<const char*>(c->w.w_gate) + es * l * f.d_ff * c->D, f.d_ff};
+    gu.seg[1] = {static_cast<const char*>(c->w.w_up) + es * l * f.d_ff * c->D, f.d_ff};
+    gu.n_seg = 2; gu.klass = COD_K_MLP;
+    gu.C = c->gemm_out; gu.ldc = 2 * f.d_ff; gu.splits = pick_splits(c, gu.ldc, c->D, R);
+    if ((rc = cod_launch_gemm(c, gu, s)) != COD_OK) return rc;
+    if ((rc = cod_launch_swiglu_finish(c, c->gemm_out, gu.splits, R, s)) != COD_OK) return rc;
+    GemmArgs dn{};
+    dn.A = c->hmid; dn.lda = f.d_ff; dn.n_rows = R; dn.K = f.d_ff;
+    dn.seg[0] = {static_cast<const char*>(c->w.w_down) + es * l * c->D * f.d_ff, c->D};
+    dn.n_seg = 1; dn.klass = COD_K_MLP;
+    dn.C = c->gemm_out; dn.ldc = c->D; dn.splits = pick_splits(c, c->D, f.d_ff, R);
+    if ((rc = cod_launch_gemm(c, dn, s)) != COD_OK) return rc;
+    if ((rc = cod_launch_resid_norm(c, c->gemm_out, dn.splits, R, c->x, gain,
                                     (last && taps) ? taps->x_final : nullptr, s)) != COD_OK)
       return rc;
   }

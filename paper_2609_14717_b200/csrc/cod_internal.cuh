@@ -133,6 +133,7 @@ struct cod_ctx {
   float* fcE;                  // [D]     F(E_carry)
   float* rope_win;             // [R_max][hd]  cos | sin of the window rows' positions
   float* rope_blk;             // [R_max][hd]  cos | sin of the block rows' positions
+  void* hmid;                  // [R, d_ff] activated MLP rows (storage type), d_ff > 0 only
   float* gemm_out;             // split-K / unfused GEMM results
   size_t gemm_out_floats;
   void* hc;                    // [R_max, D_in] accepted rows of H packed densely (baseline mode)
@@ -223,7 +224,8 @@ int cod_launch_scatter(cod_ctx* c, const void* J, const cod_split* sp, int S, in
 int cod_launch_update_lens(cod_ctx* c, const cod_split* sp, int S, int mode, const cod_state* state,
                            cudaStream_t st);
 int cod_launch_embed_norm(cod_ctx* c, const int32_t* bonus, int S, cudaStream_t st);
-int cod_launch_qkv_finish(cod_ctx* c, const float* part, int splits, int R, cudaStream_t st);
+int cod_launch_qkv_finish(cod_ctx* c, const float* part, int splits, int R, int layer, cudaStream_t st);
+int cod_launch_swiglu_finish(cod_ctx* c, const float* part, int splits, int R, cudaStream_t st);
 int cod_launch_rope_qk(cod_ctx* c, const void* q, const void* k, const int32_t* committed_len, int S,
                        cudaStream_t st);  // standalone attention entry: rotate into c->q / c->kb
 int cod_launch_attn(cod_ctx* c, int layer, const void* q, const void* kb, const void* vb,

@@ -19,6 +19,15 @@ __device__ __forceinline__ void cod_st4(__nv_bfloat16* p, float4 v) {
 __device__ __forceinline__ float4 f4_add(float4 a, float4 b) { return make_float4(a.x + b.x, a.y + b.y, a.z + b.z, a.w + b.w); }
 __device__ __forceinline__ float f4_ss(float4 a) { return a.x * a.x + a.y * a.y + a.z * a.z + a.w * a.w; }
 
+// Sum over the `group` consecutive lanes (a power of two <= 32) a head's threads occupy.
+__device__ __forceinline__ float group_sum(float v, int group) {
+  for (int o = group >> 1; o >= 1; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+  return v;
+}
+__device__ __forceinline__ float4 f4_scale_gain(float4 v, float s, float4 g) {
+  return make_float4(v.x * s * g.x, v.y * s * g.y, v.z * s * g.z, v.w * s * g.w);
+}
+
 __device__ __forceinline__ int valid_rows(const int* n_rows_dev, int n_rows) {
   return n_rows_dev ? min(*n_rows_dev, n_rows) : n_rows;
 }
@@ -112,7 +121,7 @@ __global__ void k_kv_finish(const float* __restrict__ part, int splits, int n_ro
                             int n_kv, int hd, T* __restrict__ J, int R_total,
                             const int* __restrict__ commit_slot, const int* __restrict__ carry_slot,
                             T* __restrict__ pool, T* __restrict__ carry, int page, int n_pages, int W,
-                            int max_batch, int to_state) {
+                            int max_batch, int to_state, const T* __restrict__ g_k, float eps) {
   cod_pdl_prologue();
   const int i = blockIdx.x, l = blockIdx.y;
   if (i >= valid_rows(n_rows_dev, n_rows)) return;
@@ -142,19 +151,34 @@ __global__ void k_kv_finish(const float* __restrict__ part, int splits, int n_ro
       return;   // nowhere to go (position beyond the page table: already flagged)
     }
   }
-  // hd / 8 threads per head: 4 consecutive elements of the lower half and their RoPE partners
+  // hd / 8 threads per head: 4 consecutive elements of the lower half and their RoPE partners.
+  // With the per-head key norm (g_k non-null, gains of layer l at g_k + l * hd) a head's threads
+  // first share the key's sum of squares; whole warps stay in the loop for those shuffles.
   const int tph = half >> 2;
-  for (int e = threadIdx.x; e < n_kv * tph; e += blockDim.x) {
-    const int h = e / tph, j = (e - h * tph) * 4;
+  for (int e0 = 0; e0 < n_kv * tph; e0 += blockDim.x) {
+    const int e = e0 + threadIdx.x;
+    const bool live = e < n_kv * tph;
+    const int h = live ? e / tph : 0, j = live ? (e - h * tph) * 4 : 0;
     float4 k1 = make_float4(0.f, 0.f, 0.f, 0.f), k2 = k1, v1 = k1, v2 = k1;
     const float* p = part + static_cast<size_t>(i) * ldc + l * kvw + h * hd + j;
     const size_t slab = static_cast<size_t>(n_rows) * ldc;
-    for (int s = 0; s < splits; ++s) {
-      k1 = f4_add(k1, *reinterpret_cast<const float4*>(p + s * slab));
-      k2 = f4_add(k2, *reinterpret_cast<const float4*>(p + s * slab + half));
-      v1 = f4_add(v1, *reinterpret_cast<const float4*>(p + s * slab + Ld * kvw));
-      v2 = f4_add(v2, *reinterpret_cast<const float4*>(p + s * slab + Ld * kvw + half));
+    if (live) {
+      for (int s = 0; s < splits; ++s) {
+        k1 = f4_add(k1, *reinterpret_cast<const float4*>(p + s * slab));
+        k2 = f4_add(k2, *reinterpret_cast<const float4*>(p + s * slab + half));
+        v1 = f4_add(v1, *reinterpret_cast<const float4*>(p + s * slab + Ld * kvw));
+        v2 = f4_add(v2, *reinterpret_cast<const float4*>(p + s * slab + Ld * kvw + half));
+      }
     }
+    if (g_k != nullptr) {
+      const float ss = group_sum(f4_ss(k1) + f4_ss(k2), tph);
+      const float sc = rsqrtf(ss / static_cast<float>(hd) + eps);
+      if (live) {
+        k1 = f4_scale_gain(k1, sc, cod_ld4(g_k + l * hd + j));
+        k2 = f4_scale_gain(k2, sc, cod_ld4(g_k + l * hd + half + j));
+      }
+    }
+    if (!live) continue;
     const float4 c = *reinterpret_cast<const float4*>(cs + j), sn = *reinterpret_cast<const float4*>(cs + half + j);
     T* kd = dstK + h * h_stride;
     cod_st4(kd + j, make_float4(k1.x * c.x - k2.x * sn.x, k1.y * c.y - k2.y * sn.y, k1.z * c.z - k2.z * sn.z, k1.w * c.w - k2.w * sn.w));
@@ -257,23 +281,37 @@ __global__ void __launch_bounds__(1024) k_embed_norm(const T* __restrict__ emb, 
 template <typename T>
 __global__ void k_qkv_finish(const float* __restrict__ part, int splits, int R, int n_q, int n_kv, int hd,
                              const float* __restrict__ rope_blk, T* __restrict__ q, T* __restrict__ kb,
-                             T* __restrict__ vb, int hpb) {
+                             T* __restrict__ vb, int hpb, const T* __restrict__ g_q, const T* __restrict__ g_k,
+                             float eps) {
   cod_pdl_prologue();
   // A block covers hpb heads of one row; hd / 8 threads per head, each owning 4 consecutive
   // elements of the lower half and their partners in the upper half (the pairs RoPE mixes).
   // Heads 0..n_q-1 are q, then n_kv heads of k (both rotated), then n_kv heads of v.
+  // With per-head norms (g_q, g_k non-null) a head's threads first share its sum of squares.
   const int half = hd >> 1, tph = half >> 2;
   const int r = blockIdx.x, hh = blockIdx.y * hpb + threadIdx.x / tph, j = (threadIdx.x % tph) * 4;
-  if (hh >= n_q + 2 * n_kv) return;
+  const bool live = hh < n_q + 2 * n_kv;            // whole warps stay for the shuffles
   const int qw = n_q * hd, kvw = n_kv * hd, ldc = qw + 2 * kvw;
-  const float* p = part + static_cast<size_t>(r) * ldc + hh * hd + j;
+  const float* p = part + static_cast<size_t>(r) * ldc + (live ? hh : 0) * hd + j;
   const size_t slab = static_cast<size_t>(R) * ldc;
   float4 a = make_float4(0.f, 0.f, 0.f, 0.f), b = a;
-  for (int s = 0; s < splits; ++s) {
-    a = f4_add(a, *reinterpret_cast<const float4*>(p + s * slab));
-    b = f4_add(b, *reinterpret_cast<const float4*>(p + s * slab + half));
+  if (live) {
+    for (int s = 0; s < splits; ++s) {
+      a = f4_add(a, *reinterpret_cast<const float4*>(p + s * slab));
+      b = f4_add(b, *reinterpret_cast<const float4*>(p + s * slab + half));
+    }
   }
   const bool rot = hh < n_q + n_kv;
+  const T* gain = hh < n_q ? g_q : (rot ? g_k : nullptr);
+  if (g_q != nullptr) {                               // block-uniform: every lane takes the shuffles
+    const float ss = group_sum(f4_ss(a) + f4_ss(b), tph);
+    if (live && gain != nullptr) {
+      const float sc = rsqrtf(ss / static_cast<float>(hd) + eps);
+      a = f4_scale_gain(a, sc, cod_ld4(gain + j));
+      b = f4_scale_gain(b, sc, cod_ld4(gain + half + j));
+    }
+  }
+  if (!live) return;
   T* dst = hh < n_q ? q + static_cast<size_t>(r) * qw + hh * hd
                     : (rot ? kb + static_cast<size_t>(r) * kvw + (hh - n_q) * hd
                            : vb + static_cast<size_t>(r) * kvw + (hh - n_q - n_kv) * hd);
@@ -286,6 +324,26 @@ __global__ void k_qkv_finish(const float* __restrict__ part, int splits, int R, 
     cod_st4(dst + j, a);
     cod_st4(dst + j + half, b);
   }
+}
+
+// ------------------------------------------------------------------ gated MLP activation
+// part: [splits][R][2 * d_ff] (gate columns, then up columns) -> h[r, j] = silu(gate) * up
+template <typename T>
+__global__ void k_swiglu_finish(const float* __restrict__ part, int splits, int R, int d_ff, T* __restrict__ h) {
+  cod_pdl_prologue();
+  const int r = blockIdx.x, j = (blockIdx.y * blockDim.x + threadIdx.x) * 4;
+  if (j >= d_ff) return;
+  const float* p = part + static_cast<size_t>(r) * 2 * d_ff + j;
+  const size_t slab = static_cast<size_t>(R) * 2 * d_ff;
+  float4 g = make_float4(0.f, 0.f, 0.f, 0.f), u = g;
+#pragma unroll 4
+  for (int s = 0; s < splits; ++s) {
+    g = f4_add(g, *reinterpret_cast<const float4*>(p + s * slab));
+    u = f4_add(u, *reinterpret_cast<const float4*>(p + s * slab + d_ff));
+  }
+  cod_st4(h + static_cast<size_t>(r) * d_ff + j,
+          make_float4(g.x / (1.f + expf(-g.x)) * u.x, g.y / (1.f + expf(-g.y)) * u.y,
+                      g.z / (1.f + expf(-g.z)) * u.z, g.w / (1.f + expf(-g.w)) * u.w));
 }
 
 // Rotates caller-supplied q / k_blk (the stand-alone attention entry point).
@@ -434,8 +492,8 @@ int cod_launch_kv_finish(cod_ctx* c, const float* part, int splits, int n_rows, 
   dim3 grid(n_rows, f.n_layers);
   const int to_state = ds ? 1 : 0;
   DISPATCH_T(c,
-             (cod_launch_pdl(c, k_kv_finish<__nv_bfloat16>, grid, 128, 0, st, part, splits, n_rows, n_rows_dev, a_rows, c->rope_win, f.n_layers, f.n_kv_heads, f.head_dim, static_cast<__nv_bfloat16*>(J), R_total, sp->commit_slot, sp->carry_slot, ds ? static_cast<__nv_bfloat16*>(ds->kv_pool) : nullptr, ds ? static_cast<__nv_bfloat16*>(ds->carry_kv) : nullptr, f.page_size, f.n_pages, f.block, f.max_batch, to_state)),
-             (cod_launch_pdl(c, k_kv_finish<float>, grid, 128, 0, st, part, splits, n_rows, n_rows_dev, a_rows, c->rope_win, f.n_layers, f.n_kv_heads, f.head_dim, static_cast<float*>(J), R_total, sp->commit_slot, sp->carry_slot, ds ? static_cast<float*>(ds->kv_pool) : nullptr, ds ? static_cast<float*>(ds->carry_kv) : nullptr, f.page_size, f.n_pages, f.block, f.max_batch, to_state)));
+             (cod_launch_pdl(c, k_kv_finish<__nv_bfloat16>, grid, 128, 0, st, part, splits, n_rows, n_rows_dev, a_rows, c->rope_win, f.n_layers, f.n_kv_heads, f.head_dim, static_cast<__nv_bfloat16*>(J), R_total, sp->commit_slot, sp->carry_slot, ds ? static_cast<__nv_bfloat16*>(ds->kv_pool) : nullptr, ds ? static_cast<__nv_bfloat16*>(ds->carry_kv) : nullptr, f.page_size, f.n_pages, f.block, f.max_batch, to_state, (f.flags & COD_F_QK_NORM) ? static_cast<const __nv_bfloat16*>(c->w.g_knorm) : nullptr, f.rms_eps)),
+             (cod_launch_pdl(c, k_kv_finish<float>, grid, 128, 0, st, part, splits, n_rows, n_rows_dev, a_rows, c->rope_win, f.n_layers, f.n_kv_heads, f.head_dim, static_cast<float*>(J), R_total, sp->commit_slot, sp->carry_slot, ds ? static_cast<float*>(ds->kv_pool) : nullptr, ds ? static_cast<float*>(ds->carry_kv) : nullptr, f.page_size, f.n_pages, f.block, f.max_batch, to_state, (f.flags & COD_F_QK_NORM) ? static_cast<const float*>(c->w.g_knorm) : nullptr, f.rms_eps)));
   COD_CHECK_LAUNCH(c);
   return COD_OK;
 }
@@ -480,17 +538,31 @@ int cod_launch_embed_norm(cod_ctx* c, const int32_t* bonus, int S, cudaStream_t 
   return COD_OK;
 }
 
-int cod_launch_qkv_finish(cod_ctx* c, const float* part, int splits, int R, cudaStream_t st) {
+int cod_launch_qkv_finish(cod_ctx* c, const float* part, int splits, int R, int layer, cudaStream_t st) {
   ProfScope prof(c, COD_K_ROWOPS, st);
   const cod_config& f = c->cfg;
-  // heads per block: as many (up to 8) as still leave a couple of blocks per SM
+  // heads per block: as many (up to 8) as still leave a couple of blocks per SM; whole warps always
   const int nh = f.n_q_heads + 2 * f.n_kv_heads, tph = f.head_dim / 8;
+  const int hpb_min = 32 / tph > 1 ? 32 / tph : 1;
   int hpb = 8;
-  while (hpb > 1 && R * ((nh + hpb - 1) / hpb) < 2 * c->n_sm) hpb >>= 1;
+  while (hpb > hpb_min && R * ((nh + hpb - 1) / hpb) < 2 * c->n_sm) hpb >>= 1;
   const dim3 grid(R, (nh + hpb - 1) / hpb);
+  const bool qk = (f.flags & COD_F_QK_NORM) != 0;
+  const size_t goff = static_cast<size_t>(layer) * f.head_dim;
   DISPATCH_T(c,
-             (cod_launch_pdl(c, k_qkv_finish<__nv_bfloat16>, grid, tph * hpb, 0, st, part, splits, R, f.n_q_heads, f.n_kv_heads, f.head_dim, c->rope_blk, static_cast<__nv_bfloat16*>(c->q), static_cast<__nv_bfloat16*>(c->kb), static_cast<__nv_bfloat16*>(c->vb), hpb)),
-             (cod_launch_pdl(c, k_qkv_finish<float>, grid, tph * hpb, 0, st, part, splits, R, f.n_q_heads, f.n_kv_heads, f.head_dim, c->rope_blk, static_cast<float*>(c->q), static_cast<float*>(c->kb), static_cast<float*>(c->vb), hpb)));
+             (cod_launch_pdl(c, k_qkv_finish<__nv_bfloat16>, grid, tph * hpb, 0, st, part, splits, R, f.n_q_heads, f.n_kv_heads, f.head_dim, c->rope_blk, static_cast<__nv_bfloat16*>(c->q), static_cast<__nv_bfloat16*>(c->kb), static_cast<__nv_bfloat16*>(c->vb), hpb, qk ? static_cast<const __nv_bfloat16*>(c->w.g_qnorm) + goff : nullptr, qk ? static_cast<const __nv_bfloat16*>(c->w.g_knorm) + goff : nullptr, f.rms_eps)),
+             (cod_launch_pdl(c, k_qkv_finish<float>, grid, tph * hpb, 0, st, part, splits, R, f.n_q_heads, f.n_kv_heads, f.head_dim, c->rope_blk, static_cast<float*>(c->q), static_cast<float*>(c->kb), static_cast<float*>(c->vb), hpb, qk ? static_cast<const float*>(c->w.g_qnorm) + goff : nullptr, qk ? static_cast<const float*>(c->w.g_knorm) + goff : nullptr, f.rms_eps)));
+  COD_CHECK_LAUNCH(c);
+  return COD_OK;
+}
+
+int cod_launch_swiglu_finish(cod_ctx* c, const float* part, int splits, int R, cudaStream_t st) {
+  ProfScope prof(c, COD_K_ROWOPS, st);
+  const int d_ff = c->cfg.d_ff;
+  const dim3 grid(R, (d_ff / 4 + 255) / 256);
+  DISPATCH_T(c,
+             (cod_launch_pdl(c, k_swiglu_finish<__nv_bfloat16>, grid, 256, 0, st, part, splits, R, d_ff, static_cast<__nv_bfloat16*>(c->hmid))),
+             (cod_launch_pdl(c, k_swiglu_finish<float>, grid, 256, 0, st, part, splits, R, d_ff, static_cast<float*>(c->hmid))));
   COD_CHECK_LAUNCH(c);
   return COD_OK;
 }

@@ -51,7 +51,7 @@ def _setup(name, seed, sample):
     return wl, lay, w, ctx, cfg, st_g, cfg_o, st_o
 
 
-@pytest.mark.parametrize("name,sample", [("cfg2", [0]), ("cfg3", [5, 22])])
+@pytest.mark.parametrize("name,sample", [("cfg2", [0]), ("cfg3", [5, 22]), ("cfg2f", [0]), ("cfg3f", [9])])
 def test_full_size_round_on_sampled_sequences(name, sample):
     from paper_2609_14717_b200 import binding as B
     wl, lay, w, ctx, cfg, st_g, cfg_o, st_o = _setup(name, 11, sample)

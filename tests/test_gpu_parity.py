@@ -98,6 +98,15 @@ def _workloads():
         # wide enough for split-K, several token tiles with a ragged last one, a ragged vocab tile
         "mid_bf16": small_bf16(S=34, W=16, n_layers=2, ctx=(100, 600), d_target=512, n_cap=5, d_model=1024,
                                n_q=8, n_kv=2, vocab=3000),
+        # the complete drafter layer: gated MLP (width not a multiple of the 128-row weight tile in the
+        # float32 case, a whole number of 256-row pairs in the wide bf16 case) and per-head q/k norms
+        "tiny_f32_full": synth.scaled(synth.workload("cfg1"), S=3, ctx=(5, 140), n_rounds=6, d_ff=192, qk_norm=True,
+                                      n_layers=2),
+        "small_bf16_full": small_bf16(S=3, W=16, n_layers=2, ctx=(40, 300), d_ff=768, qk_norm=True),
+        "small_bf16_mlp_only": small_bf16(S=2, W=16, n_layers=2, ctx=(40, 300), d_ff=384),
+        "small_bf16_qknorm_only": small_bf16(S=2, W=8, n_layers=2, ctx=(40, 300), qk_norm=True),
+        "mid_bf16_full": small_bf16(S=34, W=16, n_layers=2, ctx=(100, 600), d_target=512, n_cap=5, d_model=1024,
+                                    n_q=8, n_kv=2, vocab=3000, d_ff=1536, qk_norm=True),
     }
 
 
@@ -312,7 +321,11 @@ def test_round_parity_cfg1_every_round():
     ("tiny_f32", 40.0, orc.MODE_CARRY), ("tiny_f32", 40.0, orc.MODE_BASELINE), ("tiny_f32_nonorm", 1.0, orc.MODE_CARRY),
     ("small_bf16", 30.0, orc.MODE_CARRY), ("small_bf16", 30.0, orc.MODE_BASELINE),
     ("small_bf16_W32", 1.0, orc.MODE_CARRY), ("small_bf16_W8", 30.0, orc.MODE_CARRY),
-    ("mid_bf16", 30.0, orc.MODE_CARRY), ("mid_bf16", 30.0, orc.MODE_BASELINE)])
+    ("mid_bf16", 30.0, orc.MODE_CARRY), ("mid_bf16", 30.0, orc.MODE_BASELINE),
+    ("tiny_f32_full", 40.0, orc.MODE_CARRY), ("tiny_f32_full", 40.0, orc.MODE_BASELINE),
+    ("small_bf16_full", 30.0, orc.MODE_CARRY), ("small_bf16_full", 30.0, orc.MODE_BASELINE),
+    ("small_bf16_mlp_only", 30.0, orc.MODE_CARRY), ("small_bf16_qknorm_only", 30.0, orc.MODE_CARRY),
+    ("mid_bf16_full", 30.0, orc.MODE_CARRY)])
 def test_round_parity_multi_round(name, wo_scale, mode):
     """Open-loop rounds (inputs pre-generated), ragged acceptance, attention path made to matter."""
     Hn = _H()
@@ -399,4 +412,16 @@ def test_status_word_and_argument_errors():
         ctx2.draft_round(dev["draft"], dev["target"], dev["H"], wl.S, 1, 0, P.st_g, P.split, P.next_draft, None)
     assert e.value.status == -4
     ctx2.close()
+    # the complete layer needs its own weights, and a gate/up width the contraction tiles accept
+    full = synth.scaled(wl, d_ff=128, qk_norm=True)
+    ctx3 = B.Context(B.make_config(full.shape, 2, 4, 8))
+    with pytest.raises(B.CodError) as e:
+        ctx3.set_weights(P.w_g)                                       # no w_gate / g_qnorm ...
+    assert e.value.status == -1
+    ctx3.close()
+    cfg = B.make_config(full.shape, 2, 4, 8)
+    cfg.d_ff = 100
+    with pytest.raises(B.CodError) as e:
+        B.Context(cfg)
+    assert e.value.status == -2
     P.close()
