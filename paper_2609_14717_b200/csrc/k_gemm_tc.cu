@@ -37,11 +37,23 @@ struct TcParams {
   int seg_tile_end[3];        // cumulative count of 128-row tiles after each weight segment
   int seg_N[3];
   int n_seg;
+  int staged;                 // epilogue may transpose through shared memory (16-byte aligned feature runs)
   float* C;
   int ldc;
   unsigned long long* amax;
   uint32_t* status;
 };
+
+// AND of a predicate over the 128 threads of warps 0-3 (named barrier 1)
+__device__ __forceinline__ bool bar_and_128(bool v) {
+  uint32_t r;
+  asm volatile(
+      "{\n\t.reg .pred p, q;\n\tsetp.ne.b32 q, %1, 0;\n\t"
+      "bar.red.and.pred p, 1, 128, q;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(r) : "r"(static_cast<uint32_t>(v)) : "memory");
+  return r != 0;
+}
 
 
 
@@ -152,12 +164,42 @@ k_gemm_tc(const __grid_constant__ CUtensorMap map_w0, const __grid_constant__ CU
     }
   } else if (n_kb > 0) {
     // ------------------------------------------------ epilogue warps 0..3
-    const bool ok = mbar_wait(smem_u32(acc_bar), 0, abort_flag, p.status);
+    // one verdict for the four epilogue warps (they meet at a named barrier below)
+    const bool ok = bar_and_128(mbar_wait(smem_u32(acc_bar), 0, abort_flag, p.status));
     tc_fence_after();
     const int f = f0 + warp * 32 + lane;                    // weight row within the segment
     const bool f_ok = f < seg_N;
     const uint32_t t_lane = tmem_base + (static_cast<uint32_t>(warp * 32) << 16);
-    if (ok && p.amax == nullptr) {
+    if (ok && p.amax == nullptr && p.staged && p.NT >= 32) {
+      // The accumulator has features on lanes and tokens on columns; C wants a token's features
+      // contiguous. Transpose 32 tokens at a time through the (now idle) pipeline buffers and store
+      // whole 512-byte feature runs: two 16 KB buffers, one barrier of the four warps per chunk.
+      float* C = p.C + static_cast<size_t>(split) * p.n_rows * p.ldc + col0;
+      float* stage = reinterpret_cast<float*>(sm);
+      const int f_left = seg_N - f0;                       // features of this tile that exist
+      for (int c = 0, q = 0; c < p.NT && i0 + c < n_rows; c += 32, q ^= 1) {
+        uint32_t v[32];
+        if (c + 32 <= p.NT) {
+          tmem_ld32(t_lane + c, v);
+        } else {                                           // NT is a multiple of 16: a last half chunk
+          uint32_t h[16];
+          tmem_ld16(t_lane + c, h);
+#pragma unroll
+          for (int j = 0; j < 16; ++j) { v[j] = h[j]; v[16 + j] = 0u; }
+        }
+        float* buf = stage + q * (32 * BM);
+#pragma unroll
+        for (int j = 0; j < 32; ++j) buf[j * BM + warp * 32 + lane] = __uint_as_float(v[j]);
+        asm volatile("bar.sync 1, 128;" ::: "memory");
+#pragma unroll
+        for (int t = 0; t < 8; ++t) {
+          const int tok = warp * 8 + t, i = i0 + c + tok;
+          if (c + tok < p.NT && i < n_rows && lane * 4 < f_left)
+            *reinterpret_cast<float4*>(C + static_cast<size_t>(i) * p.ldc + lane * 4) =
+                *reinterpret_cast<const float4*>(buf + tok * BM + lane * 4);
+        }
+      }
+    } else if (ok && p.amax == nullptr) {
       float* C = p.C + static_cast<size_t>(split) * p.n_rows * p.ldc;
       for (int c = 0; c < p.NT; c += 16) {
         uint32_t v[16];
@@ -270,6 +312,9 @@ int cod_launch_gemm_tc(cod_ctx* c, const GemmArgs& g, cudaStream_t st) {
   p.n_seg = g.n_seg;
   p.C = g.C;
   p.ldc = g.ldc;
+  p.staged = (g.ldc % 4 == 0) && ((reinterpret_cast<uintptr_t>(g.C) & 15u) == 0) &&
+             static_cast<size_t>(stages) * stage_bytes >= 2u * 32u * BM * sizeof(float);
+  for (int i = 0; i < g.n_seg; ++i) p.staged = p.staged && (g.seg[i].N % 4 == 0);
   p.amax = g.amax;
   p.status = c->status;
 
