@@ -360,3 +360,30 @@ def draft_round(draft: np.ndarray, target: np.ndarray, H: np.ndarray, st: Oracle
     next_draft[:, 0] = split["bonus"]
     res.update(split=split, J=J, next_draft=next_draft.astype(np.int32))
     return res
+
+
+# =========================================================================== analysis aids
+def reconvergence_count(z: np.ndarray, y: np.ndarray, length: np.ndarray) -> np.ndarray:
+    """Re-convergence count R of Section 5.2 ("Why do gains differ across datasets?", the
+    equation defining R), per sequence.
+
+    z[s, q]: the verifier's top-1 next-token prediction from the q-th rejected state;
+    y[s, q]: the token eventually committed at the position that prediction refers to;
+    length[s]: the rejected suffix length L.  Position q counts if z_{q+d} = y_q for some
+    d in {-1, 0, +1}, indices outside [0, L) ignored (a one-position tolerance for a local
+    insertion or deletion).
+    """
+    z = np.asarray(z)
+    y = np.asarray(y)
+    S = z.shape[0]
+    out = np.zeros(S, dtype=np.int32)
+    for s in range(S):
+        L = int(length[s])
+        for q in range(L):
+            hit = False
+            for d in (-1, 0, 1):
+                if 0 <= q + d < L and int(z[s, q + d]) == int(y[s, q]):
+                    hit = True
+            out[s] += 1 if hit else 0
+    return out
+

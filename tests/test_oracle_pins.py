@@ -718,3 +718,30 @@ def test_qk_norm_is_applied_before_the_rotation():
             want2 = kn[j + half] * math.cos(ang) + kn[j] * math.sin(ang)
             assert abs(res["J"][0, row, 0, h, j] - want1) < 1e-10
             assert abs(res["J"][0, row, 0, h, j + half] - want2) < 1e-10
+
+
+# ----------------------------------------------------------------------------- analysis aids
+def test_reconvergence_hand_examples():
+    z = np.array([[5, 6, 7, 8], [5, 6, 7, 8], [5, 6, 7, 8], [1, 1, 1, 1], [5, 6, 7, 8]])
+    y = np.array([[5, 6, 7, 8],      # identical: every position matches at d = 0
+                  [6, 7, 8, 9],      # continuation shifted by one (a deleted token): q = 0, 1, 2 match at d = +1
+                  [4, 5, 6, 7],      # shifted the other way (an inserted token): q = 1, 2, 3 match at d = -1
+                  [2, 2, 2, 2],      # nothing in common
+                  [7, 7, 7, 7]])     # z_2 = 7 is within one position of q = 1, 2, 3 only
+    L = np.array([4, 4, 4, 4, 4])
+    assert orc.reconvergence_count(z, y, L).tolist() == [4, 3, 3, 0, 3]
+    # the suffix length cuts both the positions counted and the neighbours looked at
+    assert orc.reconvergence_count(z, y, np.array([2, 2, 2, 2, 2])).tolist() == [2, 1, 1, 0, 0]
+    assert orc.reconvergence_count(z, y, np.zeros(5, dtype=int)).tolist() == [0] * 5
+
+
+def test_reconvergence_against_a_set_formulation_exhaustive():
+    """All z, y over a 3-letter alphabet with L = 4: position q counts iff y_q is in the set
+    {z_j : |j - q| <= 1, 0 <= j < L}."""
+    L = 4
+    for zt in itertools.product(range(3), repeat=L):
+        zz = np.array([zt])
+        for yt in itertools.product(range(3), repeat=L):
+            want = sum(1 for q in range(L) if yt[q] in {zt[j] for j in range(max(0, q - 1), min(L, q + 2))})
+            assert int(orc.reconvergence_count(zz, np.array([yt]), np.array([L]))[0]) == want
+
