@@ -146,6 +146,8 @@ typedef struct {
   float* attn_out;  /* [Ld][S*W, n_q*hd]   attention output of every layer                  */
   float* x_final;   /* [S*W, D]            residual stream before the final norm            */
   float* top_logit; /* [S*W]               the winning logit of every block row             */
+  float* carry_mass;/* [Ld][S, W, n_q]     share of each query's softmax mass that falls on the
+                                           carried rows U_l (the diagnostic of Appendix C)  */
 } cod_taps;
 
 /* Creates a context on the CURRENT CUDA device and allocates its workspace.
@@ -229,6 +231,15 @@ int cod_draft_round(cod_ctx* ctx, const int32_t* draft, const int32_t* target, c
 /* Copies the sticky device status word to *dev_flags (host) after synchronising the stream;
    clear != 0 also resets it. */
 int cod_poll_status(cod_ctx* ctx, uint32_t* dev_flags, int clear, cod_stream_t stream);
+
+/* Analysis aid — the re-convergence count R of Section 5.2 (the equation defining R), one per
+   sequence: R[s] = #{ q in [0, len[s]) : z[s, q+d] == y[s, q] for some d in {-1, 0, +1} with
+   0 <= q+d < len[s] }.  z [S, W] device int32: the verifier's top-1 next-token prediction from the
+   q-th rejected state; y [S, W] device int32: the token eventually committed at the position that
+   prediction refers to; len [S] device int32: rejected suffix length (clamped to [0, W]);
+   R [S] device int32. W = cfg.block. It selects nothing and feeds nothing back (as in the paper). */
+int cod_reconvergence_count(cod_ctx* ctx, const int32_t* z, const int32_t* y, const int32_t* len, int S,
+                            int32_t* R, cod_stream_t stream);
 
 /* Kernel classes for the optional per-kernel timing below. */
 enum cod_kernel_class {

@@ -25,7 +25,7 @@ DEV_BAD_TOKEN, DEV_PAGE_OVERFLOW, DEV_BAD_PAGE, DEV_TIMEOUT, DEV_BAD_LEN = 1, 2,
 
 EXPORTS = ("cod_create", "cod_destroy", "cod_set_weights", "cod_verify_accept", "cod_project_kv",
            "cod_scatter_kv", "cod_block_attn", "cod_lm_head_argmax", "cod_lm_head_argmax_static",
-           "cod_draft_round",
+           "cod_draft_round", "cod_reconvergence_count",
            "cod_poll_status", "cod_profile_enable", "cod_profile_read", "cod_launch_count",
            "cod_workspace_bytes", "cod_error_string")
 KERNEL_CLASSES = ("verify", "fc", "kv", "qkv", "attn", "oproj", "lmhead", "rowops", "mlp")
@@ -44,7 +44,7 @@ _WEIGHT_FIELDS = ("fc", "e_carry", "g_hidden", "wk", "wv", "wq", "wo", "g_attn",
 _SPLIT_FIELDS = ("accept_len", "bonus", "row_pos", "commit_slot", "carry_slot", "acc_rows", "acc_off",
                  "rej_rows", "rej_off")
 _STATE_FIELDS = ("kv_pool", "block_table", "committed_len", "carry_kv", "carry_len")
-_TAP_FIELDS = ("z", "attn_out", "x_final", "top_logit")
+_TAP_FIELDS = ("z", "attn_out", "x_final", "top_logit", "carry_mass")
 
 
 class CodWeights(C.Structure):
@@ -79,6 +79,7 @@ def load_library() -> C.CDLL:
     lib.cod_lm_head_argmax_static.argtypes = [vp, vp, vp, i32, i32, i32, i32, C.c_float, vp, vp, vp]
     lib.cod_draft_round.argtypes = [vp, vp, vp, vp, i32, i32, i32, C.POINTER(CodState), C.POINTER(CodSplit),
                                     vp, C.POINTER(CodTaps), vp]
+    lib.cod_reconvergence_count.argtypes = [vp, vp, vp, vp, i32, vp, vp]
     lib.cod_poll_status.argtypes = [vp, C.POINTER(C.c_uint32), i32, vp]
     lib.cod_profile_enable.argtypes = [vp, C.c_uint32]
     lib.cod_profile_read.argtypes = [vp, i32, C.POINTER(C.c_float), C.POINTER(C.c_int32)]
@@ -183,6 +184,7 @@ class Taps:
         self.attn_out = torch.zeros((cfg.n_layers, R, cfg.n_q_heads * cfg.head_dim), **f32)
         self.x_final = torch.zeros((R, cfg.d_model), **f32)
         self.top_logit = torch.zeros(R, **f32)
+        self.carry_mass = torch.zeros((cfg.n_layers, S, cfg.block, cfg.n_q_heads), **f32)
 
     def struct(self) -> CodTaps:
         return CodTaps(*[_ptr(getattr(self, n)) for n in _TAP_FIELDS])
@@ -251,6 +253,10 @@ class Context:
             self._h, _ptr(draft), _ptr(target), _ptr(H), S, n_forced, mode, C.byref(st),
             C.byref(sp) if sp is not None else None, _ptr(next_draft),
             C.byref(tp) if tp is not None else None, _stream()))
+
+    def reconvergence_count(self, z, y, length, S, out) -> None:
+        _check("cod_reconvergence_count", lib().cod_reconvergence_count(
+            self._h, _ptr(z), _ptr(y), _ptr(length), S, _ptr(out), _stream()))
 
     # ---- bookkeeping
     def poll_status(self, clear: bool = True) -> int:

@@ -368,7 +368,8 @@ int cod_draft_round(cod_ctx* c, const int32_t* draft, const int32_t* target, con
     if ((rc = cod_launch_qkv_finish(c, c->gemm_out, g.splits, R, l, s)) != COD_OK) return rc;
 
     float* tap_o = (taps && taps->attn_out) ? taps->attn_out + static_cast<size_t>(l) * R * c->qw : nullptr;
-    if ((rc = cod_launch_attn(c, l, c->q, c->kb, c->vb, st, S, mode == COD_CARRY ? 1 : 0, c->o, tap_o, nullptr, s)) != COD_OK)
+    float* tap_m = (taps && taps->carry_mass) ? taps->carry_mass + static_cast<size_t>(l) * R * f.n_q_heads : nullptr;
+    if ((rc = cod_launch_attn(c, l, c->q, c->kb, c->vb, st, S, mode == COD_CARRY ? 1 : 0, c->o, tap_o, tap_m, s)) != COD_OK)
       return rc;
 
     GemmArgs o{};
@@ -409,6 +410,14 @@ int cod_draft_round(cod_ctx* c, const int32_t* draft, const int32_t* target, con
   // part 5
   if ((rc = lm_head_impl(c, R, s)) != COD_OK) return rc;
   return cod_launch_finalize(c, R, f.block, sp->bonus, c->tok, next_draft, taps ? taps->top_logit : nullptr, s);
+}
+
+int cod_reconvergence_count(cod_ctx* c, const int32_t* z, const int32_t* y, const int32_t* len, int S,
+                            int32_t* R, cod_stream_t stream) {
+  if (!c || !z || !y || !len || !R) return COD_ERR_INVALID_ARG;
+  if (check_S(c, S) != COD_OK) return COD_ERR_INVALID_ARG;
+  c->pdl = true;
+  return cod_launch_reconvergence(c, z, y, len, S, R, static_cast<cudaStream_t>(stream));
 }
 
 int cod_poll_status(cod_ctx* c, uint32_t* dev_flags, int clear, cod_stream_t stream) {

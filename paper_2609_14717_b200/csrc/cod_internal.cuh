@@ -209,6 +209,8 @@ int cod_launch_attn_simt(cod_ctx* c, int layer, const void* q, const void* kb, c
                          const cod_state* stt, int S, int use_carry, void* out, float* tap, float* mass,
                          cudaStream_t st);
 // cos/sin tables of the block rows only, at positions committed_len[s] + i
+int cod_launch_reconvergence(cod_ctx* c, const int32_t* z, const int32_t* y, const int32_t* len, int S,
+                             int32_t* R, cudaStream_t st);
 int cod_launch_rope_blk_only(cod_ctx* c, const int32_t* committed_len, int S, cudaStream_t st);
 int cod_launch_fcE(cod_ctx* c, cudaStream_t st);
 int cod_launch_gather_rows(cod_ctx* c, const void* src, const int* rows, const int* n_dev, int n_max, int width,

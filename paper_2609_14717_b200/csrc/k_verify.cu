@@ -141,3 +141,31 @@ int cod_launch_rope_blk_only(cod_ctx* c, const int32_t* committed_len, int S, cu
   COD_CHECK_LAUNCH(c);
   return COD_OK;
 }
+
+// Re-convergence count of Section 5.2: one warp per sequence, a lane per rejected position.
+__global__ void k_reconvergence(const int32_t* __restrict__ z, const int32_t* __restrict__ y,
+                                const int32_t* __restrict__ len, int S, int W, int32_t* __restrict__ R) {
+  cod_pdl_prologue();
+  const int s = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5), lane = threadIdx.x & 31;
+  if (s >= S) return;
+  const int L = min(max(len[s], 0), W);
+  int cnt = 0;
+  for (int q = lane; q < L; q += 32) {
+    const int t = y[s * W + q];
+    bool hit = z[s * W + q] == t;
+    if (q > 0) hit = hit || z[s * W + q - 1] == t;
+    if (q + 1 < L) hit = hit || z[s * W + q + 1] == t;
+    cnt += hit ? 1 : 0;
+  }
+  for (int o = 16; o >= 1; o >>= 1) cnt += __shfl_xor_sync(0xffffffffu, cnt, o);
+  if (lane == 0) R[s] = cnt;
+}
+
+int cod_launch_reconvergence(cod_ctx* c, const int32_t* z, const int32_t* y, const int32_t* len, int S,
+                             int32_t* R, cudaStream_t st) {
+  ProfScope prof(c, COD_K_VERIFY, st);
+  cod_launch_pdl(c, k_reconvergence, (S + 3) / 4, 128, 0, st, z, y, len, S, c->cfg.block, R);
+  COD_CHECK_LAUNCH(c);
+  return COD_OK;
+}
+

@@ -294,6 +294,8 @@ def _check_round(P, res_o, L0, tol):
     for l in range(sh.n_layers):
         assert rel_err(P.taps.attn_out[l].cpu().numpy(), res_o["attn_out"][l]) <= tol
     assert rel_err(P.taps.x_final.cpu().numpy(), res_o["x_final"]) <= tol
+    # share of attention on the carried rows (a probability: absolute difference)
+    assert np.max(np.abs(P.taps.carry_mass.cpu().numpy() - res_o["carry_mass"])) <= tol
     nd = P.next_draft.cpu().numpy()
     assert np.array_equal(nd[:, 0], res_o["split"]["bonus"])
     sure = res_o["gap"] >= Hn.GAP
@@ -425,3 +427,25 @@ def test_status_word_and_argument_errors():
         B.Context(cfg)
     assert e.value.status == -2
     P.close()
+
+
+def test_reconvergence_count_bit_exact():
+    """Random suffixes over a small alphabet (many coincidences), every length 0..W, W = 16 and 32."""
+    B = _B()
+    Hn = _H()
+    for W, S in ((16, 40), (32, 7)):
+        wl = small_bf16(S=1, W=W, n_layers=1)
+        ctx = B.Context(B.make_config(wl.shape, S, 4, 8))
+        rng = np.random.default_rng(W)
+        z = rng.integers(0, 4, size=(S, W)).astype(np.int32)
+        y = rng.integers(0, 4, size=(S, W)).astype(np.int32)
+        y[::3] = np.roll(z[::3], 1, axis=1)                       # shifted copies: the +-1 tolerance at work
+        length = (np.arange(S) % (W + 1)).astype(np.int32)
+        out = torch.full((S,), -1, dtype=torch.int32, device="cuda")
+        ctx.reconvergence_count(Hn.dev_i32(z), Hn.dev_i32(y), Hn.dev_i32(length), S, out)
+        torch.cuda.synchronize()
+        want = orc.reconvergence_count(z, y, length)
+        assert np.array_equal(out.cpu().numpy(), want)
+        assert want.max() > 3 and want.min() == 0
+        ctx.close()
+
