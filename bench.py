@@ -4,10 +4,12 @@ K/V projection with E_carry, scatter, block attention in every drafter layer, LM
 
     python bench.py --gpus 1 --steps 64 --warmup 3            # batch-1 configuration (default)
     python bench.py --workload cfg3                           # batch 32
+    python bench.py --workload cfg2f                          # batch 1, complete drafter layer (MLP, q/k norm)
     python bench.py --impl reference                          # the CPU oracle on the host cores
 
-Prints ONE JSON line.  Inputs are seeded and synthetic (see the design doc for the recipe); the
-weights (about 2 GB) are re-read from HBM every round, so no L2 flush is needed between steps.
+Prints ONE JSON line.  Inputs are seeded and synthetic (the recipe is in the docstrings of
+paper_2609_14717_b200/synth.py: weights ~ N(0, 0.02), hidden states with a per-layer RMS ramp,
+randomly permuted page tables, geometric acceptance lengths); the weights (about 2 GB) are re-read from HBM every round, so no L2 flush is needed between steps.
 With N > 1 (torchrun) every rank runs an independent replica: the round has no exchange step.
 """
 from __future__ import annotations

@@ -2,7 +2,7 @@
 
 A plain, slow, float64 numpy statement of what the round computes, written from
 the paper (Section 2 "Carryover Drafting", Eq. 1, Eq. 2; Appendix A, Algorithm 1
-and its "Cache semantics" paragraph).  It exists to judge the CUDA library; it
+and its "Cache semantics" paragraph).  It exists to check the CUDA library; it
 shares no code with it and is never on the product path: only the tests, the
 smoke check and the benchmark's CPU-baseline leg may import it.
 
