@@ -150,6 +150,34 @@ def verify_accept(draft: np.ndarray, target: np.ndarray, committed_len: np.ndarr
     }
 
 
+def verify_accept_stochastic(p_tok: np.ndarray, q_tok: np.ndarray, u: np.ndarray, target: np.ndarray,
+                             committed_len: np.ndarray, block_table: np.ndarray, page: int,
+                             n_forced: int) -> Dict[str, np.ndarray]:
+    """Speculative-sampling verification (Appendix A, "Why verification remains valid": the usual
+    target acceptance and residual correction applied with the drafter's actual proposal
+    distribution q).
+
+    Row p of the window is accepted with probability min(1, P(x_p) / Q(x_p)), x_p the drafted
+    token, and acceptance is again a PREFIX rule: the first rejected row ends it.  Inputs are the two
+    probabilities of the drafted token and a uniform number per row; the decision is
+    u * q < p, taken in float32 (one rounded product and a comparison, so every implementation
+    takes the same decision).  target[s, m] is the token the target's sampler supplies after the
+    accepted prefix: drawn from the residual norm(max(0, P - Q)) at the first rejected row, or
+    from P after a fully accepted window.  Everything downstream (row split, slots) is as in
+    verify_accept.
+    """
+    p32 = np.asarray(p_tok, dtype=np.float32)
+    q32 = np.asarray(q_tok, dtype=np.float32)
+    u32 = np.asarray(u, dtype=np.float32)
+    S, W = p32.shape
+    ok = (u32 * q32) < p32                       # float32 product, rounded once
+    # express the rule through the greedy routine: a window whose "draft" equals the "target"
+    # exactly on the rows the coin accepted
+    fake_target = np.array(target, dtype=np.int64)
+    fake_draft = np.where(ok, fake_target[:, :W], fake_target[:, :W] + 1)
+    return verify_accept(fake_draft, fake_target, committed_len, block_table, page, n_forced)
+
+
 # =========================================================================== shared pieces
 def rope(x: np.ndarray, pos, theta: float) -> np.ndarray:
     """Rotate-half rotary embedding of x[..., hd] at absolute position(s) pos.

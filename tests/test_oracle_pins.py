@@ -745,3 +745,51 @@ def test_reconvergence_against_a_set_formulation_exhaustive():
             want = sum(1 for q in range(L) if yt[q] in {zt[j] for j in range(max(0, q - 1), min(L, q + 2))})
             assert int(orc.reconvergence_count(zz, np.array([yt]), np.array([L]))[0]) == want
 
+
+# ----------------------------------------------------------------------------- stochastic verification
+def test_stochastic_accept_rule_by_hand_and_limits():
+    W, page = 4, 16
+    bt = np.arange(8).reshape(1, 8)
+    L = np.array([5])
+    tgt = np.array([[10, 11, 12, 13, 14]])
+    run = lambda p, q, u, nf=0: orc.verify_accept_stochastic(np.array([p]), np.array([q]), np.array([u]), tgt, L, bt, page, nf)
+    # p >= q: always accepted whatever u in [0, 1)
+    r = run([0.5, 0.5, 0.5, 0.5], [0.5, 0.4, 0.1, 0.5], [0.999, 0.999, 0.999, 0.999])
+    assert r["accept_len"][0] == 4 and r["bonus"][0] == 14
+    # row 2: p/q = 0.25, u = 0.3 -> rejected; later rows do not count even though they would pass
+    r = run([0.5, 0.5, 0.1, 0.9], [0.5, 0.5, 0.4, 0.1], [0.0, 0.9, 0.3, 0.0])
+    assert r["accept_len"][0] == 2 and r["bonus"][0] == 12
+    assert r["carry_slot"].tolist() == [-1, -1, 0, 1] and r["commit_slot"].tolist() == [5, 6, -1, -1]
+    # same row with u = 0.2 < 0.25 -> accepted
+    r = run([0.5, 0.5, 0.1, 0.9], [0.5, 0.5, 0.4, 0.1], [0.0, 0.9, 0.2, 0.0])
+    assert r["accept_len"][0] == 4
+    # p = 0 is never accepted (u * q < 0 is false), unless the row is the forced anchor
+    assert run([0.0, 1, 1, 1], [0.3, 1, 1, 1], [0.0, 0, 0, 0])["accept_len"][0] == 0
+    assert run([0.0, 1, 1, 1], [0.3, 1, 1, 1], [0.0, 0, 0, 0], nf=1)["accept_len"][0] == 4
+
+
+def test_stochastic_acceptance_frequency_is_min_1_p_over_q():
+    """Over many uniform draws a one-row window is accepted with frequency min(1, p/q)."""
+    rng = np.random.default_rng(0)
+    n = 40000
+    bt = np.zeros((n, 2), dtype=np.int64)
+    tgt = np.zeros((n, 2), dtype=np.int64)
+    for p, q in ((0.2, 0.8), (0.6, 0.3), (0.05, 0.5)):
+        u = rng.random((n, 1), dtype=np.float32)
+        r = orc.verify_accept_stochastic(np.full((n, 1), p), np.full((n, 1), q), u, tgt, np.zeros(n, dtype=int), bt, 16, 0)
+        freq = r["accept_len"].mean()
+        assert abs(freq - min(1.0, p / q)) < 4 * math.sqrt(0.25 / n)
+
+
+def test_stochastic_rule_with_degenerate_probabilities_is_the_greedy_rule():
+    """p in {0, 1} with q = 1: the coin never matters and the rule is 'draft equals target'."""
+    wl = synth.scaled(synth.workload("cfg1"), S=6, ctx=(10, 50))
+    lay = synth.make_layout(wl, 3)
+    rd = synth.make_round(wl, 3, 0)
+    match = (rd["draft"] == rd["target"][:, :wl.shape.W]).astype(np.float32)
+    u = np.random.default_rng(1).random(match.shape, dtype=np.float32)
+    a = orc.verify_accept_stochastic(match, np.ones_like(match), u, rd["target"], lay["committed_len"], lay["block_table"], 16, 1)
+    b = orc.verify_accept(rd["draft"], rd["target"], lay["committed_len"], lay["block_table"], 16, 1)
+    for k in b:
+        assert np.array_equal(a[k], b[k])
+
