@@ -169,6 +169,20 @@ int cod_set_weights(cod_ctx* ctx, const cod_weights* w, cod_stream_t stream);
 int cod_verify_accept(cod_ctx* ctx, const int32_t* draft, const int32_t* target, int S,
                       int n_forced, const cod_state* st, cod_split* out, cod_stream_t stream);
 
+/* Part 1 at temperature 1 — speculative-sampling verification (Appendix A, "Why verification
+   remains valid": the usual target acceptance and residual correction, applied with the drafter's
+   actual proposal distribution q). Row p is accepted while u[s,p] * q_tok[s,p] < p_tok[s,p]
+   (float32: one rounded product, then the comparison), i.e. with probability min(1, P(x)/Q(x)) for
+   the drafted token x; the first n_forced rows are always accepted; the first rejected row ends
+   acceptance. p_tok, q_tok, u [S, W] device float32: target and drafter probability of the drafted
+   token, and a uniform number in [0, 1). target [S, W+1] device int32: target[s, m] is the token the
+   target's sampler supplies after the accepted prefix (drawn from the residual norm(max(0, P - Q)) at
+   the first rejected row, from P after a fully accepted window); the library only reads target[s, m_s].
+   Output and state use are those of cod_verify_accept. */
+int cod_verify_accept_stochastic(cod_ctx* ctx, const int32_t* target, const float* p_tok,
+                                 const float* q_tok, const float* u, int S, int n_forced,
+                                 const cod_state* st, cod_split* out, cod_stream_t stream);
+
 /* Part 2 — J_l = (K_l(Z), V_l(Z)), Z = F(H + [rejected] E_carry) (Eq. 1-2; Algorithm 1).
    H [S*W, D_in] device. J [Ld][S*W][2][n_kv][hd] device; keys rotated (RoPE) at row_pos.
    COD_CARRY writes every row; COD_BASELINE writes accepted rows only and leaves the
@@ -231,6 +245,12 @@ int cod_draft_round(cod_ctx* ctx, const int32_t* draft, const int32_t* target, c
 /* Copies the sticky device status word to *dev_flags (host) after synchronising the stream;
    clear != 0 also resets it. */
 int cod_poll_status(cod_ctx* ctx, uint32_t* dev_flags, int clear, cod_stream_t stream);
+
+/* cod_draft_round with cod_verify_accept_stochastic as its first part; everything else identical. */
+int cod_draft_round_stochastic(cod_ctx* ctx, const int32_t* target, const float* p_tok,
+                               const float* q_tok, const float* u, const void* H, int S, int n_forced,
+                               int mode, cod_state* st, cod_split* split_out, int32_t* next_draft,
+                               const cod_taps* taps, cod_stream_t stream);
 
 /* Analysis aid — the re-convergence count R of Section 5.2 (the equation defining R), one per
    sequence: R[s] = #{ q in [0, len[s]) : z[s, q+d] == y[s, q] for some d in {-1, 0, +1} with

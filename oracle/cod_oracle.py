@@ -390,6 +390,22 @@ def draft_round(draft: np.ndarray, target: np.ndarray, H: np.ndarray, st: Oracle
     return res
 
 
+def draft_round_stochastic(target: np.ndarray, p_tok: np.ndarray, q_tok: np.ndarray, u: np.ndarray,
+                           H: np.ndarray, st: OracleState, w: Dict[str, np.ndarray], n_forced: int,
+                           mode: int) -> Dict[str, np.ndarray]:
+    """draft_round with speculative-sampling verification as its first step (Appendix A, "Why
+    verification remains valid": Carryover changes the proposal distribution, not the rule)."""
+    cfg = st.cfg
+    split = verify_accept_stochastic(p_tok, q_tok, u, target, st.committed_len, st.block_table, cfg.page, n_forced)
+    J = project_kv(H, split, w, cfg, mode)
+    scatter_kv(J, split, st, mode)
+    res = draft_block(st, split["bonus"], w, use_carry=(mode == MODE_CARRY))
+    next_draft = res["tok"].copy()
+    next_draft[:, 0] = split["bonus"]
+    res.update(split=split, J=J, next_draft=next_draft.astype(np.int32))
+    return res
+
+
 # =========================================================================== analysis aids
 def reconvergence_count(z: np.ndarray, y: np.ndarray, length: np.ndarray) -> np.ndarray:
     """Re-convergence count R of Section 5.2 ("Why do gains differ across datasets?", the

@@ -25,7 +25,8 @@ DEV_BAD_TOKEN, DEV_PAGE_OVERFLOW, DEV_BAD_PAGE, DEV_TIMEOUT, DEV_BAD_LEN = 1, 2,
 
 EXPORTS = ("cod_create", "cod_destroy", "cod_set_weights", "cod_verify_accept", "cod_project_kv",
            "cod_scatter_kv", "cod_block_attn", "cod_lm_head_argmax", "cod_lm_head_argmax_static",
-           "cod_draft_round", "cod_reconvergence_count",
+           "cod_draft_round", "cod_reconvergence_count", "cod_verify_accept_stochastic",
+           "cod_draft_round_stochastic",
            "cod_poll_status", "cod_profile_enable", "cod_profile_read", "cod_launch_count",
            "cod_workspace_bytes", "cod_error_string")
 KERNEL_CLASSES = ("verify", "fc", "kv", "qkv", "attn", "oproj", "lmhead", "rowops", "mlp")
@@ -80,6 +81,9 @@ def load_library() -> C.CDLL:
     lib.cod_draft_round.argtypes = [vp, vp, vp, vp, i32, i32, i32, C.POINTER(CodState), C.POINTER(CodSplit),
                                     vp, C.POINTER(CodTaps), vp]
     lib.cod_reconvergence_count.argtypes = [vp, vp, vp, vp, i32, vp, vp]
+    lib.cod_verify_accept_stochastic.argtypes = [vp, vp, vp, vp, vp, i32, i32, C.POINTER(CodState), C.POINTER(CodSplit), vp]
+    lib.cod_draft_round_stochastic.argtypes = [vp, vp, vp, vp, vp, vp, i32, i32, i32, C.POINTER(CodState),
+                                               C.POINTER(CodSplit), vp, C.POINTER(CodTaps), vp]
     lib.cod_poll_status.argtypes = [vp, C.POINTER(C.c_uint32), i32, vp]
     lib.cod_profile_enable.argtypes = [vp, C.c_uint32]
     lib.cod_profile_read.argtypes = [vp, i32, C.POINTER(C.c_float), C.POINTER(C.c_int32)]
@@ -251,6 +255,21 @@ class Context:
         tp = taps.struct() if taps is not None else None
         _check("cod_draft_round", lib().cod_draft_round(
             self._h, _ptr(draft), _ptr(target), _ptr(H), S, n_forced, mode, C.byref(st),
+            C.byref(sp) if sp is not None else None, _ptr(next_draft),
+            C.byref(tp) if tp is not None else None, _stream()))
+
+    def verify_accept_stochastic(self, target, p_tok, q_tok, u, S, n_forced, state: State, split: Split) -> None:
+        st, sp = state.struct(), split.struct()
+        _check("cod_verify_accept_stochastic", lib().cod_verify_accept_stochastic(
+            self._h, _ptr(target), _ptr(p_tok), _ptr(q_tok), _ptr(u), S, n_forced, C.byref(st), C.byref(sp), _stream()))
+
+    def draft_round_stochastic(self, target, p_tok, q_tok, u, H, S, n_forced, mode, state: State,
+                               split: Optional[Split], next_draft, taps: Optional[Taps] = None) -> None:
+        st = state.struct()
+        sp = split.struct() if split is not None else None
+        tp = taps.struct() if taps is not None else None
+        _check("cod_draft_round_stochastic", lib().cod_draft_round_stochastic(
+            self._h, _ptr(target), _ptr(p_tok), _ptr(q_tok), _ptr(u), _ptr(H), S, n_forced, mode, C.byref(st),
             C.byref(sp) if sp is not None else None, _ptr(next_draft),
             C.byref(tp) if tp is not None else None, _stream()))
 

@@ -242,6 +242,16 @@ int cod_verify_accept(cod_ctx* c, const int32_t* draft, const int32_t* target, i
   return cod_launch_verify(c, draft, target, S, n_forced, st, out, static_cast<cudaStream_t>(stream));
 }
 
+int cod_verify_accept_stochastic(cod_ctx* c, const int32_t* target, const float* p_tok, const float* q_tok,
+                                 const float* u, int S, int n_forced, const cod_state* st, cod_split* out,
+                                 cod_stream_t stream) {
+  if (!c || !target || !p_tok || !q_tok || !u || !st || !st->committed_len || !st->block_table || split_has_null(out))
+    return COD_ERR_INVALID_ARG;
+  if (check_S(c, S) != COD_OK || n_forced < 0 || n_forced > 1) return COD_ERR_INVALID_ARG;
+  c->pdl = true;
+  return cod_launch_verify(c, nullptr, target, S, n_forced, st, out, static_cast<cudaStream_t>(stream), p_tok, q_tok, u);
+}
+
 // fc and K/V contractions of the kept rows; the finish kernel writes J or the state.
 static int project_impl(cod_ctx* c, const void* H, const cod_split* sp, int S, int mode, void* J,
                         const cod_state* dest, float* tap_z, cudaStream_t st) {
@@ -332,10 +342,13 @@ int cod_lm_head_argmax(cod_ctx* c, const float* x, int n_rows, int32_t* tok, flo
   return cod_launch_finalize(c, n_rows, 1, nullptr, tok, nullptr, top_logit, s);
 }
 
-int cod_draft_round(cod_ctx* c, const int32_t* draft, const int32_t* target, const void* H, int S,
-                    int n_forced, int mode, cod_state* st, cod_split* split_out, int32_t* next_draft,
-                    const cod_taps* taps, cod_stream_t stream) {
-  if (!c || !draft || !target || !H || !next_draft || state_has_null(st)) return COD_ERR_INVALID_ARG;
+static int round_impl(cod_ctx* c, const int32_t* draft, const int32_t* target, const float* p_tok,
+                      const float* q_tok, const float* u, const void* H, int S, int n_forced, int mode,
+                      cod_state* st, cod_split* split_out, int32_t* next_draft, const cod_taps* taps,
+                      cod_stream_t stream) {
+  const bool stochastic = p_tok != nullptr;
+  if (!c || (!stochastic && !draft) || !target || !H || !next_draft || state_has_null(st)) return COD_ERR_INVALID_ARG;
+  if (stochastic && (!q_tok || !u)) return COD_ERR_INVALID_ARG;
   if (misaligned(H) || misaligned(st->kv_pool) || misaligned(st->carry_kv)) return COD_ERR_INVALID_ARG;
   if (split_out && split_has_null(split_out)) return COD_ERR_INVALID_ARG;
   if (check_S(c, S) != COD_OK || n_forced < 0 || n_forced > 1) return COD_ERR_INVALID_ARG;
@@ -350,7 +363,7 @@ int cod_draft_round(cod_ctx* c, const int32_t* draft, const int32_t* target, con
   c->pdl = true;
 
   // parts 1-3
-  if ((rc = cod_launch_verify(c, draft, target, S, n_forced, st, sp, s)) != COD_OK) return rc;
+  if ((rc = cod_launch_verify(c, draft, target, S, n_forced, st, sp, s, p_tok, q_tok, u)) != COD_OK) return rc;
   if ((rc = project_impl(c, H, sp, S, mode, nullptr, st, taps ? taps->z : nullptr, s)) != COD_OK) return rc;
   if ((rc = cod_launch_update_lens(c, sp, S, mode, st, s)) != COD_OK) return rc;
 
@@ -410,6 +423,21 @@ int cod_draft_round(cod_ctx* c, const int32_t* draft, const int32_t* target, con
   // part 5
   if ((rc = lm_head_impl(c, R, s)) != COD_OK) return rc;
   return cod_launch_finalize(c, R, f.block, sp->bonus, c->tok, next_draft, taps ? taps->top_logit : nullptr, s);
+}
+
+int cod_draft_round(cod_ctx* c, const int32_t* draft, const int32_t* target, const void* H, int S,
+                    int n_forced, int mode, cod_state* st, cod_split* split_out, int32_t* next_draft,
+                    const cod_taps* taps, cod_stream_t stream) {
+  if (!draft) return COD_ERR_INVALID_ARG;
+  return round_impl(c, draft, target, nullptr, nullptr, nullptr, H, S, n_forced, mode, st, split_out, next_draft, taps, stream);
+}
+
+int cod_draft_round_stochastic(cod_ctx* c, const int32_t* target, const float* p_tok, const float* q_tok,
+                               const float* u, const void* H, int S, int n_forced, int mode, cod_state* st,
+                               cod_split* split_out, int32_t* next_draft, const cod_taps* taps,
+                               cod_stream_t stream) {
+  if (!p_tok || !q_tok || !u) return COD_ERR_INVALID_ARG;
+  return round_impl(c, nullptr, target, p_tok, q_tok, u, H, S, n_forced, mode, st, split_out, next_draft, taps, stream);
 }
 
 int cod_reconvergence_count(cod_ctx* c, const int32_t* z, const int32_t* y, const int32_t* len, int S,

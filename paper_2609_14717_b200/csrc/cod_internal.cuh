@@ -189,8 +189,10 @@ inline cudaError_t cod_launch_pdl(const cod_ctx* c, void (*kernel)(KArgs...), di
 
 // ---------------------------------------------------------------------------- launchers
 // Every launcher enqueues on `st`, bumps ctx->launches, and returns a cod_status.
+// p_tok / q_tok / u all null: greedy rule (draft == target); all non-null: speculative sampling (draft unused)
 int cod_launch_verify(cod_ctx* c, const int32_t* draft, const int32_t* target, int S, int n_forced,
-                      const cod_state* state, const cod_split* out, cudaStream_t st);
+                      const cod_state* state, const cod_split* out, cudaStream_t st, const float* p_tok = nullptr,
+                      const float* q_tok = nullptr, const float* u = nullptr);
 int cod_launch_gemm(cod_ctx* c, const GemmArgs& g, cudaStream_t st);
 int cod_launch_gemm_simt(cod_ctx* c, const GemmArgs& g, cudaStream_t st);
 bool cod_gemm_tc_supported(const cod_ctx* c, const GemmArgs& g);

@@ -10,7 +10,8 @@ __global__ void __launch_bounds__(1024)
 k_verify_accept(const int32_t* __restrict__ draft, const int32_t* __restrict__ target, int S, int W,
                 int n_forced, int vocab, int page, int max_pages, int n_pages,
                 const int32_t* __restrict__ committed_len, const int32_t* __restrict__ block_table,
-                cod_split out, uint32_t* status) {
+                cod_split out, uint32_t* status, const float* __restrict__ p_tok,
+                const float* __restrict__ q_tok, const float* __restrict__ u) {
   cod_pdl_prologue();
   extern __shared__ int sm[];
   int* s_m = sm;              // [S]
@@ -24,9 +25,13 @@ k_verify_accept(const int32_t* __restrict__ draft, const int32_t* __restrict__ t
       const int p = p0 + lane;
       bool ok = true;
       if (p < W) {
-        const int d = draft[s * W + p], t = target[s * (W + 1) + p];
-        if (d < 0 || d >= vocab || t < 0 || t >= vocab) flags |= COD_DEV_BAD_TOKEN;
-        ok = (p < n_forced) || (d == t);
+        if (p_tok == nullptr) {                       // greedy: the drafted token is the target's token
+          const int d = draft[s * W + p], t = target[s * (W + 1) + p];
+          if (d < 0 || d >= vocab || t < 0 || t >= vocab) flags |= COD_DEV_BAD_TOKEN;
+          ok = (p < n_forced) || (d == t);
+        } else {                                      // speculative sampling: accept with probability min(1, P/Q)
+          ok = (p < n_forced) || (__fmul_rn(u[s * W + p], q_tok[s * W + p]) < p_tok[s * W + p]);
+        }
       }
       const unsigned miss = __ballot_sync(0xffffffffu, !ok);
       if (miss) m = p0 + __ffs(miss) - 1;
@@ -120,13 +125,14 @@ __global__ void k_rope_tables(const int32_t* __restrict__ committed_len, const i
 }
 
 int cod_launch_verify(cod_ctx* c, const int32_t* draft, const int32_t* target, int S, int n_forced,
-                      const cod_state* state, const cod_split* out, cudaStream_t st) {
+                      const cod_state* state, const cod_split* out, cudaStream_t st, const float* p_tok,
+                      const float* q_tok, const float* u) {
   ProfScope prof(c, COD_K_VERIFY, st);
   const int W = c->cfg.block;
   const size_t smem = static_cast<size_t>(2 * S + 2) * sizeof(int);
   cod_launch_pdl(c, k_verify_accept, 1, 1024, smem, st, draft, target, S, W, n_forced, c->cfg.vocab, c->cfg.page_size,
                                          c->cfg.max_pages_per_seq, c->cfg.n_pages, state->committed_len,
-                                         state->block_table, *out, c->status);
+                                         state->block_table, *out, c->status, p_tok, q_tok, u);
   COD_CHECK_LAUNCH(c);
   cod_launch_pdl(c, k_rope_tables, S * W, 64, 0, st, state->committed_len, out->accept_len, c->inv_freq_d, S, W, c->half,
                                       c->rope_win, c->rope_blk);

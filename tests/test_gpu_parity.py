@@ -449,3 +449,60 @@ def test_reconvergence_count_bit_exact():
         assert want.max() > 3 and want.min() == 0
         ctx.close()
 
+
+@pytest.mark.parametrize("W,S", [(16, 32), (32, 5), (8, 64)])
+def test_verify_accept_stochastic_bit_exact(W, S):
+    """u * q < p in float32 on both sides: identical decisions, including p = 0, q = 0, p = q and
+    products that round to the boundary."""
+    B = _B()
+    Hn = _H()
+    wl = small_bf16(S=S, W=W, n_layers=1, ctx=(0, 200))
+    lay = synth.make_layout(wl, 9)
+    ctx = B.Context(B.make_config(wl.shape, S, int(lay["max_pages_per_seq"]), int(lay["n_pages"])))
+    st = B.State(ctx.cfg, "bf16", S, lay["block_table"], lay["committed_len"])
+    sp = B.Split(S, W)
+    rng = np.random.default_rng(W * 100 + S)
+    for n_forced in (0, 1):
+        p = rng.random((S, W), dtype=np.float32)
+        q = rng.random((S, W), dtype=np.float32)
+        u = rng.random((S, W), dtype=np.float32)
+        p[rng.random((S, W)) < 0.5] = 1.0                    # long accepted prefixes too
+        p[0, :] = 0.0; q[1, :] = 0.0; q[2, :] = p[2, :]; u[3, :] = 0.0
+        p[4, :] = (u[4, :] * q[4, :]).astype(np.float32)     # exactly on the boundary: not accepted
+        tgt = rng.integers(0, wl.shape.vocab, size=(S, W + 1)).astype(np.int32)
+        ctx.verify_accept_stochastic(Hn.dev_i32(tgt), torch.from_numpy(p).cuda(), torch.from_numpy(q).cuda(),
+                                     torch.from_numpy(u).cuda(), S, n_forced, st, sp)
+        torch.cuda.synchronize()
+        want = orc.verify_accept_stochastic(p, q, u, tgt, lay["committed_len"], lay["block_table"], wl.shape.page, n_forced)
+        got = sp.to_host()
+        for k, v in want.items():
+            assert np.array_equal(got[k], v), k
+        assert want["accept_len"][4] == n_forced and want["accept_len"].max() > 2
+    assert ctx.poll_status() == 0
+    ctx.close()
+
+
+def test_round_parity_with_stochastic_verification():
+    Hn = _H()
+    B = _B()
+    wl = _workloads()["small_bf16"]
+    P = Hn.Pair(wl, seed=6, attn_split_len=64, wo_scale=30.0, poison=True)
+    rng = np.random.default_rng(12)
+    S, W = wl.S, wl.shape.W
+    ms = set()
+    for r in range(4):
+        rd, dev = P.round_inputs(r)
+        p = rng.random((S, W), dtype=np.float32); q = rng.random((S, W), dtype=np.float32) * 0.6
+        u = rng.random((S, W), dtype=np.float32)
+        L0 = P.st_o.committed_len.copy()
+        res_o = orc.draft_round_stochastic(rd["target"], p, q, u, rd["H"], P.st_o, P.w_o, 1, orc.MODE_CARRY)
+        P.ctx.draft_round_stochastic(dev["target"], torch.from_numpy(p).cuda(), torch.from_numpy(q).cuda(),
+                                     torch.from_numpy(u).cuda(), dev["H"], S, 1, B.COD_CARRY, P.st_g, P.split,
+                                     P.next_draft, P.taps)
+        torch.cuda.synchronize()
+        _check_round(P, res_o, L0, Hn.TOL["bf16"])
+        ms.update(res_o["split"]["accept_len"].tolist())
+    assert len(ms) > 2
+    assert P.ctx.poll_status() == 0
+    P.close()
+
