@@ -341,6 +341,55 @@ def lm_head_argmax(x: np.ndarray, w: Dict[str, np.ndarray], cfg: OracleConfig):
     return tok, gap, logits
 
 
+# --------------------------------------------------------------------------- sampling head
+def counter_uniform(seed: int, step: int, row: np.ndarray, col: np.ndarray) -> np.ndarray:
+    """The counter-based uniform number U(seed, step, row, col) in (0, 1) both sides draw for the
+    Gumbel-max sample of the LM head (the paper fixes no generator; this one is the reading taken).
+
+    A 32-bit integer hash: h = mix(mix(mix(seed_lo ^ K0) + seed_hi) + step) ... of the four counters
+    chained through the 'murmur3 finaliser' mix(x): x ^= x >> 16; x *= 0x85EBCA6B; x ^= x >> 13;
+    x *= 0xC2B2AE35; x ^= x >> 16 (all modulo 2^32).  U = ((h >> 9) + 0.5) * 2^-23 = (2k + 1) / 2^24, exactly
+    representable in float32.
+    """
+    M = np.uint64(0xFFFFFFFF)
+
+    def mix(x):
+        x = x & M
+        x ^= x >> np.uint64(16)
+        x = (x * np.uint64(0x85EBCA6B)) & M
+        x ^= x >> np.uint64(13)
+        x = (x * np.uint64(0xC2B2AE35)) & M
+        x ^= x >> np.uint64(16)
+        return x
+
+    seed = int(seed)
+    h = mix(np.uint64((seed & 0xFFFFFFFF) ^ 0x9E3779B9))
+    h = mix((h + np.uint64((seed >> 32) & 0xFFFFFFFF)) & M)
+    h = mix((h + np.uint64(int(step) & 0xFFFFFFFF)) & M)
+    h = mix((h + np.asarray(row, dtype=np.uint64)) & M)
+    h = mix((h + np.asarray(col, dtype=np.uint64)) & M)
+    return ((h >> np.uint64(9)).astype(np.float64) + 0.5) * 2.0 ** -23
+
+
+def lm_head_sample(x: np.ndarray, w: Dict[str, np.ndarray], cfg: OracleConfig, seed: int, step: int):
+    """A token per row drawn from softmax(N_f(x) Emb^T) by the Gumbel-max rule:
+    tok = argmax_v (logit_v - log(-log U_v)), lowest index on ties, U from counter_uniform with
+    row = the row index and col = the token id.  Returns tok, q_tok = softmax(logits)[tok],
+    the log-sum-exp of the logits and the top-2 gap of the PERTURBED logits (near-ties may
+    legitimately fall either way on another implementation)."""
+    y = rmsnorm(x, w["g_final"], cfg.rms_eps)
+    logits = y @ w["emb"].T
+    R, V = logits.shape
+    U = counter_uniform(seed, step, np.arange(R)[:, None], np.arange(V)[None, :])
+    pert = logits - np.log(-np.log(U))
+    tok = np.argmax(pert, axis=1).astype(np.int32)
+    mx = logits.max(axis=1)
+    lse = mx + np.log(np.exp(logits - mx[:, None]).sum(axis=1))
+    q_tok = np.exp(logits[np.arange(R), tok] - lse)
+    top2 = np.partition(pert, -2, axis=1)[:, -2:]
+    return tok, q_tok, lse, top2[:, 1] - top2[:, 0]
+
+
 # =========================================================================== the drafter pass
 def draft_block(st: OracleState, bonus: np.ndarray, w: Dict[str, np.ndarray],
                 use_carry: bool, keep_logits: bool = False) -> Dict[str, np.ndarray]:

@@ -44,8 +44,6 @@ struct AttnParams {
 };
 
 
-
-
 template <bool DUAL>
 struct Geo {
   static constexpr int TILES = DUAL ? 2 : 1;             // 64-key tiles per iteration
@@ -494,7 +492,6 @@ __global__ void k_attn_tc_combine(const float* __restrict__ part_o, const float*
   if (tap) *reinterpret_cast<float4*>(tap + ob) = make_float4(acc[0] * inv, acc[1] * inv, acc[2] * inv, acc[3] * inv);
   if (mass && lane == 0) mass[item] = lc * inv;
 }
-
 
 
 template <bool DUAL>

@@ -56,14 +56,6 @@ __device__ __forceinline__ bool bar_and_128(bool v) {
 }
 
 
-
-
-
-
-
-
-
-
 __global__ void __launch_bounds__(NTHREADS, 1)
 k_gemm_tc(const __grid_constant__ CUtensorMap map_w0, const __grid_constant__ CUtensorMap map_w1,
           const __grid_constant__ CUtensorMap map_w2, const __grid_constant__ CUtensorMap map_a, const TcParams p) {
@@ -263,7 +255,6 @@ k_gemm_tc(const __grid_constant__ CUtensorMap map_w0, const __grid_constant__ CU
 }
 
 // ------------------------------------------------------------------ host side
-
 
 
 }  // namespace

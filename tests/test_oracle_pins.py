@@ -793,3 +793,57 @@ def test_stochastic_rule_with_degenerate_probabilities_is_the_greedy_rule():
     for k in b:
         assert np.array_equal(a[k], b[k])
 
+
+# ----------------------------------------------------------------------------- sampling head
+def _mix32_py(x):
+    x &= 0xFFFFFFFF
+    x ^= x >> 16; x = (x * 0x85EBCA6B) & 0xFFFFFFFF
+    x ^= x >> 13; x = (x * 0xC2B2AE35) & 0xFFFFFFFF
+    x ^= x >> 16
+    return x
+
+
+def test_counter_uniform_against_plain_python_integers_and_statistics():
+    seed, step = 0x1234567890ABCDEF, 7
+    rows, cols = np.array([[0], [3], [511]]), np.array([[0, 1, 151935, 77777]])
+    U = orc.counter_uniform(seed, step, rows, cols)
+    for i, r in enumerate(rows[:, 0]):
+        for j, c in enumerate(cols[0]):
+            h = _mix32_py((seed & 0xFFFFFFFF) ^ 0x9E3779B9)
+            h = _mix32_py(h + (seed >> 32))
+            h = _mix32_py(h + step)
+            h = _mix32_py(h + int(r))
+            h = _mix32_py(h + int(c))
+            assert U[i, j] == ((h >> 9) + 0.5) / 2 ** 23
+    # the finaliser's published test value: mix(1) = 0x514E28B7
+    assert _mix32_py(1) == 0x514E28B7
+    # open interval, exactly representable in float32, flat histogram, no visible row/column correlation
+    big = orc.counter_uniform(1, 0, np.arange(64)[:, None], np.arange(4096)[None, :])
+    assert big.min() > 0 and big.max() < 1 and np.array_equal(big.astype(np.float32).astype(np.float64), big)
+    hist = np.histogram(big, bins=16, range=(0, 1))[0] / big.size
+    assert np.abs(hist - 1 / 16).max() < 0.004
+    assert abs(np.corrcoef(big[:-1].ravel(), big[1:].ravel())[0, 1]) < 0.01
+    assert abs(np.corrcoef(big[:, :-1].ravel(), big[:, 1:].ravel())[0, 1]) < 0.01
+    assert not np.array_equal(big, orc.counter_uniform(1, 1, np.arange(64)[:, None], np.arange(4096)[None, :]))
+
+
+def test_gumbel_max_sample_follows_the_softmax_and_reports_its_probability():
+    """Draw the same 3 rows over 4000 steps: token frequencies match softmax(logits); q_tok is the
+    softmax probability of the drawn token; lse is the log of the partition sum."""
+    wl = synth.scaled(synth.workload("cfg1"), vocab=12)
+    cfg = oracle_config(wl.shape)
+    w = orc.prepare_weights(synth.make_weights(wl.shape, 2))
+    w["emb"] = w["emb"] * 5.0                        # a peaked but not degenerate distribution
+    x = np.random.default_rng(0).standard_normal((3, cfg.d_model))
+    _, _, logits = orc.lm_head_argmax(x, w, cfg)
+    sm = torch.softmax(torch.from_numpy(logits), dim=1).numpy()
+    counts = np.zeros_like(sm)
+    n = 4000
+    for step in range(n):
+        tok, q, lse, _ = orc.lm_head_sample(x, w, cfg, seed=99, step=step)
+        counts[np.arange(3), tok] += 1
+        assert np.allclose(q, sm[np.arange(3), tok], rtol=1e-12)
+        assert np.allclose(lse, torch.logsumexp(torch.from_numpy(logits), dim=1).numpy(), rtol=1e-12)
+    assert 0.05 < sm.max() < 0.95
+    assert np.abs(counts / n - sm).max() < 4 * math.sqrt(0.25 / n)
+
