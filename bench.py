@@ -510,7 +510,15 @@ def run_micro(args):
         ctx.set_weights(w)
         x = torch.randn(wl.R, sh.d_model, generator=gen, device="cuda")
         tok = torch.zeros(wl.R, dtype=torch.int32, device="cuda")
-        call = lambda: ctx.lm_head_argmax(x, wl.R, tok)
+        if args.micro == "lmsample":      # the Gumbel-max draw fused into the same contraction
+            qv = torch.zeros(wl.R, dtype=torch.float32, device="cuda")
+            step_no = [0]
+
+            def call():
+                step_no[0] += 1
+                ctx.lm_head_sample(x, wl.R, args.seed, step_no[0], tok, qv, None)
+        else:
+            call = lambda: ctx.lm_head_argmax(x, wl.R, tok)
         nbytes = float(sh.vocab * sh.d_model * 2 + wl.R * sh.d_model * 2)
         flops = 2.0 * wl.R * sh.d_model * sh.vocab
     for _ in range(Wm):
@@ -607,7 +615,7 @@ def main():
     ap.add_argument("--no-graph", action="store_true", help="time plain stream launches instead of graph replays")
     ap.add_argument("--sweep", action="store_true", help="carryover-overhead sweep over batch, block and rejected fraction")
     ap.add_argument("--attn-split", type=int, default=0, help="keys per attention split (0 = library default)")
-    ap.add_argument("--micro", default=None, choices=["attn", "lmhead"],
+    ap.add_argument("--micro", default=None, choices=["attn", "lmhead", "lmsample"],
                     help="time one entry point alone (small footprint; meant for profiler captures)")
     args = ap.parse_args()
     if args.warmup < 3:

@@ -214,6 +214,19 @@ int cod_block_attn(cod_ctx* ctx, int layer, const void* q, const void* k_blk, co
 int cod_lm_head_argmax(cod_ctx* ctx, const float* x, int n_rows, int32_t* tok, float* top_logit,
                        cod_stream_t stream);
 
+/* Part 5 at temperature 1 — a token per row DRAWN from softmax(Emb . N_f(x[r])) by the Gumbel-max
+   rule, tok[r] = lowest-index argmax_v (logit_v - log(-log U(seed, step, r, v))), fused into the
+   LM-head contraction like the argmax; logits are never materialised. U is a counter-based uniform
+   number: with mix(x) the 32-bit finaliser (x ^= x >> 16; x *= 0x85EBCA6B; x ^= x >> 13;
+   x *= 0xC2B2AE35; x ^= x >> 16), h = mix(mix(mix(mix(mix(seed_lo ^ 0x9E3779B9) + seed_hi) + step) + r) + v)
+   and U = ((h >> 9) + 0.5) * 2^-23 (the paper fixes no generator; any caller can reproduce this one).
+   q_tok (nullable) [n_rows] device float: the soft-max probability of the drawn token — the
+   proposal probability Q(x) that cod_verify_accept_stochastic wants next round;
+   lse (nullable) [n_rows] device float: log-sum-exp of the row's logits.
+   bf16 contexts on the tensor-core kernels only; otherwise COD_ERR_UNSUPPORTED. */
+int cod_lm_head_sample(cod_ctx* ctx, const float* x, int n_rows, unsigned long long seed, uint32_t step,
+                       int32_t* tok, float* q_tok, float* lse, cod_stream_t stream);
+
 /* The same argmax as cod_lm_head_argmax for callers that may not allocate device memory: it needs
    no cod_ctx and calls no cudaMalloc / cudaFree or any allocating routine. (The paper has no
    counterpart for this entry point; it exists for integration.) Such callers are, for example, a

@@ -371,16 +371,19 @@ def counter_uniform(seed: int, step: int, row: np.ndarray, col: np.ndarray) -> n
     return ((h >> np.uint64(9)).astype(np.float64) + 0.5) * 2.0 ** -23
 
 
-def lm_head_sample(x: np.ndarray, w: Dict[str, np.ndarray], cfg: OracleConfig, seed: int, step: int):
+def lm_head_sample(x: np.ndarray, w: Dict[str, np.ndarray], cfg: OracleConfig, seed: int, step: int,
+                   row_ids: Optional[np.ndarray] = None):
     """A token per row drawn from softmax(N_f(x) Emb^T) by the Gumbel-max rule:
     tok = argmax_v (logit_v - log(-log U_v)), lowest index on ties, U from counter_uniform with
     row = the row index and col = the token id.  Returns tok, q_tok = softmax(logits)[tok],
     the log-sum-exp of the logits and the top-2 gap of the PERTURBED logits (near-ties may
-    legitimately fall either way on another implementation)."""
+    legitimately fall either way on another implementation).  row_ids (default 0..R-1) are the
+    row counters of the noise, for callers that pass a subset of a larger batch's rows."""
     y = rmsnorm(x, w["g_final"], cfg.rms_eps)
     logits = y @ w["emb"].T
     R, V = logits.shape
-    U = counter_uniform(seed, step, np.arange(R)[:, None], np.arange(V)[None, :])
+    rows = np.arange(R) if row_ids is None else np.asarray(row_ids)
+    U = counter_uniform(seed, step, rows[:, None], np.arange(V)[None, :])
     pert = logits - np.log(-np.log(U))
     tok = np.argmax(pert, axis=1).astype(np.int32)
     mx = logits.max(axis=1)

@@ -57,6 +57,7 @@ size_t carve(cod_ctx* c) {
   cv.take(c->attn_o, sizeof(float) * parts * f.head_dim);
   cv.take(c->attn_ml, sizeof(float) * parts * 4);
   cv.take(c->amax, sizeof(unsigned long long) * R);
+  cv.take(c->lse_part, sizeof(float2) * R * ((static_cast<size_t>(f.vocab) + 127) / 128));
   cv.take(c->tok, sizeof(int32_t) * R);
   cv.take(c->sp.accept_len, sizeof(int32_t) * f.max_batch);
   cv.take(c->sp.bonus, sizeof(int32_t) * f.max_batch);
@@ -423,6 +424,25 @@ static int round_impl(cod_ctx* c, const int32_t* draft, const int32_t* target, c
   // part 5
   if ((rc = lm_head_impl(c, R, s)) != COD_OK) return rc;
   return cod_launch_finalize(c, R, f.block, sp->bonus, c->tok, next_draft, taps ? taps->top_logit : nullptr, s);
+}
+
+int cod_lm_head_sample(cod_ctx* c, const float* x, int n_rows, unsigned long long seed, uint32_t step,
+                       int32_t* tok, float* q_tok, float* lse, cod_stream_t stream) {
+  if (!c || !x || !tok || misaligned(x)) return COD_ERR_INVALID_ARG;
+  if (n_rows < 1 || n_rows > c->R_max) return COD_ERR_INVALID_ARG;
+  if (!c->has_weights) return COD_ERR_NO_WEIGHTS;
+  GemmArgs g{};
+  g.A = c->a; g.lda = c->D; g.n_rows = n_rows; g.K = c->D;
+  g.seg[0] = {c->w.emb, c->cfg.vocab}; g.n_seg = 1;
+  g.splits = 1; g.amax = c->amax; g.klass = COD_K_LMHEAD;
+  g.lse_part = c->lse_part; g.sample_state = cod_sample_state(seed, step);
+  if (c->force_simt || !(cod_gemm_tc2_supported(c, g) || cod_gemm_tc_supported(c, g))) return COD_ERR_UNSUPPORTED;
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  c->pdl = true;
+  int rc = cod_launch_resid_norm(c, nullptr, 0, n_rows, const_cast<float*>(x), c->w.g_final, nullptr, s);
+  if (rc != COD_OK) return rc;
+  if ((rc = cod_launch_gemm(c, g, s)) != COD_OK) return rc;
+  return cod_launch_finalize_sample(c, n_rows, g.sample_state, tok, q_tok, lse, s);
 }
 
 int cod_draft_round(cod_ctx* c, const int32_t* draft, const int32_t* target, const void* H, int S,

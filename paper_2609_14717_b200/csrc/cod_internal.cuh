@@ -106,6 +106,10 @@ struct GemmArgs {
   int splits;             // split-K factor (1 = none)
   int n_acc;              // paired kernel: accumulators per CTA pair (1 or 2); 0 = let the launcher choose
   unsigned long long* amax;  // if non-null: per-row packed argmax over N instead of storing C
+  // sampling form of the argmax epilogue (tensor-core kernels only): keys carry logit + Gumbel noise and
+  // every 128-row weight tile also leaves (m, sum exp(logit - m)) per token row in lse_part[tile][n_rows]
+  float2* lse_part;       // null: plain argmax
+  uint32_t sample_state;  // hash state after seed and step
   int klass;              // cod_kernel_class, for the optional timing
 };
 
@@ -134,6 +138,7 @@ struct cod_ctx {
   float* rope_win;             // [R_max][hd]  cos | sin of the window rows' positions
   float* rope_blk;             // [R_max][hd]  cos | sin of the block rows' positions
   void* hmid;                  // [R, d_ff] activated MLP rows (storage type), d_ff > 0 only
+  float2* lse_part;            // [ceil(vocab / 128)][R] soft-max partials of the sampling LM head
   float* gemm_out;             // split-K / unfused GEMM results
   size_t gemm_out_floats;
   void* hc;                    // [R_max, D_in] accepted rows of H packed densely (baseline mode)
@@ -213,6 +218,9 @@ int cod_launch_attn_simt(cod_ctx* c, int layer, const void* q, const void* kb, c
 // cos/sin tables of the block rows only, at positions committed_len[s] + i
 int cod_launch_reconvergence(cod_ctx* c, const int32_t* z, const int32_t* y, const int32_t* len, int S,
                              int32_t* R, cudaStream_t st);
+int cod_launch_finalize_sample(cod_ctx* c, int R, uint32_t state, int32_t* tok, float* q_tok, float* lse,
+                               cudaStream_t st);
+uint32_t cod_sample_state(unsigned long long seed, uint32_t step);   // hash state after seed and step
 int cod_launch_rope_blk_only(cod_ctx* c, const int32_t* committed_len, int S, cudaStream_t st);
 int cod_launch_fcE(cod_ctx* c, cudaStream_t st);
 int cod_launch_gather_rows(cod_ctx* c, const void* src, const int* rows, const int* n_dev, int n_max, int width,

@@ -41,6 +41,8 @@ struct TcParams {
   float* C;
   int ldc;
   unsigned long long* amax;
+  float2* lse_part;           // sampling form of the argmax epilogue (null: plain argmax)
+  uint32_t sample_state;
   uint32_t* status;
 };
 
@@ -202,6 +204,33 @@ k_gemm_tc(const __grid_constant__ CUtensorMap map_w0, const __grid_constant__ CU
           if (f_ok && i < n_rows) C[static_cast<size_t>(i) * p.ldc + col0 + warp * 32 + lane] = __uint_as_float(v[j]);
         }
       }
+    } else if (ok && p.lse_part != nullptr) {
+      // sampling form: Gumbel noise on every logit before the argmax, and soft-max partials per column.
+      // Scratch in the idle pipeline buffers: row states, then per-warp (m, sum) of every column.
+      uint32_t* hrow = reinterpret_cast<uint32_t*>(sm);
+      float* red_m = reinterpret_cast<float*>(sm + 4096);
+      float* red_s = red_m + 4 * 256;
+      for (int t = threadIdx.x; t < 256; t += 128) hrow[t] = mix32(p.sample_state + static_cast<uint32_t>(i0 + t));
+      asm volatile("bar.sync 1, 128;" ::: "memory");
+      for (int c = 0; c < p.NT; c += 32) {
+        uint32_t v[32];
+        if (c + 32 <= p.NT) {
+          tmem_ld32(t_lane + c, v);
+        } else {                                   // NT is a multiple of 16: a last half chunk
+          uint32_t h[16];
+          tmem_ld16(t_lane + c, h);
+#pragma unroll
+          for (int j = 0; j < 16; ++j) { v[j] = h[j]; v[16 + j] = 0xFF800000u; }   // -inf: never wins, adds nothing
+        }
+        unsigned long long best;
+        float m_ref, s_sum;
+        sample_chunk(v, f_ok, static_cast<uint32_t>(col0 + warp * 32 + lane), hrow + c, lane, best, m_ref, s_sum);
+        if (c + lane < p.NT) {
+          red[warp * p.NT + c + lane] = best;
+          red_m[warp * 256 + c + lane] = m_ref;
+          red_s[warp * 256 + c + lane] = s_sum;
+        }
+      }
     } else if (ok) {
       // per-token (max, lowest row) over this warp's 32 weight rows, 32 token columns at a time
       const unsigned long long low = static_cast<unsigned long long>(0xFFFFFFFFu - static_cast<unsigned>(col0 + warp * 32 + lane));
@@ -244,6 +273,18 @@ k_gemm_tc(const __grid_constant__ CUtensorMap map_w0, const __grid_constant__ CU
 #pragma unroll
         for (int w = 1; w < 4; ++w) best = red[w * p.NT + t] > best ? red[w * p.NT + t] : best;
         atomicMax(p.amax + i0 + t, best);
+        if (p.lse_part != nullptr) {                   // this tile's soft-max partial of token row i0 + t
+          const float* red_m = reinterpret_cast<const float*>(sm + 4096);
+          const float* red_s = red_m + 4 * 256;
+          float m = red_m[t];
+#pragma unroll
+          for (int w = 1; w < 4; ++w) m = fmaxf(m, red_m[w * 256 + t]);
+          float sum = 0.f;
+#pragma unroll
+          for (int w = 0; w < 4; ++w)
+            if (red_m[w * 256 + t] > -INFINITY) sum += red_s[w * 256 + t] * __expf(red_m[w * 256 + t] - m);
+          p.lse_part[static_cast<size_t>(col0 / BM) * p.n_rows + i0 + t] = make_float2(m, sum);
+        }
       }
     }
   }
@@ -307,6 +348,8 @@ int cod_launch_gemm_tc(cod_ctx* c, const GemmArgs& g, cudaStream_t st) {
              static_cast<size_t>(stages) * stage_bytes >= 2u * 32u * BM * sizeof(float);
   for (int i = 0; i < g.n_seg; ++i) p.staged = p.staged && (g.seg[i].N % 4 == 0);
   p.amax = g.amax;
+  p.lse_part = g.amax ? g.lse_part : nullptr;
+  p.sample_state = g.sample_state;
   p.status = c->status;
 
   CUtensorMap mw[3], ma;
@@ -328,3 +371,53 @@ int cod_launch_gemm_tc(cod_ctx* c, const GemmArgs& g, cudaStream_t st) {
   COD_CHECK_LAUNCH(c);
   return COD_OK;
 }
+
+// ------------------------------------------------------------------ read-out of the sampling head
+// One warp per token row: merges the per-tile soft-max partials (m_t, s_t) into the log-sum-exp,
+// takes the winning (perturbed logit, index) key, removes the winner's noise again (it is a pure
+// function of seed, step, row and index) and reports q = exp(logit - lse).
+namespace {
+__global__ void k_finalize_sample(const unsigned long long* __restrict__ amax, const float2* __restrict__ lse_part,
+                                  int n_tiles, int R, uint32_t state, int32_t* __restrict__ tok,
+                                  float* __restrict__ q_tok, float* __restrict__ lse_out) {
+  cod_pdl_prologue();
+  const int r = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5), lane = threadIdx.x & 31;
+  if (r >= R) return;
+  float m = -INFINITY, s = 0.f;
+  for (int t = lane; t < n_tiles; t += 32) {
+    const float2 ms = lse_part[static_cast<size_t>(t) * R + r];
+    if (ms.x > -INFINITY) {
+      const float mn = fmaxf(m, ms.x);
+      s = s * __expf(m - mn) + ms.y * __expf(ms.x - mn);      // exp(-inf) = 0 covers the first term
+      m = mn;
+    }
+  }
+  for (int o = 16; o >= 1; o >>= 1) {
+    const float mo = __shfl_xor_sync(0xffffffffu, m, o), so = __shfl_xor_sync(0xffffffffu, s, o);
+    const float mn = fmaxf(m, mo);
+    if (mn > -INFINITY) s = s * __expf(m - mn) + so * __expf(mo - mn);
+    m = mn;
+  }
+  if (lane == 0) {
+    const unsigned long long key = amax[r];
+    const int idx = cod_unpack_index(key);
+    const float pert = tc::order_key_to_float(static_cast<unsigned>(key >> 32));
+    const float raw = pert - tc::gumbel_noise(tc::mix32(state + static_cast<uint32_t>(r)), static_cast<uint32_t>(idx));
+    const float lse = m + logf(s);
+    tok[r] = idx;
+    if (q_tok) q_tok[r] = expf(raw - lse);
+    if (lse_out) lse_out[r] = lse;
+  }
+}
+}  // namespace
+
+int cod_launch_finalize_sample(cod_ctx* c, int R, uint32_t state, int32_t* tok, float* q_tok, float* lse,
+                               cudaStream_t st) {
+  ProfScope prof(c, COD_K_ROWOPS, st);
+  const int n_tiles = (c->cfg.vocab + BM - 1) / BM;
+  cod_launch_pdl(c, k_finalize_sample, (R + 3) / 4, 128, 0, st, c->amax, c->lse_part, n_tiles, R, state, tok, q_tok, lse);
+  COD_CHECK_LAUNCH(c);
+  return COD_OK;
+}
+uint32_t cod_sample_state(unsigned long long seed, uint32_t step) { return tc::sample_state(seed, step); }
+

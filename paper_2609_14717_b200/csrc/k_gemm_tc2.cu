@@ -47,6 +47,8 @@ struct Tc2Params {
   float* C;
   int ldc;
   unsigned long long* amax;
+  float2* lse_part;           // sampling form of the argmax epilogue (null: plain argmax)
+  uint32_t sample_state;
   uint32_t* status;
 };
 
@@ -203,6 +205,25 @@ k_gemm_tc2(const __grid_constant__ CUtensorMap map_w0, const __grid_constant__ C
           if (f_ok && i < n_rows) C[static_cast<size_t>(i) * p.ldc + col0 + qw * 32 + lane] = __uint_as_float(v[j]);
         }
       }
+    } else if (ok && p.lse_part != nullptr) {
+      // sampling form: Gumbel noise on every logit before the argmax, and soft-max partials per column.
+      // Scratch in the idle pipeline buffers: row states, then per-warp (m, sum) of every column.
+      uint32_t* hrow = reinterpret_cast<uint32_t*>(sm);
+      float* red_m = reinterpret_cast<float*>(sm + 4096);
+      float* red_s = red_m + 4 * NTOK;
+      for (int t = c_begin + qw * 32 + lane; t < c_end; t += 128) hrow[t] = mix32(p.sample_state + static_cast<uint32_t>(i0 + t));
+      asm volatile("bar.sync %0, 128;" ::"r"(1 + grp) : "memory");
+      for (int c = c_begin; c < c_end; c += 32) {
+        if (i0 + c >= n_rows) break;
+        uint32_t v[32];
+        tmem_ld32(t_lane + c, v);
+        unsigned long long best;
+        float m_ref, s_sum;
+        sample_chunk(v, f_ok, static_cast<uint32_t>(col0 + qw * 32 + lane), hrow + c, lane, best, m_ref, s_sum);
+        red[qw * NTOK + c + lane] = best;
+        red_m[qw * NTOK + c + lane] = m_ref;
+        red_s[qw * NTOK + c + lane] = s_sum;
+      }
     } else if (ok) {
       const unsigned long long low = static_cast<unsigned long long>(0xFFFFFFFFu - static_cast<unsigned>(col0 + qw * 32 + lane));
       for (int c = c_begin; c < c_end; c += 32) {
@@ -231,6 +252,18 @@ k_gemm_tc2(const __grid_constant__ CUtensorMap map_w0, const __grid_constant__ C
 #pragma unroll
         for (int w = 1; w < 4; ++w) best = red[w * NTOK + t] > best ? red[w * NTOK + t] : best;
         if (best) atomicMax(p.amax + i0 + t, best);
+        if (p.lse_part != nullptr) {                   // this tile's soft-max partial of token row i0 + t
+          const float* red_m = reinterpret_cast<const float*>(sm + 4096);
+          const float* red_s = red_m + 4 * NTOK;
+          float m = red_m[t];
+#pragma unroll
+          for (int w = 1; w < 4; ++w) m = fmaxf(m, red_m[w * NTOK + t]);
+          float sum = 0.f;
+#pragma unroll
+          for (int w = 0; w < 4; ++w)
+            if (red_m[w * NTOK + t] > -INFINITY) sum += red_s[w * NTOK + t] * __expf(red_m[w * NTOK + t] - m);
+          p.lse_part[static_cast<size_t>(col0 / BM) * p.n_rows + i0 + t] = make_float2(m, sum);
+        }
       }
     }
   }
@@ -319,6 +352,8 @@ int cod_launch_gemm_tc2(cod_ctx* c, const GemmArgs& g, cudaStream_t st) {
   p.staged = (g.ldc % 4 == 0) && ((reinterpret_cast<uintptr_t>(g.C) & 15u) == 0);
   for (int i = 0; i < g.n_seg; ++i) p.staged = p.staged && (g.seg[i].N % 4 == 0);
   p.amax = g.amax;
+  p.lse_part = g.amax ? g.lse_part : nullptr;
+  p.sample_state = g.sample_state;
   p.status = c->status;
 
   CUtensorMap mw[3], ma;

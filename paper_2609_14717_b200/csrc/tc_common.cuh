@@ -217,6 +217,76 @@ __device__ __forceinline__ unsigned long long warp_colmax32(unsigned long long (
   return k[0];
 }
 
+// Column-wise sum over the 32 lanes of a warp for 32 columns at once (same exchange pattern as
+// warp_colmax32): afterwards lane L holds the sum of column L.
+__device__ __forceinline__ float warp_colsum32(float (&e)[32], int lane) {
+#pragma unroll
+  for (int off = 16; off >= 1; off >>= 1) {
+    const bool hi = (lane & off) != 0;
+#pragma unroll
+    for (int c = 0; c < off; ++c) {
+      const float send = hi ? e[c] : e[c + off];
+      const float mine = hi ? e[c + off] : e[c];
+      e[c] = mine + __shfl_xor_sync(0xffffffffu, send, off);
+    }
+  }
+  return e[0];
+}
+__device__ __forceinline__ float order_key_to_float(unsigned k) {     // inverse of order_key
+  return __uint_as_float((k & 0x80000000u) ? (k & 0x7FFFFFFFu) : ~k);
+}
+
+// ---------------------------------------------------------------------------- sampling head
+// Counter-based uniform number of the Gumbel-max draw: a chain of the 32-bit 'murmur3 finaliser'
+// over (seed, step, row, column); U = ((h >> 9) + 0.5) * 2^-23 lies in (0, 1) and is exact in float.
+__host__ __device__ __forceinline__ uint32_t mix32(uint32_t x) {
+  x ^= x >> 16; x *= 0x85EBCA6Bu; x ^= x >> 13; x *= 0xC2B2AE35u; x ^= x >> 16;
+  return x;
+}
+__host__ __device__ __forceinline__ uint32_t sample_state(unsigned long long seed, uint32_t step) {
+  uint32_t h = mix32(static_cast<uint32_t>(seed) ^ 0x9E3779B9u);
+  h = mix32(h + static_cast<uint32_t>(seed >> 32));
+  return mix32(h + step);
+}
+// -log(-log U) for the element (row state h_row = mix32(state + row), column col). U comes within
+// 2^-24 of 1, where -log U must keep its relative accuracy (those are the large-noise elements that
+// tend to win the argmax): there -log U = -log1p(-w) with w = 1 - U (exact in float) is taken from
+// its series, elsewhere from the fast logarithm; the outer logarithm's argument is never near 1 in
+// relative terms that matter (absolute error 2^-22).
+__device__ __forceinline__ float gumbel_noise(uint32_t h_row, uint32_t col) {
+  const uint32_t h = mix32(h_row + col);
+  const float u = (static_cast<float>(h >> 9) + 0.5f) * 1.1920928955078125e-07f;   // 2^-23
+  const float w = 1.0f - u;
+  const float t_series = w * fmaf(w, fmaf(w, 0.3333333433f, 0.5f), 1.0f);          // w < 2^-6: error < w^3 / 4
+  const float t = w < 0.015625f ? t_series : -__logf(u);
+  return -__logf(t);
+}
+// One chunk of 32 token columns in one warp of the LM-head epilogue, sampling form. v: the raw
+// logits of this lane's vocabulary row (index vocab_idx, valid if f_ok) for the 32 columns;
+// hrow: the 32 columns' row states. Returns for column `lane`: the packed (perturbed logit,
+// ~index) key of the warp's best row, and the sum of exp(raw - m) over the warp's valid rows
+// with m = that best perturbed logit (noise >= -2.9, so raw - m <= 2.9: no overflow).
+__device__ __forceinline__ void sample_chunk(const uint32_t (&v)[32], bool f_ok, uint32_t vocab_idx,
+                                             const uint32_t* hrow, int lane, unsigned long long& best,
+                                             float& m_ref, float& s_sum) {
+  const unsigned long long low = static_cast<unsigned long long>(0xFFFFFFFFu - vocab_idx);
+  unsigned long long k[32];
+#pragma unroll
+  for (int j = 0; j < 32; ++j) {
+    const float pert = __uint_as_float(v[j]) + gumbel_noise(hrow[j], vocab_idx);
+    k[j] = f_ok ? ((static_cast<unsigned long long>(order_key(pert)) << 32) | low) : 0ull;
+  }
+  best = warp_colmax32(k, lane);
+  m_ref = best ? order_key_to_float(static_cast<unsigned>(best >> 32)) : -INFINITY;
+  float e[32];
+#pragma unroll
+  for (int j = 0; j < 32; ++j) {
+    const float mj = __shfl_sync(0xffffffffu, m_ref, j);
+    e[j] = (f_ok && mj > -INFINITY) ? __expf(__uint_as_float(v[j]) - mj) : 0.f;
+  }
+  s_sum = warp_colsum32(e, lane);
+}
+
 // ---------------------------------------------------------------------------- tensor maps (host)
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
                                   const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,

@@ -133,3 +133,36 @@ def test_full_size_attention_alone_on_identical_inputs(name, sample):
         assert np.max(np.abs(mass.cpu().numpy()[sample] - mref)) <= TOL
     assert ctx.poll_status() == 0
     ctx.close()
+
+
+@pytest.mark.parametrize("name,rows", [("cfg2", list(range(16))), ("cfg3", [0, 1, 37, 255, 256, 300, 510, 511])])
+def test_full_size_sampling_head_on_sampled_rows(name, rows):
+    """cod_lm_head_sample over the full vocabulary (151936) at 16 and 512 rows; the oracle draws the
+    sampled rows with the same row counters."""
+    from paper_2609_14717_b200 import binding as B
+    wl = synth.scaled(synth.workload(name), n_rounds=1, ctx=(16, 16), n_layers=1)
+    sh = wl.shape
+    lay = synth.make_layout(wl, 3)
+    w = synth.make_weights(sh, 3)
+    ctx = B.Context(B.make_config(sh, wl.S, int(lay["max_pages_per_seq"]), int(lay["n_pages"])))
+    ctx.set_weights(B.weights_to_device(w, sh.dtype))
+    R = wl.R
+    x = np.random.default_rng(5).standard_normal((R, sh.d_model)).astype(np.float32)
+    tok = torch.zeros(R, dtype=torch.int32, device="cuda")
+    q = torch.zeros(R, dtype=torch.float32, device="cuda")
+    lse = torch.zeros(R, dtype=torch.float32, device="cuda")
+    ctx.lm_head_sample(torch.from_numpy(x).cuda(), R, 20260925, 3, tok, q, lse)
+    torch.cuda.synchronize()
+    w_o = {"g_final": np.asarray(w["g_final"], dtype=np.float64), "emb": np.asarray(w["emb"], dtype=np.float64)}
+    rows = np.array(rows)
+    t_o, q_o, lse_o, gap = orc.lm_head_sample(x[rows], w_o, oracle_config(sh), 20260925, 3, row_ids=rows)
+    tg, qg, lg = tok.cpu().numpy()[rows], q.cpu().numpy()[rows], lse.cpu().numpy()[rows]
+    assert np.max(np.abs(lg - lse_o)) <= TOL * max(1.0, float(np.abs(lse_o).max()))
+    sure = gap >= GAP
+    assert sure.sum() >= len(rows) // 2
+    assert np.array_equal(tg[sure], t_o[sure])
+    same = tg == t_o
+    assert np.max(np.abs(qg[same] / q_o[same] - 1.0)) <= 3 * TOL
+    assert ctx.poll_status() == 0
+    ctx.close()
+

@@ -506,3 +506,45 @@ def test_round_parity_with_stochastic_verification():
     assert P.ctx.poll_status() == 0
     P.close()
 
+
+@pytest.mark.parametrize("name", ["small_bf16", "small_bf16_W8", "mid_bf16"])
+def test_lm_head_sample_parity(name):
+    """Gumbel-max draw fused into the LM head: same counter-based noise on both sides, so the drawn
+    token must agree wherever the oracle's perturbed top-2 gap is clear; q and the log-sum-exp agree
+    to the bf16 bound. Several steps: different noise, different tokens."""
+    B = _B()
+    Hn = _H()
+    wl = _workloads()[name]
+    P = Hn.Pair(wl, seed=8, fill_pool=False)
+    sh = wl.shape
+    R = wl.R
+    x = np.random.default_rng(4).standard_normal((R, sh.d_model)).astype(np.float32)
+    xg = torch.from_numpy(x).cuda()
+    tok = torch.zeros(R, dtype=torch.int32, device="cuda")
+    q = torch.zeros(R, dtype=torch.float32, device="cuda")
+    lse = torch.zeros(R, dtype=torch.float32, device="cuda")
+    w_o = dict(P.w_o); w_o["emb"] = P.w_o["emb"]
+    seen, exempt = set(), 0
+    for step in range(3):
+        P.ctx.lm_head_sample(xg.clone(), R, 0xDEADBEEF12345, step, tok, q, lse)
+        torch.cuda.synchronize()
+        t_o, q_o, lse_o, gap = orc.lm_head_sample(x, w_o, P.cfg_o, 0xDEADBEEF12345, step)
+        _, _, logits = orc.lm_head_argmax(x, w_o, P.cfg_o)
+        scale = np.abs(logits).max()
+        assert np.max(np.abs(lse.cpu().numpy() - lse_o)) <= Hn.TOL["bf16"] * scale
+        sure = gap >= Hn.GAP
+        exempt += int((~sure).sum())
+        tg = tok.cpu().numpy()
+        assert np.array_equal(tg[sure], t_o[sure])
+        same = tg == t_o
+        assert np.max(np.abs(q.cpu().numpy()[same] / q_o[same] - 1.0)) <= 3 * Hn.TOL["bf16"]
+        seen.update(tg.tolist())
+        # a different step is a different draw
+        if step:
+            assert not np.array_equal(tg, prev)
+        prev = tg.copy()
+    assert exempt <= 0.05 * 3 * R
+    assert len(seen) > R // 2                                   # really sampling, not the argmax
+    assert P.ctx.poll_status() == 0
+    P.close()
+
