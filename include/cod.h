@@ -259,11 +259,17 @@ int cod_draft_round(cod_ctx* ctx, const int32_t* draft, const int32_t* target, c
    clear != 0 also resets it. */
 int cod_poll_status(cod_ctx* ctx, uint32_t* dev_flags, int clear, cod_stream_t stream);
 
-/* cod_draft_round with cod_verify_accept_stochastic as its first part; everything else identical. */
+/* cod_draft_round at temperature 1: cod_verify_accept_stochastic is its first part, and if q_next is
+   non-null the next block is DRAWN by the rule of cod_lm_head_sample (row counter r = s*W + i, the
+   given seed and step) instead of taken greedily: next_draft[s, 0] = bonus, next_draft[s, i] = the
+   drawn token, q_next [S, W] device float = its soft-max probability (q_next[s, 0] belongs to the
+   row-0 draw, which the bonus token replaces). With q_next == NULL the block is the greedy argmax and
+   the proposal is a point mass (the next verification then takes q_tok = 1). */
 int cod_draft_round_stochastic(cod_ctx* ctx, const int32_t* target, const float* p_tok,
                                const float* q_tok, const float* u, const void* H, int S, int n_forced,
                                int mode, cod_state* st, cod_split* split_out, int32_t* next_draft,
-                               const cod_taps* taps, cod_stream_t stream);
+                               const cod_taps* taps, float* q_next, unsigned long long seed,
+                               uint32_t step, cod_stream_t stream);
 
 /* Analysis aid — the re-convergence count R of Section 5.2 (the equation defining R), one per
    sequence: R[s] = #{ q in [0, len[s]) : z[s, q+d] == y[s, q] for some d in {-1, 0, +1} with

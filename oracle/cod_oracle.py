@@ -444,14 +444,21 @@ def draft_round(draft: np.ndarray, target: np.ndarray, H: np.ndarray, st: Oracle
 
 def draft_round_stochastic(target: np.ndarray, p_tok: np.ndarray, q_tok: np.ndarray, u: np.ndarray,
                            H: np.ndarray, st: OracleState, w: Dict[str, np.ndarray], n_forced: int,
-                           mode: int) -> Dict[str, np.ndarray]:
+                           mode: int, sample: Optional[tuple] = None) -> Dict[str, np.ndarray]:
     """draft_round with speculative-sampling verification as its first step (Appendix A, "Why
-    verification remains valid": Carryover changes the proposal distribution, not the rule)."""
+    verification remains valid": Carryover changes the proposal distribution, not the rule).
+    sample = (seed, step): the next block is drawn by lm_head_sample (row counters 0..R-1) instead
+    of taken greedily; the result then also holds q_next and the perturbed top-2 gap."""
     cfg = st.cfg
     split = verify_accept_stochastic(p_tok, q_tok, u, target, st.committed_len, st.block_table, cfg.page, n_forced)
     J = project_kv(H, split, w, cfg, mode)
     scatter_kv(J, split, st, mode)
     res = draft_block(st, split["bonus"], w, use_carry=(mode == MODE_CARRY))
+    if sample is not None:
+        tok, q, _, gap = lm_head_sample(res["x_final"], w, cfg, sample[0], sample[1])
+        res["tok"] = tok.reshape(st.S, cfg.W)
+        res["gap"] = gap.reshape(st.S, cfg.W)
+        res["q_next"] = q.reshape(st.S, cfg.W)
     next_draft = res["tok"].copy()
     next_draft[:, 0] = split["bonus"]
     res.update(split=split, J=J, next_draft=next_draft.astype(np.int32))

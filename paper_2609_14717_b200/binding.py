@@ -84,7 +84,8 @@ def load_library() -> C.CDLL:
     lib.cod_lm_head_sample.argtypes = [vp, vp, i32, C.c_uint64, C.c_uint32, vp, vp, vp, vp]
     lib.cod_verify_accept_stochastic.argtypes = [vp, vp, vp, vp, vp, i32, i32, C.POINTER(CodState), C.POINTER(CodSplit), vp]
     lib.cod_draft_round_stochastic.argtypes = [vp, vp, vp, vp, vp, vp, i32, i32, i32, C.POINTER(CodState),
-                                               C.POINTER(CodSplit), vp, C.POINTER(CodTaps), vp]
+                                               C.POINTER(CodSplit), vp, C.POINTER(CodTaps), vp, C.c_uint64,
+                                               C.c_uint32, vp]
     lib.cod_poll_status.argtypes = [vp, C.POINTER(C.c_uint32), i32, vp]
     lib.cod_profile_enable.argtypes = [vp, C.c_uint32]
     lib.cod_profile_read.argtypes = [vp, i32, C.POINTER(C.c_float), C.POINTER(C.c_int32)]
@@ -265,14 +266,15 @@ class Context:
             self._h, _ptr(target), _ptr(p_tok), _ptr(q_tok), _ptr(u), S, n_forced, C.byref(st), C.byref(sp), _stream()))
 
     def draft_round_stochastic(self, target, p_tok, q_tok, u, H, S, n_forced, mode, state: State,
-                               split: Optional[Split], next_draft, taps: Optional[Taps] = None) -> None:
+                               split: Optional[Split], next_draft, taps: Optional[Taps] = None,
+                               q_next=None, seed: int = 0, step: int = 0) -> None:
         st = state.struct()
         sp = split.struct() if split is not None else None
         tp = taps.struct() if taps is not None else None
         _check("cod_draft_round_stochastic", lib().cod_draft_round_stochastic(
             self._h, _ptr(target), _ptr(p_tok), _ptr(q_tok), _ptr(u), _ptr(H), S, n_forced, mode, C.byref(st),
             C.byref(sp) if sp is not None else None, _ptr(next_draft),
-            C.byref(tp) if tp is not None else None, _stream()))
+            C.byref(tp) if tp is not None else None, _ptr(q_next), seed, step, _stream()))
 
     def lm_head_sample(self, x, n_rows, seed, step, tok, q_tok=None, lse=None) -> None:
         _check("cod_lm_head_sample", lib().cod_lm_head_sample(

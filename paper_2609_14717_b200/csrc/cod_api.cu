@@ -346,7 +346,7 @@ int cod_lm_head_argmax(cod_ctx* c, const float* x, int n_rows, int32_t* tok, flo
 static int round_impl(cod_ctx* c, const int32_t* draft, const int32_t* target, const float* p_tok,
                       const float* q_tok, const float* u, const void* H, int S, int n_forced, int mode,
                       cod_state* st, cod_split* split_out, int32_t* next_draft, const cod_taps* taps,
-                      cod_stream_t stream) {
+                      cod_stream_t stream, float* q_next = nullptr, unsigned long long seed = 0, uint32_t step = 0) {
   const bool stochastic = p_tok != nullptr;
   if (!c || (!stochastic && !draft) || !target || !H || !next_draft || state_has_null(st)) return COD_ERR_INVALID_ARG;
   if (stochastic && (!q_tok || !u)) return COD_ERR_INVALID_ARG;
@@ -422,6 +422,16 @@ static int round_impl(cod_ctx* c, const int32_t* draft, const int32_t* target, c
       return rc;
   }
   // part 5
+  if (q_next != nullptr) {                      // temperature 1: the block is drawn, with its proposal probabilities
+    GemmArgs g{};
+    g.A = c->a; g.lda = c->D; g.n_rows = R; g.K = c->D;
+    g.seg[0] = {c->w.emb, f.vocab}; g.n_seg = 1;
+    g.splits = 1; g.amax = c->amax; g.klass = COD_K_LMHEAD;
+    g.lse_part = c->lse_part; g.sample_state = cod_sample_state(seed, step);
+    if (c->force_simt || !(cod_gemm_tc2_supported(c, g) || cod_gemm_tc_supported(c, g))) return COD_ERR_UNSUPPORTED;
+    if ((rc = cod_launch_gemm(c, g, s)) != COD_OK) return rc;
+    return cod_launch_finalize_sample(c, R, g.sample_state, c->tok, q_next, nullptr, s, sp->bonus, next_draft);
+  }
   if ((rc = lm_head_impl(c, R, s)) != COD_OK) return rc;
   return cod_launch_finalize(c, R, f.block, sp->bonus, c->tok, next_draft, taps ? taps->top_logit : nullptr, s);
 }
@@ -455,9 +465,10 @@ int cod_draft_round(cod_ctx* c, const int32_t* draft, const int32_t* target, con
 int cod_draft_round_stochastic(cod_ctx* c, const int32_t* target, const float* p_tok, const float* q_tok,
                                const float* u, const void* H, int S, int n_forced, int mode, cod_state* st,
                                cod_split* split_out, int32_t* next_draft, const cod_taps* taps,
-                               cod_stream_t stream) {
+                               float* q_next, unsigned long long seed, uint32_t step, cod_stream_t stream) {
   if (!p_tok || !q_tok || !u) return COD_ERR_INVALID_ARG;
-  return round_impl(c, nullptr, target, p_tok, q_tok, u, H, S, n_forced, mode, st, split_out, next_draft, taps, stream);
+  return round_impl(c, nullptr, target, p_tok, q_tok, u, H, S, n_forced, mode, st, split_out, next_draft, taps, stream,
+                    q_next, seed, step);
 }
 
 int cod_reconvergence_count(cod_ctx* c, const int32_t* z, const int32_t* y, const int32_t* len, int S,

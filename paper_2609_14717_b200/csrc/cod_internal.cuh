@@ -219,7 +219,7 @@ int cod_launch_attn_simt(cod_ctx* c, int layer, const void* q, const void* kb, c
 int cod_launch_reconvergence(cod_ctx* c, const int32_t* z, const int32_t* y, const int32_t* len, int S,
                              int32_t* R, cudaStream_t st);
 int cod_launch_finalize_sample(cod_ctx* c, int R, uint32_t state, int32_t* tok, float* q_tok, float* lse,
-                               cudaStream_t st);
+                               cudaStream_t st, const int32_t* bonus = nullptr, int32_t* next_draft = nullptr);
 uint32_t cod_sample_state(unsigned long long seed, uint32_t step);   // hash state after seed and step
 int cod_launch_rope_blk_only(cod_ctx* c, const int32_t* committed_len, int S, cudaStream_t st);
 int cod_launch_fcE(cod_ctx* c, cudaStream_t st);

@@ -379,7 +379,8 @@ int cod_launch_gemm_tc(cod_ctx* c, const GemmArgs& g, cudaStream_t st) {
 namespace {
 __global__ void k_finalize_sample(const unsigned long long* __restrict__ amax, const float2* __restrict__ lse_part,
                                   int n_tiles, int R, uint32_t state, int32_t* __restrict__ tok,
-                                  float* __restrict__ q_tok, float* __restrict__ lse_out) {
+                                  float* __restrict__ q_tok, float* __restrict__ lse_out, int W,
+                                  const int32_t* __restrict__ bonus, int32_t* __restrict__ next_draft) {
   cod_pdl_prologue();
   const int r = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5), lane = threadIdx.x & 31;
   if (r >= R) return;
@@ -404,18 +405,20 @@ __global__ void k_finalize_sample(const unsigned long long* __restrict__ amax, c
     const float pert = tc::order_key_to_float(static_cast<unsigned>(key >> 32));
     const float raw = pert - tc::gumbel_noise(tc::mix32(state + static_cast<uint32_t>(r)), static_cast<uint32_t>(idx));
     const float lse = m + logf(s);
-    tok[r] = idx;
+    if (tok) tok[r] = idx;
     if (q_tok) q_tok[r] = expf(raw - lse);
     if (lse_out) lse_out[r] = lse;
+    if (next_draft) next_draft[r] = (r % W == 0) ? bonus[r / W] : idx;     // row 0 of a block is the bonus token
   }
 }
 }  // namespace
 
 int cod_launch_finalize_sample(cod_ctx* c, int R, uint32_t state, int32_t* tok, float* q_tok, float* lse,
-                               cudaStream_t st) {
+                               cudaStream_t st, const int32_t* bonus, int32_t* next_draft) {
   ProfScope prof(c, COD_K_ROWOPS, st);
   const int n_tiles = (c->cfg.vocab + BM - 1) / BM;
-  cod_launch_pdl(c, k_finalize_sample, (R + 3) / 4, 128, 0, st, c->amax, c->lse_part, n_tiles, R, state, tok, q_tok, lse);
+  cod_launch_pdl(c, k_finalize_sample, (R + 3) / 4, 128, 0, st, c->amax, c->lse_part, n_tiles, R, state, tok, q_tok, lse, c->cfg.block,
+                 bonus, next_draft);
   COD_CHECK_LAUNCH(c);
   return COD_OK;
 }

@@ -503,6 +503,24 @@ def test_round_parity_with_stochastic_verification():
         _check_round(P, res_o, L0, Hn.TOL["bf16"])
         ms.update(res_o["split"]["accept_len"].tolist())
     assert len(ms) > 2
+    # a temperature-1 round end to end: stochastic verification, then the next block drawn with its q
+    rd, dev = P.round_inputs(4)
+    p = rng.random((S, W), dtype=np.float32); q = rng.random((S, W), dtype=np.float32) * 0.6
+    u = rng.random((S, W), dtype=np.float32)
+    L0 = P.st_o.committed_len.copy()
+    res_o = orc.draft_round_stochastic(rd["target"], p, q, u, rd["H"], P.st_o, P.w_o, 1, orc.MODE_CARRY, sample=(77, 4))
+    q_next = torch.zeros((S, W), dtype=torch.float32, device="cuda")
+    P.ctx.draft_round_stochastic(dev["target"], torch.from_numpy(p).cuda(), torch.from_numpy(q).cuda(),
+                                 torch.from_numpy(u).cuda(), dev["H"], S, 1, B.COD_CARRY, P.st_g, P.split,
+                                 P.next_draft, P.taps, q_next=q_next, seed=77, step=4)
+    torch.cuda.synchronize()
+    _check_round(P, res_o, L0, Hn.TOL["bf16"])                  # next_draft compared where the perturbed gap is clear
+    nd = P.next_draft.cpu().numpy()
+    same = nd == res_o["next_draft"]
+    same[:, 0] = False
+    assert same.sum() > (S * (W - 1)) // 2
+    assert np.max(np.abs(q_next.cpu().numpy()[same] / res_o["q_next"][same] - 1.0)) <= 3 * Hn.TOL["bf16"]
+    assert len(np.unique(nd[:, 1:])) > 8                        # drawn, not the (nearly constant) argmax
     assert P.ctx.poll_status() == 0
     P.close()
 
