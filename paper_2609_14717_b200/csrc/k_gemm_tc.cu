@@ -58,6 +58,10 @@ __device__ __forceinline__ bool bar_and_128(bool v) {
 }
 
 
+// SAMPLE selects the sampling form of the argmax epilogue and WIDE the transposing store epilogue
+// (32 token rows and more) at compile time, so the kernel a batch-1 round launches a dozen times
+// carries neither: with ~45 short kernels per round, instruction fetch of cold code shows.
+template <bool SAMPLE, bool WIDE>
 __global__ void __launch_bounds__(NTHREADS, 1)
 k_gemm_tc(const __grid_constant__ CUtensorMap map_w0, const __grid_constant__ CUtensorMap map_w1,
           const __grid_constant__ CUtensorMap map_w2, const __grid_constant__ CUtensorMap map_a, const TcParams p) {
@@ -164,7 +168,7 @@ k_gemm_tc(const __grid_constant__ CUtensorMap map_w0, const __grid_constant__ CU
     const int f = f0 + warp * 32 + lane;                    // weight row within the segment
     const bool f_ok = f < seg_N;
     const uint32_t t_lane = tmem_base + (static_cast<uint32_t>(warp * 32) << 16);
-    if (ok && p.amax == nullptr && p.staged && p.NT >= 32) {
+    if (WIDE && ok && p.amax == nullptr) {
       // The accumulator has features on lanes and tokens on columns; C wants a token's features
       // contiguous. Transpose 32 tokens at a time through the (now idle) pipeline buffers and store
       // whole 512-byte feature runs: two 16 KB buffers, one barrier of the four warps per chunk.
@@ -204,7 +208,7 @@ k_gemm_tc(const __grid_constant__ CUtensorMap map_w0, const __grid_constant__ CU
           if (f_ok && i < n_rows) C[static_cast<size_t>(i) * p.ldc + col0 + warp * 32 + lane] = __uint_as_float(v[j]);
         }
       }
-    } else if (ok && p.lse_part != nullptr) {
+    } else if (SAMPLE && ok) {
       // sampling form: Gumbel noise on every logit before the argmax, and soft-max partials per column.
       // Scratch in the idle pipeline buffers: row states, then per-warp (m, sum) of every column.
       uint32_t* hrow = reinterpret_cast<uint32_t*>(sm);
@@ -273,7 +277,7 @@ k_gemm_tc(const __grid_constant__ CUtensorMap map_w0, const __grid_constant__ CU
 #pragma unroll
         for (int w = 1; w < 4; ++w) best = red[w * p.NT + t] > best ? red[w * p.NT + t] : best;
         atomicMax(p.amax + i0 + t, best);
-        if (p.lse_part != nullptr) {                   // this tile's soft-max partial of token row i0 + t
+        if (SAMPLE) {                                  // this tile's soft-max partial of token row i0 + t
           const float* red_m = reinterpret_cast<const float*>(sm + 4096);
           const float* red_s = red_m + 4 * 256;
           float m = red_m[t];
@@ -360,14 +364,22 @@ int cod_launch_gemm_tc(cod_ctx* c, const GemmArgs& g, cudaStream_t st) {
   if (!make_map_2d(&ma, g.A, g.n_rows, g.K, g.lda, p.NT)) return COD_ERR_CUDA;
 
   const size_t smem = static_cast<size_t>(stages) * stage_bytes + 1024 /* alignment slack */ + 34 * 8 + 4 * p.NT * 8;
-  static size_t configured = 0;
-  if (smem > configured) {
-    if (cudaFuncSetAttribute(k_gemm_tc, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem)) != cudaSuccess)
-      return COD_ERR_CUDA;
-    configured = smem;
+  // three instantiations: plain (narrow store or argmax), wide store, sampling argmax
+  const int variant = p.lse_part != nullptr ? 2 : ((p.amax == nullptr && p.staged && p.NT >= 32) ? 1 : 0);
+  static size_t configured[3] = {0, 0, 0};
+  if (smem > configured[variant]) {
+    const int bytes = static_cast<int>(smem);
+    const cudaError_t e =
+        variant == 2 ? cudaFuncSetAttribute(k_gemm_tc<true, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes)
+        : variant == 1 ? cudaFuncSetAttribute(k_gemm_tc<false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes)
+                       : cudaFuncSetAttribute(k_gemm_tc<false, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
+    if (e != cudaSuccess) return COD_ERR_CUDA;
+    configured[variant] = smem;
   }
   dim3 grid((g.n_rows + p.NT - 1) / p.NT, tiles, splits);
-  cod_launch_pdl(c, k_gemm_tc, grid, NTHREADS, smem, st, mw[0], mw[1], mw[2], ma, p);
+  if (variant == 2) cod_launch_pdl(c, k_gemm_tc<true, false>, grid, NTHREADS, smem, st, mw[0], mw[1], mw[2], ma, p);
+  else if (variant == 1) cod_launch_pdl(c, k_gemm_tc<false, true>, grid, NTHREADS, smem, st, mw[0], mw[1], mw[2], ma, p);
+  else cod_launch_pdl(c, k_gemm_tc<false, false>, grid, NTHREADS, smem, st, mw[0], mw[1], mw[2], ma, p);
   COD_CHECK_LAUNCH(c);
   return COD_OK;
 }

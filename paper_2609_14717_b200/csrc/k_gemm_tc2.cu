@@ -53,6 +53,8 @@ struct Tc2Params {
 };
 
 
+// SAMPLE selects the sampling form of the argmax epilogue at compile time (see k_gemm_tc).
+template <bool SAMPLE>
 __global__ void __launch_bounds__(NTHREADS, 1)
 k_gemm_tc2(const __grid_constant__ CUtensorMap map_w0, const __grid_constant__ CUtensorMap map_w1,
            const __grid_constant__ CUtensorMap map_w2, const __grid_constant__ CUtensorMap map_a, const Tc2Params p) {
@@ -205,7 +207,7 @@ k_gemm_tc2(const __grid_constant__ CUtensorMap map_w0, const __grid_constant__ C
           if (f_ok && i < n_rows) C[static_cast<size_t>(i) * p.ldc + col0 + qw * 32 + lane] = __uint_as_float(v[j]);
         }
       }
-    } else if (ok && p.lse_part != nullptr) {
+    } else if (SAMPLE && ok) {
       // sampling form: Gumbel noise on every logit before the argmax, and soft-max partials per column.
       // Scratch in the idle pipeline buffers: row states, then per-warp (m, sum) of every column.
       uint32_t* hrow = reinterpret_cast<uint32_t*>(sm);
@@ -252,7 +254,7 @@ k_gemm_tc2(const __grid_constant__ CUtensorMap map_w0, const __grid_constant__ C
 #pragma unroll
         for (int w = 1; w < 4; ++w) best = red[w * NTOK + t] > best ? red[w * NTOK + t] : best;
         if (best) atomicMax(p.amax + i0 + t, best);
-        if (p.lse_part != nullptr) {                   // this tile's soft-max partial of token row i0 + t
+        if (SAMPLE) {                                  // this tile's soft-max partial of token row i0 + t
           const float* red_m = reinterpret_cast<const float*>(sm + 4096);
           const float* red_s = red_m + 4 * NTOK;
           float m = red_m[t];
@@ -365,11 +367,13 @@ int cod_launch_gemm_tc2(cod_ctx* c, const GemmArgs& g, cudaStream_t st) {
 
   const size_t smem = static_cast<size_t>(p.stages) * (A_TILE_BYTES + p.n_acc * B_TILE_BYTES) + 1024 + 18 * 8 +
                       static_cast<size_t>(4) * p.n_acc * NT * 8;
-  static size_t configured = 0;
-  if (smem > configured) {
-    if (cudaFuncSetAttribute(k_gemm_tc2, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem)) != cudaSuccess)
-      return COD_ERR_CUDA;
-    configured = smem;
+  static size_t configured[2] = {0, 0};
+  const int sample = p.lse_part != nullptr ? 1 : 0;
+  if (smem > configured[sample]) {
+    const cudaError_t e = sample ? cudaFuncSetAttribute(k_gemm_tc2<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem))
+                                 : cudaFuncSetAttribute(k_gemm_tc2<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem));
+    if (e != cudaSuccess) return COD_ERR_CUDA;
+    configured[sample] = smem;
   }
   cudaLaunchConfig_t cfg{};
   cfg.gridDim = dim3(2, pairs * p.n_tiles_n, splits);
@@ -385,7 +389,9 @@ int cod_launch_gemm_tc2(cod_ctx* c, const GemmArgs& g, cudaStream_t st) {
   attr[1].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = attr;
   cfg.numAttrs = c->pdl ? 2 : 1;
-  if (cudaLaunchKernelEx(&cfg, k_gemm_tc2, mw[0], mw[1], mw[2], ma, p) != cudaSuccess) return COD_ERR_CUDA;
+  const cudaError_t le = sample ? cudaLaunchKernelEx(&cfg, k_gemm_tc2<true>, mw[0], mw[1], mw[2], ma, p)
+                                : cudaLaunchKernelEx(&cfg, k_gemm_tc2<false>, mw[0], mw[1], mw[2], ma, p);
+  if (le != cudaSuccess) return COD_ERR_CUDA;
   COD_CHECK_LAUNCH(c);
   return COD_OK;
 }
