@@ -202,7 +202,7 @@ def time_oracle(wl, seed, weights, n_rounds, S_sample, budget_s=None):
         t0 = time.perf_counter()
         orc.draft_round(rd["draft"], rd["target"], rd["H"], st, w64, sub.n_forced, orc.MODE_CARRY)
         times.append(time.perf_counter() - t0)
-        if budget_s is not None and sum(times) > budget_s and len(times) >= 1:
+        if budget_s is not None and sum(times) > budget_s and len(times) >= 3:
             break
     return times
 
@@ -438,7 +438,8 @@ def run_gpu(args):
     cpu = None
     if world == 1 and not args.no_cpu_baseline:
         S_sample = 1 if wl.S == 1 else 2
-        times = time_oracle(wl, seed, weights, n_rounds=3, S_sample=S_sample, budget_s=25.0)
+        # about 12 s of oracle work (at least 3 rounds, at most what the page tables were sized for)
+        times = time_oracle(wl, seed, weights, n_rounds=max(3, min(64, wl.n_rounds - 1)), S_sample=S_sample, budget_s=12.0)
         mean = sum(times) / len(times)
         cpu = {"value": (S_sample / wl.S) / mean, "unit": UNIT, "cores": cores_used(), "kind": "oracle",
                "sample": f"{len(times)} whole rounds of {S_sample} of {wl.S} sequences at full shapes "
