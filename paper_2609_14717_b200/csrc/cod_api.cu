@@ -41,6 +41,10 @@ size_t carve(cod_ctx* c) {
   widest = widest > static_cast<size_t>(2 * f.d_ff) ? widest : static_cast<size_t>(2 * f.d_ff);
   c->gemm_out_floats = static_cast<size_t>(COD_MAX_SPLITS) * R * widest;
   cv.take(c->gemm_out, sizeof(float) * c->gemm_out_floats);
+  // the side branch (first layer's Q/K/V chain next to the context projection) pays off where the
+  // round is a chain of short, latency-bound kernels: up to 128 rows
+  c->side_rows = static_cast<int>(R < 128 ? R : 128);
+  cv.take(c->gemm_out2, sizeof(float) * COD_MAX_SPLITS * c->side_rows * (c->qw + 2 * c->kvw));
   cv.take(c->hc, es * R * c->D_in);
   cv.take(c->z, es * R * D);
   cv.take(c->x, sizeof(float) * R * D);
@@ -200,6 +204,9 @@ int cod_create(const cod_config* cfg, cod_ctx** out) {
   c->prof_ev = static_cast<cudaEvent_t*>(calloc(2 * COD_PROF_SLOTS, sizeof(cudaEvent_t)));
   c->prof_class = static_cast<unsigned char*>(calloc(COD_PROF_SLOTS, 1));
   if (!c->prof_ev || !c->prof_class) ok = false;
+  if (ok) ok = cudaStreamCreateWithFlags(&c->side, cudaStreamNonBlocking) == cudaSuccess &&
+               cudaEventCreateWithFlags(&c->ev_fork, cudaEventDisableTiming) == cudaSuccess &&
+               cudaEventCreateWithFlags(&c->ev_join, cudaEventDisableTiming) == cudaSuccess;
   for (int i = 0; ok && i < 2 * COD_PROF_SLOTS; ++i) ok = cudaEventCreate(&c->prof_ev[i]) == cudaSuccess;
   if (!ok) { cudaFree(c->ws); cudaGetLastError(); free(c->prof_ev); free(c->prof_class); delete c; return COD_ERR_CUDA; }
   *out = c;
@@ -210,6 +217,9 @@ int cod_destroy(cod_ctx* c) {
   if (!c) return COD_ERR_INVALID_ARG;
   cudaDeviceSynchronize();
   cudaFree(c->ws);
+  if (c->ev_fork) cudaEventDestroy(c->ev_fork);
+  if (c->ev_join) cudaEventDestroy(c->ev_join);
+  if (c->side) cudaStreamDestroy(c->side);
   for (int i = 0; i < 2 * COD_PROF_SLOTS; ++i) cudaEventDestroy(c->prof_ev[i]);
   free(c->prof_ev);
   free(c->prof_class);
@@ -363,23 +373,45 @@ static int round_impl(cod_ctx* c, const int32_t* draft, const int32_t* target, c
   int rc;
   c->pdl = true;
 
-  // parts 1-3
+  // part 1
   if ((rc = cod_launch_verify(c, draft, target, S, n_forced, st, sp, s, p_tok, q_tok, u)) != COD_OK) return rc;
-  if ((rc = project_impl(c, H, sp, S, mode, nullptr, st, taps ? taps->z : nullptr, s)) != COD_OK) return rc;
-  if ((rc = cod_launch_update_lens(c, sp, S, mode, st, s)) != COD_OK) return rc;
+
+  // The first layer's embedding + Q/K/V chain of the NEXT block needs only the bonus tokens and the
+  // position tables of part 1; the context projection (parts 2-3) needs only the row split. For
+  // small rounds (a chain of short kernels) the former runs on a side stream next to the latter
+  // and joins before the first attention; under stream capture the fork and join become graph edges.
+  const bool fork = R <= c->side_rows && c->gemm_out2 != nullptr;
+  cudaStream_t sq = fork ? c->side : s;                      // stream of the first layer's Q/K/V chain
+  float* slab_q = fork ? c->gemm_out2 : c->gemm_out;
+  if (fork) {
+    if (cudaEventRecord(c->ev_fork, s) != cudaSuccess || cudaStreamWaitEvent(c->side, c->ev_fork, 0) != cudaSuccess)
+      return COD_ERR_CUDA;
+  } else {
+    // parts 2-3 first, on the one stream
+    if ((rc = project_impl(c, H, sp, S, mode, nullptr, st, taps ? taps->z : nullptr, s)) != COD_OK) return rc;
+    if ((rc = cod_launch_update_lens(c, sp, S, mode, st, s)) != COD_OK) return rc;
+  }
 
   // the next block: [bonus, MASK, ...] through every drafter layer
-  if ((rc = cod_launch_embed_norm(c, sp->bonus, S, s)) != COD_OK) return rc;
+  if ((rc = cod_launch_embed_norm(c, sp->bonus, S, sq)) != COD_OK) return rc;
   for (int l = 0; l < f.n_layers; ++l) {
+    cudaStream_t sl = l == 0 ? sq : s;
     GemmArgs g{};
     g.A = c->a; g.lda = c->D; g.n_rows = R; g.K = c->D;
     g.seg[0] = {static_cast<const char*>(c->w.wq) + es * l * c->qw * c->D, c->qw};
     g.seg[1] = {static_cast<const char*>(c->w.wk) + es * l * c->kvw * c->D, c->kvw};
     g.seg[2] = {static_cast<const char*>(c->w.wv) + es * l * c->kvw * c->D, c->kvw};
     g.n_seg = 3; g.klass = COD_K_QKV;
-    g.C = c->gemm_out; g.ldc = c->qw + 2 * c->kvw; g.splits = pick_splits(c, g.ldc, c->D, R);
-    if ((rc = cod_launch_gemm(c, g, s)) != COD_OK) return rc;
-    if ((rc = cod_launch_qkv_finish(c, c->gemm_out, g.splits, R, l, s)) != COD_OK) return rc;
+    g.C = l == 0 ? slab_q : c->gemm_out; g.ldc = c->qw + 2 * c->kvw; g.splits = pick_splits(c, g.ldc, c->D, R);
+    if ((rc = cod_launch_gemm(c, g, sl)) != COD_OK) return rc;
+    if ((rc = cod_launch_qkv_finish(c, g.C, g.splits, R, l, sl)) != COD_OK) return rc;
+    if (l == 0 && fork) {
+      // parts 2-3 on the caller's stream meanwhile, then the join
+      if ((rc = project_impl(c, H, sp, S, mode, nullptr, st, taps ? taps->z : nullptr, s)) != COD_OK) return rc;
+      if ((rc = cod_launch_update_lens(c, sp, S, mode, st, s)) != COD_OK) return rc;
+      if (cudaEventRecord(c->ev_join, c->side) != cudaSuccess || cudaStreamWaitEvent(s, c->ev_join, 0) != cudaSuccess)
+        return COD_ERR_CUDA;
+    }
 
     float* tap_o = (taps && taps->attn_out) ? taps->attn_out + static_cast<size_t>(l) * R * c->qw : nullptr;
     float* tap_m = (taps && taps->carry_mass) ? taps->carry_mass + static_cast<size_t>(l) * R * f.n_q_heads : nullptr;

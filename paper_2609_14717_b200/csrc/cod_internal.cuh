@@ -140,6 +140,10 @@ struct cod_ctx {
   void* hmid;                  // [R, d_ff] activated MLP rows (storage type), d_ff > 0 only
   float2* lse_part;            // [ceil(vocab / 128)][R] soft-max partials of the sampling LM head
   float* gemm_out;             // split-K / unfused GEMM results
+  float* gemm_out2;            // a second, small slab buffer for the side branch of the round (null: no side branch)
+  int side_rows;               // the side branch is used for rounds of at most this many rows
+  cudaStream_t side;           // side branch of the round: the first layer's embedding / Q/K/V chain
+  cudaEvent_t ev_fork, ev_join;
   size_t gemm_out_floats;
   void* hc;                    // [R_max, D_in] accepted rows of H packed densely (baseline mode)
   void* z;                     // [R_max, D]
