@@ -67,6 +67,9 @@ class OracleConfig:
     hidden_norm: bool
     d_ff: int = 0            # > 0: every drafter layer has a gated MLP of this width
     qk_norm: bool = False    # per-head RMS norm of queries and keys before the rotation
+    carry_variant: str = "embedding"   # "embedding": E_carry on rejected rows (Eq. 2, the paper's choice);
+                                       # "none": rejected rows pass F unmarked; "projector": rejected rows
+                                       # pass their own fusion map F_rej (Table 4(b)'s two alternatives)
 
     @property
     def d_in(self) -> int:
@@ -219,8 +222,13 @@ def fuse_features(H: np.ndarray, rejected: np.ndarray, w: Dict[str, np.ndarray],
     """Z = F(H^keep) with E_carry added to the rejected rows first (Eq. 2; Algorithm 1
     right column, steps 2-3: the embedding is added "before projection by F")."""
     Hk = np.asarray(H, dtype=np.float64).copy()
-    Hk[rejected] = Hk[rejected] + w["e_carry"]
+    if cfg.carry_variant == "embedding":
+        Hk[rejected] = Hk[rejected] + w["e_carry"]
     Z = Hk @ w["fc"].T
+    if cfg.carry_variant == "projector":
+        # Section 5 "How should rejected states be distinguished?": a separate projector for the
+        # rejected rows instead of the embedding (its shape is not given; taken as F's)
+        Z[rejected] = Hk[rejected] @ w["fc_rej"].T
     if cfg.hidden_norm:
         Z = rmsnorm(Z, w["g_hidden"], cfg.rms_eps)
     return Z

@@ -52,6 +52,7 @@ class DrafterShape:
     h_rms: Optional[Tuple[float, float]] = None  # per-layer RMS range of H
     d_ff: int = 0         # width of the gated MLP of a drafter layer; 0 = attention sub-layer only
     qk_norm: bool = False # per-head RMS norm (with gain) of queries and keys before the rotation
+    carry_variant: str = "embedding"  # how rejected rows are told apart: "embedding" (E_carry), "none", "projector"
 
     @property
     def d_in(self) -> int:
@@ -151,7 +152,7 @@ def _normal(rng: np.random.Generator, shape, scale: float = 1.0) -> np.ndarray:
 
 # --------------------------------------------------------------------------- weights
 _WEIGHT_ORDER = ("fc", "e_carry", "g_hidden", "wk", "wv", "wq", "wo", "g_attn", "g_final", "emb",
-                 "w_gate", "w_up", "w_down", "g_mlp", "g_qnorm", "g_knorm")   # new names go last: stream index = position
+                 "w_gate", "w_up", "w_down", "g_mlp", "g_qnorm", "g_knorm", "fc_rej")   # new names go last: stream index = position
 
 
 def weight_shapes(sh: DrafterShape) -> Dict[str, Tuple[int, ...]]:
@@ -173,6 +174,8 @@ def weight_shapes(sh: DrafterShape) -> Dict[str, Tuple[int, ...]]:
                     "g_mlp": (Ld, D)})
     if sh.qk_norm:
         out.update({"g_qnorm": (Ld, sh.hd), "g_knorm": (Ld, sh.hd)})
+    if sh.carry_variant == "projector":
+        out["fc_rej"] = (D, sh.d_in)
     return out
 
 

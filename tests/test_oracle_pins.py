@@ -847,3 +847,30 @@ def test_gumbel_max_sample_follows_the_softmax_and_reports_its_probability():
     assert 0.05 < sm.max() < 0.95
     assert np.abs(counts / n - sm).max() < 4 * math.sqrt(0.25 / n)
 
+
+# ----------------------------------------------------------------------------- other ways to mark rejected rows
+def test_carry_variants_relate_as_they_must():
+    """'none' is the embedding variant with E_carry = 0; 'projector' with F_rej = F is 'none';
+    with another F_rej only the rejected rows change, and they are exactly F_rej h (one-hot probes)."""
+    base = synth.scaled(synth.workload("cfg1"), S=2, ctx=(10, 40), hidden_norm=False)
+    wl_n, wl_p = synth.scaled(base, carry_variant="none"), synth.scaled(base, carry_variant="projector")
+    w = orc.prepare_weights(synth.make_weights(wl_p.shape, 3))
+    rd = synth.make_round(base, 3, 0)
+    lay = synth.make_layout(base, 3)
+    split = orc.verify_accept(rd["draft"], rd["target"], lay["committed_len"], lay["block_table"], 16, 1)
+    W = base.shape.W
+    rejected = (np.tile(np.arange(W), base.S) >= np.repeat(split["accept_len"], W))
+    assert rejected.any() and (~rejected).any()
+    Z_e = orc.fuse_features(rd["H"], rejected, w, oracle_config(base.shape))
+    w0 = dict(w); w0["e_carry"] = np.zeros_like(w["e_carry"])
+    Z_e0 = orc.fuse_features(rd["H"], rejected, w0, oracle_config(base.shape))
+    Z_n = orc.fuse_features(rd["H"], rejected, w, oracle_config(wl_n.shape))
+    assert np.array_equal(Z_n, Z_e0) and not np.array_equal(Z_n, Z_e)
+    wp = dict(w); wp["fc_rej"] = w["fc"]
+    assert np.array_equal(orc.fuse_features(rd["H"], rejected, wp, oracle_config(wl_p.shape)), Z_n)
+    Z_p = orc.fuse_features(rd["H"], rejected, w, oracle_config(wl_p.shape))
+    assert np.array_equal(Z_p[~rejected], Z_n[~rejected]) and not np.allclose(Z_p[rejected], Z_n[rejected])
+    r = int(np.flatnonzero(rejected)[0])
+    want = [sum(w["fc_rej"][i, k] * float(rd["H"][r, k]) for k in range(base.shape.d_in)) for i in range(4)]
+    assert np.allclose(Z_p[r, :4], want, atol=1e-12)
+
