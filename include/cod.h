@@ -63,6 +63,9 @@ enum cod_mode {
 /* cod_config.flags */
 #define COD_F_HIDDEN_NORM 1u /* RMS-normalise (with gain g_hidden) the output of F */
 #define COD_F_NO_TENSOR_CORES 2u /* use the plain-FMA kernels only (an on-GPU cross-check) */
+#define COD_F_NO_CARRY_EMBED 8u /* rejected rows pass F unmarked ("no explicit discrimination", Section 5) */
+#define COD_F_REJ_PROJECTOR 16u /* rejected rows pass their own fusion map fc_rej instead of F + E_carry
+                                   ("separate projector", Section 5; its shape is taken as F's) */
 #define COD_F_QK_NORM 4u /* per-head RMS norm with gain (g_qnorm, g_knorm) of queries and of all keys,
                             cached and block keys alike, before the rotation */
 
@@ -115,6 +118,7 @@ typedef struct {
   const void* g_mlp;    /* [Ld][D]              gain of the pre-MLP norm                           */
   const void* g_qnorm;  /* [Ld][hd]             gain of the per-head query norm                    */
   const void* g_knorm;  /* [Ld][hd]             gain of the per-head key norm                      */
+  const void* fc_rej;   /* [D, D_in]            COD_F_REJ_PROJECTOR only: fusion map of rejected rows      */
 } cod_weights;
 
 /* Mutable drafter state of a batch (device, caller-owned). */

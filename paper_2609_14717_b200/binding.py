@@ -21,6 +21,8 @@ COD_CARRY, COD_BASELINE = 0, 1
 COD_F_HIDDEN_NORM = 1
 COD_F_NO_TENSOR_CORES = 2
 COD_F_QK_NORM = 4
+COD_F_NO_CARRY_EMBED = 8
+COD_F_REJ_PROJECTOR = 16
 DEV_BAD_TOKEN, DEV_PAGE_OVERFLOW, DEV_BAD_PAGE, DEV_TIMEOUT, DEV_BAD_LEN = 1, 2, 4, 8, 16
 
 EXPORTS = ("cod_create", "cod_destroy", "cod_set_weights", "cod_verify_accept", "cod_project_kv",
@@ -41,7 +43,8 @@ class CodConfig(C.Structure):
 
 
 _WEIGHT_FIELDS = ("fc", "e_carry", "g_hidden", "wk", "wv", "wq", "wo", "g_attn", "g_final", "emb",
-                  "w_gate", "w_up", "w_down", "g_mlp", "g_qnorm", "g_knorm")   # the last six: complete layer only
+                  "w_gate", "w_up", "w_down", "g_mlp", "g_qnorm", "g_knorm",   # these six: complete layer only
+                  "fc_rej")                                                     # separate-projector variant only
 _SPLIT_FIELDS = ("accept_len", "bonus", "row_pos", "commit_slot", "carry_slot", "acc_rows", "acc_off",
                  "rej_rows", "rej_off")
 _STATE_FIELDS = ("kv_pool", "block_table", "committed_len", "carry_kv", "carry_len")
@@ -331,7 +334,8 @@ def make_config(sh, max_batch: int, max_pages_per_seq: int, n_pages: int, attn_s
         page_size=sh.page, max_batch=max_batch, max_pages_per_seq=max_pages_per_seq, n_pages=n_pages,
         dtype=COD_BF16 if sh.dtype == "bf16" else COD_F32,
         flags=(COD_F_HIDDEN_NORM if sh.hidden_norm else 0) | (COD_F_NO_TENSOR_CORES if no_tensor_cores else 0)
-        | (COD_F_QK_NORM if sh.qk_norm else 0),
+        | (COD_F_QK_NORM if sh.qk_norm else 0)
+        | {"embedding": 0, "none": COD_F_NO_CARRY_EMBED, "projector": COD_F_REJ_PROJECTOR}[sh.carry_variant],
         rope_theta=sh.rope_theta, rms_eps=sh.rms_eps,
         attn_split_len=attn_split_len, d_ff=sh.d_ff)
 

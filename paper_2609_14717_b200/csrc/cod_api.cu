@@ -39,6 +39,7 @@ size_t carve(cod_ctx* c) {
   widest = widest > static_cast<size_t>(2 * f.n_layers * c->kvw) ? widest : static_cast<size_t>(2 * f.n_layers * c->kvw);
   widest = widest > static_cast<size_t>(c->qw + 2 * c->kvw) ? widest : static_cast<size_t>(c->qw + 2 * c->kvw);
   widest = widest > static_cast<size_t>(2 * f.d_ff) ? widest : static_cast<size_t>(2 * f.d_ff);
+  if ((f.flags & COD_F_REJ_PROJECTOR) && widest < 2 * D) widest = 2 * D;
   c->gemm_out_floats = static_cast<size_t>(COD_MAX_SPLITS) * R * widest;
   cv.take(c->gemm_out, sizeof(float) * c->gemm_out_floats);
   // the side branch (first layer's Q/K/V chain next to the context projection) pays off where the
@@ -141,7 +142,9 @@ int cod_create(const cod_config* cfg, cod_ctx** out) {
   if ((f.d_target * f.n_cap) % 8 || f.d_model % 8 || f.d_model > 32768) return COD_ERR_UNSUPPORTED;
   if ((f.n_kv_heads * f.head_dim) % 64) return COD_ERR_UNSUPPORTED;
   if (f.d_ff < 0) return COD_ERR_INVALID_ARG;
-  if (f.d_ff % 64) return COD_ERR_UNSUPPORTED;   // gate and up share one contraction: tiles must not straddle them
+  if (f.d_ff % 64) return COD_ERR_UNSUPPORTED;
+  if ((f.flags & COD_F_NO_CARRY_EMBED) && (f.flags & COD_F_REJ_PROJECTOR)) return COD_ERR_INVALID_ARG;
+  if ((f.flags & COD_F_REJ_PROJECTOR) && f.d_model % 64) return COD_ERR_UNSUPPORTED;   // F | F_rej share one contraction   // gate and up share one contraction: tiles must not straddle them
   if (static_cast<int64_t>(f.n_pages) * f.page_size > (1ll << 31) - 1) return COD_ERR_UNSUPPORTED;
 
   cod_ctx* c = new (std::nothrow) cod_ctx();
@@ -238,6 +241,7 @@ int cod_set_weights(cod_ctx* c, const cod_weights* w, cod_stream_t stream) {
   if (c->cfg.flags & COD_F_QK_NORM)
     for (const void* p : {w->g_qnorm, w->g_knorm})
       if (!p || misaligned(p)) return COD_ERR_INVALID_ARG;
+  if ((c->cfg.flags & COD_F_REJ_PROJECTOR) && (!w->fc_rej || misaligned(w->fc_rej))) return COD_ERR_INVALID_ARG;
   c->w = *w;
   c->has_weights = true;
   c->pdl = false;
@@ -279,9 +283,13 @@ static int project_impl(cod_ctx* c, const void* H, const cod_split* sp, int S, i
   GemmArgs g{};
   g.A = H; g.lda = c->D_in; g.a_rows = nullptr; g.n_rows_dev = n_dev; g.n_rows = R; g.K = c->D_in;
   g.seg[0] = {c->w.fc, c->D}; g.n_seg = 1; g.klass = COD_K_FC;
-  g.C = c->gemm_out; g.ldc = c->D; g.splits = pick_splits(c, c->D, c->D_in, R);
+  // separate-projector variant, carry mode: F h and F_rej h of every row from one two-segment contraction,
+  // the finish kernel keeps the one the row's status selects (the baseline keeps accepted rows only: F alone)
+  const bool two = (f.flags & COD_F_REJ_PROJECTOR) && mode == COD_CARRY;
+  if (two) { g.seg[1] = {c->w.fc_rej, c->D}; g.n_seg = 2; }
+  g.C = c->gemm_out; g.ldc = two ? 2 * c->D : c->D; g.splits = pick_splits(c, g.ldc, c->D_in, R);
   if ((rc = cod_launch_gemm(c, g, st)) != COD_OK) return rc;
-  if ((rc = cod_launch_fc_finish(c, c->gemm_out, g.splits, R, n_dev, a_rows, sp->carry_slot, tap_z, st)) != COD_OK)
+  if ((rc = cod_launch_fc_finish(c, c->gemm_out, g.splits, R, n_dev, a_rows, sp->carry_slot, tap_z, st, g.ldc)) != COD_OK)
     return rc;
 
   GemmArgs k{};

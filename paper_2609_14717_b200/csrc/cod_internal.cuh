@@ -230,7 +230,7 @@ int cod_launch_fcE(cod_ctx* c, cudaStream_t st);
 int cod_launch_gather_rows(cod_ctx* c, const void* src, const int* rows, const int* n_dev, int n_max, int width,
                            void* dst, cudaStream_t st);
 int cod_launch_fc_finish(cod_ctx* c, const float* part, int splits, int n_rows, const int* n_rows_dev,
-                         const int* a_rows, const int* carry_slot, float* tap_z, cudaStream_t st);
+                         const int* a_rows, const int* carry_slot, float* tap_z, cudaStream_t st, int ldp = 0);   // ldp: row stride of part (0 = D; 2 D = F h | F_rej h)
 // dest_state == nullptr: write J; else write the pool / carry slot directly
 int cod_launch_kv_finish(cod_ctx* c, const float* part, int splits, int n_rows, const int* n_rows_dev,
                          const int* a_rows, const cod_split* sp, void* J, const cod_state* dest_state,

@@ -68,7 +68,7 @@ template <typename T, int NV>
 __global__ void __launch_bounds__(1024) k_fc_finish(const float* __restrict__ part, int splits, int n_rows, const int* n_rows_dev,
                             const int* __restrict__ a_rows, const int* __restrict__ carry_slot,
                             const float* __restrict__ fcE, const T* __restrict__ gain, int D, float eps,
-                            int do_norm, T* __restrict__ z, int z_compact, float* __restrict__ tap) {
+                            int do_norm, T* __restrict__ z, int z_compact, float* __restrict__ tap, int ldp) {
   cod_pdl_prologue();
   __shared__ float red[33];
   const int i = blockIdx.x;
@@ -82,14 +82,16 @@ __global__ void __launch_bounds__(1024) k_fc_finish(const float* __restrict__ pa
   for (int t = 0; t < NV; ++t) {
     const int j = threadIdx.x + t * blockDim.x;
     v[t] = make_float4(0.f, 0.f, 0.f, 0.f);
-    if (j < nv && rej) v[t] = *reinterpret_cast<const float4*>(fcE + 4 * j);
+    if (j < nv && rej && fcE != nullptr) v[t] = *reinterpret_cast<const float4*>(fcE + 4 * j);
   }
+  // ldp = D: one projection per row. ldp = 2 D: F h and F_rej h side by side, rejected rows take the second.
+  const float* prow = part + static_cast<size_t>(i) * ldp + ((ldp > D && rej) ? D : 0);
 #pragma unroll 4
   for (int s = 0; s < splits; ++s) {        // slots inside, four slabs unrolled: their loads are all in flight together
 #pragma unroll
     for (int t = 0; t < NV; ++t) {
       const int j = threadIdx.x + t * blockDim.x;
-      if (j < nv) v[t] = f4_add(v[t], *reinterpret_cast<const float4*>(part + (static_cast<size_t>(s) * n_rows + i) * D + 4 * j));
+      if (j < nv) v[t] = f4_add(v[t], *reinterpret_cast<const float4*>(prow + static_cast<size_t>(s) * n_rows * ldp + 4 * j));
     }
   }
 #pragma unroll
@@ -465,19 +467,22 @@ int cod_launch_fcE(cod_ctx* c, cudaStream_t st) {
 }
 
 int cod_launch_fc_finish(cod_ctx* c, const float* part, int splits, int n_rows, const int* n_rows_dev,
-                         const int* a_rows, const int* carry_slot, float* tap_z, cudaStream_t st) {
+                         const int* a_rows, const int* carry_slot, float* tap_z, cudaStream_t st, int ldp) {
   ProfScope prof(c, COD_K_ROWOPS, st);
   if (n_rows <= 0) return COD_OK;
   const int nt = row_threads(c->D);
   const int do_norm = (c->cfg.flags & COD_F_HIDDEN_NORM) ? 1 : 0;
+  // F(E_carry) is added to rejected rows only in the embedding variant
+  const float* fcE = (c->cfg.flags & (COD_F_NO_CARRY_EMBED | COD_F_REJ_PROJECTOR)) ? nullptr : c->fcE;
+  if (ldp <= 0) ldp = c->D;
   if (row_narrow(c->D)) {
     DISPATCH_T(c,
-               (cod_launch_pdl(c, k_fc_finish<__nv_bfloat16, 1>, n_rows, nt, 0, st, part, splits, n_rows, n_rows_dev, a_rows, carry_slot, c->fcE, static_cast<const __nv_bfloat16*>(c->w.g_hidden), c->D, c->cfg.rms_eps, do_norm, static_cast<__nv_bfloat16*>(c->z), a_rows ? 1 : 0, tap_z)),
-               (cod_launch_pdl(c, k_fc_finish<float, 1>, n_rows, nt, 0, st, part, splits, n_rows, n_rows_dev, a_rows, carry_slot, c->fcE, static_cast<const float*>(c->w.g_hidden), c->D, c->cfg.rms_eps, do_norm, static_cast<float*>(c->z), a_rows ? 1 : 0, tap_z)));
+               (cod_launch_pdl(c, k_fc_finish<__nv_bfloat16, 1>, n_rows, nt, 0, st, part, splits, n_rows, n_rows_dev, a_rows, carry_slot, fcE, static_cast<const __nv_bfloat16*>(c->w.g_hidden), c->D, c->cfg.rms_eps, do_norm, static_cast<__nv_bfloat16*>(c->z), a_rows ? 1 : 0, tap_z, ldp)),
+               (cod_launch_pdl(c, k_fc_finish<float, 1>, n_rows, nt, 0, st, part, splits, n_rows, n_rows_dev, a_rows, carry_slot, fcE, static_cast<const float*>(c->w.g_hidden), c->D, c->cfg.rms_eps, do_norm, static_cast<float*>(c->z), a_rows ? 1 : 0, tap_z, ldp)));
   } else {
     DISPATCH_T(c,
-               (cod_launch_pdl(c, k_fc_finish<__nv_bfloat16, ROW_WIDE_NV>, n_rows, nt, 0, st, part, splits, n_rows, n_rows_dev, a_rows, carry_slot, c->fcE, static_cast<const __nv_bfloat16*>(c->w.g_hidden), c->D, c->cfg.rms_eps, do_norm, static_cast<__nv_bfloat16*>(c->z), a_rows ? 1 : 0, tap_z)),
-               (cod_launch_pdl(c, k_fc_finish<float, ROW_WIDE_NV>, n_rows, nt, 0, st, part, splits, n_rows, n_rows_dev, a_rows, carry_slot, c->fcE, static_cast<const float*>(c->w.g_hidden), c->D, c->cfg.rms_eps, do_norm, static_cast<float*>(c->z), a_rows ? 1 : 0, tap_z)));
+               (cod_launch_pdl(c, k_fc_finish<__nv_bfloat16, ROW_WIDE_NV>, n_rows, nt, 0, st, part, splits, n_rows, n_rows_dev, a_rows, carry_slot, fcE, static_cast<const __nv_bfloat16*>(c->w.g_hidden), c->D, c->cfg.rms_eps, do_norm, static_cast<__nv_bfloat16*>(c->z), a_rows ? 1 : 0, tap_z, ldp)),
+               (cod_launch_pdl(c, k_fc_finish<float, ROW_WIDE_NV>, n_rows, nt, 0, st, part, splits, n_rows, n_rows_dev, a_rows, carry_slot, fcE, static_cast<const float*>(c->w.g_hidden), c->D, c->cfg.rms_eps, do_norm, static_cast<float*>(c->z), a_rows ? 1 : 0, tap_z, ldp)));
   }
   COD_CHECK_LAUNCH(c);
   return COD_OK;

@@ -105,6 +105,10 @@ def _workloads():
         "small_bf16_full": small_bf16(S=3, W=16, n_layers=2, ctx=(40, 300), d_ff=768, qk_norm=True),
         "small_bf16_mlp_only": small_bf16(S=2, W=16, n_layers=2, ctx=(40, 300), d_ff=384),
         "small_bf16_qknorm_only": small_bf16(S=2, W=8, n_layers=2, ctx=(40, 300), qk_norm=True),
+        # the two other ways of marking rejected rows (Section 5): none at all, a separate projector
+        "small_bf16_nomark": small_bf16(S=3, W=16, n_layers=1, ctx=(40, 300), carry_variant="none"),
+        "small_bf16_proj": small_bf16(S=3, W=16, n_layers=2, ctx=(40, 300), carry_variant="projector"),
+        "tiny_f32_proj": synth.scaled(synth.workload("cfg1"), S=3, ctx=(5, 140), n_rounds=6, carry_variant="projector"),
         "mid_bf16_full": small_bf16(S=34, W=16, n_layers=2, ctx=(100, 600), d_target=512, n_cap=5, d_model=1024,
                                     n_q=8, n_kv=2, vocab=3000, d_ff=1536, qk_norm=True),
     }
@@ -327,7 +331,9 @@ def test_round_parity_cfg1_every_round():
     ("tiny_f32_full", 40.0, orc.MODE_CARRY), ("tiny_f32_full", 40.0, orc.MODE_BASELINE),
     ("small_bf16_full", 30.0, orc.MODE_CARRY), ("small_bf16_full", 30.0, orc.MODE_BASELINE),
     ("small_bf16_mlp_only", 30.0, orc.MODE_CARRY), ("small_bf16_qknorm_only", 30.0, orc.MODE_CARRY),
-    ("mid_bf16_full", 30.0, orc.MODE_CARRY)])
+    ("mid_bf16_full", 30.0, orc.MODE_CARRY),
+    ("small_bf16_nomark", 30.0, orc.MODE_CARRY), ("small_bf16_proj", 30.0, orc.MODE_CARRY),
+    ("small_bf16_proj", 30.0, orc.MODE_BASELINE), ("tiny_f32_proj", 40.0, orc.MODE_CARRY)])
 def test_round_parity_multi_round(name, wo_scale, mode):
     """Open-loop rounds (inputs pre-generated), ragged acceptance, attention path made to matter."""
     Hn = _H()
