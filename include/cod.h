@@ -13,6 +13,13 @@
  *   4. the next block ([bonus, MASK, ...]) attends to [C_l; U_l; block];
  *   5. the tied LM head with a fused argmax gives the next proposals.
  *
+ * Beyond that default round: the complete drafter layer (cod_config.d_ff,
+ * COD_F_QK_NORM), the round at temperature 1 (cod_verify_accept_stochastic,
+ * cod_lm_head_sample, cod_draft_round_stochastic), the two other ways of
+ * marking rejected rows the paper compares (COD_F_NO_CARRY_EMBED,
+ * COD_F_REJ_PROJECTOR) and two analysis aids (cod_taps.carry_mass,
+ * cod_reconvergence_count).
+ *
  * Conventions
  *   - Every function returns 0 (COD_OK) or a negative cod_status. Nothing throws.
  *   - "device" pointers are CUDA device addresses owned by the caller and only
@@ -20,7 +27,10 @@
  *   - All work is enqueued on the caller's stream (a cudaStream_t passed as
  *     void*); no call synchronises the host except cod_create, cod_destroy
  *     and cod_poll_status. Results are valid once the stream has been
- *     synchronised by the caller.
+ *     synchronised by the caller. For small rounds cod_draft_round also uses a
+ *     second stream owned by the context, forked from and joined back into the
+ *     caller's stream with events (under stream capture these become graph
+ *     edges); a context therefore serves one round at a time.
  *   - After cod_create the library allocates nothing (the workspace is sized
  *     from cod_config at creation).
  *   - What only the device can see (a position beyond the page table, a token
