@@ -67,6 +67,8 @@ class OracleConfig:
     hidden_norm: bool
     d_ff: int = 0            # > 0: every drafter layer has a gated MLP of this width
     qk_norm: bool = False    # per-head RMS norm of queries and keys before the rotation
+    carry_rounds: int = 1    # k: rejected rows are retained for k rounds (the paper uses and trains k = 1;
+                             # Section 6 names retention beyond one round as what different rollouts would allow)
     carry_variant: str = "embedding"   # "embedding": E_carry on rejected rows (Eq. 2, the paper's choice);
                                        # "none": rejected rows pass F unmarked; "projector": rejected rows
                                        # pass their own fusion map F_rej (Table 4(b)'s two alternatives)
@@ -85,7 +87,8 @@ class OracleState:
     """Committed drafter KV C_l (paged), carried KV U_l, and their lengths.
 
     pool  [Ld, n_pages, n_kv, 2, page, hd]   index 3: 0 = K (already rotated), 1 = V
-    carry [Ld, S, n_kv, 2, W, hd]            rows >= carry_len[s] are NaN (never to be read)
+    carry [Ld, S, n_kv, 2, k*W, hd]          rows >= carry_len[s] are NaN (never to be read)
+    carry_hist[s]                            lengths of the (at most k) rounds' segments held in U, oldest first
     """
 
     def __init__(self, cfg: OracleConfig, S: int, n_pages: int, block_table: np.ndarray,
@@ -95,7 +98,8 @@ class OracleState:
         self.pool = np.zeros((cfg.n_layers, n_pages, cfg.n_kv, 2, cfg.page, cfg.hd), dtype=np.float64)
         self.block_table = np.array(block_table, dtype=np.int64)
         self.committed_len = np.array(committed_len, dtype=np.int64)
-        self.carry = np.full((cfg.n_layers, S, cfg.n_kv, 2, cfg.W, cfg.hd), np.nan, dtype=np.float64)
+        self.carry = np.full((cfg.n_layers, S, cfg.n_kv, 2, cfg.carry_rounds * cfg.W, cfg.hd), np.nan, dtype=np.float64)
+        self.carry_hist = [[] for _ in range(S)]
         # Algorithm 1: "Initialize U_l = empty".
         self.carry_len = np.zeros(S, dtype=np.int64)
 
@@ -277,13 +281,28 @@ def scatter_kv(J: np.ndarray, split: Dict[str, np.ndarray], st: OracleState, mod
                 pg = int(st.block_table[s, pos // page])
                 st.pool[l, pg, :, 0, pos % page, :] = J[l, s * W + p, 0]
                 st.pool[l, pg, :, 1, pos % page, :] = J[l, s * W + p, 1]
-            st.carry[l, s] = np.nan                       # the previous U_l is gone
-            if mode == MODE_CARRY:
+            if mode != MODE_CARRY:
+                st.carry[l, s] = np.nan                   # the baseline column keeps no U at all
+        if mode == MODE_CARRY:
+            # U holds the rejected rows of the last k rounds, oldest first (k = 1: "U_l <- J_l rejected",
+            # the previous U discarded). A round that rejects nothing still ages the older segments.
+            c_old = int(st.carry_len[s])
+            hist = st.carry_hist[s][-(cfg.carry_rounds - 1):] if cfg.carry_rounds > 1 else []
+            keep = sum(hist)                              # rows of the k - 1 newest rounds, at the end of U
+            drop = c_old - keep
+            st.carry_hist[s] = hist + [W - m]
+            for l in range(cfg.n_layers):
+                kept = st.carry[l, s, :, :, drop:c_old, :].copy()
+                st.carry[l, s] = np.nan
+                st.carry[l, s, :, :, :keep, :] = kept
                 for p in range(m, W):
-                    st.carry[l, s, :, 0, p - m, :] = J[l, s * W + p, 0]
-                    st.carry[l, s, :, 1, p - m, :] = J[l, s * W + p, 1]
+                    st.carry[l, s, :, 0, keep + p - m, :] = J[l, s * W + p, 0]
+                    st.carry[l, s, :, 1, keep + p - m, :] = J[l, s * W + p, 1]
+            st.carry_len[s] = keep + (W - m)
+        else:
+            st.carry_hist[s] = []
+            st.carry_len[s] = 0
         st.committed_len[s] = L + m
-        st.carry_len[s] = (W - m) if mode == MODE_CARRY else 0
 
 
 # =========================================================================== part 4

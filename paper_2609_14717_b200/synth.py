@@ -53,6 +53,7 @@ class DrafterShape:
     d_ff: int = 0         # width of the gated MLP of a drafter layer; 0 = attention sub-layer only
     qk_norm: bool = False # per-head RMS norm (with gain) of queries and keys before the rotation
     carry_variant: str = "embedding"  # how rejected rows are told apart: "embedding" (E_carry), "none", "projector"
+    carry_rounds: int = 1 # rounds for which rejected rows stay in the carry slot (the paper's setting: 1)
 
     @property
     def d_in(self) -> int:

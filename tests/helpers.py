@@ -12,7 +12,7 @@ def oracle_config(sh: synth.DrafterShape) -> orc.OracleConfig:
         d_target=sh.d_target, n_cap=sh.n_cap, d_model=sh.d_model, n_layers=sh.n_layers,
         n_q=sh.n_q, n_kv=sh.n_kv, hd=sh.hd, vocab=sh.vocab, mask_token_id=sh.mask_token_id,
         W=sh.W, page=sh.page, rope_theta=sh.rope_theta, rms_eps=sh.rms_eps,
-        hidden_norm=sh.hidden_norm, d_ff=sh.d_ff, qk_norm=sh.qk_norm, carry_variant=sh.carry_variant)
+        hidden_norm=sh.hidden_norm, d_ff=sh.d_ff, qk_norm=sh.qk_norm, carry_variant=sh.carry_variant, carry_rounds=sh.carry_rounds)
 
 
 def oracle_state(wl: synth.Workload, seed: int, fill_pool: bool = True):

@@ -874,3 +874,48 @@ def test_carry_variants_relate_as_they_must():
     want = [sum(w["fc_rej"][i, k] * float(rd["H"][r, k]) for k in range(base.shape.d_in)) for i in range(4)]
     assert np.allclose(Z_p[r, :4], want, atol=1e-12)
 
+
+# ----------------------------------------------------------------------------- retention beyond one round
+def test_carry_retention_holds_exactly_the_last_k_rounds_in_order():
+    """After every round U must be the rejected rows of the last k rounds, oldest first, each row
+    equal to the K/V the projection made for it in ITS round (positions kept)."""
+    for k in (1, 2, 3):
+        wl = synth.scaled(synth.workload("cfg1"), S=2, ctx=(10, 40), carry_rounds=k, n_rounds=8)
+        cfg, st, _ = oracle_state(wl, 9)
+        w = orc.prepare_weights(synth.make_weights(wl.shape, 9))
+        segs = [[], []]                                   # per sequence: list of (K rows, V rows) per round
+        for r in range(6):
+            rd = synth.make_round(wl, 9, r)
+            res = orc.draft_round(rd["draft"], rd["target"], rd["H"], st, w, 1, orc.MODE_CARRY)
+            for s in range(2):
+                m = int(res["split"]["accept_len"][s])
+                rows = slice(s * cfg.W + m, (s + 1) * cfg.W)
+                segs[s].append(res["J"][:, rows])            # [Ld, W - m, 2, n_kv, hd]
+                want = np.concatenate(segs[s][-k:], axis=1)
+                c = int(st.carry_len[s])
+                assert c == want.shape[1] == sum(st.carry_hist[s]) and len(st.carry_hist[s]) <= k
+                got = np.transpose(st.carry[:, s, :, :, :c, :], (0, 3, 2, 1, 4))       # -> [Ld, c, 2, n_kv, hd]
+                assert np.array_equal(got, want)
+                assert np.isnan(st.carry[:, s, :, :, c:, :]).all()
+        assert max(int(x) for x in st.carry_len) <= k * cfg.W
+
+
+def test_retained_rows_change_the_next_draft_and_k1_is_the_papers_round():
+    wl1 = synth.scaled(synth.workload("cfg1"), S=2, ctx=(10, 40), n_rounds=6)
+    wl2 = synth.scaled(wl1, carry_rounds=2)
+    w = orc.prepare_weights(synth.make_weights(wl1.shape, 4))
+    w["wo"] = w["wo"] * 40.0
+    _, st1, _ = oracle_state(wl1, 4)
+    _, st2, _ = oracle_state(wl2, 4)
+    differs = False
+    for r in range(4):
+        rd = synth.make_round(wl1, 4, r)
+        a = orc.draft_round(rd["draft"], rd["target"], rd["H"], st1, w, 1, orc.MODE_CARRY)
+        b = orc.draft_round(rd["draft"], rd["target"], rd["H"], st2, w, 1, orc.MODE_CARRY)
+        assert np.array_equal(st1.pool, st2.pool)                      # the committed cache never depends on U
+        if r == 0:
+            assert np.array_equal(a["x_final"], b["x_final"])          # nothing older to retain yet
+        else:
+            differs |= np.abs(a["x_final"] - b["x_final"]).max() > 1e-6
+    assert differs
+
