@@ -107,6 +107,9 @@ typedef struct {
   int32_t d_ff;              /* width of the gated MLP that follows the attention sub-layer of every
                                 drafter layer (a multiple of 64); 0 = no MLP. The paper leaves the
                                 drafter body open (Section 2.1); this is the complete-layer reading  */
+  int32_t carry_rounds;      /* k: rounds for which rejected rows stay in the carry slot (0 or 1: the paper's
+                                one-round slot; k > 1: U_l = the rejected rows of the last k rounds, oldest
+                                first - the retention beyond a single round that Section 6 leaves open)   */
 } cod_config;
 
 /* Borrowed device pointers, element type per cod_config.dtype, each matrix [out, in]. */
@@ -136,8 +139,10 @@ typedef struct {
   void* kv_pool;          /* [Ld][n_pages][n_kv][2][page][hd]  C_l; index 3: 0 = K (rotated), 1 = V */
   int32_t* block_table;   /* [S][max_pages_per_seq]            physical page of each logical page  */
   int32_t* committed_len; /* [S]   L_s; cod_scatter_kv adds the accepted rows                      */
-  void* carry_kv;         /* [Ld][max_batch][n_kv][2][W][hd]   U_l (rows >= carry_len are stale)   */
-  int32_t* carry_len;     /* [S]   c_s in 0..W, overwritten every round                            */
+  void* carry_kv;         /* [Ld][max_batch][n_kv][2][k*W][hd] U_l (rows >= carry_len are stale)   */
+  int32_t* carry_len;     /* [S]   c_s in 0..k*W, overwritten every round                          */
+  int32_t* carry_hist;    /* [S][k] carry_rounds = k > 1 only (else may be NULL): lengths of the k
+                                    newest rounds' segments of U_l, oldest first; starts as zeros   */
 } cod_state;
 
 /* Output of cod_verify_accept (device, caller-owned). Row ids are s*W + p. */

@@ -39,7 +39,7 @@ class CodConfig(C.Structure):
         "d_target", "n_cap", "d_model", "n_layers", "n_q_heads", "n_kv_heads", "head_dim", "vocab",
         "mask_token_id", "block", "page_size", "max_batch", "max_pages_per_seq", "n_pages", "dtype")] + [
         ("flags", C.c_uint32), ("rope_theta", C.c_float), ("rms_eps", C.c_float),
-        ("attn_split_len", C.c_int32), ("d_ff", C.c_int32)]
+        ("attn_split_len", C.c_int32), ("d_ff", C.c_int32), ("carry_rounds", C.c_int32)]
 
 
 _WEIGHT_FIELDS = ("fc", "e_carry", "g_hidden", "wk", "wv", "wq", "wo", "g_attn", "g_final", "emb",
@@ -47,7 +47,7 @@ _WEIGHT_FIELDS = ("fc", "e_carry", "g_hidden", "wk", "wv", "wq", "wo", "g_attn",
                   "fc_rej")                                                     # separate-projector variant only
 _SPLIT_FIELDS = ("accept_len", "bonus", "row_pos", "commit_slot", "carry_slot", "acc_rows", "acc_off",
                  "rej_rows", "rej_off")
-_STATE_FIELDS = ("kv_pool", "block_table", "committed_len", "carry_kv", "carry_len")
+_STATE_FIELDS = ("kv_pool", "block_table", "committed_len", "carry_kv", "carry_len", "carry_hist")
 _TAP_FIELDS = ("z", "attn_out", "x_final", "top_logit", "carry_mass")
 
 
@@ -177,9 +177,11 @@ class State:
                                    dtype=td, device=device)
         self.block_table = torch.from_numpy(np.ascontiguousarray(block_table, dtype=np.int32)).to(device)
         self.committed_len = torch.from_numpy(np.ascontiguousarray(committed_len, dtype=np.int32)).to(device)
-        self.carry_kv = torch.zeros((cfg.n_layers, cfg.max_batch, cfg.n_kv_heads, 2, cfg.block, cfg.head_dim),
+        k = max(1, int(cfg.carry_rounds))                       # rounds of rejected rows the carry slot holds
+        self.carry_kv = torch.zeros((cfg.n_layers, cfg.max_batch, cfg.n_kv_heads, 2, k * cfg.block, cfg.head_dim),
                                     dtype=td, device=device)
         self.carry_len = torch.zeros(S, dtype=torch.int32, device=device)
+        self.carry_hist = torch.zeros((S, k), dtype=torch.int32, device=device) if k > 1 else None
 
     def struct(self) -> CodState:
         return CodState(*[_ptr(getattr(self, n)) for n in _STATE_FIELDS])
@@ -337,7 +339,7 @@ def make_config(sh, max_batch: int, max_pages_per_seq: int, n_pages: int, attn_s
         | (COD_F_QK_NORM if sh.qk_norm else 0)
         | {"embedding": 0, "none": COD_F_NO_CARRY_EMBED, "projector": COD_F_REJ_PROJECTOR}[sh.carry_variant],
         rope_theta=sh.rope_theta, rms_eps=sh.rms_eps,
-        attn_split_len=attn_split_len, d_ff=sh.d_ff)
+        attn_split_len=attn_split_len, d_ff=sh.d_ff, carry_rounds=sh.carry_rounds)
 
 
 def weights_to_device(w: Dict[str, np.ndarray], dtype: str) -> Dict[str, torch.Tensor]:

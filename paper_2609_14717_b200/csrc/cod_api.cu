@@ -61,6 +61,10 @@ size_t carve(cod_ctx* c) {
   cv.take(c->zero_page, 4096);
   cv.take(c->attn_o, sizeof(float) * parts * f.head_dim);
   cv.take(c->attn_ml, sizeof(float) * parts * 4);
+  if (c->carry_cap > f.block) {
+    cv.take(c->carry_base, sizeof(int) * f.max_batch);
+    cv.take(c->carry_drop, sizeof(int) * f.max_batch);
+  }
   cv.take(c->amax, sizeof(unsigned long long) * R);
   cv.take(c->lse_part, sizeof(float2) * R * ((static_cast<size_t>(f.vocab) + 127) / 128));
   cv.take(c->tok, sizeof(int32_t) * R);
@@ -103,6 +107,8 @@ int pick_splits(const cod_ctx* c, int n_out, int K, int rows) {
   return (kb + per - 1) / per;            // no empty split
 }
 
+bool hist_missing(const cod_ctx* c, const cod_state* s) { return c->carry_cap > c->cfg.block && !s->carry_hist; }
+
 int check_S(const cod_ctx* c, int S) { return (S >= 1 && S <= c->cfg.max_batch) ? COD_OK : COD_ERR_INVALID_ARG; }
 
 }  // namespace
@@ -141,7 +147,7 @@ int cod_create(const cod_config* cfg, cod_ctx** out) {
   if (f.block > COD_MAX_W || f.block * (f.n_q_heads / f.n_kv_heads) > 128) return COD_ERR_UNSUPPORTED;
   if ((f.d_target * f.n_cap) % 8 || f.d_model % 8 || f.d_model > 32768) return COD_ERR_UNSUPPORTED;
   if ((f.n_kv_heads * f.head_dim) % 64) return COD_ERR_UNSUPPORTED;
-  if (f.d_ff < 0) return COD_ERR_INVALID_ARG;
+  if (f.d_ff < 0 || f.carry_rounds < 0 || f.carry_rounds > 8) return COD_ERR_INVALID_ARG;
   if (f.d_ff % 64) return COD_ERR_UNSUPPORTED;
   if ((f.flags & COD_F_NO_CARRY_EMBED) && (f.flags & COD_F_REJ_PROJECTOR)) return COD_ERR_INVALID_ARG;
   if ((f.flags & COD_F_REJ_PROJECTOR) && f.d_model % 64) return COD_ERR_UNSUPPORTED;   // F | F_rej share one contraction   // gate and up share one contraction: tiles must not straddle them
@@ -159,9 +165,10 @@ int cod_create(const cod_config* cfg, cod_ctx** out) {
   c->R_max = f.max_batch * f.block;
   c->half = f.head_dim / 2;
   c->force_simt = (f.flags & COD_F_NO_TENSOR_CORES) != 0;
+  c->carry_cap = (f.carry_rounds > 1 ? f.carry_rounds : 1) * f.block;
   if (cudaDeviceGetAttribute(&c->n_sm, cudaDevAttrMultiProcessorCount, c->device) != cudaSuccess || c->n_sm < 1) c->n_sm = 148;
   c->split_len = f.attn_split_len > 0 ? f.attn_split_len : 512;
-  const int64_t max_keys = static_cast<int64_t>(f.max_pages_per_seq) * f.page_size + 2 * f.block;
+  const int64_t max_keys = static_cast<int64_t>(f.max_pages_per_seq) * f.page_size + c->carry_cap + f.block;
   c->max_splits = static_cast<int>((max_keys + c->split_len - 1) / c->split_len);
 
   {
@@ -319,8 +326,10 @@ int cod_scatter_kv(cod_ctx* c, const void* J, const cod_split* split, int S, int
   if (check_S(c, S) != COD_OK || (mode != COD_CARRY && mode != COD_BASELINE)) return COD_ERR_INVALID_ARG;
   cudaStream_t s = static_cast<cudaStream_t>(stream);
   c->pdl = true;
-  int rc = cod_launch_scatter(c, J, split, S, mode, st, s);
-  if (rc != COD_OK) return rc;
+  if (hist_missing(c, st)) return COD_ERR_INVALID_ARG;
+  int rc = COD_OK;
+  if (c->carry_base && (rc = cod_launch_carry_age(c, split, S, mode, st, s)) != COD_OK) return rc;
+  if ((rc = cod_launch_scatter(c, J, split, S, mode, st, s)) != COD_OK) return rc;
   return cod_launch_update_lens(c, split, S, mode, st, s);
 }
 
@@ -383,6 +392,11 @@ static int round_impl(cod_ctx* c, const int32_t* draft, const int32_t* target, c
 
   // part 1
   if ((rc = cod_launch_verify(c, draft, target, S, n_forced, st, sp, s, p_tok, q_tok, u)) != COD_OK) return rc;
+
+  // retention beyond one round: the oldest round leaves U and the kept rows move to the front before
+  // this round's rejected rows are written behind them
+  if (hist_missing(c, st)) return COD_ERR_INVALID_ARG;
+  if (c->carry_base && (rc = cod_launch_carry_age(c, sp, S, mode, st, s)) != COD_OK) return rc;
 
   // The first layer's embedding + Q/K/V chain of the NEXT block needs only the bonus tokens and the
   // position tables of part 1; the context projection (parts 2-3) needs only the row split. For

@@ -140,6 +140,9 @@ struct cod_ctx {
   void* hmid;                  // [R, d_ff] activated MLP rows (storage type), d_ff > 0 only
   float2* lse_part;            // [ceil(vocab / 128)][R] soft-max partials of the sampling LM head
   float* gemm_out;             // split-K / unfused GEMM results
+  int carry_cap;               // rows of one (layer, sequence, head, K|V) carry slot: carry_rounds * block
+  int* carry_base;             // [max_batch] rows of U kept from earlier rounds (carry_rounds > 1), else null
+  int* carry_drop;             // [max_batch] rows of U that leave this round (carry_rounds > 1), else null
   float* gemm_out2;            // a second, small slab buffer for the side branch of the round (null: no side branch)
   int side_rows;               // the side branch is used for rounds of at most this many rows
   cudaStream_t side;           // side branch of the round: the first layer's embedding / Q/K/V chain
@@ -225,6 +228,8 @@ int cod_launch_reconvergence(cod_ctx* c, const int32_t* z, const int32_t* y, con
 int cod_launch_finalize_sample(cod_ctx* c, int R, uint32_t state, int32_t* tok, float* q_tok, float* lse,
                                cudaStream_t st, const int32_t* bonus = nullptr, int32_t* next_draft = nullptr);
 uint32_t cod_sample_state(unsigned long long seed, uint32_t step);   // hash state after seed and step
+// carry_rounds > 1: drops the oldest round's rows of U, moves the kept ones to the front, shifts the history
+int cod_launch_carry_age(cod_ctx* c, const cod_split* sp, int S, int mode, const cod_state* st, cudaStream_t stream);
 int cod_launch_rope_blk_only(cod_ctx* c, const int32_t* committed_len, int S, cudaStream_t st);
 int cod_launch_fcE(cod_ctx* c, cudaStream_t st);
 int cod_launch_gather_rows(cod_ctx* c, const void* src, const int* rows, const int* n_dev, int n_max, int width,

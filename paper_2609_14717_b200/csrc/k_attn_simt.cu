@@ -22,7 +22,7 @@ k_attn_split(const T* __restrict__ q, const T* __restrict__ kb, const T* __restr
              const int* __restrict__ committed_len, const int* __restrict__ carry_len, int use_carry,
              int layer, int W, int rep, int n_kv, int page, int max_pages, int n_pages, int max_batch,
              int split_len, int max_splits, float* __restrict__ part_o, float* __restrict__ part_ml,
-             uint32_t* status) {
+             uint32_t* status, int cap /* rows of a carry slot */) {
   cod_pdl_prologue();
   extern __shared__ float smem[];
   const int M = W * rep;
@@ -35,7 +35,7 @@ k_attn_split(const T* __restrict__ q, const T* __restrict__ kb, const T* __restr
   int c = use_carry ? carry_len[s] : 0;
   uint32_t flags = 0;
   if (L < 0 || L > max_pages * page) { flags |= COD_DEV_BAD_LEN; L = max(0, min(L, max_pages * page)); }
-  if (c < 0 || c > W) { flags |= COD_DEV_BAD_LEN; c = max(0, min(c, W)); }
+  if (c < 0 || c > cap) { flags |= COD_DEV_BAD_LEN; c = max(0, min(c, cap)); }
   const int T_total = L + c + W;
   const int t0 = k * split_len;
   if (t0 >= T_total) return;
@@ -77,8 +77,8 @@ k_attn_split(const T* __restrict__ q, const T* __restrict__ kb, const T* __restr
           kp = pool + ((((static_cast<size_t>(layer) * n_pages + pg) * n_kv + h) * 2) * page + tt % page) * HD;
           vp = kp + static_cast<size_t>(page) * HD;
         } else if (tt < L + c) {
-          kp = carry + ((((static_cast<size_t>(layer) * max_batch + s) * n_kv + h) * 2) * W + (tt - L)) * HD;
-          vp = kp + static_cast<size_t>(W) * HD;
+          kp = carry + ((((static_cast<size_t>(layer) * max_batch + s) * n_kv + h) * 2) * cap + (tt - L)) * HD;
+          vp = kp + static_cast<size_t>(cap) * HD;
         } else {
           const int i = tt - L - c;
           kp = kb + static_cast<size_t>(s * W + i) * kvw + h * HD;
@@ -157,7 +157,7 @@ __global__ void k_attn_combine(const float* __restrict__ part_o, const float* __
                                const int* __restrict__ committed_len, const int* __restrict__ carry_len,
                                int use_carry, int S, int W, int rep, int n_kv, int page, int max_pages,
                                int split_len, int max_splits, T* __restrict__ out, float* __restrict__ tap,
-                               float* __restrict__ mass) {
+                               float* __restrict__ mass, int cap) {
   cod_pdl_prologue();
   const int lane = threadIdx.x & 31;
   const int item = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);   // (s, i, g)
@@ -166,7 +166,7 @@ __global__ void k_attn_combine(const float* __restrict__ part_o, const float* __
   const int g = item % n_q, i = (item / n_q) % W, s = item / (n_q * W);
   const int h = g / rep, mrow = i * rep + (g - h * rep), M = W * rep;
   const int L = max(0, min(committed_len[s], max_pages * page));
-  const int c = use_carry ? max(0, min(carry_len[s], W)) : 0;
+  const int c = use_carry ? max(0, min(carry_len[s], cap)) : 0;
   const int n_splits = (L + c + W + split_len - 1) / split_len;
   const size_t base = (static_cast<size_t>(s) * n_kv + h) * max_splits;
 
@@ -210,7 +210,7 @@ int launch_split(cod_ctx* c, int layer, const void* q, const void* kb, const voi
                                        static_cast<const T*>(stt->kv_pool), static_cast<const T*>(stt->carry_kv),
                                        stt->block_table, stt->committed_len, stt->carry_len, use_carry, layer, f.block,
                                        rep, f.n_kv_heads, f.page_size, f.max_pages_per_seq, f.n_pages, f.max_batch,
-                                       c->split_len, c->max_splits, c->attn_o, c->attn_ml, c->status);
+                                       c->split_len, c->max_splits, c->attn_o, c->attn_ml, c->status, c->carry_cap);
   COD_CHECK_LAUNCH(c);
   return COD_OK;
 }
@@ -230,7 +230,7 @@ int launch_all(cod_ctx* c, int layer, const void* q, const void* kb, const void*
   cod_launch_pdl(c, k_attn_combine<T, HD>, (items + 3) / 4, 128, 0, st, c->attn_o, c->attn_ml, stt->committed_len, stt->carry_len,
                                                          use_carry, S, f.block, rep, f.n_kv_heads, f.page_size,
                                                          f.max_pages_per_seq, c->split_len, c->max_splits,
-                                                         static_cast<T*>(out), tap, mass);
+                                                         static_cast<T*>(out), tap, mass, c->carry_cap);
   COD_CHECK_LAUNCH(c);
   return COD_OK;
 }

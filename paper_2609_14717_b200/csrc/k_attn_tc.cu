@@ -36,6 +36,7 @@ struct AttnParams {
   const __nv_bfloat16 *pool, *carry;
   const int *block_table, *committed_len, *carry_len;
   int use_carry, layer, W, rep, n_kv, n_pages, max_pages, max_batch;
+  int cap;                              // rows of a carry slot (retention rounds * W)
   int split_len;                        // keys of the paged region per CTA (multiple of 128)
   int max_parts;                        // partial slots per (sequence, KV head)
   float* part_o;                        // [S][n_kv][max_parts][M][hd]
@@ -94,7 +95,7 @@ k_attn_tc(const __grid_constant__ CUtensorMap map_pool, const __grid_constant__ 
   int L = p.committed_len[s];
   int c = p.use_carry ? p.carry_len[s] : 0;
   if (L < 0 || L > p.max_pages * PAGE) { flags |= COD_DEV_BAD_LEN; L = max(0, min(L, p.max_pages * PAGE)); }
-  if (c < 0 || c > p.W) { flags |= COD_DEV_BAD_LEN; c = max(0, min(c, p.W)); }
+  if (c < 0 || c > p.cap) { flags |= COD_DEV_BAD_LEN; c = max(0, min(c, p.cap)); }
   const int F = (L / PAGE) * PAGE;                       // keys held in whole pages
   const int n_reg = (F + p.split_len - 1) / p.split_len; // CTAs over the paged region
   if (split > n_reg) return;
@@ -282,7 +283,7 @@ k_attn_tc(const __grid_constant__ CUtensorMap map_pool, const __grid_constant__ 
                 if (pg < 0 || pg >= p.n_pages) { flags |= COD_DEV_BAD_PAGE; }
                 else src = p.pool + ((((static_cast<size_t>(p.layer) * p.n_pages + pg) * p.n_kv + h) * 2 + kv) * PAGE + g) * HD;
               } else if (g < Lr + c) {
-                src = p.carry + ((((static_cast<size_t>(p.layer) * p.max_batch + s) * p.n_kv + h) * 2 + kv) * p.W + (g - Lr)) * HD;
+                src = p.carry + ((((static_cast<size_t>(p.layer) * p.max_batch + s) * p.n_kv + h) * 2 + kv) * p.cap + (g - Lr)) * HD;
               } else if (g < n_tail) {
                 src = (kv ? p.vb : p.kb) + static_cast<size_t>(s * p.W + (g - Lr - c)) * (p.n_kv * HD) + h * HD;
               }
@@ -506,6 +507,7 @@ int launch(cod_ctx* c, int layer, const void* q, const void* kb, const void* vb,
   p.q = static_cast<const __nv_bfloat16*>(q); p.kb = static_cast<const __nv_bfloat16*>(kb); p.vb = static_cast<const __nv_bfloat16*>(vb);
   p.pool = static_cast<const __nv_bfloat16*>(stt->kv_pool); p.carry = static_cast<const __nv_bfloat16*>(stt->carry_kv);
   p.block_table = stt->block_table; p.committed_len = stt->committed_len; p.carry_len = stt->carry_len;
+  p.cap = c->carry_cap;
   p.use_carry = use_carry; p.layer = layer; p.W = f.block; p.rep = f.n_q_heads / f.n_kv_heads; p.n_kv = f.n_kv_heads;
   p.n_pages = f.n_pages; p.max_pages = f.max_pages_per_seq; p.max_batch = f.max_batch;
   p.split_len = c->tc_split_len; p.max_parts = c->tc_max_parts;

@@ -123,7 +123,8 @@ __global__ void k_kv_finish(const float* __restrict__ part, int splits, int n_ro
                             int n_kv, int hd, T* __restrict__ J, int R_total,
                             const int* __restrict__ commit_slot, const int* __restrict__ carry_slot,
                             T* __restrict__ pool, T* __restrict__ carry, int page, int n_pages, int W,
-                            int max_batch, int to_state, const T* __restrict__ g_k, float eps) {
+                            int max_batch, int to_state, const T* __restrict__ g_k, float eps, int cap,
+                            const int* __restrict__ carry_base) {
   cod_pdl_prologue();
   const int i = blockIdx.x, l = blockIdx.y;
   if (i >= valid_rows(n_rows_dev, n_rows)) return;
@@ -145,10 +146,11 @@ __global__ void k_kv_finish(const float* __restrict__ part, int splits, int n_ro
       h_stride = static_cast<size_t>(2) * page * hd;
       kv_stride = static_cast<size_t>(page) * hd;
     } else if (uslot >= 0 && carry) {
-      const int s = uslot / W, u = uslot - s * W;
-      dstK = carry + (((static_cast<size_t>(l) * max_batch + s) * n_kv) * 2) * W * hd + static_cast<size_t>(u) * hd;
-      h_stride = static_cast<size_t>(2) * W * hd;
-      kv_stride = static_cast<size_t>(W) * hd;
+      // a carry slot holds cap = k * W rows; the new round's rows follow the carry_base[s] retained ones
+      const int s = uslot / W, u = uslot - s * W + (carry_base ? carry_base[s] : 0);
+      dstK = carry + (((static_cast<size_t>(l) * max_batch + s) * n_kv) * 2) * cap * hd + static_cast<size_t>(u) * hd;
+      h_stride = static_cast<size_t>(2) * cap * hd;
+      kv_stride = static_cast<size_t>(cap) * hd;
     } else {
       return;   // nowhere to go (position beyond the page table: already flagged)
     }
@@ -197,7 +199,7 @@ template <typename T>
 __global__ void k_scatter_kv(const T* __restrict__ J, int R_total, int n_kv, int hd,
                              const int* __restrict__ commit_slot, const int* __restrict__ carry_slot,
                              T* __restrict__ pool, T* __restrict__ carry, int page, int n_pages, int W,
-                             int max_batch, int use_carry) {
+                             int max_batch, int use_carry, int cap, const int* __restrict__ carry_base) {
   cod_pdl_prologue();
   const int row = blockIdx.x, l = blockIdx.y;
   const int kvw = n_kv * hd;
@@ -210,10 +212,10 @@ __global__ void k_scatter_kv(const T* __restrict__ J, int R_total, int n_kv, int
     h_stride = static_cast<size_t>(2) * page * hd;
     kv_stride = static_cast<size_t>(page) * hd;
   } else if (uslot >= 0 && use_carry) {
-    const int s = uslot / W, u = uslot - s * W;
-    dst = carry + (((static_cast<size_t>(l) * max_batch + s) * n_kv) * 2) * W * hd + static_cast<size_t>(u) * hd;
-    h_stride = static_cast<size_t>(2) * W * hd;
-    kv_stride = static_cast<size_t>(W) * hd;
+    const int s = uslot / W, u = uslot - s * W + (carry_base ? carry_base[s] : 0);
+    dst = carry + (((static_cast<size_t>(l) * max_batch + s) * n_kv) * 2) * cap * hd + static_cast<size_t>(u) * hd;
+    h_stride = static_cast<size_t>(2) * cap * hd;
+    kv_stride = static_cast<size_t>(cap) * hd;
   } else {
     return;
   }
@@ -229,7 +231,8 @@ __global__ void k_scatter_kv(const T* __restrict__ J, int R_total, int n_kv, int
 }
 
 __global__ void k_update_lens(const int* __restrict__ accept_len, int S, int W, int mode, int max_tokens,
-                              int* __restrict__ committed_len, int* __restrict__ carry_len, uint32_t* status) {
+                              int* __restrict__ committed_len, int* __restrict__ carry_len, uint32_t* status,
+                              const int* __restrict__ carry_base) {
   cod_pdl_prologue();
   const int s = blockIdx.x * blockDim.x + threadIdx.x;
   if (s >= S) return;
@@ -237,7 +240,49 @@ __global__ void k_update_lens(const int* __restrict__ accept_len, int S, int W, 
   const int L = committed_len[s] + m;
   if (L > max_tokens) atomicOr(status, COD_DEV_PAGE_OVERFLOW);
   committed_len[s] = L;
-  carry_len[s] = mode == COD_CARRY ? W - m : 0;
+  carry_len[s] = mode == COD_CARRY ? (carry_base ? carry_base[s] : 0) + W - m : 0;
+}
+
+// ------------------------------------------------------------------ carry retention (carry_rounds = k > 1)
+// Per sequence: the oldest of the k retained rounds leaves U. hist[s][0..k) holds the segment lengths,
+// oldest first (zeros at the start: empty rounds). base[s] = rows that stay; the history shifts and
+// takes the new round's W - m. The baseline drafter keeps no U: history and base are cleared.
+__global__ void k_carry_age_hist(const int* __restrict__ accept_len, const int* __restrict__ carry_len, int S, int W,
+                                 int k, int mode, int* __restrict__ hist, int* __restrict__ base, int* __restrict__ drop) {
+  cod_pdl_prologue();
+  const int s = blockIdx.x * blockDim.x + threadIdx.x;
+  if (s >= S) return;
+  int* h = hist + static_cast<size_t>(s) * k;
+  if (mode != COD_CARRY) {
+    for (int j = 0; j < k; ++j) h[j] = 0;
+    base[s] = 0; drop[s] = 0;
+    return;
+  }
+  int keep = 0;
+  for (int j = 1; j < k; ++j) { keep += h[j]; h[j - 1] = h[j]; }
+  h[k - 1] = W - accept_len[s];
+  keep = max(0, min(keep, carry_len[s]));
+  base[s] = keep;
+  drop[s] = max(0, carry_len[s] - keep);
+}
+// Moves rows [drop, drop + keep) of every (layer, sequence, head, K|V) slot to the front. One block per
+// slot; rows go one at a time in increasing order (destination below source), a barrier between the
+// read and the write of a row.
+template <typename T>
+__global__ void k_carry_shift(T* __restrict__ carry, const int* __restrict__ base, const int* __restrict__ drop,
+                              int max_batch, int n_kv, int cap, int hd) {
+  cod_pdl_prologue();
+  const int s = blockIdx.x, slot = blockIdx.y, l = blockIdx.z;          // slot = head * 2 + (K|V)
+  const int keep = base[s], d = drop[s];
+  if (d == 0 || keep == 0) return;
+  T* p = carry + ((static_cast<size_t>(l) * max_batch + s) * n_kv * 2 + slot) * cap * hd;
+  for (int i = 0; i < keep; ++i) {
+    T v = T();
+    if (threadIdx.x < hd) v = p[static_cast<size_t>(i + d) * hd + threadIdx.x];
+    __syncthreads();
+    if (threadIdx.x < hd) p[static_cast<size_t>(i) * hd + threadIdx.x] = v;
+    __syncthreads();
+  }
 }
 
 // ------------------------------------------------------------------ block input
@@ -497,8 +542,8 @@ int cod_launch_kv_finish(cod_ctx* c, const float* part, int splits, int n_rows, 
   dim3 grid(n_rows, f.n_layers);
   const int to_state = ds ? 1 : 0;
   DISPATCH_T(c,
-             (cod_launch_pdl(c, k_kv_finish<__nv_bfloat16>, grid, 128, 0, st, part, splits, n_rows, n_rows_dev, a_rows, c->rope_win, f.n_layers, f.n_kv_heads, f.head_dim, static_cast<__nv_bfloat16*>(J), R_total, sp->commit_slot, sp->carry_slot, ds ? static_cast<__nv_bfloat16*>(ds->kv_pool) : nullptr, ds ? static_cast<__nv_bfloat16*>(ds->carry_kv) : nullptr, f.page_size, f.n_pages, f.block, f.max_batch, to_state, (f.flags & COD_F_QK_NORM) ? static_cast<const __nv_bfloat16*>(c->w.g_knorm) : nullptr, f.rms_eps)),
-             (cod_launch_pdl(c, k_kv_finish<float>, grid, 128, 0, st, part, splits, n_rows, n_rows_dev, a_rows, c->rope_win, f.n_layers, f.n_kv_heads, f.head_dim, static_cast<float*>(J), R_total, sp->commit_slot, sp->carry_slot, ds ? static_cast<float*>(ds->kv_pool) : nullptr, ds ? static_cast<float*>(ds->carry_kv) : nullptr, f.page_size, f.n_pages, f.block, f.max_batch, to_state, (f.flags & COD_F_QK_NORM) ? static_cast<const float*>(c->w.g_knorm) : nullptr, f.rms_eps)));
+             (cod_launch_pdl(c, k_kv_finish<__nv_bfloat16>, grid, 128, 0, st, part, splits, n_rows, n_rows_dev, a_rows, c->rope_win, f.n_layers, f.n_kv_heads, f.head_dim, static_cast<__nv_bfloat16*>(J), R_total, sp->commit_slot, sp->carry_slot, ds ? static_cast<__nv_bfloat16*>(ds->kv_pool) : nullptr, ds ? static_cast<__nv_bfloat16*>(ds->carry_kv) : nullptr, f.page_size, f.n_pages, f.block, f.max_batch, to_state, (f.flags & COD_F_QK_NORM) ? static_cast<const __nv_bfloat16*>(c->w.g_knorm) : nullptr, f.rms_eps, c->carry_cap, c->carry_base)),
+             (cod_launch_pdl(c, k_kv_finish<float>, grid, 128, 0, st, part, splits, n_rows, n_rows_dev, a_rows, c->rope_win, f.n_layers, f.n_kv_heads, f.head_dim, static_cast<float*>(J), R_total, sp->commit_slot, sp->carry_slot, ds ? static_cast<float*>(ds->kv_pool) : nullptr, ds ? static_cast<float*>(ds->carry_kv) : nullptr, f.page_size, f.n_pages, f.block, f.max_batch, to_state, (f.flags & COD_F_QK_NORM) ? static_cast<const float*>(c->w.g_knorm) : nullptr, f.rms_eps, c->carry_cap, c->carry_base)));
   COD_CHECK_LAUNCH(c);
   return COD_OK;
 }
@@ -511,8 +556,8 @@ int cod_launch_scatter(cod_ctx* c, const void* J, const cod_split* sp, int S, in
   dim3 grid(R, f.n_layers);
   const int use_carry = mode == COD_CARRY;
   DISPATCH_T(c,
-             (cod_launch_pdl(c, k_scatter_kv<__nv_bfloat16>, grid, 128, 0, st, static_cast<const __nv_bfloat16*>(J), R, f.n_kv_heads, f.head_dim, sp->commit_slot, sp->carry_slot, static_cast<__nv_bfloat16*>(ds->kv_pool), static_cast<__nv_bfloat16*>(ds->carry_kv), f.page_size, f.n_pages, f.block, f.max_batch, use_carry)),
-             (cod_launch_pdl(c, k_scatter_kv<float>, grid, 128, 0, st, static_cast<const float*>(J), R, f.n_kv_heads, f.head_dim, sp->commit_slot, sp->carry_slot, static_cast<float*>(ds->kv_pool), static_cast<float*>(ds->carry_kv), f.page_size, f.n_pages, f.block, f.max_batch, use_carry)));
+             (cod_launch_pdl(c, k_scatter_kv<__nv_bfloat16>, grid, 128, 0, st, static_cast<const __nv_bfloat16*>(J), R, f.n_kv_heads, f.head_dim, sp->commit_slot, sp->carry_slot, static_cast<__nv_bfloat16*>(ds->kv_pool), static_cast<__nv_bfloat16*>(ds->carry_kv), f.page_size, f.n_pages, f.block, f.max_batch, use_carry, c->carry_cap, c->carry_base)),
+             (cod_launch_pdl(c, k_scatter_kv<float>, grid, 128, 0, st, static_cast<const float*>(J), R, f.n_kv_heads, f.head_dim, sp->commit_slot, sp->carry_slot, static_cast<float*>(ds->kv_pool), static_cast<float*>(ds->carry_kv), f.page_size, f.n_pages, f.block, f.max_batch, use_carry, c->carry_cap, c->carry_base)));
   COD_CHECK_LAUNCH(c);
   return COD_OK;
 }
@@ -521,7 +566,22 @@ int cod_launch_update_lens(cod_ctx* c, const cod_split* sp, int S, int mode, con
   ProfScope prof(c, COD_K_ROWOPS, st);
   cod_launch_pdl(c, k_update_lens, (S + 127) / 128, 128, 0, st, sp->accept_len, S, c->cfg.block, mode,
                                                  c->cfg.max_pages_per_seq * c->cfg.page_size, ds->committed_len,
-                                                 ds->carry_len, c->status);
+                                                 ds->carry_len, c->status, c->carry_base);
+  COD_CHECK_LAUNCH(c);
+  return COD_OK;
+}
+
+int cod_launch_carry_age(cod_ctx* c, const cod_split* sp, int S, int mode, const cod_state* ds, cudaStream_t st) {
+  ProfScope prof(c, COD_K_ROWOPS, st);
+  const cod_config& f = c->cfg;
+  const int k = c->carry_cap / f.block;
+  cod_launch_pdl(c, k_carry_age_hist, (S + 127) / 128, 128, 0, st, sp->accept_len, ds->carry_len, S, f.block, k, mode,
+                 ds->carry_hist, c->carry_base, c->carry_drop);
+  COD_CHECK_LAUNCH(c);
+  const dim3 grid(S, f.n_kv_heads * 2, f.n_layers);
+  DISPATCH_T(c,
+             (cod_launch_pdl(c, k_carry_shift<__nv_bfloat16>, grid, 128, 0, st, static_cast<__nv_bfloat16*>(ds->carry_kv), c->carry_base, c->carry_drop, f.max_batch, f.n_kv_heads, c->carry_cap, f.head_dim)),
+             (cod_launch_pdl(c, k_carry_shift<float>, grid, 128, 0, st, static_cast<float*>(ds->carry_kv), c->carry_base, c->carry_drop, f.max_batch, f.n_kv_heads, c->carry_cap, f.head_dim)));
   COD_CHECK_LAUNCH(c);
   return COD_OK;
 }

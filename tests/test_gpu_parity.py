@@ -109,6 +109,10 @@ def _workloads():
         "small_bf16_nomark": small_bf16(S=3, W=16, n_layers=1, ctx=(40, 300), carry_variant="none"),
         "small_bf16_proj": small_bf16(S=3, W=16, n_layers=2, ctx=(40, 300), carry_variant="projector"),
         "tiny_f32_proj": synth.scaled(synth.workload("cfg1"), S=3, ctx=(5, 140), n_rounds=6, carry_variant="projector"),
+        # rejected rows retained for k > 1 rounds: the carry slot holds k * W rows, the oldest round leaves
+        "small_bf16_keep2": small_bf16(S=3, W=16, n_layers=2, ctx=(40, 300), carry_rounds=2, n_rounds=6),
+        "small_bf16_W32_keep2": small_bf16(S=2, W=32, n_layers=1, ctx=(100, 200), carry_rounds=2, n_rounds=6),
+        "tiny_f32_keep3": synth.scaled(synth.workload("cfg1"), S=3, ctx=(5, 140), n_rounds=8, carry_rounds=3),
         "mid_bf16_full": small_bf16(S=34, W=16, n_layers=2, ctx=(100, 600), d_target=512, n_cap=5, d_model=1024,
                                     n_q=8, n_kv=2, vocab=3000, d_ff=1536, qk_norm=True),
     }
@@ -168,7 +172,11 @@ def test_project_and_scatter_unfused(name, mode):
                     assert torch.equal(pool_g[:, pg, :, :, off, :], Jh[:, row].transpose(1, 2))
                     touched[:, pg, :, :, off, :] = True
                 elif mode == orc.MODE_CARRY:
-                    assert torch.equal(carry_g[:, s, :, :, p - ms, :], Jh[:, row].transpose(1, 2))
+                    kept_rows = int(P.st_o.carry_len[s]) - (sh.W - ms)       # rows retained from earlier rounds (0 for k = 1)
+                    assert torch.equal(carry_g[:, s, :, :, kept_rows + p - ms, :], Jh[:, row].transpose(1, 2))
+            c = int(P.st_o.carry_len[s])
+            if mode == orc.MODE_CARRY and c:                                 # the whole slot, retained rows included
+                assert rel_err(carry_g[:, s, :, :, :c, :].float().numpy(), P.st_o.carry[:, s, :, :, :c, :]) <= tol
         assert torch.equal(pool_g[~touched], pool0.cpu()[~touched])           # nothing else moved
     assert P.ctx.poll_status() == 0
     P.close()
@@ -333,7 +341,9 @@ def test_round_parity_cfg1_every_round():
     ("small_bf16_mlp_only", 30.0, orc.MODE_CARRY), ("small_bf16_qknorm_only", 30.0, orc.MODE_CARRY),
     ("mid_bf16_full", 30.0, orc.MODE_CARRY),
     ("small_bf16_nomark", 30.0, orc.MODE_CARRY), ("small_bf16_proj", 30.0, orc.MODE_CARRY),
-    ("small_bf16_proj", 30.0, orc.MODE_BASELINE), ("tiny_f32_proj", 40.0, orc.MODE_CARRY)])
+    ("small_bf16_proj", 30.0, orc.MODE_BASELINE), ("tiny_f32_proj", 40.0, orc.MODE_CARRY),
+    ("small_bf16_keep2", 30.0, orc.MODE_CARRY), ("small_bf16_keep2", 30.0, orc.MODE_BASELINE),
+    ("small_bf16_W32_keep2", 1.0, orc.MODE_CARRY), ("tiny_f32_keep3", 40.0, orc.MODE_CARRY)])
 def test_round_parity_multi_round(name, wo_scale, mode):
     """Open-loop rounds (inputs pre-generated), ragged acceptance, attention path made to matter."""
     Hn = _H()
