@@ -17,7 +17,8 @@
  * COD_F_QK_NORM), the round at temperature 1 (cod_verify_accept_stochastic,
  * cod_lm_head_sample, cod_draft_round_stochastic), the two other ways of
  * marking rejected rows the paper compares (COD_F_NO_CARRY_EMBED,
- * COD_F_REJ_PROJECTOR) and two analysis aids (cod_taps.carry_mass,
+ * COD_F_REJ_PROJECTOR), retention of rejected rows over several rounds
+ * (cod_config.carry_rounds) and two analysis aids (cod_taps.carry_mass,
  * cod_reconvergence_count).
  *
  * Conventions
