@@ -333,7 +333,15 @@ int cod_launch_gemm_tc(cod_ctx* c, const GemmArgs& g, cudaStream_t st) {
   const uint32_t stage_bytes = A_TILE_BYTES + static_cast<uint32_t>(p.NT) * BK * 2;
   int stages = static_cast<int>((200u * 1024u) / stage_bytes);
   if (stages > 8) stages = 8;
-  if (p.NT <= 32 && stages > 5) stages = 5;      // small tiles: leave room for two CTAs per SM
+  // small tiles: leave room for two CTAs per SM - three when the grid is several waves deep (the LM head
+  // at batch 1: 1187 CTAs), where a third resident CTA covers the other two's fill and drain bubbles
+  // (203 -> 191 us); shallower grids keep the deeper ring, each CTA being alone on its share of an SM
+  if (p.NT <= 32) {
+    int tiles_all = 0;
+    for (int i = 0; i < g.n_seg; ++i) tiles_all += (g.seg[i].N + BM - 1) / BM;
+    const int cap = static_cast<long long>(tiles_all) * splits >= 3ll * c->n_sm ? 4 : 5;
+    if (stages > cap) stages = cap;
+  }
   if (stages > p.kb_per_split) stages = p.kb_per_split;
   if (stages < 1) stages = 1;
   p.stages = stages;
