@@ -67,6 +67,9 @@ size_t carve(cod_ctx* c) {
   }
   cv.take(c->amax, sizeof(unsigned long long) * R);
   cv.take(c->lse_part, sizeof(float2) * R * ((static_cast<size_t>(f.vocab) + 127) / 128));
+  // the LM head streams the whole embedding table every round: a tile-major copy for the tensor-core path
+  if (f.dtype == COD_BF16 && !(f.flags & COD_F_NO_TENSOR_CORES) && f.d_model % 8 == 0)
+    cv.take(c->emb_tiled, cod_retile_bytes(f.vocab, f.d_model));
   cv.take(c->tok, sizeof(int32_t) * R);
   cv.take(c->sp.accept_len, sizeof(int32_t) * f.max_batch);
   cv.take(c->sp.bonus, sizeof(int32_t) * f.max_batch);
@@ -252,6 +255,10 @@ int cod_set_weights(cod_ctx* c, const cod_weights* w, cod_stream_t stream) {
   c->w = *w;
   c->has_weights = true;
   c->pdl = false;
+  if (c->emb_tiled) {
+    const int rc = cod_launch_retile(c, w->emb, c->cfg.vocab, c->D, c->emb_tiled, static_cast<cudaStream_t>(stream));
+    if (rc != COD_OK) return rc;
+  }
   return cod_launch_fcE(c, static_cast<cudaStream_t>(stream));
 }
 
@@ -352,7 +359,7 @@ int cod_block_attn(cod_ctx* c, int layer, const void* q, const void* k_blk, cons
 static int lm_head_impl(cod_ctx* c, int n_rows, cudaStream_t st) {
   GemmArgs g{};
   g.A = c->a; g.lda = c->D; g.n_rows = n_rows; g.K = c->D;
-  g.seg[0] = {c->w.emb, c->cfg.vocab}; g.n_seg = 1;
+  g.seg[0] = {c->w.emb, c->cfg.vocab, c->emb_tiled}; g.n_seg = 1;
   g.splits = 1; g.amax = c->amax; g.klass = COD_K_LMHEAD;
   return cod_launch_gemm(c, g, st);
 }
@@ -479,7 +486,7 @@ static int round_impl(cod_ctx* c, const int32_t* draft, const int32_t* target, c
   if (q_next != nullptr) {                      // temperature 1: the block is drawn, with its proposal probabilities
     GemmArgs g{};
     g.A = c->a; g.lda = c->D; g.n_rows = R; g.K = c->D;
-    g.seg[0] = {c->w.emb, f.vocab}; g.n_seg = 1;
+    g.seg[0] = {c->w.emb, f.vocab, c->emb_tiled}; g.n_seg = 1;
     g.splits = 1; g.amax = c->amax; g.klass = COD_K_LMHEAD;
     g.lse_part = c->lse_part; g.sample_state = cod_sample_state(seed, step);
     if (c->force_simt || !(cod_gemm_tc2_supported(c, g) || cod_gemm_tc_supported(c, g))) return COD_ERR_UNSUPPORTED;
@@ -497,7 +504,7 @@ int cod_lm_head_sample(cod_ctx* c, const float* x, int n_rows, unsigned long lon
   if (!c->has_weights) return COD_ERR_NO_WEIGHTS;
   GemmArgs g{};
   g.A = c->a; g.lda = c->D; g.n_rows = n_rows; g.K = c->D;
-  g.seg[0] = {c->w.emb, c->cfg.vocab}; g.n_seg = 1;
+  g.seg[0] = {c->w.emb, c->cfg.vocab, c->emb_tiled}; g.n_seg = 1;
   g.splits = 1; g.amax = c->amax; g.klass = COD_K_LMHEAD;
   g.lse_part = c->lse_part; g.sample_state = cod_sample_state(seed, step);
   if (c->force_simt || !(cod_gemm_tc2_supported(c, g) || cod_gemm_tc_supported(c, g))) return COD_ERR_UNSUPPORTED;

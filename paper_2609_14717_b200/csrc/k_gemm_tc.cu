@@ -41,6 +41,7 @@ struct TcParams {
   float* C;
   int ldc;
   unsigned long long* amax;
+  const uint8_t* wt[3];       // per weight segment: tile-major copy (16 KB tiles), or null
   float2* lse_part;           // sampling form of the argmax epilogue (null: plain argmax)
   uint32_t sample_state;
   uint32_t* status;
@@ -93,6 +94,8 @@ k_gemm_tc(const __grid_constant__ CUtensorMap map_w0, const __grid_constant__ CU
   for (int s = 0; s < sidx; ++s) col0 += p.seg_N[s];
   const int seg_N = p.seg_N[sidx];
   const CUtensorMap* map_w = sidx == 0 ? &map_w0 : (sidx == 1 ? &map_w1 : &map_w2);
+  // tile-major copy of this segment: tile (tile_in_seg, kb) is 16 KB at ((tile_in_seg * kb_total) + kb) * 16 KB
+  const uint8_t* wt = p.wt[sidx] ? p.wt[sidx] + static_cast<size_t>(tile_in_seg) * p.kb_total * A_TILE_BYTES : nullptr;
 
   const int kb0 = split * p.kb_per_split, kb1 = min(p.kb_total, kb0 + p.kb_per_split);
   const int n_pre = min(p.stages, kb1 - kb0);     // stages whose weight tile is requested ahead of the dependency
@@ -115,7 +118,8 @@ k_gemm_tc(const __grid_constant__ CUtensorMap map_w0, const __grid_constant__ CU
   const uint32_t tmem_base = *tmem_slot;
   if (warp == 4 && lane == 0)
     for (int it = 0; it < n_pre; ++it)
-      tma_load_2d(base + it * stage_bytes, map_w, (kb0 + it) * BK, f0, smem_u32(full_bar + it));
+      if (wt) bulk_load(base + it * stage_bytes, wt + static_cast<size_t>(kb0 + it) * A_TILE_BYTES, A_TILE_BYTES, smem_u32(full_bar + it));
+      else tma_load_2d(base + it * stage_bytes, map_w, (kb0 + it) * BK, f0, smem_u32(full_bar + it));
 
   cod_pdl_prologue();
   const int n_rows = p.n_rows_dev ? min(*p.n_rows_dev, p.n_rows) : p.n_rows;
@@ -137,7 +141,10 @@ k_gemm_tc(const __grid_constant__ CUtensorMap map_w0, const __grid_constant__ CU
         mbar_expect_tx(fb, stage_bytes);
         const uint32_t a_dst = base + s * stage_bytes;
         const int k = (kb0 + it) * BK;
-        if (it >= n_pre) tma_load_2d(a_dst, map_w, k, f0, fb);
+        if (it >= n_pre) {
+          if (wt) bulk_load(a_dst, wt + static_cast<size_t>(kb0 + it) * A_TILE_BYTES, A_TILE_BYTES, fb);
+          else tma_load_2d(a_dst, map_w, k, f0, fb);
+        }
         tma_load_2d(a_dst + A_TILE_BYTES, &map_a, k, i0, fb);
       }
     }
@@ -360,6 +367,7 @@ int cod_launch_gemm_tc(cod_ctx* c, const GemmArgs& g, cudaStream_t st) {
              static_cast<size_t>(stages) * stage_bytes >= 2u * 32u * BM * sizeof(float);
   for (int i = 0; i < g.n_seg; ++i) p.staged = p.staged && (g.seg[i].N % 4 == 0);
   p.amax = g.amax;
+  for (int i = 0; i < 3; ++i) p.wt[i] = i < g.n_seg ? static_cast<const uint8_t*>(g.seg[i].Bt) : nullptr;
   p.lse_part = g.amax ? g.lse_part : nullptr;
   p.sample_state = g.sample_state;
   p.status = c->status;
@@ -443,4 +451,31 @@ int cod_launch_finalize_sample(cod_ctx* c, int R, uint32_t state, int32_t* tok, 
   return COD_OK;
 }
 uint32_t cod_sample_state(unsigned long long seed, uint32_t step) { return tc::sample_state(seed, step); }
+
+// ------------------------------------------------------------------ tile-major weight copy
+namespace {
+__global__ void k_retile(const __nv_bfloat16* __restrict__ B, int N, int K, uint8_t* __restrict__ Bt) {
+  const int kb = blockIdx.x, tile = blockIdx.y, kb_total = gridDim.x;
+  uint4* dst = reinterpret_cast<uint4*>(Bt + (static_cast<size_t>(tile) * kb_total + kb) * A_TILE_BYTES);
+  for (int idx = threadIdx.x; idx < BM * 8; idx += blockDim.x) {        // 16-byte chunks: 128 rows x 8
+    const int r = idx >> 3, ch = idx & 7;
+    const int row = tile * BM + r, col = kb * BK + ch * 8;
+    uint4 v = make_uint4(0u, 0u, 0u, 0u);
+    if (row < N && col < K) v = *reinterpret_cast<const uint4*>(B + static_cast<size_t>(row) * K + col);   // K % 8 == 0
+    dst[r * 8 + (ch ^ (r & 7))] = v;                                       // the 128-byte swizzle
+  }
+}
+}  // namespace
+
+size_t cod_retile_bytes(int N, int K) {
+  return static_cast<size_t>((N + BM - 1) / BM) * ((K + BK - 1) / BK) * A_TILE_BYTES;
+}
+
+int cod_launch_retile(cod_ctx* c, const void* B, int N, int K, void* Bt, cudaStream_t st) {
+  if (K % 8) return COD_ERR_UNSUPPORTED;
+  const dim3 grid((K + BK - 1) / BK, (N + BM - 1) / BM);
+  k_retile<<<grid, 256, 0, st>>>(static_cast<const __nv_bfloat16*>(B), N, K, static_cast<uint8_t*>(Bt));
+  COD_CHECK_LAUNCH(c);
+  return COD_OK;
+}
 
