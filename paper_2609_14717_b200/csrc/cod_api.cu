@@ -68,8 +68,24 @@ size_t carve(cod_ctx* c) {
   cv.take(c->amax, sizeof(unsigned long long) * R);
   cv.take(c->lse_part, sizeof(float2) * R * ((static_cast<size_t>(f.vocab) + 127) / 128));
   // the LM head streams the whole embedding table every round: a tile-major copy for the tensor-core path
-  if (f.dtype == COD_BF16 && !(f.flags & COD_F_NO_TENSOR_CORES) && f.d_model % 8 == 0)
-    cv.take(c->emb_tiled, cod_retile_bytes(f.vocab, f.d_model));
+  // (conditions on the configuration only: the measuring pass of this function assigns no pointers)
+  const bool tile_ok = f.dtype == COD_BF16 && !(f.flags & COD_F_NO_TENSOR_CORES) && f.d_model % 8 == 0 &&
+                       (f.d_target * f.n_cap) % 8 == 0;
+  if (tile_ok) cv.take(c->emb_tiled, cod_retile_bytes(f.vocab, f.d_model));
+  // ... and of the other matrices where the single-CTA kernel (up to 128 rows) will stream them
+  if (tile_ok && f.max_batch * f.block <= 128) {
+    const int Ld = f.n_layers, kvw = c->kvw, qw = c->qw, Dm = c->D;
+    if (Dm % 128 == 0) cv.take(c->wt.fc, cod_retile_bytes(Dm, c->D_in));
+    if (Dm % 128 == 0 && (f.flags & COD_F_REJ_PROJECTOR)) cv.take(c->wt.fc_rej, cod_retile_bytes(Dm, c->D_in));
+    if (kvw % 128 == 0) { cv.take(c->wt.wk, Ld * cod_retile_bytes(kvw, Dm)); cv.take(c->wt.wv, Ld * cod_retile_bytes(kvw, Dm)); }
+    if (qw % 128 == 0) cv.take(c->wt.wq, Ld * cod_retile_bytes(qw, Dm));
+    if (Dm % 128 == 0 && qw % 8 == 0) cv.take(c->wt.wo, Ld * cod_retile_bytes(Dm, qw));
+    if (f.d_ff > 0 && f.d_ff % 128 == 0) {
+      cv.take(c->wt.w_gate, Ld * cod_retile_bytes(f.d_ff, Dm));
+      cv.take(c->wt.w_up, Ld * cod_retile_bytes(f.d_ff, Dm));
+      if (Dm % 128 == 0) cv.take(c->wt.w_down, Ld * cod_retile_bytes(Dm, f.d_ff));
+    }
+  }
   cv.take(c->tok, sizeof(int32_t) * R);
   cv.take(c->sp.accept_len, sizeof(int32_t) * f.max_batch);
   cv.take(c->sp.bonus, sizeof(int32_t) * f.max_batch);
@@ -256,7 +272,22 @@ int cod_set_weights(cod_ctx* c, const cod_weights* w, cod_stream_t stream) {
   c->has_weights = true;
   c->pdl = false;
   if (c->emb_tiled) {
-    const int rc = cod_launch_retile(c, w->emb, c->cfg.vocab, c->D, c->emb_tiled, static_cast<cudaStream_t>(stream));
+    cudaStream_t ss = static_cast<cudaStream_t>(stream);
+    int rc = cod_launch_retile(c, w->emb, c->cfg.vocab, c->D, c->emb_tiled, ss);
+    const cod_config& f = c->cfg;
+    // a stacked matrix [Ld][N, K] whose N is a whole number of tiles re-tiles as one matrix of Ld * N rows
+    auto all = [&](const void* src, char* dst, int N, int K, int layers) {
+      if (dst && rc == COD_OK) rc = cod_launch_retile(c, src, layers * N, K, dst, ss);
+    };
+    all(w->fc, c->wt.fc, c->D, c->D_in, 1);
+    all(w->fc_rej, c->wt.fc_rej, c->D, c->D_in, 1);
+    all(w->wk, c->wt.wk, c->kvw, c->D, f.n_layers);
+    all(w->wv, c->wt.wv, c->kvw, c->D, f.n_layers);
+    all(w->wq, c->wt.wq, c->qw, c->D, f.n_layers);
+    all(w->wo, c->wt.wo, c->D, c->qw, f.n_layers);
+    all(w->w_gate, c->wt.w_gate, f.d_ff, c->D, f.n_layers);
+    all(w->w_up, c->wt.w_up, f.d_ff, c->D, f.n_layers);
+    all(w->w_down, c->wt.w_down, c->D, f.d_ff, f.n_layers);
     if (rc != COD_OK) return rc;
   }
   return cod_launch_fcE(c, static_cast<cudaStream_t>(stream));
@@ -296,11 +327,11 @@ static int project_impl(cod_ctx* c, const void* H, const cod_split* sp, int S, i
   }
   GemmArgs g{};
   g.A = H; g.lda = c->D_in; g.a_rows = nullptr; g.n_rows_dev = n_dev; g.n_rows = R; g.K = c->D_in;
-  g.seg[0] = {c->w.fc, c->D}; g.n_seg = 1; g.klass = COD_K_FC;
+  g.seg[0] = {c->w.fc, c->D, c->wt.fc}; g.n_seg = 1; g.klass = COD_K_FC;
   // separate-projector variant, carry mode: F h and F_rej h of every row from one two-segment contraction,
   // the finish kernel keeps the one the row's status selects (the baseline keeps accepted rows only: F alone)
   const bool two = (f.flags & COD_F_REJ_PROJECTOR) && mode == COD_CARRY;
-  if (two) { g.seg[1] = {c->w.fc_rej, c->D}; g.n_seg = 2; }
+  if (two) { g.seg[1] = {c->w.fc_rej, c->D, c->wt.fc_rej}; g.n_seg = 2; }
   g.C = c->gemm_out; g.ldc = two ? 2 * c->D : c->D; g.splits = pick_splits(c, g.ldc, c->D_in, R);
   if ((rc = cod_launch_gemm(c, g, st)) != COD_OK) return rc;
   if ((rc = cod_launch_fc_finish(c, c->gemm_out, g.splits, R, n_dev, a_rows, sp->carry_slot, tap_z, st, g.ldc)) != COD_OK)
@@ -308,8 +339,8 @@ static int project_impl(cod_ctx* c, const void* H, const cod_split* sp, int S, i
 
   GemmArgs k{};
   k.A = c->z; k.lda = c->D; k.a_rows = nullptr; k.n_rows_dev = n_dev; k.n_rows = R; k.K = c->D;
-  k.seg[0] = {c->w.wk, f.n_layers * c->kvw};
-  k.seg[1] = {c->w.wv, f.n_layers * c->kvw};
+  k.seg[0] = {c->w.wk, f.n_layers * c->kvw, c->wt.wk};
+  k.seg[1] = {c->w.wv, f.n_layers * c->kvw, c->wt.wv};
   k.n_seg = 2; k.klass = COD_K_KV;
   k.C = c->gemm_out; k.ldc = 2 * f.n_layers * c->kvw; k.splits = pick_splits(c, k.ldc, c->D, R);
   if ((rc = cod_launch_gemm(c, k, st)) != COD_OK) return rc;
@@ -427,9 +458,10 @@ static int round_impl(cod_ctx* c, const int32_t* draft, const int32_t* target, c
     cudaStream_t sl = l == 0 ? sq : s;
     GemmArgs g{};
     g.A = c->a; g.lda = c->D; g.n_rows = R; g.K = c->D;
-    g.seg[0] = {static_cast<const char*>(c->w.wq) + es * l * c->qw * c->D, c->qw};
-    g.seg[1] = {static_cast<const char*>(c->w.wk) + es * l * c->kvw * c->D, c->kvw};
-    g.seg[2] = {static_cast<const char*>(c->w.wv) + es * l * c->kvw * c->D, c->kvw};
+    auto tiled = [&](const char* base, int N, int K) -> const void* { return base ? base + l * cod_retile_bytes(N, K) : nullptr; };
+    g.seg[0] = {static_cast<const char*>(c->w.wq) + es * l * c->qw * c->D, c->qw, tiled(c->wt.wq, c->qw, c->D)};
+    g.seg[1] = {static_cast<const char*>(c->w.wk) + es * l * c->kvw * c->D, c->kvw, tiled(c->wt.wk, c->kvw, c->D)};
+    g.seg[2] = {static_cast<const char*>(c->w.wv) + es * l * c->kvw * c->D, c->kvw, tiled(c->wt.wv, c->kvw, c->D)};
     g.n_seg = 3; g.klass = COD_K_QKV;
     g.C = l == 0 ? slab_q : c->gemm_out; g.ldc = c->qw + 2 * c->kvw; g.splits = pick_splits(c, g.ldc, c->D, R);
     if ((rc = cod_launch_gemm(c, g, sl)) != COD_OK) return rc;
@@ -449,7 +481,7 @@ static int round_impl(cod_ctx* c, const int32_t* draft, const int32_t* target, c
 
     GemmArgs o{};
     o.A = c->o; o.lda = c->qw; o.n_rows = R; o.K = c->qw;
-    o.seg[0] = {static_cast<const char*>(c->w.wo) + es * l * c->D * c->qw, c->D};
+    o.seg[0] = {static_cast<const char*>(c->w.wo) + es * l * c->D * c->qw, c->D, tiled(c->wt.wo, c->D, c->qw)};
     o.n_seg = 1; o.klass = COD_K_OPROJ;
     o.C = c->gemm_out; o.ldc = c->D; o.splits = pick_splits(c, c->D, c->qw, R);
     if ((rc = cod_launch_gemm(c, o, s)) != COD_OK) return rc;
@@ -466,15 +498,15 @@ static int round_impl(cod_ctx* c, const int32_t* draft, const int32_t* target, c
     if ((rc = cod_launch_resid_norm(c, c->gemm_out, o.splits, R, c->x, g_mlp, nullptr, s)) != COD_OK) return rc;
     GemmArgs gu{};
     gu.A = c->a; gu.lda = c->D; gu.n_rows = R; gu.K = c->D;
-    gu.seg[0] = {static_cast<const char*>(c->w.w_gate) + es * l * f.d_ff * c->D, f.d_ff};
-    gu.seg[1] = {static_cast<const char*>(c->w.w_up) + es * l * f.d_ff * c->D, f.d_ff};
+    gu.seg[0] = {static_cast<const char*>(c->w.w_gate) + es * l * f.d_ff * c->D, f.d_ff, tiled(c->wt.w_gate, f.d_ff, c->D)};
+    gu.seg[1] = {static_cast<const char*>(c->w.w_up) + es * l * f.d_ff * c->D, f.d_ff, tiled(c->wt.w_up, f.d_ff, c->D)};
     gu.n_seg = 2; gu.klass = COD_K_MLP;
     gu.C = c->gemm_out; gu.ldc = 2 * f.d_ff; gu.splits = pick_splits(c, gu.ldc, c->D, R);
     if ((rc = cod_launch_gemm(c, gu, s)) != COD_OK) return rc;
     if ((rc = cod_launch_swiglu_finish(c, c->gemm_out, gu.splits, R, s)) != COD_OK) return rc;
     GemmArgs dn{};
     dn.A = c->hmid; dn.lda = f.d_ff; dn.n_rows = R; dn.K = f.d_ff;
-    dn.seg[0] = {static_cast<const char*>(c->w.w_down) + es * l * c->D * f.d_ff, c->D};
+    dn.seg[0] = {static_cast<const char*>(c->w.w_down) + es * l * c->D * f.d_ff, c->D, tiled(c->wt.w_down, c->D, f.d_ff)};
     dn.n_seg = 1; dn.klass = COD_K_MLP;
     dn.C = c->gemm_out; dn.ldc = c->D; dn.splits = pick_splits(c, c->D, f.d_ff, R);
     if ((rc = cod_launch_gemm(c, dn, s)) != COD_OK) return rc;

@@ -141,6 +141,10 @@ struct cod_ctx {
   void* hmid;                  // [R, d_ff] activated MLP rows (storage type), d_ff > 0 only
   float2* lse_part;            // [ceil(vocab / 128)][R] soft-max partials of the sampling LM head
   void* emb_tiled;             // tile-major copy of the embedding table (bf16 tensor-core path), made by cod_set_weights
+  // tile-major copies of the other weight matrices, for rounds of up to 128 rows (null where the matrix
+  // does not cut into whole 128-row tiles per layer, or for large-batch-only contexts); per layer l a
+  // matrix [N, K] starts at l * cod_retile_bytes(N, K)
+  struct { char *fc, *fc_rej, *wk, *wv, *wq, *wo, *w_gate, *w_up, *w_down; } wt;
   float* gemm_out;             // split-K / unfused GEMM results
   int carry_cap;               // rows of one (layer, sequence, head, K|V) carry slot: carry_rounds * block
   int* carry_base;             // [max_batch] rows of U kept from earlier rounds (carry_rounds > 1), else null
