@@ -34,7 +34,7 @@ METRIC = "drafting rounds/s"
 UNIT = "rounds/s"
 # dram__bytes_read.sum + dram__bytes_write.sum per launch of the dominant kernel, from the ncu
 # capture summarised under profiles/ (None until a capture exists for the current kernel).
-NCU_TRAFFIC_BYTES = {"cfg2": 1276240352, "cfg3": 1311827456}   # profiles/lmhead_k_gemm_tc*_cfg*.md
+NCU_TRAFFIC_BYTES = {"cfg2": 1249087584, "cfg3": 1311827456}   # profiles/lmhead_k_gemm_tc*_cfg*.md
 
 
 def load_peaks():
