@@ -178,8 +178,8 @@ int cod_destroy(cod_ctx* ctx);
 /* Records the weight pointers (they must stay valid while the context is used) and
    precomputes F(E_carry) = fc . e_carry: F is linear and bias-free, so
    F(h + E_carry) = F(h) + F(E_carry) (Eq. 2 with Algorithm 1's "add before F").
-   bf16 contexts also SNAPSHOT the embedding table - and, when max_batch * block <= 128, every
-   weight matrix - into tile-major copies inside the workspace (contiguous 16 KB tiles stream
+   bf16 contexts with max_batch * block <= 128 also SNAPSHOT every weight matrix, the embedding
+   table included, into tile-major copies inside the workspace (contiguous 16 KB tiles stream
    from HBM measurably faster than 128 separate rows; the workspace grows by the size of the
    copied matrices): after changing weight values in place, call cod_set_weights again. */
 int cod_set_weights(cod_ctx* ctx, const cod_weights* w, cod_stream_t stream);

@@ -67,13 +67,14 @@ size_t carve(cod_ctx* c) {
   }
   cv.take(c->amax, sizeof(unsigned long long) * R);
   cv.take(c->lse_part, sizeof(float2) * R * ((static_cast<size_t>(f.vocab) + 127) / 128));
-  // the LM head streams the whole embedding table every round: a tile-major copy for the tensor-core path
+  // rounds of up to 128 rows stream every weight matrix through the single-CTA kernel: tile-major copies
   // (conditions on the configuration only: the measuring pass of this function assigns no pointers)
   const bool tile_ok = f.dtype == COD_BF16 && !(f.flags & COD_F_NO_TENSOR_CORES) && f.d_model % 8 == 0 &&
                        (f.d_target * f.n_cap) % 8 == 0;
-  if (tile_ok) cv.take(c->emb_tiled, cod_retile_bytes(f.vocab, f.d_model));
-  // ... and of the other matrices where the single-CTA kernel (up to 128 rows) will stream them
-  if (tile_ok && f.max_batch * f.block <= 128) {
+  // (contexts sized for more than 128 rows run the paired kernel, which reads the caller's matrices: no copies)
+  const bool tile_all = tile_ok && f.max_batch * f.block <= 128;
+  if (tile_all) cv.take(c->emb_tiled, cod_retile_bytes(f.vocab, f.d_model));
+  if (tile_all) {
     const int Ld = f.n_layers, kvw = c->kvw, qw = c->qw, Dm = c->D;
     if (Dm % 128 == 0) cv.take(c->wt.fc, cod_retile_bytes(Dm, c->D_in));
     if (Dm % 128 == 0 && (f.flags & COD_F_REJ_PROJECTOR)) cv.take(c->wt.fc_rej, cod_retile_bytes(Dm, c->D_in));
