@@ -450,11 +450,11 @@ static int round_impl(cod_ctx* c, const int32_t* draft, const int32_t* target, c
   } else {
     // parts 2-3 first, on the one stream
     if ((rc = project_impl(c, H, sp, S, mode, nullptr, st, taps ? taps->z : nullptr, s)) != COD_OK) return rc;
-    if ((rc = cod_launch_update_lens(c, sp, S, mode, st, s)) != COD_OK) return rc;
   }
 
-  // the next block: [bonus, MASK, ...] through every drafter layer
-  if ((rc = cod_launch_embed_norm(c, sp->bonus, S, sq)) != COD_OK) return rc;
+  // the next block: [bonus, MASK, ...] through every drafter layer (the embedding kernel also
+  // performs part 3's length update: nothing before the first attention reads the lengths)
+  if ((rc = cod_launch_embed_norm(c, sp->bonus, S, sq, sp, mode, st)) != COD_OK) return rc;
   for (int l = 0; l < f.n_layers; ++l) {
     cudaStream_t sl = l == 0 ? sq : s;
     GemmArgs g{};
@@ -470,7 +470,6 @@ static int round_impl(cod_ctx* c, const int32_t* draft, const int32_t* target, c
     if (l == 0 && fork) {
       // parts 2-3 on the caller's stream meanwhile, then the join
       if ((rc = project_impl(c, H, sp, S, mode, nullptr, st, taps ? taps->z : nullptr, s)) != COD_OK) return rc;
-      if ((rc = cod_launch_update_lens(c, sp, S, mode, st, s)) != COD_OK) return rc;
       if (cudaEventRecord(c->ev_join, c->side) != cudaSuccess || cudaStreamWaitEvent(s, c->ev_join, 0) != cudaSuccess)
         return COD_ERR_CUDA;
     }

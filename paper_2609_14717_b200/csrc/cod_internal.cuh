@@ -257,7 +257,9 @@ int cod_launch_scatter(cod_ctx* c, const void* J, const cod_split* sp, int S, in
                        const cod_state* state, cudaStream_t st);
 int cod_launch_update_lens(cod_ctx* c, const cod_split* sp, int S, int mode, const cod_state* state,
                            cudaStream_t st);
-int cod_launch_embed_norm(cod_ctx* c, const int32_t* bonus, int S, cudaStream_t st);
+// sp non-null: the kernel also performs cod_launch_update_lens's update (inside a round)
+int cod_launch_embed_norm(cod_ctx* c, const int32_t* bonus, int S, cudaStream_t st, const cod_split* sp = nullptr,
+                          int mode = 0, const cod_state* ds = nullptr);
 int cod_launch_qkv_finish(cod_ctx* c, const float* part, int splits, int R, int layer, cudaStream_t st);
 int cod_launch_swiglu_finish(cod_ctx* c, const float* part, int splits, int R, cudaStream_t st);
 int cod_launch_rope_qk(cod_ctx* c, const void* q, const void* k, const int32_t* committed_len, int S,

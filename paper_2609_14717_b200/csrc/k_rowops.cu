@@ -230,17 +230,26 @@ __global__ void k_scatter_kv(const T* __restrict__ J, int R_total, int n_kv, int
   }
 }
 
-__global__ void k_update_lens(const int* __restrict__ accept_len, int S, int W, int mode, int max_tokens,
-                              int* __restrict__ committed_len, int* __restrict__ carry_len, uint32_t* status,
-                              const int* __restrict__ carry_base) {
+// committed_len[s] += m_s; carry_len[s] = kept rows + W - m_s (0 for the baseline drafter)
+struct LensUpdate {
+  const int* accept_len;      // null: no update
+  int S, W, mode, max_tokens;
+  int* committed_len;
+  int* carry_len;
+  uint32_t* status;
+  const int* carry_base;
+};
+__device__ __forceinline__ void cod_update_lens_one(const LensUpdate& u, int s) {
+  const int m = u.accept_len[s];
+  const int L = u.committed_len[s] + m;
+  if (L > u.max_tokens) atomicOr(u.status, COD_DEV_PAGE_OVERFLOW);
+  u.committed_len[s] = L;
+  u.carry_len[s] = u.mode == COD_CARRY ? (u.carry_base ? u.carry_base[s] : 0) + u.W - m : 0;
+}
+__global__ void k_update_lens(LensUpdate u) {
   cod_pdl_prologue();
   const int s = blockIdx.x * blockDim.x + threadIdx.x;
-  if (s >= S) return;
-  const int m = accept_len[s];
-  const int L = committed_len[s] + m;
-  if (L > max_tokens) atomicOr(status, COD_DEV_PAGE_OVERFLOW);
-  committed_len[s] = L;
-  carry_len[s] = mode == COD_CARRY ? (carry_base ? carry_base[s] : 0) + W - m : 0;
+  if (s < u.S) cod_update_lens_one(u, s);
 }
 
 // ------------------------------------------------------------------ carry retention (carry_rounds = k > 1)
@@ -290,10 +299,14 @@ __global__ void k_carry_shift(T* __restrict__ carry, const int* __restrict__ bas
 template <typename T, int NV>
 __global__ void __launch_bounds__(1024) k_embed_norm(const T* __restrict__ emb, const int* __restrict__ bonus, int W, int mask_id,
                              int vocab, const T* __restrict__ gain, int D, float eps, float* __restrict__ x,
-                             T* __restrict__ a, unsigned long long* __restrict__ amax) {
+                             T* __restrict__ a, unsigned long long* __restrict__ amax, LensUpdate lu) {
   cod_pdl_prologue();
   __shared__ float red[33];
   const int r = blockIdx.x, s = r / W, p = r - s * W;
+  // inside a round this kernel also carries the length update of part 3 (one launch fewer on the
+  // critical path; nothing between part 1 and the first attention reads the lengths)
+  if (blockIdx.x == 0 && lu.accept_len != nullptr)
+    for (int q = threadIdx.x; q < lu.S; q += blockDim.x) cod_update_lens_one(lu, q);
   int tok = p == 0 ? bonus[s] : mask_id;
   if (tok < 0 || tok >= vocab) tok = 0;
   const int nv = D >> 2;
@@ -564,9 +577,9 @@ int cod_launch_scatter(cod_ctx* c, const void* J, const cod_split* sp, int S, in
 
 int cod_launch_update_lens(cod_ctx* c, const cod_split* sp, int S, int mode, const cod_state* ds, cudaStream_t st) {
   ProfScope prof(c, COD_K_ROWOPS, st);
-  cod_launch_pdl(c, k_update_lens, (S + 127) / 128, 128, 0, st, sp->accept_len, S, c->cfg.block, mode,
-                                                 c->cfg.max_pages_per_seq * c->cfg.page_size, ds->committed_len,
-                                                 ds->carry_len, c->status, c->carry_base);
+  const LensUpdate u{sp->accept_len, S, c->cfg.block, mode, c->cfg.max_pages_per_seq * c->cfg.page_size,
+                     ds->committed_len, ds->carry_len, c->status, c->carry_base};
+  cod_launch_pdl(c, k_update_lens, (S + 127) / 128, 128, 0, st, u);
   COD_CHECK_LAUNCH(c);
   return COD_OK;
 }
@@ -586,18 +599,22 @@ int cod_launch_carry_age(cod_ctx* c, const cod_split* sp, int S, int mode, const
   return COD_OK;
 }
 
-int cod_launch_embed_norm(cod_ctx* c, const int32_t* bonus, int S, cudaStream_t st) {
+int cod_launch_embed_norm(cod_ctx* c, const int32_t* bonus, int S, cudaStream_t st, const cod_split* sp, int mode,
+                          const cod_state* ds) {
   ProfScope prof(c, COD_K_ROWOPS, st);
   const cod_config& f = c->cfg;
   const int R = S * f.block;
+  LensUpdate u{};                                   // sp == null: no length update rides along
+  if (sp) u = LensUpdate{sp->accept_len, S, f.block, mode, f.max_pages_per_seq * f.page_size, ds->committed_len,
+                         ds->carry_len, c->status, c->carry_base};
   if (row_narrow(c->D)) {
     DISPATCH_T(c,
-               (cod_launch_pdl(c, k_embed_norm<__nv_bfloat16, 1>, R, row_threads(c->D), 0, st, static_cast<const __nv_bfloat16*>(c->w.emb), bonus, f.block, f.mask_token_id, f.vocab, static_cast<const __nv_bfloat16*>(c->w.g_attn), c->D, f.rms_eps, c->x, static_cast<__nv_bfloat16*>(c->a), c->amax)),
-               (cod_launch_pdl(c, k_embed_norm<float, 1>, R, row_threads(c->D), 0, st, static_cast<const float*>(c->w.emb), bonus, f.block, f.mask_token_id, f.vocab, static_cast<const float*>(c->w.g_attn), c->D, f.rms_eps, c->x, static_cast<float*>(c->a), c->amax)));
+               (cod_launch_pdl(c, k_embed_norm<__nv_bfloat16, 1>, R, row_threads(c->D), 0, st, static_cast<const __nv_bfloat16*>(c->w.emb), bonus, f.block, f.mask_token_id, f.vocab, static_cast<const __nv_bfloat16*>(c->w.g_attn), c->D, f.rms_eps, c->x, static_cast<__nv_bfloat16*>(c->a), c->amax, u)),
+               (cod_launch_pdl(c, k_embed_norm<float, 1>, R, row_threads(c->D), 0, st, static_cast<const float*>(c->w.emb), bonus, f.block, f.mask_token_id, f.vocab, static_cast<const float*>(c->w.g_attn), c->D, f.rms_eps, c->x, static_cast<float*>(c->a), c->amax, u)));
   } else {
     DISPATCH_T(c,
-               (cod_launch_pdl(c, k_embed_norm<__nv_bfloat16, ROW_WIDE_NV>, R, row_threads(c->D), 0, st, static_cast<const __nv_bfloat16*>(c->w.emb), bonus, f.block, f.mask_token_id, f.vocab, static_cast<const __nv_bfloat16*>(c->w.g_attn), c->D, f.rms_eps, c->x, static_cast<__nv_bfloat16*>(c->a), c->amax)),
-               (cod_launch_pdl(c, k_embed_norm<float, ROW_WIDE_NV>, R, row_threads(c->D), 0, st, static_cast<const float*>(c->w.emb), bonus, f.block, f.mask_token_id, f.vocab, static_cast<const float*>(c->w.g_attn), c->D, f.rms_eps, c->x, static_cast<float*>(c->a), c->amax)));
+               (cod_launch_pdl(c, k_embed_norm<__nv_bfloat16, ROW_WIDE_NV>, R, row_threads(c->D), 0, st, static_cast<const __nv_bfloat16*>(c->w.emb), bonus, f.block, f.mask_token_id, f.vocab, static_cast<const __nv_bfloat16*>(c->w.g_attn), c->D, f.rms_eps, c->x, static_cast<__nv_bfloat16*>(c->a), c->amax, u)),
+               (cod_launch_pdl(c, k_embed_norm<float, ROW_WIDE_NV>, R, row_threads(c->D), 0, st, static_cast<const float*>(c->w.emb), bonus, f.block, f.mask_token_id, f.vocab, static_cast<const float*>(c->w.g_attn), c->D, f.rms_eps, c->x, static_cast<float*>(c->a), c->amax, u)));
   }
   COD_CHECK_LAUNCH(c);
   return COD_OK;

@@ -2,16 +2,52 @@
 // "GreedyVerify"), plus the cos/sin tables of the positions this round touches.
 #include "cod_internal.cuh"
 
+// cos/sin of pos * theta^(-2j/hd) for the window rows (pos = L_s + p) and the next block's
+// rows (pos = L_s + m_s + i). The angle is formed and reduced modulo 2*pi in double, so
+// positions of tens of thousands lose nothing in float.
+struct RopeTabs {
+  const double* inv_freq;     // null: the verify kernel leaves the tables to k_rope_tables
+  int half;
+  float* rope_win;
+  float* rope_blk;
+};
+__device__ __forceinline__ void rope_entry(const RopeTabs& t, int r, int j, int pos_win, int pos_blk) {
+  const double two_pi = 6.283185307179586476925286766559;
+  const double f = t.inv_freq[j];
+  float sn, cs;
+  if (t.rope_win) {
+    double a = static_cast<double>(pos_win) * f;
+    a -= two_pi * rint(a / two_pi);
+    sincosf(static_cast<float>(a), &sn, &cs);
+    t.rope_win[r * 2 * t.half + j] = cs; t.rope_win[r * 2 * t.half + t.half + j] = sn;
+  }
+  if (t.rope_blk) {
+    double b = static_cast<double>(pos_blk) * f;
+    b -= two_pi * rint(b / two_pi);
+    sincosf(static_cast<float>(b), &sn, &cs);
+    t.rope_blk[r * 2 * t.half + j] = cs; t.rope_blk[r * 2 * t.half + t.half + j] = sn;
+  }
+}
+__global__ void k_rope_tables(const int32_t* __restrict__ committed_len, const int32_t* __restrict__ accept_len,
+                              int S, int W, RopeTabs t) {
+  cod_pdl_prologue();
+  const int r = blockIdx.x, s = r / W, p = r - s * W;
+  const int L = max(committed_len[s], 0);
+  const int m = accept_len ? accept_len[s] : 0;
+  for (int j = threadIdx.x; j < t.half; j += blockDim.x) rope_entry(t, r, j, L + p, L + m + p);
+}
+
 // One block. A warp handles one sequence at a time: each lane compares one window row,
 // a ballot finds the first mismatch (acceptance is a PREFIX rule: a later match after the
 // first mismatch does not count). Then a scan over sequences gives the CSR offsets and
-// all threads write the per-row arrays.
+// all threads write the per-row arrays (and, for small rounds, the cos/sin tables: one launch
+// fewer at the head of the critical path).
 __global__ void __launch_bounds__(1024)
 k_verify_accept(const int32_t* __restrict__ draft, const int32_t* __restrict__ target, int S, int W,
                 int n_forced, int vocab, int page, int max_pages, int n_pages,
                 const int32_t* __restrict__ committed_len, const int32_t* __restrict__ block_table,
                 cod_split out, uint32_t* status, const float* __restrict__ p_tok,
-                const float* __restrict__ q_tok, const float* __restrict__ u) {
+                const float* __restrict__ q_tok, const float* __restrict__ u, RopeTabs tabs) {
   cod_pdl_prologue();
   extern __shared__ int sm[];
   int* s_m = sm;              // [S]
@@ -97,31 +133,12 @@ k_verify_accept(const int32_t* __restrict__ draft, const int32_t* __restrict__ t
     if (r >= R - acc_total) out.rej_rows[r] = -1;
   }
   if (flags) atomicOr(status, flags);
-}
-
-// cos/sin of pos * theta^(-2j/hd) for the window rows (pos = L_s + p) and the next block's
-// rows (pos = L_s + m_s + i). The angle is formed and reduced modulo 2*pi in double, so
-// positions of tens of thousands lose nothing in float.
-__global__ void k_rope_tables(const int32_t* __restrict__ committed_len, const int32_t* __restrict__ accept_len,
-                              const double* __restrict__ inv_freq, int S, int W, int half,
-                              float* __restrict__ rope_win, float* __restrict__ rope_blk) {
-  cod_pdl_prologue();
-  const int r = blockIdx.x, s = r / W, p = r - s * W;
-  const int L = max(committed_len[s], 0);
-  const int m = accept_len ? accept_len[s] : 0;
-  const double two_pi = 6.283185307179586476925286766559;
-  for (int j = threadIdx.x; j < half; j += blockDim.x) {
-    const double f = inv_freq[j];
-    double a = static_cast<double>(L + p) * f;
-    a -= two_pi * rint(a / two_pi);
-    float sn, cs;
-    sincosf(static_cast<float>(a), &sn, &cs);
-    if (rope_win) { rope_win[r * 2 * half + j] = cs; rope_win[r * 2 * half + half + j] = sn; }
-    double b = static_cast<double>(L + m + p) * f;
-    b -= two_pi * rint(b / two_pi);
-    sincosf(static_cast<float>(b), &sn, &cs);
-    if (rope_blk) { rope_blk[r * 2 * half + j] = cs; rope_blk[r * 2 * half + half + j] = sn; }
-  }
+  if (tabs.inv_freq != nullptr)
+    for (int e = threadIdx.x; e < R * tabs.half; e += blockDim.x) {
+      const int r = e / tabs.half, j = e - r * tabs.half, s = r / W, p = r - s * W;
+      const int L = max(committed_len[s], 0);
+      rope_entry(tabs, r, j, L + p, L + s_m[s] + p);
+    }
 }
 
 int cod_launch_verify(cod_ctx* c, const int32_t* draft, const int32_t* target, int S, int n_forced,
@@ -130,20 +147,24 @@ int cod_launch_verify(cod_ctx* c, const int32_t* draft, const int32_t* target, i
   ProfScope prof(c, COD_K_VERIFY, st);
   const int W = c->cfg.block;
   const size_t smem = static_cast<size_t>(2 * S + 2) * sizeof(int);
+  const RopeTabs tabs{c->inv_freq_d, c->half, c->rope_win, c->rope_blk};
+  const bool fold = S * W * c->half <= 4096;        // a few table entries per thread at most
   cod_launch_pdl(c, k_verify_accept, 1, 1024, smem, st, draft, target, S, W, n_forced, c->cfg.vocab, c->cfg.page_size,
                                          c->cfg.max_pages_per_seq, c->cfg.n_pages, state->committed_len,
-                                         state->block_table, *out, c->status, p_tok, q_tok, u);
+                                         state->block_table, *out, c->status, p_tok, q_tok, u,
+                                         fold ? tabs : RopeTabs{nullptr, 0, nullptr, nullptr});
   COD_CHECK_LAUNCH(c);
-  cod_launch_pdl(c, k_rope_tables, S * W, 64, 0, st, state->committed_len, out->accept_len, c->inv_freq_d, S, W, c->half,
-                                      c->rope_win, c->rope_blk);
-  COD_CHECK_LAUNCH(c);
+  if (!fold) {
+    cod_launch_pdl(c, k_rope_tables, S * W, 64, 0, st, state->committed_len, out->accept_len, S, W, tabs);
+    COD_CHECK_LAUNCH(c);
+  }
   return COD_OK;
 }
 
 int cod_launch_rope_blk_only(cod_ctx* c, const int32_t* committed_len, int S, cudaStream_t st) {
   ProfScope prof(c, COD_K_VERIFY, st);
-  cod_launch_pdl(c, k_rope_tables, S * c->cfg.block, 64, 0, st, committed_len, nullptr, c->inv_freq_d, S, c->cfg.block, c->half,
-                                                 nullptr, c->rope_blk);
+  cod_launch_pdl(c, k_rope_tables, S * c->cfg.block, 64, 0, st, committed_len, nullptr, S, c->cfg.block,
+                 RopeTabs{c->inv_freq_d, c->half, nullptr, c->rope_blk});
   COD_CHECK_LAUNCH(c);
   return COD_OK;
 }
