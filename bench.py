@@ -301,8 +301,24 @@ def run_gpu(args):
     H_dev = [h.cuda() for h in H_pin]
     d_dev = [d.cuda() for d in d_pin]
     t_dev = [t.cuda() for t in t_pin]
-    stage_H, stage_d, stage_t = torch.empty_like(H_dev[0]), torch.empty_like(d_dev[0]), torch.empty_like(t_dev[0])
+    # end-to-end staging: a round's three inputs sit in ONE pinned host buffer (256-byte aligned parts), so a
+    # step pays for one host-to-device copy; stage_H / stage_d / stage_t are views of its device twin
+    def _packed(parts, device, pin):
+        offs, n = [], 0
+        for t in parts:
+            offs.append(n)
+            n += (t.numel() * t.element_size() + 255) // 256 * 256
+        buf = torch.empty(n, dtype=torch.uint8, device=device, pin_memory=pin)
+        views = [buf[o:o + t.numel() * t.element_size()].view(t.dtype).view(t.shape) for o, t in zip(offs, parts)]
+        return buf, views
+    stage_buf, (stage_H, stage_d, stage_t) = _packed((H_pin[0], d_pin[0], t_pin[0]), "cuda", False)
+    pin_bufs = []
+    for i in range(ring):
+        buf, (vh, vd, vt) = _packed((H_pin[i], d_pin[i], t_pin[i]), "cpu", True)
+        vh.copy_(H_pin[i]); vd.copy_(d_pin[i]); vt.copy_(t_pin[i])
+        pin_bufs.append(buf)
     next_draft = torch.zeros((wl.S, sh.W), dtype=torch.int32, device="cuda")
+    out_pin = torch.zeros((wl.S, sh.W), dtype=torch.int32).pin_memory()
     L0 = state.committed_len.clone()
 
     def reset():
@@ -351,14 +367,14 @@ def run_gpu(args):
         def step(r):
             i = r % ring
             if e2e:
-                stage_H.copy_(H_pin[i], non_blocking=True)
-                stage_d.copy_(d_pin[i], non_blocking=True)
-                stage_t.copy_(t_pin[i], non_blocking=True)
+                stage_buf.copy_(pin_bufs[i], non_blocking=True)
                 if use_graph:
                     graphs[(0, mode, True)].replay()
                 else:
                     launch_round(i, mode, staged=True)
-                return next_draft.cpu()
+                out_pin.copy_(next_draft, non_blocking=True)  # the step's result, read on the host
+                torch.cuda.current_stream().synchronize()
+                return out_pin
             if use_graph:
                 graphs[(i, mode, False)].replay()
             else:
@@ -445,7 +461,7 @@ def run_gpu(args):
                "sample": f"{len(times)} whole rounds of {S_sample} of {wl.S} sequences at full shapes "
                          f"(float64 numpy, {mean:.2f} s each); rounds/s scaled by {S_sample}/{wl.S}"}
 
-    h2d = int(H_pin[0].numel() * H_pin[0].element_size() + d_pin[0].numel() * 4 + t_pin[0].numel() * 4)
+    h2d = int(stage_buf.numel())                            # the one packed copy (parts padded to 256 bytes)
     line = {
         "metric": METRIC, "value": job_throughput(ms, K, world), "unit": UNIT, "n_gpus": world, "steps": K, "warmup": Wm,
         "ms_per_step": ms / K, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
