@@ -368,6 +368,30 @@ def lm_head_argmax(x: np.ndarray, w: Dict[str, np.ndarray], cfg: OracleConfig):
     return tok, gap, logits
 
 
+def lm_head_rank(x: np.ndarray, ref_tok: np.ndarray, w: Dict[str, np.ndarray], cfg: OracleConfig,
+                 tol: float = 0.0):
+    """Rank of a reference token among the drafter's candidates (Section 5.1 "Target-token recall at
+    matched anchors": Recall@k asks whether the target's top token is among the drafter's k best, i.e.
+    whether this rank is below k).  rank[r] = number of vocabulary entries v != ref_tok[r] whose logit
+    N_f(x[r]) . Emb[v] is above the reference token's, ties going to the lower index.
+
+    Returns (rank, ref_logit, rank_lo, rank_hi): rank_lo / rank_hi count the entries above
+    ref_logit + tol resp. above ref_logit - tol, the window inside which an implementation in other
+    arithmetic may legitimately land."""
+    y = rmsnorm(x, w["g_final"], cfg.rms_eps)
+    logits = y @ w["emb"].T
+    R, V = logits.shape
+    ref_tok = np.asarray(ref_tok, dtype=np.int64)
+    ref = logits[np.arange(R), ref_tok]
+    idx = np.arange(V)[None, :]
+    other = idx != ref_tok[:, None]
+    above = (logits > ref[:, None]) | ((logits == ref[:, None]) & (idx < ref_tok[:, None]))
+    rank = (above & other).sum(axis=1).astype(np.int32)
+    rank_lo = ((logits > ref[:, None] + tol) & other).sum(axis=1).astype(np.int32)
+    rank_hi = ((logits > ref[:, None] - tol) & other).sum(axis=1).astype(np.int32)
+    return rank, ref, rank_lo, rank_hi
+
+
 # --------------------------------------------------------------------------- sampling head
 def counter_uniform(seed: int, step: int, row: np.ndarray, col: np.ndarray) -> np.ndarray:
     """The counter-based uniform number U(seed, step, row, col) in (0, 1) both sides draw for the

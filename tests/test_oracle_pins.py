@@ -848,6 +848,49 @@ def test_gumbel_max_sample_follows_the_softmax_and_reports_its_probability():
     assert np.abs(counts / n - sm).max() < 4 * math.sqrt(0.25 / n)
 
 
+def test_rank_of_a_reference_token_sort_position_argmax_and_recall():
+    """lm_head_rank against a stable sort (torch), the argmax (rank 0), hand-planted ties and the
+    Recall@k reading of Section 5.1 (a hit iff rank < k: monotone in k, certain at k = V)."""
+    wl = synth.scaled(synth.workload("cfg1"), vocab=40)
+    cfg = oracle_config(wl.shape)
+    w = orc.prepare_weights(synth.make_weights(wl.shape, 5))
+    rng = np.random.default_rng(3)
+    R, V = 9, 40
+    x = rng.standard_normal((R, cfg.d_model))
+    ref = rng.integers(0, V, size=R)
+    tok, _, logits = orc.lm_head_argmax(x, w, cfg)
+    rank, ref_logit, lo, hi = orc.lm_head_rank(x, ref, w, cfg, tol=0.0)
+    # position of the reference token in a descending stable sort (ties keep index order)
+    order = torch.sort(torch.from_numpy(-logits), dim=1, stable=True).indices.numpy()
+    for r in range(R):
+        assert rank[r] == int(np.where(order[r] == ref[r])[0][0])
+        assert ref_logit[r] == logits[r, ref[r]]
+    assert np.array_equal(lo, rank) and np.array_equal(hi, rank)          # no exact ties in random data
+    # the argmax has rank 0, and only it
+    r0, _, _, _ = orc.lm_head_rank(x, tok, w, cfg)
+    assert np.array_equal(r0, np.zeros(R, dtype=np.int32))
+    assert ((rank == 0) == (ref == tok)).all()
+    # planted ties: identical embedding rows give identical logits; the lower index ranks first
+    w2 = dict(w); w2["emb"] = w["emb"].copy()
+    w2["emb"][7] = w2["emb"][3]; w2["emb"][21] = w2["emb"][3]
+    ra, _, _, _ = orc.lm_head_rank(x, np.full(R, 3), w2, cfg)
+    rb, _, _, _ = orc.lm_head_rank(x, np.full(R, 7), w2, cfg)
+    rc, _, lo_c, hi_c = orc.lm_head_rank(x, np.full(R, 21), w2, cfg, tol=1e-9)
+    assert np.array_equal(rb, ra + 1) and np.array_equal(rc, ra + 2)
+    assert np.array_equal(lo_c, ra) and np.array_equal(hi_c, ra + 2)      # the window spans the tie group
+    # Recall@k = mean(rank < k): monotone in k, 1 at k = V; Recall@1 = agreement with the argmax
+    rec = [float((rank < k).mean()) for k in range(1, V + 1)]
+    assert all(b >= a for a, b in zip(rec, rec[1:])) and rec[-1] == 1.0
+    assert rec[0] == float((ref == tok).mean())
+    # brute force over rows and vocabulary, plain Python
+    for r in range(R):
+        cnt = 0
+        for v in range(V):
+            if v != ref[r] and (logits[r, v] > logits[r, ref[r]] or (logits[r, v] == logits[r, ref[r]] and v < ref[r])):
+                cnt += 1
+        assert cnt == rank[r]
+
+
 # ----------------------------------------------------------------------------- other ways to mark rejected rows
 def test_carry_variants_relate_as_they_must():
     """'none' is the embedding variant with E_carry = 0; 'projector' with F_rej = F is 'none';
