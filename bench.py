@@ -534,6 +534,9 @@ def run_micro(args):
             def call():
                 step_no[0] += 1
                 ctx.lm_head_sample(x, wl.R, args.seed, step_no[0], tok, qv, None)
+        elif args.micro == "lmrank":      # rank of a reference token, counted in the same contraction
+            ref = torch.randint(0, sh.vocab, (wl.R,), generator=gen, device="cuda", dtype=torch.int32)
+            call = lambda: ctx.lm_head_rank(x, wl.R, ref, tok)
         else:
             call = lambda: ctx.lm_head_argmax(x, wl.R, tok)
         nbytes = float(sh.vocab * sh.d_model * 2 + wl.R * sh.d_model * 2)
@@ -632,7 +635,7 @@ def main():
     ap.add_argument("--no-graph", action="store_true", help="time plain stream launches instead of graph replays")
     ap.add_argument("--sweep", action="store_true", help="carryover-overhead sweep over batch, block and rejected fraction")
     ap.add_argument("--attn-split", type=int, default=0, help="keys per attention split (0 = library default)")
-    ap.add_argument("--micro", default=None, choices=["attn", "lmhead", "lmsample"],
+    ap.add_argument("--micro", default=None, choices=["attn", "lmhead", "lmsample", "lmrank"],
                     help="time one entry point alone (small footprint; meant for profiler captures)")
     args = ap.parse_args()
     if args.warmup < 3:

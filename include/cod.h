@@ -18,8 +18,8 @@
  * cod_lm_head_sample, cod_draft_round_stochastic), the two other ways of
  * marking rejected rows the paper compares (COD_F_NO_CARRY_EMBED,
  * COD_F_REJ_PROJECTOR), retention of rejected rows over several rounds
- * (cod_config.carry_rounds) and two analysis aids (cod_taps.carry_mass,
- * cod_reconvergence_count).
+ * (cod_config.carry_rounds) and three analysis aids (cod_taps.carry_mass,
+ * cod_reconvergence_count, cod_lm_head_rank).
  *
  * Conventions
  *   - Every function returns 0 (COD_OK) or a negative cod_status. Nothing throws.
@@ -250,6 +250,19 @@ int cod_lm_head_argmax(cod_ctx* ctx, const float* x, int n_rows, int32_t* tok, f
    bf16 contexts on the tensor-core kernels only; otherwise COD_ERR_UNSUPPORTED. */
 int cod_lm_head_sample(cod_ctx* ctx, const float* x, int n_rows, unsigned long long seed, uint32_t step,
                        int32_t* tok, float* q_tok, float* lse, cod_stream_t stream);
+
+/* Rank of a reference token among the drafter's candidates (Section 5.1 "Target-token recall at
+   matched anchors": with ref_tok the target's top token, Recall@k is the share of rows with
+   rank < k). rank[r] = number of vocabulary entries v != ref_tok[r] with
+   Emb[v] . N_f(x[r]) above Emb[ref_tok[r]] . N_f(x[r]), ties going to the lower index. The count
+   is taken inside the LM-head contraction; logits are never materialised. The reference logit is a
+   separate float dot product of the same operands, so entries within rounding distance of it may
+   fall on either side.
+   x [n_rows, D] device float32; ref_tok [n_rows] device int32 (out of range: COD_DEV_BAD_TOKEN,
+   token 0 is used); rank [n_rows] device int32; ref_logit (nullable) [n_rows] device float.
+   bf16 contexts on the tensor-core kernels only; otherwise COD_ERR_UNSUPPORTED. */
+int cod_lm_head_rank(cod_ctx* ctx, const float* x, int n_rows, const int32_t* ref_tok, int32_t* rank,
+                     float* ref_logit, cod_stream_t stream);
 
 /* The same argmax as cod_lm_head_argmax for callers that may not allocate device memory: it needs
    no cod_ctx and calls no cudaMalloc / cudaFree or any allocating routine. (The paper has no

@@ -369,7 +369,7 @@ def lm_head_argmax(x: np.ndarray, w: Dict[str, np.ndarray], cfg: OracleConfig):
 
 
 def lm_head_rank(x: np.ndarray, ref_tok: np.ndarray, w: Dict[str, np.ndarray], cfg: OracleConfig,
-                 tol: float = 0.0):
+                 tol: float = 0.0, round_act=None):
     """Rank of a reference token among the drafter's candidates (Section 5.1 "Target-token recall at
     matched anchors": Recall@k asks whether the target's top token is among the drafter's k best, i.e.
     whether this rank is below k).  rank[r] = number of vocabulary entries v != ref_tok[r] whose logit
@@ -377,8 +377,12 @@ def lm_head_rank(x: np.ndarray, ref_tok: np.ndarray, w: Dict[str, np.ndarray], c
 
     Returns (rank, ref_logit, rank_lo, rank_hi): rank_lo / rank_hi count the entries above
     ref_logit + tol resp. above ref_logit - tol, the window inside which an implementation in other
-    arithmetic may legitimately land."""
+    arithmetic may legitimately land.  A rank is an integer decided by floating point: round_act
+    (default none), applied to the normalised activations, lets a test take that decision in the
+    operand precision of the implementation it checks (e.g. rounding to bfloat16)."""
     y = rmsnorm(x, w["g_final"], cfg.rms_eps)
+    if round_act is not None:
+        y = round_act(y)
     logits = y @ w["emb"].T
     R, V = logits.shape
     ref_tok = np.asarray(ref_tok, dtype=np.int64)

@@ -28,7 +28,7 @@ DEV_BAD_TOKEN, DEV_PAGE_OVERFLOW, DEV_BAD_PAGE, DEV_TIMEOUT, DEV_BAD_LEN = 1, 2,
 EXPORTS = ("cod_create", "cod_destroy", "cod_set_weights", "cod_verify_accept", "cod_project_kv",
            "cod_scatter_kv", "cod_block_attn", "cod_lm_head_argmax", "cod_lm_head_argmax_static",
            "cod_draft_round", "cod_reconvergence_count", "cod_verify_accept_stochastic",
-           "cod_draft_round_stochastic", "cod_lm_head_sample",
+           "cod_draft_round_stochastic", "cod_lm_head_sample", "cod_lm_head_rank",
            "cod_poll_status", "cod_profile_enable", "cod_profile_read", "cod_launch_count",
            "cod_workspace_bytes", "cod_error_string")
 KERNEL_CLASSES = ("verify", "fc", "kv", "qkv", "attn", "oproj", "lmhead", "rowops", "mlp")
@@ -85,6 +85,7 @@ def load_library() -> C.CDLL:
                                     vp, C.POINTER(CodTaps), vp]
     lib.cod_reconvergence_count.argtypes = [vp, vp, vp, vp, i32, vp, vp]
     lib.cod_lm_head_sample.argtypes = [vp, vp, i32, C.c_uint64, C.c_uint32, vp, vp, vp, vp]
+    lib.cod_lm_head_rank.argtypes = [vp, vp, i32, vp, vp, vp, vp]
     lib.cod_verify_accept_stochastic.argtypes = [vp, vp, vp, vp, vp, i32, i32, C.POINTER(CodState), C.POINTER(CodSplit), vp]
     lib.cod_draft_round_stochastic.argtypes = [vp, vp, vp, vp, vp, vp, i32, i32, i32, C.POINTER(CodState),
                                                C.POINTER(CodSplit), vp, C.POINTER(CodTaps), vp, C.c_uint64,
@@ -284,6 +285,10 @@ class Context:
     def lm_head_sample(self, x, n_rows, seed, step, tok, q_tok=None, lse=None) -> None:
         _check("cod_lm_head_sample", lib().cod_lm_head_sample(
             self._h, _ptr(x), n_rows, seed, step, _ptr(tok), _ptr(q_tok), _ptr(lse), _stream()))
+
+    def lm_head_rank(self, x, n_rows, ref_tok, rank, ref_logit=None) -> None:
+        _check("cod_lm_head_rank", lib().cod_lm_head_rank(
+            self._h, _ptr(x), n_rows, _ptr(ref_tok), _ptr(rank), _ptr(ref_logit), _stream()))
 
     def reconvergence_count(self, z, y, length, S, out) -> None:
         _check("cod_reconvergence_count", lib().cod_reconvergence_count(

@@ -548,6 +548,28 @@ int cod_lm_head_sample(cod_ctx* c, const float* x, int n_rows, unsigned long lon
   return cod_launch_finalize_sample(c, n_rows, g.sample_state, tok, q_tok, lse, s);
 }
 
+int cod_lm_head_rank(cod_ctx* c, const float* x, int n_rows, const int32_t* ref_tok, int32_t* rank,
+                     float* ref_logit, cod_stream_t stream) {
+  if (!c || !x || !ref_tok || !rank || misaligned(x)) return COD_ERR_INVALID_ARG;
+  if (n_rows < 1 || n_rows > c->R_max) return COD_ERR_INVALID_ARG;
+  if (!c->has_weights) return COD_ERR_NO_WEIGHTS;
+  GemmArgs g{};
+  g.A = c->a; g.lda = c->D; g.n_rows = n_rows; g.K = c->D;
+  g.seg[0] = {c->w.emb, c->cfg.vocab, c->emb_tiled}; g.n_seg = 1;
+  g.splits = 1; g.klass = COD_K_LMHEAD;
+  g.rank_ref = ref_logit ? ref_logit : reinterpret_cast<float*>(c->lse_part);   // scratch of the sampling head otherwise
+  g.rank_tok = c->tok;
+  g.rank_out = reinterpret_cast<unsigned int*>(rank);
+  if (c->force_simt || !cod_gemm_tc_supported(c, g)) return COD_ERR_UNSUPPORTED;
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  c->pdl = true;
+  int rc = cod_launch_resid_norm(c, nullptr, 0, n_rows, const_cast<float*>(x), c->w.g_final, nullptr, s);
+  if (rc != COD_OK) return rc;
+  if ((rc = cod_launch_rank_ref(c, n_rows, ref_tok, const_cast<float*>(g.rank_ref), c->tok, rank, s)) != COD_OK) return rc;
+  ProfScope prof(c, COD_K_LMHEAD, s);
+  return cod_launch_gemm_tc(c, g, s);
+}
+
 int cod_draft_round(cod_ctx* c, const int32_t* draft, const int32_t* target, const void* H, int S,
                     int n_forced, int mode, cod_state* st, cod_split* split_out, int32_t* next_draft,
                     const cod_taps* taps, cod_stream_t stream) {

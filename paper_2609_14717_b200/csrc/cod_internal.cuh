@@ -112,6 +112,11 @@ struct GemmArgs {
   float2* lse_part;       // null: plain argmax
   uint32_t sample_state;  // hash state after seed and step
   int klass;              // cod_kernel_class, for the optional timing
+  // rank form (k_gemm_tc only): rank_out[i] += number of weight rows n != rank_tok[i] whose product with
+  // row i lies above rank_ref[i] (ties: lower n first); nothing else is stored
+  const float* rank_ref;
+  const int32_t* rank_tok;
+  unsigned int* rank_out;
 };
 
 #define COD_PROF_SLOTS 4096
@@ -260,6 +265,9 @@ int cod_launch_update_lens(cod_ctx* c, const cod_split* sp, int S, int mode, con
 // sp non-null: the kernel also performs cod_launch_update_lens's update (inside a round)
 int cod_launch_embed_norm(cod_ctx* c, const int32_t* bonus, int S, cudaStream_t st, const cod_split* sp = nullptr,
                           int mode = 0, const cod_state* ds = nullptr);
+// reference logits ref[r] = a[r] . Emb[tok[r]] of the rank form; also sanitises the tokens and zeroes the counts
+int cod_launch_rank_ref(cod_ctx* c, int n_rows, const int32_t* ref_tok, float* ref, int32_t* tok_clean,
+                        int32_t* rank, cudaStream_t st);
 int cod_launch_qkv_finish(cod_ctx* c, const float* part, int splits, int R, int layer, cudaStream_t st);
 int cod_launch_swiglu_finish(cod_ctx* c, const float* part, int splits, int R, cudaStream_t st);
 int cod_launch_rope_qk(cod_ctx* c, const void* q, const void* k, const int32_t* committed_len, int S,

@@ -45,6 +45,10 @@ struct TcParams {
   float2* lse_part;           // sampling form of the argmax epilogue (null: plain argmax)
   uint32_t sample_state;
   uint32_t* status;
+  // rank form (RANK kernels): per token row, how many weight rows score above a reference row
+  const float* rank_ref;      // [n_rows] the reference row's logit
+  const int32_t* rank_tok;    // [n_rows] the reference row's index (excluded from the count)
+  unsigned int* rank_out;     // [n_rows] counts, zero before the launch
 };
 
 // AND of a predicate over the 128 threads of warps 0-3 (named barrier 1)
@@ -59,10 +63,11 @@ __device__ __forceinline__ bool bar_and_128(bool v) {
 }
 
 
-// SAMPLE selects the sampling form of the argmax epilogue and WIDE the transposing store epilogue
-// (32 token rows and more) at compile time, so the kernel a batch-1 round launches a dozen times
-// carries neither: with ~45 short kernels per round, instruction fetch of cold code shows.
-template <bool SAMPLE, bool WIDE>
+// SAMPLE selects the sampling form of the argmax epilogue, WIDE the transposing store epilogue
+// (32 token rows and more) and RANK the counting epilogue at compile time, so the kernel a batch-1
+// round launches a dozen times carries none of them: with ~45 short kernels per round, instruction
+// fetch of cold code shows.
+template <bool SAMPLE, bool WIDE, bool RANK>
 __global__ void __launch_bounds__(NTHREADS, 1)
 k_gemm_tc(const __grid_constant__ CUtensorMap map_w0, const __grid_constant__ CUtensorMap map_w1,
           const __grid_constant__ CUtensorMap map_w2, const __grid_constant__ CUtensorMap map_a, const TcParams p) {
@@ -175,7 +180,43 @@ k_gemm_tc(const __grid_constant__ CUtensorMap map_w0, const __grid_constant__ CU
     const int f = f0 + warp * 32 + lane;                    // weight row within the segment
     const bool f_ok = f < seg_N;
     const uint32_t t_lane = tmem_base + (static_cast<uint32_t>(warp * 32) << 16);
-    if (WIDE && ok && p.amax == nullptr) {
+    if (RANK) {
+      // Per token column: how many of this warp's 32 weight rows lie above the column's reference
+      // logit (ties: the lower index first; the reference row itself never counts). One ballot per
+      // column, lane j keeps column c + j. References sit in the idle pipeline buffers.
+      float* ref_v = reinterpret_cast<float*>(sm);
+      int* ref_t = reinterpret_cast<int*>(sm + 1024);
+      unsigned int* cnt = reinterpret_cast<unsigned int*>(red);
+      for (int t = threadIdx.x; t < p.NT; t += 128) {
+        const bool in = i0 + t < n_rows;
+        ref_v[t] = in ? p.rank_ref[i0 + t] : INFINITY;
+        ref_t[t] = in ? p.rank_tok[i0 + t] : -1;
+      }
+      asm volatile("bar.sync 1, 128;" ::: "memory");
+      const int idx = col0 + warp * 32 + lane;
+      for (int c = 0; c < p.NT && ok; c += 32) {
+        uint32_t v[32];
+        if (c + 32 <= p.NT) {
+          tmem_ld32(t_lane + c, v);
+        } else {                                   // NT is a multiple of 16: a last half chunk
+          uint32_t h[16];
+          tmem_ld16(t_lane + c, h);
+#pragma unroll
+          for (int j = 0; j < 16; ++j) { v[j] = h[j]; v[16 + j] = 0xFF800000u; }
+        }
+        unsigned int mine = 0;
+#pragma unroll
+        for (int j = 0; j < 32; ++j) {
+          const int cj = min(c + j, p.NT - 1);
+          const float x = __uint_as_float(v[j]), rv = ref_v[cj];
+          const int rt = ref_t[cj];
+          const bool above = f_ok && c + j < p.NT && idx != rt && (x > rv || (x == rv && idx < rt));
+          const unsigned int b = __ballot_sync(0xffffffffu, above);
+          if (lane == j) mine = __popc(b);
+        }
+        if (c + lane < p.NT) cnt[warp * p.NT + c + lane] = mine;
+      }
+    } else if (WIDE && ok && p.amax == nullptr) {
       // The accumulator has features on lanes and tokens on columns; C wants a token's features
       // contiguous. Transpose 32 tokens at a time through the (now idle) pipeline buffers and store
       // whole 512-byte feature runs: two 16 KB buffers, one barrier of the four warps per chunk.
@@ -275,6 +316,15 @@ k_gemm_tc(const __grid_constant__ CUtensorMap map_w0, const __grid_constant__ CU
     // give copies that may still be in flight time to land before the shared memory is released
     for (int i = 0; i < 64; ++i) __nanosleep(1000);
     __syncthreads();
+  }
+  else if (RANK) {
+    if (n_kb > 0) {
+      const unsigned int* cnt = reinterpret_cast<const unsigned int*>(red);
+      for (int t = threadIdx.x; t < p.NT; t += NTHREADS) {
+        const unsigned int total = cnt[t] + cnt[p.NT + t] + cnt[2 * p.NT + t] + cnt[3 * p.NT + t];
+        if (i0 + t < n_rows && total) atomicAdd(p.rank_out + i0 + t, total);
+      }
+    }
   }
   else if (p.amax != nullptr && n_kb > 0) {
     // the four epilogue warps merged their per-token keys in shared memory: one atomic per token
@@ -380,22 +430,24 @@ int cod_launch_gemm_tc(cod_ctx* c, const GemmArgs& g, cudaStream_t st) {
   if (!make_map_2d(&ma, g.A, g.n_rows, g.K, g.lda, p.NT)) return COD_ERR_CUDA;
 
   const size_t smem = static_cast<size_t>(stages) * stage_bytes + 1024 /* alignment slack */ + 34 * 8 + 4 * p.NT * 8;
-  // three instantiations: plain (narrow store or argmax), wide store, sampling argmax
-  const int variant = p.lse_part != nullptr ? 2 : ((p.amax == nullptr && p.staged && p.NT >= 32) ? 1 : 0);
-  static size_t configured[3] = {0, 0, 0};
+  // four instantiations: plain (narrow store or argmax), wide store, sampling argmax, rank count
+  const bool rank = g.rank_out != nullptr;
+  if (rank) {
+    if (g.amax != nullptr || g.rank_ref == nullptr || g.rank_tok == nullptr) return COD_ERR_INVALID_ARG;
+    p.rank_ref = g.rank_ref; p.rank_tok = g.rank_tok; p.rank_out = g.rank_out;
+  }
+  const int variant = rank ? 3 : (p.lse_part != nullptr ? 2 : ((p.amax == nullptr && p.staged && p.NT >= 32) ? 1 : 0));
+  using kernel_t = void (*)(const CUtensorMap, const CUtensorMap, const CUtensorMap, const CUtensorMap, const TcParams);
+  static const kernel_t kernels[4] = {k_gemm_tc<false, false, false>, k_gemm_tc<false, true, false>,
+                                      k_gemm_tc<true, false, false>, k_gemm_tc<false, false, true>};
+  static size_t configured[4] = {0, 0, 0, 0};
   if (smem > configured[variant]) {
-    const int bytes = static_cast<int>(smem);
-    const cudaError_t e =
-        variant == 2 ? cudaFuncSetAttribute(k_gemm_tc<true, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes)
-        : variant == 1 ? cudaFuncSetAttribute(k_gemm_tc<false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes)
-                       : cudaFuncSetAttribute(k_gemm_tc<false, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
-    if (e != cudaSuccess) return COD_ERR_CUDA;
+    if (cudaFuncSetAttribute(kernels[variant], cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem)) != cudaSuccess)
+      return COD_ERR_CUDA;
     configured[variant] = smem;
   }
   dim3 grid((g.n_rows + p.NT - 1) / p.NT, tiles, splits);
-  if (variant == 2) cod_launch_pdl(c, k_gemm_tc<true, false>, grid, NTHREADS, smem, st, mw[0], mw[1], mw[2], ma, p);
-  else if (variant == 1) cod_launch_pdl(c, k_gemm_tc<false, true>, grid, NTHREADS, smem, st, mw[0], mw[1], mw[2], ma, p);
-  else cod_launch_pdl(c, k_gemm_tc<false, false>, grid, NTHREADS, smem, st, mw[0], mw[1], mw[2], ma, p);
+  cod_launch_pdl(c, kernels[variant], grid, NTHREADS, smem, st, mw[0], mw[1], mw[2], ma, p);
   COD_CHECK_LAUNCH(c);
   return COD_OK;
 }

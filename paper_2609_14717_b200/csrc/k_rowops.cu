@@ -638,6 +638,42 @@ int cod_launch_qkv_finish(cod_ctx* c, const float* part, int splits, int R, int 
   return COD_OK;
 }
 
+// ------------------------------------------------------------------ reference logits of the rank head
+// ref[r] = a[r] . Emb[tok[r]] in float (the operands the contraction reads); out-of-range tokens are
+// flagged and replaced by 0; the row's count starts at zero.
+template <typename T>
+__global__ void k_rank_ref(const T* __restrict__ a, const T* __restrict__ emb, const int32_t* __restrict__ ref_tok,
+                           int D, int vocab, float* __restrict__ ref, int32_t* __restrict__ tok_clean,
+                           int32_t* __restrict__ rank, uint32_t* status) {
+  cod_pdl_prologue();
+  __shared__ float red[33];
+  const int r = blockIdx.x;
+  int tok = ref_tok[r];
+  if (tok < 0 || tok >= vocab) {
+    if (threadIdx.x == 0) atomicOr(status, COD_DEV_BAD_TOKEN);
+    tok = 0;
+  }
+  const T* x = a + static_cast<size_t>(r) * D;
+  const T* e = emb + static_cast<size_t>(tok) * D;
+  float acc = 0.f;
+  for (int j = threadIdx.x * 4; j < D; j += blockDim.x * 4) {       // D % 8 == 0
+    const float4 u = cod_ld4(x + j), v = cod_ld4(e + j);
+    acc = fmaf(u.x, v.x, fmaf(u.y, v.y, fmaf(u.z, v.z, fmaf(u.w, v.w, acc))));
+  }
+  acc = cod_block_sum(acc, red);
+  if (threadIdx.x == 0) { ref[r] = acc; tok_clean[r] = tok; rank[r] = 0; }
+}
+
+int cod_launch_rank_ref(cod_ctx* c, int n_rows, const int32_t* ref_tok, float* ref, int32_t* tok_clean,
+                        int32_t* rank, cudaStream_t st) {
+  ProfScope prof(c, COD_K_ROWOPS, st);
+  DISPATCH_T(c,
+             (cod_launch_pdl(c, k_rank_ref<__nv_bfloat16>, n_rows, 256, 0, st, static_cast<const __nv_bfloat16*>(c->a), static_cast<const __nv_bfloat16*>(c->w.emb), ref_tok, c->D, c->cfg.vocab, ref, tok_clean, rank, c->status)),
+             (cod_launch_pdl(c, k_rank_ref<float>, n_rows, 256, 0, st, static_cast<const float*>(c->a), static_cast<const float*>(c->w.emb), ref_tok, c->D, c->cfg.vocab, ref, tok_clean, rank, c->status)));
+  COD_CHECK_LAUNCH(c);
+  return COD_OK;
+}
+
 int cod_launch_swiglu_finish(cod_ctx* c, const float* part, int splits, int R, cudaStream_t st) {
   ProfScope prof(c, COD_K_ROWOPS, st);
   const int d_ff = c->cfg.d_ff;

@@ -166,3 +166,42 @@ def test_full_size_sampling_head_on_sampled_rows(name, rows):
     assert ctx.poll_status() == 0
     ctx.close()
 
+
+
+@pytest.mark.parametrize("name,rows", [("cfg2", list(range(16))), ("cfg3", [0, 1, 37, 255, 256, 300, 510, 511])])
+def test_full_size_rank_head_on_sampled_rows(name, rows):
+    """cod_lm_head_rank over the full vocabulary (151936) at 16 and 512 rows (one and two token tiles of
+    the contraction); the oracle ranks the sampled rows from bfloat16 activations. References: the
+    oracle's j-th best token for small j (what Recall@k looks at) and random tokens."""
+    from paper_2609_14717_b200 import binding as B
+    wl = synth.scaled(synth.workload(name), n_rounds=1, ctx=(16, 16), n_layers=1)
+    sh = wl.shape
+    lay = synth.make_layout(wl, 3)
+    w = synth.make_weights(sh, 3)
+    ctx = B.Context(B.make_config(sh, wl.S, int(lay["max_pages_per_seq"]), int(lay["n_pages"])))
+    ctx.set_weights(B.weights_to_device(w, sh.dtype))
+    R = wl.R
+    rng = np.random.default_rng(7)
+    x = rng.standard_normal((R, sh.d_model)).astype(np.float32)
+    w_o = {"g_final": np.asarray(w["g_final"], dtype=np.float64), "emb": np.asarray(w["emb"], dtype=np.float64)}
+    cfg_o = oracle_config(sh)
+    rows = np.array(rows)
+    rnd = lambda y: torch.from_numpy(np.asarray(y, dtype=np.float32)).to(torch.bfloat16).to(torch.float64).numpy()
+    _, _, logits = orc.lm_head_argmax(x[rows], w_o, cfg_o)
+    order = np.argsort(-logits, axis=1, kind="stable")
+    ref = rng.integers(0, sh.vocab, size=R).astype(np.int32)
+    picks = [0, 1, 3, 15, 16, 63, 1000, 0]
+    for i, r in enumerate(rows):
+        ref[r] = order[i, picks[i % len(picks)]]
+    rank = torch.full((R,), -3, dtype=torch.int32, device="cuda")
+    ctx.lm_head_rank(torch.from_numpy(x).cuda(), R, torch.from_numpy(ref).cuda(), rank)
+    torch.cuda.synchronize()
+    r_o, _, lo, hi = orc.lm_head_rank(x[rows], ref[rows], w_o, cfg_o, tol=1e-3, round_act=rnd)
+    g = rank.cpu().numpy()
+    assert (g >= 0).all() and (g < sh.vocab).all()
+    assert ((lo <= g[rows]) & (g[rows] <= hi)).all(), (g[rows], lo, hi)
+    exact = lo == hi
+    assert exact.sum() >= len(rows) // 2
+    assert np.array_equal(g[rows][exact], r_o[exact])
+    assert ctx.poll_status() == 0
+    ctx.close()

@@ -582,3 +582,76 @@ def test_lm_head_sample_parity(name):
     assert P.ctx.poll_status() == 0
     P.close()
 
+
+def _bf16_round(y):
+    return torch.from_numpy(np.asarray(y, dtype=np.float32)).to(torch.bfloat16).to(torch.float64).numpy()
+
+
+def _rank_refs(x, w_o, cfg_o, rng):
+    """Reference tokens spread over the ranking: the oracle's j-th best token for assorted j (the small
+    ranks Recall@k looks at), and uniformly random tokens."""
+    _, _, logits = orc.lm_head_argmax(x, w_o, cfg_o)
+    order = np.argsort(-logits, axis=1, kind="stable")
+    V = logits.shape[1]
+    picks = [0, 1, 2, 5, 15, 16, 100 % V, V - 1]
+    ref = np.empty(x.shape[0], dtype=np.int32)
+    for r in range(x.shape[0]):
+        ref[r] = order[r, picks[r % len(picks)]] if r % 3 else rng.integers(0, V)
+    return ref
+
+
+@pytest.mark.parametrize("name", ["small_bf16", "small_bf16_W8", "mid_bf16"])
+def test_lm_head_rank_parity(name):
+    """Rank of a reference token counted inside the LM-head contraction. The decision 'above the
+    reference' is taken on both sides from bfloat16 activations (the kernel's operand precision); what
+    is left is summation order, so the count must sit in the oracle's +-1e-3 window and equal the
+    oracle's rank wherever that window is a single value."""
+    B = _B()
+    Hn = _H()
+    wl = _workloads()[name]
+    P = Hn.Pair(wl, seed=9, fill_pool=False)
+    sh = wl.shape
+    R = wl.R
+    rng = np.random.default_rng(6)
+    x = rng.standard_normal((R, sh.d_model)).astype(np.float32)
+    ref = _rank_refs(x, P.w_o, P.cfg_o, rng)
+    rank = torch.full((R,), -7, dtype=torch.int32, device="cuda")
+    ref_logit = torch.zeros(R, dtype=torch.float32, device="cuda")
+    P.ctx.lm_head_rank(torch.from_numpy(x).cuda(), R, torch.from_numpy(ref).cuda(), rank, ref_logit)
+    torch.cuda.synchronize()
+    r_o, l_o, lo, hi = orc.lm_head_rank(x, ref, P.w_o, P.cfg_o, tol=1e-3, round_act=_bf16_round)
+    g = rank.cpu().numpy()
+    assert np.max(np.abs(ref_logit.cpu().numpy() - l_o)) <= 1e-3
+    assert ((lo <= g) & (g <= hi)).all(), (g, lo, hi)
+    exact = lo == hi
+    assert exact.sum() >= R // 2
+    assert np.array_equal(g[exact], r_o[exact])
+    # without the optional output, and a second call on the same context: same counts
+    rank2 = torch.full((R,), 5, dtype=torch.int32, device="cuda")
+    P.ctx.lm_head_rank(torch.from_numpy(x).cuda(), R, torch.from_numpy(ref).cuda(), rank2)
+    torch.cuda.synchronize()
+    assert np.array_equal(rank2.cpu().numpy(), g)
+    assert P.ctx.poll_status() == 0
+    # an out-of-range reference is flagged and counted as token 0
+    bad = torch.from_numpy(ref).cuda().clone()
+    bad[0] = sh.vocab
+    P.ctx.lm_head_rank(torch.from_numpy(x).cuda(), R, bad, rank2)
+    torch.cuda.synchronize()
+    assert P.ctx.poll_status() == B.DEV_BAD_TOKEN
+    r0, _, lo0, hi0 = orc.lm_head_rank(x[:1], np.zeros(1, dtype=np.int32), P.w_o, P.cfg_o, tol=1e-3, round_act=_bf16_round)
+    assert lo0[0] <= int(rank2[0]) <= hi0[0]
+    P.close()
+
+
+def test_lm_head_rank_unsupported_in_float32():
+    B = _B()
+    Hn = _H()
+    P = Hn.Pair(_workloads()["tiny_f32"], seed=1, fill_pool=False)
+    R = P.wl.R
+    x = torch.zeros(R, P.wl.shape.d_model, device="cuda")
+    rank = torch.zeros(R, dtype=torch.int32, device="cuda")
+    with pytest.raises(B.CodError) as e:
+        P.ctx.lm_head_rank(x, R, torch.zeros(R, dtype=torch.int32, device="cuda"), rank)
+    assert e.value.status == -2                                 # COD_ERR_UNSUPPORTED
+    P.close()
+
