@@ -701,7 +701,15 @@ int cod_launch_rope_qk(cod_ctx* c, const void* q, const void* k, const int32_t* 
 int cod_launch_resid_norm(cod_ctx* c, const float* part, int splits, int R, float* x, const void* gain,
                           float* tap_x, cudaStream_t st) {
   ProfScope prof(c, COD_K_ROWOPS, st);
-  if (row_narrow(c->D)) {
+  // More rows than one wave of one-slot-per-thread blocks holds (three 640-thread blocks per SM at D = 2560):
+  // two slots per thread and half the threads, so every row is resident at once.
+  const int nt1 = row_threads(c->D);
+  if (row_narrow(c->D) && R > (2048 / nt1) * c->n_sm && nt1 >= 256) {
+    const int nt2 = ((c->D / 8 + 31) / 32) * 32;
+    DISPATCH_T(c,
+               (cod_launch_pdl(c, k_resid_norm<__nv_bfloat16, 2>, R, nt2, 0, st, part, splits, R, c->D, x, static_cast<const __nv_bfloat16*>(gain), c->cfg.rms_eps, static_cast<__nv_bfloat16*>(c->a), tap_x, c->amax)),
+               (cod_launch_pdl(c, k_resid_norm<float, 2>, R, nt2, 0, st, part, splits, R, c->D, x, static_cast<const float*>(gain), c->cfg.rms_eps, static_cast<float*>(c->a), tap_x, c->amax)));
+  } else if (row_narrow(c->D)) {
     DISPATCH_T(c,
                (cod_launch_pdl(c, k_resid_norm<__nv_bfloat16, 1>, R, row_threads(c->D), 0, st, part, splits, R, c->D, x, static_cast<const __nv_bfloat16*>(gain), c->cfg.rms_eps, static_cast<__nv_bfloat16*>(c->a), tap_x, c->amax)),
                (cod_launch_pdl(c, k_resid_norm<float, 1>, R, row_threads(c->D), 0, st, part, splits, R, c->D, x, static_cast<const float*>(gain), c->cfg.rms_eps, static_cast<float*>(c->a), tap_x, c->amax)));
