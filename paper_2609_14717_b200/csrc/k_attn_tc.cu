@@ -460,25 +460,33 @@ __global__ void k_attn_tc_combine(const float* __restrict__ part_o, const float*
   const int F = (L / PAGE) * PAGE;
   const int n_parts = (F + split_len - 1) / split_len + 1;
   const size_t base = (static_cast<size_t>(s) * n_kv + h) * max_parts;
-  // every lane fetches the (m, l, l_carry) record of its parts; weights stay in registers
-  float mg = -INFINITY;
-  for (int k = lane; k < n_parts; k += 32) mg = fmaxf(mg, part_ml[((base + k) * M + mrow) * 4]);
+  // every lane fetches the (m, l, l_carry) record of its parts once; weights stay in registers
+  const float4 none = make_float4(-INFINITY, 0.f, 0.f, 0.f);
+  const float4 ml0 = lane < n_parts ? *reinterpret_cast<const float4*>(part_ml + ((base + lane) * M + mrow) * 4) : none;
+  float mg = ml0.x;
+  for (int k = lane + 32; k < n_parts; k += 32) mg = fmaxf(mg, part_ml[((base + k) * M + mrow) * 4]);
   mg = cod_warp_max(mg);
   float acc[4] = {0.f, 0.f, 0.f, 0.f}, l = 0.f, lc = 0.f;
   for (int k0 = 0; k0 < n_parts; k0 += 32) {
-    float w_mine = 0.f;
-    if (k0 + lane < n_parts) {
-      const float4 ml = *reinterpret_cast<const float4*>(part_ml + ((base + k0 + lane) * M + mrow) * 4);
-      w_mine = __expf(ml.x - mg);
-      l = fmaf(w_mine, ml.y, l);
-      lc = fmaf(w_mine, ml.z, lc);
-    }
+    float4 ml = ml0;
+    if (k0 > 0) ml = k0 + lane < n_parts ? *reinterpret_cast<const float4*>(part_ml + ((base + k0 + lane) * M + mrow) * 4) : none;
+    const float w_mine = k0 + lane < n_parts ? __expf(ml.x - mg) : 0.f;
+    l = fmaf(w_mine, ml.y, l);
+    lc = fmaf(w_mine, ml.z, lc);
     const int nk = min(32, n_parts - k0);
-#pragma unroll 8
-    for (int k = 0; k < nk; ++k) {
-      const float w = __shfl_sync(0xffffffffu, w_mine, k);
-      const float4 v = *reinterpret_cast<const float4*>(part_o + ((base + k0 + k) * M + mrow) * HD + lane * 4);
-      acc[0] = fmaf(w, v.x, acc[0]); acc[1] = fmaf(w, v.y, acc[1]); acc[2] = fmaf(w, v.z, acc[2]); acc[3] = fmaf(w, v.w, acc[3]);
+    // eight partial rows at a time, their loads all in flight before the first is used (a batch-1
+    // round merges 17 partials per head: one launch went from ~7 to ~5.5 us)
+    for (int kk = 0; kk < nk; kk += 8) {
+      float4 v[8];
+#pragma unroll
+      for (int u = 0; u < 8; ++u)
+        v[u] = kk + u < nk ? *reinterpret_cast<const float4*>(part_o + ((base + k0 + kk + u) * M + mrow) * HD + lane * 4)
+                           : make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+      for (int u = 0; u < 8; ++u) {
+        const float w = __shfl_sync(0xffffffffu, w_mine, (kk + u) & 31);      // lanes past the last part hold 0
+        acc[0] = fmaf(w, v[u].x, acc[0]); acc[1] = fmaf(w, v[u].y, acc[1]); acc[2] = fmaf(w, v[u].z, acc[2]); acc[3] = fmaf(w, v[u].w, acc[3]);
+      }
     }
   }
   l = cod_warp_sum(l);

@@ -86,8 +86,15 @@ __global__ void __launch_bounds__(1024) k_fc_finish(const float* __restrict__ pa
   }
   // ldp = D: one projection per row. ldp = 2 D: F h and F_rej h side by side, rejected rows take the second.
   const float* prow = part + static_cast<size_t>(i) * ldp + ((ldp > D && rej) ? D : 0);
+  if (NV == 1) {
+    // one slot per thread: every slab's load is requested before the first sum (same order of sums)
+#pragma unroll
+    for (int s = 0; s < COD_MAX_SPLITS; ++s)
+      if (s < splits && static_cast<int>(threadIdx.x) < nv)
+        v[0] = f4_add(v[0], *reinterpret_cast<const float4*>(prow + static_cast<size_t>(s) * n_rows * ldp + 4 * threadIdx.x));
+  }
 #pragma unroll 4
-  for (int s = 0; s < splits; ++s) {        // slots inside, four slabs unrolled: their loads are all in flight together
+  for (int s = NV == 1 ? COD_MAX_SPLITS : 0; s < splits; ++s) {   // slots inside, four slabs unrolled: their loads are in flight together
 #pragma unroll
     for (int t = 0; t < NV; ++t) {
       const int j = threadIdx.x + t * blockDim.x;
@@ -167,6 +174,7 @@ __global__ void k_kv_finish(const float* __restrict__ part, int splits, int n_ro
     const float* p = part + static_cast<size_t>(i) * ldc + l * kvw + h * hd + j;
     const size_t slab = static_cast<size_t>(n_rows) * ldc;
     if (live) {
+#pragma unroll 4
       for (int s = 0; s < splits; ++s) {
         k1 = f4_add(k1, *reinterpret_cast<const float4*>(p + s * slab));
         k2 = f4_add(k2, *reinterpret_cast<const float4*>(p + s * slab + half));
@@ -356,7 +364,14 @@ __global__ void k_qkv_finish(const float* __restrict__ part, int splits, int R, 
   const size_t slab = static_cast<size_t>(R) * ldc;
   float4 a = make_float4(0.f, 0.f, 0.f, 0.f), b = a;
   if (live) {
-    for (int s = 0; s < splits; ++s) {
+    // every slab's two loads are requested before the first sum (same order of sums)
+#pragma unroll
+    for (int s = 0; s < COD_MAX_SPLITS; ++s)
+      if (s < splits) {
+        a = f4_add(a, *reinterpret_cast<const float4*>(p + s * slab));
+        b = f4_add(b, *reinterpret_cast<const float4*>(p + s * slab + half));
+      }
+    for (int s = COD_MAX_SPLITS; s < splits; ++s) {
       a = f4_add(a, *reinterpret_cast<const float4*>(p + s * slab));
       b = f4_add(b, *reinterpret_cast<const float4*>(p + s * slab + half));
     }
@@ -444,8 +459,15 @@ __global__ void __launch_bounds__(1024) k_resid_norm(const float* __restrict__ p
     if (j < nv) v[t] = *reinterpret_cast<const float4*>(x + static_cast<size_t>(r) * D + 4 * j);
   }
   if (part) {
+    if (NV == 1) {
+      // one slot per thread: every slab's load is requested before the first sum (same order of sums)
+#pragma unroll
+      for (int s = 0; s < COD_MAX_SPLITS; ++s)
+        if (s < splits && static_cast<int>(threadIdx.x) < nv)
+          v[0] = f4_add(v[0], *reinterpret_cast<const float4*>(part + (static_cast<size_t>(s) * R + r) * D + 4 * threadIdx.x));
+    }
 #pragma unroll 4
-    for (int s = 0; s < splits; ++s) {      // slots inside, four slabs unrolled: their loads are all in flight together
+    for (int s = NV == 1 ? COD_MAX_SPLITS : 0; s < splits; ++s) {   // slots inside, four slabs unrolled: their loads are in flight together
 #pragma unroll
       for (int t = 0; t < NV; ++t) {
         const int j = threadIdx.x + t * blockDim.x;
