@@ -155,6 +155,8 @@ struct cod_ctx {
   int* carry_base;             // [max_batch] rows of U kept from earlier rounds (carry_rounds > 1), else null
   int* carry_drop;             // [max_batch] rows of U that leave this round (carry_rounds > 1), else null
   float* gemm_out2;            // a second, small slab buffer for the side branch of the round (null: no side branch)
+  int* attn_order;             // [max_batch * tc_max_parts] longest-first work list of the tensor-core attention
+  bool attn_order_stale;       // the lengths may have changed since the list was built
   int side_rows;               // the side branch is used for rounds of at most this many rows
   cudaStream_t side;           // side branch of the round: the first layer's embedding / Q/K/V chain
   cudaEvent_t ev_fork, ev_join;

@@ -41,6 +41,8 @@ struct AttnParams {
   int max_parts;                        // partial slots per (sequence, KV head)
   float* part_o;                        // [S][n_kv][max_parts][M][hd]
   float* part_ml;                       // [S][n_kv][max_parts][M][4]   m (natural log units), l, l_carry
+  const int* order;                     // null: CTA (x, y, z) = (part, head, sequence). Else CTA (x, y) = (head, i) works
+                                        // on part order[i] = sequence << 16 | part, longest first; -1: nothing
   uint32_t* status;
 };
 
@@ -88,7 +90,12 @@ k_attn_tc(const __grid_constant__ CUtensorMap map_pool, const __grid_constant__ 
   int* page_ids = reinterpret_cast<int*>(bars + 28);       // [split_len / 16] <= 256 entries
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int split = blockIdx.x, h = blockIdx.y, s = blockIdx.z;
+  int split = blockIdx.x, h = blockIdx.y, s = blockIdx.z;
+  if (p.order != nullptr) {
+    const int item = p.order[blockIdx.y];
+    if (item < 0) return;
+    h = blockIdx.x; s = item >> 16; split = item & 0xFFFF;
+  }
   const int M = p.W * p.rep;
 
   uint32_t flags = 0;
@@ -443,6 +450,46 @@ k_attn_tc(const __grid_constant__ CUtensorMap map_pool, const __grid_constant__ 
   }
 }
 
+// Work order for grids several waves deep: every (sequence, part) that exists, longest first, so the
+// last wave is made of short parts instead of whichever sequences come last (a counting sort by
+// iteration count in one block; the order inside a bucket is arbitrary and affects no result).
+template <int KEYS_IT>
+__global__ void k_attn_order(const int* __restrict__ committed_len, int S, int max_pages, int split_len,
+                             int max_parts, int* __restrict__ order) {
+  cod_pdl_prologue();
+  constexpr int NB = 4096 / 64 + 3;              // keys: 0 absent, 1 tail, 1 + iterations of a paged part
+  __shared__ int hist[NB], cur[NB], n_items;
+  for (int k = threadIdx.x; k < NB; k += blockDim.x) hist[k] = 0;
+  __syncthreads();
+  const int n_max = S * max_parts;
+  auto key_of = [&](int i) -> int {
+    const int s = i / max_parts, split = i - s * max_parts;
+    const int L = max(0, min(committed_len[s], max_pages * PAGE));
+    const int F = (L / PAGE) * PAGE;
+    const int n_reg = (F + split_len - 1) / split_len;
+    if (split > n_reg) return 0;
+    if (split == n_reg) return 1;
+    const int keys = min(F, (split + 1) * split_len) - split * split_len;
+    return min(NB - 1, 1 + (keys + KEYS_IT - 1) / KEYS_IT);
+  };
+  for (int i = threadIdx.x; i < n_max; i += blockDim.x) atomicAdd(&hist[key_of(i)], 1);
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    int pos = 0;
+    for (int k = NB - 1; k >= 1; --k) { cur[k] = pos; pos += hist[k]; }
+    n_items = pos;
+  }
+  __syncthreads();
+  for (int i = threadIdx.x; i < n_max; i += blockDim.x) {
+    const int k = key_of(i);
+    if (k > 0) {
+      const int s = i / max_parts;
+      order[atomicAdd(&cur[k], 1)] = (s << 16) | (i - s * max_parts);
+    }
+  }
+  for (int i = n_items + threadIdx.x; i < n_max; i += blockDim.x) order[i] = -1;
+}
+
 // Merges the partials of one (row, query head); one warp each. Empty partials carry m = -inf, l = 0.
 template <bool DUAL>
 __global__ void k_attn_tc_combine(const float* __restrict__ part_o, const float* __restrict__ part_ml,
@@ -527,6 +574,18 @@ int launch(cod_ctx* c, int layer, const void* q, const void* kb, const void* vb,
     configured = true;
   }
   dim3 grid(c->tc_max_parts, f.n_kv_heads, S);
+  // more than two waves of CTAs: longest parts first (the list holds until the lengths change)
+  if (c->attn_order != nullptr && static_cast<long long>(S) * f.n_kv_heads * c->tc_max_parts > 4ll * c->n_sm && S < 32768 &&
+      static_cast<long long>(S) * c->tc_max_parts <= 65535) {
+    if (c->attn_order_stale) {
+      cod_launch_pdl(c, k_attn_order<G::KEYS_IT>, 1, 256, 0, st, stt->committed_len, S, f.max_pages_per_seq, c->tc_split_len,
+                     c->tc_max_parts, c->attn_order);
+      COD_CHECK_LAUNCH(c);
+      c->attn_order_stale = false;
+    }
+    p.order = c->attn_order;
+    grid = dim3(f.n_kv_heads, S * c->tc_max_parts, 1);
+  }
   cod_launch_pdl(c, k_attn_tc<DUAL>, grid, NTHREADS, G::SMEM, st, mp, mz, p);
   COD_CHECK_LAUNCH(c);
   const int items = S * f.block * f.n_q_heads;

@@ -174,7 +174,7 @@ k_gemm_tc(const __grid_constant__ CUtensorMap map_w0, const __grid_constant__ CU
     }
   } else if (n_kb > 0) {
     // ------------------------------------------------ epilogue warps 0..3
-    // one verdict for the four epilogue warps (they meet at a named barrier below)
+    // one decision for the four epilogue warps (they meet at a named barrier below)
     const bool ok = bar_and_128(mbar_wait(smem_u32(acc_bar), 0, abort_flag, p.status));
     tc_fence_after();
     const int f = f0 + warp * 32 + lane;                    // weight row within the segment

@@ -164,7 +164,7 @@ k_gemm_tc2(const __grid_constant__ CUtensorMap map_w0, const __grid_constant__ C
   // Warp w reads tensor-memory lanes 32 * (w % 4) .. +31 (the only lanes it may touch); warps 0-3
   // take the first half of the token columns, warps 4-7 the second.
   if (n_kb > 0) {
-    // one verdict for everyone (the warps meet at named barriers below)
+    // one decision for everyone (the warps meet at named barriers below)
     const bool ok = __syncthreads_and(mbar_wait(smem_u32(acc_bar), 0, abort_flag, p.status)) != 0;
     tc_fence_after();
     const int qw = warp & 3, grp = warp >> 2;
