@@ -507,7 +507,15 @@ __global__ void k_attn_tc_combine(const float* __restrict__ part_o, const float*
   const int F = (L / PAGE) * PAGE;
   const int n_parts = (F + split_len - 1) / split_len + 1;
   const size_t base = (static_cast<size_t>(s) * n_kv + h) * max_parts;
-  // every lane fetches the (m, l, l_carry) record of its parts once; weights stay in registers
+  // The first four partial rows are requested together with the (m, l, l_carry) records (they need only
+  // the part count): at large batches the partials have left L2 by now and every dependent trip costs.
+  // Every lane fetches the record of its parts once; weights stay in registers.
+  constexpr int C0 = 4;
+  const float4 zero4 = make_float4(0.f, 0.f, 0.f, 0.f);
+  float4 v0[C0];
+#pragma unroll
+  for (int u = 0; u < C0; ++u)
+    v0[u] = u < n_parts ? *reinterpret_cast<const float4*>(part_o + ((base + u) * M + mrow) * HD + lane * 4) : zero4;
   const float4 none = make_float4(-INFINITY, 0.f, 0.f, 0.f);
   const float4 ml0 = lane < n_parts ? *reinterpret_cast<const float4*>(part_ml + ((base + lane) * M + mrow) * 4) : none;
   float mg = ml0.x;
@@ -521,17 +529,25 @@ __global__ void k_attn_tc_combine(const float* __restrict__ part_o, const float*
     l = fmaf(w_mine, ml.y, l);
     lc = fmaf(w_mine, ml.z, lc);
     const int nk = min(32, n_parts - k0);
-    // eight partial rows at a time, their loads all in flight before the first is used (a batch-1
-    // round merges 17 partials per head: one launch went from ~7 to ~5.5 us)
-    for (int kk = 0; kk < nk; kk += 8) {
+    int kk = 0;
+    if (k0 == 0) {
+#pragma unroll
+      for (int u = 0; u < C0; ++u) {
+        const float w = __shfl_sync(0xffffffffu, w_mine, u);                  // lanes past the last part hold 0
+        acc[0] = fmaf(w, v0[u].x, acc[0]); acc[1] = fmaf(w, v0[u].y, acc[1]); acc[2] = fmaf(w, v0[u].z, acc[2]); acc[3] = fmaf(w, v0[u].w, acc[3]);
+      }
+      kk = C0;
+    }
+    // then eight partial rows at a time, their loads all in flight before the first is used (a batch-1
+    // round merges 17 partials per head)
+    for (; kk < nk; kk += 8) {
       float4 v[8];
 #pragma unroll
       for (int u = 0; u < 8; ++u)
-        v[u] = kk + u < nk ? *reinterpret_cast<const float4*>(part_o + ((base + k0 + kk + u) * M + mrow) * HD + lane * 4)
-                           : make_float4(0.f, 0.f, 0.f, 0.f);
+        v[u] = kk + u < nk ? *reinterpret_cast<const float4*>(part_o + ((base + k0 + kk + u) * M + mrow) * HD + lane * 4) : zero4;
 #pragma unroll
       for (int u = 0; u < 8; ++u) {
-        const float w = __shfl_sync(0xffffffffu, w_mine, (kk + u) & 31);      // lanes past the last part hold 0
+        const float w = __shfl_sync(0xffffffffu, w_mine, (kk + u) & 31);
         acc[0] = fmaf(w, v[u].x, acc[0]); acc[1] = fmaf(w, v[u].y, acc[1]); acc[2] = fmaf(w, v[u].z, acc[2]); acc[3] = fmaf(w, v[u].w, acc[3]);
       }
     }
