@@ -113,6 +113,9 @@ def _workloads():
         "small_bf16_keep2": small_bf16(S=3, W=16, n_layers=2, ctx=(40, 300), carry_rounds=2, n_rounds=6),
         "small_bf16_W32_keep2": small_bf16(S=2, W=32, n_layers=1, ctx=(100, 200), carry_rounds=2, n_rounds=6),
         "tiny_f32_keep3": synth.scaled(synth.workload("cfg1"), S=3, ctx=(5, 140), n_rounds=8, carry_rounds=3),
+        # enough (sequence, head, part) CTAs for the attention kernel's longest-first work list (more than two
+        # waves of the machine at 128 keys per part), with empty, one-page and ragged contexts among them
+        "order_bf16": small_bf16(S=48, W=16, n_layers=2, ctx=(0, 900), d_model=1024, n_q=8, n_kv=2, vocab=1500),
         "mid_bf16_full": small_bf16(S=34, W=16, n_layers=2, ctx=(100, 600), d_target=512, n_cap=5, d_model=1024,
                                     n_q=8, n_kv=2, vocab=3000, d_ff=1536, qk_norm=True),
     }
@@ -205,7 +208,7 @@ def _set_carry(P, rng, lens):
 
 @pytest.mark.parametrize("name,split_len", [("tiny_f32", 32), ("tiny_f32", 0), ("small_bf16", 64),
                                             ("small_bf16_W32", 32), ("small_bf16_W8", 0), ("long_bf16", 1024),
-                                            ("long_bf16", 256), ("long_bf16_W32", 512), ("mid_bf16", 0)])
+                                            ("long_bf16", 256), ("long_bf16_W32", 512), ("mid_bf16", 0), ("order_bf16", 128)])
 def test_block_attn_parity(name, split_len):
     B, Hn = _B(), _H()
     wl = _workloads()[name]
@@ -221,9 +224,14 @@ def test_block_attn_parity(name, split_len):
         for layer in range(sh.n_layers):
             for use_carry in (True, False):
                 ref, mref = orc.block_attn(layer, q, kb, vb, P.st_o, use_carry)
+                n0 = P.ctx.launch_count()
                 P.ctx.block_attn(layer, B.to_device(q, sh.dtype), B.to_device(kb, sh.dtype), B.to_device(vb, sh.dtype),
                                  P.st_g, wl.S, use_carry, out, mass)
                 torch.cuda.synchronize()
+                if name == "order_bf16":                 # tables, rotation, work list, attention, merge
+                    assert P.ctx.launch_count() - n0 == 5
+                elif name == "mid_bf16":                 # a shallow grid runs without the work list
+                    assert P.ctx.launch_count() - n0 == 4
                 got = out.float().cpu().numpy()
                 assert np.isfinite(got).all()            # poisoned pages / stale carry rows never read
                 assert rel_err(got, ref) <= tol
@@ -339,7 +347,7 @@ def test_round_parity_cfg1_every_round():
     ("tiny_f32_full", 40.0, orc.MODE_CARRY), ("tiny_f32_full", 40.0, orc.MODE_BASELINE),
     ("small_bf16_full", 30.0, orc.MODE_CARRY), ("small_bf16_full", 30.0, orc.MODE_BASELINE),
     ("small_bf16_mlp_only", 30.0, orc.MODE_CARRY), ("small_bf16_qknorm_only", 30.0, orc.MODE_CARRY),
-    ("mid_bf16_full", 30.0, orc.MODE_CARRY),
+    ("mid_bf16_full", 30.0, orc.MODE_CARRY), ("order_bf16", 30.0, orc.MODE_CARRY),
     ("small_bf16_nomark", 30.0, orc.MODE_CARRY), ("small_bf16_proj", 30.0, orc.MODE_CARRY),
     ("small_bf16_proj", 30.0, orc.MODE_BASELINE), ("tiny_f32_proj", 40.0, orc.MODE_CARRY),
     ("small_bf16_keep2", 30.0, orc.MODE_CARRY), ("small_bf16_keep2", 30.0, orc.MODE_BASELINE),
