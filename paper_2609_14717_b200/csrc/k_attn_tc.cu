@@ -590,8 +590,8 @@ int launch(cod_ctx* c, int layer, const void* q, const void* kb, const void* vb,
     configured = true;
   }
   dim3 grid(c->tc_max_parts, f.n_kv_heads, S);
-  // more than two waves of CTAs: longest parts first (the list holds until the lengths change)
-  if (c->attn_order != nullptr && static_cast<long long>(S) * f.n_kv_heads * c->tc_max_parts > 4ll * c->n_sm && S < 32768 &&
+  // more CTAs than fit on the machine at once: longest parts first (the list holds until the lengths change)
+  if (c->attn_order != nullptr && static_cast<long long>(S) * f.n_kv_heads * c->tc_max_parts > 2ll * c->n_sm && S < 32768 &&
       static_cast<long long>(S) * c->tc_max_parts <= 65535) {
     if (c->attn_order_stale) {
       cod_launch_pdl(c, k_attn_order<G::KEYS_IT>, 1, 256, 0, st, stt->committed_len, S, f.max_pages_per_seq, c->tc_split_len,
