@@ -8,6 +8,7 @@ tests/golden/README.md.
 """
 import itertools
 import math
+import os
 
 import numpy as np
 import pytest
@@ -411,7 +412,9 @@ def test_attention_closed_forms():
     vb = np.array([[[[0.0, 1.0, 0.0, 0.0]]]])
     # q and k_blk sit at the same position, so the rotation leaves their product unchanged
     out, _ = orc.block_attn(0, q, kb, vb, st, use_carry=True)
-    assert np.allclose(out[0, 0, 0], [0.25, 0.75, 0.0, 0.0], atol=1e-14)
+    golden = os.path.join(os.path.dirname(__file__), "golden", "attention_two_keys.txt")
+    want = np.loadtxt(golden, comments="#")
+    assert want.shape == (4,) and np.allclose(out[0, 0, 0], want, atol=1e-14)
 
 
 def test_attention_masked_carry_equals_baseline_and_mass():
@@ -592,6 +595,127 @@ def test_round_is_deterministic_and_next_draft_shape():
     nd = outs[0]["next_draft"]
     assert nd.shape == (wl.S, wl.shape.W) and np.array_equal(nd[:, 0], outs[0]["split"]["bonus"])
     assert np.array_equal(nd[:, 1:], outs[0]["tok"][:, 1:])
+
+
+# ----------------------------------------------------------------------------- the drafter pass: attention sub-layer
+def _body_case(n_layers, seed=9, S=2):
+    """A tiny drafter (D = 32) after one carry-mode round, so C_l, U_l and the bonus tokens are real;
+    the attention matrices are scaled up so the sub-layer moves the residual stream by O(1)."""
+    wl = synth.scaled(synth.workload("cfg1"), S=S, ctx=(5, 30), n_layers=n_layers, d_target=16, n_cap=2,
+                      d_model=32, n_q=4, n_kv=2, hd=8, vocab=64, W=4, n_rounds=2,
+                      accept=("rej_uniform", 1, 3))
+    cfg, st, _ = oracle_state(wl, seed)
+    w = orc.prepare_weights(synth.make_weights(wl.shape, seed))
+    for k in ("wq", "wk", "wv", "wo"):
+        w[k] = w[k] * 12.0
+    rd = synth.make_round(wl, seed, 0)
+    res = orc.draft_round(rd["draft"], rd["target"], rd["H"], st, w, 1, orc.MODE_CARRY, keep_logits=True)
+    assert st.carry_len.max() > 0                              # carried rows are part of what is read
+    return wl, cfg, st, w, res
+
+
+def _matvec_loops(Wm, v):
+    """y_i = sum_k W[i, k] v[k] for a matrix stored [out, in], written out."""
+    return [sum(float(Wm[i, k]) * v[k] for k in range(Wm.shape[1])) for i in range(Wm.shape[0])]
+
+
+def _rms_gain_loops(x, g, eps):
+    ms = sum(v * v for v in x) / len(x)
+    return [float(g[k]) * x[k] / math.sqrt(ms + eps) for k in range(len(x))]
+
+
+def test_draft_block_one_layer_written_out_by_hand():
+    """One drafter layer, no MLP: for every block row a = g_attn * x0 / rms(x0); q, k_b, v_b = W a with explicit
+    sums; the (separately pinned) block attention on them; x1 = x0 + W_o o; y = g_final * x1 / rms(x1);
+    token = first index of the largest Emb[v] . y."""
+    wl, cfg, st, w, res = _body_case(n_layers=1)
+    S, W, D = wl.S, cfg.W, cfg.d_model
+    bonus = res["split"]["bonus"]
+    x0 = []
+    for s in range(S):
+        for i in range(W):
+            t = int(bonus[s]) if i == 0 else cfg.mask_token_id
+            x0.append([float(v) for v in w["emb"][t]])
+    q = np.zeros((S, W, cfg.n_q, cfg.hd)); kb = np.zeros((S, W, cfg.n_kv, cfg.hd)); vb = np.zeros_like(kb)
+    for r in range(S * W):
+        a = _rms_gain_loops(x0[r], w["g_attn"][0], cfg.rms_eps)
+        q[r // W, r % W] = np.array(_matvec_loops(w["wq"][0], a)).reshape(cfg.n_q, cfg.hd)
+        kb[r // W, r % W] = np.array(_matvec_loops(w["wk"][0], a)).reshape(cfg.n_kv, cfg.hd)
+        vb[r // W, r % W] = np.array(_matvec_loops(w["wv"][0], a)).reshape(cfg.n_kv, cfg.hd)
+    o, _ = orc.block_attn(0, q, kb, vb, st, use_carry=True)
+    o = o.reshape(S * W, cfg.n_q * cfg.hd)
+    assert np.allclose(res["attn_out"][0], o, atol=1e-10)
+    for r in range(S * W):
+        wo_o = _matvec_loops(w["wo"][0], [float(v) for v in o[r]])
+        x1 = [x0[r][i] + wo_o[i] for i in range(D)]
+        assert np.allclose(res["x_final"][r], x1, atol=1e-10)
+        assert max(abs(v) for v in wo_o) > 1e-2                # the branch under test is not negligible
+        y = _rms_gain_loops(x1, w["g_final"], cfg.rms_eps)
+        logits = [sum(float(w["emb"][v, k]) * y[k] for k in range(D)) for v in range(cfg.vocab)]
+        assert np.allclose(res["logits"][r], logits, atol=1e-10)
+        assert int(res["tok"].reshape(-1)[r]) == logits.index(max(logits))
+
+
+def _torch_body(cfg, st, w, bonus, S, *, gains=None, wo_of=None, order=None, norm_input=True, residual=True):
+    """The attention-only drafter body through torch float64 linear / rms_norm, the oracle's own block
+    attention as the (pinned) inner step.  The keyword switches build the plausible mistakes."""
+    F = torch.nn.functional
+    W = cfg.W
+    toks = np.full((S, W), cfg.mask_token_id, dtype=np.int64)
+    toks[:, 0] = bonus
+    x = torch.from_numpy(w["emb"])[torch.from_numpy(toks.reshape(-1))]
+    gains = w["g_attn"] if gains is None else gains
+    outs = []
+    for l in (range(cfg.n_layers) if order is None else order):
+        a = F.rms_norm(x, (cfg.d_model,), torch.from_numpy(np.ascontiguousarray(gains[l])), cfg.rms_eps)
+        if not norm_input:
+            a = x
+        q = F.linear(a, torch.from_numpy(w["wq"][l])).numpy().reshape(S, W, cfg.n_q, cfg.hd)
+        kb = F.linear(a, torch.from_numpy(w["wk"][l])).numpy().reshape(S, W, cfg.n_kv, cfg.hd)
+        vb = F.linear(a, torch.from_numpy(w["wv"][l])).numpy().reshape(S, W, cfg.n_kv, cfg.hd)
+        o, _ = orc.block_attn(l, q, kb, vb, st, use_carry=True)
+        o = torch.from_numpy(o.reshape(S * W, -1))
+        outs.append(o.numpy())
+        wo = w["wo"][l] if wo_of is None else wo_of(w["wo"][l])
+        upd = F.linear(o, torch.from_numpy(np.ascontiguousarray(wo)))
+        x = x + upd if residual else upd
+    return x.numpy(), outs
+
+
+def test_draft_block_two_layers_against_torch_ops():
+    """Two layers: layer order, g_attn indexed by layer, the residual carried from layer to layer."""
+    wl, cfg, st, w, res = _body_case(n_layers=2, seed=11)
+    x, outs = _torch_body(cfg, st, w, res["split"]["bonus"], wl.S)
+    assert np.allclose(res["x_final"], x, atol=1e-11)
+    for l in range(2):
+        assert np.allclose(res["attn_out"][l], outs[l], atol=1e-11)
+    y = torch.nn.functional.rms_norm(torch.from_numpy(x), (cfg.d_model,), torch.from_numpy(w["g_final"]), cfg.rms_eps)
+    logits = torch.nn.functional.linear(y, torch.from_numpy(w["emb"])).numpy()
+    assert np.allclose(res["logits"], logits, atol=1e-11)
+    assert np.array_equal(res["tok"].reshape(-1), logits.argmax(1))
+
+
+def test_draft_block_pins_would_catch_the_plausible_mistakes():
+    """Each mistake a reader might make in the body changes x_final by far more than the pins' tolerance,
+    so the two tests above do tell them apart from the right computation."""
+    wl, cfg, st, w, res = _body_case(n_layers=2, seed=11)
+    bonus, S = res["split"]["bonus"], wl.S
+    good = res["x_final"]
+    wrong = {
+        "gains of the two layers swapped": dict(gains=w["g_attn"][::-1]),
+        "no gain": dict(gains=np.ones_like(w["g_attn"])),
+        "final gain in place of the layer's": dict(gains=np.stack([w["g_final"]] * 2)),
+        "W_o transposed": dict(wo_of=lambda m: m.T),
+        "q/k/v from the un-normalised stream": dict(norm_input=False),
+        "residual dropped": dict(residual=False),
+        "layers in the wrong order": dict(order=[1, 0]),
+    }
+    for what, kw in wrong.items():
+        x, _ = _torch_body(cfg, st, w, bonus, S, **kw)
+        assert np.abs(x - good).max() > 1e-3, what
+    # the embedding of the block: bonus in row 0, MASK elsewhere
+    x, _ = _torch_body(cfg, st, w, (bonus + 1) % cfg.vocab, S)
+    assert np.abs(x - good).max() > 1e-3
 
 
 # ----------------------------------------------------------------------------- the complete layer
