@@ -31,9 +31,19 @@ normalisation and positional encoding", Section 2.1), the readings taken are:
     g // (n_q / n_kv);
   * the LM head is the transposed embedding table; argmax ties go to the lowest id.
 
+Two ways to run it.  Exact (the default, and the only truth any tolerance is
+judged against): float64 everywhere on the given inputs.  Storage-rounded (a
+DIAGNOSTIC, never the pass/fail truth): the same steps with a caller-supplied
+``round_store`` applied wherever an implementation that keeps bfloat16 tensors
+between its steps would store one (the fused features z, cached K/V, normalised
+activations, the block's rotated q/k and v, attention outputs, MLP activations,
+the LM head's input); it separates storage noise from a real defect when an
+error sits near a bound.  With ``round_store=None`` no arithmetic changes.
+
 Parity status: every function here is pinned by tests/test_oracle_pins.py
 against closed forms, brute force, invariants the paper states, and library
-special cases.  What stays unpinned is the choice of the readings above
+special cases (the drafter pass's attention sub-layer by a hand-written layer
+and by torch linear / rms_norm).  What stays unpinned is the choice of the readings above
 themselves: the paper ships no reference numbers for this path, so they are
 pinned to their written definition only ("parity unpinned" against the authors'
 system for the drafter-body glue).
@@ -238,8 +248,13 @@ def fuse_features(H: np.ndarray, rejected: np.ndarray, w: Dict[str, np.ndarray],
     return Z
 
 
+def _stored(x: np.ndarray, round_store) -> np.ndarray:
+    """x as an implementation with reduced-precision storage would hold it (diagnostic mode only)."""
+    return x if round_store is None else np.asarray(round_store(x), dtype=np.float64)
+
+
 def project_kv(H: np.ndarray, split: Dict[str, np.ndarray], w: Dict[str, np.ndarray],
-               cfg: OracleConfig, mode: int) -> np.ndarray:
+               cfg: OracleConfig, mode: int, round_store=None) -> np.ndarray:
     """J_l = (K_l(Z), V_l(Z)) for every drafter layer (Eq. 1; Algorithm 1 step "J_l").
 
     Carry mode keeps all window rows; baseline mode keeps the accepted rows only
@@ -252,7 +267,7 @@ def project_kv(H: np.ndarray, split: Dict[str, np.ndarray], w: Dict[str, np.ndar
     p_of_row = np.tile(np.arange(W), R // W)
     rejected = p_of_row >= m_of_row
     keep = np.ones(R, dtype=bool) if mode == MODE_CARRY else ~rejected
-    Z = fuse_features(H, rejected, w, cfg)
+    Z = _stored(fuse_features(H, rejected, w, cfg), round_store)
     J = np.full((cfg.n_layers, R, 2, cfg.n_kv, cfg.hd), np.nan, dtype=np.float64)
     pos = np.asarray(split["row_pos"], dtype=np.float64)
     for l in range(cfg.n_layers):
@@ -260,7 +275,8 @@ def project_kv(H: np.ndarray, split: Dict[str, np.ndarray], w: Dict[str, np.ndar
         V = (Z @ w["wv"][l].T).reshape(R, cfg.n_kv, cfg.hd)
         if cfg.qk_norm:
             K = rmsnorm(K, w["g_knorm"][l], cfg.rms_eps)
-        K = rope(K, pos[:, None], cfg.rope_theta)
+        K = _stored(rope(K, pos[:, None], cfg.rope_theta), round_store)
+        V = _stored(V, round_store)
         J[l, keep, 0] = K[keep]
         J[l, keep, 1] = V[keep]
     return J
@@ -324,7 +340,7 @@ def gather_ctx(st: OracleState, layer: int, s: int, use_carry: bool):
 
 
 def block_attn(layer: int, q: np.ndarray, k_blk: np.ndarray, v_blk: np.ndarray,
-               st: OracleState, use_carry: bool):
+               st: OracleState, use_carry: bool, round_store=None):
     """Block attention over [C_l; U_l; block] (Section 2 "Preliminaries": draft positions
     attend to the keys and values made from target hidden states; Algorithm 1: "the next
     draft reads ctx_l").
@@ -341,11 +357,12 @@ def block_attn(layer: int, q: np.ndarray, k_blk: np.ndarray, v_blk: np.ndarray,
     for s in range(S):
         L = int(st.committed_len[s])
         pos = (L + np.arange(W)).astype(np.float64)
-        qr = rope(np.asarray(q[s], dtype=np.float64), pos[:, None], cfg.rope_theta)
-        kr = rope(np.asarray(k_blk[s], dtype=np.float64), pos[:, None], cfg.rope_theta)
+        qr = _stored(rope(np.asarray(q[s], dtype=np.float64), pos[:, None], cfg.rope_theta), round_store)
+        kr = _stored(rope(np.asarray(k_blk[s], dtype=np.float64), pos[:, None], cfg.rope_theta), round_store)
+        vr = _stored(np.asarray(v_blk[s], dtype=np.float64), round_store)
         Kctx, Vctx, c = gather_ctx(st, layer, s, use_carry)
         K = np.concatenate([Kctx, np.transpose(kr, (1, 0, 2))], axis=1)        # [n_kv, T, hd]
-        V = np.concatenate([Vctx, np.transpose(np.asarray(v_blk[s], dtype=np.float64), (1, 0, 2))], axis=1)
+        V = np.concatenate([Vctx, np.transpose(vr, (1, 0, 2))], axis=1)
         for g in range(cfg.n_q):
             h = g // rep
             sc = (qr[:, g, :] @ K[h].T) / np.sqrt(np.float64(cfg.hd))          # [W, T]
@@ -354,13 +371,13 @@ def block_attn(layer: int, q: np.ndarray, k_blk: np.ndarray, v_blk: np.ndarray,
             pr = pr / pr.sum(axis=1, keepdims=True)
             out[s, :, g, :] = pr @ V[h]
             mass[s, :, g] = pr[:, L:L + c].sum(axis=1)
-    return out, mass
+    return _stored(out, round_store), mass
 
 
 # =========================================================================== part 5
-def lm_head_argmax(x: np.ndarray, w: Dict[str, np.ndarray], cfg: OracleConfig):
+def lm_head_argmax(x: np.ndarray, w: Dict[str, np.ndarray], cfg: OracleConfig, round_store=None):
     """logits = N_f(x) Emb^T; token = lowest-index argmax; also the top-2 logit gap."""
-    y = rmsnorm(x, w["g_final"], cfg.rms_eps)
+    y = _stored(rmsnorm(x, w["g_final"], cfg.rms_eps), round_store)
     logits = y @ w["emb"].T
     tok = np.argmax(logits, axis=1).astype(np.int32)          # first occurrence = lowest id
     top2 = np.partition(logits, -2, axis=1)[:, -2:]
@@ -450,7 +467,7 @@ def lm_head_sample(x: np.ndarray, w: Dict[str, np.ndarray], cfg: OracleConfig, s
 
 # =========================================================================== the drafter pass
 def draft_block(st: OracleState, bonus: np.ndarray, w: Dict[str, np.ndarray],
-                use_carry: bool, keep_logits: bool = False) -> Dict[str, np.ndarray]:
+                use_carry: bool, keep_logits: bool = False, round_store=None) -> Dict[str, np.ndarray]:
     """One parallel block prediction from [bonus, MASK, ...] reading ctx_l in every layer."""
     cfg = st.cfg
     S, W, D = st.S, cfg.W, cfg.d_model
@@ -460,20 +477,24 @@ def draft_block(st: OracleState, bonus: np.ndarray, w: Dict[str, np.ndarray],
     attn_out = np.zeros((cfg.n_layers, S * W, cfg.n_q * cfg.hd), dtype=np.float64)
     mass = np.zeros((cfg.n_layers, S, W, cfg.n_q), dtype=np.float64)
     for l in range(cfg.n_layers):
-        a = rmsnorm(x, w["g_attn"][l], cfg.rms_eps)
+        a = _stored(rmsnorm(x, w["g_attn"][l], cfg.rms_eps), round_store)
         q = (a @ w["wq"][l].T).reshape(S, W, cfg.n_q, cfg.hd)
         kb = (a @ w["wk"][l].T).reshape(S, W, cfg.n_kv, cfg.hd)
         vb = (a @ w["wv"][l].T).reshape(S, W, cfg.n_kv, cfg.hd)
         if cfg.qk_norm:
             q = rmsnorm(q, w["g_qnorm"][l], cfg.rms_eps)
             kb = rmsnorm(kb, w["g_knorm"][l], cfg.rms_eps)
-        o, mass[l] = block_attn(l, q, kb, vb, st, use_carry)
+        o, mass[l] = block_attn(l, q, kb, vb, st, use_carry, round_store)
         attn_out[l] = o.reshape(S * W, cfg.n_q * cfg.hd)
         x = x + attn_out[l] @ w["wo"][l].T
         if cfg.d_ff > 0:
-            b = rmsnorm(x, w["g_mlp"][l], cfg.rms_eps)
-            x = x + gated_mlp(b, w["w_gate"][l], w["w_up"][l], w["w_down"][l])
-    tok, gap, logits = lm_head_argmax(x, w, cfg)
+            b = _stored(rmsnorm(x, w["g_mlp"][l], cfg.rms_eps), round_store)
+            if round_store is None:
+                x = x + gated_mlp(b, w["w_gate"][l], w["w_up"][l], w["w_down"][l])
+            else:                                         # the gated activation is a stored tensor too
+                act = _stored(silu(b @ w["w_gate"][l].T) * (b @ w["w_up"][l].T), round_store)
+                x = x + act @ w["w_down"][l].T
+    tok, gap, logits = lm_head_argmax(x, w, cfg, round_store)
     res = {"tok": tok.reshape(S, W), "gap": gap.reshape(S, W), "x_final": x,
            "attn_out": attn_out, "carry_mass": mass}
     if keep_logits:
@@ -483,14 +504,15 @@ def draft_block(st: OracleState, bonus: np.ndarray, w: Dict[str, np.ndarray],
 
 def draft_round(draft: np.ndarray, target: np.ndarray, H: np.ndarray, st: OracleState,
                 w: Dict[str, np.ndarray], n_forced: int, mode: int,
-                keep_logits: bool = False) -> Dict[str, np.ndarray]:
+                keep_logits: bool = False, round_store=None) -> Dict[str, np.ndarray]:
     """verify-accept -> project -> scatter -> draft the next block (Algorithm 1, then
     "the next draft reads ctx_l").  Mutates st.  next_draft = [bonus, tok_1 .. tok_{W-1}]."""
     cfg = st.cfg
     split = verify_accept(draft, target, st.committed_len, st.block_table, cfg.page, n_forced)
-    J = project_kv(H, split, w, cfg, mode)
+    J = project_kv(H, split, w, cfg, mode, round_store)
     scatter_kv(J, split, st, mode)
-    res = draft_block(st, split["bonus"], w, use_carry=(mode == MODE_CARRY), keep_logits=keep_logits)
+    res = draft_block(st, split["bonus"], w, use_carry=(mode == MODE_CARRY), keep_logits=keep_logits,
+                      round_store=round_store)
     next_draft = res["tok"].copy()
     next_draft[:, 0] = split["bonus"]
     res.update(split=split, J=J, next_draft=next_draft.astype(np.int32))

@@ -1086,3 +1086,35 @@ def test_retained_rows_change_the_next_draft_and_k1_is_the_papers_round():
             differs |= np.abs(a["x_final"] - b["x_final"]).max() > 1e-6
     assert differs
 
+
+
+# ----------------------------------------------------------------------------- the storage-rounded diagnostic mode
+def test_storage_rounded_mode_changes_nothing_unless_asked_and_rounds_where_it_says():
+    """round_store = identity is the exact oracle bit for bit; a bfloat16 round_store is called on the
+    tensors an implementation with bf16 hand-offs stores (z, cached K and V per layer, a, rotated q / k_b,
+    v_b, o per layer, b and the gated activation per layer, y), and moves the result by bf16-sized amounts only."""
+    wl = _full_layer_workload(qk_norm=False)
+    w = orc.prepare_weights(synth.make_weights(wl.shape, 3))
+    rd = synth.make_round(wl, 3, 0)
+    runs = {}
+    calls = []
+
+    def bf16(x):
+        calls.append(np.shape(x))
+        return synth.round_bf16(np.asarray(x, dtype=np.float32)).astype(np.float64)
+
+    for name, hook in (("exact", None), ("identity", lambda x: x), ("bf16", bf16)):
+        _, st, _ = oracle_state(wl, 3)
+        runs[name] = orc.draft_round(rd["draft"], rd["target"], rd["H"], st, w, 1, orc.MODE_CARRY, round_store=hook)
+        runs[name]["pool"] = st.pool
+    for k in ("x_final", "attn_out", "J", "tok"):
+        assert np.array_equal(runs["exact"][k], runs["identity"][k], equal_nan=True)
+    Ld, S = wl.shape.n_layers, wl.S
+    # z, (K, V) per layer | per layer: a, then per sequence (q, k_b, v_b), o, b, act | y
+    assert len(calls) == 1 + 2 * Ld + Ld * (1 + 3 * S + 1 + 2) + 1
+    J = runs["bf16"]["J"]
+    kept = ~np.isnan(J)
+    assert np.array_equal(J[kept], synth.round_bf16(J[kept].astype(np.float32)).astype(np.float64))
+    for k in ("x_final", "attn_out"):
+        d = np.abs(runs["bf16"][k] - runs["exact"][k]).max() / np.abs(runs["exact"][k]).max()
+        assert 1e-5 < d < 2e-2, (k, d)
