@@ -278,7 +278,8 @@ int cod_lm_head_rank(cod_ctx* ctx, const float* x, int n_rows, const int32_t* re
    All calls on a device share the scratch, which keeps the last call's contents (what must start
    at zero is cleared by the call itself): calls that overlap on the GPU race with each other.
    The first call on a device looks up the scratch's device address with that device current; it
-   should be made before any stream capture begins. Device-side status bits are not reported. */
+   should be made before any stream capture begins. There is no status word to poll here: a row
+   whose contraction did not complete comes back as tok = -1, every other row as an id in [0, vocab). */
 int cod_lm_head_argmax_static(const void* emb, const void* g_final, const float* x, int n_rows,
                               int d_model, int vocab, int dtype, float rms_eps, int32_t* tok,
                               float* top_logit, cod_stream_t stream);

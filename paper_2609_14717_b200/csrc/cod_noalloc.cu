@@ -15,7 +15,10 @@
 //     kernels clear what has to start at zero (the argmax keys) themselves, but two calls whose
 //     kernels overlap on the GPU (different streams, no dependency) race on the scratch;
 //   * the first call on each device looks up the array's device address (cudaGetSymbolAddress,
-//     with that device current). Make that first call before any stream capture begins.
+//     with that device current). Make that first call before any stream capture begins;
+//   * there is no context, hence no status word to poll: a row whose contraction did not complete
+//     (a bounded device wait that ran out) comes back as tok = -1, every other row as a token id in
+//     [0, vocab). Callers that need to know check for negative tokens.
 #include <string.h>
 
 #include "cod_internal.cuh"
@@ -34,19 +37,24 @@ static __device__ __align__(256) unsigned char g_static_scratch[COD_STATIC_SCRAT
 
 constexpr int MAX_DEVICES = 64;
 unsigned char* g_scratch_addr[MAX_DEVICES];   // per device, filled on first use
+int g_sm_count[MAX_DEVICES];                  // per device, filled with the address
 
-int scratch_for_current_device(unsigned char** out) {
+int scratch_for_current_device(unsigned char** out, int* n_sm) {
   int dev = -1;
   if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= MAX_DEVICES) return COD_ERR_CUDA;
   if (!g_scratch_addr[dev]) {
     void* p = nullptr;
-    if (cudaGetSymbolAddress(&p, g_static_scratch) != cudaSuccess || !p) {
+    int sms = 0;
+    if (cudaGetSymbolAddress(&p, g_static_scratch) != cudaSuccess || !p ||
+        cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sms < 1) {
       cudaGetLastError();
       return COD_ERR_CUDA;
     }
+    g_sm_count[dev] = sms;
     g_scratch_addr[dev] = static_cast<unsigned char*>(p);
   }
   *out = g_scratch_addr[dev];
+  *n_sm = g_sm_count[dev];
   return COD_OK;
 }
 
@@ -63,7 +71,8 @@ extern "C" int cod_lm_head_argmax_static(const void* emb, const void* g_final, c
   if (n_rows > COD_STATIC_MAX_ROWS || d_model > COD_STATIC_MAX_DMODEL) return COD_ERR_TOO_LARGE;
 
   unsigned char* scratch = nullptr;
-  int rc = scratch_for_current_device(&scratch);
+  int n_sm = 0;
+  int rc = scratch_for_current_device(&scratch, &n_sm);
   if (rc != COD_OK) return rc;
 
   // A context on the stack that points the existing kernels at the static scratch. Nothing here
@@ -77,7 +86,7 @@ extern "C" int cod_lm_head_argmax_static(const void* emb, const void* g_final, c
   c.cfg.block = 1;
   c.D = d_model;
   c.R_max = COD_STATIC_MAX_ROWS;
-  c.n_sm = 148;
+  c.n_sm = n_sm;
   c.w.emb = emb;
   c.w.g_final = g_final;
   c.has_weights = true;

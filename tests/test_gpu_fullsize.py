@@ -1,6 +1,6 @@
-"""Parity at the sizes and in the launch configuration bench.py times (batch-1 and batch-32
-configurations, default split lengths, tensor-core kernels), on outputs the oracle can
-afford: the whole batch-1 round, and two sampled sequences of the batch-32 round."""
+"""Parity at the sizes and in the launch configuration bench.py times (batch-1, batch-32 and long-context
+configurations and a 1024-row sweep point, default split lengths, tensor-core kernels), on outputs the
+oracle can afford: the whole batch-1 round, and sampled sequences of the larger batches."""
 import numpy as np
 import pytest
 import torch
@@ -11,20 +11,43 @@ from tests.helpers import oracle_config, rel_err
 
 pytestmark = pytest.mark.gpu
 TOL, GAP = 2e-2, 1e-2
-# Inside a whole round the inputs of layer l > 0 already differ between the two sides: the residual
-# stream, the normalised activations, q/k/v and the attention output are stored in bf16 between the
-# kernels (five layers deep), and in this random-weight model the attention branch dominates the
-# residual stream, so those roundings compound (about 0.5 % per layer; the plain-FMA kernels show the
-# same growth). Each part ALONE, on identical inputs, is held to TOL (K/V rows below, the stand-alone
-# attention test below, the LM-head tests); the downstream taps of the fused round get this bound.
+# Two oracle runs judge the downstream taps of a whole round. The EXACT float64 oracle is the truth. The
+# library hands bfloat16 tensors from kernel to kernel (z, a, q/k/v, o) five layers deep, and the round is
+# sensitive to that: the oracle's storage-rounded mode (bf16 at exactly those hand-off points, float64
+# otherwise) measures how far bf16 hand-offs ALONE move each tap from the exact result - up to ~3e-2 of the
+# tensor's maximum in the deeper layers on these inputs, and two such runs whose pre-rounding values differ
+# by 3e-7 relative end up as far from each other as from the exact result (the rounding noise decorrelates
+# after the first layer, so the diagnostic run bounds the noise, it does not cancel it). Hence: layer 0 is
+# held to TOL against the exact oracle; a deeper tap may exceed TOL only as far as twice the distance the
+# storage-rounded oracle itself shows at that tap in that round, and never beyond TOL_COMPOUNDED. Each part
+# alone, on identical inputs, is held to TOL (K/V rows below, the stand-alone attention test, the LM head).
 TOL_COMPOUNDED = 5e-2
+
+
+def _bf16_store(x):
+    return synth.round_bf16(np.asarray(x, dtype=np.float32)).astype(np.float64)
+
+
+def _row_err(a, ref, width):
+    """max over rows of `width` elements of max|a - ref| / max|ref| of that row: a wrong head or row of
+    small magnitude cannot hide behind the tensor-wide maximum."""
+    a = np.asarray(a, dtype=np.float64).reshape(-1, width)
+    ref = np.asarray(ref, dtype=np.float64).reshape(-1, width)
+    den = np.abs(ref).max(axis=1)
+    return float((np.abs(a - ref).max(axis=1) / np.where(den > 0, den, 1.0)).max())
+
+
+def _named(name):
+    if name == "sweep_S64_W16_m8":
+        return synth.sweep_point(64, 16, 8)
+    return synth.workload(name)
 
 
 def _setup(name, seed, sample):
     """GPU state for the whole batch; oracle state for the sampled sequences only (they are
     independent of the rest), with identical pool contents for those sequences."""
     from paper_2609_14717_b200 import binding as B
-    wl = synth.scaled(synth.workload(name), n_rounds=4)
+    wl = synth.scaled(_named(name), n_rounds=4)
     sh = wl.shape
     lay = synth.make_layout(wl, seed)
     n_pages, mp = int(lay["n_pages"]), int(lay["max_pages_per_seq"])
@@ -51,23 +74,34 @@ def _setup(name, seed, sample):
     return wl, lay, w, ctx, cfg, st_g, cfg_o, st_o
 
 
-@pytest.mark.parametrize("name,sample", [("cfg2", [0]), ("cfg3", [5, 22]), ("cfg2f", [0]), ("cfg3f", [9])])
-def test_full_size_round_on_sampled_sequences(name, sample):
+@pytest.mark.parametrize("name,sample,mode_name,rounds", [
+    ("cfg2", [0], "carry", 2), ("cfg3", [5, 22], "carry", 2), ("cfg2f", [0], "carry", 2), ("cfg3f", [9], "carry", 2),
+    ("cfg4", [2], "carry", 1),                                  # 4 x 32K keys, block 32: one sequence, one round
+    ("sweep_S64_W16_m8", [3, 40], "carry", 1),                  # 1024 window rows at full width
+    ("sweep_S64_W16_m8", [3, 40], "baseline", 1)])
+def test_full_size_round_on_sampled_sequences(name, sample, mode_name, rounds):
+    import copy
+
     from paper_2609_14717_b200 import binding as B
     wl, lay, w, ctx, cfg, st_g, cfg_o, st_o = _setup(name, 11, sample)
+    st_r = copy.deepcopy(st_o)                                 # state of the storage-rounded diagnostic run
     sh = wl.shape
     w_o = orc.prepare_weights(w)
+    mode_g, mode_o = (B.COD_CARRY, orc.MODE_CARRY) if mode_name == "carry" else (B.COD_BASELINE, orc.MODE_BASELINE)
     split, taps = B.Split(wl.S, sh.W), B.Taps(cfg, wl.S)
     nd = torch.zeros((wl.S, sh.W), dtype=torch.int32, device="cuda")
     rows = np.concatenate([np.arange(s * sh.W, (s + 1) * sh.W) for s in sample])
-    exempt = 0
-    for r in range(2):
+    exempt = compared = 0
+    width = sh.n_q * sh.hd
+    for r in range(rounds):
         rd = synth.make_round(wl, 11, r)
         ctx.draft_round(torch.from_numpy(rd["draft"]).cuda(), torch.from_numpy(rd["target"]).cuda(),
-                        B.to_device(rd["H"], sh.dtype), wl.S, wl.n_forced, B.COD_CARRY, st_g, split, nd, taps)
+                        B.to_device(rd["H"], sh.dtype), wl.S, wl.n_forced, mode_g, st_g, split, nd, taps)
         torch.cuda.synchronize()
         L0 = st_o.committed_len.copy()
-        res = orc.draft_round(rd["draft"][sample], rd["target"][sample], rd["H"][rows], st_o, w_o, wl.n_forced, orc.MODE_CARRY)
+        args = (rd["draft"][sample], rd["target"][sample], rd["H"][rows])
+        res = orc.draft_round(*args, st_o, w_o, wl.n_forced, mode_o, keep_logits=True)
+        res_r = orc.draft_round(*args, st_r, w_o, wl.n_forced, mode_o, round_store=_bf16_store)
         got = split.to_host()
         # integers: exact (slot numbers differ because the oracle uses a compact page table)
         assert np.array_equal(got["accept_len"], rd["m"])
@@ -89,16 +123,39 @@ def test_full_size_round_on_sampled_sequences(name, sample):
                 c = int(st_o.carry_len[j])
                 if c:
                     ref.append(st_o.carry[l, j, :, :, :c, :].reshape(-1, sh.hd)); gpu.append(carry_g[l, s, :, :, :c, :].float().cpu().numpy().reshape(-1, sh.hd))
-                assert rel_err(np.concatenate([a.reshape(-1) for a in gpu]), np.concatenate([a.reshape(-1) for a in ref])) <= TOL
+                gpu = np.concatenate([a.reshape(-1) for a in gpu]); ref = np.concatenate([a.reshape(-1) for a in ref])
+                assert rel_err(gpu, ref) <= TOL
+                assert _row_err(gpu, ref, sh.hd) <= TOL, ("K/V per (row, head)", _row_err(gpu, ref, sh.hd))
+        e_exact, e_round, e_store = [], [], []
         for l in range(sh.n_layers):
-            assert rel_err(taps.attn_out[l].cpu().numpy()[rows], res["attn_out"][l]) <= (TOL if l == 0 else TOL_COMPOUNDED)
-        assert rel_err(taps.x_final.cpu().numpy()[rows], res["x_final"]) <= TOL_COMPOUNDED
+            g_l = taps.attn_out[l].cpu().numpy()[rows]
+            e_exact.append(rel_err(g_l, res["attn_out"][l])); e_round.append(rel_err(g_l, res_r["attn_out"][l]))
+            e_store.append(rel_err(res_r["attn_out"][l], res["attn_out"][l]))
+        xg = taps.x_final.cpu().numpy()[rows]
+        e_exact.append(rel_err(xg, res["x_final"])); e_round.append(rel_err(xg, res_r["x_final"]))
+        e_store.append(rel_err(res_r["x_final"], res["x_final"]))
+        fmt = lambda v: " ".join(f"{e:.2e}" for e in v)
+        print(f"\n{name} {mode_name} round {r}: attn_out[0..{sh.n_layers - 1}], x_final"
+              f"\n   library vs exact oracle            {fmt(e_exact)}"
+              f"\n   library vs storage-rounded oracle  {fmt(e_round)}"
+              f"\n   storage-rounded vs exact oracle    {fmt(e_store)}"
+              f"\n   per (row, head), layer 0, vs exact {_row_err(taps.attn_out[0].cpu().numpy()[rows], res['attn_out'][0], sh.hd):.2e}")
+        assert e_exact[0] <= TOL
+        for l, (eg, es) in enumerate(zip(e_exact, e_store)):
+            assert eg <= min(TOL_COMPOUNDED, max(TOL, 2.0 * es)), (l, eg, es)
+        # tokens: equal wherever the exact oracle's top-2 gap is at least GAP; the rest is counted, not waved through
         sure = res["gap"] >= GAP
-        sure[:, 0] = False
+        sure[:, 0] = False                                     # row 0 of next_draft is the bonus token
         assert np.array_equal(nd.cpu().numpy()[sample][sure], res["next_draft"][sure])
-        exempt += int((~sure[:, 1:]).sum())
+        exempt += int((~sure[:, 1:]).sum()); compared += int(sure[:, 1:].sum())
+        top_err = float(np.abs(taps.top_logit.cpu().numpy()[rows] - res["logits"].max(axis=1)).max())
+        print(f"   tokens compared {int(sure[:, 1:].sum())}, exempt (oracle gap < {GAP}) {int((~sure[:, 1:]).sum())}, "
+              f"max |top logit - oracle max logit| {top_err:.2e}")
+        assert top_err <= TOL * max(1.0, float(np.abs(res["logits"]).max()))
     assert ctx.poll_status() == 0
-    assert exempt <= len(sample) * sh.W          # only a handful of near-ties may be exempt
+    # exempt is by construction the number of near-ties in the oracle's own gap histogram; if a quarter of
+    # the positions were near-ties the token check would say too little
+    assert exempt < 0.25 * (exempt + compared), (exempt, compared)
     ctx.close()
 
 

@@ -9,8 +9,9 @@ import numpy as np
 import pytest
 import torch
 
+from oracle import cod_oracle as orc
 from paper_2609_14717_b200 import synth
-from tests.helpers import small_bf16
+from tests.helpers import oracle_config, small_bf16
 
 pytestmark = pytest.mark.gpu
 
@@ -26,6 +27,8 @@ def test_static_scratch_argmax_matches_the_context_path_twice_in_a_row(dtype):
     w_dev = B.weights_to_device(w, sh.dtype)
     ctx.set_weights(w_dev)
     gen = torch.Generator(device="cuda").manual_seed(5)
+    w_o = {"g_final": np.asarray(w["g_final"], dtype=np.float64), "emb": np.asarray(w["emb"], dtype=np.float64)}
+    tol = 2e-2 if dtype == "bf16" else 1e-3
     for n_rows in (48, 7):                                     # two calls in a row, the second smaller
         x = torch.randn(n_rows, sh.d_model, generator=gen, device="cuda")
         tok_ref = torch.zeros(n_rows, dtype=torch.int32, device="cuda")
@@ -41,6 +44,12 @@ def test_static_scratch_argmax_matches_the_context_path_twice_in_a_row(dtype):
         ref = top_ref[:ctx_rows].cpu().numpy()
         assert np.max(np.abs(top[:ctx_rows].cpu().numpy() - ref)) <= (2e-2 if dtype == "bf16" else 1e-3) * np.max(np.abs(ref))
         assert (tok >= 0).all() and (tok < sh.vocab).all()
+        # and against the CPU oracle's LM head on all rows: tokens where its top-2 gap is clear, top logit to tolerance
+        t_o, gap, logits = orc.lm_head_argmax(x.cpu().numpy().astype(np.float64), w_o, oracle_config(sh))
+        sure = gap >= 1e-2
+        assert sure.sum() >= n_rows // 2
+        assert np.array_equal(tok.cpu().numpy()[sure], t_o[sure])
+        assert np.max(np.abs(top.cpu().numpy() - logits.max(axis=1))) <= tol * np.max(np.abs(logits))
     # beyond the fixed capacity: refused, nothing launched
     big = torch.zeros(65, sh.d_model, device="cuda")
     with pytest.raises(B.CodError) as e:
@@ -48,3 +57,33 @@ def test_static_scratch_argmax_matches_the_context_path_twice_in_a_row(dtype):
                                 None, sh.rms_eps)
     assert e.value.status == -6
     ctx.close()
+
+
+def test_static_scratch_argmax_at_its_size_limits_against_the_oracle():
+    """Exactly 64 rows x 8192 columns (the whole scratch in use, the wide-row kernels), twice in a row; one
+    column group beyond the limit is refused."""
+    from paper_2609_14717_b200 import binding as B
+    D, V, R = 8192, 1536, 64
+    rng = np.random.default_rng(31)
+    emb = synth.round_bf16(rng.standard_normal((V, D), dtype=np.float32) * np.float32(0.02))
+    g = synth.round_bf16(np.float32(1.0) + np.float32(0.1) * rng.standard_normal(D, dtype=np.float32))
+    emb_d, g_d = B.to_device(emb, "bf16"), B.to_device(g, "bf16")
+    sh = synth.scaled(synth.workload("cfg3"), d_model=D, vocab=V).shape
+    w_o = {"g_final": g.astype(np.float64), "emb": emb.astype(np.float64)}
+    for rep in range(2):
+        x = rng.standard_normal((R, D), dtype=np.float32)
+        tok = torch.full((R,), -1, dtype=torch.int32, device="cuda")
+        top = torch.zeros(R, dtype=torch.float32, device="cuda")
+        B.lm_head_argmax_static(emb_d, g_d, torch.from_numpy(x).cuda(), tok, top, sh.rms_eps)
+        torch.cuda.synchronize()
+        t_o, gap, logits = orc.lm_head_argmax(x.astype(np.float64), w_o, oracle_config(sh))
+        sure = gap >= 1e-2
+        assert sure.sum() >= R // 2
+        assert np.array_equal(tok.cpu().numpy()[sure], t_o[sure])
+        assert np.max(np.abs(top.cpu().numpy() - logits.max(axis=1))) <= 2e-2 * np.max(np.abs(logits))
+    wide = torch.zeros(R, D + 8, device="cuda")
+    with pytest.raises(B.CodError) as e:
+        B.lm_head_argmax_static(torch.zeros(V, D + 8, dtype=torch.bfloat16, device="cuda"),
+                                torch.ones(D + 8, dtype=torch.bfloat16, device="cuda"), wide,
+                                torch.zeros(R, dtype=torch.int32, device="cuda"), None, sh.rms_eps)
+    assert e.value.status == -6
