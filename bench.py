@@ -780,9 +780,9 @@ def run_sweep(args):
                 H = B.to_device(rd["H"], "bf16")
                 nd = torch.zeros((S, W), dtype=torch.int32, device="cuda")
                 L0 = state.committed_len.clone()
-                res = {}
+                graphs = {}
                 for mode, name in ((B.COD_CARRY, "carry"), (B.COD_BASELINE, "baseline")):
-                    def one():
+                    def one(mode=mode):
                         ctx.draft_round(d, t, H, S, nf, mode, state, None, nd, None)
                     state.committed_len.copy_(L0); state.carry_len.zero_()
                     side = torch.cuda.Stream(); side.wait_stream(torch.cuda.current_stream())
@@ -792,20 +792,30 @@ def run_sweep(args):
                     g = torch.cuda.CUDAGraph()
                     with torch.cuda.graph(g):
                         one()
-                    state.committed_len.copy_(L0); state.carry_len.zero_()
-                    for _ in range(Wm):
-                        g.replay()
-                    torch.cuda.synchronize()
-                    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-                    e0.record()
-                    for _ in range(K):
-                        g.replay()
-                    e1.record(); torch.cuda.synchronize()
-                    res[name] = e0.elapsed_time(e1) / K * 1e3
+                    graphs[name] = g
+                # interleaved passes (C B C B ...), each from the restored state; medians reported
+                times = {"carry": [], "baseline": []}
+                for rep in range(args.sweep_reps):
+                    for name in ("carry", "baseline"):
+                        state.committed_len.copy_(L0); state.carry_len.zero_()
+                        for _ in range(Wm):
+                            graphs[name].replay()
+                        torch.cuda.synchronize()
+                        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                        e0.record()
+                        for _ in range(K):
+                            graphs[name].replay()
+                        e1.record(); torch.cuda.synchronize()
+                        times[name].append(e0.elapsed_time(e1) / K * 1e3)
+                res = {k: statistics.median(v) for k, v in times.items()}
+                paired = [100.0 * (c_ - b_) / b_ for c_, b_ in zip(times["carry"], times["baseline"])]
                 status = ctx.poll_status()
                 rows.append({"S": S, "W": W, "m": m, "rejected": W - m, "n_forced": nf, "carry_us": res["carry"],
-                             "baseline_us": res["baseline"], "overhead_pct": 100.0 * (res["carry"] - res["baseline"]) / res["baseline"],
-                             "device_status": status})
+                             "baseline_us": res["baseline"], "overhead_pct": statistics.median(paired),
+                             "overhead_pct_min": min(paired), "overhead_pct_max": max(paired),
+                             "carry_us_min_max": [min(times["carry"]), max(times["carry"])],
+                             "baseline_us_min_max": [min(times["baseline"]), max(times["baseline"])],
+                             "passes": args.sweep_reps, "device_status": status})
                 ctx.close()
                 del state
                 torch.cuda.empty_cache()
@@ -825,6 +835,7 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-graph", action="store_true", help="time plain stream launches instead of graph replays")
     ap.add_argument("--sweep", action="store_true", help="carryover-overhead sweep over batch, block and rejected fraction")
+    ap.add_argument("--sweep-reps", type=int, default=7, help="--sweep: interleaved passes per mode and point")
     ap.add_argument("--attn-split", type=int, default=0, help="keys per attention split (0 = library default)")
     ap.add_argument("--micro", default=None, choices=["attn", "lmhead", "lmsample", "lmrank", "gemm"],
                     help="time one entry point alone (small footprint; meant for profiler captures)")

@@ -328,7 +328,12 @@ static int project_impl(cod_ctx* c, const void* H, const cod_split* sp, int S, i
                         const cod_state* dest, float* tap_z, cudaStream_t st) {
   const cod_config& f = c->cfg;
   const int R = S * f.block;
-  const int* a_rows = mode == COD_BASELINE ? sp->acc_rows : nullptr;
+  // The baseline drafter projects accepted rows only. Rounds of up to 128 rows run on the weight-streaming
+  // kernel, where extra token columns cost nothing: there the baseline contracts all R rows in place (no
+  // packing pass, the same launches as the carry round) and the finish kernels keep the accepted ones; with no
+  // accepted row at all both contractions still leave at once. Larger rounds pack the accepted rows first.
+  const bool dense_base = mode == COD_BASELINE && R <= 128 && c->cfg.dtype == COD_BF16 && !c->force_simt;
+  const int* a_rows = mode == COD_BASELINE && !dense_base ? sp->acc_rows : nullptr;
   const int* n_dev = mode == COD_BASELINE ? sp->acc_off + S : nullptr;
   int rc;
 
@@ -337,7 +342,7 @@ static int project_impl(cod_ctx* c, const void* H, const cod_split* sp, int S, i
     H = c->hc;
   }
   GemmArgs g{};
-  g.A = H; g.lda = c->D_in; g.a_rows = nullptr; g.n_rows_dev = n_dev; g.n_rows = R; g.K = c->D_in;
+  g.A = H; g.lda = c->D_in; g.a_rows = nullptr; g.n_rows_dev = n_dev; g.rows_gate = dense_base; g.n_rows = R; g.K = c->D_in;
   g.seg[0] = {c->w.fc, c->D, c->wt.fc}; g.n_seg = 1; g.klass = COD_K_FC;
   // separate-projector variant, carry mode: F h and F_rej h of every row from one two-segment contraction,
   // the finish kernel keeps the one the row's status selects (the baseline keeps accepted rows only: F alone)
@@ -345,17 +350,17 @@ static int project_impl(cod_ctx* c, const void* H, const cod_split* sp, int S, i
   if (two) { g.seg[1] = {c->w.fc_rej, c->D, c->wt.fc_rej}; g.n_seg = 2; }
   g.C = c->gemm_out; g.ldc = two ? 2 * c->D : c->D; g.splits = pick_splits(c, g.ldc, c->D_in, R);
   if ((rc = cod_launch_gemm(c, g, st)) != COD_OK) return rc;
-  if ((rc = cod_launch_fc_finish(c, c->gemm_out, g.splits, R, n_dev, a_rows, sp->carry_slot, tap_z, st, g.ldc)) != COD_OK)
+  if ((rc = cod_launch_fc_finish(c, c->gemm_out, g.splits, R, n_dev, a_rows, sp->carry_slot, tap_z, st, g.ldc, dense_base)) != COD_OK)
     return rc;
 
   GemmArgs k{};
-  k.A = c->z; k.lda = c->D; k.a_rows = nullptr; k.n_rows_dev = n_dev; k.n_rows = R; k.K = c->D;
+  k.A = c->z; k.lda = c->D; k.a_rows = nullptr; k.n_rows_dev = n_dev; k.rows_gate = dense_base; k.n_rows = R; k.K = c->D;
   k.seg[0] = {c->w.wk, f.n_layers * c->kvw, c->wt.wk};
   k.seg[1] = {c->w.wv, f.n_layers * c->kvw, c->wt.wv};
   k.n_seg = 2; k.klass = COD_K_KV;
   k.C = c->gemm_out; k.ldc = 2 * f.n_layers * c->kvw; k.splits = pick_splits(c, k.ldc, c->D, R);
   if ((rc = cod_launch_gemm(c, k, st)) != COD_OK) return rc;
-  return cod_launch_kv_finish(c, c->gemm_out, k.splits, R, n_dev, a_rows, sp, J, dest, R, st);
+  return cod_launch_kv_finish(c, c->gemm_out, k.splits, R, n_dev, a_rows, sp, J, dest, R, st, dense_base);
 }
 
 int cod_project_kv(cod_ctx* c, const void* H, const cod_split* split, int S, int mode, void* J,

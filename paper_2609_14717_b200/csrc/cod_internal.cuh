@@ -98,6 +98,7 @@ struct GemmArgs {
   int lda;
   const int* a_rows;      // optional gather list: row(i) = a_rows[i]; else row(i) = i
   const int* n_rows_dev;  // optional device count of valid rows (<= n_rows)
+  int rows_gate;          // n_rows_dev only gates the launch: all n_rows rows if it is positive, none if it is zero
   int n_rows;             // rows (or their upper bound when n_rows_dev is set)
   int K;
   GemmSeg seg[3];         // weight segments laid side by side along N
@@ -255,11 +256,11 @@ int cod_launch_fcE(cod_ctx* c, cudaStream_t st);
 int cod_launch_gather_rows(cod_ctx* c, const void* src, const int* rows, const int* n_dev, int n_max, int width,
                            void* dst, cudaStream_t st);
 int cod_launch_fc_finish(cod_ctx* c, const float* part, int splits, int n_rows, const int* n_rows_dev,
-                         const int* a_rows, const int* carry_slot, float* tap_z, cudaStream_t st, int ldp = 0);   // ldp: row stride of part (0 = D; 2 D = F h | F_rej h)
+                         const int* a_rows, const int* carry_slot, float* tap_z, cudaStream_t st, int ldp = 0, int dense_base = 0);   // ldp: row stride of part (0 = D; 2 D = F h | F_rej h)
 // dest_state == nullptr: write J; else write the pool / carry slot directly
 int cod_launch_kv_finish(cod_ctx* c, const float* part, int splits, int n_rows, const int* n_rows_dev,
                          const int* a_rows, const cod_split* sp, void* J, const cod_state* dest_state,
-                         int R_total, cudaStream_t st);
+                         int R_total, cudaStream_t st, int dense_base = 0);
 int cod_launch_scatter(cod_ctx* c, const void* J, const cod_split* sp, int S, int mode,
                        const cod_state* state, cudaStream_t st);
 int cod_launch_update_lens(cod_ctx* c, const cod_split* sp, int S, int mode, const cod_state* state,

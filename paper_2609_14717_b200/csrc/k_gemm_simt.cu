@@ -17,7 +17,7 @@ __global__ void __launch_bounds__(NT) k_gemm_simt(GemmArgs g) {
   __shared__ float As[BK][BM + 1];
   __shared__ float Bs[BK][BN + 1];
 
-  const int n_rows = g.n_rows_dev ? min(*g.n_rows_dev, g.n_rows) : g.n_rows;
+  const int n_rows = g.n_rows_dev ? (g.rows_gate ? (*g.n_rows_dev > 0 ? g.n_rows : 0) : min(*g.n_rows_dev, g.n_rows)) : g.n_rows;
   const int i0 = blockIdx.y * BM;
   if (i0 >= n_rows) return;
 

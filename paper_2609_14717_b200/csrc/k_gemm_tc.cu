@@ -31,6 +31,7 @@ struct TcParams {
   int kb_total, kb_per_split;
   int n_rows;                 // rows (upper bound when n_rows_dev is set)
   const int* n_rows_dev;
+  int rows_gate;              // n_rows_dev only gates: all rows if positive, none if zero
   int NT;                     // token rows per CTA = MMA N (multiple of 16, <= 256)
   int tmem_cols;              // power of two >= max(32, NT)
   int stages;
@@ -127,7 +128,7 @@ k_gemm_tc(const __grid_constant__ CUtensorMap map_w0, const __grid_constant__ CU
       else tma_load_2d(base + it * stage_bytes, map_w, (kb0 + it) * BK, f0, smem_u32(full_bar + it));
 
   cod_pdl_prologue();
-  const int n_rows = p.n_rows_dev ? min(*p.n_rows_dev, p.n_rows) : p.n_rows;
+  const int n_rows = p.n_rows_dev ? (p.rows_gate ? (*p.n_rows_dev > 0 ? p.n_rows : 0) : min(*p.n_rows_dev, p.n_rows)) : p.n_rows;
   const int n_kb = i0 < n_rows ? kb1 - kb0 : 0;   // 0: no token rows here, only the requested weights to absorb
 
   if (warp == 4) {
@@ -382,6 +383,7 @@ int cod_launch_gemm_tc(cod_ctx* c, const GemmArgs& g, cudaStream_t st) {
   if (splits != g.splits) return COD_ERR_INVALID_ARG;               // the caller sized the partial slabs
   p.n_rows = g.n_rows;
   p.n_rows_dev = g.n_rows_dev;
+  p.rows_gate = g.rows_gate;
   const int r16 = (g.n_rows + 15) / 16 * 16;
   p.NT = r16 < 256 ? r16 : 256;
   int cols = 32;

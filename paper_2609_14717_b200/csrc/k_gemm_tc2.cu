@@ -312,7 +312,7 @@ void cod_plan_gemm_tc2(int n_sm, int n_out, int K, int rows, int max_splits, int
 
 // Used for more than 128 token rows; every weight segment but the last must be whole 256-row pairs.
 bool cod_gemm_tc2_supported(const cod_ctx* c, const GemmArgs& g) {
-  if (c->cfg.dtype != COD_BF16 || g.a_rows != nullptr || g.n_rows <= 128) return false;
+  if (c->cfg.dtype != COD_BF16 || g.a_rows != nullptr || g.rows_gate || g.n_rows <= 128) return false;
   if (g.K % 8 || g.lda % 8) return false;
   if ((reinterpret_cast<uintptr_t>(g.A) & 15u) != 0) return false;
   for (int i = 0; i < g.n_seg; ++i) {

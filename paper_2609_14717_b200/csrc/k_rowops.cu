@@ -68,13 +68,16 @@ template <typename T, int NV>
 __global__ void __launch_bounds__(1024) k_fc_finish(const float* __restrict__ part, int splits, int n_rows, const int* n_rows_dev,
                             const int* __restrict__ a_rows, const int* __restrict__ carry_slot,
                             const float* __restrict__ fcE, const T* __restrict__ gain, int D, float eps,
-                            int do_norm, T* __restrict__ z, int z_compact, float* __restrict__ tap, int ldp) {
+                            int do_norm, T* __restrict__ z, int z_compact, float* __restrict__ tap, int ldp, int dense_base) {
   cod_pdl_prologue();
   __shared__ float red[33];
   const int i = blockIdx.x;
-  if (i >= valid_rows(n_rows_dev, n_rows)) return;
+  // dense_base: the baseline drafter on ALL window rows (the contraction ran on every row because extra token
+  // columns are free while it streams weights); only accepted rows exist for it, and none if none was accepted
+  if (i >= (dense_base ? (*n_rows_dev > 0 ? n_rows : 0) : valid_rows(n_rows_dev, n_rows))) return;
   const int row = a_rows ? a_rows[i] : i;
   const bool rej = carry_slot[row] >= 0;
+  if (dense_base && rej) return;
   const int nv = D >> 2;
   float4 v[NV];
   float ss = 0.f;
@@ -131,11 +134,12 @@ __global__ void k_kv_finish(const float* __restrict__ part, int splits, int n_ro
                             const int* __restrict__ commit_slot, const int* __restrict__ carry_slot,
                             T* __restrict__ pool, T* __restrict__ carry, int page, int n_pages, int W,
                             int max_batch, int to_state, const T* __restrict__ g_k, float eps, int cap,
-                            const int* __restrict__ carry_base) {
+                            const int* __restrict__ carry_base, int dense_base) {
   cod_pdl_prologue();
   const int i = blockIdx.x, l = blockIdx.y;
-  if (i >= valid_rows(n_rows_dev, n_rows)) return;
+  if (i >= (dense_base ? (*n_rows_dev > 0 ? n_rows : 0) : valid_rows(n_rows_dev, n_rows))) return;
   const int row = a_rows ? a_rows[i] : i;
+  if (dense_base && carry_slot[row] >= 0) return;   // the baseline drafter keeps no rejected row
   const int kvw = n_kv * hd, half = hd >> 1, ldc = 2 * Ld * kvw;
   const float* cs = rope_win + static_cast<size_t>(row) * hd;
 
@@ -547,7 +551,7 @@ int cod_launch_fcE(cod_ctx* c, cudaStream_t st) {
 }
 
 int cod_launch_fc_finish(cod_ctx* c, const float* part, int splits, int n_rows, const int* n_rows_dev,
-                         const int* a_rows, const int* carry_slot, float* tap_z, cudaStream_t st, int ldp) {
+                         const int* a_rows, const int* carry_slot, float* tap_z, cudaStream_t st, int ldp, int dense_base) {
   ProfScope prof(c, COD_K_ROWOPS, st);
   if (n_rows <= 0) return COD_OK;
   const int nt = row_threads(c->D);
@@ -557,12 +561,12 @@ int cod_launch_fc_finish(cod_ctx* c, const float* part, int splits, int n_rows, 
   if (ldp <= 0) ldp = c->D;
   if (row_narrow(c->D)) {
     DISPATCH_T(c,
-               (cod_launch_pdl(c, k_fc_finish<__nv_bfloat16, 1>, n_rows, nt, 0, st, part, splits, n_rows, n_rows_dev, a_rows, carry_slot, fcE, static_cast<const __nv_bfloat16*>(c->w.g_hidden), c->D, c->cfg.rms_eps, do_norm, static_cast<__nv_bfloat16*>(c->z), a_rows ? 1 : 0, tap_z, ldp)),
-               (cod_launch_pdl(c, k_fc_finish<float, 1>, n_rows, nt, 0, st, part, splits, n_rows, n_rows_dev, a_rows, carry_slot, fcE, static_cast<const float*>(c->w.g_hidden), c->D, c->cfg.rms_eps, do_norm, static_cast<float*>(c->z), a_rows ? 1 : 0, tap_z, ldp)));
+               (cod_launch_pdl(c, k_fc_finish<__nv_bfloat16, 1>, n_rows, nt, 0, st, part, splits, n_rows, n_rows_dev, a_rows, carry_slot, fcE, static_cast<const __nv_bfloat16*>(c->w.g_hidden), c->D, c->cfg.rms_eps, do_norm, static_cast<__nv_bfloat16*>(c->z), a_rows ? 1 : 0, tap_z, ldp, dense_base)),
+               (cod_launch_pdl(c, k_fc_finish<float, 1>, n_rows, nt, 0, st, part, splits, n_rows, n_rows_dev, a_rows, carry_slot, fcE, static_cast<const float*>(c->w.g_hidden), c->D, c->cfg.rms_eps, do_norm, static_cast<float*>(c->z), a_rows ? 1 : 0, tap_z, ldp, dense_base)));
   } else {
     DISPATCH_T(c,
-               (cod_launch_pdl(c, k_fc_finish<__nv_bfloat16, ROW_WIDE_NV>, n_rows, nt, 0, st, part, splits, n_rows, n_rows_dev, a_rows, carry_slot, fcE, static_cast<const __nv_bfloat16*>(c->w.g_hidden), c->D, c->cfg.rms_eps, do_norm, static_cast<__nv_bfloat16*>(c->z), a_rows ? 1 : 0, tap_z, ldp)),
-               (cod_launch_pdl(c, k_fc_finish<float, ROW_WIDE_NV>, n_rows, nt, 0, st, part, splits, n_rows, n_rows_dev, a_rows, carry_slot, fcE, static_cast<const float*>(c->w.g_hidden), c->D, c->cfg.rms_eps, do_norm, static_cast<float*>(c->z), a_rows ? 1 : 0, tap_z, ldp)));
+               (cod_launch_pdl(c, k_fc_finish<__nv_bfloat16, ROW_WIDE_NV>, n_rows, nt, 0, st, part, splits, n_rows, n_rows_dev, a_rows, carry_slot, fcE, static_cast<const __nv_bfloat16*>(c->w.g_hidden), c->D, c->cfg.rms_eps, do_norm, static_cast<__nv_bfloat16*>(c->z), a_rows ? 1 : 0, tap_z, ldp, dense_base)),
+               (cod_launch_pdl(c, k_fc_finish<float, ROW_WIDE_NV>, n_rows, nt, 0, st, part, splits, n_rows, n_rows_dev, a_rows, carry_slot, fcE, static_cast<const float*>(c->w.g_hidden), c->D, c->cfg.rms_eps, do_norm, static_cast<float*>(c->z), a_rows ? 1 : 0, tap_z, ldp, dense_base)));
   }
   COD_CHECK_LAUNCH(c);
   return COD_OK;
@@ -570,15 +574,15 @@ int cod_launch_fc_finish(cod_ctx* c, const float* part, int splits, int n_rows, 
 
 int cod_launch_kv_finish(cod_ctx* c, const float* part, int splits, int n_rows, const int* n_rows_dev,
                          const int* a_rows, const cod_split* sp, void* J, const cod_state* ds, int R_total,
-                         cudaStream_t st) {
+                         cudaStream_t st, int dense_base) {
   ProfScope prof(c, COD_K_ROWOPS, st);
   if (n_rows <= 0) return COD_OK;
   const cod_config& f = c->cfg;
   dim3 grid(n_rows, f.n_layers);
   const int to_state = ds ? 1 : 0;
   DISPATCH_T(c,
-             (cod_launch_pdl(c, k_kv_finish<__nv_bfloat16>, grid, 128, 0, st, part, splits, n_rows, n_rows_dev, a_rows, c->rope_win, f.n_layers, f.n_kv_heads, f.head_dim, static_cast<__nv_bfloat16*>(J), R_total, sp->commit_slot, sp->carry_slot, ds ? static_cast<__nv_bfloat16*>(ds->kv_pool) : nullptr, ds ? static_cast<__nv_bfloat16*>(ds->carry_kv) : nullptr, f.page_size, f.n_pages, f.block, f.max_batch, to_state, (f.flags & COD_F_QK_NORM) ? static_cast<const __nv_bfloat16*>(c->w.g_knorm) : nullptr, f.rms_eps, c->carry_cap, c->carry_base)),
-             (cod_launch_pdl(c, k_kv_finish<float>, grid, 128, 0, st, part, splits, n_rows, n_rows_dev, a_rows, c->rope_win, f.n_layers, f.n_kv_heads, f.head_dim, static_cast<float*>(J), R_total, sp->commit_slot, sp->carry_slot, ds ? static_cast<float*>(ds->kv_pool) : nullptr, ds ? static_cast<float*>(ds->carry_kv) : nullptr, f.page_size, f.n_pages, f.block, f.max_batch, to_state, (f.flags & COD_F_QK_NORM) ? static_cast<const float*>(c->w.g_knorm) : nullptr, f.rms_eps, c->carry_cap, c->carry_base)));
+             (cod_launch_pdl(c, k_kv_finish<__nv_bfloat16>, grid, 128, 0, st, part, splits, n_rows, n_rows_dev, a_rows, c->rope_win, f.n_layers, f.n_kv_heads, f.head_dim, static_cast<__nv_bfloat16*>(J), R_total, sp->commit_slot, sp->carry_slot, ds ? static_cast<__nv_bfloat16*>(ds->kv_pool) : nullptr, ds ? static_cast<__nv_bfloat16*>(ds->carry_kv) : nullptr, f.page_size, f.n_pages, f.block, f.max_batch, to_state, (f.flags & COD_F_QK_NORM) ? static_cast<const __nv_bfloat16*>(c->w.g_knorm) : nullptr, f.rms_eps, c->carry_cap, c->carry_base, dense_base)),
+             (cod_launch_pdl(c, k_kv_finish<float>, grid, 128, 0, st, part, splits, n_rows, n_rows_dev, a_rows, c->rope_win, f.n_layers, f.n_kv_heads, f.head_dim, static_cast<float*>(J), R_total, sp->commit_slot, sp->carry_slot, ds ? static_cast<float*>(ds->kv_pool) : nullptr, ds ? static_cast<float*>(ds->carry_kv) : nullptr, f.page_size, f.n_pages, f.block, f.max_batch, to_state, (f.flags & COD_F_QK_NORM) ? static_cast<const float*>(c->w.g_knorm) : nullptr, f.rms_eps, c->carry_cap, c->carry_base, dense_base)));
   COD_CHECK_LAUNCH(c);
   return COD_OK;
 }
