@@ -828,7 +828,7 @@ def main():
     ap.add_argument("--steps", type=int, default=64)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--workload", default=None, choices=["cfg1", "cfg2", "cfg3", "cfg4", "cfg5", "cfg2f", "cfg3f"],
+    ap.add_argument("--workload", default=None, choices=["cfg1", "cfg2", "cfg3", "cfg4", "cfg5", "cfg2f", "cfg3f", "cfg3p"],
                     help="default: cfg3 (batch 32) on the line and cfg2 (batch 1) under \"batch1\"; cfg2f / cfg3f: the "
                          "same with the complete drafter layer (gated MLP 9728, q/k norms)")
     ap.add_argument("--seed", type=int, default=0)

@@ -47,6 +47,7 @@ size_t carve(cod_ctx* c) {
   c->side_rows = static_cast<int>(R < 128 ? R : 128);
   cv.take(c->gemm_out2, sizeof(float) * COD_MAX_SPLITS * c->side_rows * (c->qw + 2 * c->kvw));
   cv.take(c->hc, es * R * c->D_in);
+  cv.take(c->perm, sizeof(int) * R);
   cv.take(c->z, es * R * D);
   cv.take(c->x, sizeof(float) * R * D);
   cv.take(c->a, es * R * D);
@@ -349,8 +350,22 @@ static int project_impl(cod_ctx* c, const void* H, const cod_split* sp, int S, i
   const bool two = (f.flags & COD_F_REJ_PROJECTOR) && mode == COD_CARRY;
   if (two) { g.seg[1] = {c->w.fc_rej, c->D, c->wt.fc_rej}; g.n_seg = 2; }
   g.C = c->gemm_out; g.ldc = two ? 2 * c->D : c->D; g.splits = pick_splits(c, g.ldc, c->D_in, R);
+  // More than 128 rows (tensor-bound): the contraction is grouped by row instead - the window is packed
+  // accepted-first, rows [0, n_acc) meet F and rows [n_acc, R) meet F_rej in one launch, every row contracted
+  // once. Up to 128 rows both matrices are streamed whole whatever the rows, and routing would save nothing.
+  bool grouped = false;
+  if (two && R > 128) {
+    GemmArgs t = g;
+    t.A = c->hc; t.ldc = c->D; t.group_split_dev = sp->acc_off + S;
+    if (!c->force_simt && cod_gemm_tc2_supported(c, t)) {
+      if ((rc = cod_launch_gather_grouped(c, H, sp, S, R, c->D_in, c->hc, c->perm, st)) != COD_OK) return rc;
+      g = t;
+      grouped = true;
+    }
+  }
   if ((rc = cod_launch_gemm(c, g, st)) != COD_OK) return rc;
-  if ((rc = cod_launch_fc_finish(c, c->gemm_out, g.splits, R, n_dev, a_rows, sp->carry_slot, tap_z, st, g.ldc, dense_base)) != COD_OK)
+  if ((rc = cod_launch_fc_finish(c, c->gemm_out, g.splits, R, n_dev, grouped ? c->perm : a_rows, sp->carry_slot, tap_z, st,
+                                 g.ldc, dense_base, grouped ? 1 : 0)) != COD_OK)
     return rc;
 
   GemmArgs k{};

@@ -99,6 +99,8 @@ struct GemmArgs {
   const int* a_rows;      // optional gather list: row(i) = a_rows[i]; else row(i) = i
   const int* n_rows_dev;  // optional device count of valid rows (<= n_rows)
   int rows_gate;          // n_rows_dev only gates the launch: all n_rows rows if it is positive, none if it is zero
+  const int* group_split_dev;  // paired kernel, two segments: rows [0, *g) meet segment 0, rows [*g, n_rows) segment 1, both
+                          // write the SAME columns [0, seg[0].N) (a contraction grouped by row); null: segments side by side
   int n_rows;             // rows (or their upper bound when n_rows_dev is set)
   int K;
   GemmSeg seg[3];         // weight segments laid side by side along N
@@ -163,6 +165,7 @@ struct cod_ctx {
   cudaEvent_t ev_fork, ev_join;
   size_t gemm_out_floats;
   void* hc;                    // [R_max, D_in] accepted rows of H packed densely (baseline mode)
+  int* perm;                  // [R] window rows in the order accepted-first (grouped contraction of the separate projector)
   void* z;                     // [R_max, D]
   float* x;                    // [R_max, D]   residual stream
   void* a;                     // [R_max, D]   normalised activations
@@ -255,8 +258,11 @@ int cod_launch_rope_blk_only(cod_ctx* c, const int32_t* committed_len, int S, cu
 int cod_launch_fcE(cod_ctx* c, cudaStream_t st);
 int cod_launch_gather_rows(cod_ctx* c, const void* src, const int* rows, const int* n_dev, int n_max, int width,
                            void* dst, cudaStream_t st);
+// dst = src rows in the order acc_rows[0 .. *n_acc) then rej_rows[0 .. R - *n_acc); perm receives that order
+int cod_launch_gather_grouped(cod_ctx* c, const void* src, const cod_split* sp, int S, int R, int width, void* dst, int* perm,
+                              cudaStream_t st);
 int cod_launch_fc_finish(cod_ctx* c, const float* part, int splits, int n_rows, const int* n_rows_dev,
-                         const int* a_rows, const int* carry_slot, float* tap_z, cudaStream_t st, int ldp = 0, int dense_base = 0);   // ldp: row stride of part (0 = D; 2 D = F h | F_rej h)
+                         const int* a_rows, const int* carry_slot, float* tap_z, cudaStream_t st, int ldp = 0, int dense_base = 0, int z_by_row = 0);   // ldp: row stride of part (0 = D; 2 D = F h | F_rej h)
 // dest_state == nullptr: write J; else write the pool / carry slot directly
 int cod_launch_kv_finish(cod_ctx* c, const float* part, int splits, int n_rows, const int* n_rows_dev,
                          const int* a_rows, const cod_split* sp, void* J, const cod_state* dest_state,

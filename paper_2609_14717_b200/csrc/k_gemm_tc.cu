@@ -363,7 +363,7 @@ k_gemm_tc(const __grid_constant__ CUtensorMap map_w0, const __grid_constant__ CU
 }  // namespace
 
 bool cod_gemm_tc_supported(const cod_ctx* c, const GemmArgs& g) {
-  if (c->cfg.dtype != COD_BF16 || g.a_rows != nullptr) return false;
+  if (c->cfg.dtype != COD_BF16 || g.a_rows != nullptr || g.group_split_dev != nullptr) return false;
   if (g.K % 8 || g.lda % 8 || g.n_rows < 1) return false;
   if ((reinterpret_cast<uintptr_t>(g.A) & 15u) != 0) return false;
   for (int i = 0; i < g.n_seg; ++i) {

@@ -37,6 +37,7 @@ struct Tc2Params {
   int K, kb_total, kb_per_split;
   int n_rows;
   const int* n_rows_dev;
+  const int* group_split_dev; // two segments grouped by row: segment 0 owns rows [0, *g), segment 1 rows [*g, n_rows); same columns
   int pair_end[3];            // cumulative count of 256-row tile pairs after each weight segment
   int seg_N[3];
   int n_seg;
@@ -112,8 +113,14 @@ k_gemm_tc2(const __grid_constant__ CUtensorMap map_w0, const __grid_constant__ C
 
   cod_pdl_prologue();
   const int n_rows = p.n_rows_dev ? min(*p.n_rows_dev, p.n_rows) : p.n_rows;
+  int row_lo = 0, row_hi = n_rows;                // token rows this tile's weight segment is meant for
+  if (p.group_split_dev != nullptr) {
+    const int g = max(0, min(*p.group_split_dev, n_rows));
+    if (sidx == 0) row_hi = g; else row_lo = g;
+    col0 = f0;                                    // both groups' results share the columns
+  }
   // NOTE: both CTAs of a pair take the same decision here (it depends on the pair's tile only)
-  const int n_kb = i0 < n_rows ? kb1 - kb0 : 0;   // 0: no token rows here, only the requested weights to absorb
+  const int n_kb = (i0 < row_hi && i0 + NTOK > row_lo) ? kb1 - kb0 : 0;   // 0: no token rows here, only the requested weights to absorb
 
   if (warp == 4) {
     if (lane == 0) {
@@ -180,7 +187,8 @@ k_gemm_tc2(const __grid_constant__ CUtensorMap map_w0, const __grid_constant__ C
       float* C = p.C + static_cast<size_t>(split) * p.n_rows * p.ldc + col0;
       float* stage = reinterpret_cast<float*>(sm) + grp * (2 * 32 * BM);
       const int f_left = seg_N - f0;                       // features of this CTA that exist
-      for (int c = c_begin, q = 0; c < c_end && i0 + c < n_rows; c += 32, q ^= 1) {
+      for (int c = c_begin, q = 0; c < c_end && i0 + c < row_hi; c += 32, q ^= 1) {
+        if (i0 + c + 32 <= row_lo) continue;               // (the whole group of four warps skips together)
         uint32_t v[32];
         tmem_ld32(t_lane + c, v);
         float* buf = stage + q * (32 * BM);
@@ -190,7 +198,7 @@ k_gemm_tc2(const __grid_constant__ CUtensorMap map_w0, const __grid_constant__ C
 #pragma unroll
         for (int t = 0; t < 8; ++t) {
           const int tok = qw * 8 + t, i = i0 + c + tok;
-          if (i < n_rows && lane * 4 < f_left)
+          if (i >= row_lo && i < row_hi && lane * 4 < f_left)
             *reinterpret_cast<float4*>(C + static_cast<size_t>(i) * p.ldc + lane * 4) =
                 *reinterpret_cast<const float4*>(buf + tok * BM + lane * 4);
         }
@@ -198,13 +206,14 @@ k_gemm_tc2(const __grid_constant__ CUtensorMap map_w0, const __grid_constant__ C
     } else if (ok && p.amax == nullptr) {
       float* C = p.C + static_cast<size_t>(split) * p.n_rows * p.ldc;
       for (int c = c_begin; c < c_end; c += 16) {
-        if (i0 + c >= n_rows) break;
+        if (i0 + c >= row_hi) break;
+        if (i0 + c + 16 <= row_lo) continue;
         uint32_t v[16];
         tmem_ld16(t_lane + c, v);
 #pragma unroll
         for (int j = 0; j < 16; ++j) {
           const int i = i0 + c + j;
-          if (f_ok && i < n_rows) C[static_cast<size_t>(i) * p.ldc + col0 + qw * 32 + lane] = __uint_as_float(v[j]);
+          if (f_ok && i >= row_lo && i < row_hi) C[static_cast<size_t>(i) * p.ldc + col0 + qw * 32 + lane] = __uint_as_float(v[j]);
         }
       }
     } else if (SAMPLE && ok) {
@@ -332,6 +341,8 @@ int cod_launch_gemm_tc2(cod_ctx* c, const GemmArgs& g, cudaStream_t st) {
   if (splits != g.splits) return COD_ERR_INVALID_ARG;
   p.n_rows = g.n_rows;
   p.n_rows_dev = g.n_rows_dev;
+  p.group_split_dev = g.group_split_dev;
+  if (g.group_split_dev && (g.n_seg != 2 || g.amax != nullptr || g.seg[0].N != g.seg[1].N)) return COD_ERR_INVALID_ARG;
   int pairs = 0;
   for (int i = 0; i < 3; ++i) {
     if (i < g.n_seg) {

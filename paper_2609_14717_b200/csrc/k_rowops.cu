@@ -62,6 +62,21 @@ __global__ void k_gather_rows(const T* __restrict__ src, const int* __restrict__
   for (int e = threadIdx.x; e < width / VEC; e += blockDim.x) d4[e] = s4[e];
 }
 
+// dst[i] = src[perm[i]] with perm = the accepted rows (in order), then the rejected rows (in order): the window
+// grouped by row status, so that a contraction can meet each group with its own weights.
+template <typename T>
+__global__ void k_gather_grouped(const T* __restrict__ src, const int* __restrict__ acc_rows, const int* __restrict__ n_acc_dev,
+                                 const int* __restrict__ rej_rows, int width, T* __restrict__ dst, int* __restrict__ perm) {
+  cod_pdl_prologue();
+  const int i = blockIdx.x, n_acc = *n_acc_dev;
+  const int row = i < n_acc ? acc_rows[i] : rej_rows[i - n_acc];
+  if (threadIdx.x == 0) perm[i] = row;
+  constexpr int VEC = 16 / sizeof(T);
+  const uint4* s4 = reinterpret_cast<const uint4*>(src + static_cast<size_t>(row) * width);
+  uint4* d4 = reinterpret_cast<uint4*>(dst + static_cast<size_t>(i) * width);
+  for (int e = threadIdx.x; e < width / VEC; e += blockDim.x) d4[e] = s4[e];
+}
+
 // ------------------------------------------------------------------ fc finish
 // z[row] = N_h( sum_splits part[i] + [row rejected] F(E_carry) )   (one block per kept row)
 template <typename T, int NV>
@@ -541,6 +556,17 @@ int cod_launch_gather_rows(cod_ctx* c, const void* src, const int* rows, const i
   return COD_OK;
 }
 
+int cod_launch_gather_grouped(cod_ctx* c, const void* src, const cod_split* sp, int S, int R, int width, void* dst, int* perm,
+                              cudaStream_t st) {
+  ProfScope prof(c, COD_K_ROWOPS, st);
+  if (R <= 0) return COD_OK;
+  DISPATCH_T(c,
+             (cod_launch_pdl(c, k_gather_grouped<__nv_bfloat16>, R, 256, 0, st, static_cast<const __nv_bfloat16*>(src), sp->acc_rows, sp->acc_off + S, sp->rej_rows, width, static_cast<__nv_bfloat16*>(dst), perm)),
+             (cod_launch_pdl(c, k_gather_grouped<float>, R, 256, 0, st, static_cast<const float*>(src), sp->acc_rows, sp->acc_off + S, sp->rej_rows, width, static_cast<float*>(dst), perm)));
+  COD_CHECK_LAUNCH(c);
+  return COD_OK;
+}
+
 int cod_launch_fcE(cod_ctx* c, cudaStream_t st) {
   ProfScope prof(c, COD_K_ROWOPS, st);
   DISPATCH_T(c,
@@ -551,7 +577,8 @@ int cod_launch_fcE(cod_ctx* c, cudaStream_t st) {
 }
 
 int cod_launch_fc_finish(cod_ctx* c, const float* part, int splits, int n_rows, const int* n_rows_dev,
-                         const int* a_rows, const int* carry_slot, float* tap_z, cudaStream_t st, int ldp, int dense_base) {
+                         const int* a_rows, const int* carry_slot, float* tap_z, cudaStream_t st, int ldp, int dense_base,
+                         int z_by_row) {
   ProfScope prof(c, COD_K_ROWOPS, st);
   if (n_rows <= 0) return COD_OK;
   const int nt = row_threads(c->D);
@@ -561,12 +588,12 @@ int cod_launch_fc_finish(cod_ctx* c, const float* part, int splits, int n_rows, 
   if (ldp <= 0) ldp = c->D;
   if (row_narrow(c->D)) {
     DISPATCH_T(c,
-               (cod_launch_pdl(c, k_fc_finish<__nv_bfloat16, 1>, n_rows, nt, 0, st, part, splits, n_rows, n_rows_dev, a_rows, carry_slot, fcE, static_cast<const __nv_bfloat16*>(c->w.g_hidden), c->D, c->cfg.rms_eps, do_norm, static_cast<__nv_bfloat16*>(c->z), a_rows ? 1 : 0, tap_z, ldp, dense_base)),
-               (cod_launch_pdl(c, k_fc_finish<float, 1>, n_rows, nt, 0, st, part, splits, n_rows, n_rows_dev, a_rows, carry_slot, fcE, static_cast<const float*>(c->w.g_hidden), c->D, c->cfg.rms_eps, do_norm, static_cast<float*>(c->z), a_rows ? 1 : 0, tap_z, ldp, dense_base)));
+               (cod_launch_pdl(c, k_fc_finish<__nv_bfloat16, 1>, n_rows, nt, 0, st, part, splits, n_rows, n_rows_dev, a_rows, carry_slot, fcE, static_cast<const __nv_bfloat16*>(c->w.g_hidden), c->D, c->cfg.rms_eps, do_norm, static_cast<__nv_bfloat16*>(c->z), (a_rows && !z_by_row) ? 1 : 0, tap_z, ldp, dense_base)),
+               (cod_launch_pdl(c, k_fc_finish<float, 1>, n_rows, nt, 0, st, part, splits, n_rows, n_rows_dev, a_rows, carry_slot, fcE, static_cast<const float*>(c->w.g_hidden), c->D, c->cfg.rms_eps, do_norm, static_cast<float*>(c->z), (a_rows && !z_by_row) ? 1 : 0, tap_z, ldp, dense_base)));
   } else {
     DISPATCH_T(c,
-               (cod_launch_pdl(c, k_fc_finish<__nv_bfloat16, ROW_WIDE_NV>, n_rows, nt, 0, st, part, splits, n_rows, n_rows_dev, a_rows, carry_slot, fcE, static_cast<const __nv_bfloat16*>(c->w.g_hidden), c->D, c->cfg.rms_eps, do_norm, static_cast<__nv_bfloat16*>(c->z), a_rows ? 1 : 0, tap_z, ldp, dense_base)),
-               (cod_launch_pdl(c, k_fc_finish<float, ROW_WIDE_NV>, n_rows, nt, 0, st, part, splits, n_rows, n_rows_dev, a_rows, carry_slot, fcE, static_cast<const float*>(c->w.g_hidden), c->D, c->cfg.rms_eps, do_norm, static_cast<float*>(c->z), a_rows ? 1 : 0, tap_z, ldp, dense_base)));
+               (cod_launch_pdl(c, k_fc_finish<__nv_bfloat16, ROW_WIDE_NV>, n_rows, nt, 0, st, part, splits, n_rows, n_rows_dev, a_rows, carry_slot, fcE, static_cast<const __nv_bfloat16*>(c->w.g_hidden), c->D, c->cfg.rms_eps, do_norm, static_cast<__nv_bfloat16*>(c->z), (a_rows && !z_by_row) ? 1 : 0, tap_z, ldp, dense_base)),
+               (cod_launch_pdl(c, k_fc_finish<float, ROW_WIDE_NV>, n_rows, nt, 0, st, part, splits, n_rows, n_rows_dev, a_rows, carry_slot, fcE, static_cast<const float*>(c->w.g_hidden), c->D, c->cfg.rms_eps, do_norm, static_cast<float*>(c->z), (a_rows && !z_by_row) ? 1 : 0, tap_z, ldp, dense_base)));
   }
   COD_CHECK_LAUNCH(c);
   return COD_OK;

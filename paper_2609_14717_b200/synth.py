@@ -113,6 +113,10 @@ def workload(name: str) -> Workload:
         # the same batches with a complete drafter layer: gated MLP of width 9728 and q/k norms
         base = workload(name[:-1])
         return replace(base, name=name, shape=replace(base.shape, d_ff=9728, qk_norm=True))
+    if name == "cfg3p":
+        # batch 32 with the separate projector for rejected rows (Section 5, Table 4(b)) instead of the embedding
+        base = workload("cfg3")
+        return replace(base, name=name, shape=replace(base.shape, carry_variant="projector"))
     raise KeyError(name)
 
 

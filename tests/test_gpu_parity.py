@@ -109,6 +109,10 @@ def _workloads():
         "small_bf16_nomark": small_bf16(S=3, W=16, n_layers=1, ctx=(40, 300), carry_variant="none"),
         "small_bf16_proj": small_bf16(S=3, W=16, n_layers=2, ctx=(40, 300), carry_variant="projector"),
         "tiny_f32_proj": synth.scaled(synth.workload("cfg1"), S=3, ctx=(5, 140), n_rounds=6, carry_variant="projector"),
+        # ... and at more than 128 rows, where the projector variant becomes ONE contraction grouped by row status
+        # (accepted rows meet F, rejected rows F_rej; 544 rows = two token tiles with the group boundary inside one)
+        "mid_bf16_proj": small_bf16(S=34, W=16, n_layers=2, ctx=(100, 600), d_target=512, n_cap=5, d_model=1024,
+                                    n_q=8, n_kv=2, vocab=3000, carry_variant="projector"),
         # rejected rows retained for k > 1 rounds: the carry slot holds k * W rows, the oldest round leaves
         "small_bf16_keep2": small_bf16(S=3, W=16, n_layers=2, ctx=(40, 300), carry_rounds=2, n_rounds=6),
         "small_bf16_W32_keep2": small_bf16(S=2, W=32, n_layers=1, ctx=(100, 200), carry_rounds=2, n_rounds=6),
@@ -350,6 +354,7 @@ def test_round_parity_cfg1_every_round():
     ("mid_bf16_full", 30.0, orc.MODE_CARRY), ("order_bf16", 30.0, orc.MODE_CARRY),
     ("small_bf16_nomark", 30.0, orc.MODE_CARRY), ("small_bf16_proj", 30.0, orc.MODE_CARRY),
     ("small_bf16_proj", 30.0, orc.MODE_BASELINE), ("tiny_f32_proj", 40.0, orc.MODE_CARRY),
+    ("mid_bf16_proj", 30.0, orc.MODE_CARRY), ("mid_bf16_proj", 30.0, orc.MODE_BASELINE),
     ("small_bf16_keep2", 30.0, orc.MODE_CARRY), ("small_bf16_keep2", 30.0, orc.MODE_BASELINE),
     ("small_bf16_W32_keep2", 1.0, orc.MODE_CARRY), ("tiny_f32_keep3", 40.0, orc.MODE_CARRY)])
 def test_round_parity_multi_round(name, wo_scale, mode):
