@@ -332,6 +332,19 @@ enum cod_kernel_class {
   COD_K_CLASSES = 9
 };
 
+/* Failure detection (the paper has no counterpart). Every device-side wait of the tensor-core kernels
+   (an mbarrier poll in a copy / MMA pipeline) is bounded by the SM cycle counter; when the bound runs out
+   the CTA raises COD_DEV_TIMEOUT in the status word, lets what is in flight land, frees its tensor memory
+   and returns, so the context stays usable. cod_set_wait_limit sets that bound in SM cycles for the
+   context's later launches of the weight-streaming contraction (sm_cycles <= 0: the built-in bound, about
+   2 s). */
+int cod_set_wait_limit(cod_ctx* ctx, long long sm_cycles);
+/* Self-test of that path: while on != 0, the weight-streaming contraction kernel (rounds and calls of up to
+   128 rows) requests NO operand copies, so its consumers' waits run out after the wait limit and the calls
+   end with COD_DEV_TIMEOUT set and no result (tokens come back as -1). Nothing faults and nothing is left in
+   flight. Set a short wait limit first; switch it off again (and clear the status word) before real work. */
+int cod_selftest_expire_wait(cod_ctx* ctx, int on);
+
 /* Measurement aid (the paper has no counterpart): while class_mask has bit (1 << k) set,
    every launch of class k is bracketed by CUDA events on the launching stream (at most
    4096 launches are recorded between two calls). class_mask = 0 switches it off.

@@ -29,7 +29,8 @@ EXPORTS = ("cod_create", "cod_destroy", "cod_set_weights", "cod_verify_accept", 
            "cod_scatter_kv", "cod_block_attn", "cod_lm_head_argmax", "cod_lm_head_argmax_static",
            "cod_draft_round", "cod_reconvergence_count", "cod_verify_accept_stochastic",
            "cod_draft_round_stochastic", "cod_lm_head_sample", "cod_lm_head_rank",
-           "cod_poll_status", "cod_profile_enable", "cod_profile_read", "cod_launch_count",
+           "cod_poll_status", "cod_set_wait_limit", "cod_selftest_expire_wait",
+           "cod_profile_enable", "cod_profile_read", "cod_launch_count",
            "cod_workspace_bytes", "cod_error_string")
 KERNEL_CLASSES = ("verify", "fc", "kv", "qkv", "attn", "oproj", "lmhead", "rowops", "mlp")
 
@@ -299,6 +300,14 @@ class Context:
         flags = C.c_uint32(0)
         _check("cod_poll_status", lib().cod_poll_status(self._h, C.byref(flags), int(clear), _stream()))
         return int(flags.value)
+
+    def set_wait_limit(self, sm_cycles: int) -> None:
+        """Bound of the device-side waits of the weight-streaming contraction, in SM cycles (0: built-in)."""
+        _check("cod_set_wait_limit", lib().cod_set_wait_limit(self._h, C.c_longlong(sm_cycles)))
+
+    def selftest_expire_wait(self, on: bool) -> None:
+        """While on, that kernel requests no operands: its waits run out and raise COD_DEV_TIMEOUT."""
+        _check("cod_selftest_expire_wait", lib().cod_selftest_expire_wait(self._h, int(bool(on))))
 
     def profile_enable(self, classes=()) -> None:
         mask = 0

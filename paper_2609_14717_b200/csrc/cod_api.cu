@@ -635,6 +635,18 @@ int cod_poll_status(cod_ctx* c, uint32_t* dev_flags, int clear, cod_stream_t str
   return COD_OK;
 }
 
+int cod_set_wait_limit(cod_ctx* c, long long sm_cycles) {
+  if (!c) return COD_ERR_INVALID_ARG;
+  c->wait_limit = sm_cycles > 0 ? sm_cycles : 0;
+  return COD_OK;
+}
+
+int cod_selftest_expire_wait(cod_ctx* c, int on) {
+  if (!c) return COD_ERR_INVALID_ARG;
+  c->selftest_skip_copies = on ? 1 : 0;
+  return COD_OK;
+}
+
 int cod_profile_enable(cod_ctx* c, uint32_t class_mask) {
   if (!c) return COD_ERR_INVALID_ARG;
   c->prof_mask = class_mask & ((1u << COD_K_CLASSES) - 1u);

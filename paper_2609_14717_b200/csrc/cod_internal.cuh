@@ -165,6 +165,8 @@ struct cod_ctx {
   cudaEvent_t ev_fork, ev_join;
   size_t gemm_out_floats;
   void* hc;                    // [R_max, D_in] accepted rows of H packed densely (baseline mode)
+  long long wait_limit;        // SM cycles a bounded device wait may last (0: the built-in limit, about 2 s)
+  int selftest_skip_copies;    // cod_selftest_expire_wait: single-CTA contractions request no operands
   int* perm;                  // [R] window rows in the order accepted-first (grouped contraction of the separate projector)
   void* z;                     // [R_max, D]
   float* x;                    // [R_max, D]   residual stream

@@ -46,6 +46,8 @@ struct TcParams {
   float2* lse_part;           // sampling form of the argmax epilogue (null: plain argmax)
   uint32_t sample_state;
   uint32_t* status;
+  long long wait_limit;       // SM cycles a bounded wait may last
+  int skip_copies;            // self-test of the failure path: the producer requests nothing, so the waits run out
   // rank form (RANK kernels): per token row, how many weight rows score above a reference row
   const float* rank_ref;      // [n_rows] the reference row's logit
   const int32_t* rank_tok;    // [n_rows] the reference row's index (excluded from the count)
@@ -122,7 +124,7 @@ k_gemm_tc(const __grid_constant__ CUtensorMap map_w0, const __grid_constant__ CU
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
-  if (warp == 4 && lane == 0)
+  if (warp == 4 && lane == 0 && !p.skip_copies)
     for (int it = 0; it < n_pre; ++it)
       if (wt) bulk_load(base + it * stage_bytes, wt + static_cast<size_t>(kb0 + it) * A_TILE_BYTES, A_TILE_BYTES, smem_u32(full_bar + it));
       else tma_load_2d(base + it * stage_bytes, map_w, (kb0 + it) * BK, f0, smem_u32(full_bar + it));
@@ -133,16 +135,16 @@ k_gemm_tc(const __grid_constant__ CUtensorMap map_w0, const __grid_constant__ CU
 
   if (warp == 4) {
     // ------------------------------------------------ TMA producer
-    if (lane == 0) {
+    if (lane == 0 && !p.skip_copies) {
       if (n_kb == 0) {
         for (int it = 0; it < n_pre; ++it) {
           mbar_expect_tx(smem_u32(full_bar + it), A_TILE_BYTES);
-          if (!mbar_wait(smem_u32(full_bar + it), 0, abort_flag, p.status)) break;
+          if (!mbar_wait(smem_u32(full_bar + it), 0, abort_flag, p.status, p.wait_limit)) break;
         }
       }
       for (int it = 0; it < n_kb; ++it) {
         const int s = it % p.stages, use = it / p.stages;
-        if (use > 0 && !mbar_wait(smem_u32(empty_bar + s), (use - 1) & 1, abort_flag, p.status)) break;
+        if (use > 0 && !mbar_wait(smem_u32(empty_bar + s), (use - 1) & 1, abort_flag, p.status, p.wait_limit)) break;
         const uint32_t fb = smem_u32(full_bar + s);
         mbar_expect_tx(fb, stage_bytes);
         const uint32_t a_dst = base + s * stage_bytes;
@@ -161,7 +163,7 @@ k_gemm_tc(const __grid_constant__ CUtensorMap map_w0, const __grid_constant__ CU
       bool ok = true;
       for (int it = 0; it < n_kb && ok; ++it) {
         const int s = it % p.stages, use = it / p.stages;
-        ok = mbar_wait(smem_u32(full_bar + s), use & 1, abort_flag, p.status);
+        ok = mbar_wait(smem_u32(full_bar + s), use & 1, abort_flag, p.status, p.wait_limit);
         if (!ok) break;
         tc_fence_after();
         const uint32_t a_addr = base + s * stage_bytes;
@@ -176,7 +178,7 @@ k_gemm_tc(const __grid_constant__ CUtensorMap map_w0, const __grid_constant__ CU
   } else if (n_kb > 0) {
     // ------------------------------------------------ epilogue warps 0..3
     // one decision for the four epilogue warps (they meet at a named barrier below)
-    const bool ok = bar_and_128(mbar_wait(smem_u32(acc_bar), 0, abort_flag, p.status));
+    const bool ok = bar_and_128(mbar_wait(smem_u32(acc_bar), 0, abort_flag, p.status, p.wait_limit));
     tc_fence_after();
     const int f = f0 + warp * 32 + lane;                    // weight row within the segment
     const bool f_ok = f < seg_N;
@@ -423,6 +425,8 @@ int cod_launch_gemm_tc(cod_ctx* c, const GemmArgs& g, cudaStream_t st) {
   p.lse_part = g.amax ? g.lse_part : nullptr;
   p.sample_state = g.sample_state;
   p.status = c->status;
+  p.wait_limit = c->wait_limit > 0 ? c->wait_limit : WAIT_LIMIT_CYCLES;
+  p.skip_copies = c->selftest_skip_copies;
 
   CUtensorMap mw[3], ma;
   for (int i = 0; i < 3; ++i) {

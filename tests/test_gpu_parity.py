@@ -458,6 +458,39 @@ def test_status_word_and_argument_errors():
     P.close()
 
 
+def test_bounded_wait_runs_out_cleanly_and_the_context_stays_usable():
+    """Failure detection without a fault: with the self-test switch on, the weight-streaming contraction
+    requests no operands, so its consumers' bounded waits expire (after ~2e5 SM cycles here); every CTA
+    raises COD_DEV_TIMEOUT, frees its tensor memory and returns. Nothing traps, nothing stays in flight.
+    The same context then runs a normal round that matches the oracle."""
+    Hn, B = _H(), _B()
+    P = Hn.Pair(_workloads()["small_bf16"], seed=4, wo_scale=30.0)
+    sh = P.wl.shape
+    n = 24
+    x = torch.randn(n, sh.d_model, device="cuda")
+    tok = torch.full((n,), 7, dtype=torch.int32, device="cuda")
+    P.ctx.set_wait_limit(200_000)
+    P.ctx.selftest_expire_wait(True)
+    P.ctx.lm_head_argmax(x, n, tok)
+    torch.cuda.synchronize()
+    assert P.ctx.poll_status(clear=True) == B.DEV_TIMEOUT
+    assert (tok.cpu().numpy() == -1).all()                    # no row completed: the documented "no result"
+    P.ctx.selftest_expire_wait(False)
+    P.ctx.set_wait_limit(0)
+    # ... and the context is as good as new
+    P.ctx.lm_head_argmax(x, n, tok)
+    torch.cuda.synchronize()
+    t_o, gap, _ = orc.lm_head_argmax(x.cpu().numpy().astype(np.float64), P.w_o, P.cfg_o)
+    sure = gap >= Hn.GAP
+    assert np.array_equal(tok.cpu().numpy()[sure], t_o[sure])
+    for r in range(2):
+        L0 = P.st_o.committed_len.copy()
+        res_o = P.run_round(r, orc.MODE_CARRY)
+        _check_round(P, res_o, L0, Hn.TOL[sh.dtype])
+    assert P.ctx.poll_status() == 0
+    P.close()
+
+
 def test_reconvergence_count_bit_exact():
     """Random suffixes over a small alphabet (many coincidences), every length 0..W, W = 16 and 32."""
     B = _B()
