@@ -676,6 +676,75 @@ def run_micro_round(args):
     ctx.close()
 
 
+def run_timeline(args):
+    """--micro timeline: ONE graph-replayed round of the workload seen through CUPTI activity records
+    (torch.profiler): every kernel's start, end and its share of the dependency chain - the time from the later
+    of (its start, its predecessor's end) to its own end, which is what the round pays for it when launches
+    overlap programmatically. A profiler view for finding where a round's time goes; never a bench value."""
+    import torch
+    from torch.profiler import ProfilerActivity, profile
+
+    import __graft_entry__ as entry
+    from paper_2609_14717_b200 import binding as B
+
+    entry.build()
+    torch.cuda.set_device(0)
+    wl = bench_workload(args.workload, 40)
+    sh = wl.shape
+    lay = synth.make_layout(wl, args.seed)
+    cfg = B.make_config(sh, wl.S, int(lay["max_pages_per_seq"]), int(lay["n_pages"]), attn_split_len=args.attn_split)
+    ctx = B.Context(cfg)
+    td = B.torch_dtype(sh.dtype)
+    gen = torch.Generator(device="cuda").manual_seed(args.seed)
+    rnd = lambda *shape, scale=1.0: (torch.randn(*shape, generator=gen, device="cuda") * scale).to(td)
+    ctx.set_weights({k: (rnd(*v, scale=0.02) if not k.startswith("g_") else torch.ones(*v, device="cuda", dtype=td))
+                     for k, v in synth.weight_shapes(sh).items()})
+    state = B.State(cfg, sh.dtype, wl.S, lay["block_table"], lay["committed_len"])
+    for l in range(sh.n_layers):
+        state.kv_pool[l].copy_(rnd(*state.kv_pool[l].shape))
+    rd = synth.make_round(wl, args.seed, 0)
+    d, t = torch.from_numpy(rd["draft"]).cuda(), torch.from_numpy(rd["target"]).cuda()
+    H = B.to_device(rd["H"], sh.dtype)
+    nd = torch.zeros((wl.S, sh.W), dtype=torch.int32, device="cuda")
+    mode = B.COD_BASELINE if args.baseline else B.COD_CARRY
+    one = lambda: ctx.draft_round(d, t, H, wl.S, wl.n_forced, mode, state, None, nd, None)
+    side = torch.cuda.Stream()
+    side.wait_stream(torch.cuda.current_stream())
+    with torch.cuda.stream(side):
+        one()
+    torch.cuda.current_stream().wait_stream(side)
+    torch.cuda.synchronize()
+    g = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(g):
+        one()
+    for _ in range(max(args.warmup, 3)):
+        g.replay()
+    torch.cuda.synchronize()
+    with profile(activities=[ProfilerActivity.CUDA]) as prof:
+        for _ in range(3):
+            g.replay()
+        torch.cuda.synchronize()
+    ev = sorted((e for e in prof.events() if e.device_type == torch.autograd.DeviceType.CUDA),
+                key=lambda e: e.time_range.start)
+    rows = [(e.name, e.time_range.start, e.time_range.end) for e in ev]
+    first = [i for i, r in enumerate(rows) if "k_verify_accept" in r[0]]
+    last = rows[first[-1]:]
+    t0, prev_end, out, agg = last[0][1], last[0][1], [], {}
+    for name, s0, e0 in last:
+        short = name.replace("(anonymous namespace)::", "").replace("void ", "").split("(")[0]
+        chain = e0 - max(s0, prev_end)
+        out.append({"kernel": short, "start_us": s0 - t0, "end_us": e0 - t0, "chain_us": max(chain, 0.0)})
+        a = agg.setdefault(short, [0, 0.0])
+        a[0] += 1
+        a[1] += max(chain, 0.0)
+        prev_end = max(prev_end, e0)
+    print(json.dumps({"micro": "timeline", "workload": wl.name, "round_us": prev_end - t0,
+                      "chain_us_by_kernel": {k: {"launches": v[0], "chain_us": v[1]} for k, v in
+                                             sorted(agg.items(), key=lambda kv: -kv[1][1])},
+                      "kernels": out if args.verbose else None}))
+    ctx.close()
+
+
 def run_micro(args):
     """--micro attn|lmhead: one entry point alone on the workload's shapes (one drafter layer, so the
     device footprint stays small enough for a profiler capture). Prints its own JSON line."""
@@ -686,6 +755,8 @@ def run_micro(args):
 
     if args.micro == "gemm":
         return run_micro_round(args)
+    if args.micro == "timeline":
+        return run_timeline(args)
     entry.build()
     torch.cuda.set_device(0)
     peaks = load_peaks()
@@ -837,10 +908,11 @@ def main():
     ap.add_argument("--sweep", action="store_true", help="carryover-overhead sweep over batch, block and rejected fraction")
     ap.add_argument("--sweep-reps", type=int, default=7, help="--sweep: interleaved passes per mode and point")
     ap.add_argument("--attn-split", type=int, default=0, help="keys per attention split (0 = library default)")
-    ap.add_argument("--micro", default=None, choices=["attn", "lmhead", "lmsample", "lmrank", "gemm"],
+    ap.add_argument("--micro", default=None, choices=["attn", "lmhead", "lmsample", "lmrank", "gemm", "timeline"],
                     help="time one entry point alone (small footprint; meant for profiler captures)")
     ap.add_argument("--shape", default=None, choices=["fc", "kv", "qkv", "oproj", "lmhead", "attn"],
                     help="--micro gemm: the contraction class to time inside a one-layer round")
+    ap.add_argument("--verbose", action="store_true", help="--micro timeline: also list every launch")
     ap.add_argument("--baseline", action="store_true", help="--micro gemm: run the rounds in baseline mode")
     ap.add_argument("--record-traffic", default=None, metavar="NCU_CSV",
                     help="store the DRAM bytes of an ncu capture (one launch) in profiles/dram_traffic.txt")

@@ -121,6 +121,12 @@ k_gemm_tc2(const __grid_constant__ CUtensorMap map_w0, const __grid_constant__ C
   }
   // NOTE: both CTAs of a pair take the same decision here (it depends on the pair's tile only)
   const int n_kb = (i0 < row_hi && i0 + NTOK > row_lo) ? kb1 - kb0 : 0;   // 0: no token rows here, only the requested weights to absorb
+  // accumulators whose 256 token rows miss this segment's row range altogether are neither fed nor multiplied
+  // (a contraction grouped by row: the group boundary usually leaves one of the two accumulators empty)
+  uint32_t acc_on = 0;
+  for (int a = 0; a < p.n_acc; ++a)
+    if (i0 + a * NT < row_hi && i0 + (a + 1) * NT > row_lo) acc_on |= 1u << a;
+  const uint32_t stage_tx = 2 * (A_TILE_BYTES + static_cast<uint32_t>(__popc(acc_on)) * B_TILE_BYTES);
 
   if (warp == 4) {
     if (lane == 0) {
@@ -134,12 +140,12 @@ k_gemm_tc2(const __grid_constant__ CUtensorMap map_w0, const __grid_constant__ C
         const int s = it % STAGES, use = it / STAGES;
         if (use > 0 && !mbar_wait(smem_u32(empty_bar + s), (use - 1) & 1, abort_flag, p.status)) break;
         const uint32_t fb = smem_u32(full_bar + s);
-        if (rank == 0) mbar_expect_tx(fb, 2 * STAGE_BYTES);     // both CTAs' bytes land on the leader's barrier
+        if (rank == 0) mbar_expect_tx(fb, stage_tx);            // both CTAs' bytes land on the leader's barrier
         const uint32_t a_dst = base + s * STAGE_BYTES;
         const int k = (kb0 + it) * BK;
         if (it >= n_pre) tma_load_2d_pair(a_dst, map_w, k, f0, fb & PEER_MASK);
         for (int a = 0; a < p.n_acc; ++a)      // accumulator a covers tokens [i0 + a*256, +256): this CTA stages its half
-          tma_load_2d_pair(a_dst + A_TILE_BYTES + a * B_TILE_BYTES, &map_a, k, i0 + a * NT + rank * (NT / 2), fb & PEER_MASK);
+          if (acc_on & (1u << a)) tma_load_2d_pair(a_dst + A_TILE_BYTES + a * B_TILE_BYTES, &map_a, k, i0 + a * NT + rank * (NT / 2), fb & PEER_MASK);
       }
     }
   } else if (warp == 5) {
@@ -155,6 +161,7 @@ k_gemm_tc2(const __grid_constant__ CUtensorMap map_w0, const __grid_constant__ C
         const uint32_t a_addr = base + s * STAGE_BYTES;
         const uint64_t a_desc = desc_kmajor_sw128(a_addr);
         for (int a = 0; a < p.n_acc; ++a) {
+          if (!(acc_on & (1u << a))) continue;
           const uint64_t b_desc = desc_kmajor_sw128(a_addr + A_TILE_BYTES + a * B_TILE_BYTES);
 #pragma unroll
           for (int k = 0; k < BK / UK; ++k)
