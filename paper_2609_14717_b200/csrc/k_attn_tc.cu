@@ -583,7 +583,9 @@ int launch(cod_ctx* c, int layer, const void* q, const void* kb, const void* vb,
   p.n_pages = f.n_pages; p.max_pages = f.max_pages_per_seq; p.max_batch = f.max_batch;
   p.split_len = c->tc_split_len; p.max_parts = c->tc_max_parts;
   p.part_o = c->attn_o; p.part_ml = c->attn_ml; p.status = c->status;
-  static bool configured = false;
+  // the attribute belongs to (kernel, device): one flag per device the process may use
+  static bool configured_dev[64] = {};
+  bool& configured = configured_dev[c->device & 63];
   if (!configured) {
     if (cudaFuncSetAttribute(k_attn_tc<DUAL>, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(G::SMEM)) != cudaSuccess)
       return COD_ERR_CUDA;

@@ -446,7 +446,9 @@ int cod_launch_gemm_tc(cod_ctx* c, const GemmArgs& g, cudaStream_t st) {
   using kernel_t = void (*)(const CUtensorMap, const CUtensorMap, const CUtensorMap, const CUtensorMap, const TcParams);
   static const kernel_t kernels[4] = {k_gemm_tc<false, false, false>, k_gemm_tc<false, true, false>,
                                       k_gemm_tc<true, false, false>, k_gemm_tc<false, false, true>};
-  static size_t configured[4] = {0, 0, 0, 0};
+  // the attribute belongs to (kernel, device): one record per device the process may use
+  static size_t configured_dev[64][4] = {};
+  size_t* configured = configured_dev[c->device & 63];
   if (smem > configured[variant]) {
     if (cudaFuncSetAttribute(kernels[variant], cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem)) != cudaSuccess)
       return COD_ERR_CUDA;

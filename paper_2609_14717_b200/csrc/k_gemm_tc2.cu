@@ -385,7 +385,9 @@ int cod_launch_gemm_tc2(cod_ctx* c, const GemmArgs& g, cudaStream_t st) {
 
   const size_t smem = static_cast<size_t>(p.stages) * (A_TILE_BYTES + p.n_acc * B_TILE_BYTES) + 1024 + 18 * 8 +
                       static_cast<size_t>(4) * p.n_acc * NT * 8;
-  static size_t configured[2] = {0, 0};
+  // the attribute belongs to (kernel, device): one record per device the process may use
+  static size_t configured_dev[64][2] = {};
+  size_t* configured = configured_dev[c->device & 63];
   const int sample = p.lse_part != nullptr ? 1 : 0;
   if (smem > configured[sample]) {
     const cudaError_t e = sample ? cudaFuncSetAttribute(k_gemm_tc2<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem))
