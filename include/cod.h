@@ -74,6 +74,11 @@ enum cod_mode {
 /* cod_config.flags */
 #define COD_F_HIDDEN_NORM 1u /* RMS-normalise (with gain g_hidden) the output of F */
 #define COD_F_NO_TENSOR_CORES 2u /* use the plain-FMA kernels only (an on-GPU cross-check) */
+/* Attention grids several waves deep run either as one CTA per (sequence, head, part) or as persistent CTAs that
+   walk the longest-first work list without draining their pipelines between items. Same results either way; the
+   library picks by geometry (persistent for 128 query rows per head group, i.e. block 32). These two force it: */
+#define COD_F_ATTN_ONE_ITEM_CTAS 32u
+#define COD_F_ATTN_PERSISTENT 64u
 #define COD_F_NO_CARRY_EMBED 8u /* rejected rows pass F unmarked ("no explicit discrimination", Section 5) */
 #define COD_F_REJ_PROJECTOR 16u /* rejected rows pass their own fusion map fc_rej instead of F + E_carry
                                    ("separate projector", Section 5; its shape is taken as F's) */

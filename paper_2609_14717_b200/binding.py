@@ -20,6 +20,8 @@ COD_F32, COD_BF16 = 0, 1
 COD_CARRY, COD_BASELINE = 0, 1
 COD_F_HIDDEN_NORM = 1
 COD_F_NO_TENSOR_CORES = 2
+COD_F_ATTN_ONE_ITEM_CTAS = 32
+COD_F_ATTN_PERSISTENT = 64
 COD_F_QK_NORM = 4
 COD_F_NO_CARRY_EMBED = 8
 COD_F_REJ_PROJECTOR = 16
@@ -342,14 +344,14 @@ def lm_head_argmax_static(emb: torch.Tensor, g_final: torch.Tensor, x: torch.Ten
 
 
 def make_config(sh, max_batch: int, max_pages_per_seq: int, n_pages: int, attn_split_len: int = 0,
-                no_tensor_cores: bool = False) -> CodConfig:
+                no_tensor_cores: bool = False, extra_flags: int = 0) -> CodConfig:
     """cod_config from a synthetic DrafterShape."""
     return CodConfig(
         d_target=sh.d_target, n_cap=sh.n_cap, d_model=sh.d_model, n_layers=sh.n_layers, n_q_heads=sh.n_q,
         n_kv_heads=sh.n_kv, head_dim=sh.hd, vocab=sh.vocab, mask_token_id=sh.mask_token_id, block=sh.W,
         page_size=sh.page, max_batch=max_batch, max_pages_per_seq=max_pages_per_seq, n_pages=n_pages,
         dtype=COD_BF16 if sh.dtype == "bf16" else COD_F32,
-        flags=(COD_F_HIDDEN_NORM if sh.hidden_norm else 0) | (COD_F_NO_TENSOR_CORES if no_tensor_cores else 0)
+        flags=extra_flags | (COD_F_HIDDEN_NORM if sh.hidden_norm else 0) | (COD_F_NO_TENSOR_CORES if no_tensor_cores else 0)
         | (COD_F_QK_NORM if sh.qk_norm else 0)
         | {"embedding": 0, "none": COD_F_NO_CARRY_EMBED, "projector": COD_F_REJ_PROJECTOR}[sh.carry_variant],
         rope_theta=sh.rope_theta, rms_eps=sh.rms_eps,

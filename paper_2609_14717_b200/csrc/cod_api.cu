@@ -63,6 +63,7 @@ size_t carve(cod_ctx* c) {
   cv.take(c->attn_o, sizeof(float) * parts * f.head_dim);
   cv.take(c->attn_ml, sizeof(float) * parts * 4);
   if (c->tc_max_parts > 0) cv.take(c->attn_order, sizeof(int) * f.max_batch * c->tc_max_parts);
+  cv.take(c->attn_counter, 256);
   if (c->carry_cap > f.block) {
     cv.take(c->carry_base, sizeof(int) * f.max_batch);
     cv.take(c->carry_drop, sizeof(int) * f.max_batch);
@@ -187,6 +188,8 @@ int cod_create(const cod_config* cfg, cod_ctx** out) {
   c->R_max = f.max_batch * f.block;
   c->half = f.head_dim / 2;
   c->force_simt = (f.flags & COD_F_NO_TENSOR_CORES) != 0;
+  c->attn_one_item_ctas = (f.flags & COD_F_ATTN_ONE_ITEM_CTAS) != 0;
+  c->attn_persistent = (f.flags & COD_F_ATTN_PERSISTENT) != 0;
   c->carry_cap = (f.carry_rounds > 1 ? f.carry_rounds : 1) * f.block;
   if (cudaDeviceGetAttribute(&c->n_sm, cudaDevAttrMultiProcessorCount, c->device) != cudaSuccess || c->n_sm < 1) c->n_sm = 148;
   c->split_len = f.attn_split_len > 0 ? f.attn_split_len : 512;

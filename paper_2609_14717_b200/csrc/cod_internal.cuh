@@ -159,6 +159,7 @@ struct cod_ctx {
   int* carry_drop;             // [max_batch] rows of U that leave this round (carry_rounds > 1), else null
   float* gemm_out2;            // a second, small slab buffer for the side branch of the round (null: no side branch)
   int* attn_order;             // [max_batch * tc_max_parts] longest-first work list of the tensor-core attention
+  int* attn_counter;           // work units the persistent attention CTAs have taken beyond their first (zero between launches)
   bool attn_order_stale;       // the lengths may have changed since the list was built
   int side_rows;               // the side branch is used for rounds of at most this many rows
   cudaStream_t side;           // side branch of the round: the first layer's embedding / Q/K/V chain
@@ -166,6 +167,8 @@ struct cod_ctx {
   size_t gemm_out_floats;
   void* hc;                    // [R_max, D_in] accepted rows of H packed densely (baseline mode)
   long long wait_limit;        // SM cycles a bounded device wait may last (0: the built-in limit, about 2 s)
+  int attn_one_item_ctas;      // 1: work-list attention as one CTA per item (the persistent form off; for A/B runs)
+  int attn_persistent;         // 1: the persistent form whatever the geometry
   int selftest_skip_copies;    // cod_selftest_expire_wait: single-CTA contractions request no operands
   int* perm;                  // [R] window rows in the order accepted-first (grouped contraction of the separate projector)
   void* z;                     // [R_max, D]

@@ -43,6 +43,8 @@ struct AttnParams {
   float* part_ml;                       // [S][n_kv][max_parts][M][4]   m (natural log units), l, l_carry
   const int* order;                     // null: CTA (x, y, z) = (part, head, sequence). Else CTA (x, y) = (head, i) works
                                         // on part order[i] = sequence << 16 | part, longest first; -1: nothing
+  int n_list;                           // entries of order[] (persistent kernel)
+  int* work_counter;                    // persistent kernel: units taken beyond each CTA's first (zero before the launch)
   uint32_t* status;
 };
 
@@ -63,7 +65,7 @@ struct Geo {
   static constexpr uint32_t OFF_K = OFF_P + P_BUF;       // P is single-buffered
   static constexpr uint32_t OFF_V = OFF_K + NK * SLOT;
   static constexpr uint32_t OFF_CTL = OFF_V + NV * SLOT;
-  static constexpr uint32_t SMEM = OFF_CTL + 256 + 1024 + 1024;   // barriers, page ids, alignment slack
+  static constexpr uint32_t SMEM = OFF_CTL + 512 + 1024 + 1024;   // barriers and the unit ring, page ids, alignment slack
   // tensor memory columns: S[2] (64 each) then O (128)
   static constexpr uint32_t COL_S = 0, COL_O = 128, TMEM_COLS = 256;
 };
@@ -450,6 +452,467 @@ k_attn_tc(const __grid_constant__ CUtensorMap map_pool, const __grid_constant__ 
   }
 }
 
+// ---------------------------------------------------------------------------------------------------------
+// The same attention as k_attn_tc for grids several waves deep, as a PERSISTENT kernel: two CTAs per SM walk the
+// longest-first work list with a fixed stride, and the pipeline never drains between work items. All ring slots,
+// score buffers and barrier phases are indexed by ONE step counter g that runs across items, so at an item
+// boundary the producers simply keep going: the next item's first K/V tiles are requested as soon as the slots
+// free up (the K producer also requests the next item's Q tile then, by TMA), and they stream while the soft-max
+// threads store the finished item's partial result. What a one-item CTA pays per item - launch, barrier set-up,
+// tensor-memory allocation, a Q gather, a first load with nothing else in flight, the drain - is paid once per
+// CTA here; with ~2.7 items per CTA at batch 32 that was a fifth of the kernel's time (bytes in flight dip
+// whenever CTAs turn over, and an HBM-bound kernel is only as fast as its bytes in flight).
+// Differences inside an item: Q arrives by two 5-D TMA boxes instead of a gather; the page of each tile comes
+// straight from the block table, one step ahead, into a register; tail items (partial page + carried + block
+// rows, gathered with plain loads by the soft-max threads) complete their slot with one elected arrival, so a
+// barrier serves TMA-fed and gathered tiles alike; the first PV of an item waits until the soft-max threads have
+// read the previous item's O out of tensor memory (o_free).
+// Twelve warps in three warpgroups: 0-3 soft-max; 4 the K (and Q) producer, 5 the MMA issuer, 6 the V producer;
+// 7-11 only hand their registers over. After the common set-up the warpgroups rebalance their register budgets
+// (setmaxnreg): the soft-max rows' 64 scores stay in registers at 144 per thread, everyone else keeps 48.
+// The increase WAITS, without any bound, until the CTA's own pool holds the registers: the budgets must fit what
+// the CTA was launched with (PS_REGS_LAUNCH per thread; the host checks the compiled kernel before the first launch),
+// and ptxas applies a raised budget only to code inside the branch that executes the instruction.
+constexpr int NTHREADS_PS = 384, PS_REGS_LAUNCH = 80, PS_REGS_SOFTMAX = 144, PS_REGS_OTHER = 48;
+static_assert(128 * PS_REGS_SOFTMAX + (NTHREADS_PS - 128) * PS_REGS_OTHER <= NTHREADS_PS * PS_REGS_LAUNCH, "setmaxnreg budgets exceed the CTA's pool");
+template <bool DUAL>
+__global__ void __launch_bounds__(NTHREADS_PS, 2)
+k_attn_ps(const __grid_constant__ CUtensorMap map_pool, const __grid_constant__ CUtensorMap map_zero,
+          const __grid_constant__ CUtensorMap map_q, const AttnParams p) {
+  cod_pdl_prologue();
+  using G = Geo<DUAL>;
+  extern __shared__ uint8_t smem_raw[];
+  const uint32_t raw = smem_u32(smem_raw);
+  const uint32_t base = (raw + 1023u) & ~1023u;
+  uint8_t* sm = smem_raw + (base - raw);
+  uint64_t* bars = reinterpret_cast<uint64_t*>(sm + G::OFF_CTL);
+  uint64_t* k_full = bars;                  // [NK]
+  uint64_t* k_empty = bars + 5;             // [NK]
+  uint64_t* v_full = bars + 10;             // [NV]
+  uint64_t* v_empty = bars + 15;            // [NV]
+  uint64_t* s_full = bars + 20;             // [2]
+  uint64_t* p_full = bars + 22;             // [2]
+  uint64_t* o_full = bars + 24;             // [2]
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 26);
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+  uint64_t* q_full = bars + 27;             // the item's Q tile has landed
+  uint64_t* o_free = bars + 28;             // the previous item's O has been read out of tensor memory
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int M = p.W * p.rep;
+  uint32_t flags = 0;
+
+  // One work item = (sequence, KV head, part). Every role decodes the same sequence of items for this CTA.
+  struct Item { int s, h, split, F, Lr, c, n_tail, k_begin, k_end, n_it; bool is_tail; uint32_t bad; };
+  // Work unit w = list entry w / n_kv, head w % n_kv. A CTA's first unit is its own index; every further one is
+  // the next the whole grid has not taken yet (a device counter): over the longest-first list that is the
+  // longest-processing-time rule, which a fixed assignment cannot match when CTAs progress at different rates.
+  // The K producer's first lane takes the unit and publishes it to the other roles through a small ring.
+  int* witem = reinterpret_cast<int*>(bars + 40);     // [8]
+  uint64_t* item_bar = bars + 32;                     // [8] unit j of this CTA has been published
+  auto take_unit = [&](int j) {                       // (K producer, lane 0)
+    int w = j == 0 ? static_cast<int>(blockIdx.x) : static_cast<int>(gridDim.x) + atomicAdd(p.work_counter, 1);
+    if (w / p.n_kv >= p.n_list || p.order[w / p.n_kv] < 0) w = -1;      // the list is packed: nothing further
+    witem[j & 7] = w;
+    mbar_arrive(smem_u32(item_bar + (j & 7)));
+  };
+  auto unit_of = [&](int j, bool& ok) -> int {        // every role; ok false: a wait ran out
+    ok = mbar_wait(smem_u32(item_bar + (j & 7)), (j >> 3) & 1, abort_flag, p.status);
+    return ok ? witem[j & 7] : -1;
+  };
+  auto decode = [&](int w, Item& t) {
+    const int idx = w / p.n_kv;
+    const int item = p.order[idx];
+    t.h = w - idx * p.n_kv; t.s = item >> 16; t.split = item & 0xFFFF;
+    int L = p.committed_len[t.s];
+    int c = p.use_carry ? p.carry_len[t.s] : 0;
+    t.bad = 0;
+    if (L < 0 || L > p.max_pages * PAGE) { t.bad = COD_DEV_BAD_LEN; L = max(0, min(L, p.max_pages * PAGE)); }
+    if (c < 0 || c > p.cap) { t.bad = COD_DEV_BAD_LEN; c = max(0, min(c, p.cap)); }
+    t.c = c;
+    t.F = (L / PAGE) * PAGE;
+    const int n_reg = (t.F + p.split_len - 1) / p.split_len;
+    t.is_tail = t.split >= n_reg;                     // (the list holds existing parts only: == n_reg)
+    t.Lr = L - t.F;
+    t.n_tail = t.Lr + c + p.W;
+    t.k_begin = t.is_tail ? 0 : t.split * p.split_len;
+    t.k_end = t.is_tail ? t.n_tail : min(t.F, t.k_begin + p.split_len);
+    t.n_it = (t.k_end - t.k_begin + G::KEYS_IT - 1) / G::KEYS_IT;
+  };
+
+  if (threadIdx.x == 0) {
+    for (int i = 0; i < G::NK; ++i) { mbar_init(smem_u32(k_full + i), 1); mbar_init(smem_u32(k_empty + i), 1); }
+    for (int i = 0; i < G::NV; ++i) { mbar_init(smem_u32(v_full + i), 1); mbar_init(smem_u32(v_empty + i), 1); }
+    for (int i = 0; i < 2; ++i) { mbar_init(smem_u32(s_full + i), 1); mbar_init(smem_u32(p_full + i), 128); mbar_init(smem_u32(o_full + i), 1); }
+    mbar_init(smem_u32(q_full), 1);
+    mbar_init(smem_u32(o_free), 128);
+    for (int i = 0; i < 8; ++i) mbar_init(smem_u32(item_bar + i), 1);
+    *abort_flag = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  if (warp == 5) tmem_alloc(smem_u32(tmem_slot), G::TMEM_COLS);
+  if (warp < 4) {
+    // query rows beyond the real ones stay zero for the whole kernel (the Q boxes never touch them)
+    for (int idx = threadIdx.x; idx < (G::MROWS - M) * 16; idx += 128) {
+      const int r = M + (idx >> 4), ch = idx & 15;
+      *reinterpret_cast<uint4*>(sm + (ch >> 3) * G::Q_HALF + r * 128 + ((ch & 7) << 4)) = make_uint4(0u, 0u, 0u, 0u);
+    }
+    fence_async_smem();
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = *tmem_slot;
+
+  if (warp >= 4) {
+  asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(PS_REGS_OTHER));
+  if (warp == 4 || warp == 6) {
+    // ------------------------------------------------ TMA producers: warp 4 K tiles (and the Q tile), warp 6 V tiles
+    const bool is_v = warp == 6;
+    const int pages_it = G::KEYS_IT / PAGE;             // 8 or 4 pages per step, one per lane
+    const int ring = is_v ? G::NV : G::NK;
+    uint64_t* full = is_v ? v_full : k_full;
+    uint64_t* empty = is_v ? v_empty : k_empty;
+    const uint32_t ring_off = is_v ? G::OFF_V : G::OFF_K;
+    const bool lane_on = lane < pages_it;
+    const uint32_t in_slot = (lane / (KT / PAGE)) * TILE_BYTES + (lane % (KT / PAGE)) * (PAGE * 128);
+    int g = 0, j = 0;
+    bool ok = true;
+    Item t;
+    for (;; ++j) {
+      if (!is_v && lane == 0) take_unit(j);
+      const int w = unit_of(j, ok);
+      if (!ok || w < 0) break;
+      decode(w, t);
+      if (!is_v) {
+        // Q of this item, once every QK of the previous item has retired (QKs retire in order)
+        if (lane == 0 && g > 0) ok = mbar_wait(smem_u32(k_empty + (g - 1) % G::NK), ((g - 1) / G::NK) & 1, abort_flag, p.status);
+        ok = __shfl_sync(0xffffffffu, ok, 0);
+        if (!ok) break;
+        if (lane == 0) {
+          const uint32_t qb = smem_u32(q_full);
+          mbar_expect_tx(qb, static_cast<uint32_t>(M) * HD * 2);
+          tma_load_5d(base, &map_q, 0, 0, 0, t.h, t.s * p.W, qb);
+          tma_load_5d(base + G::Q_HALF, &map_q, 0, 1, 0, t.h, t.s * p.W, qb);
+        }
+      }
+      if (!t.is_tail) {
+        // this lane's physical page comes from the block table, one step ahead of its use
+        const int* table = p.block_table + t.s * p.max_pages + t.k_begin / PAGE + lane;
+        int pg_next = (lane_on && t.k_begin + lane * PAGE < t.k_end) ? table[0] : -1;
+        for (int it = 0; it < t.n_it; ++it) {
+          const int gg = g + it;
+          const int key0 = t.k_begin + it * G::KEYS_IT + lane * PAGE;
+          int pg = pg_next;
+          if (lane_on && key0 + G::KEYS_IT < t.k_end) pg_next = table[(it + 1) * pages_it];
+          int row = -1;                                 // first row of this lane's page tile in the pool map
+          if (lane_on && key0 < t.k_end) {
+            if (pg < 0 || pg >= p.n_pages) { flags |= COD_DEV_BAD_PAGE; pg = -1; }
+            if (pg >= 0) row = (((p.layer * p.n_pages + pg) * p.n_kv + t.h) * 2 + (is_v ? 1 : 0)) * PAGE;
+          }
+          const int slot = gg % ring, use = gg / ring;
+          if (lane == 0 && use > 0) ok = mbar_wait(smem_u32(empty + slot), (use - 1) & 1, abort_flag, p.status);
+          ok = __shfl_sync(0xffffffffu, ok, 0);
+          if (!ok) break;
+          const uint32_t fb = smem_u32(full + slot);
+          if (lane == 0) mbar_expect_tx(fb, G::SLOT);
+          __syncwarp();
+          if (lane_on) {
+            const uint32_t dst = base + ring_off + slot * G::SLOT + in_slot;
+            if (row >= 0) {
+              tma_load_3d(dst, &map_pool, 0, 0, row, fb);
+              tma_load_3d(dst + HALF_BYTES, &map_pool, 0, 1, row, fb);
+            } else {
+              tma_load_3d(dst, &map_zero, 0, 0, 0, fb);
+              tma_load_3d(dst + HALF_BYTES, &map_zero, 0, 1, 0, fb);
+            }
+          }
+        }
+      }
+      if (!ok) break;
+      g += t.n_it;
+    }
+  } else if (warp == 5) {
+    // ------------------------------------------------ MMA issuer
+    if (lane == 0) {
+      const uint32_t idesc_qk = instr_desc(G::MROWS, KT, 0);
+      const uint32_t idesc_pv = instr_desc(G::MROWS, HD, 1);
+      const uint64_t q_desc = desc_kmajor_sw128(base);
+      bool ok = true;
+      auto issue_qk = [&](int gg) -> bool {
+        const int slot = gg % G::NK;
+        if (!mbar_wait(smem_u32(k_full + slot), (gg / G::NK) & 1, abort_flag, p.status)) return false;
+        tc_fence_after();
+#pragma unroll
+        for (int tl = 0; tl < G::TILES; ++tl) {
+          const uint64_t k_desc = desc_kmajor_sw128(base + G::OFF_K + slot * G::SLOT + tl * TILE_BYTES);
+          const uint32_t d = tmem_base + G::COL_S + (gg & 1) * KT + (static_cast<uint32_t>(16 * tl) << 16);
+#pragma unroll
+          for (int k = 0; k < HD / 16; ++k) {
+            const uint32_t qa = (k < 4 ? 0u : (G::Q_HALF >> 4)) + (k & 3) * 2;
+            const uint32_t ka = (k < 4 ? 0u : (HALF_BYTES >> 4)) + (k & 3) * 2;
+            umma_bf16(d, q_desc + qa, k_desc + ka, idesc_qk, k ? 1u : 0u);
+          }
+        }
+        umma_commit(smem_u32(s_full + (gg & 1)));
+        umma_commit(smem_u32(k_empty + slot));
+        return true;
+      };
+      int g = 0, j = 0;
+      Item t;
+      for (;; ++j) {
+        const int w = unit_of(j, ok);
+        if (!ok || w < 0) break;
+        decode(w, t);
+        ok = mbar_wait(smem_u32(q_full), j & 1, abort_flag, p.status);
+        if (!ok) break;
+        ok = issue_qk(g);
+        for (int it = 0; it < t.n_it && ok; ++it) {
+          const int gg = g + it;
+          if (it + 1 < t.n_it) ok = issue_qk(gg + 1);
+          if (!ok) break;
+          const int slot = gg % G::NV;
+          ok = mbar_wait(smem_u32(p_full + (gg & 1)), (gg >> 1) & 1, abort_flag, p.status) &&
+               mbar_wait(smem_u32(v_full + slot), (gg / G::NV) & 1, abort_flag, p.status);
+          // the first PV of an item overwrites O: the previous item's O must have been read
+          if (ok && it == 0 && j > 0) ok = mbar_wait(smem_u32(o_free), (j - 1) & 1, abort_flag, p.status);
+          if (!ok) break;
+          tc_fence_after();
+#pragma unroll
+          for (int tl = 0; tl < G::TILES; ++tl) {
+            const uint64_t p_desc = desc_kmajor_sw128(base + G::OFF_P + tl * G::P_TILE);
+            const uint64_t v_desc = desc_mnmajor_sw128(base + G::OFF_V + slot * G::SLOT + tl * TILE_BYTES, HALF_BYTES);
+            const uint32_t d = tmem_base + G::COL_O + (static_cast<uint32_t>(16 * tl) << 16);
+#pragma unroll
+            for (int kk = 0; kk < KT / 16; ++kk)       // 16 keys per MMA: 32 bytes along P's rows, 16 rows of V
+              umma_bf16(d, p_desc + kk * 2, v_desc + kk * ((16 * 128) >> 4), idesc_pv, (it | kk) ? 1u : 0u);
+          }
+          umma_commit(smem_u32(o_full + (gg & 1)));
+          umma_commit(smem_u32(v_empty + slot));
+        }
+        if (!ok) break;
+        g += t.n_it;
+      }
+    }
+  }
+  } else {
+    asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(PS_REGS_SOFTMAX));
+    // ------------------------------------------------ softmax: one thread per (row, tile), as in k_attn_tc
+    const int T = threadIdx.x;
+    const int tile = DUAL ? (lane >> 4) : 0;
+    const int r = DUAL ? (16 * warp + (lane & 15)) : T;
+    const uint32_t t_lane = tmem_base + (static_cast<uint32_t>(32 * warp) << 16);
+    const float sl2 = rsqrtf(static_cast<float>(HD)) * 1.4426950408889634f;   // raw score -> log2 units
+    const float rescale_gap = 8.f / sl2;
+    bool ok = true;
+    int g = 0, j = 0;
+    Item t;
+    for (;; ++j) {
+      const int w = unit_of(j, ok);
+      ok = __all_sync(0xffffffffu, ok);
+      if (!ok || w < 0) break;
+      decode(w, t);
+      float m_ref = -INFINITY, l_run = 0.f, lc_run = 0.f;
+      const int s = t.s, h = t.h, c = t.c, Lr = t.Lr, F = t.F, n_it = t.n_it, k_begin = t.k_begin, k_end = t.k_end,
+                n_tail = t.n_tail, split = t.split;
+      const bool is_tail = t.is_tail;
+      flags |= t.bad;
+#pragma unroll 1
+      for (int it = 0; it < n_it && ok; ++it) {
+        const int gg = g + it;
+        if (is_tail) {
+          // gather this step's rows (partial page, carried rows, block rows) with plain loads: first the K
+          // rows (the MMA warp asks for them first), then the V rows; one elected arrival completes the slot
+          constexpr int GB = 8;                               // independent 16-byte loads in flight per thread
+#pragma unroll 1
+          for (int kv = 0; kv < 2; ++kv) {
+            const int ring = kv ? G::NV : G::NK;
+            const int slot = gg % ring, use = gg / ring;
+            uint64_t* full = kv ? v_full : k_full;
+            uint64_t* empty = kv ? v_empty : k_empty;
+            if (use > 0) {
+              ok = __all_sync(0xffffffffu, mbar_wait(smem_u32(empty + slot), (use - 1) & 1, abort_flag, p.status));
+              if (!ok) break;
+            }
+            for (int idx0 = T; idx0 < G::KEYS_IT * 16; idx0 += 128 * GB) {
+              uint4 val[GB];
+              uint32_t dst[GB];
+#pragma unroll
+              for (int u = 0; u < GB; ++u) {
+                const int idx = idx0 + u * 128;
+                const int ch = idx & 15, jk = idx >> 4;                         // chunk, key within the step
+                const int gk = it * G::KEYS_IT + jk;
+                const __nv_bfloat16* src = nullptr;
+                if (gk < Lr) {
+                  int pg = p.block_table[s * p.max_pages + F / PAGE];
+                  if (pg < 0 || pg >= p.n_pages) { flags |= COD_DEV_BAD_PAGE; }
+                  else src = p.pool + ((((static_cast<size_t>(p.layer) * p.n_pages + pg) * p.n_kv + h) * 2 + kv) * PAGE + gk) * HD;
+                } else if (gk < Lr + c) {
+                  src = p.carry + ((((static_cast<size_t>(p.layer) * p.max_batch + s) * p.n_kv + h) * 2 + kv) * p.cap + (gk - Lr)) * HD;
+                } else if (gk < n_tail) {
+                  src = (kv ? p.vb : p.kb) + static_cast<size_t>(s * p.W + (gk - Lr - c)) * (p.n_kv * HD) + h * HD;
+                }
+                val[u] = src ? *reinterpret_cast<const uint4*>(src + ch * 8) : make_uint4(0u, 0u, 0u, 0u);
+                const int jj = jk & (KT - 1), tl = jk / KT;
+                dst[u] = (kv ? G::OFF_V : G::OFF_K) + slot * G::SLOT + tl * TILE_BYTES +
+                         (ch >> 3) * HALF_BYTES + jj * 128 + (((ch & 7) ^ (jj & 7)) << 4);
+              }
+#pragma unroll
+              for (int u = 0; u < GB; ++u) *reinterpret_cast<uint4*>(sm + dst[u]) = val[u];
+            }
+            fence_async_smem();
+            asm volatile("bar.sync 2, 128;" ::: "memory");
+            if (T == 0) mbar_arrive(smem_u32(full + slot));
+          }
+          if (!ok) break;
+        }
+
+        ok = __all_sync(0xffffffffu, mbar_wait(smem_u32(s_full + (gg & 1)), (gg >> 1) & 1, abort_flag, p.status));
+        if (!ok) break;
+        tc_fence_after();
+        const int key_t0 = k_begin + it * G::KEYS_IT + tile * KT;         // first key of this thread's tile
+        const int n_valid = max(0, min(KT, k_end - key_t0));
+        float sc[KT];
+        {
+          uint32_t v[32];
+          tmem_ld32(t_lane + G::COL_S + (gg & 1) * KT, v);
+#pragma unroll
+          for (int q = 0; q < 32; ++q) sc[q] = __uint_as_float(v[q]);
+          tmem_ld32(t_lane + G::COL_S + (gg & 1) * KT + 32, v);
+#pragma unroll
+          for (int q = 0; q < 32; ++q) sc[32 + q] = __uint_as_float(v[q]);
+        }
+        if (n_valid < KT) {                                  // only the last step of a part is ragged
+#pragma unroll
+          for (int q = 0; q < KT; ++q) sc[q] = q < n_valid ? sc[q] : -INFINITY;
+        }
+        float mx4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};      // four independent chains
+#pragma unroll
+        for (int q = 0; q < KT; q += 4) {
+          mx4[0] = fmaxf(mx4[0], sc[q]); mx4[1] = fmaxf(mx4[1], sc[q + 1]);
+          mx4[2] = fmaxf(mx4[2], sc[q + 2]); mx4[3] = fmaxf(mx4[3], sc[q + 3]);
+        }
+        const float mx = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3]));
+        const bool need = mx > m_ref + rescale_gap;        // also true for the first finite maximum
+        if (__any_sync(0xffffffffu, need)) {
+          const float m_new = need ? mx : m_ref;
+          const float factor = need ? ex2_approx((m_ref - m_new) * sl2) : 1.f;     // ex2(-inf) = 0
+          if (it > 0) {
+            // O is relative to the old reference: once PV(g-1) has landed, scale this warp's rows
+            ok = __all_sync(0xffffffffu, mbar_wait(smem_u32(o_full + ((gg - 1) & 1)), ((gg - 1) >> 1) & 1, abort_flag, p.status));
+            if (!ok) break;
+            tc_fence_after();
+#pragma unroll
+            for (int q4 = 0; q4 < HD / 32; ++q4) {
+              uint32_t v[32];
+              tmem_ld32(t_lane + G::COL_O + q4 * 32, v);
+#pragma unroll
+              for (int q = 0; q < 32; ++q) v[q] = __float_as_uint(__uint_as_float(v[q]) * factor);
+              tmem_st32(t_lane + G::COL_O + q4 * 32, v);
+            }
+          }
+          l_run *= factor;
+          lc_run *= factor;
+          m_ref = m_new;
+        }
+        if (gg >= 1) {   // the P buffer about to be overwritten was read by PV(g-1) (possibly the previous item's last)
+          ok = __all_sync(0xffffffffu, mbar_wait(smem_u32(o_full + ((gg - 1) & 1)), ((gg - 1) >> 1) & 1, abort_flag, p.status));
+          if (!ok) break;
+        }
+        const float neg = m_ref == -INFINITY ? 0.f : -m_ref * sl2;
+        float ps4[4] = {0.f, 0.f, 0.f, 0.f}, pcar = 0.f;
+        uint8_t* prow = sm + G::OFF_P + tile * G::P_TILE + r * 128;
+        const int car0 = is_tail ? Lr - (it * G::KEYS_IT + tile * KT) : KT;  // carried keys: [car0, car0 + c)
+#pragma unroll
+        for (int ch = 0; ch < 8; ++ch) {
+          uint32_t packed[4];
+#pragma unroll
+          for (int e = 0; e < 4; ++e) {
+            const int q = ch * 8 + e * 2;
+            const float p0 = ex2_approx(fmaf(sc[q], sl2, neg)), p1 = ex2_approx(fmaf(sc[q + 1], sl2, neg));
+            ps4[e] += p0 + p1;
+            if (is_tail) {
+              if (q >= car0 && q < car0 + c) pcar += p0;
+              if (q + 1 >= car0 && q + 1 < car0 + c) pcar += p1;
+            }
+            const __nv_bfloat162 b = __floats2bfloat162_rn(p0, p1);
+            packed[e] = *reinterpret_cast<const uint32_t*>(&b);
+          }
+          *reinterpret_cast<uint4*>(prow + ((ch ^ (r & 7)) << 4)) = make_uint4(packed[0], packed[1], packed[2], packed[3]);
+        }
+        fence_async_smem();
+        tc_fence_before();
+        mbar_arrive(smem_u32(p_full + (gg & 1)));
+        l_run += (ps4[0] + ps4[1]) + (ps4[2] + ps4[3]);
+        lc_run += pcar;
+      }
+      if (!ok) break;
+
+      // the item's partial result: O out of tensor memory once its last PV has landed (see k_attn_tc), then
+      // the accumulator is handed back to the MMA issuer
+      const int gl = g + n_it - 1;
+      ok = __all_sync(0xffffffffu, mbar_wait(smem_u32(o_full + (gl & 1)), (gl >> 1) & 1, abort_flag, p.status));
+      if (!ok) break;
+      tc_fence_after();
+      float w_me = 1.f, w_other = 0.f;
+      float m_out = m_ref;
+      if (DUAL) {
+        const float m_o = __shfl_xor_sync(0xffffffffu, m_ref, 16);
+        const float l_o = __shfl_xor_sync(0xffffffffu, l_run, 16), lc_o = __shfl_xor_sync(0xffffffffu, lc_run, 16);
+        m_out = fmaxf(m_ref, m_o);
+        const float base_m = m_out == -INFINITY ? 0.f : m_out;
+        w_me = ex2_approx((m_ref - base_m) * sl2);
+        w_other = ex2_approx((m_o - base_m) * sl2);
+        l_run = w_me * l_run + w_other * l_o;
+        lc_run = w_me * lc_run + w_other * lc_o;
+      }
+      const size_t rowi = ((static_cast<size_t>(s) * p.n_kv + h) * p.max_parts + split) * M + min(r, M - 1);
+      float4* po = reinterpret_cast<float4*>(p.part_o + rowi * HD);
+#pragma unroll
+      for (int q4 = 0; q4 < HD / 32; ++q4) {
+        uint32_t v[32];
+        tmem_ld32(t_lane + G::COL_O + q4 * 32, v);
+        float o[32];
+#pragma unroll
+        for (int q = 0; q < 32; ++q) {
+          o[q] = __uint_as_float(v[q]) * w_me;
+          if (DUAL) o[q] += __shfl_xor_sync(0xffffffffu, __uint_as_float(v[q]), 16) * w_other;
+        }
+        if (q4 == HD / 32 - 1) {                            // every column has been read: O may be overwritten
+          tc_fence_before();
+          mbar_arrive(smem_u32(o_free));
+        }
+        // the two lanes of a row share the stores: even chunks from the first tile's lane
+        if (r < M && (!DUAL || ((q4 & 1) == tile))) {
+#pragma unroll
+          for (int q = 0; q < 8; ++q) po[q4 * 8 + q] = make_float4(o[4 * q], o[4 * q + 1], o[4 * q + 2], o[4 * q + 3]);
+        }
+      }
+      if (r < M && tile == 0) {
+        float* ml = p.part_ml + rowi * 4;
+        ml[0] = m_out * rsqrtf(static_cast<float>(HD));      // natural-log units of the scaled score
+        ml[1] = l_run;
+        ml[2] = lc_run;
+      }
+      g += n_it;
+    }
+  }
+
+  // ---------------------------------------------------- teardown
+  if (flags) atomicOr(p.status, flags);
+  tc_fence_before();
+  __syncthreads();
+  if (*abort_flag) {
+    for (int i = 0; i < 64; ++i) __nanosleep(1000);
+    __syncthreads();
+  }
+  if (warp == 5) {
+    __syncwarp();
+    tc_fence_after();
+    tmem_dealloc(tmem_base, G::TMEM_COLS);
+  }
+}
+
 // Work order for grids several waves deep: every (sequence, part) that exists, longest first, so the
 // last wave is made of short parts instead of whichever sequences come last (a counting sort by
 // iteration count in one block; the order inside a bucket is arbitrary and affects no result).
@@ -495,8 +958,9 @@ template <bool DUAL>
 __global__ void k_attn_tc_combine(const float* __restrict__ part_o, const float* __restrict__ part_ml,
                                   const int* __restrict__ committed_len, int S, int W, int rep, int n_kv,
                                   int max_pages, int split_len, int max_parts, __nv_bfloat16* __restrict__ out,
-                                  float* __restrict__ tap, float* __restrict__ mass) {
+                                  float* __restrict__ tap, float* __restrict__ mass, int* __restrict__ work_counter) {
   cod_pdl_prologue();
+  if (work_counter != nullptr && blockIdx.x == 0 && threadIdx.x == 0) *work_counter = 0;   // for the next persistent attention launch
   const int lane = threadIdx.x & 31;
   const int item = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
   const int n_q = n_kv * rep;
@@ -602,14 +1066,42 @@ int launch(cod_ctx* c, int layer, const void* q, const void* kb, const void* vb,
       c->attn_order_stale = false;
     }
     p.order = c->attn_order;
+    p.n_list = S * c->tc_max_parts;
+    p.work_counter = c->attn_counter;
     grid = dim3(f.n_kv_heads, S * c->tc_max_parts, 1);
+    // the persistent form: two CTAs per SM walk the list (query rows must fill whole boxes: M = W * rep)
+    CUtensorMap mq;
+    // (measured: with 128 query rows per head group - block 32 - the persistent form is 7 % faster at 4 x 32K keys;
+    // with 64 rows the two interleaved tiles already keep HBM at what it gives this access pattern, ~6 TB/s, and
+    // the one-item CTAs of the hardware scheduler come out 6 % ahead at batch 32, so they stay)
+    if ((!DUAL || c->attn_persistent) && !c->attn_one_item_ctas &&
+        make_map_q(&mq, q, static_cast<uint64_t>(f.max_batch) * f.block, p.rep, f.n_kv_heads, f.block)) {
+      static bool configured_ps[64] = {};
+      if (!configured_ps[c->device & 63]) {
+        cudaFuncAttributes fa;
+        if (cudaFuncGetAttributes(&fa, k_attn_ps<DUAL>) != cudaSuccess) return COD_ERR_CUDA;
+        if (fa.numRegs < PS_REGS_LAUNCH) return COD_ERR_UNSUPPORTED;   // the CTA's register pool would be smaller than the budgets assume
+        if (cudaFuncSetAttribute(k_attn_ps<DUAL>, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(G::SMEM)) != cudaSuccess)
+          return COD_ERR_CUDA;
+        configured_ps[c->device & 63] = true;
+      }
+      const long long work = static_cast<long long>(S) * c->tc_max_parts * f.n_kv_heads;
+      const int groups = 2 * c->n_sm / f.n_kv_heads > 0 ? 2 * c->n_sm / f.n_kv_heads : 1;          // head groups resident at once
+      const int ctas = static_cast<int>(work / f.n_kv_heads < groups ? work : static_cast<long long>(groups) * f.n_kv_heads);
+      cod_launch_pdl(c, k_attn_ps<DUAL>, dim3(ctas, 1, 1), NTHREADS_PS, G::SMEM, st, mp, mz, mq, p);
+      COD_CHECK_LAUNCH(c);
+    } else {
+      cod_launch_pdl(c, k_attn_tc<DUAL>, grid, NTHREADS, G::SMEM, st, mp, mz, p);
+      COD_CHECK_LAUNCH(c);
+    }
+  } else {
+    cod_launch_pdl(c, k_attn_tc<DUAL>, grid, NTHREADS, G::SMEM, st, mp, mz, p);
+    COD_CHECK_LAUNCH(c);
   }
-  cod_launch_pdl(c, k_attn_tc<DUAL>, grid, NTHREADS, G::SMEM, st, mp, mz, p);
-  COD_CHECK_LAUNCH(c);
   const int items = S * f.block * f.n_q_heads;
   cod_launch_pdl(c, k_attn_tc_combine<DUAL>, (items + 3) / 4, 128, 0, st, c->attn_o, c->attn_ml, stt->committed_len, S, f.block, p.rep,
                                                            f.n_kv_heads, f.max_pages_per_seq, c->tc_split_len,
-                                                           c->tc_max_parts, static_cast<__nv_bfloat16*>(out), tap, mass);
+                                                           c->tc_max_parts, static_cast<__nv_bfloat16*>(out), tap, mass, c->attn_counter);
   COD_CHECK_LAUNCH(c);
   return COD_OK;
 }

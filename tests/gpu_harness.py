@@ -21,7 +21,7 @@ class Pair:
     """One workload instantiated on both sides with identical weights, layout and pool."""
 
     def __init__(self, wl: synth.Workload, seed: int, attn_split_len: int = 0, wo_scale: float = 1.0,
-                 fill_pool: bool = True, max_batch: int | None = None, poison: bool = False):
+                 fill_pool: bool = True, max_batch: int | None = None, poison: bool = False, extra_flags: int = 0):
         self.wl, self.seed = wl, seed
         sh = wl.shape
         self.cfg_o = oracle_config(sh)
@@ -34,7 +34,7 @@ class Pair:
         self.w_host = w
         self.w_o = orc.prepare_weights(w)
         self.st_o = orc.OracleState(self.cfg_o, wl.S, n_pages, lay["block_table"], lay["committed_len"])
-        self.cfg_g = B.make_config(sh, max_batch or wl.S, mp, n_pages, attn_split_len)
+        self.cfg_g = B.make_config(sh, max_batch or wl.S, mp, n_pages, attn_split_len, extra_flags=extra_flags)
         self.ctx = B.Context(self.cfg_g)
         self.w_g = B.weights_to_device(w, sh.dtype)
         self.ctx.set_weights(self.w_g)

@@ -120,6 +120,8 @@ def _workloads():
         # enough (sequence, head, part) CTAs for the attention kernel's longest-first work list (more than two
         # waves of the machine at 128 keys per part), with empty, one-page and ragged contexts among them
         "order_bf16": small_bf16(S=48, W=16, n_layers=2, ctx=(0, 900), d_model=1024, n_q=8, n_kv=2, vocab=1500),
+        # the same with block 32 (128 query rows per head group): there the work list is walked by PERSISTENT CTAs
+        "order_bf16_W32": small_bf16(S=40, W=32, n_layers=2, ctx=(0, 900), d_model=1024, n_q=8, n_kv=2, vocab=1500),
         "mid_bf16_full": small_bf16(S=34, W=16, n_layers=2, ctx=(100, 600), d_target=512, n_cap=5, d_model=1024,
                                     n_q=8, n_kv=2, vocab=3000, d_ff=1536, qk_norm=True),
     }
@@ -210,14 +212,17 @@ def _set_carry(P, rng, lens):
     P.st_g.carry_len.copy_(torch.tensor(lens, dtype=torch.int32))
 
 
-@pytest.mark.parametrize("name,split_len", [("tiny_f32", 32), ("tiny_f32", 0), ("small_bf16", 64),
-                                            ("small_bf16_W32", 32), ("small_bf16_W8", 0), ("long_bf16", 1024),
-                                            ("long_bf16", 256), ("long_bf16_W32", 512), ("mid_bf16", 0), ("order_bf16", 128)])
-def test_block_attn_parity(name, split_len):
+@pytest.mark.parametrize("name,split_len,flags", [
+    ("tiny_f32", 32, 0), ("tiny_f32", 0, 0), ("small_bf16", 64, 0), ("small_bf16_W32", 32, 0), ("small_bf16_W8", 0, 0),
+    ("long_bf16", 1024, 0), ("long_bf16", 256, 0), ("long_bf16_W32", 512, 0), ("mid_bf16", 0, 0), ("order_bf16", 128, 0),
+    # the work list walked by persistent CTAs: block 32 by default, block 16 when forced; and block 32 forced back
+    # to one CTA per item
+    ("order_bf16_W32", 128, 0), ("order_bf16", 128, 64), ("order_bf16_W32", 256, 32)])
+def test_block_attn_parity(name, split_len, flags):
     B, Hn = _B(), _H()
     wl = _workloads()[name]
     sh = wl.shape
-    P = Hn.Pair(wl, seed=4, attn_split_len=split_len, poison=True)
+    P = Hn.Pair(wl, seed=4, attn_split_len=split_len, poison=True, extra_flags=flags)
     rng = np.random.default_rng(11)
     tol = Hn.TOL[sh.dtype]
     out = torch.zeros((wl.S, sh.W, sh.n_q, sh.hd), dtype=B.torch_dtype(sh.dtype), device="cuda")
@@ -232,7 +237,7 @@ def test_block_attn_parity(name, split_len):
                 P.ctx.block_attn(layer, B.to_device(q, sh.dtype), B.to_device(kb, sh.dtype), B.to_device(vb, sh.dtype),
                                  P.st_g, wl.S, use_carry, out, mass)
                 torch.cuda.synchronize()
-                if name == "order_bf16":                 # tables, rotation, work list, attention, merge
+                if name.startswith("order_bf16"):        # tables, rotation, work list, attention, merge
                     assert P.ctx.launch_count() - n0 == 5
                 elif name == "small_bf16":               # a grid that fits the machine at once runs without the work list
                     assert P.ctx.launch_count() - n0 == 4
@@ -351,7 +356,7 @@ def test_round_parity_cfg1_every_round():
     ("tiny_f32_full", 40.0, orc.MODE_CARRY), ("tiny_f32_full", 40.0, orc.MODE_BASELINE),
     ("small_bf16_full", 30.0, orc.MODE_CARRY), ("small_bf16_full", 30.0, orc.MODE_BASELINE),
     ("small_bf16_mlp_only", 30.0, orc.MODE_CARRY), ("small_bf16_qknorm_only", 30.0, orc.MODE_CARRY),
-    ("mid_bf16_full", 30.0, orc.MODE_CARRY), ("order_bf16", 30.0, orc.MODE_CARRY),
+    ("mid_bf16_full", 30.0, orc.MODE_CARRY), ("order_bf16", 30.0, orc.MODE_CARRY), ("order_bf16_W32", 30.0, orc.MODE_CARRY),
     ("small_bf16_nomark", 30.0, orc.MODE_CARRY), ("small_bf16_proj", 30.0, orc.MODE_CARRY),
     ("small_bf16_proj", 30.0, orc.MODE_BASELINE), ("tiny_f32_proj", 40.0, orc.MODE_CARRY),
     ("mid_bf16_proj", 30.0, orc.MODE_CARRY), ("mid_bf16_proj", 30.0, orc.MODE_BASELINE),
