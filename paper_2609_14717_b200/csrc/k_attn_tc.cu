@@ -49,6 +49,34 @@ struct AttnParams {
 };
 
 
+// One query row's 64 scores -> probabilities exp2(s * sl2 + neg), stored as bf16 into the row of the P tile
+// (16-byte chunks XOR-swizzled by the row) and summed. TAIL: also the mass on the carried keys [car0, car0 + c)
+// (only tail tiles hold carried keys; the common tile carries none of that bookkeeping).
+template <bool TAIL>
+__device__ __forceinline__ void softmax_store(const float (&sc)[64], float sl2, float neg, uint8_t* prow, int r, int car0,
+                                              int c, float& psum, float& pcar) {
+  float ps4[4] = {0.f, 0.f, 0.f, 0.f};
+  pcar = 0.f;
+#pragma unroll
+  for (int ch = 0; ch < 8; ++ch) {
+    uint32_t packed[4];
+#pragma unroll
+    for (int e = 0; e < 4; ++e) {
+      const int j = ch * 8 + e * 2;
+      const float p0 = tc::ex2_approx(fmaf(sc[j], sl2, neg)), p1 = tc::ex2_approx(fmaf(sc[j + 1], sl2, neg));
+      ps4[e] += p0 + p1;
+      if (TAIL) {
+        if (j >= car0 && j < car0 + c) pcar += p0;
+        if (j + 1 >= car0 && j + 1 < car0 + c) pcar += p1;
+      }
+      const __nv_bfloat162 b = __floats2bfloat162_rn(p0, p1);
+      packed[e] = *reinterpret_cast<const uint32_t*>(&b);
+    }
+    *reinterpret_cast<uint4*>(prow + ((ch ^ (r & 7)) << 4)) = make_uint4(packed[0], packed[1], packed[2], packed[3]);
+  }
+  psum = (ps4[0] + ps4[1]) + (ps4[2] + ps4[3]);
+}
+
 template <bool DUAL>
 struct Geo {
   static constexpr int TILES = DUAL ? 2 : 1;             // 64-key tiles per iteration
@@ -363,30 +391,15 @@ k_attn_tc(const __grid_constant__ CUtensorMap map_pool, const __grid_constant__ 
         if (!ok) break;
       }
       const float neg = m_ref == -INFINITY ? 0.f : -m_ref * sl2;
-      float ps4[4] = {0.f, 0.f, 0.f, 0.f}, pcar = 0.f;
+      float psum, pcar;
       uint8_t* prow = sm + G::OFF_P + tile * G::P_TILE + r * 128;
       const int car0 = is_tail ? Lr - (it * G::KEYS_IT + tile * KT) : KT;  // carried keys: [car0, car0 + c)
-#pragma unroll
-      for (int ch = 0; ch < 8; ++ch) {
-        uint32_t packed[4];
-#pragma unroll
-        for (int e = 0; e < 4; ++e) {
-          const int j = ch * 8 + e * 2;
-          const float p0 = ex2_approx(fmaf(sc[j], sl2, neg)), p1 = ex2_approx(fmaf(sc[j + 1], sl2, neg));
-          ps4[e] += p0 + p1;
-          if (is_tail) {
-            if (j >= car0 && j < car0 + c) pcar += p0;
-            if (j + 1 >= car0 && j + 1 < car0 + c) pcar += p1;
-          }
-          const __nv_bfloat162 b = __floats2bfloat162_rn(p0, p1);
-          packed[e] = *reinterpret_cast<const uint32_t*>(&b);
-        }
-        *reinterpret_cast<uint4*>(prow + ((ch ^ (r & 7)) << 4)) = make_uint4(packed[0], packed[1], packed[2], packed[3]);
-      }
+      if (is_tail) softmax_store<true>(sc, sl2, neg, prow, r, car0, c, psum, pcar);
+      else softmax_store<false>(sc, sl2, neg, prow, r, car0, c, psum, pcar);
       fence_async_smem();
       tc_fence_before();
       mbar_arrive(smem_u32(p_full + (it & 1)));
-      l_run += (ps4[0] + ps4[1]) + (ps4[2] + ps4[3]);
+      l_run += psum;
       lc_run += pcar;
     }
 
@@ -820,30 +833,15 @@ k_attn_ps(const __grid_constant__ CUtensorMap map_pool, const __grid_constant__ 
           if (!ok) break;
         }
         const float neg = m_ref == -INFINITY ? 0.f : -m_ref * sl2;
-        float ps4[4] = {0.f, 0.f, 0.f, 0.f}, pcar = 0.f;
+        float psum, pcar;
         uint8_t* prow = sm + G::OFF_P + tile * G::P_TILE + r * 128;
         const int car0 = is_tail ? Lr - (it * G::KEYS_IT + tile * KT) : KT;  // carried keys: [car0, car0 + c)
-#pragma unroll
-        for (int ch = 0; ch < 8; ++ch) {
-          uint32_t packed[4];
-#pragma unroll
-          for (int e = 0; e < 4; ++e) {
-            const int q = ch * 8 + e * 2;
-            const float p0 = ex2_approx(fmaf(sc[q], sl2, neg)), p1 = ex2_approx(fmaf(sc[q + 1], sl2, neg));
-            ps4[e] += p0 + p1;
-            if (is_tail) {
-              if (q >= car0 && q < car0 + c) pcar += p0;
-              if (q + 1 >= car0 && q + 1 < car0 + c) pcar += p1;
-            }
-            const __nv_bfloat162 b = __floats2bfloat162_rn(p0, p1);
-            packed[e] = *reinterpret_cast<const uint32_t*>(&b);
-          }
-          *reinterpret_cast<uint4*>(prow + ((ch ^ (r & 7)) << 4)) = make_uint4(packed[0], packed[1], packed[2], packed[3]);
-        }
+        if (is_tail) softmax_store<true>(sc, sl2, neg, prow, r, car0, c, psum, pcar);
+        else softmax_store<false>(sc, sl2, neg, prow, r, car0, c, psum, pcar);
         fence_async_smem();
         tc_fence_before();
         mbar_arrive(smem_u32(p_full + (gg & 1)));
-        l_run += (ps4[0] + ps4[1]) + (ps4[2] + ps4[3]);
+        l_run += psum;
         lc_run += pcar;
       }
       if (!ok) break;
