@@ -377,6 +377,7 @@ def measure_workload(name, args, rank, world, local, peaks, with_cpu):
         buf, (vh, vd, vt) = _packed((H_pin[i], d_pin[i], t_pin[i]), "cpu", True)
         vh.copy_(H_pin[i]); vd.copy_(d_pin[i]); vt.copy_(t_pin[i])
         pin_bufs.append(buf)
+    stage_buf.copy_(pin_bufs[0])                            # the staged graph's warm-up launch reads it
     next_draft = torch.zeros((wl.S, sh.W), dtype=torch.int32, device="cuda")
     out_pin = torch.zeros((wl.S, sh.W), dtype=torch.int32).pin_memory()
     L0 = state.committed_len.clone()
