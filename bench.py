@@ -344,7 +344,7 @@ def measure_workload(name, args, rank, world, local, peaks, with_cpu):
     weights = synth.make_weights(sh, seed)
     lay = synth.make_layout(wl, seed)
     n_pages, mp = int(lay["n_pages"]), int(lay["max_pages_per_seq"])
-    cfg = B.make_config(sh, wl.S, mp, n_pages, attn_split_len=args.attn_split)
+    cfg = B.make_config(sh, wl.S, mp, n_pages, attn_split_len=args.attn_split, extra_flags=args.flags)
     ctx = B.Context(cfg)
     w_dev = B.weights_to_device(weights, sh.dtype)
     ctx.set_weights(w_dev)
@@ -642,7 +642,7 @@ def run_micro_round(args):
     wl = synth.scaled(bench_workload(args.workload, K + Wm + 2), n_layers=1)
     sh = wl.shape
     lay = synth.make_layout(wl, args.seed)
-    cfg = B.make_config(sh, wl.S, int(lay["max_pages_per_seq"]), int(lay["n_pages"]), attn_split_len=args.attn_split)
+    cfg = B.make_config(sh, wl.S, int(lay["max_pages_per_seq"]), int(lay["n_pages"]), attn_split_len=args.attn_split, extra_flags=args.flags)
     ctx = B.Context(cfg)
     td = B.torch_dtype(sh.dtype)
     gen = torch.Generator(device="cuda").manual_seed(args.seed)
@@ -693,7 +693,7 @@ def run_timeline(args):
     wl = bench_workload(args.workload, 40)
     sh = wl.shape
     lay = synth.make_layout(wl, args.seed)
-    cfg = B.make_config(sh, wl.S, int(lay["max_pages_per_seq"]), int(lay["n_pages"]), attn_split_len=args.attn_split)
+    cfg = B.make_config(sh, wl.S, int(lay["max_pages_per_seq"]), int(lay["n_pages"]), attn_split_len=args.attn_split, extra_flags=args.flags)
     ctx = B.Context(cfg)
     td = B.torch_dtype(sh.dtype)
     gen = torch.Generator(device="cuda").manual_seed(args.seed)
@@ -765,7 +765,7 @@ def run_micro(args):
     sh = wl.shape
     lay = synth.make_layout(wl, args.seed)
     n_pages, mp = int(lay["n_pages"]), int(lay["max_pages_per_seq"])
-    cfg = B.make_config(sh, wl.S, mp, n_pages, attn_split_len=args.attn_split)
+    cfg = B.make_config(sh, wl.S, mp, n_pages, attn_split_len=args.attn_split, extra_flags=args.flags)
     ctx = B.Context(cfg)
     td = B.torch_dtype(sh.dtype)
     gen = torch.Generator(device="cuda").manual_seed(args.seed)
@@ -909,6 +909,8 @@ def main():
     ap.add_argument("--sweep", action="store_true", help="carryover-overhead sweep over batch, block and rejected fraction")
     ap.add_argument("--sweep-reps", type=int, default=7, help="--sweep: interleaved passes per mode and point")
     ap.add_argument("--attn-split", type=int, default=0, help="keys per attention split (0 = library default)")
+    ap.add_argument("--flags", type=int, default=0,
+                    help="extra cod_config flags OR-ed in (e.g. 64 = persistent attention, 32 = one-item attention CTAs)")
     ap.add_argument("--micro", default=None, choices=["attn", "lmhead", "lmsample", "lmrank", "gemm", "timeline"],
                     help="time one entry point alone (small footprint; meant for profiler captures)")
     ap.add_argument("--shape", default=None, choices=["fc", "kv", "qkv", "oproj", "lmhead", "attn"],

@@ -49,6 +49,27 @@ struct AttnParams {
 };
 
 
+// L2 eviction hints. The K/V stream is read once per call: marked evict-first it does not push out what the call
+// itself will read again (the partial results written below, marked evict-last, which the merge kernel reads).
+__device__ __forceinline__ uint64_t l2_policy_evict_first() {
+  uint64_t pol;
+  asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(pol));
+  return pol;
+}
+__device__ __forceinline__ uint64_t l2_policy_evict_last() {
+  uint64_t pol;
+  asm volatile("createpolicy.fractional.L2::evict_last.b64 %0, 1.0;" : "=l"(pol));
+  return pol;
+}
+__device__ __forceinline__ void tma_load_3d_hint(uint32_t dst, const CUtensorMap* map, int c0, int c1, int c2, uint32_t bar, uint64_t pol) {
+  asm volatile(
+      "cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint [%0], [%1, {%2, %3, %4}], [%5], %6;"
+      ::"r"(dst), "l"(reinterpret_cast<uint64_t>(map)), "r"(c0), "r"(c1), "r"(c2), "r"(bar), "l"(pol) : "memory");
+}
+__device__ __forceinline__ void st_float4_hint(float4* ptr, float a, float b, float c, float d, uint64_t pol) {
+  asm volatile("st.global.L2::cache_hint.v4.f32 [%0], {%1, %2, %3, %4}, %5;" ::"l"(ptr), "f"(a), "f"(b), "f"(c), "f"(d), "l"(pol) : "memory");
+}
+
 // One query row's 64 scores -> probabilities exp2(s * sl2 + neg), stored as bf16 into the row of the P tile
 // (16-byte chunks XOR-swizzled by the row) and summed. TAIL: also the mass on the carried keys [car0, car0 + c)
 // (only tail tiles hold carried keys; the common tile carries none of that bookkeeping).
@@ -199,6 +220,7 @@ k_attn_tc(const __grid_constant__ CUtensorMap map_pool, const __grid_constant__ 
       uint64_t* full = is_v ? v_full : k_full;
       uint64_t* empty = is_v ? v_empty : k_empty;
       const uint32_t ring_off = is_v ? G::OFF_V : G::OFF_K;
+      const uint64_t pol_stream = l2_policy_evict_first();
       bool ok = true;
       for (int it = 0; it < n_it && ok; ++it) {
         const int key0 = k_begin + it * G::KEYS_IT + lane * PAGE;
@@ -218,8 +240,8 @@ k_attn_tc(const __grid_constant__ CUtensorMap map_pool, const __grid_constant__ 
         if (lane < pages_it) {
           const uint32_t dst = base + ring_off + slot * G::SLOT + in_slot;
           if (row >= 0) {
-            tma_load_3d(dst, &map_pool, 0, 0, row, fb);
-            tma_load_3d(dst + HALF_BYTES, &map_pool, 0, 1, row, fb);
+            tma_load_3d_hint(dst, &map_pool, 0, 0, row, fb, pol_stream);
+            tma_load_3d_hint(dst + HALF_BYTES, &map_pool, 0, 1, row, fb, pol_stream);
           } else {
             tma_load_3d(dst, &map_zero, 0, 0, 0, fb);
             tma_load_3d(dst + HALF_BYTES, &map_zero, 0, 1, 0, fb);
@@ -424,6 +446,7 @@ k_attn_tc(const __grid_constant__ CUtensorMap map_pool, const __grid_constant__ 
         }
         const size_t rowi = ((static_cast<size_t>(s) * p.n_kv + h) * p.max_parts + split) * M + min(r, M - 1);
         float4* po = reinterpret_cast<float4*>(p.part_o + rowi * HD);
+      const uint64_t pol_keep = l2_policy_evict_last();
 #pragma unroll
         for (int q4 = 0; q4 < HD / 32; ++q4) {
           uint32_t v[32];
@@ -437,7 +460,7 @@ k_attn_tc(const __grid_constant__ CUtensorMap map_pool, const __grid_constant__ 
           // the two lanes of a row share the stores: even chunks from the first tile's lane
           if (r < M && (!DUAL || ((q4 & 1) == tile))) {
 #pragma unroll
-            for (int j = 0; j < 8; ++j) po[q4 * 8 + j] = make_float4(o[4 * j], o[4 * j + 1], o[4 * j + 2], o[4 * j + 3]);
+            for (int j = 0; j < 8; ++j) st_float4_hint(po + q4 * 8 + j, o[4 * j], o[4 * j + 1], o[4 * j + 2], o[4 * j + 3], pol_keep);
           }
         }
         if (r < M && tile == 0) {
@@ -588,6 +611,7 @@ k_attn_ps(const __grid_constant__ CUtensorMap map_pool, const __grid_constant__ 
     uint64_t* empty = is_v ? v_empty : k_empty;
     const uint32_t ring_off = is_v ? G::OFF_V : G::OFF_K;
     const bool lane_on = lane < pages_it;
+    const uint64_t pol_stream = l2_policy_evict_first();
     const uint32_t in_slot = (lane / (KT / PAGE)) * TILE_BYTES + (lane % (KT / PAGE)) * (PAGE * 128);
     int g = 0, j = 0;
     bool ok = true;
@@ -633,8 +657,8 @@ k_attn_ps(const __grid_constant__ CUtensorMap map_pool, const __grid_constant__ 
           if (lane_on) {
             const uint32_t dst = base + ring_off + slot * G::SLOT + in_slot;
             if (row >= 0) {
-              tma_load_3d(dst, &map_pool, 0, 0, row, fb);
-              tma_load_3d(dst + HALF_BYTES, &map_pool, 0, 1, row, fb);
+              tma_load_3d_hint(dst, &map_pool, 0, 0, row, fb, pol_stream);
+              tma_load_3d_hint(dst + HALF_BYTES, &map_pool, 0, 1, row, fb, pol_stream);
             } else {
               tma_load_3d(dst, &map_zero, 0, 0, 0, fb);
               tma_load_3d(dst + HALF_BYTES, &map_zero, 0, 1, 0, fb);
@@ -866,6 +890,7 @@ k_attn_ps(const __grid_constant__ CUtensorMap map_pool, const __grid_constant__ 
       }
       const size_t rowi = ((static_cast<size_t>(s) * p.n_kv + h) * p.max_parts + split) * M + min(r, M - 1);
       float4* po = reinterpret_cast<float4*>(p.part_o + rowi * HD);
+      const uint64_t pol_keep = l2_policy_evict_last();
 #pragma unroll
       for (int q4 = 0; q4 < HD / 32; ++q4) {
         uint32_t v[32];
@@ -883,7 +908,7 @@ k_attn_ps(const __grid_constant__ CUtensorMap map_pool, const __grid_constant__ 
         // the two lanes of a row share the stores: even chunks from the first tile's lane
         if (r < M && (!DUAL || ((q4 & 1) == tile))) {
 #pragma unroll
-          for (int q = 0; q < 8; ++q) po[q4 * 8 + q] = make_float4(o[4 * q], o[4 * q + 1], o[4 * q + 2], o[4 * q + 3]);
+          for (int q = 0; q < 8; ++q) st_float4_hint(po + q4 * 8 + q, o[4 * q], o[4 * q + 1], o[4 * q + 2], o[4 * q + 3], pol_keep);
         }
       }
       if (r < M && tile == 0) {
