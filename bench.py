@@ -639,7 +639,9 @@ def run_micro_round(args):
     torch.cuda.set_device(0)
     peaks = load_peaks()
     K, Wm = args.steps, args.warmup
-    wl = synth.scaled(bench_workload(args.workload, K + Wm + 2), n_layers=1)
+    wl = bench_workload(args.workload, K + Wm + 2)
+    if args.layers > 0:
+        wl = synth.scaled(wl, n_layers=args.layers)
     sh = wl.shape
     lay = synth.make_layout(wl, args.seed)
     cfg = B.make_config(sh, wl.S, int(lay["max_pages_per_seq"]), int(lay["n_pages"]), attn_split_len=args.attn_split, extra_flags=args.flags)
@@ -909,6 +911,8 @@ def main():
     ap.add_argument("--sweep", action="store_true", help="carryover-overhead sweep over batch, block and rejected fraction")
     ap.add_argument("--sweep-reps", type=int, default=7, help="--sweep: interleaved passes per mode and point")
     ap.add_argument("--attn-split", type=int, default=0, help="keys per attention split (0 = library default)")
+    ap.add_argument("--layers", type=int, default=1,
+                    help="--micro gemm: drafter layers of the rounds it runs (default 1; 0 = the workload's own depth)")
     ap.add_argument("--flags", type=int, default=0,
                     help="extra cod_config flags OR-ed in (e.g. 64 = persistent attention, 32 = one-item attention CTAs)")
     ap.add_argument("--micro", default=None, choices=["attn", "lmhead", "lmsample", "lmrank", "gemm", "timeline"],

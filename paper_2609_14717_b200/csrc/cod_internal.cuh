@@ -28,6 +28,13 @@ __device__ __forceinline__ void cod_pdl_prologue() {
   if (gridDim.x * gridDim.y * gridDim.z <= 1024u) asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
 }
 
+// Drops one 128-byte line (address aligned to 128 bytes) from L2 without writing it back: for scratch data that
+// has been read for the last time. Whatever is read there before the next write is indeterminate, and the caller
+// orders the drop after every read of the line (the readers synchronise with the dropping thread first).
+__device__ __forceinline__ void cod_discard_line(const void* p) {
+  asm volatile("discard.global.L2 [%0], 128;" ::"l"(p) : "memory");
+}
+
 // ---------------------------------------------------------------------------- element access
 __device__ __forceinline__ float cod_ld(const float* p) { return *p; }
 __device__ __forceinline__ float cod_ld(const __nv_bfloat16* p) { return __bfloat162float(*p); }

@@ -1041,6 +1041,11 @@ __global__ void k_attn_tc_combine(const float* __restrict__ part_o, const float*
   }
   l = cod_warp_sum(l);
   lc = cod_warp_sum(lc);
+  // this warp was the only reader of its partial rows (512 bytes each): they are dead now and leave L2 without a
+  // write-back (the warp barrier orders every lane's reads before the drop)
+  __syncwarp();
+  for (int k = lane >> 2; k < n_parts; k += 8)          // lane 4 k + q drops line q of part k
+    cod_discard_line(part_o + ((base + k) * M + mrow) * HD + (lane & 3) * 32);
   const float inv = 1.f / l;
   const size_t ob = static_cast<size_t>(item) * HD + lane * 4;
   const __nv_bfloat162 b0 = __floats2bfloat162_rn(acc[0] * inv, acc[1] * inv), b1 = __floats2bfloat162_rn(acc[2] * inv, acc[3] * inv);

@@ -21,6 +21,15 @@
 #include "tc_common.cuh"
 
 namespace {
+// A weight tile is read once per launch: fetched with an L2 evict-first hint it leaves the cache before the token
+// operand every pair re-reads and before the float partial sums the finishing kernel is about to read.
+__device__ __forceinline__ void tma_load_2d_pair_stream(uint32_t dst, const CUtensorMap* map, int c0, int c1, uint32_t leader_bar) {
+  uint64_t pol;
+  asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(pol));
+  asm volatile(
+      "cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint [%0], [%1, {%2, %3}], [%4], %5;"
+      ::"r"(dst), "l"(reinterpret_cast<uint64_t>(map)), "r"(c0), "r"(c1), "r"(leader_bar), "l"(pol) : "memory");
+}
 
 using namespace tc;
 
@@ -109,7 +118,7 @@ k_gemm_tc2(const __grid_constant__ CUtensorMap map_w0, const __grid_constant__ C
   const uint32_t tmem_base = *tmem_slot;
   if (warp == 4 && lane == 0)
     for (int it = 0; it < n_pre; ++it)
-      tma_load_2d_pair(base + it * STAGE_BYTES, map_w, (kb0 + it) * BK, f0, smem_u32(full_bar + it) & PEER_MASK);
+      tma_load_2d_pair_stream(base + it * STAGE_BYTES, map_w, (kb0 + it) * BK, f0, smem_u32(full_bar + it) & PEER_MASK);
 
   cod_pdl_prologue();
   const int n_rows = p.n_rows_dev ? min(*p.n_rows_dev, p.n_rows) : p.n_rows;
@@ -143,7 +152,7 @@ k_gemm_tc2(const __grid_constant__ CUtensorMap map_w0, const __grid_constant__ C
         if (rank == 0) mbar_expect_tx(fb, stage_tx);            // both CTAs' bytes land on the leader's barrier
         const uint32_t a_dst = base + s * STAGE_BYTES;
         const int k = (kb0 + it) * BK;
-        if (it >= n_pre) tma_load_2d_pair(a_dst, map_w, k, f0, fb & PEER_MASK);
+        if (it >= n_pre) tma_load_2d_pair_stream(a_dst, map_w, k, f0, fb & PEER_MASK);
         for (int a = 0; a < p.n_acc; ++a)      // accumulator a covers tokens [i0 + a*256, +256): this CTA stages its half
           if (acc_on & (1u << a)) tma_load_2d_pair(a_dst + A_TILE_BYTES + a * B_TILE_BYTES, &map_a, k, i0 + a * NT + rank * (NT / 2), fb & PEER_MASK);
       }

@@ -122,6 +122,15 @@ __global__ void __launch_bounds__(1024) k_fc_finish(const float* __restrict__ pa
 #pragma unroll
   for (int t = 0; t < NV; ++t) ss += f4_ss(v[t]);
   ss = cod_block_sum(ss, red);
+  // the partial sums are dead: their lines leave L2 without a write-back (the block has met since their last read)
+  if ((D & 31) == 0 && (ldp & 31) == 0) {
+#pragma unroll
+    for (int t = 0; t < NV; ++t) {
+      const int j = threadIdx.x + t * blockDim.x;
+      if (j < nv)
+        for (int s = j & 7; s < splits; s += 8) cod_discard_line(prow + static_cast<size_t>(s) * n_rows * ldp + 4 * (j & ~7));
+    }
+  }
   const float scale = do_norm ? rsqrtf(ss / static_cast<float>(D) + eps) : 1.f;
 #pragma unroll
   for (int t = 0; t < NV; ++t) {
@@ -200,6 +209,13 @@ __global__ void k_kv_finish(const float* __restrict__ part, int splits, int n_ro
         v1 = f4_add(v1, *reinterpret_cast<const float4*>(p + s * slab + Ld * kvw));
         v2 = f4_add(v2, *reinterpret_cast<const float4*>(p + s * slab + Ld * kvw + half));
       }
+    }
+    if ((half & 31) == 0) {          // the partial sums are dead: dropped from L2, no write-back (see k_qkv_finish)
+      __syncwarp();
+      const int g8 = threadIdx.x & 7;                // the eight lanes share the drops
+      if (live)
+        for (int idx = g8; idx < 4 * splits; idx += 8)
+          cod_discard_line(p - 4 * g8 + (idx >> 2) * slab + ((idx >> 1) & 1) * (Ld * kvw) + (idx & 1) * half);
     }
     if (g_k != nullptr) {
       const float ss = group_sum(f4_ss(k1) + f4_ss(k2), tph);
@@ -395,6 +411,15 @@ __global__ void k_qkv_finish(const float* __restrict__ part, int splits, int R, 
       b = f4_add(b, *reinterpret_cast<const float4*>(p + s * slab + half));
     }
   }
+  // The partial sums are dead once summed: the lines are dropped from L2 instead of being written back to HBM
+  // later, under some HBM-bound kernel. Eight consecutive lanes share a 128-byte line; the first of them drops it
+  // after the warp has met (all of the line's reads are then complete).
+  if ((half & 31) == 0) {
+    __syncwarp();
+    const int g8 = threadIdx.x & 7;                  // the eight lanes share the drops: line (s, half) to lane 2 s + half
+    if (live)
+      for (int idx = g8; idx < 2 * splits; idx += 8) cod_discard_line(p - 4 * g8 + (idx >> 1) * slab + (idx & 1) * half);
+  }
   const bool rot = hh < n_q + n_kv;
   const T* gain = hh < n_q ? g_q : (rot ? g_k : nullptr);
   if (g_q != nullptr) {                               // block-uniform: every lane takes the shuffles
@@ -504,6 +529,15 @@ __global__ void __launch_bounds__(1024) k_resid_norm(const float* __restrict__ p
     }
   }
   ss = cod_block_sum(ss, red);
+  // the partial sums are dead: their lines leave L2 without a write-back (the block has met since their last read)
+  if (part && (D & 31) == 0) {
+#pragma unroll
+    for (int t = 0; t < NV; ++t) {
+      const int j = threadIdx.x + t * blockDim.x;
+      if (j < nv)
+        for (int s = j & 7; s < splits; s += 8) cod_discard_line(part + (static_cast<size_t>(s) * R + r) * D + 4 * (j & ~7));
+    }
+  }
   const float scale = rsqrtf(ss / static_cast<float>(D) + eps);
 #pragma unroll
   for (int t = 0; t < NV; ++t) {
