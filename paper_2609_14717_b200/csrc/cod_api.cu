@@ -190,6 +190,7 @@ int cod_create(const cod_config* cfg, cod_ctx** out) {
   c->force_simt = (f.flags & COD_F_NO_TENSOR_CORES) != 0;
   c->attn_one_item_ctas = (f.flags & COD_F_ATTN_ONE_ITEM_CTAS) != 0;
   c->attn_persistent = (f.flags & COD_F_ATTN_PERSISTENT) != 0;
+  c->attn_run_ahead = true;
   c->carry_cap = (f.carry_rounds > 1 ? f.carry_rounds : 1) * f.block;
   if (cudaDeviceGetAttribute(&c->n_sm, cudaDevAttrMultiProcessorCount, c->device) != cudaSuccess || c->n_sm < 1) c->n_sm = 148;
   c->split_len = f.attn_split_len > 0 ? f.attn_split_len : 512;
@@ -511,8 +512,12 @@ static int round_impl(cod_ctx* c, const int32_t* draft, const int32_t* target, c
 
     float* tap_o = (taps && taps->attn_out) ? taps->attn_out + static_cast<size_t>(l) * R * c->qw : nullptr;
     float* tap_m = (taps && taps->carry_mass) ? taps->carry_mass + static_cast<size_t>(l) * R * f.n_q_heads : nullptr;
-    if ((rc = cod_launch_attn(c, l, c->q, c->kb, c->vb, st, S, mode == COD_CARRY ? 1 : 0, c->o, tap_o, tap_m, s)) != COD_OK)
-      return rc;
+    // after the join the first attention's stream predecessor is the context projection, which writes the pool,
+    // the carry slots and (through the other branch) the lengths: that launch must not run ahead of it
+    c->attn_run_ahead = !(l == 0 && fork);
+    rc = cod_launch_attn(c, l, c->q, c->kb, c->vb, st, S, mode == COD_CARRY ? 1 : 0, c->o, tap_o, tap_m, s);
+    c->attn_run_ahead = true;
+    if (rc != COD_OK) return rc;
 
     GemmArgs o{};
     o.A = c->o; o.lda = c->qw; o.n_rows = R; o.K = c->qw;

@@ -31,6 +31,9 @@ __device__ __forceinline__ void cod_pdl_prologue() {
 // Drops one 128-byte line (address aligned to 128 bytes) from L2 without writing it back: for scratch data that
 // has been read for the last time. Whatever is read there before the next write is indeterminate, and the caller
 // orders the drop after every read of the line (the readers synchronise with the dropping thread first).
+// Worth its instructions only when the scratch is large enough to be pushed out to HBM under a memory-bound kernel:
+// rounds of more token rows than this (one block per row in the kernels that use it).
+#define COD_DROP_MIN_ROWS 128
 __device__ __forceinline__ void cod_discard_line(const void* p) {
   asm volatile("discard.global.L2 [%0], 128;" ::"l"(p) : "memory");
 }
@@ -176,6 +179,7 @@ struct cod_ctx {
   long long wait_limit;        // SM cycles a bounded device wait may last (0: the built-in limit, about 2 s)
   int attn_one_item_ctas;      // 1: work-list attention as one CTA per item (the persistent form off; for A/B runs)
   int attn_persistent;         // 1: the persistent form whatever the geometry
+  bool attn_run_ahead;         // false while the next attention launch follows a kernel that writes the KV state or the lengths
   int selftest_skip_copies;    // cod_selftest_expire_wait: single-CTA contractions request no operands
   int* perm;                  // [R] window rows in the order accepted-first (grouped contraction of the separate projector)
   void* z;                     // [R_max, D]

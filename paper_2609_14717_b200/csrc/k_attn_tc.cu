@@ -43,6 +43,7 @@ struct AttnParams {
   float* part_ml;                       // [S][n_kv][max_parts][M][4]   m (natural log units), l, l_carry
   const int* order;                     // null: CTA (x, y, z) = (part, head, sequence). Else CTA (x, y) = (head, i) works
                                         // on part order[i] = sequence << 16 | part, longest first; -1: nothing
+  int run_ahead;                // the launch's stream predecessor writes only q / k_blk / v_blk (see k_attn_tc)
   int n_list;                           // entries of order[] (persistent kernel)
   int* work_counter;                    // persistent kernel: units taken beyond each CTA's first (zero before the launch)
   uint32_t* status;
@@ -122,7 +123,11 @@ struct Geo {
 template <bool DUAL>
 __global__ void __launch_bounds__(NTHREADS, 2)
 k_attn_tc(const __grid_constant__ CUtensorMap map_pool, const __grid_constant__ CUtensorMap map_zero, const AttnParams p) {
-  cod_pdl_prologue();
+  // Small grids (no work list) run ahead of the dependency: barriers, tensor memory, page ids and the paged K/V
+  // stream touch nothing the previous kernel of the stream writes (it produces q, k_blk, v_blk or the work list;
+  // everything older has completed before this grid may start), so only the warps that read those wait for it.
+  const bool early = p.order == nullptr && p.run_ahead;
+  if (!early) cod_pdl_prologue();
   using G = Geo<DUAL>;
   extern __shared__ uint8_t smem_raw[];
   const uint32_t raw = smem_u32(smem_raw);
@@ -137,6 +142,7 @@ k_attn_tc(const __grid_constant__ CUtensorMap map_pool, const __grid_constant__ 
   uint64_t* p_full = bars + 22;             // [2]
   uint64_t* o_full = bars + 24;             // [2]
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 26);
+  uint64_t* q_ready = bars + 27;            // the Q tile is in shared memory
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
   int* page_ids = reinterpret_cast<int*>(bars + 28);       // [split_len / 16] <= 256 entries
 
@@ -168,14 +174,28 @@ k_attn_tc(const __grid_constant__ CUtensorMap map_pool, const __grid_constant__ 
     for (int i = 0; i < G::NK; ++i) { mbar_init(smem_u32(k_full + i), is_tail ? 128 : 1); mbar_init(smem_u32(k_empty + i), 1); }
     for (int i = 0; i < G::NV; ++i) { mbar_init(smem_u32(v_full + i), is_tail ? 128 : 1); mbar_init(smem_u32(v_empty + i), 1); }
     for (int i = 0; i < 2; ++i) { mbar_init(smem_u32(s_full + i), 1); mbar_init(smem_u32(p_full + i), 128); mbar_init(smem_u32(o_full + i), 1); }
+    mbar_init(smem_u32(q_ready), 128);
     *abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
   if (warp == 5) tmem_alloc(smem_u32(tmem_slot), G::TMEM_COLS);
+  if (warp == 4 && !is_tail) {
+    // physical page of every logical page this CTA will touch, fetched once
+    for (int i = lane; i < (k_end - k_begin + PAGE - 1) / PAGE; i += 32) {
+      int pg = p.block_table[s * p.max_pages + k_begin / PAGE + i];
+      if (pg < 0 || pg >= p.n_pages) { flags |= COD_DEV_BAD_PAGE; pg = -1; }
+      page_ids[i] = pg;
+    }
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = *tmem_slot;
 
   // Q tile: [half][row][64 elements], 128-byte rows, chunks of 16 bytes XOR-swizzled by (row & 7);
   // rows beyond the real query rows are zero.
   if (warp < 4) {
+    if (early) cod_pdl_prologue();
     const int qw = p.n_kv * p.rep * HD;
     constexpr int QB = 8;                                   // independent 16-byte loads in flight per thread
     for (int idx0 = threadIdx.x; idx0 < G::MROWS * 16; idx0 += 128 * QB) {
@@ -196,19 +216,8 @@ k_attn_tc(const __grid_constant__ CUtensorMap map_pool, const __grid_constant__ 
       }
     }
     fence_async_smem();
-  } else if (warp == 4 && !is_tail) {
-    // physical page of every logical page this CTA will touch, fetched once
-    for (int i = lane; i < (k_end - k_begin + PAGE - 1) / PAGE; i += 32) {
-      int pg = p.block_table[s * p.max_pages + k_begin / PAGE + i];
-      if (pg < 0 || pg >= p.n_pages) { flags |= COD_DEV_BAD_PAGE; pg = -1; }
-      page_ids[i] = pg;
-    }
-    __syncwarp();
+    mbar_arrive(smem_u32(q_ready));
   }
-  tc_fence_before();
-  __syncthreads();
-  tc_fence_after();
-  const uint32_t tmem_base = *tmem_slot;
 
   if (warp == 4 || warp == 6) {
     // ------------------------------------------------ TMA producers (paged region only): warp 4 streams
@@ -275,7 +284,7 @@ k_attn_tc(const __grid_constant__ CUtensorMap map_pool, const __grid_constant__ 
         umma_commit(smem_u32(k_empty + slot));
         return true;
       };
-      ok = issue_qk(0);
+      ok = mbar_wait(smem_u32(q_ready), 0, abort_flag, p.status) && issue_qk(0);
       for (int it = 0; it < n_it && ok; ++it) {
         if (it + 1 < n_it) ok = issue_qk(it + 1);
         if (!ok) break;
@@ -1044,8 +1053,9 @@ __global__ void k_attn_tc_combine(const float* __restrict__ part_o, const float*
   // this warp was the only reader of its partial rows (512 bytes each): they are dead now and leave L2 without a
   // write-back (the warp barrier orders every lane's reads before the drop)
   __syncwarp();
-  for (int k = lane >> 2; k < n_parts; k += 8)          // lane 4 k + q drops line q of part k
-    cod_discard_line(part_o + ((base + k) * M + mrow) * HD + (lane & 3) * 32);
+  if (S * W > COD_DROP_MIN_ROWS)
+    for (int k = lane >> 2; k < n_parts; k += 8)        // lane 4 k + q drops line q of part k
+      cod_discard_line(part_o + ((base + k) * M + mrow) * HD + (lane & 3) * 32);
   const float inv = 1.f / l;
   const size_t ob = static_cast<size_t>(item) * HD + lane * 4;
   const __nv_bfloat162 b0 = __floats2bfloat162_rn(acc[0] * inv, acc[1] * inv), b1 = __floats2bfloat162_rn(acc[2] * inv, acc[3] * inv);
@@ -1075,6 +1085,7 @@ int launch(cod_ctx* c, int layer, const void* q, const void* kb, const void* vb,
   p.n_pages = f.n_pages; p.max_pages = f.max_pages_per_seq; p.max_batch = f.max_batch;
   p.split_len = c->tc_split_len; p.max_parts = c->tc_max_parts;
   p.part_o = c->attn_o; p.part_ml = c->attn_ml; p.status = c->status;
+  p.run_ahead = c->attn_run_ahead ? 1 : 0;
   // the attribute belongs to (kernel, device): one flag per device the process may use
   static bool configured_dev[64] = {};
   bool& configured = configured_dev[c->device & 63];

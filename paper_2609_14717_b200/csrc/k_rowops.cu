@@ -123,7 +123,7 @@ __global__ void __launch_bounds__(1024) k_fc_finish(const float* __restrict__ pa
   for (int t = 0; t < NV; ++t) ss += f4_ss(v[t]);
   ss = cod_block_sum(ss, red);
   // the partial sums are dead: their lines leave L2 without a write-back (the block has met since their last read)
-  if ((D & 31) == 0 && (ldp & 31) == 0) {
+  if ((D & 31) == 0 && (ldp & 31) == 0 && gridDim.x > COD_DROP_MIN_ROWS) {
 #pragma unroll
     for (int t = 0; t < NV; ++t) {
       const int j = threadIdx.x + t * blockDim.x;
@@ -210,7 +210,7 @@ __global__ void k_kv_finish(const float* __restrict__ part, int splits, int n_ro
         v2 = f4_add(v2, *reinterpret_cast<const float4*>(p + s * slab + Ld * kvw + half));
       }
     }
-    if ((half & 31) == 0) {          // the partial sums are dead: dropped from L2, no write-back (see k_qkv_finish)
+    if ((half & 31) == 0 && gridDim.x > COD_DROP_MIN_ROWS) {          // the partial sums are dead: dropped from L2, no write-back (see k_qkv_finish)
       __syncwarp();
       const int g8 = threadIdx.x & 7;                // the eight lanes share the drops
       if (live)
@@ -414,7 +414,7 @@ __global__ void k_qkv_finish(const float* __restrict__ part, int splits, int R, 
   // The partial sums are dead once summed: the lines are dropped from L2 instead of being written back to HBM
   // later, under some HBM-bound kernel. Eight consecutive lanes share a 128-byte line; the first of them drops it
   // after the warp has met (all of the line's reads are then complete).
-  if ((half & 31) == 0) {
+  if ((half & 31) == 0 && gridDim.x > COD_DROP_MIN_ROWS) {
     __syncwarp();
     const int g8 = threadIdx.x & 7;                  // the eight lanes share the drops: line (s, half) to lane 2 s + half
     if (live)
@@ -530,7 +530,7 @@ __global__ void __launch_bounds__(1024) k_resid_norm(const float* __restrict__ p
   }
   ss = cod_block_sum(ss, red);
   // the partial sums are dead: their lines leave L2 without a write-back (the block has met since their last read)
-  if (part && (D & 31) == 0) {
+  if (part && (D & 31) == 0 && gridDim.x > COD_DROP_MIN_ROWS) {
 #pragma unroll
     for (int t = 0; t < NV; ++t) {
       const int j = threadIdx.x + t * blockDim.x;
