@@ -9,6 +9,7 @@
 
 #define COD_MAX_SPLITS 8          // split-K partial slabs the GEMM workspace can hold
 #define COD_MAX_W 128             // largest supported block size
+#define COD_L2_KEEP_BYTES (48ll << 20)   // weight bytes of the fc projection asked to stay in L2 between small rounds
 
 // ---------------------------------------------------------------------------- dependent launches
 // With few token rows a round is ~45 short kernels, and every kernel is launched with programmatic

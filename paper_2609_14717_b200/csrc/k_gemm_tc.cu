@@ -48,6 +48,7 @@ struct TcParams {
   uint32_t* status;
   long long wait_limit;       // SM cycles a bounded wait may last
   int skip_copies;            // self-test of the failure path: the producer requests nothing, so the waits run out
+  int pin_tiles;              // weight tiles [0, pin_tiles) of the launch are fetched evict-last (kept in L2 for the next round)
   // rank form (RANK kernels): per token row, how many weight rows score above a reference row
   const float* rank_ref;      // [n_rows] the reference row's logit
   const int32_t* rank_tok;    // [n_rows] the reference row's index (excluded from the count)
@@ -65,6 +66,19 @@ __device__ __forceinline__ bool bar_and_128(bool v) {
   return r != 0;
 }
 
+
+// Weight tiles with an L2 eviction hint: a weight is read once per launch, so its lines should leave L2 first
+// (evict-first) - except a prefix of one launch per round that fits L2 and is asked to stay (evict-last), so that
+// the next round finds it there.
+__device__ __forceinline__ void bulk_load_hint(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar, uint64_t pol) {
+  asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint [%0], [%1], %2, [%3], %4;"
+               ::"r"(dst), "l"(src), "r"(bytes), "r"(bar), "l"(pol) : "memory");
+}
+__device__ __forceinline__ void tma_load_2d_hint(uint32_t dst, const CUtensorMap* map, int c0, int c1, uint32_t bar, uint64_t pol) {
+  asm volatile(
+      "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint [%0], [%1, {%2, %3}], [%4], %5;"
+      ::"r"(dst), "l"(reinterpret_cast<uint64_t>(map)), "r"(c0), "r"(c1), "r"(bar), "l"(pol) : "memory");
+}
 
 // SAMPLE selects the sampling form of the argmax epilogue, WIDE the transposing store epilogue
 // (32 token rows and more) and RANK the counting epilogue at compile time, so the kernel a batch-1
@@ -124,10 +138,13 @@ k_gemm_tc(const __grid_constant__ CUtensorMap map_w0, const __grid_constant__ CU
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
+  uint64_t pol_w;
+  if (m_tile < p.pin_tiles) asm volatile("createpolicy.fractional.L2::evict_last.b64 %0, 1.0;" : "=l"(pol_w));
+  else asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(pol_w));
   if (warp == 4 && lane == 0 && !p.skip_copies)
     for (int it = 0; it < n_pre; ++it)
-      if (wt) bulk_load(base + it * stage_bytes, wt + static_cast<size_t>(kb0 + it) * A_TILE_BYTES, A_TILE_BYTES, smem_u32(full_bar + it));
-      else tma_load_2d(base + it * stage_bytes, map_w, (kb0 + it) * BK, f0, smem_u32(full_bar + it));
+      if (wt) bulk_load_hint(base + it * stage_bytes, wt + static_cast<size_t>(kb0 + it) * A_TILE_BYTES, A_TILE_BYTES, smem_u32(full_bar + it), pol_w);
+      else tma_load_2d_hint(base + it * stage_bytes, map_w, (kb0 + it) * BK, f0, smem_u32(full_bar + it), pol_w);
 
   cod_pdl_prologue();
   const int n_rows = p.n_rows_dev ? (p.rows_gate ? (*p.n_rows_dev > 0 ? p.n_rows : 0) : min(*p.n_rows_dev, p.n_rows)) : p.n_rows;
@@ -150,8 +167,8 @@ k_gemm_tc(const __grid_constant__ CUtensorMap map_w0, const __grid_constant__ CU
         const uint32_t a_dst = base + s * stage_bytes;
         const int k = (kb0 + it) * BK;
         if (it >= n_pre) {
-          if (wt) bulk_load(a_dst, wt + static_cast<size_t>(kb0 + it) * A_TILE_BYTES, A_TILE_BYTES, fb);
-          else tma_load_2d(a_dst, map_w, k, f0, fb);
+          if (wt) bulk_load_hint(a_dst, wt + static_cast<size_t>(kb0 + it) * A_TILE_BYTES, A_TILE_BYTES, fb, pol_w);
+          else tma_load_2d_hint(a_dst, map_w, k, f0, fb, pol_w);
         }
         tma_load_2d(a_dst + A_TILE_BYTES, &map_a, k, i0, fb);
       }
@@ -427,6 +444,10 @@ int cod_launch_gemm_tc(cod_ctx* c, const GemmArgs& g, cudaStream_t st) {
   p.status = c->status;
   p.wait_limit = c->wait_limit > 0 ? c->wait_limit : WAIT_LIMIT_CYCLES;
   p.skip_copies = c->selftest_skip_copies;
+  // The round's first weight stream (the fc projection) keeps a prefix of its tiles in L2 for the next round: every
+  // other stream of the round is evict-first, so about a third of the 126 MB survives a round (measured at batch 1:
+  // 40-64 MB kept -> 410 -> 405 us per round; 96 MB -> no gain, the prefix then evicts itself).
+  p.pin_tiles = g.klass == COD_K_FC ? static_cast<int>(COD_L2_KEEP_BYTES / (static_cast<long long>(g.K) * BM * 2)) : 0;
 
   CUtensorMap mw[3], ma;
   for (int i = 0; i < 3; ++i) {
