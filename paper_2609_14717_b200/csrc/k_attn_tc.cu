@@ -990,7 +990,7 @@ template <bool DUAL>
 __global__ void k_attn_tc_combine(const float* __restrict__ part_o, const float* __restrict__ part_ml,
                                   const int* __restrict__ committed_len, int S, int W, int rep, int n_kv,
                                   int max_pages, int split_len, int max_parts, __nv_bfloat16* __restrict__ out,
-                                  float* __restrict__ tap, float* __restrict__ mass, int* __restrict__ work_counter) {
+                                  float* __restrict__ tap, float* __restrict__ mass, int* __restrict__ work_counter, int drop) {
   cod_pdl_prologue();
   if (work_counter != nullptr && blockIdx.x == 0 && threadIdx.x == 0) *work_counter = 0;   // for the next persistent attention launch
   const int lane = threadIdx.x & 31;
@@ -1053,7 +1053,7 @@ __global__ void k_attn_tc_combine(const float* __restrict__ part_o, const float*
   // this warp was the only reader of its partial rows (512 bytes each): they are dead now and leave L2 without a
   // write-back (the warp barrier orders every lane's reads before the drop)
   __syncwarp();
-  if (S * W > COD_DROP_MIN_ROWS)
+  if (drop)
     for (int k = lane >> 2; k < n_parts; k += 8)        // lane 4 k + q drops line q of part k
       cod_discard_line(part_o + ((base + k) * M + mrow) * HD + (lane & 3) * 32);
   const float inv = 1.f / l;
@@ -1138,9 +1138,11 @@ int launch(cod_ctx* c, int layer, const void* q, const void* kb, const void* vb,
     COD_CHECK_LAUNCH(c);
   }
   const int items = S * f.block * f.n_q_heads;
+  // partials worth dropping from L2 once merged: when the launch may have written more than a few MB of them
+  const int drop = static_cast<long long>(S) * f.n_kv_heads * c->tc_max_parts * f.block * p.rep * HD * 4 > (8ll << 20) ? 1 : 0;
   cod_launch_pdl(c, k_attn_tc_combine<DUAL>, (items + 3) / 4, 128, 0, st, c->attn_o, c->attn_ml, stt->committed_len, S, f.block, p.rep,
                                                            f.n_kv_heads, f.max_pages_per_seq, c->tc_split_len,
-                                                           c->tc_max_parts, static_cast<__nv_bfloat16*>(out), tap, mass, c->attn_counter);
+                                                           c->tc_max_parts, static_cast<__nv_bfloat16*>(out), tap, mass, c->attn_counter, drop);
   COD_CHECK_LAUNCH(c);
   return COD_OK;
 }
