@@ -986,8 +986,10 @@ __global__ void k_attn_order(const int* __restrict__ committed_len, int S, int m
 }
 
 // Merges the partials of one (row, query head); one warp each. Empty partials carry m = -inf, l = 0.
-template <bool DUAL>
-__global__ void k_attn_tc_combine(const float* __restrict__ part_o, const float* __restrict__ part_ml,
+// FEW: no (sequence, head) has more than four parts (large batches: long parts). The kernel is bound by how many
+// warps wait on L2 at once, and without the eight-row batches of the general loop it fits eight blocks per SM.
+template <bool DUAL, bool FEW>
+__global__ void __launch_bounds__(128, FEW ? 8 : 1) k_attn_tc_combine(const float* __restrict__ part_o, const float* __restrict__ part_ml,
                                   const int* __restrict__ committed_len, int S, int W, int rep, int n_kv,
                                   int max_pages, int split_len, int max_parts, __nv_bfloat16* __restrict__ out,
                                   float* __restrict__ tap, float* __restrict__ mass, int* __restrict__ work_counter, int drop) {
@@ -1036,6 +1038,7 @@ __global__ void k_attn_tc_combine(const float* __restrict__ part_o, const float*
     }
     // then eight partial rows at a time, their loads all in flight before the first is used (a batch-1
     // round merges 17 partials per head)
+    if (!FEW)
     for (; kk < nk; kk += 8) {
       float4 v[8];
 #pragma unroll
@@ -1140,9 +1143,14 @@ int launch(cod_ctx* c, int layer, const void* q, const void* kb, const void* vb,
   const int items = S * f.block * f.n_q_heads;
   // partials worth dropping from L2 once merged: when the launch may have written more than a few MB of them
   const int drop = static_cast<long long>(S) * f.n_kv_heads * c->tc_max_parts * f.block * p.rep * HD * 4 > (8ll << 20) ? 1 : 0;
-  cod_launch_pdl(c, k_attn_tc_combine<DUAL>, (items + 3) / 4, 128, 0, st, c->attn_o, c->attn_ml, stt->committed_len, S, f.block, p.rep,
-                                                           f.n_kv_heads, f.max_pages_per_seq, c->tc_split_len,
-                                                           c->tc_max_parts, static_cast<__nv_bfloat16*>(out), tap, mass, c->attn_counter, drop);
+  if (c->tc_max_parts <= 4)
+    cod_launch_pdl(c, k_attn_tc_combine<DUAL, true>, (items + 3) / 4, 128, 0, st, c->attn_o, c->attn_ml, stt->committed_len, S, f.block, p.rep,
+                   f.n_kv_heads, f.max_pages_per_seq, c->tc_split_len, c->tc_max_parts, static_cast<__nv_bfloat16*>(out), tap, mass,
+                   c->attn_counter, drop);
+  else
+    cod_launch_pdl(c, k_attn_tc_combine<DUAL, false>, (items + 3) / 4, 128, 0, st, c->attn_o, c->attn_ml, stt->committed_len, S, f.block, p.rep,
+                   f.n_kv_heads, f.max_pages_per_seq, c->tc_split_len, c->tc_max_parts, static_cast<__nv_bfloat16*>(out), tap, mass,
+                   c->attn_counter, drop);
   COD_CHECK_LAUNCH(c);
   return COD_OK;
 }
