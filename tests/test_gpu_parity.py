@@ -380,6 +380,46 @@ def test_round_parity_multi_round(name, wo_scale, mode):
     P.close()
 
 
+@pytest.mark.parametrize("name,mode", [
+    ("small_bf16", orc.MODE_CARRY), ("small_bf16", orc.MODE_BASELINE), ("mid_bf16", orc.MODE_CARRY),
+    ("order_bf16", orc.MODE_CARRY), ("small_bf16_full", orc.MODE_CARRY)])
+def test_round_parity_through_cuda_graph_replays(name, mode):
+    """The launch form the benchmark times: one round captured into a CUDA graph (programmatic edges between the
+    kernels, fork and join of the small-round side stream as graph edges), replayed on fresh inputs written into
+    the captured buffers. Round 0 runs as plain launches (it also warms the lazily configured kernels), rounds
+    1-4 are replays; every round is held against the oracle like the stream-launched rounds."""
+    Hn = _H()
+    wl = _workloads()[name]
+    P = Hn.Pair(wl, seed=11, attn_split_len=64, wo_scale=30.0, poison=True)
+    tol = Hn.TOL[wl.shape.dtype]
+    rd, dev = P.round_inputs(0)
+    buf = {k: v.clone() for k, v in dev.items()}            # the buffers the graph is bound to
+    L0 = P.st_o.committed_len.copy()
+    res_o = P.run_round(0, mode, rd=rd, dev=buf)
+    _check_round(P, res_o, L0, tol)
+    side = torch.cuda.Stream()
+    side.wait_stream(torch.cuda.current_stream())
+    g = torch.cuda.CUDAGraph()
+    with torch.cuda.stream(side):
+        with torch.cuda.graph(g, stream=side):
+            P.ctx.draft_round(buf["draft"], buf["target"], buf["H"], wl.S, wl.n_forced, mode, P.st_g, P.split,
+                              P.next_draft, P.taps)
+    torch.cuda.current_stream().wait_stream(side)
+    torch.cuda.synchronize()
+    for r in range(1, 5):
+        rd, dev = P.round_inputs(r)
+        for k in buf:
+            buf[k].copy_(dev[k])
+        L0 = P.st_o.committed_len.copy()
+        res_o = orc.draft_round(rd["draft"], rd["target"], rd["H"], P.st_o, P.w_o, wl.n_forced, mode)
+        g.replay()
+        torch.cuda.synchronize()
+        _check_round(P, res_o, L0, tol)
+    assert P.ctx.poll_status() == 0
+    del g
+    P.close()
+
+
 def test_full_acceptance_carry_equals_baseline_bitwise():
     """m = W for every sequence: U is empty and the carry-mode round is the baseline round."""
     Hn = _H()
