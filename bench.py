@@ -764,6 +764,8 @@ def run_micro(args):
     torch.cuda.set_device(0)
     peaks = load_peaks()
     wl = synth.scaled(bench_workload(args.workload, 4), n_layers=1)
+    if args.vocab > 0:
+        wl = synth.scaled(wl, vocab=args.vocab)
     sh = wl.shape
     lay = synth.make_layout(wl, args.seed)
     n_pages, mp = int(lay["n_pages"]), int(lay["max_pages_per_seq"])
@@ -911,6 +913,7 @@ def main():
     ap.add_argument("--sweep", action="store_true", help="carryover-overhead sweep over batch, block and rejected fraction")
     ap.add_argument("--sweep-reps", type=int, default=7, help="--sweep: interleaved passes per mode and point")
     ap.add_argument("--attn-split", type=int, default=0, help="keys per attention split (0 = library default)")
+    ap.add_argument("--vocab", type=int, default=0, help="--micro lmhead*: override the vocabulary size (0 = the workload's)")
     ap.add_argument("--layers", type=int, default=1,
                     help="--micro gemm: drafter layers of the rounds it runs (default 1; 0 = the workload's own depth)")
     ap.add_argument("--flags", type=int, default=0,

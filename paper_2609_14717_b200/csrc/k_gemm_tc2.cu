@@ -51,6 +51,7 @@ struct Tc2Params {
   int seg_N[3];
   int n_seg;
   int n_tiles_n;              // token tiles
+  int tail_pairs;             // the last tail_pairs weight tiles run as two launches of one accumulator each (see the launcher)
   int n_acc;                  // accumulators per pair: 1 (256 token rows) or 2 (512)
   int stages;
   int staged;                 // epilogue transposes through shared memory (needs 16-byte aligned feature runs)
@@ -86,7 +87,13 @@ k_gemm_tc2(const __grid_constant__ CUtensorMap map_w0, const __grid_constant__ C
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int rank = blockIdx.x;                    // position in the pair; 0 leads
-  const int n_tile = blockIdx.y % p.n_tiles_n, pair = blockIdx.y / p.n_tiles_n, split = blockIdx.z;
+  const int n_tile = blockIdx.y % p.n_tiles_n, split = blockIdx.z;
+  int pair = blockIdx.y / p.n_tiles_n;
+  int half = -1;                                  // >= 0: this pair works on one accumulator (256 token rows) of a tail tile
+  if (p.tail_pairs > 0) {
+    const int whole = p.pair_end[p.n_seg - 1] - p.tail_pairs;
+    if (pair >= whole) { half = (pair - whole) & 1; pair = whole + ((pair - whole) >> 1); }
+  }
   const int i0 = n_tile * NTOK;
 
   int sidx = 0;
@@ -128,6 +135,7 @@ k_gemm_tc2(const __grid_constant__ CUtensorMap map_w0, const __grid_constant__ C
     if (sidx == 0) row_hi = g; else row_lo = g;
     col0 = f0;                                    // both groups' results share the columns
   }
+  if (half >= 0) { row_lo = max(row_lo, half * NT); row_hi = min(row_hi, (half + 1) * NT); }
   // NOTE: both CTAs of a pair take the same decision here (it depends on the pair's tile only)
   const int n_kb = (i0 < row_hi && i0 + NTOK > row_lo) ? kb1 - kb0 : 0;   // 0: no token rows here, only the requested weights to absorb
   // accumulators whose 256 token rows miss this segment's row range altogether are neither fed nor multiplied
@@ -241,7 +249,8 @@ k_gemm_tc2(const __grid_constant__ CUtensorMap map_w0, const __grid_constant__ C
       for (int t = c_begin + qw * 32 + lane; t < c_end; t += 128) hrow[t] = mix32(p.sample_state + static_cast<uint32_t>(i0 + t));
       asm volatile("bar.sync %0, 128;" ::"r"(1 + grp) : "memory");
       for (int c = c_begin; c < c_end; c += 32) {
-        if (i0 + c >= n_rows) break;
+        if (i0 + c >= row_hi) break;
+        if (i0 + c + 32 <= row_lo) continue;
         uint32_t v[32];
         tmem_ld32(t_lane + c, v);
         unsigned long long best;
@@ -254,7 +263,8 @@ k_gemm_tc2(const __grid_constant__ CUtensorMap map_w0, const __grid_constant__ C
     } else if (ok) {
       const unsigned long long low = static_cast<unsigned long long>(0xFFFFFFFFu - static_cast<unsigned>(col0 + qw * 32 + lane));
       for (int c = c_begin; c < c_end; c += 32) {
-        if (i0 + c >= n_rows) break;
+        if (i0 + c >= row_hi) break;
+        if (i0 + c + 32 <= row_lo) continue;
         uint32_t v[32];
         tmem_ld32(t_lane + c, v);
         unsigned long long k[32];
@@ -274,7 +284,7 @@ k_gemm_tc2(const __grid_constant__ CUtensorMap map_w0, const __grid_constant__ C
     __syncthreads();
   } else if (p.amax != nullptr && n_kb > 0) {
     for (int t = threadIdx.x; t < NTOK; t += NTHREADS) {
-      if (i0 + t < n_rows) {
+      if (i0 + t >= row_lo && i0 + t < row_hi) {
         unsigned long long best = red[t];
 #pragma unroll
         for (int w = 1; w < 4; ++w) best = red[w * NTOK + t] > best ? red[w * NTOK + t] : best;
@@ -404,8 +414,17 @@ int cod_launch_gemm_tc2(cod_ctx* c, const GemmArgs& g, cudaStream_t st) {
     if (e != cudaSuccess) return COD_ERR_CUDA;
     configured[sample] = smem;
   }
+  // The argmax launches (no split-K, all rows in one two-accumulator tile) run in waves of one pair per two SMs; the
+  // weight tiles beyond the last whole wave would hold two SMs each for a whole tile time while the rest idle
+  // (151936 columns: 594 tiles = 8 waves of 74 + 2). Those tiles are launched as two pairs each, one accumulator
+  // (256 token rows) per pair: half the time for the leftover wave.
+  p.tail_pairs = 0;
+  const int per_wave = c->n_sm / 2;
+  if (g.amax != nullptr && splits == 1 && p.n_acc == 2 && p.n_tiles_n == 1 && per_wave > 0 && pairs > per_wave &&
+      2 * (pairs % per_wave) <= per_wave)
+    p.tail_pairs = pairs % per_wave;
   cudaLaunchConfig_t cfg{};
-  cfg.gridDim = dim3(2, pairs * p.n_tiles_n, splits);
+  cfg.gridDim = dim3(2, (pairs + p.tail_pairs) * p.n_tiles_n, splits);
   cfg.blockDim = dim3(NTHREADS, 1, 1);
   cfg.dynamicSmemBytes = smem;
   cfg.stream = st;
