@@ -31,7 +31,8 @@ __device__ __forceinline__ void cod_pdl_prologue() {
 
 // Drops one 128-byte line (address aligned to 128 bytes) from L2 without writing it back: for scratch data that
 // has been read for the last time. Whatever is read there before the next write is indeterminate, and the caller
-// orders the drop after every read of the line (the readers synchronise with the dropping thread first).
+// orders the drop after every read of the line: the readers synchronise with the dropping thread first, and the
+// dropping thread is itself one of the line's readers (the lanes that share a line read it with one instruction).
 // Worth its instructions only when the scratch is large enough to be pushed out to HBM under a memory-bound kernel:
 // rounds of more token rows than this (one block per row in the kernels that use it).
 #define COD_DROP_MIN_ROWS 128

@@ -1057,8 +1057,8 @@ __global__ void __launch_bounds__(128, FEW ? 8 : 1) k_attn_tc_combine(const floa
   // write-back (the warp barrier orders every lane's reads before the drop)
   __syncwarp();
   if (drop)
-    for (int k = lane >> 2; k < n_parts; k += 8)        // lane 4 k + q drops line q of part k
-      cod_discard_line(part_o + ((base + k) * M + mrow) * HD + (lane & 3) * 32);
+    for (int k = lane & 7; k < n_parts; k += 8)         // a lane drops the line its own 16 bytes came from, for every eighth part
+      cod_discard_line(part_o + ((base + k) * M + mrow) * HD + (lane >> 3) * 32);
   const float inv = 1.f / l;
   const size_t ob = static_cast<size_t>(item) * HD + lane * 4;
   const __nv_bfloat162 b0 = __floats2bfloat162_rn(acc[0] * inv, acc[1] * inv), b1 = __floats2bfloat162_rn(acc[2] * inv, acc[3] * inv);
